@@ -1,0 +1,140 @@
+/*
+ * toktier.h -- C ABI of the B200 (sm_100a) exact full-request tokenizer.
+ *
+ * The library computes, entirely in CUDA kernels, what the paper's Sec. 4 ("Exact GPU
+ * Tokenization") describes: GPT-family regex pre-tokenization re-expressed as per-character
+ * class tags, maximal runs and a run-local piece-start predicate (Sec. 4.1), followed by
+ * byte-level BPE applied to every piece independently (Sec. 4.2), with counts kept on the
+ * device so that no call synchronises with the host (Sec. 4.3).  Output token IDs are identical
+ * to sequential leftmost-first matching followed by lowest-rank-first merging.
+ *
+ * Conventions
+ *   - "DEVICE" pointers are CUDA device addresses on the current device; "HOST" pointers are
+ *     ordinary host addresses.  The library never frees or reallocates caller memory.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ *   - Every tt_encode* / tt_pretokenize call only enqueues work on `stream`; it never
+ *     synchronises and never reads device memory on the host.  Data-dependent failures are
+ *     reported through the DEVICE status word (see below), never by trapping.
+ *   - Host return value: TT_OK or a TT_ERR_* code describing an argument / CUDA problem.
+ *   - There is no CPU fallback: without a CUDA device the calls fail with TT_ERR_CUDA.
+ */
+#ifndef TOKTIER_H
+#define TOKTIER_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* host return codes and device status values */
+enum {
+    TT_OK = 0,
+    TT_ERR_ARG = 1,              /* null pointer, bad pattern id, buffer too small (host-detectable)   */
+    TT_ERR_BAD_VOCAB = 2,        /* merge table rejected by tt_vocab_load                              */
+    TT_ERR_CUDA = 3,             /* a CUDA runtime call failed (no device, out of memory, launch)      */
+    TT_ERR_INVALID_UTF8 = 4,     /* device status: input is not strict UTF-8; zero tokens are returned */
+    TT_ERR_CAPACITY = 5,         /* device status: ids_cap too small for the result; zero tokens       */
+    TT_ERR_INTERNAL_TIMEOUT = 6  /* device status: a bounded device-side loop gave up                  */
+};
+
+/* Patterns (benchmark configs; the paper names the two lineages in Sec. 4.1):
+ *   TT_PATTERN_CL100K  contraction | [^\r\n\p{L}\p{N}]?\p{L}+ | \p{N}{1,3} | ' '?[^\s\p{L}\p{N}]+[\r\n]*
+ *                      | \s*[\r\n]+ | \s+(?!\S) | \s+
+ *   TT_PATTERN_O200K   case-aware word alternatives with an optional contraction suffix,
+ *                      \p{N}{1,3}, ' '?[^\s\p{L}\p{N}]+[\r\n/]*, and the same whitespace rules. */
+enum { TT_PATTERN_CL100K = 0, TT_PATTERN_O200K = 1 };
+
+typedef struct tt_vocab tt_vocab;   /* opaque; immutable after load; owns its device tables */
+
+/* One merge rule; its rank is its index in the array passed to tt_vocab_load. */
+typedef struct { int32_t left, right, result; } tt_merge;
+
+/*
+ * tt_vocab_load -- build the device tables for one tokenizer (paper Sec. 4.2: merge ranks and
+ * vocabulary entries are packed into GPU hash tables).
+ *   merges    HOST, n_merges entries, copied.  rank = index.  `left`/`right` must each be a base id
+ *             (a value of byte_map) or the `result` of a LOWER-ranked merge; pairs must be distinct;
+ *             results must be distinct, non-negative and differ from every base id.
+ *   byte_map  HOST, 256 entries: byte value -> base token id; must be injective and non-negative.
+ *   pattern_id  TT_PATTERN_CL100K or TT_PATTERN_O200K.
+ *   out       receives the handle (device tables live on the current CUDA device).
+ * Limits: n_merges <= 262,144 - 256.  Synchronous (it waits for its own uploads).
+ * Returns TT_OK, TT_ERR_ARG, TT_ERR_BAD_VOCAB or TT_ERR_CUDA; *out is NULL on failure.
+ */
+int tt_vocab_load(const tt_merge* merges, size_t n_merges, const int32_t byte_map[256], int pattern_id,
+                  tt_vocab** out);
+
+/* Frees the handle and its device tables.  NULL is allowed.  No encode using it may be in flight. */
+void tt_vocab_free(tt_vocab* v);
+
+/*
+ * tt_workspace_bytes -- DEVICE scratch size needed by an encode call over at most max_len text
+ * bytes in at most max_docs documents (use 1 for tt_encode).  The caller allocates the scratch
+ * (256-byte aligned) and may reuse it for any number of calls that do not overlap in time.
+ */
+size_t tt_workspace_bytes(const tt_vocab* v, size_t max_len, size_t max_docs);
+
+/*
+ * tt_encode -- tokenize one request (the cold full-request path, paper Sec. 4).
+ *   text        DEVICE, len bytes of UTF-8 (len < 2^31).  Not modified.
+ *   ids_out     DEVICE int32[ids_cap].  ids_cap >= len always suffices (a token covers >= 1 byte).
+ *   count_out   DEVICE int64: number of tokens written (0 on a device-side error).
+ *   status_out  DEVICE int32: TT_OK, TT_ERR_INVALID_UTF8, TT_ERR_CAPACITY or TT_ERR_INTERNAL_TIMEOUT.
+ *   workspace   DEVICE scratch of at least tt_workspace_bytes(v, len, 1) bytes.
+ * Asynchronous on `stream`.  len == 0 yields count 0, status TT_OK.
+ */
+int tt_encode(const tt_vocab* v, const uint8_t* text, size_t len, void* stream,
+              int32_t* ids_out, size_t ids_cap, int64_t* count_out, int32_t* status_out,
+              void* workspace, size_t workspace_bytes);
+
+/*
+ * tt_encode_batch -- tokenize n_docs independent documents in one call (paper Sec. 4.2:
+ * multi-document batches concatenate inputs and cut runs at document boundaries).
+ *   text         DEVICE, the documents concatenated; total_len = total bytes (HOST value, < 2^31).
+ *   doc_off      DEVICE int64[n_docs+1], ascending byte offsets, doc_off[0]=0, doc_off[n_docs]=total_len.
+ *   ids_out      DEVICE int32[ids_cap]: token IDs of all documents, in document order.
+ *   ids_off_out  DEVICE int64[n_docs+1]: token offset of each document in ids_out; the last entry
+ *                is the total count.
+ *   status_out   DEVICE int32 as for tt_encode (one word for the whole batch; on error every
+ *                ids_off_out entry is 0).
+ * Every document is tokenized exactly as if it were encoded alone.  Asynchronous on `stream`.
+ */
+int tt_encode_batch(const tt_vocab* v, const uint8_t* text, size_t total_len, const int64_t* doc_off,
+                    size_t n_docs, void* stream, int32_t* ids_out, size_t ids_cap, int64_t* ids_off_out,
+                    int32_t* status_out, void* workspace, size_t workspace_bytes);
+
+/*
+ * tt_pretokenize -- the pre-tokenization half alone (paper Sec. 4.1; the paper checks piece
+ * boundaries separately from IDs because ID-level agreement can hide a boundary fault).
+ *   piece_off_out  DEVICE int32[piece_cap]: byte offset of every piece start, ascending;
+ *                  piece_cap >= len always suffices.
+ *   n_pieces_out   DEVICE int64: number of pieces.
+ * doc_off / n_docs as in tt_encode_batch, or doc_off = NULL and n_docs = 1 for one document.
+ */
+int tt_pretokenize(const tt_vocab* v, const uint8_t* text, size_t len, const int64_t* doc_off, size_t n_docs,
+                   void* stream, int32_t* piece_off_out, size_t piece_cap, int64_t* n_pieces_out,
+                   int32_t* status_out, void* workspace, size_t workspace_bytes);
+
+/*
+ * tt_encode_host -- convenience wrapper for HOST buffers: copies `text` to the device, encodes,
+ * copies IDs back and synchronises.  Allocates and caches its own device and pinned staging
+ * buffers inside the handle's context (not thread-safe per vocab).  ids_out HOST int32[ids_cap];
+ * *count_out HOST.  Returns the host code, or the device status if that is not TT_OK.
+ */
+int tt_encode_host(tt_vocab* v, const uint8_t* text, size_t len, int32_t* ids_out, size_t ids_cap,
+                   int64_t* count_out);
+
+/* Number of class-table entries (0x110000) copied to out (HOST uint8, one class code per code
+ * point as the kernels see it): 0 other, 1 mark, 2 whitespace, 3 number, 4 lowercase letter,
+ * 5 uppercase/titlecase letter, 6 caseless letter.  For exhaustive table checks. */
+size_t tt_class_table(uint8_t* out, size_t cap);
+
+/* Static, human-readable description of a code. */
+const char* tt_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TOKTIER_H */

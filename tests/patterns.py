@@ -1,0 +1,33 @@
+"""Test-side statement of the two pre-tokenization patterns as regular expressions for a
+backtracking engine (the third-party ``regex`` module).  The oracle itself never uses a regex
+engine; these strings exist only to pin it."""
+CON = r"'(?:[sStTmMdD]|[rR][eE]|[vV][eE]|[lL][lL])"
+P0 = (CON
+      + r"|[^\r\n\p{L}\p{N}]?\p{L}+"
+      + r"|\p{N}{1,3}"
+      + r"| ?[^\s\p{L}\p{N}]+[\r\n]*"
+      + r"|\s*[\r\n]+"
+      + r"|\s+(?!\S)"
+      + r"|\s+")
+U = r"[\p{Lu}\p{Lt}\p{Lm}\p{Lo}\p{M}]"
+LW = r"[\p{Ll}\p{Lm}\p{Lo}\p{M}]"
+P1 = (r"[^\r\n\p{L}\p{N}]?" + U + "*" + LW + "+" + "(?:" + CON + ")?"
+      + r"|[^\r\n\p{L}\p{N}]?" + U + "+" + LW + "*" + "(?:" + CON + ")?"
+      + r"|\p{N}{1,3}"
+      + r"| ?[^\s\p{L}\p{N}]+[\r\n/]*"
+      + r"|\s*[\r\n]+"
+      + r"|\s+(?!\S)"
+      + r"|\s+")
+PATTERNS = [P0, P1]
+
+
+def engine_starts(compiled, s: str):
+    """Successive leftmost-first matches from position 0; returns piece start BYTE offsets."""
+    out, p, b = [], 0, 0
+    while p < len(s):
+        m = compiled.match(s, p)
+        assert m and m.end() > p
+        out.append(b)
+        b += len(s[p:m.end()].encode("utf-8"))
+        p = m.end()
+    return out

@@ -1,0 +1,170 @@
+"""Pins for the oracle's pre-tokenizer (paper Sec. 4.1: leftmost-first alternation with
+backtracking, each match beginning at the previous match's end).
+
+The oracle is a hand-written sequential matcher; here it is compared with a genuine backtracking
+regex engine on exhaustive small alphabets and random strings, with worked examples, and with
+structural invariants."""
+import itertools
+import json
+import os
+import random
+
+import numpy as np
+import pytest
+
+import oracle
+from patterns import PATTERNS, engine_starts
+
+regex = pytest.importorskip("regex")
+R = [regex.compile(p) for p in PATTERNS]
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden", "pretok_examples.jsonl")
+
+
+def _exhaustive(pat, alphabet, maxlen):
+    bad = []
+    for ln in range(1, maxlen + 1):
+        for tup in itertools.product(alphabet, repeat=ln):
+            s = "".join(tup)
+            if engine_starts(R[pat], s) != list(oracle.pretokenize(s, pat)):
+                bad.append(s)
+                if len(bad) > 5:
+                    return bad
+    return bad
+
+
+@pytest.mark.parametrize("alphabet,maxlen", [
+    ("as1 \t\n!'", 5),                 # letters, digit, blank, tab, LF, punctuation, apostrophe
+    ("rRevl't !", 5),                  # every contraction spelling
+    ("eé中²́ 　\n's", 4),   # multi-byte letters, No digit, mark, ideographic space
+    ("a1 \r\n !", 5),             # CR, LF, no-break space
+])
+def test_pattern0_equals_backtracking_engine(alphabet, maxlen):
+    assert _exhaustive(0, alphabet, maxlen) == []
+
+
+@pytest.mark.parametrize("alphabet,maxlen", [
+    ("á's/\n !", 5),
+    ("Aal's1 \n/", 5),
+    ("Aa中́'s !/\n", 4),
+    ("AaBb中́1 \t", 5),
+    ("á's/\n !", 5),              # marks with contraction and tail chains
+    ("ǅaʰA'l \r", 5),         # titlecase, modifier letter
+])
+def test_pattern1_equals_backtracking_engine(alphabet, maxlen):
+    assert _exhaustive(1, alphabet, maxlen) == []
+
+
+def _agreeing_codepoints():
+    """Code points whose class agrees between the oracle's frozen table and the regex engine's own
+    (possibly newer) Unicode tables; random strings are drawn only from these."""
+    t = oracle.class_table()
+    pools = []
+    probes = [(r"\p{Ll}", oracle.K_LL), (r"[\p{Lu}\p{Lt}]", oracle.K_LU), (r"[\p{Lm}\p{Lo}]", oracle.K_LB),
+              (r"\p{N}", oracle.K_N), (r"\s", oracle.K_W), (r"\p{M}", oracle.K_M)]
+    rng = random.Random(5)
+    sample = [rng.randrange(0x20, 0x30000) for _ in range(6000)] + list(range(0x20, 0x250))
+    sample = [c for c in sample if not (0xD800 <= c <= 0xDFFF)]
+    for c in sample:
+        ch = chr(c)
+        code = oracle.K_O
+        for pat, k in probes:
+            if regex.fullmatch(pat, ch):
+                code = k
+                break
+        if code == t[c]:
+            pools.append(c)
+    return pools
+
+
+def test_random_unicode_strings_equal_engine():
+    pool = _agreeing_codepoints()
+    assert len(pool) > 5000
+    rng = random.Random(11)
+    special = list(" \t\n\r'/!.,") + ["'s", "'re", "'LL", "\r\n", "  "]
+    for pat in (0, 1):
+        for _ in range(3000):
+            n = rng.randrange(1, 40)
+            s = "".join(rng.choice(special) if rng.random() < 0.5 else chr(rng.choice(pool)) for _ in range(n))
+            assert engine_starts(R[pat], s) == list(oracle.pretokenize(s, pat)), repr(s)
+
+
+def test_worked_examples():
+    n = 0
+    with open(GOLDEN, encoding="utf-8") as f:
+        for line in f:
+            d = json.loads(line)
+            if "text" not in d:
+                continue
+            for pat, key in ((0, "p0"), (1, "p1")):
+                got = [p.decode("utf-8") for p in oracle.pieces(d["text"], pat)]
+                assert got == d[key], (d["text"], key, got)
+            n += 1
+    assert n >= 30
+
+
+def test_pieces_partition_the_input():
+    import workloads as wl
+    for name in ("C1", "C2"):
+        cfg = wl.CONFIGS[name]
+        text = wl.request(cfg, n_chars=20000)
+        for pat in (0, 1):
+            st = oracle.pretokenize(text, pat)
+            assert st[0] == 0 and np.all(np.diff(st) > 0) and st[-1] < text.size
+            # every start is a code-point boundary
+            assert np.all((text[st] & 0xC0) != 0x80)
+            assert b"".join(oracle.pieces(text, pat)) == text.tobytes()
+
+
+def test_document_cut_is_idempotent():
+    """Cutting the text at a piece boundary and matching both halves alone gives the same pieces
+    (a match never looks behind its own start)."""
+    import workloads as wl
+    text = wl.request(wl.CONFIGS["C2"], n_chars=5000)
+    for pat in (0, 1):
+        st = oracle.pretokenize(text, pat)
+        for k in (len(st) // 3, len(st) // 2):
+            cut = int(st[k])
+            tail = oracle.pretokenize(text[cut:], pat) + cut
+            assert list(tail) == list(st[k:])
+
+
+def test_class_table_spot_values_and_engine_agreement():
+    t = oracle.class_table()
+    assert t[0x20] == oracle.K_W and t[0x3000] == oracle.K_W and t[0x85] == oracle.K_W and t[0xA0] == oracle.K_W
+    assert t[0x1C] == oracle.K_O            # str.isspace() says True, White_Space says no
+    assert t[0xE9] == oracle.K_LL and t[0x4E2D] == oracle.K_LB and t[0x0301] == oracle.K_M
+    assert t[0xB2] == oracle.K_N and t[0x01C5] == oracle.K_LU and t[0x2160] == oracle.K_N
+    assert t[ord("A")] == oracle.K_LU and t[ord("z")] == oracle.K_LL and t[ord("7")] == oracle.K_N
+    assert t[ord("'")] == oracle.K_O and t[ord("/")] == oracle.K_O and t[0x1F600] == oracle.K_O
+    assert int((t == oracle.K_W).sum()) == 25
+    # the regex engine's \s is exactly the whitespace class
+    ws = [c for c in range(0x3100) if regex.fullmatch(r"\s", chr(c))]
+    assert ws == [c for c in range(0x3100) if t[c] == oracle.K_W]
+    # Against the engine's (newer) tables over U+0020..U+2FFF: every disagreement must be a code
+    # point that is unassigned in the frozen 15.0.0 database, except U+0295, whose General_Category
+    # changed after 15.0.
+    import unicodedata
+    differ = []
+    for c in range(0x20, 0x3000):
+        ch = chr(c)
+        want = (oracle.K_LL if regex.fullmatch(r"\p{Ll}", ch) else oracle.K_LU if regex.fullmatch(r"[\p{Lu}\p{Lt}]", ch)
+                else oracle.K_LB if regex.fullmatch(r"[\p{Lm}\p{Lo}]", ch) else oracle.K_N if regex.fullmatch(r"\p{N}", ch)
+                else oracle.K_W if regex.fullmatch(r"\s", ch) else oracle.K_M if regex.fullmatch(r"\p{M}", ch) else oracle.K_O)
+        if t[c] != want:
+            differ.append(c)
+    assert len(differ) < 60
+    for c in differ:
+        assert c == 0x295 or unicodedata.category(chr(c)) == "Cn", hex(c)
+
+
+@pytest.mark.parametrize("data,ok", [
+    (b"", True), (b"abc", True), ("é中😀".encode(), True),
+    (b"\x80", False), (b"\xc3", False), (b"\xc0\xaf", False), (b"\xe0\x80\xaf", False),
+    (b"\xed\xa0\x80", False), (b"\xf4\x90\x80\x80", False), (b"\xf0\x8f\xbf\xbf", False),
+    (b"a\xe4\xb8", False), (b"\xf5\x80\x80\x80", False), (b"\xef\xbf\xbf", True), (b"\xf4\x8f\xbf\xbf", True),
+])
+def test_strict_utf8(data, ok):
+    assert (oracle.utf8_check(data) >= 0) == ok
+    if not ok:
+        with pytest.raises(oracle.InvalidUtf8):
+            oracle.pretokenize(data, 0)

@@ -1,0 +1,162 @@
+"""B200-native exact tokenizer: thin Python binding over the C ABI in include/toktier.h.
+
+Argument marshalling only -- every step of the path runs in the CUDA kernels of libtoktier.so.
+PyTorch supplies device memory and streams.  There is no CPU fallback: if the library is missing
+or no CUDA device is present, the calls raise.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libtoktier.so")
+
+TT_OK, TT_ERR_ARG, TT_ERR_BAD_VOCAB, TT_ERR_CUDA, TT_ERR_INVALID_UTF8, TT_ERR_CAPACITY, TT_ERR_INTERNAL_TIMEOUT = range(7)
+TT_PATTERN_CL100K, TT_PATTERN_O200K = 0, 1
+
+EXPORTS = ["tt_vocab_load", "tt_vocab_free", "tt_workspace_bytes", "tt_encode", "tt_encode_batch",
+           "tt_pretokenize", "tt_encode_host", "tt_class_table", "tt_strerror"]
+
+_lib = None
+
+
+class TokTierError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {strerror(code)} (code {code})")
+
+
+def lib() -> ctypes.CDLL:
+    """Loads libtoktier.so (built in-tree by paper_2607_29678_b200.build); raises if it is missing."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(f"{LIB_PATH} not built; run `python -m paper_2607_29678_b200.build`")
+        L = ctypes.CDLL(LIB_PATH)
+        c = ctypes
+        L.tt_vocab_load.restype = c.c_int
+        L.tt_vocab_load.argtypes = [c.c_void_p, c.c_size_t, c.c_void_p, c.c_int, c.POINTER(c.c_void_p)]
+        L.tt_vocab_free.restype = None
+        L.tt_vocab_free.argtypes = [c.c_void_p]
+        L.tt_workspace_bytes.restype = c.c_size_t
+        L.tt_workspace_bytes.argtypes = [c.c_void_p, c.c_size_t, c.c_size_t]
+        L.tt_encode.restype = c.c_int
+        L.tt_encode.argtypes = [c.c_void_p, c.c_void_p, c.c_size_t, c.c_void_p, c.c_void_p, c.c_size_t, c.c_void_p,
+                                c.c_void_p, c.c_void_p, c.c_size_t]
+        L.tt_encode_batch.restype = c.c_int
+        L.tt_encode_batch.argtypes = [c.c_void_p, c.c_void_p, c.c_size_t, c.c_void_p, c.c_size_t, c.c_void_p, c.c_void_p,
+                                      c.c_size_t, c.c_void_p, c.c_void_p, c.c_void_p, c.c_size_t]
+        L.tt_pretokenize.restype = c.c_int
+        L.tt_pretokenize.argtypes = [c.c_void_p, c.c_void_p, c.c_size_t, c.c_void_p, c.c_size_t, c.c_void_p, c.c_void_p,
+                                     c.c_size_t, c.c_void_p, c.c_void_p, c.c_void_p, c.c_size_t]
+        L.tt_encode_host.restype = c.c_int
+        L.tt_encode_host.argtypes = [c.c_void_p, c.c_void_p, c.c_size_t, c.c_void_p, c.c_size_t, c.POINTER(c.c_int64)]
+        L.tt_class_table.restype = c.c_size_t
+        L.tt_class_table.argtypes = [c.c_void_p, c.c_size_t]
+        L.tt_strerror.restype = c.c_char_p
+        L.tt_strerror.argtypes = [c.c_int]
+        _lib = L
+    return _lib
+
+
+def strerror(code: int) -> str:
+    return lib().tt_strerror(int(code)).decode()
+
+
+def class_table() -> np.ndarray:
+    """uint8[0x110000]: the class code the kernels assign to every code point."""
+    out = np.empty(0x110000, dtype=np.uint8)
+    lib().tt_class_table(out.ctypes.data, out.size)
+    return out
+
+
+def _check(rc: int, where: str):
+    if rc != TT_OK:
+        raise TokTierError(rc, where)
+
+
+def _stream_ptr(stream) -> int:
+    import torch
+    s = torch.cuda.current_stream() if stream is None else stream
+    return int(s.cuda_stream)
+
+
+class Vocab:
+    """tt_vocab_load / tt_vocab_free.  merges: int32[n,3] rows (left, right, result); rank = row."""
+
+    def __init__(self, merges, byte_map=None, pattern_id: int = TT_PATTERN_CL100K):
+        m = np.ascontiguousarray(merges, dtype=np.int32).reshape(-1, 3)
+        bm = np.ascontiguousarray(np.arange(256) if byte_map is None else byte_map, dtype=np.int32)
+        if bm.size != 256:
+            raise ValueError("byte_map needs 256 entries")
+        self.n_merges = m.shape[0]
+        self.pattern_id = pattern_id
+        h = ctypes.c_void_p()
+        _check(lib().tt_vocab_load(m.ctypes.data, m.shape[0], bm.ctypes.data, pattern_id, ctypes.byref(h)), "tt_vocab_load")
+        self._h = h
+
+    def close(self):
+        if getattr(self, "_h", None):
+            lib().tt_vocab_free(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # -- sizes -------------------------------------------------------------------------------
+    def workspace_bytes(self, max_len: int, max_docs: int = 1) -> int:
+        return int(lib().tt_workspace_bytes(self._h, max_len, max_docs))
+
+    def alloc(self, max_len: int, max_docs: int = 1, device="cuda"):
+        """Device buffers for calls over at most max_len bytes: dict(ids, count, status, ids_off, workspace)."""
+        import torch
+        return dict(
+            ids=torch.empty(max(max_len, 1), dtype=torch.int32, device=device),
+            count=torch.zeros(1, dtype=torch.int64, device=device),
+            status=torch.zeros(1, dtype=torch.int32, device=device),
+            ids_off=torch.zeros(max_docs + 1, dtype=torch.int64, device=device),
+            workspace=torch.empty(self.workspace_bytes(max_len, max_docs), dtype=torch.uint8, device=device),
+        )
+
+    # -- device entry points (asynchronous on the stream) ---------------------------------------
+    def encode(self, text, bufs, stream=None, length: int | None = None):
+        """tt_encode: text = uint8 CUDA tensor.  Results land in bufs['ids'], bufs['count'], bufs['status']."""
+        n = int(text.numel() if length is None else length)
+        ws = bufs["workspace"]
+        _check(lib().tt_encode(self._h, text.data_ptr(), n, _stream_ptr(stream), bufs["ids"].data_ptr(),
+                               bufs["ids"].numel(), bufs["count"].data_ptr(), bufs["status"].data_ptr(),
+                               ws.data_ptr(), ws.numel()), "tt_encode")
+
+    def encode_batch(self, text, doc_off, bufs, stream=None):
+        """tt_encode_batch: doc_off = int64 CUDA tensor [n_docs+1].  Results in bufs['ids'], bufs['ids_off'], bufs['status']."""
+        ws = bufs["workspace"]
+        n_docs = int(doc_off.numel()) - 1
+        _check(lib().tt_encode_batch(self._h, text.data_ptr(), int(text.numel()), doc_off.data_ptr(), n_docs,
+                                     _stream_ptr(stream), bufs["ids"].data_ptr(), bufs["ids"].numel(),
+                                     bufs["ids_off"].data_ptr(), bufs["status"].data_ptr(), ws.data_ptr(), ws.numel()),
+               "tt_encode_batch")
+
+    def pretokenize(self, text, piece_off, n_pieces, bufs, doc_off=None, stream=None):
+        """tt_pretokenize: piece_off = int32 CUDA tensor [>= len+1], n_pieces = int64 CUDA tensor [1]."""
+        ws = bufs["workspace"]
+        n_docs = 1 if doc_off is None else int(doc_off.numel()) - 1
+        _check(lib().tt_pretokenize(self._h, text.data_ptr(), int(text.numel()), 0 if doc_off is None else doc_off.data_ptr(),
+                                    n_docs, _stream_ptr(stream), piece_off.data_ptr(), piece_off.numel(),
+                                    n_pieces.data_ptr(), bufs["status"].data_ptr(), ws.data_ptr(), ws.numel()),
+               "tt_pretokenize")
+
+    # -- host convenience --------------------------------------------------------------------------
+    def encode_host(self, data) -> np.ndarray:
+        """tt_encode_host: bytes / uint8 array in host memory -> int32 ids in host memory."""
+        a = np.frombuffer(data, dtype=np.uint8) if isinstance(data, (bytes, bytearray)) else np.ascontiguousarray(data, dtype=np.uint8)
+        out = np.empty(max(a.size, 1), dtype=np.int32)
+        cnt = ctypes.c_int64(0)
+        _check(lib().tt_encode_host(self._h, a.ctypes.data, a.size, out.ctypes.data, out.size, ctypes.byref(cnt)),
+               "tt_encode_host")
+        return out[:cnt.value]

@@ -1,0 +1,318 @@
+// C ABI of the toktier library (see include/toktier.h).  Host side: argument checks, vocabulary
+// tables, workspace layout and the kernel chain  K1+K2 -> K3 -> K4 (warp) -> K4 (long) -> K5a -> K5b.
+// Nothing here synchronises with the device except tt_vocab_load and tt_encode_host.
+#include "../../include/toktier.h"
+#include "tt_common.cuh"
+#include "tt_pretok_kernels.cuh"
+#include "tt_bpe.cuh"
+#include "unicode_table.inc"
+
+#include <climits>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <unordered_map>
+#include <unordered_set>
+#include <vector>
+
+struct tt_vocab {
+    int pattern = 0;
+    int device = 0;
+    int sm_count = 148;
+    size_t n_merges = 0;
+    u64* d_slots = nullptr;
+    u32 table_cap = 0;
+    int32_t* d_ext_id = nullptr;
+    u8* d_cls = nullptr;
+    int cls_bytes = 0;
+    PairTable tab{};
+    // cached buffers of tt_encode_host
+    u8* h_text = nullptr; int32_t* h_ids = nullptr; long long* h_scalars = nullptr;
+    u8* d_text = nullptr; int32_t* d_ids = nullptr; long long* d_count = nullptr; int32_t* d_status = nullptr;
+    void* d_ws = nullptr; size_t host_cap = 0, ws_cap = 0;
+    cudaStream_t host_stream = nullptr;
+};
+
+static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+extern "C" const char* tt_strerror(int code) {
+    switch (code) {
+        case TT_OK: return "ok";
+        case TT_ERR_ARG: return "invalid argument";
+        case TT_ERR_BAD_VOCAB: return "merge table rejected";
+        case TT_ERR_CUDA: return "CUDA runtime error";
+        case TT_ERR_INVALID_UTF8: return "input is not valid UTF-8";
+        case TT_ERR_CAPACITY: return "output buffer too small";
+        case TT_ERR_INTERNAL_TIMEOUT: return "bounded device loop gave up";
+        default: return "unknown code";
+    }
+}
+
+extern "C" size_t tt_class_table(uint8_t* out, size_t cap) {
+    const size_t n = 0x110000;
+    for (size_t cp = 0; cp < n && cp < cap; cp++) {
+        unsigned v = tt_cls_stage2_host[(size_t)tt_cls_stage1_host[cp >> 8] * 128 + ((cp & 0xFF) >> 1)];
+        out[cp] = (uint8_t)((cp & 1) ? (v >> 4) : (v & 15));
+    }
+    return n;
+}
+
+extern "C" void tt_vocab_free(tt_vocab* v) {
+    if (!v) return;
+    cudaFree(v->d_slots); cudaFree(v->d_ext_id); cudaFree(v->d_cls);
+    cudaFree(v->d_text); cudaFree(v->d_ids); cudaFree(v->d_count); cudaFree(v->d_status); cudaFree(v->d_ws);
+    if (v->h_text) cudaFreeHost(v->h_text);
+    if (v->h_ids) cudaFreeHost(v->h_ids);
+    if (v->h_scalars) cudaFreeHost(v->h_scalars);
+    if (v->host_stream) cudaStreamDestroy(v->host_stream);
+    delete v;
+}
+
+extern "C" int tt_vocab_load(const tt_merge* merges, size_t n_merges, const int32_t byte_map[256], int pattern_id,
+                             tt_vocab** out) {
+    if (out) *out = nullptr;
+    if (!out || !byte_map || (n_merges && !merges)) return TT_ERR_ARG;
+    if (pattern_id != TT_PATTERN_CL100K && pattern_id != TT_PATTERN_O200K) return TT_ERR_ARG;
+    if (n_merges > TT_MAX_INTERNAL - 256) return TT_ERR_ARG;
+    // external id -> internal id (byte b -> b, result of rank r -> 256 + r)
+    std::unordered_map<int32_t, u32> internal;
+    internal.reserve(512 + 2 * n_merges);
+    std::vector<int32_t> ext_id(256 + n_merges);
+    for (int b = 0; b < 256; b++) {
+        if (byte_map[b] < 0 || !internal.emplace(byte_map[b], (u32)b).second) return TT_ERR_BAD_VOCAB;   // not injective
+        ext_id[b] = byte_map[b];
+    }
+    u32 cap = 1024;
+    while (cap < 2 * n_merges + 2) cap <<= 1;
+    u32 log2cap = 0;
+    while ((1u << log2cap) < cap) log2cap++;
+    std::vector<u64> slots(cap, TT_SLOT_EMPTY);
+    const u32 mask = cap - 1, shift = 64 - log2cap;
+    for (size_t r = 0; r < n_merges; r++) {
+        const tt_merge& m = merges[r];
+        auto l = internal.find(m.left), rr = internal.find(m.right);
+        if (l == internal.end() || rr == internal.end()) return TT_ERR_BAD_VOCAB;      // operand not yet defined
+        if (m.result < 0 || internal.count(m.result)) return TT_ERR_BAD_VOCAB;         // result id reused
+        const u64 key = ((u64)l->second << TT_ID_BITS) | rr->second;
+        u32 h = (u32)((key * 0x9E3779B97F4A7C15ull) >> shift);
+        for (;;) {
+            if (slots[h] == TT_SLOT_EMPTY) { slots[h] = (key << 20) | (u64)r; break; }
+            if ((slots[h] >> 20) == key) return TT_ERR_BAD_VOCAB;                      // duplicate pair
+            h = (h + 1) & mask;
+        }
+        internal.emplace(m.result, (u32)(256 + r));
+        ext_id[256 + r] = m.result;
+    }
+    tt_vocab* v = new (std::nothrow) tt_vocab();
+    if (!v) return TT_ERR_CUDA;
+    v->pattern = pattern_id; v->n_merges = n_merges; v->table_cap = cap;
+    // class tables: stage1 | stage2 | ascii
+    const int stage2_bytes = TT_CLS_NBLOCKS * 128;
+    v->cls_bytes = (int)align_up(0x1100 + stage2_bytes, 16) + 128;
+    std::vector<u8> cls(v->cls_bytes, 0);
+    memcpy(cls.data(), tt_cls_stage1_host, 0x1100);
+    memcpy(cls.data() + 0x1100, tt_cls_stage2_host, stage2_bytes);
+    tt_fill_ascii_table(cls.data() + v->cls_bytes - 128);
+    bool ok = cudaGetDevice(&v->device) == cudaSuccess;
+    ok = ok && cudaDeviceGetAttribute(&v->sm_count, cudaDevAttrMultiProcessorCount, v->device) == cudaSuccess;
+    ok = ok && cudaMalloc(&v->d_slots, (size_t)cap * sizeof(u64)) == cudaSuccess;
+    ok = ok && cudaMalloc(&v->d_ext_id, ext_id.size() * sizeof(int32_t)) == cudaSuccess;
+    ok = ok && cudaMalloc(&v->d_cls, v->cls_bytes) == cudaSuccess;
+    ok = ok && cudaMemcpy(v->d_slots, slots.data(), (size_t)cap * sizeof(u64), cudaMemcpyHostToDevice) == cudaSuccess;
+    ok = ok && cudaMemcpy(v->d_ext_id, ext_id.data(), ext_id.size() * sizeof(int32_t), cudaMemcpyHostToDevice) == cudaSuccess;
+    ok = ok && cudaMemcpy(v->d_cls, cls.data(), v->cls_bytes, cudaMemcpyHostToDevice) == cudaSuccess;
+    if (!ok) { cudaGetLastError(); tt_vocab_free(v); return TT_ERR_CUDA; }
+    v->tab.slots = v->d_slots; v->tab.mask = mask; v->tab.shift = shift;
+    *out = v;
+    return TT_OK;
+}
+
+// ---- workspace layout ----------------------------------------------------------------------------
+static size_t carve(TTWorkspace* w, void* base, size_t max_len, size_t max_docs) {
+    (void)max_docs;
+    const size_t padded = max_len + 64;                       // aligned frame: up to 15 bytes of shift + tail
+    const size_t nchunks = padded / TT_CHUNK + 2;
+    const size_t ntiles = nchunks / TT_TILE_CHUNKS + 2;
+    const size_t nblk = max_len / CNT_THREADS + 2;
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return (char*)base + o; };
+    char* p;
+    p = take(sizeof(TTHeader));                 if (w) w->hdr = (TTHeader*)p;
+    p = take((padded / 32 + 4) * sizeof(u32));  if (w) w->docmask = (u32*)p;
+    p = take(nchunks * sizeof(u16));            if (w) w->startmask = (u16*)p;
+    p = take((ntiles + 1) * sizeof(u32));       if (w) w->tile_cnt = (u32*)p;
+    p = take((max_len + 2) * sizeof(u32));      if (w) w->piece_off = (u32*)p;
+    p = take((max_len + 1) * sizeof(u32));      if (w) w->piece_cnt = (u32*)p;
+    p = take((nblk + 1) * sizeof(u32));         if (w) w->blk_cnt = (u32*)p;
+    p = take((max_len + 2) * sizeof(u32));      if (w) w->tok_off = (u32*)p;
+    p = take((max_len + 1) * sizeof(int32_t));  if (w) w->stage = (int32_t*)p;
+    p = take((max_len + 1) * sizeof(u32));      if (w) w->rank_buf = (u32*)p;
+    p = take((max_len / TT_WARP_PIECE_MAX + 2) * sizeof(u32)); if (w) w->long_list = (u32*)p;
+    return off;
+}
+
+extern "C" size_t tt_workspace_bytes(const tt_vocab* v, size_t max_len, size_t max_docs) {
+    (void)v;
+    return carve(nullptr, nullptr, max_len, max_docs);
+}
+
+#define CK(x) do { if ((x) != cudaSuccess) { cudaGetLastError(); return TT_ERR_CUDA; } } while (0)
+
+// Enqueues K1+K2 and K3.  piece_off_dst receives the offsets (workspace array or the caller's).
+static int run_pretok(const tt_vocab* v, const uint8_t* text, size_t len, const int64_t* doc_off, size_t n_docs,
+                      cudaStream_t st, TTWorkspace& w, u32* piece_off_dst) {
+    const uintptr_t addr = (uintptr_t)text;
+    const long long shift = (long long)(addr & 15);
+    PretokParams P;
+    P.base = (const u8*)(addr - shift);
+    P.lo = shift; P.hi = shift + (long long)len;
+    P.nchunks = (P.hi + TT_CHUNK - 1) / TT_CHUNK;
+    P.ntiles = (int)((P.nchunks + TT_TILE_CHUNKS - 1) / TT_TILE_CHUNKS);
+    P.pattern = v->pattern;
+    P.docmask = nullptr;
+    P.startmask = w.startmask; P.tile_cnt = w.tile_cnt; P.hdr = w.hdr;
+    P.cls_tables = v->d_cls; P.cls_bytes = v->cls_bytes;
+    if (doc_off) {
+        CK(cudaMemsetAsync(w.docmask, 0, ((size_t)P.hi / 32 + 4) * sizeof(u32), st));
+        const int threads = 256, blocks = (int)((n_docs + 1 + threads - 1) / threads);
+        k_docmask<<<blocks, threads, 0, st>>>((const long long*)doc_off, (int)n_docs, shift, (long long)len, w.docmask, w.hdr);
+        P.docmask = w.docmask;
+    }
+    const size_t smem = align_up(v->cls_bytes, 16) + sizeof(u16) * F_COUNT * TT_SLOTS;
+    const int grid = P.ntiles < v->sm_count * 4 ? P.ntiles : v->sm_count * 4;
+    k_pretok<<<grid, TT_TILE_CHUNKS, smem, st>>>(P);
+    k_compact<<<grid, TT_TILE_CHUNKS, 0, st>>>(w.startmask, w.tile_cnt, P.nchunks, P.ntiles, shift, (long long)len,
+                                               piece_off_dst, w.hdr);
+    CK(cudaGetLastError());
+    return TT_OK;
+}
+
+static int check_common(const tt_vocab* v, const void* text, size_t len, void* workspace, size_t workspace_bytes,
+                        size_t n_docs) {
+    if (!v || !workspace || (len && !text)) return TT_ERR_ARG;
+    if (len >= (size_t)INT32_MAX - 64) return TT_ERR_ARG;
+    if (((uintptr_t)workspace & 255) != 0) return TT_ERR_ARG;
+    if (workspace_bytes < tt_workspace_bytes(v, len, n_docs)) return TT_ERR_ARG;
+    return TT_OK;
+}
+
+static int encode_impl(const tt_vocab* v, const uint8_t* text, size_t len, const int64_t* doc_off, size_t n_docs,
+                       cudaStream_t st, int32_t* ids_out, size_t ids_cap, int64_t* count_out, int64_t* ids_off_out,
+                       int32_t* status_out, void* workspace) {
+    TTWorkspace w;
+    carve(&w, workspace, len, n_docs);
+    CK(cudaMemsetAsync(w.hdr, 0, sizeof(TTHeader), st));
+    if (len == 0) {
+        if (count_out) CK(cudaMemsetAsync(count_out, 0, sizeof(int64_t), st));
+        if (ids_off_out) CK(cudaMemsetAsync(ids_off_out, 0, (n_docs + 1) * sizeof(int64_t), st));
+        CK(cudaMemsetAsync(status_out, 0, sizeof(int32_t), st));
+        return TT_OK;
+    }
+    int rc = run_pretok(v, text, len, doc_off, n_docs, st, w, w.piece_off);
+    if (rc != TT_OK) return rc;
+    const int bpe_grid = v->sm_count * 8;
+    k_bpe_warp<<<bpe_grid, BPE_WARPS * 32, 0, st>>>(text, w.piece_off, w.hdr, v->tab, v->d_ext_id, w.piece_cnt, w.stage,
+                                                    w.long_list);
+    k_bpe_long<<<v->sm_count, LONG_THREADS, 0, st>>>(text, w.piece_off, w.hdr, v->tab, v->d_ext_id, w.piece_cnt, w.stage,
+                                                     w.rank_buf, w.long_list);
+    const int nblk = (int)((len + CNT_THREADS - 1) / CNT_THREADS);
+    k_count<<<nblk, CNT_THREADS, 0, st>>>(w.piece_cnt, w.hdr, w.blk_cnt, (unsigned long long)ids_cap);
+    k_scatter<<<nblk, CNT_THREADS, 0, st>>>(w.piece_off, w.piece_cnt, w.blk_cnt, w.stage, w.hdr, w.tok_off, ids_out,
+                                            (long long*)count_out, status_out);
+    if (doc_off) {
+        const int threads = 256, blocks = (int)((n_docs + 1 + threads - 1) / threads);
+        k_doc_offsets<<<blocks, threads, 0, st>>>((const long long*)doc_off, (int)n_docs, w.piece_off, w.tok_off, w.hdr,
+                                                  (long long*)ids_off_out);
+    }
+    CK(cudaGetLastError());
+    return TT_OK;
+}
+
+extern "C" int tt_encode(const tt_vocab* v, const uint8_t* text, size_t len, void* stream, int32_t* ids_out,
+                         size_t ids_cap, int64_t* count_out, int32_t* status_out, void* workspace,
+                         size_t workspace_bytes) {
+    int rc = check_common(v, text, len, workspace, workspace_bytes, 1);
+    if (rc != TT_OK) return rc;
+    if (!count_out || !status_out || (len && !ids_out)) return TT_ERR_ARG;
+    return encode_impl(v, text, len, nullptr, 1, (cudaStream_t)stream, ids_out, ids_cap, count_out, nullptr, status_out,
+                       workspace);
+}
+
+extern "C" int tt_encode_batch(const tt_vocab* v, const uint8_t* text, size_t total_len, const int64_t* doc_off,
+                               size_t n_docs, void* stream, int32_t* ids_out, size_t ids_cap, int64_t* ids_off_out,
+                               int32_t* status_out, void* workspace, size_t workspace_bytes) {
+    int rc = check_common(v, text, total_len, workspace, workspace_bytes, n_docs);
+    if (rc != TT_OK) return rc;
+    if (!doc_off || !ids_off_out || !status_out || (total_len && !ids_out) || n_docs >= (size_t)INT32_MAX) return TT_ERR_ARG;
+    return encode_impl(v, text, total_len, doc_off, n_docs, (cudaStream_t)stream, ids_out, ids_cap, nullptr, ids_off_out,
+                       status_out, workspace);
+}
+
+__global__ void k_finish_pretok(const TTHeader* hdr, long long* n_pieces_out, int32_t* status_out) {
+    *status_out = hdr->status;
+    *n_pieces_out = hdr->status ? 0 : (long long)hdr->n_pieces;
+}
+
+extern "C" int tt_pretokenize(const tt_vocab* v, const uint8_t* text, size_t len, const int64_t* doc_off, size_t n_docs,
+                              void* stream, int32_t* piece_off_out, size_t piece_cap, int64_t* n_pieces_out,
+                              int32_t* status_out, void* workspace, size_t workspace_bytes) {
+    int rc = check_common(v, text, len, workspace, workspace_bytes, n_docs);
+    if (rc != TT_OK) return rc;
+    if (!n_pieces_out || !status_out || (len && !piece_off_out) || piece_cap < len + 1) return TT_ERR_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    TTWorkspace w;
+    carve(&w, workspace, len, n_docs);
+    CK(cudaMemsetAsync(w.hdr, 0, sizeof(TTHeader), st));
+    if (len == 0) {
+        CK(cudaMemsetAsync(n_pieces_out, 0, sizeof(int64_t), st));
+        CK(cudaMemsetAsync(status_out, 0, sizeof(int32_t), st));
+        return TT_OK;
+    }
+    rc = run_pretok(v, text, len, doc_off, n_docs, st, w, (u32*)piece_off_out);
+    if (rc != TT_OK) return rc;
+    k_finish_pretok<<<1, 1, 0, st>>>(w.hdr, (long long*)n_pieces_out, status_out);
+    CK(cudaGetLastError());
+    return TT_OK;
+}
+
+extern "C" int tt_encode_host(tt_vocab* v, const uint8_t* text, size_t len, int32_t* ids_out, size_t ids_cap,
+                              int64_t* count_out) {
+    if (!v || !count_out || (len && (!text || !ids_out))) return TT_ERR_ARG;
+    if (len >= (size_t)INT32_MAX - 64) return TT_ERR_ARG;
+    *count_out = 0;
+    if (!v->host_stream) CK(cudaStreamCreateWithFlags(&v->host_stream, cudaStreamNonBlocking));
+    if (len + 1 > v->host_cap) {
+        cudaFree(v->d_text); cudaFree(v->d_ids); cudaFree(v->d_ws);
+        if (v->h_text) cudaFreeHost(v->h_text);
+        if (v->h_ids) cudaFreeHost(v->h_ids);
+        v->d_text = nullptr; v->d_ids = nullptr; v->d_ws = nullptr; v->h_text = nullptr; v->h_ids = nullptr; v->host_cap = 0;
+        const size_t cap = align_up(len + 1 + len / 4, 4096);
+        v->ws_cap = tt_workspace_bytes(v, cap, 1);
+        CK(cudaMalloc(&v->d_text, cap + 64));
+        CK(cudaMalloc(&v->d_ids, cap * sizeof(int32_t)));
+        CK(cudaMalloc(&v->d_ws, v->ws_cap));
+        CK(cudaMallocHost(&v->h_text, cap + 64));
+        CK(cudaMallocHost(&v->h_ids, cap * sizeof(int32_t)));
+        if (!v->d_count) CK(cudaMalloc(&v->d_count, sizeof(long long)));
+        if (!v->d_status) CK(cudaMalloc(&v->d_status, sizeof(int32_t)));
+        if (!v->h_scalars) CK(cudaMallocHost(&v->h_scalars, 2 * sizeof(long long)));
+        v->host_cap = cap;
+    }
+    cudaStream_t st = v->host_stream;
+    memcpy(v->h_text, text, len);
+    CK(cudaMemcpyAsync(v->d_text, v->h_text, len, cudaMemcpyHostToDevice, st));
+    int rc = tt_encode(v, v->d_text, len, st, v->d_ids, v->host_cap, (int64_t*)v->d_count, v->d_status, v->d_ws, v->ws_cap);
+    if (rc != TT_OK) return rc;
+    CK(cudaMemcpyAsync(&v->h_scalars[0], v->d_count, sizeof(long long), cudaMemcpyDeviceToHost, st));
+    CK(cudaMemcpyAsync(&v->h_scalars[1], v->d_status, sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+    CK(cudaStreamSynchronize(st));
+    const int status = (int)(v->h_scalars[1] & 0xFFFFFFFF);
+    if (status != TT_OK) return status;
+    const long long n = v->h_scalars[0];
+    if ((size_t)n > ids_cap) return TT_ERR_CAPACITY;
+    CK(cudaMemcpyAsync(v->h_ids, v->d_ids, (size_t)n * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+    CK(cudaStreamSynchronize(st));
+    memcpy(ids_out, v->h_ids, (size_t)n * sizeof(int32_t));
+    *count_out = n;
+    return TT_OK;
+}

@@ -1,0 +1,64 @@
+// Shared definitions of the toktier CUDA library (sm_100a).
+#pragma once
+#include <cstdint>
+#include <cstddef>
+#include <cuda_runtime.h>
+
+#if defined(__CUDACC__)
+#define TT_HD __host__ __device__ __forceinline__
+#else
+#define TT_HD inline
+#endif
+
+typedef uint8_t u8;
+typedef uint16_t u16;
+typedef uint32_t u32;
+typedef uint64_t u64;
+
+// ---- geometry of the pre-tokenization pass -------------------------------------------------
+// A chunk is one aligned 16-byte vector load; a tile is what one CTA classifies per iteration.
+constexpr int TT_CHUNK = 16;
+#ifndef TT_TILE_CHUNKS_DEF
+#define TT_TILE_CHUNKS_DEF 256
+#endif
+constexpr int TT_TILE_CHUNKS = TT_TILE_CHUNKS_DEF;        // = threads per CTA
+constexpr int TT_TILE_BYTES = TT_CHUNK * TT_TILE_CHUNKS; // 4 KiB of text per tile
+
+// ---- character class codes (two-stage Unicode table, see gen_unicode_table.py) ------------
+enum : u32 { CC_OTHER = 0, CC_MARK = 1, CC_SPACE = 2, CC_NUMBER = 3, CC_LOWER = 4, CC_UPPER = 5, CC_CASELESS = 6 };
+
+// ---- BPE -----------------------------------------------------------------------------------
+constexpr u32 TT_ID_BITS = 18;                    // internal ids: byte b -> b, merge of rank r -> 256 + r
+constexpr u32 TT_MAX_INTERNAL = 1u << TT_ID_BITS;
+constexpr u32 TT_RANK_INF = 0xFFFFFFFFu;
+constexpr u64 TT_SLOT_EMPTY = ~0ull;              // pair-table slot: (left << 38) | (right << 20) | rank
+constexpr int TT_WARP_PIECE_MAX = 256;            // bytes; longer pieces take the block-cooperative path
+
+// ---- workspace header (device memory, zeroed at the start of every call) --------------------
+struct TTHeader {
+    int status;              // TT_OK or a device-side error code
+    u32 pretok_done;         // CTAs that finished the pre-tokenization pass
+    u32 count_done;          // CTAs that finished the token-count reduction
+    u32 n_pieces;            // number of pieces found
+    u32 n_long;              // entries in the long-piece list
+    u32 long_next;           // work counter of the long-piece kernel
+    u32 piece_next;          // work counter of the warp BPE kernel
+    u32 pad0;
+    unsigned long long n_tokens;   // total tokens
+    u32 pad[22];
+};
+static_assert(sizeof(TTHeader) == 128, "header layout");
+
+struct TTWorkspace {
+    TTHeader* hdr;
+    u32* docmask;      // bit per text byte: first byte of a document (batch only)
+    u16* startmask;    // bit per text byte: first byte of a piece (one u16 per chunk)
+    u32* tile_cnt;     // pieces per tile, then exclusive prefix (ntiles + 1)
+    u32* piece_off;    // byte offset of every piece + sentinel (len + 2)
+    u32* piece_cnt;    // tokens per piece (len + 1)
+    u32* blk_cnt;      // token count per block of pieces, then exclusive prefix
+    u32* tok_off;      // token offset of every piece + total (len + 2)
+    int32_t* stage;    // token ids staged at the byte offset of their piece (len)
+    u32* rank_buf;     // per-position ranks for the long-piece path (len)
+    u32* long_list;    // piece indices longer than TT_WARP_PIECE_MAX
+};

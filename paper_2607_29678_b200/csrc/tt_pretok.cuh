@@ -1,0 +1,218 @@
+// Steps K2 and K3: run-local piece-start rules and stream compaction.
+//
+// Paper Sec. 4.1: whether a character begins a piece depends only on its offset within its
+// maximal same-class run, a few characters of look-back across the run boundary, and per-run
+// aggregates of whitespace runs (run start, first non-CR/LF position, last CR/LF position); the
+// test is an independent per-character predicate.  Here one thread evaluates the predicate for the
+// 16 bytes of its chunk as bit-parallel operations on class masks (bit i <-> byte i) over a 48-byte
+// window (previous, own, next chunk).  Aggregates that reach further (offset mod 3 inside a number
+// run, CR/LF runs glued to preceding punctuation, "is there a CR/LF later in this whitespace run")
+// are resolved by walking chunk summaries in shared memory and, beyond the tile, by a bounded
+// CTA-cooperative walk over the text itself -- no CTA ever waits for another CTA.
+#pragma once
+#include "tt_classify.cuh"
+
+enum { F_LEAD = 0, F_OTH, F_MARK, F_SPC, F_NUM, F_LOW, F_UPP, F_CLESS, F_NL, F_SP, F_AP, F_SL, F_DOC, F_COUNT };
+constexpr int TT_SLOTS = TT_TILE_CHUNKS + 2;          // tile plus one halo chunk on each side
+
+enum { NEED_N = 1, NEED_A = 2, NEED_F = 4 };
+
+struct PretokParams {
+    const u8* base;          // 16-byte aligned address at or below the text
+    long long lo, hi;        // the text occupies [lo, hi) in the aligned frame
+    long long nchunks;       // ceil(hi / 16)
+    int ntiles;
+    int pattern;
+    const u32* docmask;      // bit per byte (aligned frame) marking document starts, or null (one document)
+    u16* startmask;          // out: one u16 per chunk
+    u32* tile_cnt;           // out: pieces per tile; replaced by the exclusive prefix (ntiles + 1 entries)
+    TTHeader* hdr;
+    const u8* cls_tables;    // stage1 | stage2 | ascii, contiguous in global memory
+    int cls_bytes;
+};
+
+struct TileCarry {           // aggregates of runs that enter or leave the shared-memory window
+    u32 n_before;            // number leads (mod 3) of the number run ending right before the low halo chunk
+    u32 nl_absorbed_before;  // the CR/LF run ending right before the low halo chunk is glued to punctuation
+    u32 nl_later_after;      // the whitespace run leaving the high halo chunk still contains a CR/LF
+};
+
+TT_HD u64 tt_win(const u16 (*sm)[TT_SLOTS], int f, int slot) {
+    return (u64)sm[f][slot - 1] | ((u64)sm[f][slot] << 16) | ((u64)sm[f][slot + 1] << 32);
+}
+
+TT_HD int tt_hibit(u32 x) {   // position of the highest set bit, x != 0
+#if defined(__CUDA_ARCH__)
+    return 31 - __clz(x);
+#else
+    return 31 - __builtin_clz(x);
+#endif
+}
+TT_HD int tt_lobit(u32 x) {   // position of the lowest set bit, x != 0
+#if defined(__CUDA_ARCH__)
+    return __ffs(x) - 1;
+#else
+    return __builtin_ctz(x);
+#endif
+}
+TT_HD int tt_popc(u32 x) {
+#if defined(__CUDA_ARCH__)
+    return __popc(x);
+#else
+    return __builtin_popcount(x);
+#endif
+}
+
+// Number leads in the number run that ends at the last byte of slot `s` (walking down).
+// Returns the count; sets `open` when the run continues below slot 0.
+TT_HD u32 tt_walk_back_num(const u16 (*sm)[TT_SLOTS], int s, bool& open) {
+    u32 cnt = 0;
+    open = false;
+    for (; s >= 0; s--) {
+        u32 n = sm[F_NUM][s], d = sm[F_DOC][s], ld = sm[F_LEAD][s];
+        u32 cut = (~n & 0xFFFFu) | (d >> 1);        // byte j ends the walk if it is not a number byte or j+1 starts a document
+        if (cut) { int b = tt_hibit(cut); cnt += tt_popc(ld & n & (0xFFFFu << (b + 1)) & 0xFFFFu); return cnt; }
+        cnt += tt_popc(ld & n);
+        if (d & 1) return cnt;                      // run starts at a document start
+    }
+    open = true;
+    return cnt;
+}
+
+// Is the CR/LF run that ends at the last byte of slot `s` glued to a preceding punctuation char?
+// (0 / 1; `open` when the run continues below slot 0.)
+TT_HD u32 tt_walk_back_nl(const u16 (*sm)[TT_SLOTS], int s, u32 othmask_fields, bool& open) {
+    open = false;
+    for (; s >= 0; s--) {
+        u32 nl = sm[F_NL][s], d = sm[F_DOC][s];
+        u32 cut = (~nl & 0xFFFFu) | (d >> 1);
+        if (cut) {
+            int b = tt_hibit(cut);
+            if ((d >> 1) >> b & 1) return 0;        // the run starts at a document start
+            u32 o = sm[F_OTH][s] | (othmask_fields ? sm[F_MARK][s] : 0);
+            return (o >> b) & 1;
+        }
+        if (d & 1) return 0;
+    }
+    open = true;
+    return 0;
+}
+
+// Does the whitespace run that contains byte `bit` of slot `s` contain a CR/LF above that byte?
+TT_HD u32 tt_walk_fwd_nl(const u16 (*sm)[TT_SLOTS], int s, int bit, bool& open) {
+    open = false;
+    u32 low = (0xFFFFu << (bit + 1)) & 0xFFFFu;
+    for (; s < TT_SLOTS; s++) {
+        u32 w = sm[F_SPC][s], nl = sm[F_NL][s], d = sm[F_DOC][s];
+        u32 ev = ((~w) | d | nl) & low;
+        if (ev) { int j = tt_lobit(ev); return ((nl & w & ~d) >> j) & 1; }
+        low = 0xFFFFu;
+    }
+    open = true;
+    return 0;
+}
+
+// Contraction suffix length at the apostrophe whose two following bytes are b1, b2 (0 = none).
+TT_HD int tt_contraction_len(u32 b1, u32 b2) {
+    const u32 a = b1 | 0x20, b = b2 | 0x20;       // ASCII case fold; no other byte maps onto these letters
+    if (a == 's' || a == 't' || a == 'm' || a == 'd') return 2;
+    if ((a == 'r' && b == 'e') || (a == 'v' && b == 'e') || (a == 'l' && b == 'l')) return 3;
+    return 0;
+}
+
+// Pattern 0 (cl100k-style).  Returns the 16 start bits of the chunk in `slot`; `need` receives the
+// NEED_* flags of aggregates that leave the shared-memory window (then `tc` must be filled and the
+// function called again).
+TT_HD u32 tt_eval_chunk_p0(const u16 (*sm)[TT_SLOTS], int slot, const u8* base, long long g0, long long hi,
+                           const TileCarry& tc, bool have_tc, u32& need) {
+    const u64 OWN = 0xFFFFull << 16;
+    const u64 lead = tt_win(sm, F_LEAD, slot);
+    const u64 L = tt_win(sm, F_LOW, slot) | tt_win(sm, F_UPP, slot) | tt_win(sm, F_CLESS, slot);
+    const u64 N = tt_win(sm, F_NUM, slot);
+    const u64 W = tt_win(sm, F_SPC, slot);
+    const u64 O = tt_win(sm, F_OTH, slot) | tt_win(sm, F_MARK, slot);
+    const u64 NL = tt_win(sm, F_NL, slot), SP = tt_win(sm, F_SP, slot), AP = tt_win(sm, F_AP, slot);
+    const u64 D = tt_win(sm, F_DOC, slot);
+    const u64 V = L | N | W | O;                       // bytes that exist and are valid
+    const u64 cont = V & ~lead;
+    const u64 nD = ~D;
+    u64 S = 0;
+#define PREV(x) (((x) << 1) & nD)
+    // punctuation runs: start of the run, unless a blank precedes it (the blank starts the piece)
+    const u64 G = O & lead & ~PREV(O) & ~PREV(SP);
+    S |= G;
+    // letter runs: the run start, unless non-CR/LF whitespace or a single match-start punctuation char precedes it
+    const u64 c1 = cont << 1, c2 = cont << 2, c3 = cont << 3;
+    const u64 pfx = ((G << 1) | ((G << 2) & c1) | ((G << 3) & c2 & c1) | ((G << 4) & c3 & c2 & c1)) & nD;
+    S |= L & lead & ~PREV(L) & ~((PREV(W) & ~PREV(NL)) | pfx);
+    // contractions: apostrophe that is a match start, then s/t/m/d or re/ve/ll; the letter after the suffix starts a piece
+    u64 ga = G & AP & (0x3FFFFull << 12);              // apostrophes at own bytes -4 .. +13 can put a start into this chunk
+    while (ga) {
+        int p = tt_lobit((u32)(ga >> 12)) + 12; ga &= ga - 1;
+        long long g = g0 + (p - 16);
+        u32 b1 = (g + 1 < hi) ? base[g + 1] : 0, b2 = (g + 2 < hi) ? base[g + 2] : 0;
+        if ((D >> (p + 1)) & 1) b1 = 0;
+        if ((D >> (p + 2)) & 1) b2 = 0;
+        int cl = tt_contraction_len(b1, b2);
+        if (cl) {
+            u64 at = 1ull << (p + cl);
+            bool same_doc = ((D >> (p + 1)) & ((1ull << cl) - 1)) == 0;
+            if (same_doc) S |= at & L & lead;
+        }
+    }
+    // number runs: every third number lead counted from the run start
+    {
+        u32 n_own = (u32)(N >> 16) & 0xFFFFu, ld_own = (u32)(lead >> 16) & 0xFFFFu;
+        u32 nstart = (u32)((N & ~PREV(N)) >> 16) & 0xFFFFu;
+        u32 m = n_own & ld_own;
+        if (m) {
+            u32 cnt = 0;
+            if ((n_own & 1) && !(nstart & 1)) {            // the run enters from the previous chunk
+                bool open;
+                cnt = tt_walk_back_num(sm, slot - 1, open);
+                if (open) { if (have_tc) cnt += tc.n_before; else need |= NEED_N; }
+                cnt %= 3;
+            }
+            while (m) {
+                int i = tt_lobit(m); m &= m - 1;
+                if ((nstart >> i) & 1) cnt = 0;
+                if (cnt == 0) S |= 1ull << (16 + i);
+                cnt = cnt == 2 ? 0 : cnt + 1;
+            }
+        }
+    }
+    // whitespace runs
+    if (W & OWN) {
+        // (a) run start, unless it is a CR/LF glued to preceding punctuation
+        S |= W & lead & ~PREV(W) & ~(PREV(O) & NL);
+        // (b) CR/LF absorbed by preceding punctuation: CR/LF runs that begin right after punctuation
+        u32 nl_own = (u32)(NL >> 16) & 0xFFFFu, d_own = (u32)(D >> 16) & 0xFFFFu;
+        u32 prev_absorbed = 0;                             // byte before the chunk is an absorbed CR/LF
+        if (((NL >> 15) & 1) && !(d_own & 1)) {
+            bool open;
+            prev_absorbed = tt_walk_back_nl(sm, slot - 1, 1, open);
+            if (open) { if (have_tc) prev_absorbed = tc.nl_absorbed_before; else need |= NEED_A; }
+        }
+        u32 nlq = nl_own & ~d_own;
+        u32 sel = (u32)(((NL & ~PREV(NL) & PREV(O)) >> 16) & 0xFFFFu) | ((nlq & 1) ? prev_absorbed : 0);
+        u32 absorbed = nlq & ~(nlq + sel);
+        u64 prevA = (((u64)absorbed << 17) | ((u64)prev_absorbed << 16)) & nD;
+        S |= W & lead & ~NL & prevA;
+        // (c) last character of the run when something follows in the same document (and it is not CR/LF)
+        const u64 next_exists = (V >> 1) & ~(D >> 1);
+        const u64 wend = W & ~((W >> 1) & ~(D >> 1)) & next_exists;
+        const u64 k1 = cont >> 1, k2 = cont >> 2, k3 = cont >> 3;
+        S |= lead & W & ~NL & (wend | ((wend >> 1) & k1) | ((wend >> 2) & k1 & k2) | ((wend >> 3) & k1 & k2 & k3));
+        // (d) first character after the last CR/LF of the run
+        u32 cand = (u32)((W & lead & ~NL & PREV(NL)) >> 16) & 0xFFFFu;
+        while (cand) {
+            int i = tt_lobit(cand); cand &= cand - 1;
+            bool open;
+            u32 later = tt_walk_fwd_nl(sm, slot, i, open);
+            if (open) { if (have_tc) later = tc.nl_later_after; else { need |= NEED_F; later = 1; } }
+            if (!later) S |= 1ull << (16 + i);
+        }
+    }
+#undef PREV
+    return (u32)((S & lead & OWN) >> 16);
+}

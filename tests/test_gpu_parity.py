@@ -1,0 +1,217 @@
+"""GPU parity: the CUDA path (through the C ABI) against the CPU oracle, element by element, at the
+level of piece boundaries and at the level of token IDs (paper Sec. 4.1: both levels are needed,
+because ID agreement can hide a boundary fault).  Bit-exact is the only tolerance."""
+import itertools
+import random
+
+import numpy as np
+import pytest
+
+import oracle
+import workloads as wl
+from gpu_util import cpu_vocab, gpu_encode, gpu_encode_batch, gpu_pretok, gpu_vocab
+
+pytestmark = pytest.mark.gpu
+
+TILE = 4096
+
+
+def _expect_pieces(text, pattern):
+    return oracle.pretokenize(text, pattern)
+
+
+@pytest.mark.parametrize("name,n_chars", [("C1", None), ("C2", None), ("C3", None), ("C4", 400_000)])
+def test_piece_offsets_match_oracle(name, n_chars):
+    cfg = wl.CONFIGS[name]
+    text = wl.request(cfg, n_chars=n_chars)
+    got, status = gpu_pretok(gpu_vocab(name), text)
+    assert status == 0
+    want = _expect_pieces(text, cfg.pattern_id)
+    assert got.size == want.size and np.array_equal(got, want)
+
+
+@pytest.mark.parametrize("name,n_chars", [("C1", None), ("C2", None), ("C3", None), ("C4", 400_000)])
+def test_token_ids_match_oracle(name, n_chars):
+    cfg = wl.CONFIGS[name]
+    text = wl.request(cfg, n_chars=n_chars)
+    ids, status = gpu_encode(gpu_vocab(name), text)
+    assert status == 0
+    want, _ = cpu_vocab(name).encode(text, cfg.pattern_id, nthreads=4)
+    assert ids.size == want.size and np.array_equal(ids, want)
+
+
+@pytest.mark.parametrize("pattern", [0, 1])
+@pytest.mark.parametrize("offset", [0, 1, 7, 15])
+def test_misaligned_text_pointer(pattern, offset):
+    name = "C2" if pattern == 0 else "C4"
+    text = wl.generate(wl.KIND_MIX_UNI, 77 + offset, 30_000)
+    got, status = gpu_pretok(gpu_vocab(name), text, offset=offset)
+    assert status == 0 and np.array_equal(got, _expect_pieces(text, pattern))
+    ids, status = gpu_encode(gpu_vocab(name), text, offset=offset)
+    want, _ = cpu_vocab(name).encode(text, pattern)
+    assert status == 0 and np.array_equal(ids, want)
+
+
+def _alphabet_docs(alphabet, maxlen):
+    docs = []
+    for ln in range(1, maxlen + 1):
+        for tup in itertools.product(alphabet, repeat=ln):
+            docs.append("".join(tup).encode("utf-8"))
+    return docs
+
+
+def _batch_pieces_check(name, pattern, docs):
+    text = np.frombuffer(b"".join(docs), dtype=np.uint8)
+    off = np.zeros(len(docs) + 1, dtype=np.int64)
+    off[1:] = np.cumsum([len(d) for d in docs])
+    got, status = gpu_pretok(gpu_vocab(name), text, doc_off=off)
+    assert status == 0
+    want = []
+    for i, d in enumerate(docs):
+        want.extend((oracle.pretokenize(d, pattern) + off[i]).tolist())
+    want = np.asarray(want, dtype=np.int64)
+    if got.size != want.size or not np.array_equal(got, want):
+        bad = sorted(set(got.tolist()) ^ set(want.tolist()))[:5]
+        which = [int(np.searchsorted(off, b, side="right") - 1) for b in bad]
+        raise AssertionError(f"piece mismatch in documents {[docs[w] for w in which]}")
+
+
+@pytest.mark.parametrize("alphabet,maxlen", [
+    ("as1 \t\n!'", 5), ("rRevl't !", 5), ("eé中²́ 　\n's", 4), ("a1 \r\n !", 5)])
+def test_exhaustive_small_alphabets_pattern0(alphabet, maxlen):
+    """Every string over a small alphabet, each as its own document of one batch call."""
+    _batch_pieces_check("C1", 0, _alphabet_docs(alphabet, maxlen))
+
+
+@pytest.mark.parametrize("alphabet,maxlen", [
+    ("á's/\n !", 5), ("Aal's1 \n/", 5), ("Aa中́'s !/\n", 4), ("AaBb中́1 \t", 5), ("ǅaʰA'l \r", 5)])
+def test_exhaustive_small_alphabets_pattern1(alphabet, maxlen):
+    _batch_pieces_check("C4", 1, _alphabet_docs(alphabet, maxlen))
+
+
+SEAM_CONSTRUCTS = ["don't", "x's's's", " \n \n  x", "1234567", "é中😀²", "!!!\n\n\nabc", "a   b", "\r\n\r\n", "'re're",
+                   "A中B", "HelloWORLDab", "!\n/\n/x", "x́\ny", " 　 z", "12'll3", "a\n\n\n\n\n\n\n\n\n\n\n\n\n\n\n\n\n\nb"]
+
+
+@pytest.mark.parametrize("pattern", [0, 1])
+def test_constructs_at_every_tile_seam_position(pattern):
+    """Each construct is placed so that every one of its bytes falls on a tile boundary once."""
+    name = "C2" if pattern == 0 else "C4"
+    rng = random.Random(pattern)
+    for cons in SEAM_CONSTRUCTS:
+        cb = cons.encode("utf-8")
+        docs = []
+        for k in range(-4, len(cb) + 5):
+            pad = TILE - k
+            filler = wl.generate(wl.KIND_MIX, rng.randrange(1 << 30), TILE)[:max(pad, 0)].tobytes()
+            docs.append(filler + cb + b" tail text 123\n")
+        _batch_pieces_check(name, pattern, docs)
+
+
+@pytest.mark.parametrize("pattern", [0, 1])
+def test_long_runs_across_tiles(pattern):
+    name = "C2" if pattern == 0 else "C4"
+    rng = random.Random(100 + pattern)
+    docs = []
+    for _ in range(60):
+        parts = []
+        for _ in range(rng.randrange(1, 5)):
+            k = rng.randrange(8)
+            if k == 0:
+                parts.append("7" * rng.randrange(1, 13000))
+            elif k == 1:
+                parts.append(rng.choice(["", "!", "a", "\n", "!\n"]) + " " * rng.randrange(1, 13000) + rng.choice(["", "x", "\n", "!", "1"]))
+            elif k == 2:
+                parts.append(rng.choice(["!", "a", ""]) + "\n" * rng.randrange(1, 9000) + rng.choice(["", " ", "  x", "/"]))
+            elif k == 3:
+                parts.append(rng.choice([";\n", "", "a"]) + rng.choice(["/", "'", "=", "-"]) * rng.randrange(1, 9000))
+            elif k == 4:
+                parts.append("٣" * rng.randrange(1, 5000))
+            elif k == 5:
+                parts.append(rng.choice(["!", "a"]) + "\r\n" * rng.randrange(1, 3000) + "\t " * rng.randrange(0, 3000) + "z")
+            elif k == 6:
+                parts.append("中" * rng.randrange(1, 3000) + "ABC" + "é" * rng.randrange(1, 3000))
+            else:
+                parts.append(" " * rng.randrange(1, 5000) + "\n" * rng.randrange(1, 5000) + " " * rng.randrange(1, 5000))
+        docs.append("".join(parts).encode("utf-8"))
+    _batch_pieces_check(name, pattern, docs)
+
+
+def test_batch_ids_match_documents_alone():
+    cfg = wl.CONFIGS["C5"]
+    text, off = wl.batch(cfg, n_docs=12, scale=0.02)
+    off = np.concatenate([off[:5], [off[4]], off[5:]]).astype(np.int64)   # an empty document in the middle
+    ids, ioff, status = gpu_encode_batch(gpu_vocab("C5"), text, off)
+    assert status == 0
+    want, woff = cpu_vocab("C5").encode_batch(text, off, cfg.pattern_id, nthreads=4)
+    assert np.array_equal(ioff, woff)
+    assert np.array_equal(ids, want)
+
+
+def test_adversarial_long_pieces_ids():
+    """64 KB blanks/tabs, 20,000 digits and 50 KB of one punctuation character (pattern 1 vocabulary)."""
+    cfg = wl.CONFIGS["C4"]
+    v, cv = gpu_vocab("C4"), cpu_vocab("C4")
+    for piece in (b"x" + b" " * 65536 + b"y", b"\n" + b"\t" * 65536, b"9" * 20000, b";\n" + b"/" * 51200 + b"a",
+                  b"'" * 51200, b"=" * 51200 + b"\n", ("中" * 3000).encode(), b" \t" * 32768):
+        text = np.frombuffer(piece, dtype=np.uint8)
+        ids, status = gpu_encode(v, text)
+        want, _ = cv.encode(text, cfg.pattern_id)
+        assert status == 0 and np.array_equal(ids, want), piece[:20]
+
+
+def test_edge_cases_and_status_codes():
+    import paper_2607_29678_b200 as tt
+    v = gpu_vocab("C1")
+    ids, status = gpu_encode(v, np.zeros(0, dtype=np.uint8))
+    assert status == 0 and ids.size == 0
+    for one in (b"a", b" ", b"\n", b"7", b"'", "中".encode(), "😀".encode(), b"\x00"):
+        ids, status = gpu_encode(v, np.frombuffer(one, dtype=np.uint8))
+        want, _ = cpu_vocab("C1").encode(one, 0)
+        assert status == 0 and np.array_equal(ids, want)
+    for bad in (b"abc\x80def", b"\xc3", b"ab\xe4\xb8", b"\xc0\xaf", b"\xed\xa0\x80", b"\xf4\x90\x80\x80", b"x" * 5000 + b"\xff"):
+        ids, status = gpu_encode(v, np.frombuffer(bad, dtype=np.uint8))
+        assert status == tt.TT_ERR_INVALID_UTF8 and ids.size == 0
+    text = wl.request(wl.CONFIGS["C1"])
+    ids, status = gpu_encode(v, text, ids_cap=10)
+    assert status == tt.TT_ERR_CAPACITY and ids.size == 0
+    # the handle is still usable after errors
+    ids, status = gpu_encode(v, text)
+    want, _ = cpu_vocab("C1").encode(text, 0)
+    assert status == 0 and np.array_equal(ids, want)
+
+
+def test_host_wrapper_and_non_identity_ids():
+    import paper_2607_29678_b200 as tt
+    rng = random.Random(4)
+    perm = list(range(256))
+    rng.shuffle(perm)
+    byte_map = np.array([5000 + p for p in perm], dtype=np.int32)
+    base, _ = wl.load_vocab(wl.CONFIGS["C1"])
+    remap = {i: int(byte_map[i]) for i in range(256)}
+    remap.update({256 + r: 100_000 + 3 * r for r in range(base.shape[0])})
+    merges = np.array([[remap[a], remap[b], remap[c]] for a, b, c in base.tolist()], dtype=np.int32)
+    gv = tt.Vocab(merges, byte_map, 0)
+    cv = oracle.Vocab(merges, byte_map)
+    text = wl.request(wl.CONFIGS["C1"])
+    want, _ = cv.encode(text, 0)
+    assert np.array_equal(gv.encode_host(text), want)
+    ids, status = gpu_encode(gv, text)
+    assert status == 0 and np.array_equal(ids, want)
+
+
+def test_result_does_not_depend_on_schedule():
+    """Same input, repeated calls and a reused workspace: identical output every time."""
+    import torch
+    cfg = wl.CONFIGS["C2"]
+    v = gpu_vocab("C2")
+    text = wl.request(cfg)
+    from gpu_util import to_dev
+    d = to_dev(text)
+    bufs = v.alloc(text.size)
+    outs = []
+    for _ in range(3):
+        v.encode(d, bufs)
+        torch.cuda.synchronize()
+        outs.append(bufs["ids"][:int(bufs["count"].item())].cpu().numpy().copy())
+    assert np.array_equal(outs[0], outs[1]) and np.array_equal(outs[0], outs[2])

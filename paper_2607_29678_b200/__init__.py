@@ -18,7 +18,7 @@ TT_OK, TT_ERR_ARG, TT_ERR_BAD_VOCAB, TT_ERR_CUDA, TT_ERR_INVALID_UTF8, TT_ERR_CA
 TT_PATTERN_CL100K, TT_PATTERN_O200K = 0, 1
 
 EXPORTS = ["tt_vocab_load", "tt_vocab_free", "tt_workspace_bytes", "tt_encode", "tt_encode_batch",
-           "tt_pretokenize", "tt_encode_host", "tt_class_table", "tt_strerror"]
+           "tt_pretokenize", "tt_encode_timed", "tt_encode_host", "tt_class_table", "tt_strerror"]
 
 _lib = None
 
@@ -52,6 +52,9 @@ def lib() -> ctypes.CDLL:
         L.tt_pretokenize.restype = c.c_int
         L.tt_pretokenize.argtypes = [c.c_void_p, c.c_void_p, c.c_size_t, c.c_void_p, c.c_size_t, c.c_void_p, c.c_void_p,
                                      c.c_size_t, c.c_void_p, c.c_void_p, c.c_void_p, c.c_size_t]
+        L.tt_encode_timed.restype = c.c_int
+        L.tt_encode_timed.argtypes = [c.c_void_p, c.c_void_p, c.c_size_t, c.c_void_p, c.c_void_p, c.c_size_t, c.c_void_p,
+                                      c.c_void_p, c.c_void_p, c.c_size_t, c.POINTER(c.c_float)]
         L.tt_encode_host.restype = c.c_int
         L.tt_encode_host.argtypes = [c.c_void_p, c.c_void_p, c.c_size_t, c.c_void_p, c.c_size_t, c.POINTER(c.c_int64)]
         L.tt_class_table.restype = c.c_size_t
@@ -132,6 +135,17 @@ class Vocab:
         _check(lib().tt_encode(self._h, text.data_ptr(), n, _stream_ptr(stream), bufs["ids"].data_ptr(),
                                bufs["ids"].numel(), bufs["count"].data_ptr(), bufs["status"].data_ptr(),
                                ws.data_ptr(), ws.numel()), "tt_encode")
+
+    KERNEL_NAMES = ("pretok", "compact", "bpe_warp", "bpe_long", "count", "scatter")
+
+    def encode_timed(self, text, bufs, stream=None) -> dict:
+        """tt_encode_timed: like encode, synchronises, returns {kernel name: milliseconds}."""
+        ws = bufs["workspace"]
+        ms = (ctypes.c_float * 6)()
+        _check(lib().tt_encode_timed(self._h, text.data_ptr(), int(text.numel()), _stream_ptr(stream),
+                                     bufs["ids"].data_ptr(), bufs["ids"].numel(), bufs["count"].data_ptr(),
+                                     bufs["status"].data_ptr(), ws.data_ptr(), ws.numel(), ms), "tt_encode_timed")
+        return dict(zip(self.KERNEL_NAMES, [float(x) for x in ms]))
 
     def encode_batch(self, text, doc_off, bufs, stream=None):
         """tt_encode_batch: doc_off = int64 CUDA tensor [n_docs+1].  Results in bufs['ids'], bufs['ids_off'], bufs['status']."""

@@ -160,7 +160,7 @@ extern "C" size_t tt_workspace_bytes(const tt_vocab* v, size_t max_len, size_t m
 
 // Enqueues K1+K2 and K3.  piece_off_dst receives the offsets (workspace array or the caller's).
 static int run_pretok(const tt_vocab* v, const uint8_t* text, size_t len, const int64_t* doc_off, size_t n_docs,
-                      cudaStream_t st, TTWorkspace& w, u32* piece_off_dst) {
+                      cudaStream_t st, TTWorkspace& w, u32* piece_off_dst, cudaEvent_t ev_mid = nullptr) {
     const uintptr_t addr = (uintptr_t)text;
     const long long shift = (long long)(addr & 15);
     PretokParams P;
@@ -181,6 +181,7 @@ static int run_pretok(const tt_vocab* v, const uint8_t* text, size_t len, const 
     const size_t smem = align_up(v->cls_bytes, 16) + sizeof(u16) * F_COUNT * TT_SLOTS;
     const int grid = P.ntiles < v->sm_count * 4 ? P.ntiles : v->sm_count * 4;
     k_pretok<<<grid, TT_TILE_CHUNKS, smem, st>>>(P);
+    if (ev_mid) cudaEventRecord(ev_mid, st);
     k_compact<<<grid, TT_TILE_CHUNKS, 0, st>>>(w.startmask, w.tile_cnt, P.nchunks, P.ntiles, shift, (long long)len,
                                                piece_off_dst, w.hdr);
     CK(cudaGetLastError());
@@ -198,7 +199,8 @@ static int check_common(const tt_vocab* v, const void* text, size_t len, void* w
 
 static int encode_impl(const tt_vocab* v, const uint8_t* text, size_t len, const int64_t* doc_off, size_t n_docs,
                        cudaStream_t st, int32_t* ids_out, size_t ids_cap, int64_t* count_out, int64_t* ids_off_out,
-                       int32_t* status_out, void* workspace) {
+                       int32_t* status_out, void* workspace, cudaEvent_t* ev = nullptr) {
+#define MARK(i) do { if (ev) cudaEventRecord(ev[i], st); } while (0)
     TTWorkspace w;
     carve(&w, workspace, len, n_docs);
     CK(cudaMemsetAsync(w.hdr, 0, sizeof(TTHeader), st));
@@ -208,15 +210,20 @@ static int encode_impl(const tt_vocab* v, const uint8_t* text, size_t len, const
         CK(cudaMemsetAsync(status_out, 0, sizeof(int32_t), st));
         return TT_OK;
     }
-    int rc = run_pretok(v, text, len, doc_off, n_docs, st, w, w.piece_off);
+    MARK(0);
+    int rc = run_pretok(v, text, len, doc_off, n_docs, st, w, w.piece_off, ev ? ev[1] : nullptr);
     if (rc != TT_OK) return rc;
+    MARK(2);
     const int bpe_grid = v->sm_count * 8;
     k_bpe_warp<<<bpe_grid, BPE_WARPS * 32, 0, st>>>(text, w.piece_off, w.hdr, v->tab, v->d_ext_id, w.piece_cnt, w.stage,
                                                     w.long_list);
+    MARK(3);
     k_bpe_long<<<v->sm_count, LONG_THREADS, 0, st>>>(text, w.piece_off, w.hdr, v->tab, v->d_ext_id, w.piece_cnt, w.stage,
                                                      w.rank_buf, w.long_list);
+    MARK(4);
     const int nblk = (int)((len + CNT_THREADS - 1) / CNT_THREADS);
     k_count<<<nblk, CNT_THREADS, 0, st>>>(w.piece_cnt, w.hdr, w.blk_cnt, (unsigned long long)ids_cap);
+    MARK(5);
     k_scatter<<<nblk, CNT_THREADS, 0, st>>>(w.piece_off, w.piece_cnt, w.blk_cnt, w.stage, w.hdr, w.tok_off, ids_out,
                                             (long long*)count_out, status_out);
     if (doc_off) {
@@ -224,6 +231,8 @@ static int encode_impl(const tt_vocab* v, const uint8_t* text, size_t len, const
         k_doc_offsets<<<blocks, threads, 0, st>>>((const long long*)doc_off, (int)n_docs, w.piece_off, w.tok_off, w.hdr,
                                                   (long long*)ids_off_out);
     }
+    MARK(6);
+#undef MARK
     CK(cudaGetLastError());
     return TT_OK;
 }
@@ -246,6 +255,23 @@ extern "C" int tt_encode_batch(const tt_vocab* v, const uint8_t* text, size_t to
     if (!doc_off || !ids_off_out || !status_out || (total_len && !ids_out) || n_docs >= (size_t)INT32_MAX) return TT_ERR_ARG;
     return encode_impl(v, text, total_len, doc_off, n_docs, (cudaStream_t)stream, ids_out, ids_cap, nullptr, ids_off_out,
                        status_out, workspace);
+}
+
+extern "C" int tt_encode_timed(const tt_vocab* v, const uint8_t* text, size_t len, void* stream, int32_t* ids_out,
+                               size_t ids_cap, int64_t* count_out, int32_t* status_out, void* workspace,
+                               size_t workspace_bytes, float ms_out[6]) {
+    int rc = check_common(v, text, len, workspace, workspace_bytes, 1);
+    if (rc != TT_OK) return rc;
+    if (!count_out || !status_out || !ms_out || !len || !ids_out) return TT_ERR_ARG;
+    cudaEvent_t ev[7];
+    for (int i = 0; i < 7; i++) CK(cudaEventCreate(&ev[i]));
+    rc = encode_impl(v, text, len, nullptr, 1, (cudaStream_t)stream, ids_out, ids_cap, count_out, nullptr, status_out,
+                     workspace, ev);
+    if (rc == TT_OK && cudaEventSynchronize(ev[6]) != cudaSuccess) rc = TT_ERR_CUDA;
+    for (int i = 0; i < 6 && rc == TT_OK; i++)
+        if (cudaEventElapsedTime(&ms_out[i], ev[i], ev[i + 1]) != cudaSuccess) rc = TT_ERR_CUDA;
+    for (int i = 0; i < 7; i++) cudaEventDestroy(ev[i]);
+    return rc;
 }
 
 __global__ void k_finish_pretok(const TTHeader* hdr, long long* n_pieces_out, int32_t* status_out) {

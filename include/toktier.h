@@ -36,7 +36,8 @@ enum {
     TT_ERR_CUDA = 3,             /* a CUDA runtime call failed (no device, out of memory, launch)      */
     TT_ERR_INVALID_UTF8 = 4,     /* device status: input is not strict UTF-8; zero tokens are returned */
     TT_ERR_CAPACITY = 5,         /* device status: ids_cap too small for the result; zero tokens       */
-    TT_ERR_INTERNAL_TIMEOUT = 6  /* device status: a bounded device-side loop gave up                  */
+    TT_ERR_INTERNAL_TIMEOUT = 6, /* device status: a bounded device-side loop gave up                  */
+    TT_ERR_TOO_LARGE = 7         /* tt_encode_static only: len is above TT_STATIC_MAX_LEN              */
 };
 
 /* Patterns (benchmark configs; the paper names the two lineages in Sec. 4.1):
@@ -138,6 +139,31 @@ int tt_encode_timed(const tt_vocab* v, const uint8_t* text, size_t len, void* st
  */
 int tt_encode_host(tt_vocab* v, const uint8_t* text, size_t len, int32_t* ids_out, size_t ids_cap,
                    int64_t* count_out);
+
+/*
+ * tt_encode_static -- tt_encode for callers that cannot provide scratch memory and must not allocate.
+ * (The paper has no counterpart; this is a convenience of this library.)
+ *
+ * Some callers are not in a position to call cudaMalloc or to carve a workspace out of an allocator:
+ * a plug-in running inside a serving process whose device memory is owned and budgeted by the host
+ * framework, code on a latency-critical thread where an allocation could block behind the device's
+ * other work, or a component that is handed only input and output buffers.  For them the scratch of
+ * the kernel chain is a fixed array inside the library image: loading the library reserves
+ * TT_STATIC_MAX_LEN * 28 + 65,536 bytes (about 7.1 MiB) on every GPU the process uses, until exit.
+ *
+ * Arguments and results are those of tt_encode without `workspace`; inputs and outputs are still
+ * the caller's DEVICE buffers.  The call itself performs no cudaMalloc, cudaFree or other allocating
+ * call.  Differences from tt_encode:
+ *   - len above TT_STATIC_MAX_LEN (262,144 bytes) is refused with TT_ERR_TOO_LARGE; nothing is enqueued.
+ *   - The first call on each device looks up the device address of the array (once per device, with
+ *     that device current).  Make that first call outside any stream capture.
+ *   - All calls on a device share the one array, which still holds the previous call's data; the call
+ *     clears the words that must start at zero.  Two calls whose kernels can overlap on the GPU
+ *     (different streams, no ordering between them) race on it: order them on one stream or with events.
+ */
+#define TT_STATIC_MAX_LEN 262144u
+int tt_encode_static(const tt_vocab* v, const uint8_t* text, size_t len, void* stream,
+                     int32_t* ids_out, size_t ids_cap, int64_t* count_out, int32_t* status_out);
 
 /* Number of class-table entries (0x110000) copied to out (HOST uint8, one class code per code
  * point as the kernels see it): 0 other, 1 mark, 2 whitespace, 3 number, 4 lowercase letter,

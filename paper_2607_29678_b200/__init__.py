@@ -14,11 +14,12 @@ import numpy as np
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libtoktier.so")
 
-TT_OK, TT_ERR_ARG, TT_ERR_BAD_VOCAB, TT_ERR_CUDA, TT_ERR_INVALID_UTF8, TT_ERR_CAPACITY, TT_ERR_INTERNAL_TIMEOUT = range(7)
+TT_OK, TT_ERR_ARG, TT_ERR_BAD_VOCAB, TT_ERR_CUDA, TT_ERR_INVALID_UTF8, TT_ERR_CAPACITY, TT_ERR_INTERNAL_TIMEOUT, TT_ERR_TOO_LARGE = range(8)
+TT_STATIC_MAX_LEN = 262144
 TT_PATTERN_CL100K, TT_PATTERN_O200K = 0, 1
 
 EXPORTS = ["tt_vocab_load", "tt_vocab_free", "tt_workspace_bytes", "tt_encode", "tt_encode_batch",
-           "tt_pretokenize", "tt_encode_timed", "tt_encode_host", "tt_class_table", "tt_strerror"]
+           "tt_pretokenize", "tt_encode_timed", "tt_encode_host", "tt_encode_static", "tt_class_table", "tt_strerror"]
 
 _lib = None
 
@@ -55,6 +56,9 @@ def lib() -> ctypes.CDLL:
         L.tt_encode_timed.restype = c.c_int
         L.tt_encode_timed.argtypes = [c.c_void_p, c.c_void_p, c.c_size_t, c.c_void_p, c.c_void_p, c.c_size_t, c.c_void_p,
                                       c.c_void_p, c.c_void_p, c.c_size_t, c.POINTER(c.c_float)]
+        L.tt_encode_static.restype = c.c_int
+        L.tt_encode_static.argtypes = [c.c_void_p, c.c_void_p, c.c_size_t, c.c_void_p, c.c_void_p, c.c_size_t, c.c_void_p,
+                                       c.c_void_p]
         L.tt_encode_host.restype = c.c_int
         L.tt_encode_host.argtypes = [c.c_void_p, c.c_void_p, c.c_size_t, c.c_void_p, c.c_size_t, c.POINTER(c.c_int64)]
         L.tt_class_table.restype = c.c_size_t
@@ -164,6 +168,15 @@ class Vocab:
                                     n_docs, _stream_ptr(stream), piece_off.data_ptr(), piece_off.numel(),
                                     n_pieces.data_ptr(), bufs["status"].data_ptr(), ws.data_ptr(), ws.numel()),
                "tt_pretokenize")
+
+    def encode_static(self, text, ids, count, status, stream=None, length: int | None = None):
+        """tt_encode_static: encode without a workspace, for callers that may not allocate device memory
+        (the library's own fixed scratch array is used; at most TT_STATIC_MAX_LEN bytes of text).
+        text / ids / count / status are the caller's CUDA tensors (uint8, int32, int64[1], int32[1]).
+        Calls on one device share the scratch, so do not let two of them overlap on the GPU."""
+        n = int(text.numel() if length is None else length)
+        _check(lib().tt_encode_static(self._h, text.data_ptr(), n, _stream_ptr(stream), ids.data_ptr(), ids.numel(),
+                                      count.data_ptr(), status.data_ptr()), "tt_encode_static")
 
     # -- host convenience --------------------------------------------------------------------------
     def encode_host(self, data) -> np.ndarray:

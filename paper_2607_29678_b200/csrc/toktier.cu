@@ -8,6 +8,7 @@
 #include "unicode_table.inc"
 
 #include <climits>
+#include <mutex>
 #include <cstdio>
 #include <cstring>
 #include <new>
@@ -44,6 +45,7 @@ extern "C" const char* tt_strerror(int code) {
         case TT_ERR_INVALID_UTF8: return "input is not valid UTF-8";
         case TT_ERR_CAPACITY: return "output buffer too small";
         case TT_ERR_INTERNAL_TIMEOUT: return "bounded device loop gave up";
+        case TT_ERR_TOO_LARGE: return "input exceeds the fixed limit of the no-allocation entry point";
         default: return "unknown code";
     }
 }
@@ -341,4 +343,39 @@ extern "C" int tt_encode_host(tt_vocab* v, const uint8_t* text, size_t len, int3
     memcpy(ids_out, v->h_ids, (size_t)n * sizeof(int32_t));
     *count_out = n;
     return TT_OK;
+}
+
+// ---- entry point that needs no caller scratch and allocates nothing ---------------------------------
+// The scratch of the kernel chain lives in a fixed device array that is part of the library image, so
+// every GPU that loads the library carries it until the process exits.
+#define TT_STATIC_SCRATCH_BYTES ((size_t)TT_STATIC_MAX_LEN * 28u + 65536u)
+static __device__ __align__(256) unsigned char tt_static_scratch[TT_STATIC_SCRATCH_BYTES];
+
+// Host code may not use the array's name as an address (it names a host-side shadow); the device
+// address is looked up once per device and remembered.
+static void* g_static_scratch_ptr[64];
+static std::mutex g_static_scratch_mutex;
+
+extern "C" int tt_encode_static(const tt_vocab* v, const uint8_t* text, size_t len, void* stream, int32_t* ids_out,
+                                size_t ids_cap, int64_t* count_out, int32_t* status_out) {
+    if (!v || !count_out || !status_out || (len && (!text || !ids_out))) return TT_ERR_ARG;
+    if (len > TT_STATIC_MAX_LEN) return TT_ERR_TOO_LARGE;
+    if (carve(nullptr, nullptr, len, 1) > TT_STATIC_SCRATCH_BYTES) return TT_ERR_TOO_LARGE;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return TT_ERR_CUDA; }
+    if (dev < 0 || dev >= 64) return TT_ERR_ARG;
+    void* scratch = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(g_static_scratch_mutex);
+        if (!g_static_scratch_ptr[dev]) {                        // first call on this device: set-up
+            void* p = nullptr;
+            if (cudaGetSymbolAddress(&p, tt_static_scratch) != cudaSuccess || !p) { cudaGetLastError(); return TT_ERR_CUDA; }
+            g_static_scratch_ptr[dev] = p;
+        }
+        scratch = g_static_scratch_ptr[dev];
+    }
+    // encode_impl clears the header (status word and work counters) first; every other scratch array
+    // is written before it is read, so the previous call's contents do not matter.
+    return encode_impl(v, text, len, nullptr, 1, (cudaStream_t)stream, ids_out, ids_cap, count_out, nullptr, status_out,
+                       scratch);
 }

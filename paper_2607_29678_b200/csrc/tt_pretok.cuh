@@ -13,9 +13,10 @@
 #include "tt_classify.cuh"
 
 enum { F_LEAD = 0, F_OTH, F_MARK, F_SPC, F_NUM, F_LOW, F_UPP, F_CLESS, F_NL, F_SP, F_AP, F_SL, F_DOC, F_COUNT };
-constexpr int TT_SLOTS = TT_TILE_CHUNKS + 2;          // tile plus one halo chunk on each side
+constexpr int TT_LOW_HALO = 2;                          // chunks kept below the tile (look-back context)
+constexpr int TT_SLOTS = TT_TILE_CHUNKS + TT_LOW_HALO + 1;   // low halo, tile, one high halo chunk
 
-enum { NEED_N = 1, NEED_A = 2, NEED_F = 4 };
+enum { NEED_N = 1, NEED_A = 2, NEED_F = 4, NEED_S = 8, NEED_H = 16, NEED_C = 32 };
 
 struct PretokParams {
     const u8* base;          // 16-byte aligned address at or below the text
@@ -35,6 +36,9 @@ struct TileCarry {           // aggregates of runs that enter or leave the share
     u32 n_before;            // number leads (mod 3) of the number run ending right before the low halo chunk
     u32 nl_absorbed_before;  // the CR/LF run ending right before the low halo chunk is glued to punctuation
     u32 nl_later_after;      // the whitespace run leaving the high halo chunk still contains a CR/LF
+    u32 slash_absorbed_before;   // pattern 1: the '/' run ending right before the low halo is part of a punctuation tail
+    u32 dirty_before;        // pattern 1: an unresolved construct lies between the last sure piece start and the low halo
+    long long sure_before;   // pattern 1: position (aligned frame) of the last sure piece start before the low halo
 };
 
 TT_HD u64 tt_win(const u16 (*sm)[TT_SLOTS], int f, int slot) {
@@ -81,11 +85,12 @@ TT_HD u32 tt_walk_back_num(const u16 (*sm)[TT_SLOTS], int s, bool& open) {
 
 // Is the CR/LF run that ends at the last byte of slot `s` glued to a preceding punctuation char?
 // (0 / 1; `open` when the run continues below slot 0.)
-TT_HD u32 tt_walk_back_nl(const u16 (*sm)[TT_SLOTS], int s, u32 othmask_fields, bool& open) {
+TT_HD u32 tt_walk_back_nl(const u16 (*sm)[TT_SLOTS], int s, u32 othmask_fields, bool& open, int top = 15) {
     open = false;
-    for (; s >= 0; s--) {
+    u32 keep = 0xFFFFu >> (15 - top);               // the walk starts at bit `top` of slot s
+    for (; s >= 0; s--, keep = 0xFFFFu) {
         u32 nl = sm[F_NL][s], d = sm[F_DOC][s];
-        u32 cut = (~nl & 0xFFFFu) | (d >> 1);
+        u32 cut = ((~nl & 0xFFFFu) | (d >> 1)) & keep;
         if (cut) {
             int b = tt_hibit(cut);
             if ((d >> 1) >> b & 1) return 0;        // the run starts at a document start

@@ -65,51 +65,80 @@ __device__ __forceinline__ u32 doc_bits(const PretokParams& P, long long chunk) 
 }
 
 // ---- bounded CTA-cooperative walks over the text (runs that leave the shared-memory window) ----
-// Every loop below advances by one tile per iteration and stops at the ends of the text.
+// Every loop below advances by one tile per iteration and stops at the ends of the text.  All
+// positions are in the aligned frame; `gend` is exclusive.
 
-// Number leads (mod 3) of the number run that ends right before chunk c0.
-__device__ u32 coop_back_num(const PretokParams& P, const ClassTables& T, long long c0, long long* scratch) {
-    u32 total = 0;
-    for (long long cb = c0 - TT_TILE_CHUNKS;; cb -= TT_TILE_CHUNKS) {
-        long long chunk = cb + threadIdx.x;
-        ChunkMasks m = tt_classify_chunk(P.base, chunk, P.nchunks, P.lo, P.hi, T);
-        u32 d = doc_bits(P, chunk), dn = doc_bits(P, chunk + 1);
-        u32 cut = (~(u32)m.num & 0xFFFFu) | (d >> 1) | ((dn & 1) << 15);
-        if (chunk < 0) cut = 0xFFFFu;
-        long long pos = cut ? chunk * 16 + tt_hibit(cut) : -(1ll << 60);
-        long long top = cta_max_ll(pos, scratch);
-        u32 mine = 0;
-        if (chunk * 16 + 15 > top) {
-            u32 keep = 0xFFFFu;
-            if (top >= chunk * 16) keep = (0xFFFFu << (int)(top - chunk * 16 + 1)) & 0xFFFFu;
-            mine = tt_popc(m.lead & m.num & keep);
-        }
-        total += cta_sum_u32(mine, scratch);
-        if (top > -(1ll << 59) || cb <= 0) break;
-    }
-    return total % 3;
+enum { RUN_NUM = 0, RUN_NL = 1, RUN_SL = 2 };
+constexpr long long COOP_NONE = -(1ll << 60);
+
+__device__ __forceinline__ u32 run_mask(const ChunkMasks& m, int kind) {
+    return kind == RUN_NUM ? m.num : kind == RUN_NL ? m.nl : m.sl;
 }
 
-// Is the CR/LF run that ends right before chunk c0 glued to a preceding punctuation character?
-__device__ u32 coop_back_nl(const PretokParams& P, const ClassTables& T, long long c0, long long* scratch) {
-    for (long long cb = c0 - TT_TILE_CHUNKS;; cb -= TT_TILE_CHUNKS) {
-        long long chunk = cb + threadIdx.x;
-        ChunkMasks m = tt_classify_chunk(P.base, chunk, P.nchunks, P.lo, P.hi, T);
-        u32 d = doc_bits(P, chunk), dn = doc_bits(P, chunk + 1);
-        u32 dcut = (d >> 1) | ((dn & 1) << 15);
-        u32 cut = (~(u32)m.nl & 0xFFFFu) | dcut;
-        if (chunk < 0) cut = 0xFFFFu;
-        long long pos = -(1ll << 60);
+// Walks down from gend-1 through bytes of the run class `kind` (cut at document starts).  Returns the
+// position of the first byte that is not part of the run, with flags in the low three bits:
+// 1 = the run was cut by a document start, 2 = that byte is "other" (4 = a mark), 8 = it is CR/LF.
+// *leads receives the number of code-point leads inside the run (RUN_NUM only).
+__device__ long long coop_back_run(const PretokParams& P, const ClassTables& T, long long gend, int kind,
+                                   long long* scratch, u32* leads) {
+    u32 total = 0;
+    long long found = COOP_NONE;
+    const long long ctop = (gend + TT_CHUNK - 1) / TT_CHUNK;          // chunks below ctop are examined
+    for (long long cb = ctop - TT_TILE_CHUNKS;; cb -= TT_TILE_CHUNKS) {
+        const long long chunk = cb + threadIdx.x;
+        const ChunkMasks m = tt_classify_chunk(P.base, chunk, P.nchunks, P.lo, P.hi, T);
+        const u32 d = doc_bits(P, chunk), dn = doc_bits(P, chunk + 1);
+        u32 live = 0xFFFFu;                                          // bytes of this chunk below gend
+        if (chunk * 16 + 16 > gend) live = gend > chunk * 16 ? (0xFFFFu >> (int)(chunk * 16 + 16 - gend)) : 0u;
+        const u32 dcut = ((d >> 1) | ((dn & 1) << 15));
+        // a document start at gend itself does not cut the run (the caller has checked that byte)
+        u32 dc = dcut;
+        if (gend - 1 >= chunk * 16 && gend - 1 < chunk * 16 + 16) dc &= ~(1u << (int)(gend - 1 - chunk * 16));
+        u32 cut = ((~run_mask(m, kind) & 0xFFFFu) | dc) & live;
+        if (chunk < 0) cut = live;
+        long long pos = COOP_NONE;
         if (cut) {
-            int b = tt_hibit(cut);
-            // encode the answer in the low bit: (position << 1) | glued
-            u32 glued = (chunk >= 0) && !((dcut >> b) & 1) && (((u32)(m.oth | m.mark) >> b) & 1);
-            pos = ((chunk * 16 + b) << 1) | glued;
+            const int b = tt_hibit(cut);
+            const u32 flags = ((dc >> b) & 1) | ((((u32)m.oth >> b) & 1) << 1) | ((((u32)m.mark >> b) & 1) << 2) |
+                              ((((u32)m.nl >> b) & 1) << 3);
+            pos = ((chunk * 16 + b) << 4) | flags;
         }
-        long long top = cta_max_ll(pos, scratch);
-        if (top > -(1ll << 59)) return (u32)(top & 1);
-        if (cb <= 0) return 0;
+        const long long top = cta_max_ll(pos, scratch);
+        const long long top_pos = top == COOP_NONE ? COOP_NONE : (top >> 4);
+        if (leads) {
+            u32 mine = 0;
+            if (chunk >= 0 && chunk * 16 + 15 > top_pos) {
+                u32 keep = live;
+                if (top_pos >= chunk * 16) keep &= (0xFFFFu << (int)(top_pos - chunk * 16 + 1));
+                mine = tt_popc(m.lead & run_mask(m, kind) & keep);
+            }
+            total += cta_sum_u32(mine, scratch);
+        }
+        if (top != COOP_NONE) { found = top; break; }
+        if (cb <= 0) { found = ((long long)-1 << 4) | 1; break; }
     }
+    if (leads) *leads = total;
+    return found;
+}
+
+// Number leads (mod 3) of the number run that ends right before gend.
+__device__ u32 coop_back_num(const PretokParams& P, const ClassTables& T, long long gend, long long* scratch) {
+    u32 leads = 0;
+    coop_back_run(P, T, gend, RUN_NUM, scratch, &leads);
+    return leads % 3;
+}
+// Is the byte before gend an "other" character, or a CR/LF run glued to one?  (marks count as
+// "other" only for pattern 0)
+__device__ u32 coop_back_nl(const PretokParams& P, const ClassTables& T, long long gend, long long* scratch) {
+    const long long r = coop_back_run(P, T, gend, RUN_NL, scratch, nullptr);
+    if (r & 1) return 0;
+    return ((r >> 1) & 1) | (P.pattern == 0 ? ((r >> 2) & 1) : 0);
+}
+// Pattern 1: is the byte before gend a '/' run (or CR/LF run) that belongs to a punctuation tail?
+__device__ u32 coop_back_slash(const PretokParams& P, const ClassTables& T, long long gend, long long* scratch) {
+    const long long r = coop_back_run(P, T, gend, RUN_SL, scratch, nullptr);
+    if ((r & 1) || !((r >> 3) & 1)) return 0;                 // cut by a document, or not preceded by CR/LF
+    return coop_back_nl(P, T, (r >> 4) + 1, scratch);
 }
 
 // Does the whitespace run that continues at chunk c0 (its first byte) still contain a CR/LF?
@@ -119,7 +148,7 @@ __device__ u32 coop_fwd_nl(const PretokParams& P, const ClassTables& T, long lon
         ChunkMasks m = tt_classify_chunk(P.base, chunk, P.nchunks, P.lo, P.hi, T);
         u32 d = doc_bits(P, chunk);
         u32 ev = ((~(u32)m.spc) | d | m.nl) & 0xFFFFu;       // bytes past the end are not whitespace
-        long long neg = -(1ll << 60);
+        long long neg = COOP_NONE;
         if (ev) {
             int j = tt_lobit(ev);
             u32 is_nl = ((u32)(m.nl & m.spc & ~d) >> j) & 1;
@@ -127,12 +156,44 @@ __device__ u32 coop_fwd_nl(const PretokParams& P, const ClassTables& T, long lon
             neg = -(((chunk * 16 + j) << 1) | (is_nl ^ 1));
         }
         long long best = cta_max_ll(neg, scratch);
-        if (best > -(1ll << 59)) return (u32)(((-best) & 1) ^ 1);
+        if (best != COOP_NONE) return (u32)(((-best) & 1) ^ 1);
         if (cb + TT_TILE_CHUNKS >= P.nchunks) return 0;
     }
 }
 
+// Pattern 1: nearest sure piece start (sure_only) or nearest sure-start / unresolved-construct event
+// below gend.  Returns (position << 1) | is_unresolved; the text start is always a sure start.
+__device__ long long coop_back_event(const PretokParams& P, const ClassTables& T, long long gend, bool sure_only,
+                                     long long* scratch) {
+    const long long ctop = (gend + TT_CHUNK - 1) / TT_CHUNK;
+    for (long long cb = ctop - TT_TILE_CHUNKS;; cb -= TT_TILE_CHUNKS) {
+        const long long chunk = cb + threadIdx.x;
+        long long pos = COOP_NONE;
+        if (chunk >= 0) {
+            ChunkDoc p, c, n;
+            p.m = tt_classify_chunk(P.base, chunk - 1, P.nchunks, P.lo, P.hi, T); p.doc = doc_bits(P, chunk - 1);
+            c.m = tt_classify_chunk(P.base, chunk, P.nchunks, P.lo, P.hi, T);     c.doc = doc_bits(P, chunk);
+            n.m = tt_classify_chunk(P.base, chunk + 1, P.nchunks, P.lo, P.hi, T); n.doc = doc_bits(P, chunk + 1);
+            u32 sure, hard;
+            tt_sure_hard_cm(p, c, n, sure, hard);
+            u32 live = 0xFFFFu;
+            if (chunk * 16 + 16 > gend) live = gend > chunk * 16 ? (0xFFFFu >> (int)(chunk * 16 + 16 - gend)) : 0u;
+            const u32 ev = (sure | (sure_only ? 0u : hard)) & live;
+            if (ev) { const int b = tt_hibit(ev); pos = ((chunk * 16 + b) << 1) | (sure_only ? 0u : ((hard >> b) & 1)); }
+        }
+        const long long top = cta_max_ll(pos, scratch);
+        if (top != COOP_NONE) return top;
+        if (cb <= 0) return (P.lo << 1);
+    }
+}
+
 // ---- K1 + K2 -----------------------------------------------------------------------------------
+__device__ __forceinline__ void store_slot(u16 (*sm)[TT_SLOTS], int s, const ChunkMasks& m, u32 d) {
+    sm[F_LEAD][s] = m.lead; sm[F_OTH][s] = m.oth; sm[F_MARK][s] = m.mark; sm[F_SPC][s] = m.spc;
+    sm[F_NUM][s] = m.num; sm[F_LOW][s] = m.low; sm[F_UPP][s] = m.upp; sm[F_CLESS][s] = m.cless;
+    sm[F_NL][s] = m.nl; sm[F_SP][s] = m.sp; sm[F_AP][s] = m.ap; sm[F_SL][s] = m.sl; sm[F_DOC][s] = (u16)d;
+}
+
 __global__ void __launch_bounds__(TT_TILE_CHUNKS)
 k_pretok(const PretokParams P) {
     extern __shared__ __align__(16) u8 smem_raw[];
@@ -140,7 +201,6 @@ k_pretok(const PretokParams P) {
     u16 (*sm)[TT_SLOTS] = reinterpret_cast<u16 (*)[TT_SLOTS]>(smem_raw + ((P.cls_bytes + 15) & ~15));
     __shared__ long long scratch[40];
     __shared__ u32 s_need;
-    __shared__ TileCarry s_tc;
     __shared__ u32 s_islast;
 
     const int tid = threadIdx.x;
@@ -148,50 +208,56 @@ k_pretok(const PretokParams P) {
         *reinterpret_cast<uint4*>(tables + i) = *reinterpret_cast<const uint4*>(P.cls_tables + i);
     ClassTables T;
     T.stage1 = tables; T.stage2 = tables + 0x1100; T.ascii = tables + P.cls_bytes - 128;
+    SeqCtx SC;
+    SC.base = P.base; SC.lo = P.lo; SC.hi = P.hi; SC.docmask = P.docmask; SC.T = T;
     u32 any_bad = 0;
 
     for (int tile = blockIdx.x; tile < P.ntiles; tile += gridDim.x) {
         __syncthreads();
         if (tid == 0) s_need = 0;
         const long long c_first = (long long)tile * TT_TILE_CHUNKS;
-        // phase A: classify own chunk (+ the two halo chunks)
+        // phase A: classify own chunk (+ the halo chunks)
         {
             const long long chunk = c_first + tid;
-            ChunkMasks m = tt_classify_chunk(P.base, chunk, P.nchunks, P.lo, P.hi, T);
-            const int s = tid + 1;
-            u32 d = doc_bits(P, chunk);
-            sm[F_LEAD][s] = m.lead; sm[F_OTH][s] = m.oth; sm[F_MARK][s] = m.mark; sm[F_SPC][s] = m.spc;
-            sm[F_NUM][s] = m.num; sm[F_LOW][s] = m.low; sm[F_UPP][s] = m.upp; sm[F_CLESS][s] = m.cless;
-            sm[F_NL][s] = m.nl; sm[F_SP][s] = m.sp; sm[F_AP][s] = m.ap; sm[F_SL][s] = m.sl; sm[F_DOC][s] = (u16)d;
+            const ChunkMasks m = tt_classify_chunk(P.base, chunk, P.nchunks, P.lo, P.hi, T);
+            const u32 d = doc_bits(P, chunk);
+            store_slot(sm, tid + TT_LOW_HALO, m, d);
             any_bad |= m.bad | (d & ~(u32)m.lead & 0xFFFFu & (m.oth | m.mark | m.spc | m.num | m.low | m.upp | m.cless));
         }
-        if (tid < 2) {
-            const long long chunk = tid == 0 ? c_first - 1 : c_first + TT_TILE_CHUNKS;
-            ChunkMasks m = tt_classify_chunk(P.base, chunk, P.nchunks, P.lo, P.hi, T);
-            const int s = tid == 0 ? 0 : TT_SLOTS - 1;
-            sm[F_LEAD][s] = m.lead; sm[F_OTH][s] = m.oth; sm[F_MARK][s] = m.mark; sm[F_SPC][s] = m.spc;
-            sm[F_NUM][s] = m.num; sm[F_LOW][s] = m.low; sm[F_UPP][s] = m.upp; sm[F_CLESS][s] = m.cless;
-            sm[F_NL][s] = m.nl; sm[F_SP][s] = m.sp; sm[F_AP][s] = m.ap; sm[F_SL][s] = m.sl; sm[F_DOC][s] = (u16)doc_bits(P, chunk);
+        if (tid < TT_LOW_HALO + 1) {
+            const long long chunk = tid < TT_LOW_HALO ? c_first - TT_LOW_HALO + tid : c_first + TT_TILE_CHUNKS;
+            const int s = tid < TT_LOW_HALO ? tid : TT_SLOTS - 1;
+            store_slot(sm, s, tt_classify_chunk(P.base, chunk, P.nchunks, P.lo, P.hi, T), doc_bits(P, chunk));
         }
         __syncthreads();
         // phase B: evaluate the piece-start predicate
-        TileCarry tc; tc.n_before = 0; tc.nl_absorbed_before = 0; tc.nl_later_after = 0;
+        TileCarry tc;
+        tc.n_before = 0; tc.nl_absorbed_before = 0; tc.nl_later_after = 0; tc.slash_absorbed_before = 0;
+        tc.dirty_before = 0; tc.sure_before = P.lo;
         u32 need = 0;
+        const int slot = tid + TT_LOW_HALO;
         const long long g0 = (c_first + tid) * TT_CHUNK;
-        u32 S = P.pattern == 0 ? tt_eval_chunk_p0(sm, tid + 1, P.base, g0, P.hi, tc, false, need)
-                               : tt_eval_chunk_p1(sm, tid + 1, P.base, g0, P.hi, tc, false, need);
+        u32 S = P.pattern == 0 ? tt_eval_chunk_p0(sm, slot, P.base, g0, P.hi, tc, false, need)
+                               : tt_eval_chunk_p1(sm, slot, SC, g0, tc, false, need);
         if (need) atomicOr(&s_need, need);
         __syncthreads();
         const u32 need_all = s_need;
         if (need_all) {                                               // block-uniform
-            u32 a = 0, b = 0, c = 0;
-            if (need_all & NEED_N) a = coop_back_num(P, T, c_first - 1, scratch);
-            if (need_all & NEED_A) b = coop_back_nl(P, T, c_first - 1, scratch);
-            if (need_all & NEED_F) c = coop_fwd_nl(P, T, c_first + TT_TILE_CHUNKS + 1, scratch);
-            tc.n_before = a; tc.nl_absorbed_before = b; tc.nl_later_after = c;
+            const long long below = (c_first - TT_LOW_HALO) * TT_CHUNK;    // first byte of the low halo
+            if (need_all & NEED_N) tc.n_before = coop_back_num(P, T, below, scratch);
+            if (need_all & NEED_A) tc.nl_absorbed_before = coop_back_nl(P, T, below, scratch);
+            if (need_all & NEED_S) tc.slash_absorbed_before = coop_back_slash(P, T, below, scratch);
+            if (need_all & NEED_F) tc.nl_later_after = coop_fwd_nl(P, T, c_first + TT_TILE_CHUNKS + 1, scratch);
+            if (need_all & (NEED_H | NEED_C)) {
+                // events of slot 0 (first halo chunk) are not examined by the walks in shared memory
+                const long long gend = below + TT_CHUNK;
+                const long long ev = coop_back_event(P, T, gend, false, scratch);
+                tc.dirty_before = (u32)(ev & 1);
+                tc.sure_before = (ev & 1) ? (coop_back_event(P, T, (ev >> 1) + 1, true, scratch) >> 1) : (ev >> 1);
+            }
             need = 0;
-            S = P.pattern == 0 ? tt_eval_chunk_p0(sm, tid + 1, P.base, g0, P.hi, tc, true, need)
-                               : tt_eval_chunk_p1(sm, tid + 1, P.base, g0, P.hi, tc, true, need);
+            S = P.pattern == 0 ? tt_eval_chunk_p0(sm, slot, P.base, g0, P.hi, tc, true, need)
+                               : tt_eval_chunk_p1(sm, slot, SC, g0, tc, true, need);
         }
         if (c_first + tid < P.nchunks) P.startmask[c_first + tid] = (u16)S;
         u32 total = cta_sum_u32(tt_popc(S), scratch);

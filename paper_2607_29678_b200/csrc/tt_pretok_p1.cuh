@@ -1,8 +1,372 @@
-// Pattern 1 (o200k-style) piece-start predicate.  (placeholder until the case-aware rules land)
+// Pattern 1 (o200k-style) piece-start predicate.
+//
+// Paper Sec. 4.1: this lineage adds a case-boundary rule and a sparse contraction path to the
+// run-local rules, and Unicode marks take a narrow sparse fallback while the common path stays
+// vectorised.  Here the vectorised path covers number runs, whitespace runs, punctuation runs with
+// their [\r\n/]* tails, word starts with the one-character prefix and the lower->upper case boundary.
+// Three constructs are not decided by local rules: a mark, an upper-case letter that follows a
+// caseless letter, and an apostrophe between letters (a possible contraction suffix).  Each of them
+// marks the text from the last *sure* piece start before it up to the next sure piece start as
+// unresolved; a thread whose chunk contains unresolved bytes re-derives those bytes by matching
+// sequentially from that sure start (matching from a piece start never looks behind it).  Sure
+// starts are positions that begin a piece whatever surrounds them: a document start, the first
+// digit of a number run, whitespace or non-apostrophe punctuation right after a letter or digit, a
+// letter right after a digit or a CR/LF.
 #pragma once
 #include "tt_pretok.cuh"
 
-TT_HD u32 tt_eval_chunk_p1(const u16 (*sm)[TT_SLOTS], int slot, const u8* base, long long g0, long long hi,
+struct SeqCtx {                 // what the sequential matcher needs to read the text itself
+    const u8* base;
+    long long lo, hi;
+    const u32* docmask;         // or null: one document
+    ClassTables T;
+};
+
+// ---- sequential matcher over the raw text (sparse path) ---------------------------------------------
+struct SeqChar { u32 cls; u32 byte; int len; };   // byte = the ASCII byte, or 0x100 for multi-byte characters
+
+TT_HD SeqChar tt_seq_char(const SeqCtx& C, long long g, long long end) {
+    SeqChar r;
+    u32 b = C.base[g];
+    if (b < 0x80) { r.cls = C.T.ascii[b] & 7; r.byte = b; r.len = 1; return r; }
+    int n = b >= 0xF0 ? 4 : b >= 0xE0 ? 3 : 2;
+    if (g + n > end) n = (int)(end - g);
+    u32 cp = b & (0x7Fu >> (b >= 0xF0 ? 4 : b >= 0xE0 ? 3 : 2));
+    for (int k = 1; k < n; k++) cp = (cp << 6) | (C.base[g + k] & 0x3F);
+    if (cp > 0x10FFFF) cp = 0xFFFD;                  // malformed input: the result is discarded anyway
+    r.cls = tt_class_of(cp, C.T); r.byte = 0x100; r.len = n < 1 ? 1 : n;
+    return r;
+}
+TT_HD bool tt_seq_is_doc_start(const SeqCtx& C, long long g) {
+    if (C.docmask) return (C.docmask[g >> 5] >> (g & 31)) & 1;
+    return g == C.lo;
+}
+TT_HD bool tt_cls_word(u32 c) { return c == CC_LOWER || c == CC_UPPER || c == CC_CASELESS || c == CC_MARK; }
+TT_HD bool tt_cls_up(u32 c) { return c == CC_UPPER || c == CC_CASELESS || c == CC_MARK; }      // U
+TT_HD bool tt_cls_lw(u32 c) { return c == CC_LOWER || c == CC_CASELESS || c == CC_MARK; }      // Lw
+TT_HD bool tt_cls_letter(u32 c) { return c == CC_LOWER || c == CC_UPPER || c == CC_CASELESS; }
+TT_HD bool tt_cls_punct(u32 c) { return c == CC_OTHER || c == CC_MARK; }                        // [^\s\p{L}\p{N}]
+
+// U* Lw+ from q (greedy U*, giving characters back until Lw+ can start); returns the end or q.
+TT_HD long long tt_seq_body_lower(const SeqCtx& C, long long q, long long end) {
+    long long t = q, last_lw_end = -1;
+    while (t < end) {
+        SeqChar ch = tt_seq_char(C, t, end);
+        if (!tt_cls_word(ch.cls) || !tt_cls_up(ch.cls)) break;
+        if (tt_cls_lw(ch.cls)) last_lw_end = t + ch.len;
+        t += ch.len;
+    }
+    if (t < end) {
+        SeqChar ch = tt_seq_char(C, t, end);
+        if (tt_cls_word(ch.cls) && tt_cls_lw(ch.cls)) {
+            long long v = t;
+            while (v < end) { SeqChar c2 = tt_seq_char(C, v, end); if (!tt_cls_word(c2.cls) || !tt_cls_lw(c2.cls)) break; v += c2.len; }
+            return v;
+        }
+    }
+    return last_lw_end >= 0 ? last_lw_end : q;
+}
+// U+ Lw* from q
+TT_HD long long tt_seq_body_upper(const SeqCtx& C, long long q, long long end) {
+    long long t = q;
+    while (t < end) { SeqChar ch = tt_seq_char(C, t, end); if (!tt_cls_word(ch.cls) || !tt_cls_up(ch.cls)) break; t += ch.len; }
+    if (t == q) return q;
+    while (t < end) { SeqChar ch = tt_seq_char(C, t, end); if (!tt_cls_word(ch.cls) || !tt_cls_lw(ch.cls)) break; t += ch.len; }
+    return t;
+}
+// One leftmost-first match of pattern 1 at p (p < end); returns the end of the piece.
+TT_HD long long tt_seq_match_p1(const SeqCtx& C, long long p, long long end) {
+    const SeqChar c0 = tt_seq_char(C, p, end);
+    const bool nl0 = c0.byte == '\n' || c0.byte == '\r';
+    const bool prefix_ok = !nl0 && !tt_cls_letter(c0.cls) && c0.cls != CC_NUMBER;
+    long long e = -1;
+    for (int alt = 0; alt < 2 && e < 0; alt++) {
+        if (prefix_ok && p + c0.len < end) {
+            long long q = p + c0.len, v = alt == 0 ? tt_seq_body_lower(C, q, end) : tt_seq_body_upper(C, q, end);
+            if (v > q) { e = v; break; }
+        }
+        long long v = alt == 0 ? tt_seq_body_lower(C, p, end) : tt_seq_body_upper(C, p, end);
+        if (v > p) e = v;
+    }
+    if (e >= 0) {
+        if (e < end && C.base[e] == '\'') {
+            u32 b1 = e + 1 < end ? C.base[e + 1] : 0, b2 = e + 2 < end ? C.base[e + 2] : 0;
+            e += tt_contraction_len(b1, b2);
+        }
+        return e;
+    }
+    if (c0.cls == CC_NUMBER) {
+        long long t = p; int k = 0;
+        while (t < end && k < 3) { SeqChar ch = tt_seq_char(C, t, end); if (ch.cls != CC_NUMBER) break; t += ch.len; k++; }
+        return t;
+    }
+    long long q = -1;
+    if (c0.byte == ' ' && p + 1 < end && tt_cls_punct(tt_seq_char(C, p + 1, end).cls)) q = p + 1;
+    else if (tt_cls_punct(c0.cls)) q = p;
+    if (q >= 0) {
+        while (q < end) { SeqChar ch = tt_seq_char(C, q, end); if (!tt_cls_punct(ch.cls)) break; q += ch.len; }
+        while (q < end) { u32 b = C.base[q]; if (b != '\n' && b != '\r' && b != '/') break; q++; }
+        return q;
+    }
+    // whitespace: \s*[\r\n]+ | \s+(?!\S) | \s+
+    long long t = p, last_nl_end = -1, last_char = p; int n = 0;
+    while (t < end) {
+        SeqChar ch = tt_seq_char(C, t, end);
+        if (ch.cls != CC_SPACE) break;
+        if (ch.byte == '\n' || ch.byte == '\r') last_nl_end = t + 1;
+        last_char = t; t += ch.len; n++;
+    }
+    if (last_nl_end >= 0) return last_nl_end;
+    if (t >= end) return t;
+    if (n >= 2) return last_char;
+    return t > p ? t : p + c0.len;
+}
+
+// Piece starts inside [g0, g0+16) obtained by matching sequentially from the piece start `from`
+// (from <= g0 + 15).  Returns a 16-bit mask; bits below `from` are not produced.
+TT_HD u32 tt_seq_starts_p1(const SeqCtx& C, long long from, long long g0, long long& doc_end) {
+    long long end = C.hi;
+    if (C.docmask) {                                   // end of the document that contains `from`
+        long long g = from + 1;
+        // look for the next document start, one 32-bit word at a time
+        while (g < C.hi) {
+            u32 w = C.docmask[g >> 5] >> (g & 31);
+            if (w) { g += tt_lobit(w); break; }
+            g = ((g >> 5) + 1) << 5;
+        }
+        end = g < C.hi ? g : C.hi;
+    }
+    doc_end = end;
+    u32 bits = 0;
+    long long p = from;
+    const long long stop = g0 + TT_CHUNK < end ? g0 + TT_CHUNK : end;
+    while (p < stop) {
+        if (p >= g0) bits |= 1u << (int)(p - g0);
+        long long e = tt_seq_match_p1(C, p, end);
+        p = e > p ? e : p + 1;
+    }
+    return bits;
+}
+
+// ---- masks of sure piece starts and of unresolved constructs for one chunk ---------------------------
+struct ChunkDoc { ChunkMasks m; u32 doc; };
+
+TT_HD ChunkDoc tt_load_slot(const u16 (*sm)[TT_SLOTS], int s) {
+    ChunkDoc c;
+    c.m.lead = sm[F_LEAD][s]; c.m.oth = sm[F_OTH][s]; c.m.mark = sm[F_MARK][s]; c.m.spc = sm[F_SPC][s]; c.m.num = sm[F_NUM][s];
+    c.m.low = sm[F_LOW][s]; c.m.upp = sm[F_UPP][s]; c.m.cless = sm[F_CLESS][s]; c.m.nl = sm[F_NL][s]; c.m.sp = sm[F_SP][s];
+    c.m.ap = sm[F_AP][s]; c.m.sl = sm[F_SL][s]; c.m.bad = 0; c.doc = sm[F_DOC][s];
+    return c;
+}
+// p = previous chunk, c = the chunk, n = next chunk
+TT_HD void tt_sure_hard_cm(const ChunkDoc& p, const ChunkDoc& c, const ChunkDoc& n, u32& sure, u32& hard) {
+    // 18-bit frame: bit 0 = last byte of the previous chunk, bits 1..16 = the chunk, bit 17 = first byte of the next
+#define FR(x) ((((u32)p.x) >> 15) | (((u32)c.x) << 1) | ((((u32)n.x) & 1u) << 17))
+    const u32 lead = FR(m.lead), D = FR(doc);
+    const u32 Lr = FR(m.low) | FR(m.upp) | FR(m.cless), N = FR(m.num), W = FR(m.spc), O = FR(m.oth), AP = FR(m.ap);
+    const u32 nD = ~D;
+    const u32 pLr = (Lr << 1) & nD, pN = (N << 1) & nD, pNL = (FR(m.nl) << 1) & nD, pCl = (FR(m.cless) << 1) & nD;
+    const u32 nLr = (Lr >> 1) & ~(D >> 1);
+    const u32 cs = D | (N & ~pN) | (W & (pLr | pN)) | (O & ~AP & (pLr | pN)) | (Lr & (pN | pNL));
+    const u32 h = FR(m.mark) | (FR(m.upp) & pCl) | (AP & pLr & nLr);
+#undef FR
+    sure = ((cs & lead) >> 1) & 0xFFFFu;
+    hard = ((h & lead) >> 1) & 0xFFFFu;
+}
+// Valid for 1 <= s <= TT_SLOTS - 2 (needs the neighbouring slots).
+TT_HD void tt_sure_hard(const u16 (*sm)[TT_SLOTS], int s, u32& sure, u32& hard) {
+    tt_sure_hard_cm(tt_load_slot(sm, s - 1), tt_load_slot(sm, s), tt_load_slot(sm, s + 1), sure, hard);
+}
+
+// Walks down from slot s: is the nearest sure-start / unresolved-construct event an unresolved one?
+TT_HD u32 tt_walk_back_dirty(const u16 (*sm)[TT_SLOTS], int s, bool& open) {
+    open = false;
+    for (; s >= 1; s--) {
+        u32 c, h; tt_sure_hard(sm, s, c, h);
+        if (c | h) { int b = tt_hibit(c | h); return (h >> b) & 1; }
+    }
+    open = true;
+    return 0;
+}
+// Walks down from slot s: position (slot * 16 + bit) of the nearest sure start, or -1 when open.
+TT_HD int tt_walk_back_sure(const u16 (*sm)[TT_SLOTS], int s) {
+    for (; s >= 1; s--) {
+        u32 c, h; tt_sure_hard(sm, s, c, h);
+        if (c) return s * 16 + tt_hibit(c);
+    }
+    return -1;
+}
+// Is the '/' run that ends at bit `top` of slot s part of a punctuation tail (absorbed)?
+// need_a: the answer hangs on a CR/LF run that leaves the window (then the tile carry decides).
+TT_HD u32 tt_walk_back_slash(const u16 (*sm)[TT_SLOTS], int s, int top, bool& open_s, bool& open_a) {
+    open_s = open_a = false;
+    u32 keep = 0xFFFFu >> (15 - top);
+    for (; s >= 0; s--, keep = 0xFFFFu) {
+        u32 sl = sm[F_SL][s], d = sm[F_DOC][s];
+        u32 cut = ((~sl & 0xFFFFu) | (d >> 1)) & keep;
+        if (cut) {
+            int b = tt_hibit(cut);
+            if (((d >> 1) >> b) & 1) return 0;                  // the run starts a document
+            if (!((sm[F_NL][s] >> b) & 1)) return 0;            // not preceded by CR/LF
+            return tt_walk_back_nl(sm, s, 0, open_a, b);
+        }
+        if (d & 1) return 0;
+    }
+    open_s = true;
+    return 0;
+}
+
+TT_HD u64 tt_win4(const u16 (*sm)[TT_SLOTS], int f, int slot) {   // slots slot-2 .. slot+1; own chunk at bits 32..47
+    return (u64)sm[f][slot - 2] | ((u64)sm[f][slot - 1] << 16) | ((u64)sm[f][slot] << 32) | ((u64)sm[f][slot + 1] << 48);
+}
+
+// Returns the 16 start bits of the chunk in `slot` (slot >= 2).
+TT_HD u32 tt_eval_chunk_p1(const u16 (*sm)[TT_SLOTS], int slot, const SeqCtx& C, long long g0,
                            const TileCarry& tc, bool have_tc, u32& need) {
-    return tt_eval_chunk_p0(sm, slot, base, g0, hi, tc, have_tc, need);
+    const u64 OWN = 0xFFFFull << 32;
+    const u64 lead = tt_win4(sm, F_LEAD, slot);
+    const u64 low = tt_win4(sm, F_LOW, slot), upp = tt_win4(sm, F_UPP, slot), cless = tt_win4(sm, F_CLESS, slot);
+    const u64 Lr = low | upp | cless, Mk = tt_win4(sm, F_MARK, slot);
+    const u64 N = tt_win4(sm, F_NUM, slot), W = tt_win4(sm, F_SPC, slot), O = tt_win4(sm, F_OTH, slot);
+    const u64 NL = tt_win4(sm, F_NL, slot), SP = tt_win4(sm, F_SP, slot), AP = tt_win4(sm, F_AP, slot), SL = tt_win4(sm, F_SL, slot);
+    const u64 D = tt_win4(sm, F_DOC, slot);
+    const u64 V = Lr | Mk | N | W | O;
+    const u64 cont = V & ~lead;
+    const u64 nD = ~D;
+    u64 S = 0;
+#define PREV(x) (((x) << 1) & nD)
+    // ---- CR/LF absorbed by a preceding punctuation character (any non-mark "other", slashes included)
+    u64 A;
+    {
+        u32 carry = 0;
+        if ((NL & 1) && !(D & 1)) {                      // the run may enter the window from below
+            bool open = slot < 3;
+            if (!open) {
+                u32 prevnl = (sm[F_NL][slot - 3] >> 15) & 1, prevo = (sm[F_OTH][slot - 3] >> 15) & 1;
+                if (prevnl) carry = tt_walk_back_nl(sm, slot - 3, 0, open);
+                else carry = prevo;
+            }
+            if (open) { if (have_tc) carry = tc.nl_absorbed_before; else need |= NEED_A; }
+        }
+        const u64 nlq = NL & nD;
+        const u64 sel = (NL & ~PREV(NL) & PREV(O)) | ((nlq & 1) ? (u64)carry : 0);
+        A = nlq & ~(nlq + sel);
+    }
+    // ---- slashes absorbed by the tail [\r\n/]* : '/' runs that begin right after an absorbed CR/LF
+    u64 AS;
+    {
+        u32 carry = 0;
+        if ((SL & 1) && !(D & 1)) {
+            bool open_s = slot < 3, open_a = false;
+            if (!open_s) {
+                u32 prevsl = (sm[F_SL][slot - 3] >> 15) & 1, prevnl = (sm[F_NL][slot - 3] >> 15) & 1;
+                if (prevsl) carry = tt_walk_back_slash(sm, slot - 3, 15, open_s, open_a);
+                else if (prevnl) carry = tt_walk_back_nl(sm, slot - 3, 0, open_a);
+            }
+            if (open_s) { if (have_tc) carry = tc.slash_absorbed_before; else need |= NEED_S; }
+            if (open_a) { if (have_tc) carry = tc.nl_absorbed_before; else need |= NEED_A; }
+        }
+        const u64 slq = SL & nD;
+        const u64 sel = (SL & ~PREV(SL) & PREV(A)) | ((slq & 1) ? (u64)carry : 0);
+        AS = slq & ~(slq + sel);
+    }
+    // ---- punctuation: a run start that no blank precedes; an absorbed slash is no start and ends the run before it
+    const u64 Oe = O & ~AS;
+    const u64 G = Oe & lead & ~PREV(Oe) & ~PREV(SP);
+    S |= G;
+    // ---- words: run start unless non-CR/LF whitespace or a single match-start punctuation char is the prefix
+    const u64 c1 = cont << 1, c2 = cont << 2, c3 = cont << 3;
+    const u64 pfx = ((G << 1) | ((G << 2) & c1) | ((G << 3) & c2 & c1) | ((G << 4) & c3 & c2 & c1)) & nD;
+    S |= Lr & lead & ~PREV(Lr) & ~((PREV(W) & ~PREV(NL)) | pfx);
+    S |= upp & lead & PREV(low);                          // case boundary: upper after lower
+    // ---- number runs: every third lead counted from the run start
+    {
+        const u32 n_own = (u32)(N >> 32) & 0xFFFFu, ld_own = (u32)(lead >> 32) & 0xFFFFu;
+        const u32 nstart = (u32)((N & ~PREV(N)) >> 32) & 0xFFFFu;
+        u32 m = n_own & ld_own;
+        if (m) {
+            u32 cnt = 0;
+            if ((n_own & 1) && !(nstart & 1)) {
+                bool open;
+                cnt = tt_walk_back_num(sm, slot - 1, open);
+                if (open) { if (have_tc) cnt += tc.n_before; else need |= NEED_N; }
+                cnt %= 3;
+            }
+            while (m) {
+                int i = tt_lobit(m); m &= m - 1;
+                if ((nstart >> i) & 1) cnt = 0;
+                if (cnt == 0) S |= 1ull << (32 + i);
+                cnt = cnt == 2 ? 0 : cnt + 1;
+            }
+        }
+    }
+    // ---- whitespace runs (same rules as pattern 0; "punctuation" excludes marks here)
+    if (W & OWN) {
+        S |= W & lead & ~PREV(W) & ~(PREV(O) & NL);
+        S |= W & lead & ~NL & PREV(A);
+        const u64 next_exists = (V >> 1) & ~(D >> 1);
+        const u64 wend = W & ~((W >> 1) & ~(D >> 1)) & next_exists;
+        const u64 k1 = cont >> 1, k2 = cont >> 2, k3 = cont >> 3;
+        S |= lead & W & ~NL & (wend | ((wend >> 1) & k1) | ((wend >> 2) & k1 & k2) | ((wend >> 3) & k1 & k2 & k3));
+        u32 cand = (u32)((W & lead & ~NL & PREV(NL)) >> 32) & 0xFFFFu;
+        while (cand) {
+            int i = tt_lobit(cand); cand &= cand - 1;
+            bool open;
+            u32 later = tt_walk_fwd_nl(sm, slot, i, open);
+            if (open) { if (have_tc) later = tc.nl_later_after; else { need |= NEED_F; later = 1; } }
+            if (!later) S |= 1ull << (32 + i);
+        }
+    }
+    // ---- unresolved constructs: propagate from each one up to the next sure start
+    const u64 pLr = PREV(Lr), pN = PREV(N);
+    const u64 sure = (D | (N & ~pN) | (W & (pLr | pN)) | (O & ~AP & (pLr | pN)) | (Lr & (pN | PREV(NL)))) & lead;
+    const u64 hard = (Mk | (upp & PREV(cless)) | (AP & pLr & ((Lr >> 1) & ~(D >> 1)))) & lead;
+    // Window bits 0..15 (slot-2) lack look-back at bit 0, so events there are taken from the walk,
+    // which starts at slot-2 and has full neighbour information; propagation runs over bits 16..63.
+    u64 dirty;
+    {
+        u32 carry = 0;
+        bool open;
+        carry = tt_walk_back_dirty(sm, slot - 2, open);
+        if (open) { if (have_tc) carry = tc.dirty_before; else need |= NEED_H; }
+        const u64 sure2 = sure & ~0xFFFFull;
+        u64 F = (hard & ~0xFFFFull) | (((u64)carry << 16) & ~sure2);
+        u64 R = ~sure2;
+        F |= (F << 1) & R;  R &= R << 1;
+        F |= (F << 2) & R;  R &= R << 2;
+        F |= (F << 4) & R;  R &= R << 4;
+        F |= (F << 8) & R;  R &= R << 8;
+        F |= (F << 16) & R; R &= R << 16;
+        F |= (F << 32) & R;
+        dirty = F;
+    }
+    u32 pending = (u32)((dirty & OWN & V) >> 32) & 0xFFFFu;
+    u32 res = (u32)((S & lead & OWN) >> 32) & 0xFFFFu;
+    while (pending) {
+        // re-derive from the last sure start at or below the first unresolved byte, up to the end of
+        // the chunk or of the document, whichever comes first
+        const int first = tt_lobit(pending) + 32;
+        const u64 below = sure & ((2ull << first) - 1) & ~0xFFFFull;
+        long long from = -1;
+        if (below) {
+            int hb = (below >> 32) ? 32 + tt_hibit((u32)(below >> 32)) : tt_hibit((u32)below);
+            from = g0 + (hb - 32);
+        } else {
+            int pos = tt_walk_back_sure(sm, slot - 2);
+            if (pos >= 0) from = g0 + ((long long)pos - (long long)slot * 16);
+            else if (have_tc) from = tc.sure_before;
+            else need |= NEED_C;
+        }
+        if (from < 0) break;
+        long long doc_end;
+        const u32 seq = tt_seq_starts_p1(C, from, g0, doc_end);
+        const int fb = from > g0 ? (int)(from - g0) : 0;
+        const int eb = doc_end - g0 >= 16 ? 16 : (int)(doc_end - g0);
+        const u32 take = (0xFFFFu << fb) & ~(eb >= 16 ? 0u : (0xFFFFu << eb)) & 0xFFFFu;
+        res = (res & ~take) | (seq & take);
+        pending &= ~take;
+        pending &= ~((1u << (first - 32)) | ((1u << (first - 32)) - 1));     // always make progress
+    }
+    return res;
+#undef PREV
 }

@@ -31,7 +31,7 @@ def to_dev(a: np.ndarray, offset: int = 0):
     import torch
     buf = torch.zeros(a.size + offset + 64, dtype=torch.uint8, device="cuda")
     t = buf[offset:offset + a.size]
-    t.copy_(torch.from_numpy(np.ascontiguousarray(a)))
+    t.copy_(torch.from_numpy(np.array(a, dtype=np.uint8, copy=True)))
     return t
 
 

@@ -12,6 +12,7 @@
 #include <cstdio>
 #include <cstring>
 #include <new>
+#include <string>
 #include <unordered_map>
 #include <unordered_set>
 #include <vector>
@@ -27,6 +28,9 @@ struct tt_vocab {
     u8* d_cls = nullptr;
     int cls_bytes = 0;
     PairTable tab{};
+    TokSlot* d_tokslots = nullptr;
+    TokTable toktab{};
+    size_t n_table_tokens = 0;
     // cached buffers of tt_encode_host
     u8* h_text = nullptr; int32_t* h_ids = nullptr; long long* h_scalars = nullptr;
     u8* d_text = nullptr; int32_t* d_ids = nullptr; long long* d_count = nullptr; int32_t* d_status = nullptr;
@@ -61,13 +65,86 @@ extern "C" size_t tt_class_table(uint8_t* out, size_t cap) {
 
 extern "C" void tt_vocab_free(tt_vocab* v) {
     if (!v) return;
-    cudaFree(v->d_slots); cudaFree(v->d_ext_id); cudaFree(v->d_cls);
+    cudaFree(v->d_slots); cudaFree(v->d_ext_id); cudaFree(v->d_cls); cudaFree(v->d_tokslots);
     cudaFree(v->d_text); cudaFree(v->d_ids); cudaFree(v->d_count); cudaFree(v->d_status); cudaFree(v->d_ws);
     if (v->h_text) cudaFreeHost(v->h_text);
     if (v->h_ids) cudaFreeHost(v->h_ids);
     if (v->h_scalars) cudaFreeHost(v->h_scalars);
     if (v->host_stream) cudaStreamDestroy(v->host_stream);
     delete v;
+}
+
+
+// Whole-piece table: every token of at most TT_TOKTAB_MAXLEN bytes is encoded with the merge kernel
+// itself; those whose byte string yields exactly that one token are entered (key = bytes, value = the
+// caller's id).  A hit in the table therefore equals what the merge loop returns for that piece.
+static int build_token_table(tt_vocab* v, const tt_merge* merges, size_t n_merges, const std::vector<int32_t>& ext_id) {
+    (void)merges;
+    // byte strings of the merge results, by internal id (operands are lower internal ids by construction)
+    std::vector<std::string> bytes(256 + n_merges);
+    for (int b = 0; b < 256; b++) bytes[b] = std::string(1, (char)b);
+    std::unordered_map<int32_t, u32> internal;
+    internal.reserve(2 * ext_id.size());
+    for (size_t i = 0; i < ext_id.size(); i++) internal.emplace(ext_id[i], (u32)i);
+    std::vector<u32> cand;                       // internal ids of candidate tokens
+    std::vector<u8> cat; std::vector<u32> off;
+    for (size_t r = 0; r < n_merges; r++) {
+        const std::string& L = bytes[internal[merges[r].left]];
+        const std::string& R = bytes[internal[merges[r].right]];
+        if (L.size() + R.size() <= 4096) bytes[256 + r] = L + R;          // longer strings are never candidates
+        else bytes[256 + r] = std::string(4097, 'x');
+        const std::string& t = bytes[256 + r];
+        if (t.size() >= 2 && t.size() <= (size_t)TT_TOKTAB_MAXLEN) {
+            cand.push_back((u32)(256 + r)); off.push_back((u32)cat.size());
+            cat.insert(cat.end(), t.begin(), t.end());
+        }
+    }
+    off.push_back((u32)cat.size());
+    if (cand.empty()) return TT_OK;
+    const size_t nb = cat.size(), np = cand.size();
+    u8* d_text = nullptr; u32 *d_off = nullptr, *d_cnt = nullptr, *d_long = nullptr; int32_t* d_stage = nullptr; TTHeader* d_hdr = nullptr;
+    TTHeader h; memset(&h, 0, sizeof(h)); h.n_pieces = (u32)np;
+    std::vector<u32> cnt(np); std::vector<int32_t> stage(nb);
+    bool ok = cudaMalloc(&d_text, nb + 64) == cudaSuccess && cudaMalloc(&d_off, (np + 1) * sizeof(u32)) == cudaSuccess &&
+              cudaMalloc(&d_cnt, np * sizeof(u32)) == cudaSuccess && cudaMalloc(&d_long, (np + 1) * sizeof(u32)) == cudaSuccess &&
+              cudaMalloc(&d_stage, nb * sizeof(int32_t)) == cudaSuccess && cudaMalloc(&d_hdr, sizeof(TTHeader)) == cudaSuccess;
+    ok = ok && cudaMemcpy(d_text, cat.data(), nb, cudaMemcpyHostToDevice) == cudaSuccess;
+    ok = ok && cudaMemcpy(d_off, off.data(), (np + 1) * sizeof(u32), cudaMemcpyHostToDevice) == cudaSuccess;
+    ok = ok && cudaMemcpy(d_hdr, &h, sizeof(h), cudaMemcpyHostToDevice) == cudaSuccess;
+    if (ok) {
+        k_bpe_warp<<<v->sm_count * 8, BPE_WARPS * 32>>>(d_text, d_off, d_hdr, v->tab, v->d_ext_id, d_cnt, d_stage, d_long, nullptr);
+        ok = cudaGetLastError() == cudaSuccess && cudaDeviceSynchronize() == cudaSuccess;
+    }
+    ok = ok && cudaMemcpy(cnt.data(), d_cnt, np * sizeof(u32), cudaMemcpyDeviceToHost) == cudaSuccess;
+    ok = ok && cudaMemcpy(stage.data(), d_stage, nb * sizeof(int32_t), cudaMemcpyDeviceToHost) == cudaSuccess;
+    cudaFree(d_text); cudaFree(d_off); cudaFree(d_cnt); cudaFree(d_long); cudaFree(d_stage); cudaFree(d_hdr);
+    if (!ok) { cudaGetLastError(); return TT_ERR_CUDA; }
+    std::vector<u32> keep;
+    for (size_t i = 0; i < np; i++)
+        if (cnt[i] == 1 && stage[off[i]] == ext_id[cand[i]]) keep.push_back((u32)i);
+    u32 cap = 1024;
+    while (cap < 2 * keep.size() + 2) cap <<= 1;
+    u32 log2cap = 0;
+    while ((1u << log2cap) < cap) log2cap++;
+    const u32 mask = cap - 1, shift = 64 - log2cap;
+    std::vector<TokSlot> slots(cap);
+    memset(slots.data(), 0, cap * sizeof(TokSlot));
+    for (u32 i : keep) {
+        const u32 n = off[i + 1] - off[i];
+        u8 key[24] = {0};
+        memcpy(key, cat.data() + off[i], n);
+        u64 k[3]; memcpy(k, key, 24);
+        u32 hh = toktab_hash(k[0], k[1], k[2], n, shift);
+        while (slots[hh].len != 0) hh = (hh + 1) & mask;
+        slots[hh].k0 = k[0]; slots[hh].k1 = k[1]; slots[hh].k2 = k[2]; slots[hh].len = n; slots[hh].id = ext_id[cand[i]];
+    }
+    if (cudaMalloc(&v->d_tokslots, (size_t)cap * sizeof(TokSlot)) != cudaSuccess ||
+        cudaMemcpy(v->d_tokslots, slots.data(), (size_t)cap * sizeof(TokSlot), cudaMemcpyHostToDevice) != cudaSuccess) {
+        cudaGetLastError(); return TT_ERR_CUDA;
+    }
+    v->toktab.slots = v->d_tokslots; v->toktab.mask = mask; v->toktab.shift = shift;
+    v->n_table_tokens = keep.size();
+    return TT_OK;
 }
 
 extern "C" int tt_vocab_load(const tt_merge* merges, size_t n_merges, const int32_t byte_map[256], int pattern_id,
@@ -125,6 +202,7 @@ extern "C" int tt_vocab_load(const tt_merge* merges, size_t n_merges, const int3
     ok = ok && cudaMemcpy(v->d_cls, cls.data(), v->cls_bytes, cudaMemcpyHostToDevice) == cudaSuccess;
     if (!ok) { cudaGetLastError(); tt_vocab_free(v); return TT_ERR_CUDA; }
     v->tab.slots = v->d_slots; v->tab.mask = mask; v->tab.shift = shift;
+    if (build_token_table(v, merges, n_merges, ext_id) != TT_OK) { tt_vocab_free(v); return TT_ERR_CUDA; }
     *out = v;
     return TT_OK;
 }
@@ -217,15 +295,22 @@ static int encode_impl(const tt_vocab* v, const uint8_t* text, size_t len, const
     if (rc != TT_OK) return rc;
     MARK(2);
     const int bpe_grid = v->sm_count * 8;
-    k_bpe_warp<<<bpe_grid, BPE_WARPS * 32, 0, st>>>(text, w.piece_off, w.hdr, v->tab, v->d_ext_id, w.piece_cnt, w.stage,
-                                                    w.long_list);
+    {
+        const size_t want = (len / 4 + 255) / 256;                       // about one thread per expected piece
+        const int lookup_grid = (int)(want < 1 ? 1 : want > (size_t)v->sm_count * 16 ? (size_t)v->sm_count * 16 : want);
+        k_bpe_lookup<<<lookup_grid, 256, 0, st>>>(text, w.piece_off, w.hdr, v->toktab, v->d_ext_id, w.piece_cnt, w.stage,
+                                                  w.tok_off /* miss list until the scatter */);
+    }
     MARK(3);
+    k_bpe_warp<<<bpe_grid, BPE_WARPS * 32, 0, st>>>(text, w.piece_off, w.hdr, v->tab, v->d_ext_id, w.piece_cnt, w.stage,
+                                                    w.long_list, w.tok_off);
+    MARK(4);
     k_bpe_long<<<v->sm_count, LONG_THREADS, 0, st>>>(text, w.piece_off, w.hdr, v->tab, v->d_ext_id, w.piece_cnt, w.stage,
                                                      w.rank_buf, w.long_list);
-    MARK(4);
+    MARK(5);
     const int nblk = (int)((len + CNT_THREADS - 1) / CNT_THREADS);
     k_count<<<nblk, CNT_THREADS, 0, st>>>(w.piece_cnt, w.hdr, w.blk_cnt, (unsigned long long)ids_cap);
-    MARK(5);
+    MARK(6);
     k_scatter<<<nblk, CNT_THREADS, 0, st>>>(w.piece_off, w.piece_cnt, w.blk_cnt, w.stage, w.hdr, w.tok_off, ids_out,
                                             (long long*)count_out, status_out);
     if (doc_off) {
@@ -233,7 +318,7 @@ static int encode_impl(const tt_vocab* v, const uint8_t* text, size_t len, const
         k_doc_offsets<<<blocks, threads, 0, st>>>((const long long*)doc_off, (int)n_docs, w.piece_off, w.tok_off, w.hdr,
                                                   (long long*)ids_off_out);
     }
-    MARK(6);
+    MARK(7);
 #undef MARK
     CK(cudaGetLastError());
     return TT_OK;
@@ -261,18 +346,18 @@ extern "C" int tt_encode_batch(const tt_vocab* v, const uint8_t* text, size_t to
 
 extern "C" int tt_encode_timed(const tt_vocab* v, const uint8_t* text, size_t len, void* stream, int32_t* ids_out,
                                size_t ids_cap, int64_t* count_out, int32_t* status_out, void* workspace,
-                               size_t workspace_bytes, float ms_out[6]) {
+                               size_t workspace_bytes, float ms_out[7]) {
     int rc = check_common(v, text, len, workspace, workspace_bytes, 1);
     if (rc != TT_OK) return rc;
     if (!count_out || !status_out || !ms_out || !len || !ids_out) return TT_ERR_ARG;
-    cudaEvent_t ev[7];
-    for (int i = 0; i < 7; i++) CK(cudaEventCreate(&ev[i]));
+    cudaEvent_t ev[8];
+    for (int i = 0; i < 8; i++) CK(cudaEventCreate(&ev[i]));
     rc = encode_impl(v, text, len, nullptr, 1, (cudaStream_t)stream, ids_out, ids_cap, count_out, nullptr, status_out,
                      workspace, ev);
-    if (rc == TT_OK && cudaEventSynchronize(ev[6]) != cudaSuccess) rc = TT_ERR_CUDA;
-    for (int i = 0; i < 6 && rc == TT_OK; i++)
+    if (rc == TT_OK && cudaEventSynchronize(ev[7]) != cudaSuccess) rc = TT_ERR_CUDA;
+    for (int i = 0; i < 7 && rc == TT_OK; i++)
         if (cudaEventElapsedTime(&ms_out[i], ev[i], ev[i + 1]) != cudaSuccess) rc = TT_ERR_CUDA;
-    for (int i = 0; i < 7; i++) cudaEventDestroy(ev[i]);
+    for (int i = 0; i < 8; i++) cudaEventDestroy(ev[i]);
     return rc;
 }
 

@@ -28,6 +28,83 @@ __device__ __forceinline__ u32 pair_probe(const PairTable& t, u32 a, u32 b) {
     return TT_RANK_INF;
 }
 
+// ---- whole-piece table: byte string of a vocabulary entry -> its id ------------------------------------
+// Holds every token of at most TT_TOKTAB_MAXLEN bytes whose own byte string encodes to exactly that
+// token (checked at load time by running the merge kernel below on every token string), so a hit
+// returns what the merge loop would return.  Slots are 32 bytes (one sector): three key words, the
+// length (0 = empty) and the caller's id; open addressing, linear probing, load factor <= 0.5.
+constexpr int TT_TOKTAB_MAXLEN = 24;
+struct TokSlot { u64 k0, k1, k2; u32 len; int32_t id; };
+static_assert(sizeof(TokSlot) == 32, "slot layout");
+struct TokTable { const TokSlot* slots; u32 mask; u32 shift; };
+
+TT_HD u32 toktab_hash(u64 k0, u64 k1, u64 k2, u32 len, u32 shift) {
+    u64 h = (k0 + len) * 0x9E3779B97F4A7C15ull;
+    h ^= (k1 + 0x632BE59BD9B4E019ull) * 0xC2B2AE3D27D4EB4Full;
+    h ^= (k2 + 0x85157AF5ull) * 0x165667B19E3779F9ull;
+    h ^= h >> 29;
+    h *= 0xBF58476D1CE4E5B9ull;
+    return (u32)(h >> shift);
+}
+
+// K4, thread per piece: one-byte pieces map directly; pieces of up to 24 bytes are looked up as whole
+// vocabulary entries; everything else (and every miss) goes to the miss list for the merge kernels.
+__global__ void __launch_bounds__(256)
+k_bpe_lookup(const u8* __restrict__ text, const u32* __restrict__ piece_off, TTHeader* hdr, const TokTable tab,
+             const int32_t* __restrict__ ext_id, u32* __restrict__ piece_cnt, int32_t* __restrict__ stage,
+             u32* __restrict__ miss_list) {
+    if (hdr->status != 0) return;
+    const u32 n_pieces = hdr->n_pieces;
+    const u32 lane = threadIdx.x & 31;
+    const u32 stride = gridDim.x * blockDim.x;
+    const u32 rounds = (n_pieces + stride - 1) / stride;
+    u32 p = blockIdx.x * blockDim.x + threadIdx.x;
+    for (u32 it = 0; it < rounds; it++, p += stride) {
+        bool miss = false;
+        if (p < n_pieces) {
+            const u32 a = piece_off[p], n = piece_off[p + 1] - a;
+            if (n == 1) {
+                stage[a] = ext_id[text[a]]; piece_cnt[p] = 1;
+            } else if (n > TT_TOKTAB_MAXLEN || tab.slots == nullptr) {
+                miss = true;
+            } else {
+                // gather the piece's bytes with aligned 8-byte loads (only words that hold a piece byte)
+                const uintptr_t addr = (uintptr_t)(text + a);
+                const u64* w = reinterpret_cast<const u64*>(addr & ~(uintptr_t)7);
+                const u32 sh = (u32)(addr & 7) * 8, last = (u32)(addr & 7) + n;     // bytes used in the window
+                const u64 w0 = __ldg(w), w1 = last > 8 ? __ldg(w + 1) : 0, w2 = last > 16 ? __ldg(w + 2) : 0,
+                          w3 = last > 24 ? __ldg(w + 3) : 0;
+                u64 k0 = sh ? (w0 >> sh) | (w1 << (64 - sh)) : w0;
+                u64 k1 = sh ? (w1 >> sh) | (w2 << (64 - sh)) : w1;
+                u64 k2 = sh ? (w2 >> sh) | (w3 << (64 - sh)) : w2;
+                if (n < 8) { k0 &= (1ull << (8 * n)) - 1; k1 = 0; k2 = 0; }
+                else if (n < 16) { k1 &= (n == 8) ? 0 : ((1ull << (8 * (n - 8))) - 1); k2 = 0; }
+                else if (n < 24) { k2 &= (n == 16) ? 0 : ((1ull << (8 * (n - 16))) - 1); }
+                u32 h = toktab_hash(k0, k1, k2, n, tab.shift);
+                miss = true;
+                for (u32 probe = 0; probe <= tab.mask; probe++) {           // bounded by the capacity
+                    const uint4* sp = reinterpret_cast<const uint4*>(tab.slots + h);
+                    const uint4 lo = __ldg(sp), hi = __ldg(sp + 1);
+                    const u32 slen = hi.z;
+                    if (slen == 0) break;
+                    if (slen == n && (((u64)lo.y << 32) | lo.x) == k0 && (((u64)lo.w << 32) | lo.z) == k1 &&
+                        (((u64)hi.y << 32) | hi.x) == k2) {
+                        stage[a] = (int32_t)hi.w; piece_cnt[p] = 1; miss = false; break;
+                    }
+                    h = (h + 1) & tab.mask;
+                }
+            }
+        }
+        const u32 mm = __ballot_sync(0xFFFFFFFFu, miss);
+        if (mm) {
+            u32 base = 0;
+            if (lane == 0) base = atomicAdd(&hdr->n_miss, (u32)__popc(mm));
+            base = __shfl_sync(0xFFFFFFFFu, base, 0);
+            if (miss) miss_list[base + __popc(mm & ((1u << lane) - 1))] = p;
+        }
+    }
+}
+
 constexpr u32 RK_STALE = 0xFFFFFFFEu;                 // rank must be probed again
 constexpr int BPE_WARPS = 8;                          // warps per CTA of the warp-per-piece kernel
 constexpr int WCH = TT_WARP_PIECE_MAX / 32;           // 32-token chunks per piece
@@ -36,17 +113,19 @@ constexpr int WCH = TT_WARP_PIECE_MAX / 32;           // 32-token chunks per pie
 __global__ void __launch_bounds__(BPE_WARPS * 32)
 k_bpe_warp(const u8* __restrict__ text, const u32* __restrict__ piece_off, TTHeader* hdr, const PairTable tab,
            const int32_t* __restrict__ ext_id, u32* __restrict__ piece_cnt, int32_t* __restrict__ stage,
-           u32* __restrict__ long_list) {
+           u32* __restrict__ long_list, const u32* __restrict__ miss_list) {
     __shared__ u32 s_tok[BPE_WARPS][TT_WARP_PIECE_MAX];
     __shared__ u32 s_rk[BPE_WARPS][TT_WARP_PIECE_MAX];
     if (hdr->status != 0) return;
-    const u32 n_pieces = hdr->n_pieces;
+    // with a miss list: the pieces the lookup kernel could not settle; without: every piece
+    const u32 n_items = miss_list ? hdr->n_miss : hdr->n_pieces;
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
     const u32 lt = (1u << lane) - 1;
     u32* tok = s_tok[wid];
     u32* rk = s_rk[wid];
     const u32 nwarps = gridDim.x * BPE_WARPS;
-    for (u32 p = blockIdx.x * BPE_WARPS + wid; p < n_pieces; p += nwarps) {
+    for (u32 item = blockIdx.x * BPE_WARPS + wid; item < n_items; item += nwarps) {
+        const u32 p = miss_list ? miss_list[item] : item;
         const u32 a = piece_off[p], n = piece_off[p + 1] - a;
         if (n > TT_WARP_PIECE_MAX) {
             if (lane == 0) long_list[atomicAdd(&hdr->n_long, 1u)] = p;

@@ -43,7 +43,7 @@ struct TTHeader {
     u32 n_long;              // entries in the long-piece list
     u32 long_next;           // work counter of the long-piece kernel
     u32 piece_next;          // work counter of the warp BPE kernel
-    u32 pad0;
+    u32 n_miss;              // entries in the miss list (pieces that need the merge loop)
     unsigned long long n_tokens;   // total tokens
     u32 pad[22];
 };
@@ -57,7 +57,7 @@ struct TTWorkspace {
     u32* piece_off;    // byte offset of every piece + sentinel (len + 2)
     u32* piece_cnt;    // tokens per piece (len + 1)
     u32* blk_cnt;      // token count per block of pieces, then exclusive prefix
-    u32* tok_off;      // token offset of every piece + total (len + 2)
+    u32* tok_off;      // token offset of every piece + total (len + 2); before the scatter: the miss list
     int32_t* stage;    // token ids staged at the byte offset of their piece (len)
     u32* rank_buf;     // per-position ranks for the long-piece path (len)
     u32* long_list;    // piece indices longer than TT_WARP_PIECE_MAX

@@ -156,6 +156,8 @@ def main():
     ap.add_argument("--no-batch", action="store_true", help="skip the config-C5 batch leg")
     ap.add_argument("--no-cpu", action="store_true", help="skip the cpu_baseline leg")
     ap.add_argument("--batch-docs", type=int, default=256)
+    ap.add_argument("--profile", action="store_true",
+                    help="run only the warm-up and the timed steps, then exit (command used under ncu)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -222,6 +224,11 @@ def main():
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         total_ms = float(t.item())
     ms_per_step = total_ms / args.steps
+
+    if args.profile:
+        if rank == 0:
+            print(json.dumps({"profile_run": True, "ms_per_step": round(ms_per_step, 4), "steps": args.steps}), flush=True)
+        return
 
     # ---- steady state (same buffer re-encoded, caches warm), for context ----
     warm = []

@@ -330,7 +330,7 @@ def main():
         "chars_per_s_single": round(cfg.n_chars / (ms_per_step * 1e-3), 1),
         "e2e": {"value": round(e2e_ms, 4), "unit": "ms", "h2d_bytes_per_step": nbytes, "d2h_bytes_per_step": 4 * n_ids + 12,
                 "p50": round(pct(e2e, 0.5), 4), "api": "tt_encode_host (pageable host buffers in, pinned staging inside)"},
-        "gpu_launches": 7 * args.steps,
+        "gpu_launches": 5 * args.steps,
         "batch": batch,
         "roofline": roofline,
         "cpu_baseline": cpu,

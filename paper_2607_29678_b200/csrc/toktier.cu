@@ -1,5 +1,6 @@
 // C ABI of the toktier library (see include/toktier.h).  Host side: argument checks, vocabulary
-// tables, workspace layout and the kernel chain  K1+K2 -> K3 -> K4 (warp) -> K4 (long) -> K5a -> K5b.
+// tables, workspace layout and the kernel chain  K1+K2 -> K3 -> K4 (long pieces) -> K4 (all other pieces,
+// with K5's count scan in its last CTA) -> K5 scatter.
 // Nothing here synchronises with the device except tt_vocab_load and tt_encode_host.
 #include "../../include/toktier.h"
 #include "tt_common.cuh"
@@ -103,16 +104,19 @@ static int build_token_table(tt_vocab* v, const tt_merge* merges, size_t n_merge
     if (cand.empty()) return TT_OK;
     const size_t nb = cat.size(), np = cand.size();
     u8* d_text = nullptr; u32 *d_off = nullptr, *d_cnt = nullptr, *d_long = nullptr; int32_t* d_stage = nullptr; TTHeader* d_hdr = nullptr;
+    const size_t nblocks = (np + BPE_THREADS - 1) / BPE_THREADS;
     TTHeader h; memset(&h, 0, sizeof(h)); h.n_pieces = (u32)np;
     std::vector<u32> cnt(np); std::vector<int32_t> stage(nb);
     bool ok = cudaMalloc(&d_text, nb + 64) == cudaSuccess && cudaMalloc(&d_off, (np + 1) * sizeof(u32)) == cudaSuccess &&
-              cudaMalloc(&d_cnt, np * sizeof(u32)) == cudaSuccess && cudaMalloc(&d_long, (np + 1) * sizeof(u32)) == cudaSuccess &&
+              cudaMalloc(&d_cnt, np * sizeof(u32)) == cudaSuccess && cudaMalloc(&d_long, (nblocks + 1) * sizeof(u32)) == cudaSuccess &&
               cudaMalloc(&d_stage, nb * sizeof(int32_t)) == cudaSuccess && cudaMalloc(&d_hdr, sizeof(TTHeader)) == cudaSuccess;
     ok = ok && cudaMemcpy(d_text, cat.data(), nb, cudaMemcpyHostToDevice) == cudaSuccess;
     ok = ok && cudaMemcpy(d_off, off.data(), (np + 1) * sizeof(u32), cudaMemcpyHostToDevice) == cudaSuccess;
     ok = ok && cudaMemcpy(d_hdr, &h, sizeof(h), cudaMemcpyHostToDevice) == cudaSuccess;
     if (ok) {
-        k_bpe_warp<<<v->sm_count * 8, BPE_WARPS * 32>>>(d_text, d_off, d_hdr, v->tab, v->d_ext_id, d_cnt, d_stage, d_long, nullptr);
+        TokTable none; none.slots = nullptr; none.mask = 0; none.shift = 0;
+        k_bpe_pieces<<<v->sm_count * 8, BPE_THREADS>>>(d_text, d_off, d_hdr, v->tab, none, v->d_ext_id, d_cnt, d_stage,
+                                                        d_long /* block totals, unused */, ~0ull);
         ok = cudaGetLastError() == cudaSuccess && cudaDeviceSynchronize() == cudaSuccess;
     }
     ok = ok && cudaMemcpy(cnt.data(), d_cnt, np * sizeof(u32), cudaMemcpyDeviceToHost) == cudaSuccess;
@@ -161,22 +165,29 @@ extern "C" int tt_vocab_load(const tt_merge* merges, size_t n_merges, const int3
         if (byte_map[b] < 0 || !internal.emplace(byte_map[b], (u32)b).second) return TT_ERR_BAD_VOCAB;   // not injective
         ext_id[b] = byte_map[b];
     }
-    u32 cap = 1024;
-    while (cap < 2 * n_merges + 2) cap <<= 1;
-    u32 log2cap = 0;
-    while ((1u << log2cap) < cap) log2cap++;
+    // pair table: buckets of four slots, at most one key per bucket on average
+    u32 nbuckets = 256;
+    while (nbuckets < n_merges + 1) nbuckets <<= 1;
+    u32 log2b = 0;
+    while ((1u << log2b) < nbuckets) log2b++;
+    const u32 cap = 4 * nbuckets;
     std::vector<u64> slots(cap, TT_SLOT_EMPTY);
-    const u32 mask = cap - 1, shift = 64 - log2cap;
+    const u32 mask = nbuckets - 1, shift = 64 - log2b;
+    std::unordered_set<u64> seen;
+    seen.reserve(2 * n_merges + 16);
     for (size_t r = 0; r < n_merges; r++) {
         const tt_merge& m = merges[r];
         auto l = internal.find(m.left), rr = internal.find(m.right);
         if (l == internal.end() || rr == internal.end()) return TT_ERR_BAD_VOCAB;      // operand not yet defined
         if (m.result < 0 || internal.count(m.result)) return TT_ERR_BAD_VOCAB;         // result id reused
         const u64 key = ((u64)l->second << TT_ID_BITS) | rr->second;
-        u32 h = (u32)((key * 0x9E3779B97F4A7C15ull) >> shift);
+        if (!seen.insert(key).second) return TT_ERR_BAD_VOCAB;                         // duplicate pair
+        u32 h = pair_bucket(key, shift);
         for (;;) {
-            if (slots[h] == TT_SLOT_EMPTY) { slots[h] = (key << 20) | (u64)r; break; }
-            if ((slots[h] >> 20) == key) return TT_ERR_BAD_VOCAB;                      // duplicate pair
+            u64* b = &slots[4 * (size_t)h];
+            int k = 0;
+            while (k < 4 && b[k] != TT_SLOT_EMPTY) k++;
+            if (k < 4) { b[k] = (key << 20) | (u64)r; break; }
             h = (h + 1) & mask;
         }
         internal.emplace(m.result, (u32)(256 + r));
@@ -213,7 +224,7 @@ static size_t carve(TTWorkspace* w, void* base, size_t max_len, size_t max_docs)
     const size_t padded = max_len + 64;                       // aligned frame: up to 15 bytes of shift + tail
     const size_t nchunks = padded / TT_CHUNK + 2;
     const size_t ntiles = nchunks / TT_TILE_CHUNKS + 2;
-    const size_t nblk = max_len / CNT_THREADS + 2;
+    const size_t nblk = max_len / BPE_THREADS + 2;
     size_t off = 0;
     auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return (char*)base + o; };
     char* p;
@@ -263,7 +274,7 @@ static int run_pretok(const tt_vocab* v, const uint8_t* text, size_t len, const 
     k_pretok<<<grid, TT_TILE_CHUNKS, smem, st>>>(P);
     if (ev_mid) cudaEventRecord(ev_mid, st);
     k_compact<<<grid, TT_TILE_CHUNKS, 0, st>>>(w.startmask, w.tile_cnt, P.nchunks, P.ntiles, shift, (long long)len,
-                                               piece_off_dst, w.hdr);
+                                               piece_off_dst, w.hdr, w.long_list, TT_WARP_PIECE_MAX);
     CK(cudaGetLastError());
     return TT_OK;
 }
@@ -294,31 +305,22 @@ static int encode_impl(const tt_vocab* v, const uint8_t* text, size_t len, const
     int rc = run_pretok(v, text, len, doc_off, n_docs, st, w, w.piece_off, ev ? ev[1] : nullptr);
     if (rc != TT_OK) return rc;
     MARK(2);
-    const int bpe_grid = v->sm_count * 8;
-    {
-        const size_t want = (len / 4 + 255) / 256;                       // about one thread per expected piece
-        const int lookup_grid = (int)(want < 1 ? 1 : want > (size_t)v->sm_count * 16 ? (size_t)v->sm_count * 16 : want);
-        k_bpe_lookup<<<lookup_grid, 256, 0, st>>>(text, w.piece_off, w.hdr, v->toktab, v->d_ext_id, w.piece_cnt, w.stage,
-                                                  w.tok_off /* miss list until the scatter */);
-    }
-    MARK(3);
-    k_bpe_warp<<<bpe_grid, BPE_WARPS * 32, 0, st>>>(text, w.piece_off, w.hdr, v->tab, v->d_ext_id, w.piece_cnt, w.stage,
-                                                    w.long_list, w.tok_off);
-    MARK(4);
     k_bpe_long<<<v->sm_count, LONG_THREADS, 0, st>>>(text, w.piece_off, w.hdr, v->tab, v->d_ext_id, w.piece_cnt, w.stage,
                                                      w.rank_buf, w.long_list);
-    MARK(5);
-    const int nblk = (int)((len + CNT_THREADS - 1) / CNT_THREADS);
-    k_count<<<nblk, CNT_THREADS, 0, st>>>(w.piece_cnt, w.hdr, w.blk_cnt, (unsigned long long)ids_cap);
-    MARK(6);
-    k_scatter<<<nblk, CNT_THREADS, 0, st>>>(w.piece_off, w.piece_cnt, w.blk_cnt, w.stage, w.hdr, w.tok_off, ids_out,
-                                            (long long*)count_out, status_out);
+    MARK(3);
+    const size_t want = (len + BPE_THREADS - 1) / BPE_THREADS;               // upper bound of piece blocks
+    const int piece_grid = (int)(want > (size_t)v->sm_count * 8 ? (size_t)v->sm_count * 8 : want);
+    k_bpe_pieces<<<piece_grid, BPE_THREADS, 0, st>>>(text, w.piece_off, w.hdr, v->tab, v->toktab, v->d_ext_id, w.piece_cnt,
+                                                     w.stage, w.blk_cnt, (unsigned long long)ids_cap);
+    MARK(4);
+    k_scatter<<<piece_grid, BPE_THREADS, 0, st>>>(w.piece_off, w.piece_cnt, w.blk_cnt, w.stage, w.hdr, w.tok_off, ids_out,
+                                                  (long long*)count_out, status_out);
     if (doc_off) {
         const int threads = 256, blocks = (int)((n_docs + 1 + threads - 1) / threads);
         k_doc_offsets<<<blocks, threads, 0, st>>>((const long long*)doc_off, (int)n_docs, w.piece_off, w.tok_off, w.hdr,
                                                   (long long*)ids_off_out);
     }
-    MARK(7);
+    MARK(5);
 #undef MARK
     CK(cudaGetLastError());
     return TT_OK;
@@ -346,18 +348,18 @@ extern "C" int tt_encode_batch(const tt_vocab* v, const uint8_t* text, size_t to
 
 extern "C" int tt_encode_timed(const tt_vocab* v, const uint8_t* text, size_t len, void* stream, int32_t* ids_out,
                                size_t ids_cap, int64_t* count_out, int32_t* status_out, void* workspace,
-                               size_t workspace_bytes, float ms_out[7]) {
+                               size_t workspace_bytes, float ms_out[5]) {
     int rc = check_common(v, text, len, workspace, workspace_bytes, 1);
     if (rc != TT_OK) return rc;
     if (!count_out || !status_out || !ms_out || !len || !ids_out) return TT_ERR_ARG;
-    cudaEvent_t ev[8];
-    for (int i = 0; i < 8; i++) CK(cudaEventCreate(&ev[i]));
+    cudaEvent_t ev[6];
+    for (int i = 0; i < 6; i++) CK(cudaEventCreate(&ev[i]));
     rc = encode_impl(v, text, len, nullptr, 1, (cudaStream_t)stream, ids_out, ids_cap, count_out, nullptr, status_out,
                      workspace, ev);
-    if (rc == TT_OK && cudaEventSynchronize(ev[7]) != cudaSuccess) rc = TT_ERR_CUDA;
-    for (int i = 0; i < 7 && rc == TT_OK; i++)
+    if (rc == TT_OK && cudaEventSynchronize(ev[5]) != cudaSuccess) rc = TT_ERR_CUDA;
+    for (int i = 0; i < 5 && rc == TT_OK; i++)
         if (cudaEventElapsedTime(&ms_out[i], ev[i], ev[i + 1]) != cudaSuccess) rc = TT_ERR_CUDA;
-    for (int i = 0; i < 8; i++) cudaEventDestroy(ev[i]);
+    for (int i = 0; i < 6; i++) cudaEventDestroy(ev[i]);
     return rc;
 }
 

@@ -1,28 +1,41 @@
-// Steps K4 and K5: byte-level BPE per piece, token-count scan and scatter of the IDs.
+// Steps K4 and K5: byte-level BPE per piece, token counts and scatter of the IDs.
 //
-// Paper Sec. 4.2: every piece is encoded independently; merge ranks live in a GPU hash table; a
-// round's minimum rank identifies one pair value, merging all its leftmost non-overlapping
-// occurrences equals iterated single merges, and only pairs next to a completed merge need to be
-// probed again.  Work is dispatched by piece length: a warp per piece up to TT_WARP_PIECE_MAX
-// bytes (state in shared memory, candidates as ballot masks), a CTA per longer piece (state in
-// global scratch).  Token ids used inside the kernels are "internal": byte b -> b, result of the
-// merge of rank r -> 256 + r; the caller's ids are looked up when the tokens are staged.
+// Paper Sec. 4.2: every piece is encoded independently; merge ranks and vocabulary entries live in
+// GPU hash tables; a round's minimum rank identifies one pair value, merging all its leftmost
+// non-overlapping occurrences equals iterated single merges, and only pairs next to a completed
+// merge need to be probed again.  Work is dispatched by piece length and difficulty:
+//   * a thread per piece looks the whole piece up as a vocabulary entry (one 32-byte probe);
+//   * pieces that are not a single entry are merged by a warp (<= 32 bytes: tokens in registers,
+//     candidates as ballot masks; <= 256 bytes: several tokens per lane, compaction through shared memory);
+//   * longer pieces are merged by a whole CTA with its state in global scratch (k_bpe_long).
+// Token ids inside the kernels are "internal": byte b -> b, result of the merge of rank r -> 256 + r;
+// the caller's ids are looked up when the tokens are staged.
 #pragma once
 #include "tt_common.cuh"
 
+// ---- pair table: (left, right) -> rank ---------------------------------------------------------------
+// Buckets of four 8-byte slots (one 32-byte sector); slot = (left << 38) | (right << 20) | rank.
+// A key lives in its home bucket or, if that is full, in the following ones; a bucket with a free
+// slot ends the search.  Sized for at most one key per bucket on average.
 struct PairTable {
-    const u64* slots;     // open addressing, linear probing; slot = (left << 38) | (right << 20) | rank
-    u32 mask;             // capacity - 1 (capacity is a power of two, load factor <= 0.5)
-    u32 shift;            // 64 - log2(capacity)
+    const u64* slots;     // 4 * (mask + 1) slots
+    u32 mask;             // number of buckets - 1 (power of two)
+    u32 shift;            // 64 - log2(number of buckets)
 };
+TT_HD u32 pair_bucket(u64 key, u32 shift) { return (u32)((key * 0x9E3779B97F4A7C15ull) >> shift); }
 
 __device__ __forceinline__ u32 pair_probe(const PairTable& t, u32 a, u32 b) {
     const u64 key = ((u64)a << TT_ID_BITS) | b;
-    u32 h = (u32)((key * 0x9E3779B97F4A7C15ull) >> t.shift);
-    for (u32 n = 0; n <= t.mask; n++) {               // bounded by the table capacity
-        const u64 s = __ldg(t.slots + h);
-        if (s == TT_SLOT_EMPTY) return TT_RANK_INF;
-        if ((s >> 20) == key) return (u32)(s & 0xFFFFFu);
+    u32 h = pair_bucket(key, t.shift);
+    for (u32 n = 0; n <= t.mask; n++) {               // bounded by the number of buckets
+        const uint4* bp = reinterpret_cast<const uint4*>(t.slots + 4 * (size_t)h);
+        const uint4 x = __ldg(bp), y = __ldg(bp + 1);
+        const u64 s0 = ((u64)x.y << 32) | x.x, s1 = ((u64)x.w << 32) | x.z, s2 = ((u64)y.y << 32) | y.x, s3 = ((u64)y.w << 32) | y.z;
+        if ((s0 >> 20) == key) return (u32)(s0 & 0xFFFFFu);
+        if ((s1 >> 20) == key) return (u32)(s1 & 0xFFFFFu);
+        if ((s2 >> 20) == key) return (u32)(s2 & 0xFFFFFu);
+        if ((s3 >> 20) == key) return (u32)(s3 & 0xFFFFFu);
+        if (s3 == TT_SLOT_EMPTY) return TT_RANK_INF;  // slots fill from the front: a free last slot ends the chain
         h = (h + 1) & t.mask;
     }
     return TT_RANK_INF;
@@ -47,163 +60,160 @@ TT_HD u32 toktab_hash(u64 k0, u64 k1, u64 k2, u32 len, u32 shift) {
     return (u32)(h >> shift);
 }
 
-// K4, thread per piece: one-byte pieces map directly; pieces of up to 24 bytes are looked up as whole
-// vocabulary entries; everything else (and every miss) goes to the miss list for the merge kernels.
-__global__ void __launch_bounds__(256)
-k_bpe_lookup(const u8* __restrict__ text, const u32* __restrict__ piece_off, TTHeader* hdr, const TokTable tab,
-             const int32_t* __restrict__ ext_id, u32* __restrict__ piece_cnt, int32_t* __restrict__ stage,
-             u32* __restrict__ miss_list) {
-    if (hdr->status != 0) return;
-    const u32 n_pieces = hdr->n_pieces;
-    const u32 lane = threadIdx.x & 31;
-    const u32 stride = gridDim.x * blockDim.x;
-    const u32 rounds = (n_pieces + stride - 1) / stride;
-    u32 p = blockIdx.x * blockDim.x + threadIdx.x;
-    for (u32 it = 0; it < rounds; it++, p += stride) {
-        bool miss = false;
-        if (p < n_pieces) {
-            const u32 a = piece_off[p], n = piece_off[p + 1] - a;
-            if (n == 1) {
-                stage[a] = ext_id[text[a]]; piece_cnt[p] = 1;
-            } else if (n > TT_TOKTAB_MAXLEN || tab.slots == nullptr) {
-                miss = true;
-            } else {
-                // gather the piece's bytes with aligned 8-byte loads (only words that hold a piece byte)
-                const uintptr_t addr = (uintptr_t)(text + a);
-                const u64* w = reinterpret_cast<const u64*>(addr & ~(uintptr_t)7);
-                const u32 sh = (u32)(addr & 7) * 8, last = (u32)(addr & 7) + n;     // bytes used in the window
-                const u64 w0 = __ldg(w), w1 = last > 8 ? __ldg(w + 1) : 0, w2 = last > 16 ? __ldg(w + 2) : 0,
-                          w3 = last > 24 ? __ldg(w + 3) : 0;
-                u64 k0 = sh ? (w0 >> sh) | (w1 << (64 - sh)) : w0;
-                u64 k1 = sh ? (w1 >> sh) | (w2 << (64 - sh)) : w1;
-                u64 k2 = sh ? (w2 >> sh) | (w3 << (64 - sh)) : w2;
-                if (n < 8) { k0 &= (1ull << (8 * n)) - 1; k1 = 0; k2 = 0; }
-                else if (n < 16) { k1 &= (n == 8) ? 0 : ((1ull << (8 * (n - 8))) - 1); k2 = 0; }
-                else if (n < 24) { k2 &= (n == 16) ? 0 : ((1ull << (8 * (n - 16))) - 1); }
-                u32 h = toktab_hash(k0, k1, k2, n, tab.shift);
-                miss = true;
-                for (u32 probe = 0; probe <= tab.mask; probe++) {           // bounded by the capacity
-                    const uint4* sp = reinterpret_cast<const uint4*>(tab.slots + h);
-                    const uint4 lo = __ldg(sp), hi = __ldg(sp + 1);
-                    const u32 slen = hi.z;
-                    if (slen == 0) break;
-                    if (slen == n && (((u64)lo.y << 32) | lo.x) == k0 && (((u64)lo.w << 32) | lo.z) == k1 &&
-                        (((u64)hi.y << 32) | hi.x) == k2) {
-                        stage[a] = (int32_t)hi.w; piece_cnt[p] = 1; miss = false; break;
-                    }
-                    h = (h + 1) & tab.mask;
-                }
-            }
+// Looks a piece of 2..24 bytes up; returns true and the id on a hit.
+__device__ __forceinline__ bool toktab_lookup(const TokTable& tab, const u8* __restrict__ text, u32 a, u32 n, int32_t& id) {
+    // gather the piece's bytes with aligned 8-byte loads (only words that hold a piece byte)
+    const uintptr_t addr = (uintptr_t)(text + a);
+    const u64* w = reinterpret_cast<const u64*>(addr & ~(uintptr_t)7);
+    const u32 sh = (u32)(addr & 7) * 8, last = (u32)(addr & 7) + n;     // bytes used in the window
+    const u64 w0 = __ldg(w), w1 = last > 8 ? __ldg(w + 1) : 0, w2 = last > 16 ? __ldg(w + 2) : 0, w3 = last > 24 ? __ldg(w + 3) : 0;
+    u64 k0 = sh ? (w0 >> sh) | (w1 << (64 - sh)) : w0;
+    u64 k1 = sh ? (w1 >> sh) | (w2 << (64 - sh)) : w1;
+    u64 k2 = sh ? (w2 >> sh) | (w3 << (64 - sh)) : w2;
+    if (n < 8) { k0 &= (1ull << (8 * n)) - 1; k1 = 0; k2 = 0; }
+    else if (n < 16) { k1 &= (n == 8) ? 0 : ((1ull << (8 * (n - 8))) - 1); k2 = 0; }
+    else if (n < 24) { k2 &= (n == 16) ? 0 : ((1ull << (8 * (n - 16))) - 1); }
+    u32 h = toktab_hash(k0, k1, k2, n, tab.shift);
+    for (u32 probe = 0; probe <= tab.mask; probe++) {           // bounded by the capacity
+        const uint4* sp = reinterpret_cast<const uint4*>(tab.slots + h);
+        const uint4 lo = __ldg(sp), hi = __ldg(sp + 1);
+        if (hi.z == 0) return false;
+        if (hi.z == n && (((u64)lo.y << 32) | lo.x) == k0 && (((u64)lo.w << 32) | lo.z) == k1 && (((u64)hi.y << 32) | hi.x) == k2) {
+            id = (int32_t)hi.w;
+            return true;
         }
-        const u32 mm = __ballot_sync(0xFFFFFFFFu, miss);
-        if (mm) {
-            u32 base = 0;
-            if (lane == 0) base = atomicAdd(&hdr->n_miss, (u32)__popc(mm));
-            base = __shfl_sync(0xFFFFFFFFu, base, 0);
-            if (miss) miss_list[base + __popc(mm & ((1u << lane) - 1))] = p;
-        }
+        h = (h + 1) & tab.mask;
     }
+    return false;
 }
 
 constexpr u32 RK_STALE = 0xFFFFFFFEu;                 // rank must be probed again
-constexpr int BPE_WARPS = 8;                          // warps per CTA of the warp-per-piece kernel
+constexpr int BPE_WARPS = 8;                          // warps per CTA of the piece kernels
+constexpr int BPE_THREADS = BPE_WARPS * 32;           // = pieces per CTA iteration
 constexpr int WCH = TT_WARP_PIECE_MAX / 32;           // 32-token chunks per piece
 
-// ---- K4, warp per piece ---------------------------------------------------------------------------
-__global__ void __launch_bounds__(BPE_WARPS * 32)
-k_bpe_warp(const u8* __restrict__ text, const u32* __restrict__ piece_off, TTHeader* hdr, const PairTable tab,
-           const int32_t* __restrict__ ext_id, u32* __restrict__ piece_cnt, int32_t* __restrict__ stage,
-           u32* __restrict__ long_list, const u32* __restrict__ miss_list) {
-    __shared__ u32 s_tok[BPE_WARPS][TT_WARP_PIECE_MAX];
-    __shared__ u32 s_rk[BPE_WARPS][TT_WARP_PIECE_MAX];
-    if (hdr->status != 0) return;
-    // with a miss list: the pieces the lookup kernel could not settle; without: every piece
-    const u32 n_items = miss_list ? hdr->n_miss : hdr->n_pieces;
-    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
-    const u32 lt = (1u << lane) - 1;
-    u32* tok = s_tok[wid];
-    u32* rk = s_rk[wid];
-    const u32 nwarps = gridDim.x * BPE_WARPS;
-    for (u32 item = blockIdx.x * BPE_WARPS + wid; item < n_items; item += nwarps) {
-        const u32 p = miss_list ? miss_list[item] : item;
-        const u32 a = piece_off[p], n = piece_off[p + 1] - a;
-        if (n > TT_WARP_PIECE_MAX) {
-            if (lane == 0) long_list[atomicAdd(&hdr->n_long, 1u)] = p;
-            continue;
-        }
-        if (n == 1) {
-            if (lane == 0) { stage[a] = ext_id[text[a]]; piece_cnt[p] = 1; }
-            continue;
-        }
-        __syncwarp();
-        for (u32 k = lane; k < n; k += 32) tok[k] = text[a + k];
-        __syncwarp();
-        for (u32 k = lane; k < n; k += 32) rk[k] = (k + 1 < n) ? pair_probe(tab, tok[k], tok[k + 1]) : TT_RANK_INF;
-        u32 m = n;
-        for (u32 round = 0; round < n; round++) {      // at most n - 1 merges
-            __syncwarp();
-            const int nch = (int)((m + 31) >> 5);
-            u32 t[WCH], r[WCH];
-            u32 mn = TT_RANK_INF;
-#pragma unroll
-            for (int j = 0; j < WCH; j++) {
-                if (j < nch) {
-                    const u32 k = j * 32 + lane;
-                    t[j] = k < m ? tok[k] : 0;
-                    r[j] = k < m ? rk[k] : TT_RANK_INF;
-                    mn = min(mn, r[j]);
-                }
-            }
-            mn = __reduce_min_sync(0xFFFFFFFFu, mn);
-            if (mn == TT_RANK_INF) break;
-            // candidates, then leftmost non-overlapping selection: inside a maximal run of
-            // consecutive candidates take the positions at even distance from the run start
-            u32 sel[WCH];
-            u32 prev_ones = 0;                          // length of the candidate run that ends at the previous chunk's top
-#pragma unroll
-            for (int j = 0; j < WCH; j++) {
-                if (j < nch) {
-                    const u32 c = __ballot_sync(0xFFFFFFFFu, r[j] == mn);
-                    const u32 below = ~c & lt;
-                    const u32 dist = below ? (u32)(lane - (32 - __clz(below))) : (u32)lane + prev_ones;
-                    sel[j] = __ballot_sync(0xFFFFFFFFu, ((c >> lane) & 1) && !(dist & 1));
-                    prev_ones = (c == 0xFFFFFFFFu) ? prev_ones + 32 : (u32)__clz(~c);
-                }
-            }
-            __syncwarp();
-            // compaction in place: every lane has read its elements; survivors move down
-            u32 removed = 0;
-#pragma unroll
-            for (int j = 0; j < WCH; j++) {
-                if (j < nch) {
-                    const u32 k = j * 32 + lane;
-                    const u32 s = sel[j];
-                    const bool me = (s >> lane) & 1;
-                    const bool gone = lane ? ((s >> (lane - 1)) & 1) : (j ? (sel[j - 1] >> 31) & 1 : 0);
-                    const bool next_sel = lane < 31 ? ((s >> (lane + 1)) & 1) : ((j + 1 < nch) ? (sel[j + 1] & 1) : 0);
-                    if (k < m && !gone) {
-                        const u32 np = k - removed - __popc(s & lt);
-                        tok[np] = me ? 256u + mn : t[j];
-                        rk[np] = (me || next_sel) ? RK_STALE : r[j];
-                    }
-                    removed += __popc(s);
-                }
-            }
-            m -= removed;
-            __syncwarp();
-            for (u32 k = lane; k < m; k += 32)
-                if (rk[k] == RK_STALE) rk[k] = (k + 1 < m) ? pair_probe(tab, tok[k], tok[k + 1]) : TT_RANK_INF;
-        }
-        __syncwarp();
-        for (u32 k = lane; k < m; k += 32) stage[a + k] = ext_id[tok[k]];
-        if (lane == 0) piece_cnt[p] = m;
+// ---- warp merge, up to 32 bytes: one token per lane, no shared memory ------------------------------------
+// Returns the token count; the tokens (caller's ids) are staged at stage[a ...].
+__device__ __forceinline__ u32 warp_merge_reg(const u8* __restrict__ text, u32 a, u32 n, const PairTable& tab,
+                                              const int32_t* __restrict__ ext_id, int32_t* __restrict__ stage, int lane) {
+    const u32 FULL = 0xFFFFFFFFu, lt = (1u << lane) - 1;
+    u32 t = (u32)lane < n ? text[a + lane] : 0;
+    u32 m = n;
+    u32 tn = __shfl_down_sync(FULL, t, 1);
+    u32 r = ((u32)lane + 1 < m) ? pair_probe(tab, t, tn) : TT_RANK_INF;
+    for (u32 round = 0; round < n; round++) {          // at most n - 1 merges
+        const u32 mn = __reduce_min_sync(FULL, r);
+        if (mn == TT_RANK_INF) break;
+        // leftmost non-overlapping occurrences: inside a run of consecutive candidates, every other one
+        const u32 c = __ballot_sync(FULL, r == mn);
+        const u32 below = ~c & lt;
+        const u32 dist = below ? (u32)(lane - (32 - __clz(below))) : (u32)lane;
+        const u32 sel = __ballot_sync(FULL, ((c >> lane) & 1) && !(dist & 1));
+        const bool me = (sel >> lane) & 1;
+        const bool nxt = lane < 31 ? ((sel >> (lane + 1)) & 1) : false;
+        const u32 nt = me ? 256u + mn : t;
+        const u32 nr = (me || nxt) ? RK_STALE : r;
+        // survivors move down: new lane j takes the j-th surviving old lane
+        const u32 surv = ~(sel << 1) & (m >= 32 ? FULL : ((1u << m) - 1));
+        const u32 src = __fns(surv, 0, lane + 1);
+        t = __shfl_sync(FULL, nt, src & 31);
+        r = __shfl_sync(FULL, nr, src & 31);
+        m -= __popc(sel);
+        tn = __shfl_down_sync(FULL, t, 1);
+        if ((u32)lane + 1 >= m) r = TT_RANK_INF;
+        else if (r == RK_STALE) r = pair_probe(tab, t, tn);
     }
+    if ((u32)lane < m) stage[a + lane] = ext_id[t];
+    return m;
 }
 
-// ---- K4, CTA per long piece (long whitespace / punctuation runs and other pieces > 256 bytes) -----
-constexpr int LONG_THREADS = 1024;
-constexpr u32 TOK_NEW = 0x80000000u;                  // token produced in the current round
+// ---- warp merge, 33..256 bytes: E tokens per lane in registers, compaction through shared memory ---------
+// Position k lives in lane k % 32, register k / 32.  Each round the surviving (token, rank) pairs are
+// written to their new positions in one of two shared-memory buffers (alternating, so one warp barrier
+// per round suffices) and read back; ranks next to a merge are marked stale and probed again.
+template <int E>
+__device__ __forceinline__ u32 warp_merge_perm(u64* buf /* 2 * 32 * E entries of this warp */, const u8* __restrict__ text,
+                                               u32 a, u32 n, const PairTable& tab, const int32_t* __restrict__ ext_id,
+                                               int32_t* __restrict__ stage, int lane) {
+    const u32 FULL = 0xFFFFFFFFu, lt = (1u << lane) - 1;
+    u32 t[E], r[E];
+    u32 m = n;
+    __syncwarp();
+#pragma unroll
+    for (int j = 0; j < E; j++) {
+        const u32 k = j * 32 + lane;
+        t[j] = k < n ? text[a + k] : 0;
+        buf[k] = t[j];
+    }
+    __syncwarp();
+#pragma unroll
+    for (int j = 0; j < E; j++) {
+        const u32 k = j * 32 + lane;
+        r[j] = (k + 1 < n) ? pair_probe(tab, t[j], (u32)buf[k + 1]) : TT_RANK_INF;
+    }
+    int cur = 0;
+    for (u32 round = 0; round < n; round++) {          // at most n - 1 merges
+        u32 mn = r[0];
+#pragma unroll
+        for (int j = 1; j < E; j++) mn = min(mn, r[j]);
+        mn = __reduce_min_sync(FULL, mn);
+        if (mn == TT_RANK_INF) break;
+        const int nch = (int)((m + 31) >> 5);
+        u32 sel[E];
+        u32 prev_ones = 0;                              // candidate run ending at the top of the previous word
+#pragma unroll
+        for (int j = 0; j < E; j++) {
+            sel[j] = 0;
+            if (j < nch) {
+                const u32 c = __ballot_sync(FULL, r[j] == mn);
+                const u32 below = ~c & lt;
+                const u32 dist = below ? (u32)(lane - (32 - __clz(below))) : (u32)lane + prev_ones;
+                sel[j] = __ballot_sync(FULL, ((c >> lane) & 1) && !(dist & 1));
+                prev_ones = (c == FULL) ? prev_ones + 32 : (u32)__clz(~c);
+            }
+        }
+        u64* nb = buf + (cur ^ 1) * (32 * E);
+        u32 removed = 0;
+#pragma unroll
+        for (int j = 0; j < E; j++) {
+            if (j < nch) {
+                const u32 k = j * 32 + lane;
+                const u32 s = sel[j];
+                const bool me = (s >> lane) & 1;
+                const bool gone = lane ? ((s >> (lane - 1)) & 1) : (j ? (sel[j > 0 ? j - 1 : 0] >> 31) & 1 : 0);
+                const bool next_sel = lane < 31 ? ((s >> (lane + 1)) & 1) : ((j + 1 < E) ? (sel[j + 1 < E ? j + 1 : j] & 1) : 0);
+                if (k < m && !gone) {
+                    const u32 np = k - removed - __popc(s & lt);
+                    nb[np] = ((u64)((me || next_sel) ? RK_STALE : r[j]) << 32) | (me ? 256u + mn : t[j]);
+                }
+                removed += __popc(s);
+            }
+        }
+        m -= removed;
+        cur ^= 1;
+        __syncwarp();
+#pragma unroll
+        for (int j = 0; j < E; j++) {
+            const u32 k = j * 32 + lane;
+            r[j] = TT_RANK_INF;
+            if (k < m) {
+                const u64 v = nb[k];
+                t[j] = (u32)v;
+                r[j] = (u32)(v >> 32);
+                if (k + 1 >= m) r[j] = TT_RANK_INF;
+                else if (r[j] == RK_STALE) r[j] = pair_probe(tab, t[j], (u32)nb[k + 1]);
+            }
+        }
+    }
+#pragma unroll
+    for (int j = 0; j < E; j++) {
+        const u32 k = j * 32 + lane;
+        if (k < m) stage[a + k] = ext_id[t[j]];
+    }
+    return m;
+}
 
+// ---- CTA-wide scans -----------------------------------------------------------------------------------
 __device__ __forceinline__ int cta_incl_max_scan(int v, int* scratch /* >= 33 */, int carry) {
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5, nw = blockDim.x >> 5;
     for (int o = 1; o < 32; o <<= 1) { int t = __shfl_up_sync(0xFFFFFFFFu, v, o); if (lane >= o) v = max(v, t); }
@@ -236,6 +246,84 @@ __device__ __forceinline__ u32 cta_excl_sum_scan(u32 v, u32* scratch /* >= 33 */
     *total = scratch[32];
     return scratch[wid] + x - v;
 }
+
+// ---- K4, pieces of a block of BPE_THREADS consecutive pieces ---------------------------------------------
+// Phase 1: a thread per piece (one-byte pieces map directly, pieces of up to 24 bytes are looked up as
+// whole vocabulary entries).  Phase 2: the CTA's warps merge the pieces phase 1 could not settle.
+// Phase 3: the token total of the block; the last CTA to finish turns the block totals into their
+// exclusive prefix (K5's scan) and checks the output capacity.  Pieces longer than
+// TT_WARP_PIECE_MAX were encoded before this kernel (k_bpe_long); only their counts are read here.
+// Without a token table (while the table itself is being built) every piece takes the merge path.
+__global__ void __launch_bounds__(BPE_THREADS)
+k_bpe_pieces(const u8* __restrict__ text, const u32* __restrict__ piece_off, TTHeader* hdr, const PairTable tab,
+             const TokTable toktab, const int32_t* __restrict__ ext_id, u32* __restrict__ piece_cnt,
+             int32_t* __restrict__ stage, u32* __restrict__ blk_cnt, unsigned long long ids_cap) {
+    __shared__ u64 s_buf[BPE_WARPS][2 * TT_WARP_PIECE_MAX];     // two (token, rank) buffers per warp
+    __shared__ u32 s_miss[BPE_THREADS];
+    __shared__ u32 s_nmiss, s_total, s_islast;
+    __shared__ u32 sc[40];
+    const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+    const bool dead = hdr->status != 0;
+    const u32 n_pieces = dead ? 0 : hdr->n_pieces;
+    const u32 n_blocks = (n_pieces + BPE_THREADS - 1) / BPE_THREADS;
+    for (u32 pb = blockIdx.x; pb < n_blocks; pb += gridDim.x) {
+        __syncthreads();
+        if (tid == 0) { s_nmiss = 0; s_total = 0; }
+        __syncthreads();
+        const u32 p = pb * BPE_THREADS + tid;
+        u32 cnt = 0;
+        if (p < n_pieces) {
+            const u32 a = piece_off[p], n = piece_off[p + 1] - a;
+            int32_t id;
+            if (n == 1) { stage[a] = ext_id[text[a]]; cnt = 1; }
+            else if (n > TT_WARP_PIECE_MAX) cnt = piece_cnt[p];
+            else if (n <= TT_TOKTAB_MAXLEN && toktab.slots != nullptr && toktab_lookup(toktab, text, a, n, id)) { stage[a] = id; cnt = 1; }
+            else s_miss[atomicAdd(&s_nmiss, 1u)] = p;
+            if (cnt && n <= TT_WARP_PIECE_MAX) piece_cnt[p] = cnt;
+        }
+        u32 wsum = cnt;
+        for (int o = 16; o; o >>= 1) wsum += __shfl_xor_sync(0xFFFFFFFFu, wsum, o);
+        __syncthreads();
+        const u32 nmiss = s_nmiss;
+        u32 msum = 0;
+        for (u32 e = wid; e < nmiss; e += BPE_WARPS) {
+            const u32 q = s_miss[e];
+            const u32 a = piece_off[q], n = piece_off[q + 1] - a;
+            const u32 m = n <= 32 ? warp_merge_reg(text, a, n, tab, ext_id, stage, lane)
+                        : n <= 64 ? warp_merge_perm<2>(s_buf[wid], text, a, n, tab, ext_id, stage, lane)
+                                  : warp_merge_perm<WCH>(s_buf[wid], text, a, n, tab, ext_id, stage, lane);
+            if (lane == 0) piece_cnt[q] = m;
+            msum += m;
+        }
+        if (lane == 0) atomicAdd(&s_total, wsum + msum);
+        __syncthreads();
+        if (tid == 0) blk_cnt[pb] = s_total;
+    }
+    // the last CTA to finish: exclusive prefix of the block totals, total token count, capacity check
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) s_islast = (atomicAdd(&hdr->count_done, 1u) == gridDim.x - 1);
+    __syncthreads();
+    if (!s_islast) return;
+    __threadfence();
+    unsigned long long carry = 0;
+    for (u32 b0 = 0; b0 < n_blocks; b0 += BPE_THREADS) {
+        const u32 i = b0 + tid;
+        u32 x = i < n_blocks ? blk_cnt[i] : 0, t2;
+        const u32 ex = cta_excl_sum_scan(x, sc, &t2);
+        if (i < n_blocks) blk_cnt[i] = (u32)carry + ex;
+        carry += t2;
+        __syncthreads();
+    }
+    if (tid == 0) {
+        hdr->n_tokens = carry;
+        if (!dead && carry > ids_cap) atomicMax(&hdr->status, 5 /* TT_ERR_CAPACITY */);
+    }
+}
+
+// ---- K4, CTA per long piece (long whitespace / punctuation runs and other pieces > 256 bytes) -----
+constexpr int LONG_THREADS = 1024;
+constexpr u32 TOK_NEW = 0x80000000u;                  // token produced in the current round
 
 __global__ void __launch_bounds__(LONG_THREADS)
 k_bpe_long(const u8* __restrict__ text, const u32* __restrict__ piece_off, TTHeader* hdr, const PairTable tab,
@@ -316,48 +404,15 @@ k_bpe_long(const u8* __restrict__ text, const u32* __restrict__ piece_off, TTHea
     }
 }
 
-// ---- K5a: token counts per block of pieces, then their exclusive prefix ---------------------------
-constexpr int CNT_THREADS = 1024;
-
-__global__ void __launch_bounds__(CNT_THREADS)
-k_count(const u32* __restrict__ piece_cnt, TTHeader* hdr, u32* __restrict__ blk_cnt, unsigned long long ids_cap) {
-    __shared__ u32 sc[40];
-    __shared__ u32 s_islast;
-    const u32 n_pieces = hdr->n_pieces;
-    const bool dead = hdr->status != 0;
-    const u32 p = blockIdx.x * CNT_THREADS + threadIdx.x;
-    u32 v = (!dead && p < n_pieces) ? piece_cnt[p] : 0, tot;
-    cta_excl_sum_scan(v, sc, &tot);
-    if (threadIdx.x == 0) blk_cnt[blockIdx.x] = tot;
-    __threadfence();
-    __syncthreads();
-    if (threadIdx.x == 0) s_islast = (atomicAdd(&hdr->count_done, 1u) == gridDim.x - 1);
-    __syncthreads();
-    if (!s_islast) return;
-    __threadfence();
-    const u32 nblk = gridDim.x;
-    unsigned long long carry = 0;
-    for (u32 b0 = 0; b0 < nblk; b0 += CNT_THREADS) {
-        const u32 i = b0 + threadIdx.x;
-        u32 x = i < nblk ? blk_cnt[i] : 0, t2;
-        const u32 ex = cta_excl_sum_scan(x, sc, &t2);
-        if (i < nblk) blk_cnt[i] = (u32)carry + ex;
-        carry += t2;
-        __syncthreads();
-    }
-    if (threadIdx.x == 0) {
-        hdr->n_tokens = carry;
-        if (!dead && carry > ids_cap) atomicMax(&hdr->status, 5 /* TT_ERR_CAPACITY */);
-    }
-}
-
-// ---- K5b: token offsets per piece and coalesced scatter of the staged ids --------------------------
-__global__ void __launch_bounds__(CNT_THREADS)
+// ---- K5: token offsets per piece and coalesced scatter of the staged ids ----------------------------------
+// One CTA per block of BPE_THREADS pieces (the same partition as k_bpe_pieces, whose last CTA left the
+// exclusive prefix of the block totals in blk_base).
+__global__ void __launch_bounds__(BPE_THREADS)
 k_scatter(const u32* __restrict__ piece_off, const u32* __restrict__ piece_cnt, const u32* __restrict__ blk_base,
           const int32_t* __restrict__ stage, TTHeader* hdr, u32* __restrict__ tok_off, int32_t* __restrict__ ids_out,
           long long* __restrict__ count_out, int32_t* __restrict__ status_out) {
     __shared__ u32 sc[40];
-    __shared__ u32 s_big[CNT_THREADS][3];
+    __shared__ u32 s_big[BPE_THREADS][3];
     __shared__ u32 s_nbig;
     const int status = hdr->status;
     const u32 n_pieces = hdr->n_pieces;
@@ -367,27 +422,31 @@ k_scatter(const u32* __restrict__ piece_off, const u32* __restrict__ piece_cnt, 
         if (status || n_pieces == 0) tok_off[0] = 0;
     }
     if (status != 0) return;
-    if (threadIdx.x == 0) s_nbig = 0;
-    const u32 p = blockIdx.x * CNT_THREADS + threadIdx.x;
-    const u32 c = p < n_pieces ? piece_cnt[p] : 0;
-    u32 tot;
-    const u32 dst = blk_base[blockIdx.x] + cta_excl_sum_scan(c, sc, &tot);
-    if (p < n_pieces) {
-        tok_off[p] = dst;
-        if (p == n_pieces - 1) tok_off[n_pieces] = dst + c;
-        const u32 src = piece_off[p];
-        if (c <= 8) {
-            for (u32 k = 0; k < c; k++) ids_out[dst + k] = stage[src + k];
-        } else {
-            const u32 slot = atomicAdd(&s_nbig, 1u);
-            s_big[slot][0] = src; s_big[slot][1] = dst; s_big[slot][2] = c;
+    const u32 n_blocks = (n_pieces + BPE_THREADS - 1) / BPE_THREADS;
+    for (u32 pb = blockIdx.x; pb < n_blocks; pb += gridDim.x) {
+        __syncthreads();
+        if (threadIdx.x == 0) s_nbig = 0;
+        const u32 p = pb * BPE_THREADS + threadIdx.x;
+        const u32 c = p < n_pieces ? piece_cnt[p] : 0;
+        u32 tot;
+        const u32 dst = blk_base[pb] + cta_excl_sum_scan(c, sc, &tot);
+        if (p < n_pieces) {
+            tok_off[p] = dst;
+            if (p == n_pieces - 1) tok_off[n_pieces] = dst + c;
+            const u32 src = piece_off[p];
+            if (c <= 8) {
+                for (u32 k = 0; k < c; k++) ids_out[dst + k] = stage[src + k];
+            } else {
+                const u32 slot = atomicAdd(&s_nbig, 1u);
+                s_big[slot][0] = src; s_big[slot][1] = dst; s_big[slot][2] = c;
+            }
         }
-    }
-    __syncthreads();
-    const u32 nbig = s_nbig;
-    for (u32 e = 0; e < nbig; e++) {
-        const u32 src = s_big[e][0], d2 = s_big[e][1], cc = s_big[e][2];
-        for (u32 k = threadIdx.x; k < cc; k += CNT_THREADS) ids_out[d2 + k] = stage[src + k];
+        __syncthreads();
+        const u32 nbig = s_nbig;
+        for (u32 e = 0; e < nbig; e++) {
+            const u32 src = s_big[e][0], d2 = s_big[e][1], cc = s_big[e][2];
+            for (u32 k = threadIdx.x; k < cc; k += BPE_THREADS) ids_out[d2 + k] = stage[src + k];
+        }
     }
 }
 

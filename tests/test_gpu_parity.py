@@ -215,3 +215,37 @@ def test_result_does_not_depend_on_schedule():
         torch.cuda.synchronize()
         outs.append(bufs["ids"][:int(bufs["count"].item())].cpu().numpy().copy())
     assert np.array_equal(outs[0], outs[1]) and np.array_equal(outs[0], outs[2])
+
+
+def test_full_size_c4_ids_and_pieces():
+    """The whole 3,000,000-char adversarial request of config C4 (pattern 1, 199,744 merges)."""
+    cfg = wl.CONFIGS["C4"]
+    text = wl.request(cfg)
+    got, status = gpu_pretok(gpu_vocab("C4"), text)
+    assert status == 0 and np.array_equal(got, _expect_pieces(text, 1))
+    ids, status = gpu_encode(gpu_vocab("C4"), text)
+    want, _ = cpu_vocab("C4").encode(text, 1, nthreads=8)
+    assert status == 0 and ids.size == want.size and np.array_equal(ids, want)
+
+
+def test_full_size_c5_batch_sampled_documents():
+    """One tt_encode_batch call over the full 256-request batch of config C5, in the configuration the
+    benchmark times; a sample of documents is compared with the oracle element by element, every
+    document through properties that hold at any size."""
+    cfg = wl.CONFIGS["C5"]
+    text, off = wl.batch(cfg)
+    ids, ioff, status = gpu_encode_batch(gpu_vocab("C5"), text, off)
+    assert status == 0
+    assert ioff[0] == 0 and np.all(np.diff(ioff) > 0) and ioff[-1] == ids.size
+    assert np.all(np.diff(ioff) <= np.diff(off))                      # a token covers at least one byte
+    assert ids.min() >= 0 and ids.max() < 256 + cfg.n_merges
+    cv = cpu_vocab("C5")
+    lens = np.diff(off)
+    sample = sorted({0, 255, int(np.argmin(lens)), int(np.argmax(lens)), 17, 101, 200})
+    for d in sample:
+        want, _ = cv.encode(text[off[d]:off[d + 1]], cfg.pattern_id, nthreads=8)
+        got = ids[ioff[d]:ioff[d + 1]]
+        assert got.size == want.size and np.array_equal(got, want), f"document {d}"
+    # decode(encode(x)) == x on one further document, through the vocabulary's byte strings
+    d = 64
+    assert cv.decode(ids[ioff[d]:ioff[d + 1]][:2000]) == text[off[d]:off[d + 1]].tobytes()[:len(cv.decode(ids[ioff[d]:ioff[d + 1]][:2000]))]

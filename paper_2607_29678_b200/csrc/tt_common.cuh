@@ -19,10 +19,10 @@ typedef uint64_t u64;
 // A chunk is one aligned 16-byte vector load; a tile is what one CTA classifies per iteration.
 constexpr int TT_CHUNK = 16;
 #ifndef TT_TILE_CHUNKS_DEF
-#define TT_TILE_CHUNKS_DEF 256
+#define TT_TILE_CHUNKS_DEF 128
 #endif
 constexpr int TT_TILE_CHUNKS = TT_TILE_CHUNKS_DEF;        // = threads per CTA
-constexpr int TT_TILE_BYTES = TT_CHUNK * TT_TILE_CHUNKS; // 4 KiB of text per tile
+constexpr int TT_TILE_BYTES = TT_CHUNK * TT_TILE_CHUNKS; // 2 KiB of text per tile
 
 // ---- character class codes (two-stage Unicode table, see gen_unicode_table.py) ------------
 enum : u32 { CC_OTHER = 0, CC_MARK = 1, CC_SPACE = 2, CC_NUMBER = 3, CC_LOWER = 4, CC_UPPER = 5, CC_CASELESS = 6 };

@@ -204,8 +204,12 @@ k_pretok(const PretokParams P) {
     __shared__ u32 s_islast;
 
     const int tid = threadIdx.x;
+    // the 128-byte ASCII table is always staged; the two-stage Unicode table only once a tile holds a
+    // non-ASCII byte (pattern 1 stages it at once: its sparse matcher may read beyond the tile)
+    bool tables_loaded = P.pattern != 0;
     for (int i = tid * 16; i < P.cls_bytes; i += blockDim.x * 16)
-        *reinterpret_cast<uint4*>(tables + i) = *reinterpret_cast<const uint4*>(P.cls_tables + i);
+        if (tables_loaded || i >= P.cls_bytes - 128)
+            *reinterpret_cast<uint4*>(tables + i) = *reinterpret_cast<const uint4*>(P.cls_tables + i);
     ClassTables T;
     T.stage1 = tables; T.stage2 = tables + 0x1100; T.ascii = tables + P.cls_bytes - 128;
     SeqCtx SC;
@@ -216,6 +220,29 @@ k_pretok(const PretokParams P) {
         __syncthreads();
         if (tid == 0) s_need = 0;
         const long long c_first = (long long)tile * TT_TILE_CHUNKS;
+        if (!tables_loaded) {                                         // block-uniform
+            bool hi_bit = false;
+            {
+                const long long chunk = c_first + tid;
+                if (chunk >= 0 && chunk < P.nchunks) {
+                    const uint4 v = *reinterpret_cast<const uint4*>(P.base + chunk * TT_CHUNK);
+                    hi_bit = ((v.x | v.y | v.z | v.w) & 0x80808080u) != 0;
+                }
+            }
+            if (tid < TT_LOW_HALO + 1) {
+                const long long chunk = tid < TT_LOW_HALO ? c_first - TT_LOW_HALO + tid : c_first + TT_TILE_CHUNKS;
+                if (chunk >= 0 && chunk < P.nchunks) {
+                    const uint4 v = *reinterpret_cast<const uint4*>(P.base + chunk * TT_CHUNK);
+                    hi_bit = hi_bit || ((v.x | v.y | v.z | v.w) & 0x80808080u) != 0;
+                }
+            }
+            if (__syncthreads_or(hi_bit)) {
+                for (int i = tid * 16; i < P.cls_bytes - 128; i += blockDim.x * 16)
+                    *reinterpret_cast<uint4*>(tables + i) = *reinterpret_cast<const uint4*>(P.cls_tables + i);
+                tables_loaded = true;
+                __syncthreads();
+            }
+        }
         // phase A: classify own chunk (+ the halo chunks)
         {
             const long long chunk = c_first + tid;
@@ -230,6 +257,13 @@ k_pretok(const PretokParams P) {
             store_slot(sm, s, tt_classify_chunk(P.base, chunk, P.nchunks, P.lo, P.hi, T), doc_bits(P, chunk));
         }
         __syncthreads();
+        if (P.pattern != 0) {                                          // sure starts / unresolved constructs per slot
+            u32 su, ha;
+            tt_sure_hard(sm, tid + TT_LOW_HALO, su, ha);
+            sm[F_SURE][tid + TT_LOW_HALO] = (u16)su; sm[F_HARD][tid + TT_LOW_HALO] = (u16)ha;
+            if (tid >= 1 && tid < TT_LOW_HALO) { tt_sure_hard(sm, tid, su, ha); sm[F_SURE][tid] = (u16)su; sm[F_HARD][tid] = (u16)ha; }
+            __syncthreads();
+        }
         // phase B: evaluate the piece-start predicate
         TileCarry tc;
         tc.n_before = 0; tc.nl_absorbed_before = 0; tc.nl_later_after = 0; tc.slash_absorbed_before = 0;
@@ -243,6 +277,12 @@ k_pretok(const PretokParams P) {
         __syncthreads();
         const u32 need_all = s_need;
         if (need_all) {                                               // block-uniform
+            if (!tables_loaded) {                                     // the walks below classify text outside the tile
+                for (int i = tid * 16; i < P.cls_bytes - 128; i += blockDim.x * 16)
+                    *reinterpret_cast<uint4*>(tables + i) = *reinterpret_cast<const uint4*>(P.cls_tables + i);
+                tables_loaded = true;
+                __syncthreads();
+            }
             const long long below = (c_first - TT_LOW_HALO) * TT_CHUNK;    // first byte of the low halo
             if (need_all & NEED_N) tc.n_before = coop_back_num(P, T, below, scratch);
             if (need_all & NEED_A) tc.nl_absorbed_before = coop_back_nl(P, T, below, scratch);

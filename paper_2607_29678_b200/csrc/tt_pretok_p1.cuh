@@ -178,11 +178,12 @@ TT_HD void tt_sure_hard(const u16 (*sm)[TT_SLOTS], int s, u32& sure, u32& hard) 
     tt_sure_hard_cm(tt_load_slot(sm, s - 1), tt_load_slot(sm, s), tt_load_slot(sm, s + 1), sure, hard);
 }
 
-// Walks down from slot s: is the nearest sure-start / unresolved-construct event an unresolved one?
+// Walks down from slot s over the precomputed F_SURE / F_HARD masks (valid for slots >= 1): is the
+// nearest sure-start / unresolved-construct event an unresolved one?
 TT_HD u32 tt_walk_back_dirty(const u16 (*sm)[TT_SLOTS], int s, bool& open) {
     open = false;
     for (; s >= 1; s--) {
-        u32 c, h; tt_sure_hard(sm, s, c, h);
+        const u32 c = sm[F_SURE][s], h = sm[F_HARD][s];
         if (c | h) { int b = tt_hibit(c | h); return (h >> b) & 1; }
     }
     open = true;
@@ -191,7 +192,7 @@ TT_HD u32 tt_walk_back_dirty(const u16 (*sm)[TT_SLOTS], int s, bool& open) {
 // Walks down from slot s: position (slot * 16 + bit) of the nearest sure start, or -1 when open.
 TT_HD int tt_walk_back_sure(const u16 (*sm)[TT_SLOTS], int s) {
     for (; s >= 1; s--) {
-        u32 c, h; tt_sure_hard(sm, s, c, h);
+        const u32 c = sm[F_SURE][s];
         if (c) return s * 16 + tt_hibit(c);
     }
     return -1;
@@ -318,9 +319,9 @@ TT_HD u32 tt_eval_chunk_p1(const u16 (*sm)[TT_SLOTS], int slot, const SeqCtx& C,
         }
     }
     // ---- unresolved constructs: propagate from each one up to the next sure start
-    const u64 pLr = PREV(Lr), pN = PREV(N);
-    const u64 sure = (D | (N & ~pN) | (W & (pLr | pN)) | (O & ~AP & (pLr | pN)) | (Lr & (pN | PREV(NL)))) & lead;
-    const u64 hard = (Mk | (upp & PREV(cless)) | (AP & pLr & ((Lr >> 1) & ~(D >> 1)))) & lead;
+    // sure starts / unresolved constructs of slot-1 and of the own slot (filled in after classification)
+    const u64 sure = ((u64)sm[F_SURE][slot - 1] << 16) | ((u64)sm[F_SURE][slot] << 32);
+    const u64 hard = ((u64)sm[F_HARD][slot - 1] << 16) | ((u64)sm[F_HARD][slot] << 32);
     // Window bits 0..15 (slot-2) lack look-back at bit 0, so events there are taken from the walk,
     // which starts at slot-2 and has full neighbour information; propagation runs over bits 16..63.
     u64 dirty;

@@ -1,6 +1,6 @@
 // C ABI of the toktier library (see include/toktier.h).  Host side: argument checks, vocabulary
-// tables, workspace layout and the kernel chain  K1+K2 -> K3 -> K4 (long pieces) -> K4 (all other pieces,
-// with K5's count scan in its last CTA) -> K5 scatter.
+// tables, workspace layout and the kernel chain  k_pretok (K1+K2, tile piece counts) -> k_pieces (K3 per tile in
+// shared memory, K4, K5's count scan in its last CTA) -> k_scatter (K5).
 // Nothing here synchronises with the device except tt_vocab_load and tt_encode_host.
 #include "../../include/toktier.h"
 #include "tt_common.cuh"
@@ -103,25 +103,37 @@ static int build_token_table(tt_vocab* v, const tt_merge* merges, size_t n_merge
     off.push_back((u32)cat.size());
     if (cand.empty()) return TT_OK;
     const size_t nb = cat.size(), np = cand.size();
-    u8* d_text = nullptr; u32 *d_off = nullptr, *d_cnt = nullptr, *d_long = nullptr; int32_t* d_stage = nullptr; TTHeader* d_hdr = nullptr;
-    const size_t nblocks = (np + BPE_THREADS - 1) / BPE_THREADS;
+    // start flags and per-tile piece counts of the concatenation, as k_pretok would leave them
+    const size_t nchunks = (nb + TT_CHUNK - 1) / TT_CHUNK, ntiles = (nchunks + TT_TILE_CHUNKS - 1) / TT_TILE_CHUNKS;
+    std::vector<u16> smask(nchunks + 1, 0);
+    std::vector<u32> tile_base(ntiles + 1, 0);
+    for (size_t i = 0; i < np; i++) { smask[off[i] >> 4] |= (u16)(1u << (off[i] & 15)); tile_base[off[i] / TT_TILE_BYTES + 1]++; }
+    for (size_t t = 0; t < ntiles; t++) tile_base[t + 1] += tile_base[t];
+    u8* d_text = nullptr; u16* d_mask = nullptr; u32 *d_tb = nullptr, *d_cnt = nullptr, *d_tt = nullptr; int32_t* d_stage = nullptr;
+    TTHeader* d_hdr = nullptr;
     TTHeader h; memset(&h, 0, sizeof(h)); h.n_pieces = (u32)np;
     std::vector<u32> cnt(np); std::vector<int32_t> stage(nb);
-    bool ok = cudaMalloc(&d_text, nb + 64) == cudaSuccess && cudaMalloc(&d_off, (np + 1) * sizeof(u32)) == cudaSuccess &&
-              cudaMalloc(&d_cnt, np * sizeof(u32)) == cudaSuccess && cudaMalloc(&d_long, (nblocks + 1) * sizeof(u32)) == cudaSuccess &&
-              cudaMalloc(&d_stage, nb * sizeof(int32_t)) == cudaSuccess && cudaMalloc(&d_hdr, sizeof(TTHeader)) == cudaSuccess;
+    bool ok = cudaMalloc(&d_text, nchunks * TT_CHUNK + 64) == cudaSuccess && cudaMalloc(&d_mask, (nchunks + 1) * sizeof(u16)) == cudaSuccess &&
+              cudaMalloc(&d_tb, (ntiles + 1) * sizeof(u32)) == cudaSuccess && cudaMalloc(&d_tt, (ntiles + 1) * sizeof(u32)) == cudaSuccess &&
+              cudaMalloc(&d_cnt, (np + 1) * sizeof(u32)) == cudaSuccess && cudaMalloc(&d_stage, (nb + 1) * sizeof(int32_t)) == cudaSuccess &&
+              cudaMalloc(&d_hdr, sizeof(TTHeader)) == cudaSuccess;
     ok = ok && cudaMemcpy(d_text, cat.data(), nb, cudaMemcpyHostToDevice) == cudaSuccess;
-    ok = ok && cudaMemcpy(d_off, off.data(), (np + 1) * sizeof(u32), cudaMemcpyHostToDevice) == cudaSuccess;
+    ok = ok && cudaMemcpy(d_mask, smask.data(), (nchunks + 1) * sizeof(u16), cudaMemcpyHostToDevice) == cudaSuccess;
+    ok = ok && cudaMemcpy(d_tb, tile_base.data(), (ntiles + 1) * sizeof(u32), cudaMemcpyHostToDevice) == cudaSuccess;
     ok = ok && cudaMemcpy(d_hdr, &h, sizeof(h), cudaMemcpyHostToDevice) == cudaSuccess;
     if (ok) {
-        TokTable none; none.slots = nullptr; none.mask = 0; none.shift = 0;
-        k_bpe_pieces<<<v->sm_count * 8, BPE_THREADS>>>(d_text, d_off, d_hdr, v->tab, none, v->d_ext_id, d_cnt, d_stage,
-                                                        d_long /* block totals, unused */, ~0ull);
+        PieceParams Q;
+        Q.base = d_text; Q.shift = 0; Q.hi = (long long)nb; Q.nchunks = (long long)nchunks; Q.ntiles = (int)ntiles;
+        Q.startmask = d_mask; Q.tile_base = d_tb; Q.hdr = d_hdr; Q.tab = v->tab;
+        Q.toktab.slots = nullptr; Q.toktab.mask = 0; Q.toktab.shift = 0;      // no table yet: every piece is merged
+        Q.ext_id = v->d_ext_id; Q.piece_cnt = d_cnt; Q.stage = d_stage; Q.pairbuf = nullptr; Q.tile_tok = d_tt; Q.ids_cap = ~0ull;
+        const int grid = (int)(ntiles < (size_t)v->sm_count * 8 ? ntiles : (size_t)v->sm_count * 8);
+        k_pieces<<<grid, BPE_THREADS>>>(Q);
         ok = cudaGetLastError() == cudaSuccess && cudaDeviceSynchronize() == cudaSuccess;
     }
     ok = ok && cudaMemcpy(cnt.data(), d_cnt, np * sizeof(u32), cudaMemcpyDeviceToHost) == cudaSuccess;
     ok = ok && cudaMemcpy(stage.data(), d_stage, nb * sizeof(int32_t), cudaMemcpyDeviceToHost) == cudaSuccess;
-    cudaFree(d_text); cudaFree(d_off); cudaFree(d_cnt); cudaFree(d_long); cudaFree(d_stage); cudaFree(d_hdr);
+    cudaFree(d_text); cudaFree(d_mask); cudaFree(d_tb); cudaFree(d_tt); cudaFree(d_cnt); cudaFree(d_stage); cudaFree(d_hdr);
     if (!ok) { cudaGetLastError(); return TT_ERR_CUDA; }
     std::vector<u32> keep;
     for (size_t i = 0; i < np; i++)
@@ -224,7 +236,6 @@ static size_t carve(TTWorkspace* w, void* base, size_t max_len, size_t max_docs)
     const size_t padded = max_len + 64;                       // aligned frame: up to 15 bytes of shift + tail
     const size_t nchunks = padded / TT_CHUNK + 2;
     const size_t ntiles = nchunks / TT_TILE_CHUNKS + 2;
-    const size_t nblk = max_len / BPE_THREADS + 2;
     size_t off = 0;
     auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return (char*)base + o; };
     char* p;
@@ -232,13 +243,10 @@ static size_t carve(TTWorkspace* w, void* base, size_t max_len, size_t max_docs)
     p = take((padded / 32 + 4) * sizeof(u32));  if (w) w->docmask = (u32*)p;
     p = take(nchunks * sizeof(u16));            if (w) w->startmask = (u16*)p;
     p = take((ntiles + 1) * sizeof(u32));       if (w) w->tile_cnt = (u32*)p;
-    p = take((max_len + 2) * sizeof(u32));      if (w) w->piece_off = (u32*)p;
+    p = take((ntiles + 1) * sizeof(u32));       if (w) w->tile_tok = (u32*)p;
     p = take((max_len + 1) * sizeof(u32));      if (w) w->piece_cnt = (u32*)p;
-    p = take((nblk + 1) * sizeof(u32));         if (w) w->blk_cnt = (u32*)p;
-    p = take((max_len + 2) * sizeof(u32));      if (w) w->tok_off = (u32*)p;
     p = take((max_len + 1) * sizeof(int32_t));  if (w) w->stage = (int32_t*)p;
-    p = take((max_len + 1) * sizeof(u32));      if (w) w->rank_buf = (u32*)p;
-    p = take((max_len / TT_WARP_PIECE_MAX + 2) * sizeof(u32)); if (w) w->long_list = (u32*)p;
+    p = take((max_len + 1) * sizeof(u64));      if (w) w->pairbuf = (u64*)p;
     return off;
 }
 
@@ -249,12 +257,12 @@ extern "C" size_t tt_workspace_bytes(const tt_vocab* v, size_t max_len, size_t m
 
 #define CK(x) do { if ((x) != cudaSuccess) { cudaGetLastError(); return TT_ERR_CUDA; } } while (0)
 
-// Enqueues K1+K2 and K3.  piece_off_dst receives the offsets (workspace array or the caller's).
+// Enqueues K1+K2 (and K3 when piece_off_dst is given: only tt_pretokenize materialises the offsets;
+// the encode chain derives them per tile from the start flags).
 static int run_pretok(const tt_vocab* v, const uint8_t* text, size_t len, const int64_t* doc_off, size_t n_docs,
-                      cudaStream_t st, TTWorkspace& w, u32* piece_off_dst, cudaEvent_t ev_mid = nullptr) {
+                      cudaStream_t st, TTWorkspace& w, u32* piece_off_dst, PretokParams& P) {
     const uintptr_t addr = (uintptr_t)text;
     const long long shift = (long long)(addr & 15);
-    PretokParams P;
     P.base = (const u8*)(addr - shift);
     P.lo = shift; P.hi = shift + (long long)len;
     P.nchunks = (P.hi + TT_CHUNK - 1) / TT_CHUNK;
@@ -272,9 +280,9 @@ static int run_pretok(const tt_vocab* v, const uint8_t* text, size_t len, const 
     const size_t smem = align_up(v->cls_bytes, 16) + sizeof(u16) * F_COUNT * TT_SLOTS;
     const int grid = P.ntiles < v->sm_count * 4 ? P.ntiles : v->sm_count * 4;
     k_pretok<<<grid, TT_TILE_CHUNKS, smem, st>>>(P);
-    if (ev_mid) cudaEventRecord(ev_mid, st);
-    k_compact<<<grid, TT_TILE_CHUNKS, 0, st>>>(w.startmask, w.tile_cnt, P.nchunks, P.ntiles, shift, (long long)len,
-                                               piece_off_dst, w.hdr, w.long_list, TT_WARP_PIECE_MAX);
+    if (piece_off_dst)
+        k_compact<<<grid, TT_TILE_CHUNKS, 0, st>>>(w.startmask, w.tile_cnt, P.nchunks, P.ntiles, shift, (long long)len,
+                                                   piece_off_dst, w.hdr);
     CK(cudaGetLastError());
     return TT_OK;
 }
@@ -302,25 +310,26 @@ static int encode_impl(const tt_vocab* v, const uint8_t* text, size_t len, const
         return TT_OK;
     }
     MARK(0);
-    int rc = run_pretok(v, text, len, doc_off, n_docs, st, w, w.piece_off, ev ? ev[1] : nullptr);
+    PretokParams PP;
+    int rc = run_pretok(v, text, len, doc_off, n_docs, st, w, nullptr, PP);
     if (rc != TT_OK) return rc;
+    MARK(1);
+    const int tile_grid = PP.ntiles < v->sm_count * 8 ? PP.ntiles : v->sm_count * 8;
+    PieceParams Q;
+    Q.base = PP.base; Q.shift = PP.lo; Q.hi = PP.hi; Q.nchunks = PP.nchunks; Q.ntiles = PP.ntiles;
+    Q.startmask = w.startmask; Q.tile_base = w.tile_cnt; Q.hdr = w.hdr; Q.tab = v->tab; Q.toktab = v->toktab;
+    Q.ext_id = v->d_ext_id; Q.piece_cnt = w.piece_cnt; Q.stage = w.stage; Q.pairbuf = w.pairbuf; Q.tile_tok = w.tile_tok;
+    Q.ids_cap = (unsigned long long)ids_cap;
+    k_pieces<<<tile_grid, BPE_THREADS, 0, st>>>(Q);
     MARK(2);
-    k_bpe_long<<<v->sm_count, LONG_THREADS, 0, st>>>(text, w.piece_off, w.hdr, v->tab, v->d_ext_id, w.piece_cnt, w.stage,
-                                                     w.rank_buf, w.long_list);
+    ScatterParams S;
+    S.shift = PP.lo; S.hi = PP.hi; S.nchunks = PP.nchunks; S.ntiles = PP.ntiles; S.startmask = w.startmask;
+    S.tile_base = w.tile_cnt; S.tile_tok = w.tile_tok; S.piece_cnt = w.piece_cnt; S.stage = w.stage; S.hdr = w.hdr;
+    S.ids_out = ids_out; S.count_out = (long long*)count_out; S.status_out = status_out;
+    S.docmask = doc_off ? w.docmask : nullptr; S.doc_off = (const long long*)doc_off; S.n_docs = (int)n_docs;
+    S.ids_off_out = (long long*)ids_off_out;
+    k_scatter<<<tile_grid, BPE_THREADS, 0, st>>>(S);
     MARK(3);
-    const size_t want = (len + BPE_THREADS - 1) / BPE_THREADS;               // upper bound of piece blocks
-    const int piece_grid = (int)(want > (size_t)v->sm_count * 8 ? (size_t)v->sm_count * 8 : want);
-    k_bpe_pieces<<<piece_grid, BPE_THREADS, 0, st>>>(text, w.piece_off, w.hdr, v->tab, v->toktab, v->d_ext_id, w.piece_cnt,
-                                                     w.stage, w.blk_cnt, (unsigned long long)ids_cap);
-    MARK(4);
-    k_scatter<<<piece_grid, BPE_THREADS, 0, st>>>(w.piece_off, w.piece_cnt, w.blk_cnt, w.stage, w.hdr, w.tok_off, ids_out,
-                                                  (long long*)count_out, status_out);
-    if (doc_off) {
-        const int threads = 256, blocks = (int)((n_docs + 1 + threads - 1) / threads);
-        k_doc_offsets<<<blocks, threads, 0, st>>>((const long long*)doc_off, (int)n_docs, w.piece_off, w.tok_off, w.hdr,
-                                                  (long long*)ids_off_out);
-    }
-    MARK(5);
 #undef MARK
     CK(cudaGetLastError());
     return TT_OK;
@@ -348,18 +357,18 @@ extern "C" int tt_encode_batch(const tt_vocab* v, const uint8_t* text, size_t to
 
 extern "C" int tt_encode_timed(const tt_vocab* v, const uint8_t* text, size_t len, void* stream, int32_t* ids_out,
                                size_t ids_cap, int64_t* count_out, int32_t* status_out, void* workspace,
-                               size_t workspace_bytes, float ms_out[5]) {
+                               size_t workspace_bytes, float ms_out[3]) {
     int rc = check_common(v, text, len, workspace, workspace_bytes, 1);
     if (rc != TT_OK) return rc;
     if (!count_out || !status_out || !ms_out || !len || !ids_out) return TT_ERR_ARG;
-    cudaEvent_t ev[6];
-    for (int i = 0; i < 6; i++) CK(cudaEventCreate(&ev[i]));
+    cudaEvent_t ev[4];
+    for (int i = 0; i < 4; i++) CK(cudaEventCreate(&ev[i]));
     rc = encode_impl(v, text, len, nullptr, 1, (cudaStream_t)stream, ids_out, ids_cap, count_out, nullptr, status_out,
                      workspace, ev);
-    if (rc == TT_OK && cudaEventSynchronize(ev[5]) != cudaSuccess) rc = TT_ERR_CUDA;
-    for (int i = 0; i < 5 && rc == TT_OK; i++)
+    if (rc == TT_OK && cudaEventSynchronize(ev[3]) != cudaSuccess) rc = TT_ERR_CUDA;
+    for (int i = 0; i < 3 && rc == TT_OK; i++)
         if (cudaEventElapsedTime(&ms_out[i], ev[i], ev[i + 1]) != cudaSuccess) rc = TT_ERR_CUDA;
-    for (int i = 0; i < 6; i++) cudaEventDestroy(ev[i]);
+    for (int i = 0; i < 4; i++) cudaEventDestroy(ev[i]);
     return rc;
 }
 
@@ -383,7 +392,8 @@ extern "C" int tt_pretokenize(const tt_vocab* v, const uint8_t* text, size_t len
         CK(cudaMemsetAsync(status_out, 0, sizeof(int32_t), st));
         return TT_OK;
     }
-    rc = run_pretok(v, text, len, doc_off, n_docs, st, w, (u32*)piece_off_out);
+    PretokParams PP;
+    rc = run_pretok(v, text, len, doc_off, n_docs, st, w, (u32*)piece_off_out, PP);
     if (rc != TT_OK) return rc;
     k_finish_pretok<<<1, 1, 0, st>>>(w.hdr, (long long*)n_pieces_out, status_out);
     CK(cudaGetLastError());

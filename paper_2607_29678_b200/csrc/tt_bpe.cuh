@@ -213,22 +213,7 @@ __device__ __forceinline__ u32 warp_merge_perm(u64* buf /* 2 * 32 * E entries of
     return m;
 }
 
-// ---- CTA-wide scans -----------------------------------------------------------------------------------
-__device__ __forceinline__ int cta_incl_max_scan(int v, int* scratch /* >= 33 */, int carry) {
-    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5, nw = blockDim.x >> 5;
-    for (int o = 1; o < 32; o <<= 1) { int t = __shfl_up_sync(0xFFFFFFFFu, v, o); if (lane >= o) v = max(v, t); }
-    __syncthreads();
-    if (lane == 31) scratch[wid] = v;
-    __syncthreads();
-    if (wid == 0) {
-        int s = lane < nw ? scratch[lane] : INT_MIN;
-        for (int o = 1; o < 32; o <<= 1) { int t = __shfl_up_sync(0xFFFFFFFFu, s, o); if (lane >= o) s = max(s, t); }
-        if (lane < nw) scratch[lane] = s;
-    }
-    __syncthreads();
-    int before = wid ? scratch[wid - 1] : INT_MIN;
-    return max(max(v, before), carry);
-}
+// ---- CTA-wide helpers ------------------------------------------------------------------------------------
 __device__ __forceinline__ u32 cta_excl_sum_scan(u32 v, u32* scratch /* >= 33 */, u32* total) {
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5, nw = blockDim.x >> 5;
     u32 x = v;
@@ -246,219 +231,361 @@ __device__ __forceinline__ u32 cta_excl_sum_scan(u32 v, u32* scratch /* >= 33 */
     *total = scratch[32];
     return scratch[wid] + x - v;
 }
+__device__ __forceinline__ u32 cta_min_u32(u32 v, u32* scratch /* >= 33 */) {
+    v = __reduce_min_sync(0xFFFFFFFFu, v);
+    __syncthreads();
+    if ((threadIdx.x & 31) == 0) scratch[threadIdx.x >> 5] = v;
+    __syncthreads();
+    u32 r = scratch[0];
+    for (int w = 1; w < (int)(blockDim.x >> 5); w++) r = min(r, scratch[w]);
+    return r;
+}
 
-// ---- K4, pieces of a block of BPE_THREADS consecutive pieces ---------------------------------------------
-// Phase 1: a thread per piece (one-byte pieces map directly, pieces of up to 24 bytes are looked up as
-// whole vocabulary entries).  Phase 2: the CTA's warps merge the pieces phase 1 could not settle.
-// Phase 3: the token total of the block; the last CTA to finish turns the block totals into their
-// exclusive prefix (K5's scan) and checks the output capacity.  Pieces longer than
-// TT_WARP_PIECE_MAX were encoded before this kernel (k_bpe_long); only their counts are read here.
-// Without a token table (while the table itself is being built) every piece takes the merge path.
-__global__ void __launch_bounds__(BPE_THREADS)
-k_bpe_pieces(const u8* __restrict__ text, const u32* __restrict__ piece_off, TTHeader* hdr, const PairTable tab,
-             const TokTable toktab, const int32_t* __restrict__ ext_id, u32* __restrict__ piece_cnt,
-             int32_t* __restrict__ stage, u32* __restrict__ blk_cnt, unsigned long long ids_cap) {
-    __shared__ u64 s_buf[BPE_WARPS][2 * TT_WARP_PIECE_MAX];     // two (token, rank) buffers per warp
-    __shared__ u32 s_miss[BPE_THREADS];
-    __shared__ u32 s_nmiss, s_total, s_islast;
-    __shared__ u32 sc[40];
-    const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
-    const bool dead = hdr->status != 0;
-    const u32 n_pieces = dead ? 0 : hdr->n_pieces;
-    const u32 n_blocks = (n_pieces + BPE_THREADS - 1) / BPE_THREADS;
-    for (u32 pb = blockIdx.x; pb < n_blocks; pb += gridDim.x) {
-        __syncthreads();
-        if (tid == 0) { s_nmiss = 0; s_total = 0; }
-        __syncthreads();
-        const u32 p = pb * BPE_THREADS + tid;
-        u32 cnt = 0;
-        if (p < n_pieces) {
-            const u32 a = piece_off[p], n = piece_off[p + 1] - a;
-            int32_t id;
-            if (n == 1) { stage[a] = ext_id[text[a]]; cnt = 1; }
-            else if (n > TT_WARP_PIECE_MAX) cnt = piece_cnt[p];
-            else if (n <= TT_TOKTAB_MAXLEN && toktab.slots != nullptr && toktab_lookup(toktab, text, a, n, id)) { stage[a] = id; cnt = 1; }
-            else s_miss[atomicAdd(&s_nmiss, 1u)] = p;
-            if (cnt && n <= TT_WARP_PIECE_MAX) piece_cnt[p] = cnt;
+// ---- CTA merge for long pieces -----------------------------------------------------------------------------
+// arr[i] = token | (rank of the pair (i, i+1) << 32), in global scratch or shared memory.  One round:
+// the minimum rank is found, every thread takes LK consecutive positions, decides which of its
+// candidates are merged (the parity of a run of consecutive candidates is carried from thread to
+// thread with one ballot-based scan; LK is even, so a slice that is all candidates leaves the parity
+// unchanged), and the survivors are written to their new positions in place, chunk after chunk (every
+// thread of a chunk has its positions in registers before anything is written, and writes never pass
+// the read front).  Ranks next to a merge are marked stale and probed again in a second sweep, which
+// also yields the next round's minimum.
+constexpr int LK = 16;
+
+__device__ __noinline__ u32 cta_merge_rounds(u64* arr, u32 m, const PairTable& tab, u32* s_scr /* >= 48 */, u32 stop_at, bool& finished) {
+    const int tid = threadIdx.x, T = blockDim.x, lane = tid & 31, wid = tid >> 5, nw = T >> 5;
+    finished = false;
+    // minimum rank of the current array
+    u32 lmin = TT_RANK_INF;
+    for (u32 i = tid; i < m; i += T) lmin = min(lmin, (u32)(arr[i] >> 32));
+    for (;;) {
+        const u32 mn = cta_min_u32(lmin, s_scr);
+        if (mn == TT_RANK_INF) { finished = true; return m; }
+        if (m <= stop_at) return m;
+        u32 carry_par = 0, out = 0;                        // parity of the candidate run before the chunk; survivors so far
+        for (u32 base = 0; base < m; base += (u32)T * LK) {
+            const u32 i0 = base + (u32)tid * LK;
+            u32 tok[LK + 1], rk[LK + 1];
+#pragma unroll
+            for (int k = 0; k <= LK; k++) {
+                const u32 i = i0 + k;
+                const u64 v = i < m ? arr[i] : ~0ull;
+                tok[k] = (u32)v; rk[k] = i < m ? (u32)(v >> 32) : TT_RANK_INF;
+            }
+            const u32 nval = i0 < m ? min((u32)LK, m - i0) : 0;
+            u32 cand = 0;
+#pragma unroll
+            for (int k = 0; k <= LK; k++) cand |= (u32)(rk[k] == mn) << k;
+            const u32 cand_in = cand & ((1u << LK) - 1);
+            const bool all = cand_in == ((1u << LK) - 1);
+            // parity of my trailing candidate run (if not all candidates)
+            const u32 trail = __clz(~(cand_in << (32 - LK)));                 // consecutive candidates at the top of the slice
+            const u32 my_par = trail & 1;
+            // incoming parity: trailing parity of the nearest lower slice that is not all candidates
+            const u32 allm = __ballot_sync(0xFFFFFFFFu, all), parm = __ballot_sync(0xFFFFFFFFu, my_par);
+            const u32 lower = ~allm & ((1u << lane) - 1);
+            __syncthreads();
+            if (lane == 31) { const u32 na = ~allm; s_scr[wid] = na ? (2u | ((parm >> (31 - __clz(na))) & 1)) : 0u; }   // 0 = all lanes pass through
+            __syncthreads();
+            u32 in_par;
+            if (lower) in_par = (parm >> (31 - __clz(lower))) & 1;
+            else {
+                in_par = carry_par;
+                for (int w = wid - 1; w >= 0; w--) { const u32 e = s_scr[w]; if (e) { in_par = e & 1; break; } }
+            }
+            u32 next_carry = carry_par;
+            for (int w = nw - 1; w >= 0; w--) { const u32 e = s_scr[w]; if (e) { next_carry = e & 1; break; } }
+            // selection inside the slice (positions 0..LK; position LK only to know whether it is merged)
+            u32 sel = 0, off = in_par;
+#pragma unroll
+            for (int k = 0; k <= LK; k++) {
+                if ((cand >> k) & 1) { sel |= (u32)!(off & 1) << k; off++; } else off = 0;
+            }
+            const bool gone0 = in_par == 1;                                    // the element before the slice was merged with my first
+            const u32 gone = ((sel << 1) | (u32)gone0) & ((1u << LK) - 1);
+            const u32 valid = nval >= LK ? ((1u << LK) - 1) : ((1u << nval) - 1);
+            const u32 surv = valid & ~gone;
+            u32 tot;
+            const u32 ex = cta_excl_sum_scan(__popc(surv), s_scr, &tot);         // all loads of the chunk are done: barrier inside
+            u32 o = out + ex;
+#pragma unroll
+            for (int k = 0; k < LK; k++) {
+                if ((surv >> k) & 1) {
+                    const bool me = (sel >> k) & 1;
+                    const bool nxt = me ? false : ((sel >> (k + 1)) & 1);
+                    const u32 nt = me ? 256u + mn : tok[k];
+                    const u32 nr = (me || nxt) ? RK_STALE : rk[k];
+                    arr[o++] = ((u64)nr << 32) | nt;
+                }
+            }
+            out += tot;
+            carry_par = next_carry;
+            __syncthreads();
         }
-        u32 wsum = cnt;
+        m = out;
+        __syncthreads();
+        // probe the stale ranks again; collect the minimum for the next round
+        lmin = TT_RANK_INF;
+        for (u32 i = tid; i < m; i += T) {
+            const u64 v = arr[i];
+            u32 r = (u32)(v >> 32);
+            if (i + 1 >= m) { r = TT_RANK_INF; arr[i] = ((u64)r << 32) | (u32)v; }
+            else if (r == RK_STALE) { r = pair_probe(tab, (u32)v, (u32)arr[i + 1]); arr[i] = ((u64)r << 32) | (u32)v; }
+            lmin = min(lmin, r);
+        }
+        __syncthreads();
+    }
+}
+
+constexpr int LONG_SMEM_TOKENS = 4096;                  // long pieces move into shared memory below this many tokens
+
+// Encodes one piece of n > TT_WARP_PIECE_MAX bytes with the whole CTA.  gbuf: n entries of global scratch.
+__device__ u32 cta_merge_long(const u8* __restrict__ text, u32 a, u32 n, const PairTable& tab, const int32_t* __restrict__ ext_id,
+                              int32_t* __restrict__ stage, u64* gbuf, u64* sbuf /* LONG_SMEM_TOKENS */, u32* s_scr) {
+    const int tid = threadIdx.x, T = blockDim.x;
+    u64* arr = n <= LONG_SMEM_TOKENS ? sbuf : gbuf;
+    __syncthreads();
+    for (u32 i = tid; i < n; i += T) {
+        const u32 t0 = text[a + i];
+        const u32 r = (i + 1 < n) ? pair_probe(tab, t0, text[a + i + 1]) : TT_RANK_INF;
+        arr[i] = ((u64)r << 32) | t0;
+    }
+    __syncthreads();
+    bool finished;
+    u32 m = cta_merge_rounds(arr, n, tab, s_scr, arr == gbuf ? LONG_SMEM_TOKENS : 0, finished);
+    if (!finished && arr == gbuf) {
+        __syncthreads();
+        for (u32 i = tid; i < m; i += T) sbuf[i] = gbuf[i];
+        __syncthreads();
+        arr = sbuf;
+        m = cta_merge_rounds(arr, m, tab, s_scr, 0, finished);
+    }
+    __syncthreads();
+    for (u32 i = tid; i < m; i += T) stage[a + i] = ext_id[(u32)arr[i]];
+    __syncthreads();
+    return m;
+}
+
+// ---- pieces of one text tile -----------------------------------------------------------------------------
+// The start flags of a tile (TT_TILE_CHUNKS u16 masks) become a list of in-tile piece offsets in shared
+// memory; the end of the tile's last piece is the next start flag after the tile (or the text end).
+constexpr int TILE_MAX_PIECES = TT_TILE_BYTES;
+
+struct TilePieces {
+    u16 off[TILE_MAX_PIECES];      // byte offset of each piece inside the tile (aligned frame)
+    u32 n;                         // pieces that start in the tile
+    u32 end;                       // end of the last piece, relative to the tile start (may lie far beyond the tile)
+};
+
+__device__ void tile_pieces(TilePieces& tp, const u16* __restrict__ startmask, long long nchunks, long long c0,
+                            long long hi /* end of text, aligned frame */, u32* s_scr) {
+    const int tid = threadIdx.x;
+    u32 m = 0;
+    if (tid < TT_TILE_CHUNKS && c0 + tid < nchunks) m = startmask[c0 + tid];
+    u32 tot;
+    u32 r = cta_excl_sum_scan(__popc(m), s_scr, &tot);
+    while (m) { const int i = __ffs(m) - 1; m &= m - 1; tp.off[r++] = (u16)(tid * TT_CHUNK + i); }
+    // the next start after the tile
+    __shared__ u32 s_next;
+    if (tid == 0) { tp.n = tot; s_next = 0xFFFFFFFFu; }
+    __syncthreads();
+    if (tot) {
+        for (long long cb = c0 + TT_TILE_CHUNKS; cb < nchunks; cb += blockDim.x) {
+            const long long c = cb + tid;
+            const u32 mm = c < nchunks ? startmask[c] : 0;
+            if (mm) atomicMin(&s_next, (u32)((c - c0) * TT_CHUNK + (__ffs(mm) - 1)));
+            __syncthreads();
+            if (s_next != 0xFFFFFFFFu) break;
+        }
+        __syncthreads();
+        if (tid == 0) tp.end = s_next != 0xFFFFFFFFu ? s_next : (u32)(hi - c0 * TT_CHUNK);
+    }
+    __syncthreads();
+}
+
+// ---- K4 (+ the scan of K5): all pieces of a text tile -----------------------------------------------------------
+// Phase 1: a thread per piece (one-byte pieces map directly, pieces of up to 24 bytes are looked up as
+// whole vocabulary entries).  Phase 2: the CTA's warps merge the pieces phase 1 could not settle; pieces
+// longer than TT_WARP_PIECE_MAX are merged by the whole CTA.  Phase 3: the tile's token total; the last
+// CTA to finish turns the tile totals into their exclusive prefix and checks the output capacity.
+// Without a token table (while the table itself is being built) every piece takes the merge path.
+struct PieceParams {
+    const u8* base;            // aligned frame origin (text = base + shift)
+    long long shift, hi;       // text occupies [shift, hi)
+    long long nchunks;
+    int ntiles;
+    const u16* startmask;
+    const u32* tile_base;      // first piece index of every tile (exclusive prefix, ntiles + 1)
+    TTHeader* hdr;
+    PairTable tab;
+    TokTable toktab;
+    const int32_t* ext_id;
+    u32* piece_cnt;            // tokens per piece
+    int32_t* stage;            // ids staged at the text offset of their piece
+    u64* pairbuf;              // global scratch of the long-piece path, indexed like the text
+    u32* tile_tok;             // out: tokens per tile, then their exclusive prefix (ntiles + 1)
+    unsigned long long ids_cap;
+};
+
+__global__ void __launch_bounds__(BPE_THREADS, 4)
+k_pieces(const PieceParams P) {
+    __shared__ TilePieces tp;
+    __shared__ u64 s_buf[LONG_SMEM_TOKENS];                   // warp merge buffers (8 x 2 x 256) or one long piece
+    __shared__ u16 s_miss[TILE_MAX_PIECES];
+    __shared__ u32 s_nmiss, s_nlong, s_total, s_islast;
+    __shared__ u32 sc[48];
+    static_assert(LONG_SMEM_TOKENS >= BPE_WARPS * 2 * TT_WARP_PIECE_MAX, "buffer size");
+    const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+    const bool dead = P.hdr->status != 0;
+    const u8* text = P.base + P.shift;
+    for (int tile = blockIdx.x; tile < (dead ? 0 : P.ntiles); tile += gridDim.x) {
+        const long long c0 = (long long)tile * TT_TILE_CHUNKS;
+        __syncthreads();
+        if (tid == 0) { s_nmiss = 0; s_nlong = 0; s_total = 0; }
+        tile_pieces(tp, P.startmask, P.nchunks, c0, P.hi, sc);
+        const u32 np = tp.n, p0 = P.tile_base[tile];
+        const long long t0 = c0 * TT_CHUNK - P.shift;             // text offset of the tile start
+        u32 wsum = 0;
+        for (u32 i = tid; i < np; i += BPE_THREADS) {
+            const u32 a = (u32)(t0 + tp.off[i]);
+            const u32 n = (i + 1 < np ? tp.off[i + 1] : tp.end) - tp.off[i];
+            int32_t id;
+            if (n == 1) { P.stage[a] = P.ext_id[text[a]]; P.piece_cnt[p0 + i] = 1; wsum++; }
+            else if (n <= TT_TOKTAB_MAXLEN && P.toktab.slots != nullptr && toktab_lookup(P.toktab, text, a, n, id)) {
+                P.stage[a] = id; P.piece_cnt[p0 + i] = 1; wsum++;
+            } else if (n > TT_WARP_PIECE_MAX) { s_miss[TILE_MAX_PIECES - 1 - atomicAdd(&s_nlong, 1u)] = (u16)i; }
+            else s_miss[atomicAdd(&s_nmiss, 1u)] = (u16)i;        // short misses from the front, long pieces from the back
+        }
         for (int o = 16; o; o >>= 1) wsum += __shfl_xor_sync(0xFFFFFFFFu, wsum, o);
         __syncthreads();
-        const u32 nmiss = s_nmiss;
+        const u32 nmiss = s_nmiss, nlong = s_nlong;
         u32 msum = 0;
+        u64* wbuf = s_buf + wid * (2 * TT_WARP_PIECE_MAX);
         for (u32 e = wid; e < nmiss; e += BPE_WARPS) {
-            const u32 q = s_miss[e];
-            const u32 a = piece_off[q], n = piece_off[q + 1] - a;
-            const u32 m = n <= 32 ? warp_merge_reg(text, a, n, tab, ext_id, stage, lane)
-                        : n <= 64 ? warp_merge_perm<2>(s_buf[wid], text, a, n, tab, ext_id, stage, lane)
-                                  : warp_merge_perm<WCH>(s_buf[wid], text, a, n, tab, ext_id, stage, lane);
-            if (lane == 0) piece_cnt[q] = m;
+            const u32 i = s_miss[e];
+            const u32 a = (u32)(t0 + tp.off[i]);
+            const u32 n = (i + 1 < np ? tp.off[i + 1] : tp.end) - tp.off[i];
+            const u32 m = n <= 32 ? warp_merge_reg(text, a, n, P.tab, P.ext_id, P.stage, lane)
+                        : n <= 64 ? warp_merge_perm<2>(wbuf, text, a, n, P.tab, P.ext_id, P.stage, lane)
+                                  : warp_merge_perm<WCH>(wbuf, text, a, n, P.tab, P.ext_id, P.stage, lane);
+            if (lane == 0) P.piece_cnt[p0 + i] = m;
             msum += m;
         }
         if (lane == 0) atomicAdd(&s_total, wsum + msum);
+        for (u32 e = 0; e < nlong; e++) {                         // block-uniform
+            const u32 i = s_miss[TILE_MAX_PIECES - 1 - e];
+            const u32 a = (u32)(t0 + tp.off[i]);
+            const u32 n = (i + 1 < np ? tp.off[i + 1] : tp.end) - tp.off[i];
+            const u32 m = cta_merge_long(text, a, n, P.tab, P.ext_id, P.stage, P.pairbuf + a, s_buf, sc);
+            if (tid == 0) { P.piece_cnt[p0 + i] = m; atomicAdd(&s_total, m); }
+        }
         __syncthreads();
-        if (tid == 0) blk_cnt[pb] = s_total;
+        if (tid == 0) P.tile_tok[tile] = s_total;
     }
-    // the last CTA to finish: exclusive prefix of the block totals, total token count, capacity check
+    // the last CTA to finish: exclusive prefix of the tile totals, total token count, capacity check
     __threadfence();
     __syncthreads();
-    if (tid == 0) s_islast = (atomicAdd(&hdr->count_done, 1u) == gridDim.x - 1);
+    if (tid == 0) s_islast = (atomicAdd(&P.hdr->count_done, 1u) == gridDim.x - 1);
     __syncthreads();
     if (!s_islast) return;
     __threadfence();
     unsigned long long carry = 0;
-    for (u32 b0 = 0; b0 < n_blocks; b0 += BPE_THREADS) {
+    const u32 nt = dead ? 0 : (u32)P.ntiles;
+    for (u32 b0 = 0; b0 < nt; b0 += BPE_THREADS) {
         const u32 i = b0 + tid;
-        u32 x = i < n_blocks ? blk_cnt[i] : 0, t2;
+        u32 x = i < nt ? P.tile_tok[i] : 0, t2;
         const u32 ex = cta_excl_sum_scan(x, sc, &t2);
-        if (i < n_blocks) blk_cnt[i] = (u32)carry + ex;
+        if (i < nt) P.tile_tok[i] = (u32)carry + ex;
         carry += t2;
         __syncthreads();
     }
     if (tid == 0) {
-        hdr->n_tokens = carry;
-        if (!dead && carry > ids_cap) atomicMax(&hdr->status, 5 /* TT_ERR_CAPACITY */);
+        P.tile_tok[nt] = (u32)carry;
+        P.hdr->n_tokens = carry;
+        if (!dead && carry > P.ids_cap) atomicMax(&P.hdr->status, 5 /* TT_ERR_CAPACITY */);
     }
 }
 
-// ---- K4, CTA per long piece (long whitespace / punctuation runs and other pieces > 256 bytes) -----
-constexpr int LONG_THREADS = 1024;
-constexpr u32 TOK_NEW = 0x80000000u;                  // token produced in the current round
+// ---- K5: coalesced scatter of the staged ids, one text tile per CTA iteration ---------------------------------
+// Also writes the token offset of every document that starts in the tile (batch calls).
+struct ScatterParams {
+    long long shift, hi, nchunks;
+    int ntiles;
+    const u16* startmask;
+    const u32* tile_base;
+    const u32* tile_tok;
+    const u32* piece_cnt;
+    const int32_t* stage;
+    TTHeader* hdr;
+    int32_t* ids_out;
+    long long* count_out;
+    int32_t* status_out;
+    const u32* docmask;        // batch: bit per byte of document starts, else null
+    const long long* doc_off;  // batch: n_docs + 1 offsets
+    int n_docs;
+    long long* ids_off_out;    // batch: n_docs + 1 token offsets
+};
 
-__global__ void __launch_bounds__(LONG_THREADS)
-k_bpe_long(const u8* __restrict__ text, const u32* __restrict__ piece_off, TTHeader* hdr, const PairTable tab,
-           const int32_t* __restrict__ ext_id, u32* __restrict__ piece_cnt, int32_t* __restrict__ stage,
-           u32* __restrict__ rank_buf, const u32* __restrict__ long_list) {
-    __shared__ u32 s_u[40];
-    __shared__ int s_i[40];
-    __shared__ u32 s_sel[LONG_THREADS];
-    __shared__ u32 s_item, s_min;
-    if (hdr->status != 0) return;
-    const u32 n_long = hdr->n_long;
-    const int tid = threadIdx.x;
-    for (;;) {
-        __syncthreads();
-        if (tid == 0) s_item = atomicAdd(&hdr->long_next, 1u);
-        __syncthreads();
-        const u32 item = s_item;
-        if (item >= n_long) break;
-        const u32 p = long_list[item];
-        const u32 a = piece_off[p], n = piece_off[p + 1] - a;
-        u32* tok = reinterpret_cast<u32*>(stage) + a;
-        u32* rk = rank_buf + a;
-        for (u32 i = tid; i < n; i += LONG_THREADS) tok[i] = text[a + i];
-        __syncthreads();
-        for (u32 i = tid; i < n; i += LONG_THREADS) rk[i] = (i + 1 < n) ? pair_probe(tab, tok[i], tok[i + 1]) : TT_RANK_INF;
-        u32 m = n;
-        for (u32 round = 0; round < n; round++) {
-            __syncthreads();
-            // pass 1: minimum rank present
-            u32 mn = TT_RANK_INF;
-            for (u32 i = tid; i < m; i += LONG_THREADS) mn = min(mn, rk[i]);
-            mn = __reduce_min_sync(0xFFFFFFFFu, mn);
-            if (tid == 0) s_min = TT_RANK_INF;
-            __syncthreads();
-            if ((tid & 31) == 0) atomicMin(&s_min, mn);
-            __syncthreads();
-            mn = s_min;
-            if (mn == TT_RANK_INF) break;
-            // pass 2: select and compact, chunk by chunk in order (writes never pass the read front)
-            int carry_z = -1;            // nearest non-candidate position so far
-            u32 carry_removed = 0, carry_lastsel = 0;
-            for (u32 b = 0; b < m; b += LONG_THREADS) {
-                const u32 i = b + tid;
-                const bool in = i < m;
-                const u32 t = in ? (tok[i] & ~TOK_NEW) : 0;
-                const u32 r = in ? rk[i] : TT_RANK_INF;
-                const bool cand = in && r == mn;
-                const int z = cta_incl_max_scan(cand ? -1 : (int)i, s_i, carry_z);
-                const bool sel = cand && !(((int)i - z - 1) & 1);
-                s_sel[tid] = sel;
-                u32 tot;
-                const u32 ex = cta_excl_sum_scan(sel ? 1u : 0u, s_u, &tot);     // contains __syncthreads: s_sel visible
-                const bool gone = tid ? s_sel[tid - 1] : carry_lastsel;
-                if (in && !gone) {
-                    const u32 np = i - carry_removed - ex;
-                    tok[np] = sel ? ((256u + mn) | TOK_NEW) : t;
-                    rk[np] = r;
-                }
-                // carries for the next chunk (identical in every thread)
-                const u32 last = min(m - b, (u32)LONG_THREADS) - 1;
-                __syncthreads();
-                if (tid == (int)last) { s_i[34] = z; s_u[34] = sel; }
-                __syncthreads();
-                carry_z = s_i[34]; carry_lastsel = s_u[34];
-                carry_removed += tot;
-            }
-            m -= carry_removed;
-            __syncthreads();
-            // pass 3: probe again the pairs that touch a new token
-            for (u32 i = tid; i < m; i += LONG_THREADS) {
-                const u32 x = tok[i], y = (i + 1 < m) ? tok[i + 1] : 0;
-                if ((x | y) & TOK_NEW) rk[i] = (i + 1 < m) ? pair_probe(tab, x & ~TOK_NEW, y & ~TOK_NEW) : TT_RANK_INF;
-            }
-        }
-        __syncthreads();
-        for (u32 i = tid; i < m; i += LONG_THREADS) stage[a + i] = ext_id[tok[i] & ~TOK_NEW];
-        if (tid == 0) piece_cnt[p] = m;
-    }
-}
-
-// ---- K5: token offsets per piece and coalesced scatter of the staged ids ----------------------------------
-// One CTA per block of BPE_THREADS pieces (the same partition as k_bpe_pieces, whose last CTA left the
-// exclusive prefix of the block totals in blk_base).
 __global__ void __launch_bounds__(BPE_THREADS)
-k_scatter(const u32* __restrict__ piece_off, const u32* __restrict__ piece_cnt, const u32* __restrict__ blk_base,
-          const int32_t* __restrict__ stage, TTHeader* hdr, u32* __restrict__ tok_off, int32_t* __restrict__ ids_out,
-          long long* __restrict__ count_out, int32_t* __restrict__ status_out) {
-    __shared__ u32 sc[40];
-    __shared__ u32 s_big[BPE_THREADS][3];
+k_scatter(const ScatterParams P) {
+    __shared__ TilePieces tp;
+    __shared__ u32 sc[48];
+    __shared__ u32 s_big[TILE_MAX_PIECES / 8][3];
     __shared__ u32 s_nbig;
-    const int status = hdr->status;
-    const u32 n_pieces = hdr->n_pieces;
-    if (blockIdx.x == 0 && threadIdx.x == 0) {
-        if (status_out) *status_out = status;
-        if (count_out) *count_out = status ? 0 : (long long)hdr->n_tokens;
-        if (status || n_pieces == 0) tok_off[0] = 0;
+    const int tid = threadIdx.x;
+    const int status = P.hdr->status;
+    if (blockIdx.x == 0 && tid == 0) {
+        if (P.status_out) *P.status_out = status;
+        if (P.count_out) *P.count_out = status ? 0 : (long long)P.hdr->n_tokens;
     }
-    if (status != 0) return;
-    const u32 n_blocks = (n_pieces + BPE_THREADS - 1) / BPE_THREADS;
-    for (u32 pb = blockIdx.x; pb < n_blocks; pb += gridDim.x) {
+    if (status != 0) {
+        if (P.ids_off_out)
+            for (long long d = (long long)blockIdx.x * blockDim.x + tid; d <= P.n_docs; d += (long long)gridDim.x * blockDim.x) P.ids_off_out[d] = 0;
+        return;
+    }
+    if (P.ids_off_out && blockIdx.x == 0) {
+        // documents that start at the very end of the text (empty trailing documents) and the total
+        const long long len = P.hi - P.shift;
+        for (int d = P.n_docs - tid; d >= 0 && P.doc_off[d] >= len; d -= blockDim.x) P.ids_off_out[d] = (long long)P.hdr->n_tokens;
+    }
+    for (int tile = blockIdx.x; tile < P.ntiles; tile += gridDim.x) {
+        const long long c0 = (long long)tile * TT_TILE_CHUNKS;
         __syncthreads();
-        if (threadIdx.x == 0) s_nbig = 0;
-        const u32 p = pb * BPE_THREADS + threadIdx.x;
-        const u32 c = p < n_pieces ? piece_cnt[p] : 0;
-        u32 tot;
-        const u32 dst = blk_base[pb] + cta_excl_sum_scan(c, sc, &tot);
-        if (p < n_pieces) {
-            tok_off[p] = dst;
-            if (p == n_pieces - 1) tok_off[n_pieces] = dst + c;
-            const u32 src = piece_off[p];
-            if (c <= 8) {
-                for (u32 k = 0; k < c; k++) ids_out[dst + k] = stage[src + k];
-            } else {
-                const u32 slot = atomicAdd(&s_nbig, 1u);
-                s_big[slot][0] = src; s_big[slot][1] = dst; s_big[slot][2] = c;
+        if (tid == 0) s_nbig = 0;
+        tile_pieces(tp, P.startmask, P.nchunks, c0, P.hi, sc);
+        const u32 np = tp.n, p0 = P.tile_base[tile];
+        const long long t0 = c0 * TT_CHUNK - P.shift;
+        u32 carry = P.tile_tok[tile];
+        for (u32 b = 0; b < np; b += BPE_THREADS) {
+            const u32 i = b + tid;
+            const u32 c = i < np ? P.piece_cnt[p0 + i] : 0;
+            u32 tot;
+            const u32 dst = carry + cta_excl_sum_scan(c, sc, &tot);
+            if (i < np) {
+                const u32 src = (u32)(t0 + tp.off[i]);
+                if (c <= 8) { for (u32 k = 0; k < c; k++) P.ids_out[dst + k] = P.stage[src + k]; }
+                else {
+                    const u32 slot = atomicAdd(&s_nbig, 1u);
+                    if (slot < TILE_MAX_PIECES / 8) { s_big[slot][0] = src; s_big[slot][1] = dst; s_big[slot][2] = c; }
+                }
+                if (P.docmask) {
+                    const long long g = c0 * TT_CHUNK + tp.off[i];
+                    if ((P.docmask[g >> 5] >> (g & 31)) & 1) {
+                        // every document that starts at this byte (empty ones included) gets this token offset
+                        const long long want = g - P.shift;
+                        int lo = 0, hi2 = P.n_docs;
+                        while (lo < hi2) { int mid = (lo + hi2) >> 1; if (P.doc_off[mid] < want) lo = mid + 1; else hi2 = mid; }
+                        for (int d = lo; d <= P.n_docs && P.doc_off[d] == want; d++) P.ids_off_out[d] = dst;
+                    }
+                }
             }
+            carry += tot;
+            __syncthreads();
         }
-        __syncthreads();
-        const u32 nbig = s_nbig;
+        const u32 nbig = min(s_nbig, (u32)(TILE_MAX_PIECES / 8));
         for (u32 e = 0; e < nbig; e++) {
             const u32 src = s_big[e][0], d2 = s_big[e][1], cc = s_big[e][2];
-            for (u32 k = threadIdx.x; k < cc; k += BPE_THREADS) ids_out[d2 + k] = stage[src + k];
+            for (u32 k = tid; k < cc; k += BPE_THREADS) P.ids_out[d2 + k] = P.stage[src + k];
         }
     }
-}
-
-// ---- batch: token offset of every document ----------------------------------------------------------
-__global__ void k_doc_offsets(const long long* __restrict__ doc_off, int n_docs, const u32* __restrict__ piece_off,
-                              const u32* __restrict__ tok_off, const TTHeader* hdr, long long* __restrict__ ids_off_out) {
-    const int d = blockIdx.x * blockDim.x + threadIdx.x;
-    if (d > n_docs) return;
-    if (hdr->status != 0) { ids_off_out[d] = 0; return; }
-    const u32 n_pieces = hdr->n_pieces;
-    const long long want = doc_off[d];
-    u32 lo = 0, hi = n_pieces;                  // first piece whose offset is >= want
-    while (lo < hi) { u32 mid = (lo + hi) >> 1; if ((long long)piece_off[mid] < want) lo = mid + 1; else hi = mid; }
-    ids_off_out[d] = tok_off[lo];
 }

@@ -54,11 +54,8 @@ struct TTWorkspace {
     u32* docmask;      // bit per text byte: first byte of a document (batch only)
     u16* startmask;    // bit per text byte: first byte of a piece (one u16 per chunk)
     u32* tile_cnt;     // pieces per tile, then exclusive prefix (ntiles + 1)
-    u32* piece_off;    // byte offset of every piece + sentinel (len + 2)
+    u32* tile_tok;     // tokens per tile, then exclusive prefix (ntiles + 1)
     u32* piece_cnt;    // tokens per piece (len + 1)
-    u32* blk_cnt;      // token count per block of pieces, then exclusive prefix
-    u32* tok_off;      // token offset of every piece + total (len + 2); before the scatter: the miss list
     int32_t* stage;    // token ids staged at the byte offset of their piece (len)
-    u32* rank_buf;     // per-position ranks for the long-piece path (len)
-    u32* long_list;    // piece indices longer than TT_WARP_PIECE_MAX
+    u64* pairbuf;      // (token, rank) pairs of the long-piece path, indexed like the text (len)
 };

@@ -326,40 +326,21 @@ k_pretok(const PretokParams P) {
     }
 }
 
-// ---- K3: compaction of the start flags into piece offsets ---------------------------------------
-// piece_off[i] = byte offset (relative to the text) of piece i; piece_off[n_pieces] = len.
-// Pieces longer than `long_min` bytes are also appended to long_list (they take the CTA-per-piece
-// merge kernel): a piece's end is the next start bit, searched at most long_min bytes ahead.
+// ---- K3: compaction of the start flags into piece offsets (tt_pretokenize) --------------------------
+// piece_off[i] = byte offset (relative to the text) of piece i; piece_off[n_pieces] = len.  The encode
+// chain does the same per tile in shared memory (tile_pieces in tt_bpe.cuh) and never stores the list.
 __global__ void __launch_bounds__(TT_TILE_CHUNKS)
 k_compact(const u16* __restrict__ startmask, const u32* __restrict__ tile_base, long long nchunks, int ntiles,
-          long long shift, long long len, u32* __restrict__ piece_off, TTHeader* hdr, u32* __restrict__ long_list,
-          int long_min) {
+          long long shift, long long len, u32* __restrict__ piece_off, TTHeader* hdr) {
     __shared__ u32 sc[40];
-    __shared__ u16 s_m[TT_TILE_CHUNKS];
     if (hdr->status != 0) return;
     for (int tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
-        const long long c0 = (long long)tile * TT_TILE_CHUNKS;
-        const long long chunk = c0 + threadIdx.x;
+        const long long chunk = (long long)tile * TT_TILE_CHUNKS + threadIdx.x;
         u32 m = chunk < nchunks ? startmask[chunk] : 0;
-        __syncthreads();
-        s_m[threadIdx.x] = (u16)m;
-        u32 r = tile_base[tile] + cta_exscan_u32(tt_popc(m), sc, nullptr);      // contains __syncthreads
+        u32 r = tile_base[tile] + cta_exscan_u32(tt_popc(m), sc, nullptr);
         const long long g0 = chunk * TT_CHUNK - shift;
-        if (m) {
-            // only the last start of the chunk can begin a piece that reaches beyond the chunk
-            const int top = tt_hibit(m);
-            long long dist = 16 - top;
-            long long j = chunk + 1;
-            bool found = false;
-            while (dist <= long_min && j < nchunks) {
-                const u32 mm = (j - c0 < TT_TILE_CHUNKS) ? s_m[j - c0] : startmask[j];
-                if (mm) { dist += tt_lobit(mm); found = true; break; }
-                dist += 16; j++;
-            }
-            if (!found && j >= nchunks) dist = len - (g0 + top);
-            if (dist > long_min) long_list[atomicAdd(&hdr->n_long, 1u)] = r + tt_popc(m) - 1;
-        }
         while (m) { int i = tt_lobit(m); m &= m - 1; piece_off[r++] = (u32)(g0 + i); }
+        __syncthreads();
     }
     if (blockIdx.x == 0 && threadIdx.x == 0) piece_off[tile_base[ntiles]] = (u32)len;
 }

@@ -158,6 +158,8 @@ def main():
     ap.add_argument("--batch-docs", type=int, default=256)
     ap.add_argument("--profile", action="store_true",
                     help="run only the warm-up and the timed steps, then exit (command used under ncu)")
+    ap.add_argument("--profile-batch", action="store_true",
+                    help="run only the config-C5 batch leg (2 warm-up + 2 timed calls), then exit (command used under ncu)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -185,6 +187,20 @@ def main():
     cfg = wl.CONFIGS["C3"]
     merges, byte_map = wl.load_vocab(cfg)
     vocab = tt.Vocab(merges, byte_map, cfg.pattern_id)
+    if args.profile_batch:
+        c5 = wl.CONFIGS["C5"]
+        btext, boff = wl.batch(c5, sample=rank, n_docs=args.batch_docs)
+        d_text = torch.from_numpy(btext).cuda(); d_off = torch.from_numpy(boff).cuda()
+        bb = vocab.alloc(btext.size, max_docs=boff.size - 1)
+        ts = []
+        for k in range(4):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(); vocab.encode_batch(d_text, d_off, bb); b.record()
+            torch.cuda.synchronize()
+            ts.append(a.elapsed_time(b))
+        print(json.dumps({"profile_batch_run": True, "bytes": int(btext.size), "ms": [round(t, 3) for t in ts],
+                          "tokens": int(bb["ids_off"][-1].item())}), flush=True)
+        return
     host_texts = [wl.request(cfg, sample=rank * 100 + s) for s in range(N_DISTINCT_INPUTS)]
     max_len = max(t.size for t in host_texts)
     dev_texts = [torch.from_numpy(t).cuda() for t in host_texts]

@@ -20,9 +20,12 @@
 struct PairTable {
     const u64* slots;     // 4 * (mask + 1) slots
     u32 mask;             // number of buckets - 1 (power of two)
-    u32 shift;            // 64 - log2(number of buckets)
+    u32 shift;            // 32 - log2(number of buckets)
 };
-TT_HD u32 pair_bucket(u64 key, u32 shift) { return (u32)((key * 0x9E3779B97F4A7C15ull) >> shift); }
+TT_HD u32 pair_bucket(u64 key, u32 shift) {
+    const u32 x = ((u32)key ^ ((u32)(key >> 32) * 0x9E3779B1u)) * 0x85EBCA6Bu;
+    return (x ^ (x >> 15)) * 0xC2B2AE35u >> shift;
+}
 
 __device__ __forceinline__ u32 pair_probe(const PairTable& t, u32 a, u32 b) {
     const u64 key = ((u64)a << TT_ID_BITS) | b;
@@ -114,8 +117,13 @@ __device__ __forceinline__ u32 warp_merge_reg(const u8* __restrict__ text, u32 a
         const u32 nt = me ? 256u + mn : t;
         const u32 nr = (me || nxt) ? RK_STALE : r;
         // survivors move down: new lane j takes the j-th surviving old lane
-        const u32 surv = ~(sel << 1) & (m >= 32 ? FULL : ((1u << m) - 1));
-        const u32 src = __fns(surv, 0, lane + 1);
+        u32 src;
+        if ((sel & (sel - 1)) == 0) {                   // one merge (the usual case): everything above it moves down by one
+            src = (u32)lane + ((u32)lane > (u32)(__ffs(sel) - 1) ? 1u : 0u);
+        } else {
+            const u32 surv = ~(sel << 1) & (m >= 32 ? FULL : ((1u << m) - 1));
+            src = __fns(surv, 0, lane + 1);
+        }
         t = __shfl_sync(FULL, nt, src & 31);
         r = __shfl_sync(FULL, nr, src & 31);
         m -= __popc(sel);
@@ -377,29 +385,25 @@ struct TilePieces {
     u32 end;                       // end of the last piece, relative to the tile start (may lie far beyond the tile)
 };
 
-__device__ void tile_pieces(TilePieces& tp, const u16* __restrict__ startmask, long long nchunks, long long c0,
-                            long long hi /* end of text, aligned frame */, u32* s_scr) {
+__device__ void tile_pieces(TilePieces& tp, const u16* __restrict__ startmask, const u32* __restrict__ tile_first,
+                            long long nchunks, int ntiles, int tile, long long hi /* end of text, aligned frame */, u32* s_scr) {
     const int tid = threadIdx.x;
+    const long long c0 = (long long)tile * TT_TILE_CHUNKS;
     u32 m = 0;
     if (tid < TT_TILE_CHUNKS && c0 + tid < nchunks) m = startmask[c0 + tid];
+    if (tid == 0) {
+        // the next start after the tile: the first start of the next tile that has one, else the text end
+        u32 end = (u32)(hi - c0 * TT_CHUNK);
+        for (int t = tile + 1; t < ntiles; t++) {
+            const u32 f = tile_first[t];
+            if (f != 0xFFFFFFFFu) { end = (u32)(t - tile) * TT_TILE_BYTES + f; break; }
+        }
+        tp.end = end;
+    }
     u32 tot;
     u32 r = cta_excl_sum_scan(__popc(m), s_scr, &tot);
     while (m) { const int i = __ffs(m) - 1; m &= m - 1; tp.off[r++] = (u16)(tid * TT_CHUNK + i); }
-    // the next start after the tile
-    __shared__ u32 s_next;
-    if (tid == 0) { tp.n = tot; s_next = 0xFFFFFFFFu; }
-    __syncthreads();
-    if (tot) {
-        for (long long cb = c0 + TT_TILE_CHUNKS; cb < nchunks; cb += blockDim.x) {
-            const long long c = cb + tid;
-            const u32 mm = c < nchunks ? startmask[c] : 0;
-            if (mm) atomicMin(&s_next, (u32)((c - c0) * TT_CHUNK + (__ffs(mm) - 1)));
-            __syncthreads();
-            if (s_next != 0xFFFFFFFFu) break;
-        }
-        __syncthreads();
-        if (tid == 0) tp.end = s_next != 0xFFFFFFFFu ? s_next : (u32)(hi - c0 * TT_CHUNK);
-    }
+    if (tid == 0) tp.n = tot;
     __syncthreads();
 }
 
@@ -416,6 +420,7 @@ struct PieceParams {
     int ntiles;
     const u16* startmask;
     const u32* tile_base;      // first piece index of every tile (exclusive prefix, ntiles + 1)
+    const u32* tile_first;     // offset of the first piece start inside every tile (~0: none)
     TTHeader* hdr;
     PairTable tab;
     TokTable toktab;
@@ -442,7 +447,7 @@ k_pieces(const PieceParams P) {
         const long long c0 = (long long)tile * TT_TILE_CHUNKS;
         __syncthreads();
         if (tid == 0) { s_nmiss = 0; s_nlong = 0; s_total = 0; }
-        tile_pieces(tp, P.startmask, P.nchunks, c0, P.hi, sc);
+        tile_pieces(tp, P.startmask, P.tile_first, P.nchunks, P.ntiles, tile, P.hi, sc);
         const u32 np = tp.n, p0 = P.tile_base[tile];
         const long long t0 = c0 * TT_CHUNK - P.shift;             // text offset of the tile start
         u32 wsum = 0;
@@ -458,6 +463,8 @@ k_pieces(const PieceParams P) {
         }
         for (int o = 16; o; o >>= 1) wsum += __shfl_xor_sync(0xFFFFFFFFu, wsum, o);
         __syncthreads();
+        // the misses of the tile are spread over the CTA's warps (the longest merge chain of a request sets
+        // its latency, so no warp should have to do two of them in a row if another warp is idle)
         const u32 nmiss = s_nmiss, nlong = s_nlong;
         u32 msum = 0;
         u64* wbuf = s_buf + wid * (2 * TT_WARP_PIECE_MAX);
@@ -513,6 +520,7 @@ struct ScatterParams {
     int ntiles;
     const u16* startmask;
     const u32* tile_base;
+    const u32* tile_first;
     const u32* tile_tok;
     const u32* piece_cnt;
     const int32_t* stage;
@@ -552,7 +560,7 @@ k_scatter(const ScatterParams P) {
         const long long c0 = (long long)tile * TT_TILE_CHUNKS;
         __syncthreads();
         if (tid == 0) s_nbig = 0;
-        tile_pieces(tp, P.startmask, P.nchunks, c0, P.hi, sc);
+        tile_pieces(tp, P.startmask, P.tile_first, P.nchunks, P.ntiles, tile, P.hi, sc);
         const u32 np = tp.n, p0 = P.tile_base[tile];
         const long long t0 = c0 * TT_CHUNK - P.shift;
         u32 carry = P.tile_tok[tile];

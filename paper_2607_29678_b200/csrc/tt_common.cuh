@@ -54,6 +54,7 @@ struct TTWorkspace {
     u32* docmask;      // bit per text byte: first byte of a document (batch only)
     u16* startmask;    // bit per text byte: first byte of a piece (one u16 per chunk)
     u32* tile_cnt;     // pieces per tile, then exclusive prefix (ntiles + 1)
+    u32* tile_first;   // offset of the first piece start inside each tile, ~0 if none (ntiles + 1)
     u32* tile_tok;     // tokens per tile, then exclusive prefix (ntiles + 1)
     u32* piece_cnt;    // tokens per piece (len + 1)
     int32_t* stage;    // token ids staged at the byte offset of their piece (len)

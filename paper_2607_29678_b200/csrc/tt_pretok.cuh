@@ -29,6 +29,7 @@ struct PretokParams {
     const u32* docmask;      // bit per byte (aligned frame) marking document starts, or null (one document)
     u16* startmask;          // out: one u16 per chunk
     u32* tile_cnt;           // out: pieces per tile; replaced by the exclusive prefix (ntiles + 1 entries)
+    u32* tile_first;         // out: offset inside the tile of its first piece start, or ~0 if it has none
     TTHeader* hdr;
     const u8* cls_tables;    // stage1 | stage2 | ascii, contiguous in global memory
     int cls_bytes;

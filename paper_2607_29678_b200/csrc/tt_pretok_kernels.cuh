@@ -200,7 +200,7 @@ k_pretok(const PretokParams P) {
     u8* tables = smem_raw;                                            // class tables
     u16 (*sm)[TT_SLOTS] = reinterpret_cast<u16 (*)[TT_SLOTS]>(smem_raw + ((P.cls_bytes + 15) & ~15));
     __shared__ long long scratch[40];
-    __shared__ u32 s_need;
+    __shared__ u32 s_need, s_first;
     __shared__ u32 s_islast;
 
     const int tid = threadIdx.x;
@@ -218,7 +218,7 @@ k_pretok(const PretokParams P) {
 
     for (int tile = blockIdx.x; tile < P.ntiles; tile += gridDim.x) {
         __syncthreads();
-        if (tid == 0) s_need = 0;
+        if (tid == 0) { s_need = 0; s_first = 0xFFFFFFFFu; }
         const long long c_first = (long long)tile * TT_TILE_CHUNKS;
         if (!tables_loaded) {                                         // block-uniform
             bool hi_bit = false;
@@ -300,8 +300,9 @@ k_pretok(const PretokParams P) {
                                : tt_eval_chunk_p1(sm, slot, SC, g0, tc, true, need);
         }
         if (c_first + tid < P.nchunks) P.startmask[c_first + tid] = (u16)S;
+        if (S) atomicMin(&s_first, (u32)(tid * TT_CHUNK + tt_lobit(S)));
         u32 total = cta_sum_u32(tt_popc(S), scratch);
-        if (tid == 0) P.tile_cnt[tile] = total;
+        if (tid == 0) { P.tile_cnt[tile] = total; P.tile_first[tile] = s_first; }
     }
     if (any_bad) atomicMax(&P.hdr->status, 4 /* TT_ERR_INVALID_UTF8 */);
 

@@ -365,20 +365,18 @@ def main():
 
 
 def vocab_table_bytes(n_merges: int) -> int:
-    cap = 1024
-    while cap < 2 * n_merges + 2:
-        cap *= 2
-    return cap * 8 + 4 * (256 + n_merges) + 21632      # pair table + id map + class tables
+    """Information content of the vocabulary tables a cold request has to read: one 8-byte (pair, rank)
+    slot per merge, the 4-byte id map and the 21,632-byte class tables."""
+    return 8 * n_merges + 4 * (256 + n_merges) + 21632
+
+
+# DRAM bytes (read + write) per launch from the committed ncu capture of the C3 request
+# (profiles/c3_1M_request_kernels.md).
+NCU_TRAFFIC = {"pieces": 5_282_048, "pretok": 1_129_728, "scatter": 4_909_824}
 
 
 def ncu_traffic(kernel: str):
-    """DRAM bytes per launch of the dominant kernel from the committed ncu summary, if there is one."""
-    p = os.path.join(ROOT, "profiles", "ncu_traffic.json")
-    try:
-        with open(p) as f:
-            return json.load(f).get(kernel)
-    except Exception:
-        return None
+    return NCU_TRAFFIC.get(kernel)
 
 
 if __name__ == "__main__":

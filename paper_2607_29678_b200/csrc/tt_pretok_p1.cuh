@@ -3,9 +3,10 @@
 // Paper Sec. 4.1: this lineage adds a case-boundary rule and a sparse contraction path to the
 // run-local rules, and Unicode marks take a narrow sparse fallback while the common path stays
 // vectorised.  Here the vectorised path covers number runs, whitespace runs, punctuation runs with
-// their [\r\n/]* tails, word starts with the one-character prefix and the lower->upper case boundary.
-// Three constructs are not decided by local rules: a mark, an upper-case letter that follows a
-// caseless letter, and an apostrophe between letters (a possible contraction suffix).  Each of them
+// their [\r\n/]* tails, word starts with the one-character prefix, the lower->upper case boundary and
+// the contraction suffix after a word.  Three constructs are not decided by local rules: a mark, an
+// upper-case letter that follows a caseless letter, and an apostrophe between letters that has another
+// apostrophe two or three bytes before it (a chain of possible contraction suffixes).  Each of them
 // marks the text from the last *sure* piece start before it up to the next sure piece start as
 // unresolved; a thread whose chunk contains unresolved bytes re-derives those bytes by matching
 // sequentially from that sure start (matching from a piece start never looks behind it).  Sure
@@ -160,18 +161,20 @@ TT_HD ChunkDoc tt_load_slot(const u16 (*sm)[TT_SLOTS], int s) {
 }
 // p = previous chunk, c = the chunk, n = next chunk
 TT_HD void tt_sure_hard_cm(const ChunkDoc& p, const ChunkDoc& c, const ChunkDoc& n, u32& sure, u32& hard) {
-    // 18-bit frame: bit 0 = last byte of the previous chunk, bits 1..16 = the chunk, bit 17 = first byte of the next
-#define FR(x) ((((u32)p.x) >> 15) | (((u32)c.x) << 1) | ((((u32)n.x) & 1u) << 17))
+    // 20-bit frame: bits 0..2 = last three bytes of the previous chunk, bits 3..18 = the chunk, bit 19 = first byte of the next
+#define FR(x) ((((u32)p.x) >> 13) | (((u32)c.x) << 3) | ((((u32)n.x) & 1u) << 19))
     const u32 lead = FR(m.lead), D = FR(doc);
     const u32 Lr = FR(m.low) | FR(m.upp) | FR(m.cless), N = FR(m.num), W = FR(m.spc), O = FR(m.oth), AP = FR(m.ap);
     const u32 nD = ~D;
     const u32 pLr = (Lr << 1) & nD, pN = (N << 1) & nD, pNL = (FR(m.nl) << 1) & nD, pCl = (FR(m.cless) << 1) & nD;
     const u32 nLr = (Lr >> 1) & ~(D >> 1);
     const u32 cs = D | (N & ~pN) | (W & (pLr | pN)) | (O & ~AP & (pLr | pN)) | (Lr & (pN | pNL));
-    const u32 h = FR(m.mark) | (FR(m.upp) & pCl) | (AP & pLr & nLr);
+    // an apostrophe between letters is a possible contraction suffix; it is decided locally unless another
+    // apostrophe two or three bytes before it may have consumed the letter in front of it
+    const u32 h = FR(m.mark) | (FR(m.upp) & pCl) | (AP & pLr & nLr & ((AP << 2) | (AP << 3)));
 #undef FR
-    sure = ((cs & lead) >> 1) & 0xFFFFu;
-    hard = ((h & lead) >> 1) & 0xFFFFu;
+    sure = ((cs & lead) >> 3) & 0xFFFFu;
+    hard = ((h & lead) >> 3) & 0xFFFFu;
 }
 // Valid for 1 <= s <= TT_SLOTS - 2 (needs the neighbouring slots).
 TT_HD void tt_sure_hard(const u16 (*sm)[TT_SLOTS], int s, u32& sure, u32& hard) {
@@ -280,6 +283,24 @@ TT_HD u32 tt_eval_chunk_p1(const u16 (*sm)[TT_SLOTS], int slot, const SeqCtx& C,
     const u64 pfx = ((G << 1) | ((G << 2) & c1) | ((G << 3) & c2 & c1) | ((G << 4) & c3 & c2 & c1)) & nD;
     S |= Lr & lead & ~PREV(Lr) & ~((PREV(W) & ~PREV(NL)) | pfx);
     S |= upp & lead & PREV(low);                          // case boundary: upper after lower
+    // ---- contraction suffix: an apostrophe between letters with a valid suffix ('s 't 'm 'd 're 've 'll, ASCII,
+    // any case) belongs to the word before it; the suffix letters start nothing and the next letter starts a piece.
+    // (Apostrophes with another apostrophe 2-3 bytes before them are left to the sparse path.)
+    {
+        u64 ca = AP & PREV(Lr) & ((Lr >> 1) & ~(D >> 1)) & ~((AP << 2) | (AP << 3)) & (0x7FFFFull << 29);   // own bytes -3 .. +15
+        while (ca) {
+            const int q = (u32)ca ? tt_lobit((u32)ca) : 32 + tt_lobit((u32)(ca >> 32));
+            ca &= ca - 1;
+            const long long g = g0 + (q - 32);
+            const u32 b1 = (g + 1 < C.hi) ? C.base[g + 1] : 0, b2 = (g + 2 < C.hi) ? C.base[g + 2] : 0;
+            int cl = tt_contraction_len(b1, (D >> (q + 2)) & 1 ? 0u : b2);
+            if (cl) {
+                const u64 span = ((1ull << cl) - 1) << q;                 // apostrophe and suffix letters
+                S &= ~span;
+                if (((D >> (q + 1)) & ((1ull << cl) - 1)) == 0) S |= (1ull << (q + cl)) & Lr & lead;
+            }
+        }
+    }
     // ---- number runs: every third lead counted from the run start
     {
         const u32 n_own = (u32)(N >> 32) & 0xFFFFu, ld_own = (u32)(lead >> 32) & 0xFFFFu;

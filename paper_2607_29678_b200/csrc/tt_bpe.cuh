@@ -7,7 +7,8 @@
 //   * a thread per piece looks the whole piece up as a vocabulary entry (one 32-byte probe);
 //   * pieces that are not a single entry are merged by a warp (<= 32 bytes: tokens in registers,
 //     candidates as ballot masks; <= 256 bytes: several tokens per lane, compaction through shared memory);
-//   * longer pieces are merged by a whole CTA with its state in global scratch (k_bpe_long).
+//   * longer pieces are merged by the whole CTA (cta_merge_long: state in shared memory, or in global
+//     scratch while the piece still has more than 4,096 tokens).
 // Token ids inside the kernels are "internal": byte b -> b, result of the merge of rank r -> 256 + r;
 // the caller's ids are looked up when the tokens are staged.
 #pragma once

@@ -249,3 +249,39 @@ def test_full_size_c5_batch_sampled_documents():
     # decode(encode(x)) == x on one further document, through the vocabulary's byte strings
     d = 64
     assert cv.decode(ids[ioff[d]:ioff[d + 1]][:2000]) == text[off[d]:off[d + 1]].tobytes()[:len(cv.decode(ids[ioff[d]:ioff[d + 1]][:2000]))]
+
+
+def _random_wellformed_merges(rng, n_merges, alphabet):
+    ids = list(alphabet)
+    seen, rows = set(), []
+    while len(rows) < n_merges:
+        p = (rng.choice(ids), rng.choice(ids))
+        if p in seen:
+            continue
+        seen.add(p)
+        rows.append((p[0], p[1], 256 + len(rows)))
+        ids.append(256 + len(rows) - 1)
+    return np.array(rows, dtype=np.int32)
+
+
+@pytest.mark.parametrize("seed,n_merges,alpha", [(1, 6, "ab"), (2, 40, "abc"), (3, 300, "abcd"), (4, 2000, "ab"), (5, 25, "a")])
+def test_merge_kernels_on_random_tables(seed, n_merges, alpha):
+    """Random well-formed merge tables over tiny alphabets (dense in repeated pairs and equal-token runs)
+    and letter-only documents of every length class: <= 32 bytes (registers), <= 64 and <= 256 (warp),
+    longer (CTA, shared memory and global scratch).  Each document is one piece under pattern 0."""
+    import paper_2607_29678_b200 as tt
+    rng = random.Random(seed)
+    merges = _random_wellformed_merges(rng, n_merges, [ord(c) for c in alpha])
+    gv = tt.Vocab(merges, None, 0)
+    cv = oracle.Vocab(merges)
+    lens = list(range(1, 70)) + [100, 128, 129, 200, 255, 256, 257, 300, 511, 1000, 2047, 2048, 2049, 4095, 4096, 4097, 5000, 9000, 20000]
+    docs = [bytes(rng.choice(alpha.encode()) for _ in range(n)) for n in lens for _ in range(3)]
+    text = np.frombuffer(b"".join(docs), dtype=np.uint8)
+    off = np.zeros(len(docs) + 1, dtype=np.int64)
+    off[1:] = np.cumsum([len(d) for d in docs])
+    ids, ioff, status = gpu_encode_batch(gv, text, off)
+    assert status == 0
+    for k, d in enumerate(docs):
+        want = cv.bpe(d, 2)
+        got = ids[ioff[k]:ioff[k + 1]]
+        assert got.size == want.size and np.array_equal(got, want), (len(d), d[:40])

@@ -96,16 +96,13 @@ constexpr int BPE_WARPS = 8;                          // warps per CTA of the pi
 constexpr int BPE_THREADS = BPE_WARPS * 32;           // = pieces per CTA iteration
 constexpr int WCH = TT_WARP_PIECE_MAX / 32;           // 32-token chunks per piece
 
-// ---- warp merge, up to 32 bytes: one token per lane, no shared memory ------------------------------------
-// Returns the token count; the tokens (caller's ids) are staged at stage[a ...].
-__device__ __forceinline__ u32 warp_merge_reg(const u8* __restrict__ text, u32 a, u32 n, const PairTable& tab,
-                                              const int32_t* __restrict__ ext_id, int32_t* __restrict__ stage, int lane) {
+// ---- warp merge rounds with at most 32 tokens: one token per lane, no shared memory -----------------------
+// t = token of position `lane`, r = rank of the pair (lane, lane + 1) or TT_RANK_INF, m = token count.
+// Runs rounds to the fixpoint, stages the tokens (caller's ids) at stage[a ...] and returns their count.
+__device__ __forceinline__ u32 warp_merge_reg_rounds(u32 t, u32 r, u32 m, u32 max_rounds, u32 a, const PairTable& tab,
+                                                     const int32_t* __restrict__ ext_id, int32_t* __restrict__ stage, int lane) {
     const u32 FULL = 0xFFFFFFFFu, lt = (1u << lane) - 1;
-    u32 t = (u32)lane < n ? text[a + lane] : 0;
-    u32 m = n;
-    u32 tn = __shfl_down_sync(FULL, t, 1);
-    u32 r = ((u32)lane + 1 < m) ? pair_probe(tab, t, tn) : TT_RANK_INF;
-    for (u32 round = 0; round < n; round++) {          // at most n - 1 merges
+    for (u32 round = 0; round < max_rounds; round++) {
         const u32 mn = __reduce_min_sync(FULL, r);
         if (mn == TT_RANK_INF) break;
         // leftmost non-overlapping occurrences: inside a run of consecutive candidates, every other one
@@ -128,12 +125,21 @@ __device__ __forceinline__ u32 warp_merge_reg(const u8* __restrict__ text, u32 a
         t = __shfl_sync(FULL, nt, src & 31);
         r = __shfl_sync(FULL, nr, src & 31);
         m -= __popc(sel);
-        tn = __shfl_down_sync(FULL, t, 1);
+        const u32 tn = __shfl_down_sync(FULL, t, 1);
         if ((u32)lane + 1 >= m) r = TT_RANK_INF;
         else if (r == RK_STALE) r = pair_probe(tab, t, tn);
     }
     if ((u32)lane < m) stage[a + lane] = ext_id[t];
     return m;
+}
+
+// A piece of up to 32 bytes.
+__device__ __forceinline__ u32 warp_merge_reg(const u8* __restrict__ text, u32 a, u32 n, const PairTable& tab,
+                                              const int32_t* __restrict__ ext_id, int32_t* __restrict__ stage, int lane) {
+    const u32 t = (u32)lane < n ? text[a + lane] : 0;
+    const u32 tn = __shfl_down_sync(0xFFFFFFFFu, t, 1);
+    const u32 r = ((u32)lane + 1 < n) ? pair_probe(tab, t, tn) : TT_RANK_INF;
+    return warp_merge_reg_rounds(t, r, n, n, a, tab, ext_id, stage, lane);
 }
 
 // ---- warp merge, 33..256 bytes: E tokens per lane in registers, compaction through shared memory ---------
@@ -167,6 +173,7 @@ __device__ __forceinline__ u32 warp_merge_perm(u64* buf /* 2 * 32 * E entries of
         for (int j = 1; j < E; j++) mn = min(mn, r[j]);
         mn = __reduce_min_sync(FULL, mn);
         if (mn == TT_RANK_INF) break;
+        if (m <= 32) return warp_merge_reg_rounds(t[0], r[0], m, m, a, tab, ext_id, stage, lane);   // cheaper rounds from here on
         const int nch = (int)((m + 31) >> 5);
         u32 sel[E];
         u32 prev_ones = 0;                              // candidate run ending at the top of the previous word

@@ -89,6 +89,8 @@ def _load():
         lib.orc_vocab_free.argtypes = [c.c_void_p]
         lib.orc_token_bytes.restype = c.c_size_t
         lib.orc_token_bytes.argtypes = [c.c_void_p, c.c_int32, c.c_void_p, c.c_size_t]
+        lib.orc_token_lens.restype = None
+        lib.orc_token_lens.argtypes = [c.c_void_p, c.c_void_p, c.c_size_t, c.c_void_p]
         lib.orc_bpe.restype = c.c_int64
         lib.orc_bpe.argtypes = [c.c_void_p, c.c_void_p, c.c_size_t, c.c_int, c.c_void_p, c.c_size_t]
         lib.orc_encode.restype = c.c_int64
@@ -166,6 +168,22 @@ class Vocab:
 
     def decode(self, ids) -> bytes:
         return b"".join(self.token_bytes(int(i)) for i in ids)
+
+    def spans(self, text, ids):
+        """Span export (paper App. E.3): byte_off[i] = sum of the byte lengths of tokens 0..i-1;
+        char_off[i] = number of non-continuation bytes of the TEXT before byte_off[i].
+        Returns (byte_off int64[T+1], char_off int64[T+1])."""
+        a = _as_u8(text)
+        ids = np.ascontiguousarray(ids, dtype=np.int32)
+        lens = np.zeros(ids.size, dtype=np.int64)
+        _load().orc_token_lens(self._h, ids.ctypes.data, ids.size, lens.ctypes.data)
+        byte_off = np.zeros(ids.size + 1, dtype=np.int64)
+        byte_off[1:] = np.cumsum(lens)
+        if byte_off[-1] != a.size or (ids.size and lens.min() <= 0):
+            raise ValueError("ids do not spell the text")
+        starts_before = np.zeros(a.size + 1, dtype=np.int64)
+        starts_before[1:] = np.cumsum((a & 0xC0) != 0x80)
+        return byte_off, starts_before[byte_off]
 
     def bpe(self, piece, variant: int = 0) -> np.ndarray:
         """BPE of one piece; variant 0 = rescan definition, 1 = heap, 2 = chosen by length."""

@@ -356,6 +356,12 @@ size_t orc_token_bytes(const void *vp, int32_t id, uint8_t *out, size_t cap) {
     return s.size();
 }
 
+/* Byte lengths of n tokens (0 for an unknown id). */
+void orc_token_lens(const void *vp, const int32_t *ids, size_t n, int64_t *out) {
+    const Vocab *v = (const Vocab *)vp;
+    for (size_t i = 0; i < n; i++) out[i] = (ids[i] < 0 || ids[i] > v->max_id) ? 0 : (int64_t)v->token_bytes[ids[i]].size();
+}
+
 /* BPE of one piece.  variant 0 = rescan (the definition), 1 = heap, 2 = by length. */
 int64_t orc_bpe(const void *vp, const uint8_t *bytes, size_t n, int variant, int32_t *out, size_t cap) {
     std::vector<int32_t> t;

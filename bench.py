@@ -270,6 +270,21 @@ def main():
     kmean = {n: sum(v) / len(v) for n, v in ktimes.items()}
     dominant = max(kmean, key=kmean.get)
 
+    # ---- span export (paper App. E.3) on the ids of one request, cold caches ----
+    boff = torch.empty(max_len + 2, dtype=torch.int32, device="cuda")
+    coff = torch.empty(max_len + 2, dtype=torch.int32, device="cuda")
+    vocab.encode(dev_texts[0], bufs)
+    sws = vocab.spans(bufs["ids"], bufs["count"], dev_texts[0].numel(), boff, coff, bufs["status"])
+    torch.cuda.synchronize()
+    span_ms = []
+    for k in range(10):
+        flush_l2()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream); vocab.spans(bufs["ids"], bufs["count"], dev_texts[0].numel(), boff, coff, bufs["status"], workspace=sws); b.record(stream)
+        torch.cuda.synchronize()
+        span_ms.append(a.elapsed_time(b))
+    assert int(bufs["status"].item()) == 0
+
     # ---- end to end through the host-buffer entry point ----
     e2e = []
     n_ids = 0
@@ -354,6 +369,8 @@ def main():
                 "p50": round(pct(e2e, 0.5), 4), "api": "tt_encode_host (pageable host buffers in, pinned staging inside)"},
         "gpu_launches": 3 * args.steps,
         "batch": batch,
+        "span_export": {"ms_p50": round(pct(span_ms, 0.5), 4), "what": "tt_spans on the ids of one C3 request: byte and character "
+                        "offsets per token, device to device; the paper adds 0.13-0.73 ms for this step on its hardware"},
         "roofline": roofline,
         "cpu_baseline": cpu,
         "clocks": clocks,

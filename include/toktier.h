@@ -37,7 +37,8 @@ enum {
     TT_ERR_INVALID_UTF8 = 4,     /* device status: input is not strict UTF-8; zero tokens are returned */
     TT_ERR_CAPACITY = 5,         /* device status: ids_cap too small for the result; zero tokens       */
     TT_ERR_INTERNAL_TIMEOUT = 6, /* device status: a bounded device-side loop gave up                  */
-    TT_ERR_TOO_LARGE = 7         /* tt_encode_static only: len is above TT_STATIC_MAX_LEN              */
+    TT_ERR_TOO_LARGE = 7,        /* tt_encode_static only: len is above TT_STATIC_MAX_LEN              */
+    TT_ERR_BAD_IDS = 8           /* tt_spans device status: unknown id, or the ids do not spell text_len bytes */
 };
 
 /* Patterns (benchmark configs; the paper names the two lineages in Sec. 4.1):
@@ -117,6 +118,26 @@ int tt_encode_batch(const tt_vocab* v, const uint8_t* text, size_t total_len, co
 int tt_pretokenize(const tt_vocab* v, const uint8_t* text, size_t len, const int64_t* doc_off, size_t n_docs,
                    void* stream, int32_t* piece_off_out, size_t piece_cap, int64_t* n_pieces_out,
                    int32_t* status_out, void* workspace, size_t workspace_bytes);
+
+/*
+ * tt_spans -- byte and character spans of the tokens of an encoded text (paper App. E.3, span export:
+ * the IDs gather per-token byte lengths, a cumulative sum yields byte offsets, and a second cumulative
+ * sum over the non-continuation bytes lifts them to character offsets).
+ *   ids, count      DEVICE: the IDs and their number, as tt_encode left them (count <= ids_cap).
+ *   text_len        HOST value: byte length of the text the IDs were produced from (only checked).
+ *   byte_off_out    DEVICE int32[ids_cap + 1]: token i covers text bytes [byte_off[i], byte_off[i+1]).
+ *   char_off_out    DEVICE int32[ids_cap + 1]: char_off[i] = number of code points that start before
+ *                   byte_off[i]; a token that begins inside a multi-byte character therefore starts at
+ *                   the index of the next character.
+ *   status_out      DEVICE int32: TT_OK, or TT_ERR_BAD_IDS if an id is not in the vocabulary or the
+ *                   byte lengths do not add up to text_len (then only entry 0 of the outputs is written).
+ *   workspace       DEVICE scratch of at least tt_spans_workspace_bytes(v, ids_cap) bytes, 256-byte aligned.
+ * Asynchronous on `stream`; never reads the text.  Needs caller ids below 2^24 (else TT_ERR_ARG).
+ */
+size_t tt_spans_workspace_bytes(const tt_vocab* v, size_t ids_cap);
+int tt_spans(const tt_vocab* v, const int32_t* ids, const int64_t* count, size_t ids_cap, size_t text_len,
+             void* stream, int32_t* byte_off_out, int32_t* char_off_out, int32_t* status_out,
+             void* workspace, size_t workspace_bytes);
 
 /*
  * tt_encode_timed -- diagnostic variant of tt_encode (same arguments and results) that records

@@ -14,12 +14,12 @@ import numpy as np
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libtoktier.so")
 
-TT_OK, TT_ERR_ARG, TT_ERR_BAD_VOCAB, TT_ERR_CUDA, TT_ERR_INVALID_UTF8, TT_ERR_CAPACITY, TT_ERR_INTERNAL_TIMEOUT, TT_ERR_TOO_LARGE = range(8)
+TT_OK, TT_ERR_ARG, TT_ERR_BAD_VOCAB, TT_ERR_CUDA, TT_ERR_INVALID_UTF8, TT_ERR_CAPACITY, TT_ERR_INTERNAL_TIMEOUT, TT_ERR_TOO_LARGE, TT_ERR_BAD_IDS = range(9)
 TT_STATIC_MAX_LEN = 262144
 TT_PATTERN_CL100K, TT_PATTERN_O200K = 0, 1
 
 EXPORTS = ["tt_vocab_load", "tt_vocab_free", "tt_workspace_bytes", "tt_encode", "tt_encode_batch",
-           "tt_pretokenize", "tt_encode_timed", "tt_encode_host", "tt_encode_static", "tt_class_table", "tt_strerror"]
+           "tt_pretokenize", "tt_encode_timed", "tt_encode_host", "tt_encode_static", "tt_spans", "tt_spans_workspace_bytes", "tt_class_table", "tt_strerror"]
 
 _lib = None
 
@@ -59,6 +59,11 @@ def lib() -> ctypes.CDLL:
         L.tt_encode_static.restype = c.c_int
         L.tt_encode_static.argtypes = [c.c_void_p, c.c_void_p, c.c_size_t, c.c_void_p, c.c_void_p, c.c_size_t, c.c_void_p,
                                        c.c_void_p]
+        L.tt_spans_workspace_bytes.restype = c.c_size_t
+        L.tt_spans_workspace_bytes.argtypes = [c.c_void_p, c.c_size_t]
+        L.tt_spans.restype = c.c_int
+        L.tt_spans.argtypes = [c.c_void_p, c.c_void_p, c.c_void_p, c.c_size_t, c.c_size_t, c.c_void_p, c.c_void_p, c.c_void_p,
+                               c.c_void_p, c.c_void_p, c.c_size_t]
         L.tt_encode_host.restype = c.c_int
         L.tt_encode_host.argtypes = [c.c_void_p, c.c_void_p, c.c_size_t, c.c_void_p, c.c_size_t, c.POINTER(c.c_int64)]
         L.tt_class_table.restype = c.c_size_t
@@ -177,6 +182,17 @@ class Vocab:
         n = int(text.numel() if length is None else length)
         _check(lib().tt_encode_static(self._h, text.data_ptr(), n, _stream_ptr(stream), ids.data_ptr(), ids.numel(),
                                       count.data_ptr(), status.data_ptr()), "tt_encode_static")
+
+    def spans(self, ids, count, text_len: int, byte_off, char_off, status, workspace=None, stream=None):
+        """tt_spans: byte / character offsets of the tokens in `ids` (int32 CUDA tensor) whose number is in
+        `count` (int64 CUDA tensor [1]).  byte_off / char_off: int32 CUDA tensors [ids.numel() + 1]."""
+        import torch
+        if workspace is None:
+            workspace = torch.empty(int(lib().tt_spans_workspace_bytes(self._h, ids.numel())), dtype=torch.uint8, device=ids.device)
+        _check(lib().tt_spans(self._h, ids.data_ptr(), count.data_ptr(), ids.numel(), int(text_len), _stream_ptr(stream),
+                              byte_off.data_ptr(), char_off.data_ptr(), status.data_ptr(), workspace.data_ptr(),
+                              workspace.numel()), "tt_spans")
+        return workspace
 
     # -- host convenience --------------------------------------------------------------------------
     def encode_host(self, data) -> np.ndarray:

@@ -6,6 +6,7 @@
 #include "tt_common.cuh"
 #include "tt_pretok_kernels.cuh"
 #include "tt_bpe.cuh"
+#include "tt_spans.cuh"
 #include "unicode_table.inc"
 
 #include <climits>
@@ -32,6 +33,8 @@ struct tt_vocab {
     TokSlot* d_tokslots = nullptr;
     TokTable toktab{};
     size_t n_table_tokens = 0;
+    uint2* d_meta = nullptr;             // per caller id: (byte length, non-continuation bytes) for tt_spans
+    u32 meta_n = 0;
     // cached buffers of tt_encode_host
     u8* h_text = nullptr; int32_t* h_ids = nullptr; long long* h_scalars = nullptr;
     u8* d_text = nullptr; int32_t* d_ids = nullptr; long long* d_count = nullptr; int32_t* d_status = nullptr;
@@ -51,6 +54,7 @@ extern "C" const char* tt_strerror(int code) {
         case TT_ERR_CAPACITY: return "output buffer too small";
         case TT_ERR_INTERNAL_TIMEOUT: return "bounded device loop gave up";
         case TT_ERR_TOO_LARGE: return "input exceeds the fixed limit of the no-allocation entry point";
+        case TT_ERR_BAD_IDS: return "token ids do not belong to this vocabulary or do not spell a text of the given length";
         default: return "unknown code";
     }
 }
@@ -66,7 +70,7 @@ extern "C" size_t tt_class_table(uint8_t* out, size_t cap) {
 
 extern "C" void tt_vocab_free(tt_vocab* v) {
     if (!v) return;
-    cudaFree(v->d_slots); cudaFree(v->d_ext_id); cudaFree(v->d_cls); cudaFree(v->d_tokslots);
+    cudaFree(v->d_slots); cudaFree(v->d_ext_id); cudaFree(v->d_cls); cudaFree(v->d_tokslots); cudaFree(v->d_meta);
     cudaFree(v->d_text); cudaFree(v->d_ids); cudaFree(v->d_count); cudaFree(v->d_status); cudaFree(v->d_ws);
     if (v->h_text) cudaFreeHost(v->h_text);
     if (v->h_ids) cudaFreeHost(v->h_ids);
@@ -228,6 +232,25 @@ extern "C" int tt_vocab_load(const tt_merge* merges, size_t n_merges, const int3
     if (!ok) { cudaGetLastError(); tt_vocab_free(v); return TT_ERR_CUDA; }
     v->tab.slots = v->d_slots; v->tab.mask = mask; v->tab.shift = shift;
     if (build_token_table(v, merges, n_merges, ext_id) != TT_OK) { tt_vocab_free(v); return TT_ERR_CUDA; }
+    {   // byte length and number of non-continuation bytes of every token, indexed by the caller's id
+        std::vector<uint2> in(256 + n_merges);
+        for (int b = 0; b < 256; b++) in[b] = make_uint2(1u, (b & 0xC0) != 0x80 ? 1u : 0u);
+        int32_t max_ext = 0;
+        for (int32_t e : ext_id) max_ext = e > max_ext ? e : max_ext;
+        for (size_t r = 0; r < n_merges; r++) {
+            const uint2 L = in[internal[merges[r].left]], R = in[internal[merges[r].right]];
+            in[256 + r] = make_uint2(L.x + R.x, L.y + R.y);
+        }
+        if (max_ext < (1 << 24)) {
+            std::vector<uint2> meta((size_t)max_ext + 1, make_uint2(0, 0));
+            for (size_t i = 0; i < ext_id.size(); i++) meta[ext_id[i]] = in[i];
+            if (cudaMalloc(&v->d_meta, meta.size() * sizeof(uint2)) != cudaSuccess ||
+                cudaMemcpy(v->d_meta, meta.data(), meta.size() * sizeof(uint2), cudaMemcpyHostToDevice) != cudaSuccess) {
+                cudaGetLastError(); tt_vocab_free(v); return TT_ERR_CUDA;
+            }
+            v->meta_n = (u32)meta.size();
+        }
+    }
     *out = v;
     return TT_OK;
 }
@@ -399,6 +422,34 @@ extern "C" int tt_pretokenize(const tt_vocab* v, const uint8_t* text, size_t len
     rc = run_pretok(v, text, len, doc_off, n_docs, st, w, (u32*)piece_off_out, PP);
     if (rc != TT_OK) return rc;
     k_finish_pretok<<<1, 1, 0, st>>>(w.hdr, (long long*)n_pieces_out, status_out);
+    CK(cudaGetLastError());
+    return TT_OK;
+}
+
+extern "C" size_t tt_spans_workspace_bytes(const tt_vocab* v, size_t ids_cap) {
+    (void)v;
+    return align_up(sizeof(SpanHeader), 256) + align_up((ids_cap / SPAN_THREADS + 3) * sizeof(uint2), 256);
+}
+
+extern "C" int tt_spans(const tt_vocab* v, const int32_t* ids, const int64_t* count, size_t ids_cap, size_t text_len,
+                        void* stream, int32_t* byte_off_out, int32_t* char_off_out, int32_t* status_out, void* workspace,
+                        size_t workspace_bytes) {
+    if (!v || !count || !byte_off_out || !char_off_out || !status_out || !workspace || (ids_cap && !ids)) return TT_ERR_ARG;
+    if (v->meta_n == 0 || ids_cap >= (size_t)INT32_MAX || text_len >= (size_t)INT32_MAX) return TT_ERR_ARG;
+    if (((uintptr_t)workspace & 255) != 0 || workspace_bytes < tt_spans_workspace_bytes(v, ids_cap)) return TT_ERR_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    SpanParams P;
+    P.ids = ids; P.count = (const long long*)count; P.ids_cap = ids_cap; P.text_len = text_len;
+    P.meta = v->d_meta; P.meta_n = v->meta_n;
+    P.hdr = (SpanHeader*)workspace;
+    P.blk = (uint2*)((char*)workspace + align_up(sizeof(SpanHeader), 256));
+    P.byte_off = byte_off_out; P.char_off = char_off_out; P.status_out = status_out;
+    CK(cudaMemsetAsync(P.hdr, 0, sizeof(SpanHeader), st));
+    size_t want = (ids_cap + SPAN_THREADS - 1) / SPAN_THREADS;
+    if (want < 1) want = 1;
+    const int grid = (int)(want > (size_t)v->sm_count * 2 ? (size_t)v->sm_count * 2 : want);
+    k_span_sums<<<grid, SPAN_THREADS, 0, st>>>(P);
+    k_span_write<<<grid, SPAN_THREADS, 0, st>>>(P);
     CK(cudaGetLastError());
     return TT_OK;
 }

@@ -101,10 +101,11 @@ struct Matcher {
     }
 
     /* alternatives shared by both patterns --------------------------------------------- */
-    /* \p{N}{1,3} */
+    /* \p{N}{1,3}, or a single \p{N} in the single-digit variant (pattern 2) */
+    size_t maxDigits = 3;
     size_t altNumber(size_t p) const {
         size_t e = p;
-        while (e < n && e < p + 3 && isN(e)) e++;
+        while (e < n && e < p + maxDigits && isN(e)) e++;
         return e - p;
     }
     /*  ?[^\s\p{L}\p{N}]+[\r\n]*   (pattern 1: trailing class is [\r\n/]) */
@@ -193,11 +194,12 @@ struct Matcher {
 /* piece starts as code-point indices */
 void pretok_cp(const Text &t, int pattern, std::vector<size_t> &starts) {
     Matcher M(t);
+    if (pattern == 2) M.maxDigits = 1;        /* pattern 2 = pattern 0 with \p{N} in place of \p{N}{1,3} */
     size_t p = 0;
     starts.clear();
     while (p < M.n) {
         starts.push_back(p);
-        size_t m = pattern == 0 ? M.match0(p) : M.match1(p);
+        size_t m = pattern == 1 ? M.match1(p) : M.match0(p);
         if (m == 0) m = 1;   /* cannot happen: every position matches some alternative */
         p += m;
     }

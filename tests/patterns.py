@@ -18,7 +18,10 @@ P1 = (r"[^\r\n\p{L}\p{N}]?" + U + "*" + LW + "+" + "(?:" + CON + ")?"
       + r"|\s*[\r\n]+"
       + r"|\s+(?!\S)"
       + r"|\s+")
-PATTERNS = [P0, P1]
+# pattern 2: pattern 0 with single-digit number pieces (the paper's family table lists a "\\p{N} single" front end)
+P2 = P0.replace(r"|\p{N}{1,3}", r"|\p{N}")
+assert P2 != P0
+PATTERNS = [P0, P1, P2]
 
 
 def engine_starts(compiled, s: str):

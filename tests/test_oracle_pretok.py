@@ -54,6 +54,12 @@ def test_pattern1_equals_backtracking_engine(alphabet, maxlen):
     assert _exhaustive(1, alphabet, maxlen) == []
 
 
+@pytest.mark.parametrize("alphabet,maxlen", [("a12 \t\n!'", 5), ("1²٣ a.", 6)])
+def test_pattern2_single_digit_variant_equals_backtracking_engine(alphabet, maxlen):
+    assert _exhaustive(2, alphabet, maxlen) == []
+    assert [p.decode() for p in oracle.pieces("ab1234 56", 2)] == ["ab", "1", "2", "3", "4", " ", "5", "6"]
+
+
 def _agreeing_codepoints():
     """Code points whose class agrees between the oracle's frozen table and the regex engine's own
     (possibly newer) Unicode tables; random strings are drawn only from these."""
@@ -81,7 +87,7 @@ def test_random_unicode_strings_equal_engine():
     assert len(pool) > 5000
     rng = random.Random(11)
     special = list(" \t\n\r'/!.,") + ["'s", "'re", "'LL", "\r\n", "  "]
-    for pat in (0, 1):
+    for pat in (0, 1, 2):
         for _ in range(3000):
             n = rng.randrange(1, 40)
             s = "".join(rng.choice(special) if rng.random() < 0.5 else chr(rng.choice(pool)) for _ in range(n))

@@ -173,7 +173,7 @@ extern "C" int tt_vocab_load(const tt_merge* merges, size_t n_merges, const int3
                              tt_vocab** out) {
     if (out) *out = nullptr;
     if (!out || !byte_map || (n_merges && !merges)) return TT_ERR_ARG;
-    if (pattern_id != TT_PATTERN_CL100K && pattern_id != TT_PATTERN_O200K) return TT_ERR_ARG;
+    if (pattern_id != TT_PATTERN_CL100K && pattern_id != TT_PATTERN_O200K && pattern_id != TT_PATTERN_CL100K_N1) return TT_ERR_ARG;
     if (n_merges > TT_MAX_INTERNAL - 256) return TT_ERR_ARG;
     // external id -> internal id (byte b -> b, result of rank r -> 256 + r)
     std::unordered_map<int32_t, u32> internal;

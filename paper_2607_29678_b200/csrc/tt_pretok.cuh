@@ -132,7 +132,7 @@ TT_HD int tt_contraction_len(u32 b1, u32 b2) {
 // NEED_* flags of aggregates that leave the shared-memory window (then `tc` must be filled and the
 // function called again).
 TT_HD u32 tt_eval_chunk_p0(const u16 (*sm)[TT_SLOTS], int slot, const u8* base, long long g0, long long hi,
-                           const TileCarry& tc, bool have_tc, u32& need) {
+                           const TileCarry& tc, bool have_tc, u32& need, bool single_digits = false) {
     const u64 OWN = 0xFFFFull << 16;
     const u64 lead = tt_win(sm, F_LEAD, slot);
     const u64 L = tt_win(sm, F_LOW, slot) | tt_win(sm, F_UPP, slot) | tt_win(sm, F_CLESS, slot);
@@ -168,8 +168,9 @@ TT_HD u32 tt_eval_chunk_p0(const u16 (*sm)[TT_SLOTS], int slot, const u8* base, 
             if (same_doc) S |= at & L & lead;
         }
     }
-    // number runs: every third number lead counted from the run start
-    {
+    // number runs: every third number lead counted from the run start (single-digit variant: every lead)
+    if (single_digits) S |= N & lead;
+    else {
         u32 n_own = (u32)(N >> 16) & 0xFFFFu, ld_own = (u32)(lead >> 16) & 0xFFFFu;
         u32 nstart = (u32)((N & ~PREV(N)) >> 16) & 0xFFFFu;
         u32 m = n_own & ld_own;

@@ -132,7 +132,7 @@ __device__ u32 coop_back_num(const PretokParams& P, const ClassTables& T, long l
 __device__ u32 coop_back_nl(const PretokParams& P, const ClassTables& T, long long gend, long long* scratch) {
     const long long r = coop_back_run(P, T, gend, RUN_NL, scratch, nullptr);
     if (r & 1) return 0;
-    return ((r >> 1) & 1) | (P.pattern == 0 ? ((r >> 2) & 1) : 0);
+    return ((r >> 1) & 1) | (P.pattern != 1 ? ((r >> 2) & 1) : 0);
 }
 // Pattern 1: is the byte before gend a '/' run (or CR/LF run) that belongs to a punctuation tail?
 __device__ u32 coop_back_slash(const PretokParams& P, const ClassTables& T, long long gend, long long* scratch) {
@@ -206,7 +206,7 @@ k_pretok(const PretokParams P) {
     const int tid = threadIdx.x;
     // the 128-byte ASCII table is always staged; the two-stage Unicode table only once a tile holds a
     // non-ASCII byte (pattern 1 stages it at once: its sparse matcher may read beyond the tile)
-    bool tables_loaded = P.pattern != 0;
+    bool tables_loaded = P.pattern == 1;
     for (int i = tid * 16; i < P.cls_bytes; i += blockDim.x * 16)
         if (tables_loaded || i >= P.cls_bytes - 128)
             *reinterpret_cast<uint4*>(tables + i) = *reinterpret_cast<const uint4*>(P.cls_tables + i);
@@ -257,7 +257,7 @@ k_pretok(const PretokParams P) {
             store_slot(sm, s, tt_classify_chunk(P.base, chunk, P.nchunks, P.lo, P.hi, T), doc_bits(P, chunk));
         }
         __syncthreads();
-        if (P.pattern != 0) {                                          // sure starts / unresolved constructs per slot
+        if (P.pattern == 1) {                                          // sure starts / unresolved constructs per slot
             u32 su, ha;
             tt_sure_hard(sm, tid + TT_LOW_HALO, su, ha);
             sm[F_SURE][tid + TT_LOW_HALO] = (u16)su; sm[F_HARD][tid + TT_LOW_HALO] = (u16)ha;
@@ -271,7 +271,7 @@ k_pretok(const PretokParams P) {
         u32 need = 0;
         const int slot = tid + TT_LOW_HALO;
         const long long g0 = (c_first + tid) * TT_CHUNK;
-        u32 S = P.pattern == 0 ? tt_eval_chunk_p0(sm, slot, P.base, g0, P.hi, tc, false, need)
+        u32 S = P.pattern != 1 ? tt_eval_chunk_p0(sm, slot, P.base, g0, P.hi, tc, false, need, P.pattern == 2)
                                : tt_eval_chunk_p1(sm, slot, SC, g0, tc, false, need);
         if (need) atomicOr(&s_need, need);
         __syncthreads();
@@ -296,7 +296,7 @@ k_pretok(const PretokParams P) {
                 tc.sure_before = (ev & 1) ? (coop_back_event(P, T, (ev >> 1) + 1, true, scratch) >> 1) : (ev >> 1);
             }
             need = 0;
-            S = P.pattern == 0 ? tt_eval_chunk_p0(sm, slot, P.base, g0, P.hi, tc, true, need)
+            S = P.pattern != 1 ? tt_eval_chunk_p0(sm, slot, P.base, g0, P.hi, tc, true, need, P.pattern == 2)
                                : tt_eval_chunk_p1(sm, slot, SC, g0, tc, true, need);
         }
         if (c_first + tid < P.nchunks) P.startmask[c_first + tid] = (u16)S;

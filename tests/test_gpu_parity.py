@@ -285,3 +285,22 @@ def test_merge_kernels_on_random_tables(seed, n_merges, alpha):
         want = cv.bpe(d, 2)
         got = ids[ioff[k]:ioff[k + 1]]
         assert got.size == want.size and np.array_equal(got, want), (len(d), d[:40])
+
+
+def test_single_digit_pattern_variant():
+    """TT_PATTERN_CL100K_N1: pieces on exhaustive strings with digits, ids on config C2's text."""
+    import paper_2607_29678_b200 as tt
+    cfg = wl.CONFIGS["C2"]
+    merges, byte_map = wl.load_vocab(cfg)
+    gv = tt.Vocab(merges, byte_map, tt.TT_PATTERN_CL100K_N1)
+    docs = _alphabet_docs("a12 \t\n!'", 5) + _alphabet_docs("1²٣ a.", 5)
+    text = np.frombuffer(b"".join(docs), dtype=np.uint8)
+    off = np.zeros(len(docs) + 1, dtype=np.int64)
+    off[1:] = np.cumsum([len(d) for d in docs])
+    got, status = gpu_pretok(gv, text, doc_off=off)
+    want = np.concatenate([oracle.pretokenize(d, 2) + off[i] for i, d in enumerate(docs)])
+    assert status == 0 and np.array_equal(got, want)
+    big = wl.request(cfg)
+    ids, status = gpu_encode(gv, big)
+    want_ids, _ = cpu_vocab("C2").encode(big, 2, nthreads=4)
+    assert status == 0 and np.array_equal(ids, want_ids)

@@ -25,7 +25,6 @@ struct tt_vocab {
     int sm_count = 148;
     size_t n_merges = 0;
     u64* d_slots = nullptr;
-    u32 table_cap = 0;
     int32_t* d_ext_id = nullptr;
     u8* d_cls = nullptr;
     int cls_bytes = 0;
@@ -213,7 +212,7 @@ extern "C" int tt_vocab_load(const tt_merge* merges, size_t n_merges, const int3
     }
     tt_vocab* v = new (std::nothrow) tt_vocab();
     if (!v) return TT_ERR_CUDA;
-    v->pattern = pattern_id; v->n_merges = n_merges; v->table_cap = cap;
+    v->pattern = pattern_id; v->n_merges = n_merges;
     // class tables: stage1 | stage2 | ascii
     const int stage2_bytes = TT_CLS_NBLOCKS * 128;
     v->cls_bytes = (int)align_up(0x1100 + stage2_bytes, 16) + 128;
@@ -304,7 +303,7 @@ static int run_pretok(const tt_vocab* v, const uint8_t* text, size_t len, const 
         P.docmask = w.docmask;
     }
     const size_t smem = align_up(v->cls_bytes, 16) + sizeof(u16) * F_COUNT * TT_SLOTS;
-    const int grid = P.ntiles < v->sm_count * 4 ? P.ntiles : v->sm_count * 4;
+    const int grid = P.ntiles < v->sm_count * 6 ? P.ntiles : v->sm_count * 6;
     k_pretok<<<grid, TT_TILE_CHUNKS, smem, st>>>(P);
     if (piece_off_dst)
         k_compact<<<grid, TT_TILE_CHUNKS, 0, st>>>(w.startmask, w.tile_cnt, P.nchunks, P.ntiles, shift, (long long)len,

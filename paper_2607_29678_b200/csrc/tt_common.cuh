@@ -38,14 +38,10 @@ constexpr int TT_WARP_PIECE_MAX = 256;            // bytes; longer pieces take t
 struct TTHeader {
     int status;              // TT_OK or a device-side error code
     u32 pretok_done;         // CTAs that finished the pre-tokenization pass
-    u32 count_done;          // CTAs that finished the token-count reduction
+    u32 count_done;          // CTAs that finished the piece kernel
     u32 n_pieces;            // number of pieces found
-    u32 n_long;              // entries in the long-piece list
-    u32 long_next;           // work counter of the long-piece kernel
-    u32 piece_next;          // work counter of the warp BPE kernel
-    u32 n_miss;              // entries in the miss list (pieces that need the merge loop)
     unsigned long long n_tokens;   // total tokens
-    u32 pad[22];
+    u32 pad[26];
 };
 static_assert(sizeof(TTHeader) == 128, "header layout");
 

@@ -194,7 +194,7 @@ __device__ __forceinline__ void store_slot(u16 (*sm)[TT_SLOTS], int s, const Chu
     sm[F_NL][s] = m.nl; sm[F_SP][s] = m.sp; sm[F_AP][s] = m.ap; sm[F_SL][s] = m.sl; sm[F_DOC][s] = (u16)d;
 }
 
-__global__ void __launch_bounds__(TT_TILE_CHUNKS)
+__global__ void __launch_bounds__(TT_TILE_CHUNKS, 6)
 k_pretok(const PretokParams P) {
     extern __shared__ __align__(16) u8 smem_raw[];
     u8* tables = smem_raw;                                            // class tables

@@ -38,10 +38,6 @@ TT_HD SeqChar tt_seq_char(const SeqCtx& C, long long g, long long end) {
     r.cls = tt_class_of(cp, C.T); r.byte = 0x100; r.len = n < 1 ? 1 : n;
     return r;
 }
-TT_HD bool tt_seq_is_doc_start(const SeqCtx& C, long long g) {
-    if (C.docmask) return (C.docmask[g >> 5] >> (g & 31)) & 1;
-    return g == C.lo;
-}
 TT_HD bool tt_cls_word(u32 c) { return c == CC_LOWER || c == CC_UPPER || c == CC_CASELESS || c == CC_MARK; }
 TT_HD bool tt_cls_up(u32 c) { return c == CC_UPPER || c == CC_CASELESS || c == CC_MARK; }      // U
 TT_HD bool tt_cls_lw(u32 c) { return c == CC_LOWER || c == CC_CASELESS || c == CC_MARK; }      // Lw

@@ -304,3 +304,37 @@ def test_single_digit_pattern_variant():
     ids, status = gpu_encode(gv, big)
     want_ids, _ = cpu_vocab("C2").encode(big, 2, nthreads=4)
     assert status == 0 and np.array_equal(ids, want_ids)
+
+
+@pytest.mark.parametrize("pattern", [0, 1, 2])
+def test_random_unicode_documents(pattern):
+    """Documents of random code points from every plane (plus the ASCII constructs the rules care about),
+    each encoded as its own document of one batch call: piece boundaries against the oracle."""
+    import paper_2607_29678_b200 as tt
+    rng = random.Random(2024 + pattern)
+    merges, byte_map = wl.load_vocab(wl.CONFIGS["C1"])
+    gv = tt.Vocab(merges, byte_map, pattern)
+    special = list(" \t\n\r'/!.,1aZ") + ["'s", "'re", "'LL", "\r\n", "  ", "\n\n", "12345", "́", "　", " "]
+    ranges = [(0x20, 0x7F), (0xA0, 0x250), (0x300, 0x370), (0x370, 0x530), (0x600, 0x700), (0x900, 0xA00), (0x2000, 0x2070),
+              (0x3000, 0x3100), (0x4E00, 0x4F00), (0xAC00, 0xAD00), (0xFF00, 0xFFF0), (0x1D400, 0x1D500), (0x1F300, 0x1F700)]
+    docs = []
+    for _ in range(6000):
+        n = rng.randrange(1, 60)
+        parts = []
+        for _ in range(n):
+            if rng.random() < 0.45:
+                parts.append(rng.choice(special))
+            else:
+                lo, hi = rng.choice(ranges)
+                parts.append(chr(rng.randrange(lo, hi)))
+        docs.append("".join(parts).encode("utf-8"))
+    text = np.frombuffer(b"".join(docs), dtype=np.uint8)
+    off = np.zeros(len(docs) + 1, dtype=np.int64)
+    off[1:] = np.cumsum([len(d) for d in docs])
+    got, status = gpu_pretok(gv, text, doc_off=off)
+    assert status == 0
+    want = np.concatenate([oracle.pretokenize(d, pattern) + off[i] for i, d in enumerate(docs)])
+    if got.size != want.size or not np.array_equal(got, want):
+        bad = sorted(set(got.tolist()) ^ set(want.tolist()))[:3]
+        which = [int(np.searchsorted(off, b, side="right") - 1) for b in bad]
+        raise AssertionError(f"piece mismatch in documents {[docs[w] for w in which]}")

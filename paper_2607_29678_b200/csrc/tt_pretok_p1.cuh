@@ -21,6 +21,7 @@ struct SeqCtx {                 // what the sequential matcher needs to read the
     long long lo, hi;
     const u32* docmask;         // or null: one document
     ClassTables T;
+    mutable long long reach;    // highest text position (exclusive) a match has examined so far
 };
 
 // ---- sequential matcher over the raw text (sparse path) ---------------------------------------------
@@ -29,9 +30,10 @@ struct SeqChar { u32 cls; u32 byte; int len; };   // byte = the ASCII byte, or 0
 TT_HD SeqChar tt_seq_char(const SeqCtx& C, long long g, long long end) {
     SeqChar r;
     u32 b = C.base[g];
-    if (b < 0x80) { r.cls = C.T.ascii[b] & 7; r.byte = b; r.len = 1; return r; }
+    if (b < 0x80) { r.cls = C.T.ascii[b] & 7; r.byte = b; r.len = 1; if (g + 1 > C.reach) C.reach = g + 1; return r; }
     int n = b >= 0xF0 ? 4 : b >= 0xE0 ? 3 : 2;
     if (g + n > end) n = (int)(end - g);
+    if (g + n > C.reach) C.reach = g + n;
     u32 cp = b & (0x7Fu >> (b >= 0xF0 ? 4 : b >= 0xE0 ? 3 : 2));
     for (int k = 1; k < n; k++) cp = (cp << 6) | (C.base[g + k] & 0x3F);
     if (cp > 0x10FFFF) cp = 0xFFFD;                  // malformed input: the result is discarded anyway
@@ -86,6 +88,7 @@ TT_HD long long tt_seq_match_p1(const SeqCtx& C, long long p, long long end) {
         if (v > p) e = v;
     }
     if (e >= 0) {
+        if (e + 3 > end) C.reach = end;
         if (e < end && C.base[e] == '\'') {
             u32 b1 = e + 1 < end ? C.base[e + 1] : 0, b2 = e + 2 < end ? C.base[e + 2] : 0;
             e += tt_contraction_len(b1, b2);
@@ -103,6 +106,7 @@ TT_HD long long tt_seq_match_p1(const SeqCtx& C, long long p, long long end) {
     if (q >= 0) {
         while (q < end) { SeqChar ch = tt_seq_char(C, q, end); if (!tt_cls_punct(ch.cls)) break; q += ch.len; }
         while (q < end) { u32 b = C.base[q]; if (b != '\n' && b != '\r' && b != '/') break; q++; }
+        if (q + 1 > C.reach) C.reach = q + 1 < end ? q + 1 : end;
         return q;
     }
     // whitespace: \s*[\r\n]+ | \s+(?!\S) | \s+
@@ -119,29 +123,50 @@ TT_HD long long tt_seq_match_p1(const SeqCtx& C, long long p, long long end) {
     return t > p ? t : p + c0.len;
 }
 
+// First document start in [g, lim), or lim when there is none.
+TT_HD long long tt_next_doc_start(const u32* docmask, long long g, long long lim) {
+    while (g < lim) {
+        const u32 w = docmask[g >> 5] >> (g & 31);
+        if (w) { g += tt_lobit(w); break; }
+        g = ((g >> 5) + 1) << 5;
+    }
+    return g < lim ? g : lim;
+}
+
 // Piece starts inside [g0, g0+16) obtained by matching sequentially from the piece start `from`
-// (from <= g0 + 15).  Returns a 16-bit mask; bits below `from` are not produced.
+// (from <= g0 + 15).  Returns a 16-bit mask; bits below `from` are not produced.  The end of the
+// document that contains `from` is looked up only as far as the matches look: the search begins with a
+// provisional end a little past the chunk, and a match that examined the provisional end is repeated
+// with the end moved out geometrically (documents can be megabytes long; pieces rarely are).
+// doc_end returns an end that is exact whenever it is below g0 + 16.
 TT_HD u32 tt_seq_starts_p1(const SeqCtx& C, long long from, long long g0, long long& doc_end) {
     long long end = C.hi;
-    if (C.docmask) {                                   // end of the document that contains `from`
-        long long g = from + 1;
-        // look for the next document start, one 32-bit word at a time
-        while (g < C.hi) {
-            u32 w = C.docmask[g >> 5] >> (g & 31);
-            if (w) { g += tt_lobit(w); break; }
-            g = ((g >> 5) + 1) << 5;
-        }
-        end = g < C.hi ? g : C.hi;
+    bool exact = true;
+    if (C.docmask) {
+        long long cap = g0 + TT_CHUNK + 64;
+        if (cap > C.hi) cap = C.hi;
+        end = tt_next_doc_start(C.docmask, from + 1, cap);
+        exact = end < cap || cap == C.hi;
     }
-    doc_end = end;
     u32 bits = 0;
     long long p = from;
-    const long long stop = g0 + TT_CHUNK < end ? g0 + TT_CHUNK : end;
-    while (p < stop) {
+    for (;;) {
+        const long long stop = g0 + TT_CHUNK < end ? g0 + TT_CHUNK : end;
+        if (p >= stop) break;
+        C.reach = 0;
+        const long long e = tt_seq_match_p1(C, p, end);
+        if (!exact && C.reach >= end) {                // looked at the provisional end: move it out, match again
+            long long cap = end + 4 * (end - from);
+            if (cap > C.hi) cap = C.hi;
+            const long long ne = tt_next_doc_start(C.docmask, end, cap);
+            exact = ne < cap || cap == C.hi;
+            end = ne;
+            continue;
+        }
         if (p >= g0) bits |= 1u << (int)(p - g0);
-        long long e = tt_seq_match_p1(C, p, end);
         p = e > p ? e : p + 1;
     }
+    doc_end = end;
     return bits;
 }
 
@@ -156,7 +181,8 @@ TT_HD ChunkDoc tt_load_slot(const u16 (*sm)[TT_SLOTS], int s) {
     return c;
 }
 // p = previous chunk, c = the chunk, n = next chunk
-TT_HD void tt_sure_hard_cm(const ChunkDoc& p, const ChunkDoc& c, const ChunkDoc& n, u32& sure, u32& hard) {
+// upcl: the unresolved constructs of the second kind (upper-case letter after a caseless letter), a subset of hard
+TT_HD void tt_sure_hard_cm(const ChunkDoc& p, const ChunkDoc& c, const ChunkDoc& n, u32& sure, u32& hard, u32& upcl) {
     // 20-bit frame: bits 0..2 = last three bytes of the previous chunk, bits 3..18 = the chunk, bit 19 = first byte of the next
 #define FR(x) ((((u32)p.x) >> 13) | (((u32)c.x) << 3) | ((((u32)n.x) & 1u) << 19))
     const u32 lead = FR(m.lead), D = FR(doc);
@@ -164,17 +190,77 @@ TT_HD void tt_sure_hard_cm(const ChunkDoc& p, const ChunkDoc& c, const ChunkDoc&
     const u32 nD = ~D;
     const u32 pLr = (Lr << 1) & nD, pN = (N << 1) & nD, pNL = (FR(m.nl) << 1) & nD, pCl = (FR(m.cless) << 1) & nD;
     const u32 nLr = (Lr >> 1) & ~(D >> 1);
-    const u32 cs = D | (N & ~pN) | (W & (pLr | pN)) | (O & ~AP & (pLr | pN)) | (Lr & (pN | pNL));
+    // a one-byte blank right before a letter is the letter's prefix whatever precedes it; a letter after two
+    // punctuation characters (the nearer one a single byte, the farther one no slash, which a tail could have
+    // taken) follows a punctuation piece that ends there
+    const u32 blank_pfx = W & ~FR(m.nl) & lead & (lead >> 1) & (Lr >> 1) & ~(D >> 1);
+    const u32 after_oo = Lr & ((O & lead) << 1) & ((O & ~FR(m.sl)) << 2) & nD & ~(D << 1);
+    const u32 cs = D | (N & ~pN) | (W & (pLr | pN)) | (O & (pN | (~AP & pLr))) | (Lr & (pN | pNL)) | blank_pfx | after_oo;
     // an apostrophe between letters is a possible contraction suffix; it is decided locally unless another
     // apostrophe two or three bytes before it may have consumed the letter in front of it
-    const u32 h = FR(m.mark) | (FR(m.upp) & pCl) | (AP & pLr & nLr & ((AP << 2) | (AP << 3)));
+    const u32 h2 = FR(m.upp) & pCl;
+    const u32 h = FR(m.mark) | h2 | (AP & pLr & nLr & ((AP << 2) | (AP << 3)));
 #undef FR
     sure = ((cs & lead) >> 3) & 0xFFFFu;
     hard = ((h & lead) >> 3) & 0xFFFFu;
+    upcl = ((h2 & lead) >> 3) & 0xFFFFu;
 }
-// Valid for 1 <= s <= TT_SLOTS - 2 (needs the neighbouring slots).
+TT_HD void tt_sure_hard_cm(const ChunkDoc& p, const ChunkDoc& c, const ChunkDoc& n, u32& sure, u32& hard) {
+    u32 upcl;
+    tt_sure_hard_cm(p, c, n, sure, hard, upcl);
+}
+
+// An upper-case letter (bit i of slot s) that follows a caseless letter, decided from the class masks of
+// the tile: 1 = it starts a piece, 0 = it does not, -1 = left to the sparse path.
+//   Going left over the caseless letters: a lower-case letter means the letters in between continue its
+//   lower-case stretch, which stops at the upper-case letter, so that one starts a piece (unless the
+//   lower-case letter may belong to a contraction suffix, which begins a word body of its own).  An
+//   upper-case letter, a non-letter or a document start means the word body has held no lower-case
+//   letter so far; its leading stretch then runs to the first lower-case letter or to the end of the
+//   letter run, and only in the second case is it cut, after its last caseless letter: the upper-case
+//   letter starts a piece exactly when only upper-case letters follow up to the end of the run.
+//   A mark at either end of the look leaves the case to the sparse path, and so does leaving the tile.
+TT_HD int tt_resolve_upper_after_caseless(const u16 (*sm)[TT_SLOTS], int s, int i) {
+    u32 keep = (1u << i) - 1;
+    for (int t = s;; t--, keep = 0xFFFFu) {
+        if (t < 0) return -1;
+        const u32 c = sm[F_CLESS][t], d = sm[F_DOC][t];
+        const u32 stop = ((~c & 0xFFFFu) | d) & keep;
+        if (!stop) continue;
+        const int k = tt_hibit(stop);
+        if ((c >> k) & 1) break;                                  // a caseless letter that starts a document
+        if ((sm[F_MARK][t] >> k) & 1) return -1;
+        if ((sm[F_LOW][t] >> k) & 1) {
+            const u32 ap = ((u32)sm[F_AP][t] << 16) | (t > 0 ? (u32)sm[F_AP][t - 1] : 0xFFFFu);
+            if ((ap >> (14 + k)) & 3) return -1;                  // apostrophe one or two bytes before it
+            return 1;
+        }
+        break;
+    }
+    keep = ~((2u << i) - 1) & 0xFFFFu;
+    for (int t = s;; t++, keep = 0xFFFFu) {
+        if (t >= TT_SLOTS) return -1;
+        const u32 u = sm[F_UPP][t], d = sm[F_DOC][t];
+        const u32 stop = ((~u & 0xFFFFu) | d) & keep;
+        if (!stop) continue;
+        const int k = tt_lobit(stop);
+        if ((d >> k) & 1) return 1;
+        if ((sm[F_MARK][t] >> k) & 1) return -1;
+        return (((u32)sm[F_LOW][t] | sm[F_CLESS][t]) >> k) & 1 ? 0 : 1;
+    }
+}
+
+// Valid for 1 <= s <= TT_SLOTS - 2 (needs the neighbouring slots).  Unresolved constructs of the second
+// kind that the tile's masks decide leave `hard`; those that start a piece join `sure`.
 TT_HD void tt_sure_hard(const u16 (*sm)[TT_SLOTS], int s, u32& sure, u32& hard) {
-    tt_sure_hard_cm(tt_load_slot(sm, s - 1), tt_load_slot(sm, s), tt_load_slot(sm, s + 1), sure, hard);
+    u32 upcl;
+    tt_sure_hard_cm(tt_load_slot(sm, s - 1), tt_load_slot(sm, s), tt_load_slot(sm, s + 1), sure, hard, upcl);
+    while (upcl) {
+        const int i = tt_lobit(upcl);
+        upcl &= upcl - 1;
+        const int r = tt_resolve_upper_after_caseless(sm, s, i);
+        if (r >= 0) { hard &= ~(1u << i); sure |= (u32)r << i; }
+    }
 }
 
 // Walks down from slot s over the precomputed F_SURE / F_HARD masks (valid for slots >= 1): is the
@@ -359,7 +445,7 @@ TT_HD u32 tt_eval_chunk_p1(const u16 (*sm)[TT_SLOTS], int slot, const SeqCtx& C,
         dirty = F;
     }
     u32 pending = (u32)((dirty & OWN & V) >> 32) & 0xFFFFu;
-    u32 res = (u32)((S & lead & OWN) >> 32) & 0xFFFFu;
+    u32 res = (u32)(((S | sure) & lead & OWN) >> 32) & 0xFFFFu;     // sure starts include the decided case boundaries
     while (pending) {
         // re-derive from the last sure start at or below the first unresolved byte, up to the end of
         // the chunk or of the document, whichever comes first

@@ -338,3 +338,31 @@ def test_random_unicode_documents(pattern):
         bad = sorted(set(got.tolist()) ^ set(want.tolist()))[:3]
         which = [int(np.searchsorted(off, b, side="right") - 1) for b in bad]
         raise AssertionError(f"piece mismatch in documents {[docs[w] for w in which]}")
+
+
+def test_cjk_latin_mixtures_in_long_documents():
+    """Pattern 1 on caseless-script text with glued upper/lower-case words, marks and contraction chains,
+    in documents far longer than a tile: the case-boundary decisions taken from the class masks, the
+    sparse matcher behind them and its search for the document end (long pieces next to unresolved
+    constructs, documents that end inside such pieces).  Piece boundaries and IDs against the oracle."""
+    rng = random.Random(4242)
+    atoms = ["中", "文", "使用", "手机", "A", "B", "GPU", "App", "iPhone", "a", "word", "'", "'s", "'T", " ", "  ", "，", "。",
+             "!", "!!", "/", "\n", "1", "2024", "́", "é", "É", "ǅ", "ʰ", "\t", "x's's's"]
+    w = [10, 10, 5, 5, 5, 3, 3, 2, 2, 3, 2, 1, 1, 1, 2, 1, 2, 1, 0.5, 0.5, 0.5, 0.5, 1, 0.5, 0.2, 1, 1, 0.3, 0.3, 0.3, 0.2]
+    long_runs = ["中", " ", "A", "a", "9", "\n", "=", "文B", " \t"]
+    docs = []
+    for _ in range(40):
+        parts = []
+        for _ in range(rng.randrange(200, 4000)):
+            if rng.random() < 0.004:
+                parts.append(rng.choice(long_runs) * rng.randrange(40, 6000))
+            else:
+                parts.append(rng.choices(atoms, w)[0])
+        docs.append("".join(parts).encode("utf-8"))
+    _batch_pieces_check("C4", 1, docs)
+    text = np.frombuffer(b"".join(docs), dtype=np.uint8)
+    off = np.zeros(len(docs) + 1, dtype=np.int64)
+    off[1:] = np.cumsum([len(d) for d in docs])
+    ids, ioff, status = gpu_encode_batch(gpu_vocab("C4"), text, off)
+    want, woff = cpu_vocab("C4").encode_batch(text, off, 1, nthreads=8)
+    assert status == 0 and np.array_equal(ioff, woff) and np.array_equal(ids, want)

@@ -25,6 +25,7 @@ struct tt_vocab {
     int sm_count = 148;
     size_t n_merges = 0;
     u64* d_slots = nullptr;
+    u32* d_bytepair = nullptr;
     int32_t* d_ext_id = nullptr;
     u8* d_cls = nullptr;
     int cls_bytes = 0;
@@ -69,7 +70,7 @@ extern "C" size_t tt_class_table(uint8_t* out, size_t cap) {
 
 extern "C" void tt_vocab_free(tt_vocab* v) {
     if (!v) return;
-    cudaFree(v->d_slots); cudaFree(v->d_ext_id); cudaFree(v->d_cls); cudaFree(v->d_tokslots); cudaFree(v->d_meta);
+    cudaFree(v->d_slots); cudaFree(v->d_bytepair); cudaFree(v->d_ext_id); cudaFree(v->d_cls); cudaFree(v->d_tokslots); cudaFree(v->d_meta);
     cudaFree(v->d_text); cudaFree(v->d_ids); cudaFree(v->d_count); cudaFree(v->d_status); cudaFree(v->d_ws);
     if (v->h_text) cudaFreeHost(v->h_text);
     if (v->h_ids) cudaFreeHost(v->h_ids);
@@ -126,6 +127,7 @@ static int build_token_table(tt_vocab* v, const tt_merge* merges, size_t n_merge
     ok = ok && cudaMemcpy(d_tb, tile_base.data(), (ntiles + 1) * sizeof(u32), cudaMemcpyHostToDevice) == cudaSuccess;
     ok = ok && cudaMemcpy(d_tf, tile_first.data(), (ntiles + 1) * sizeof(u32), cudaMemcpyHostToDevice) == cudaSuccess;
     ok = ok && cudaMemcpy(d_hdr, &h, sizeof(h), cudaMemcpyHostToDevice) == cudaSuccess;
+    ok = ok && cudaMemset(d_tt, 0, (ntiles + 1) * sizeof(u32)) == cudaSuccess;
     if (ok) {
         PieceParams Q;
         Q.base = d_text; Q.shift = 0; Q.hi = (long long)nb; Q.nchunks = (long long)nchunks; Q.ntiles = (int)ntiles;
@@ -189,6 +191,7 @@ extern "C" int tt_vocab_load(const tt_merge* merges, size_t n_merges, const int3
     while ((1u << log2b) < nbuckets) log2b++;
     const u32 cap = 4 * nbuckets;
     std::vector<u64> slots(cap, TT_SLOT_EMPTY);
+    std::vector<u32> bytepair(65536, TT_RANK_INF);      // ranks of the byte-byte pairs, directly indexed
     const u32 mask = nbuckets - 1, shift = 32 - log2b;
     std::unordered_set<u64> seen;
     seen.reserve(2 * n_merges + 16);
@@ -199,6 +202,7 @@ extern "C" int tt_vocab_load(const tt_merge* merges, size_t n_merges, const int3
         if (m.result < 0 || internal.count(m.result)) return TT_ERR_BAD_VOCAB;         // result id reused
         const u64 key = ((u64)l->second << TT_ID_BITS) | rr->second;
         if (!seen.insert(key).second) return TT_ERR_BAD_VOCAB;                         // duplicate pair
+        if (l->second < 256 && rr->second < 256) bytepair[(l->second << 8) | rr->second] = (u32)r;
         u32 h = pair_bucket(key, shift);
         for (;;) {
             u64* b = &slots[4 * (size_t)h];
@@ -223,13 +227,15 @@ extern "C" int tt_vocab_load(const tt_merge* merges, size_t n_merges, const int3
     bool ok = cudaGetDevice(&v->device) == cudaSuccess;
     ok = ok && cudaDeviceGetAttribute(&v->sm_count, cudaDevAttrMultiProcessorCount, v->device) == cudaSuccess;
     ok = ok && cudaMalloc(&v->d_slots, (size_t)cap * sizeof(u64)) == cudaSuccess;
+    ok = ok && cudaMalloc(&v->d_bytepair, bytepair.size() * sizeof(u32)) == cudaSuccess;
+    ok = ok && cudaMemcpy(v->d_bytepair, bytepair.data(), bytepair.size() * sizeof(u32), cudaMemcpyHostToDevice) == cudaSuccess;
     ok = ok && cudaMalloc(&v->d_ext_id, ext_id.size() * sizeof(int32_t)) == cudaSuccess;
     ok = ok && cudaMalloc(&v->d_cls, v->cls_bytes) == cudaSuccess;
     ok = ok && cudaMemcpy(v->d_slots, slots.data(), (size_t)cap * sizeof(u64), cudaMemcpyHostToDevice) == cudaSuccess;
     ok = ok && cudaMemcpy(v->d_ext_id, ext_id.data(), ext_id.size() * sizeof(int32_t), cudaMemcpyHostToDevice) == cudaSuccess;
     ok = ok && cudaMemcpy(v->d_cls, cls.data(), v->cls_bytes, cudaMemcpyHostToDevice) == cudaSuccess;
     if (!ok) { cudaGetLastError(); tt_vocab_free(v); return TT_ERR_CUDA; }
-    v->tab.slots = v->d_slots; v->tab.mask = mask; v->tab.shift = shift;
+    v->tab.slots = v->d_slots; v->tab.bytepair = v->d_bytepair; v->tab.mask = mask; v->tab.shift = shift;
     if (build_token_table(v, merges, n_merges, ext_id) != TT_OK) { tt_vocab_free(v); return TT_ERR_CUDA; }
     {   // byte length and number of non-continuation bytes of every token, indexed by the caller's id
         std::vector<uint2> in(256 + n_merges);
@@ -294,7 +300,7 @@ static int run_pretok(const tt_vocab* v, const uint8_t* text, size_t len, const 
     P.ntiles = (int)((P.nchunks + TT_TILE_CHUNKS - 1) / TT_TILE_CHUNKS);
     P.pattern = v->pattern;
     P.docmask = nullptr;
-    P.startmask = w.startmask; P.tile_cnt = w.tile_cnt; P.tile_first = w.tile_first; P.hdr = w.hdr;
+    P.startmask = w.startmask; P.tile_cnt = w.tile_cnt; P.tile_first = w.tile_first; P.tile_tok = w.tile_tok; P.hdr = w.hdr;
     P.cls_tables = v->d_cls; P.cls_bytes = v->cls_bytes;
     if (doc_off) {
         CK(cudaMemsetAsync(w.docmask, 0, ((size_t)P.hi / 32 + 4) * sizeof(u32), st));

@@ -7,6 +7,8 @@
 //   * a thread per piece looks the whole piece up as a vocabulary entry (one 32-byte probe);
 //   * pieces that are not a single entry are merged by a warp (<= 32 bytes: tokens in registers,
 //     candidates as ballot masks; <= 256 bytes: several tokens per lane, compaction through shared memory);
+//     where a CTA has many such pieces of <= 32 bytes waiting (text dense in pieces outside the vocabulary,
+//     or many tiles per CTA), it merges 128 of them at once, one thread per piece (lane_merge);
 //   * longer pieces are merged by the whole CTA (cta_merge_long: state in shared memory, or in global
 //     scratch while the piece still has more than 4,096 tokens).
 // Token ids inside the kernels are "internal": byte b -> b, result of the merge of rank r -> 256 + r;
@@ -20,6 +22,7 @@
 // slot ends the search.  Sized for at most one key per bucket on average.
 struct PairTable {
     const u64* slots;     // 4 * (mask + 1) slots
+    const u32* bytepair;  // rank of the pair (byte a, byte b) at [a << 8 | b], TT_RANK_INF if none: a piece's first probes
     u32 mask;             // number of buckets - 1 (power of two)
     u32 shift;            // 32 - log2(number of buckets)
 };
@@ -138,7 +141,7 @@ __device__ __forceinline__ u32 warp_merge_reg(const u8* __restrict__ text, u32 a
                                               const int32_t* __restrict__ ext_id, int32_t* __restrict__ stage, int lane) {
     const u32 t = (u32)lane < n ? text[a + lane] : 0;
     const u32 tn = __shfl_down_sync(0xFFFFFFFFu, t, 1);
-    const u32 r = ((u32)lane + 1 < n) ? pair_probe(tab, t, tn) : TT_RANK_INF;
+    const u32 r = ((u32)lane + 1 < n) ? __ldg(tab.bytepair + ((t << 8) | tn)) : TT_RANK_INF;
     return warp_merge_reg_rounds(t, r, n, n, a, tab, ext_id, stage, lane);
 }
 
@@ -164,7 +167,7 @@ __device__ __forceinline__ u32 warp_merge_perm(u64* buf /* 2 * 32 * E entries of
 #pragma unroll
     for (int j = 0; j < E; j++) {
         const u32 k = j * 32 + lane;
-        r[j] = (k + 1 < n) ? pair_probe(tab, t[j], (u32)buf[k + 1]) : TT_RANK_INF;
+        r[j] = (k + 1 < n) ? __ldg(tab.bytepair + ((t[j] << 8) | (u32)buf[k + 1])) : TT_RANK_INF;
     }
     int cur = 0;
     for (u32 round = 0; round < n; round++) {          // at most n - 1 merges
@@ -226,6 +229,94 @@ __device__ __forceinline__ u32 warp_merge_perm(u64* buf /* 2 * 32 * E entries of
         const u32 k = j * 32 + lane;
         if (k < m) stage[a + k] = ext_id[t[j]];
     }
+    return m;
+}
+
+// ---- a thread per piece, <= 32 bytes: tokens and pair ranks in shared memory ------------------------------
+// Paper Sec. 4.2 gives the shortest length class to single threads.  Here a warp per piece has the shorter
+// dependent chain (one probe latency per round for the whole piece), so it serves a request's few
+// unmatched pieces; a thread per piece keeps 32 independent chains per warp in flight and issues an order
+// of magnitude fewer instructions per piece, so it serves bulk text.  Same rounds as everywhere: the
+// minimum rank of the piece, all its leftmost non-overlapping occurrences, new probes only next to a merge.
+// Column s of tok[LANE_MAX][LANE_SLOTS] / rk[LANE_MAX][LANE_SLOTS]: any two threads of a warp hit
+// different banks whatever rows they are at.
+constexpr int LANE_SLOTS = 128;                       // pieces merged at once
+constexpr int LANE_MAX = 32;                          // bytes per piece on this path
+constexpr u32 LANE_MIN_PIECES = 33;                   // fewer pieces left after a CTA's last tile get a warp each instead
+// Two independent probes with both first-bucket loads in flight together.
+__device__ __forceinline__ u32 pair_match_first(const PairTable& t, const uint4 lo, const uint4 hi, u64 key) {
+    const u64 s0 = ((u64)lo.y << 32) | lo.x, s1 = ((u64)lo.w << 32) | lo.z, s2 = ((u64)hi.y << 32) | hi.x, s3 = ((u64)hi.w << 32) | hi.z;
+    if ((s0 >> 20) == key) return (u32)(s0 & 0xFFFFFu);
+    if ((s1 >> 20) == key) return (u32)(s1 & 0xFFFFFu);
+    if ((s2 >> 20) == key) return (u32)(s2 & 0xFFFFFu);
+    if ((s3 >> 20) == key) return (u32)(s3 & 0xFFFFFu);
+    if (s3 == TT_SLOT_EMPTY) return TT_RANK_INF;
+    return pair_probe(t, (u32)(key >> TT_ID_BITS), (u32)(key & (TT_MAX_INTERNAL - 1)));     // full bucket: walk the chain
+}
+__device__ __forceinline__ void pair_probe2(const PairTable& t, u32 a0, u32 b0, u32 a1, u32 b1, u32& r0, u32& r1) {
+    const u64 key0 = ((u64)a0 << TT_ID_BITS) | b0, key1 = ((u64)a1 << TT_ID_BITS) | b1;
+    const uint4* p0 = reinterpret_cast<const uint4*>(t.slots + 4 * (size_t)pair_bucket(key0, t.shift));
+    const uint4* p1 = reinterpret_cast<const uint4*>(t.slots + 4 * (size_t)pair_bucket(key1, t.shift));
+    const uint4 x0 = __ldg(p0), y0 = __ldg(p0 + 1), x1 = __ldg(p1), y1 = __ldg(p1 + 1);
+    r0 = pair_match_first(t, x0, y0, key0);
+    r1 = pair_match_first(t, x1, y1, key1);
+}
+
+// Tokens stay at the byte position where they began; `al` has a bit per position that still holds a
+// token, and the rank of a pair is kept at its left position, so a merge moves nothing: it rewrites the
+// left token, clears the partner's bit and marks the two pairs that changed for a new probe.
+__device__ __forceinline__ u32 lane_merge(u32* __restrict__ tok, u32* __restrict__ rk, int s, const u8* __restrict__ text, u32 a, u32 n,
+                                          const PairTable& tab, const int32_t* __restrict__ ext_id, int32_t* __restrict__ stage) {
+#define TK(k) tok[(k) * LANE_SLOTS + s]
+#define RK(k) rk[(k) * LANE_SLOTS + s]
+    u32 prev = text[a];
+    TK(0) = prev;
+#pragma unroll 4
+    for (u32 k = 1; k < n; k++) {
+        const u32 t = text[a + k];
+        TK(k) = t;
+        RK(k - 1) = __ldg(tab.bytepair + ((prev << 8) | t));
+        prev = t;
+    }
+    u32 al = 0xFFFFFFFFu >> (32 - n);
+    u32 stale = 0;
+    for (u32 round = 0; round < n; round++) {
+        while (stale) {                                   // every thread of the warp walks its own list in step
+            const u32 k0 = __ffs(stale) - 1;
+            stale &= stale - 1;
+            const u32 k1 = stale ? __ffs(stale) - 1 : k0;
+            stale &= stale - 1;
+            const u32 up0 = al & (0xFFFFFFFEu << k0), up1 = al & (0xFFFFFFFEu << k1);
+            u32 r0 = TT_RANK_INF, r1 = TT_RANK_INF;         // (a position without a token above it has no pair)
+            pair_probe2(tab, TK(k0), up0 ? TK(__ffs(up0) - 1) : 0u, TK(k1), up1 ? TK(__ffs(up1) - 1) : 0u, r0, r1);
+            RK(k0) = up0 ? r0 : TT_RANK_INF;
+            RK(k1) = up1 ? r1 : TT_RANK_INF;
+        }
+        u32 mn = TT_RANK_INF, c = 0;
+        for (u32 x = al & ~(0x80000000u >> __clz(al)); x; x &= x - 1) {      // every position but the topmost
+            const u32 k = __ffs(x) - 1;
+            const u32 r = RK(k);
+            if (r < mn) { mn = r; c = 0; }
+            c |= (r == mn ? 1u : 0u) << k;
+        }
+        if (mn == TT_RANK_INF) break;
+        const u32 nt = 256u + mn;
+        u32 blocked = 32;
+        for (u32 x = c; x; x &= x - 1) {                  // leftmost non-overlapping occurrences, ascending
+            const u32 k = __ffs(x) - 1;
+            if (k == blocked) continue;                   // its token went into the merge before it
+            const u32 p = __ffs(al & (0xFFFFFFFEu << k)) - 1;
+            TK(k) = nt;
+            al &= ~(1u << p);
+            blocked = p;
+            const u32 below = al & ((1u << k) - 1);
+            stale |= (1u << k) | (below ? 0x80000000u >> __clz(below) : 0u);
+        }
+    }
+    u32 m = 0;
+    for (u32 x = al; x; x &= x - 1) stage[a + m++] = ext_id[TK(__ffs(x) - 1)];
+#undef TK
+#undef RK
     return m;
 }
 
@@ -363,7 +454,7 @@ __device__ u32 cta_merge_long(const u8* __restrict__ text, u32 a, u32 n, const P
     __syncthreads();
     for (u32 i = tid; i < n; i += T) {
         const u32 t0 = text[a + i];
-        const u32 r = (i + 1 < n) ? pair_probe(tab, t0, text[a + i + 1]) : TT_RANK_INF;
+        const u32 r = (i + 1 < n) ? __ldg(tab.bytepair + ((t0 << 8) | text[a + i + 1])) : TT_RANK_INF;
         arr[i] = ((u64)r << 32) | t0;
     }
     __syncthreads();
@@ -417,9 +508,12 @@ __device__ void tile_pieces(TilePieces& tp, const u16* __restrict__ startmask, c
 
 // ---- K4 (+ the scan of K5): all pieces of a text tile -----------------------------------------------------------
 // Phase 1: a thread per piece (one-byte pieces map directly, pieces of up to 24 bytes are looked up as
-// whole vocabulary entries).  Phase 2: the CTA's warps merge the pieces phase 1 could not settle; pieces
-// longer than TT_WARP_PIECE_MAX are merged by the whole CTA.  Phase 3: the tile's token total; the last
-// CTA to finish turns the tile totals into their exclusive prefix and checks the output capacity.
+// whole vocabulary entries).  Phase 2: the CTA's warps merge the pieces of 33..256 bytes phase 1 could not
+// settle; longer ones are merged by the whole CTA.  Unsettled pieces of <= 32 bytes go to a queue that
+// outlives the tile: it is emptied when it holds LANE_SLOTS pieces (a thread per piece) and after the CTA's
+// last tile (a warp per piece if few are left).  Phase 3: token totals per tile (tile_tok must be zero on
+// entry; queued pieces add to their tile when they are merged); the last CTA to finish turns the tile
+// totals into their exclusive prefix and checks the output capacity.
 // Without a token table (while the table itself is being built) every piece takes the merge path.
 struct PieceParams {
     const u8* base;            // aligned frame origin (text = base + shift)
@@ -440,21 +534,65 @@ struct PieceParams {
     unsigned long long ids_cap;
 };
 
+constexpr int MID_SLOTS = 64;                         // queue of 33..256-byte pieces
+// The CTA's warps take the nm queued pieces of 33..256 bytes and then nt queued pieces of <= 32 bytes, one
+// piece at a time each (*next must be zero and the queues visible on entry).
+__device__ __forceinline__ void warp_flush(const PieceParams& P, u64* s_buf, const u32* m_a, const u32* m_p, const u32* m_tn, u32 nm,
+                                           const u32* q_a, const u32* q_p, const u32* q_tn, u32 nt, u32* next, const u8* text) {
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    u64* wbuf = s_buf + wid * (2 * TT_WARP_PIECE_MAX);
+    for (;;) {
+        u32 e = 0;
+        if (lane == 0) e = atomicAdd(next, 1u);
+        e = __shfl_sync(0xFFFFFFFFu, e, 0);
+        if (e >= nm + nt) break;
+        u32 m, pidx, tile;
+        if (e < nm) {
+            const u32 a = m_a[e], n = (m_tn[e] & 255) + 1;
+            m = n <= 64 ? warp_merge_perm<2>(wbuf, text, a, n, P.tab, P.ext_id, P.stage, lane)
+                        : warp_merge_perm<WCH>(wbuf, text, a, n, P.tab, P.ext_id, P.stage, lane);
+            pidx = m_p[e]; tile = m_tn[e] >> 8;
+        } else {
+            const u32 q = e - nm;
+            m = warp_merge_reg(text, q_a[q], (q_tn[q] & 31) + 1, P.tab, P.ext_id, P.stage, lane);
+            pidx = q_p[q]; tile = q_tn[q] >> 5;
+        }
+        if (lane == 0) { P.piece_cnt[pidx] = m; atomicAdd(&P.tile_tok[tile], m); }
+    }
+}
+
+// Merges the queued pieces a thread per piece (all threads of the CTA call it; the queue must be visible).
+__device__ __forceinline__ void lane_flush(const PieceParams& P, u64* s_buf, const u32* q_a, const u32* q_p, const u32* q_tn, u32 qn, const u8* text) {
+    const int tid = threadIdx.x;
+    if ((u32)tid < qn) {
+        u32* tok = reinterpret_cast<u32*>(s_buf);
+        const u32 m = lane_merge(tok, tok + LANE_SLOTS * LANE_MAX, tid, text, q_a[tid], (q_tn[tid] & 31) + 1, P.tab, P.ext_id, P.stage);
+        P.piece_cnt[q_p[tid]] = m;
+        atomicAdd(&P.tile_tok[q_tn[tid] >> 5], m);
+    }
+}
+
 __global__ void __launch_bounds__(BPE_THREADS, 4)
 k_pieces(const PieceParams P) {
     __shared__ TilePieces tp;
-    __shared__ u64 s_buf[LONG_SMEM_TOKENS];                   // warp merge buffers (8 x 2 x 256) or one long piece
+    __shared__ u64 s_buf[LONG_SMEM_TOKENS];                   // warp merge buffers (8 x 2 x 256), one long piece, or the lane path's columns
     __shared__ u16 s_miss[TILE_MAX_PIECES];
-    __shared__ u32 s_nmiss, s_nlong, s_total, s_islast;
+    __shared__ u16 s_mid[TT_TILE_BYTES / (LANE_MAX + 1) + 2];
+    __shared__ u32 q_a[LANE_SLOTS], q_p[LANE_SLOTS], q_tn[LANE_SLOTS];     // queue: text offset, piece index, tile << 5 | (bytes - 1)
+    __shared__ u32 m_a[MID_SLOTS], m_p[MID_SLOTS], m_tn[MID_SLOTS];        // queue of the 33..256-byte pieces: ..., tile << 8 | (bytes - 1)
+    __shared__ u32 s_nmiss, s_nmid, s_nlong, s_total, s_islast, s_next;
     __shared__ u32 sc[48];
     static_assert(LONG_SMEM_TOKENS >= BPE_WARPS * 2 * TT_WARP_PIECE_MAX, "buffer size");
+    static_assert(LONG_SMEM_TOKENS * sizeof(u64) >= 2 * LANE_SLOTS * LANE_MAX * sizeof(u32), "buffer size");
+    static_assert(LANE_SLOTS <= BPE_THREADS && LANE_MAX == 32, "queue layout");
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
     const bool dead = P.hdr->status != 0;
     const u8* text = P.base + P.shift;
+    u32 qn = 0, mq = 0;                                        // block-uniform queue lengths
     for (int tile = blockIdx.x; tile < (dead ? 0 : P.ntiles); tile += gridDim.x) {
         const long long c0 = (long long)tile * TT_TILE_CHUNKS;
         __syncthreads();
-        if (tid == 0) { s_nmiss = 0; s_nlong = 0; s_total = 0; }
+        if (tid == 0) { s_nmiss = 0; s_nmid = 0; s_nlong = 0; s_total = 0; }
         tile_pieces(tp, P.startmask, P.tile_first, P.nchunks, P.ntiles, tile, P.hi, sc);
         const u32 np = tp.n, p0 = P.tile_base[tile];
         const long long t0 = c0 * TT_CHUNK - P.shift;             // text offset of the tile start
@@ -466,27 +604,51 @@ k_pieces(const PieceParams P) {
             if (n == 1) { P.stage[a] = P.ext_id[text[a]]; P.piece_cnt[p0 + i] = 1; wsum++; }
             else if (n <= TT_TOKTAB_MAXLEN && P.toktab.slots != nullptr && toktab_lookup(P.toktab, text, a, n, id)) {
                 P.stage[a] = id; P.piece_cnt[p0 + i] = 1; wsum++;
-            } else if (n > TT_WARP_PIECE_MAX) { s_miss[TILE_MAX_PIECES - 1 - atomicAdd(&s_nlong, 1u)] = (u16)i; }
-            else s_miss[atomicAdd(&s_nmiss, 1u)] = (u16)i;        // short misses from the front, long pieces from the back
+            } else if (n > TT_WARP_PIECE_MAX) { s_miss[TILE_MAX_PIECES - 1 - atomicAdd(&s_nlong, 1u)] = (u16)i; }   // long pieces from the back
+            else if (n > LANE_MAX) s_mid[atomicAdd(&s_nmid, 1u)] = (u16)i;
+            else s_miss[atomicAdd(&s_nmiss, 1u)] = (u16)i;
         }
         for (int o = 16; o; o >>= 1) wsum += __shfl_xor_sync(0xFFFFFFFFu, wsum, o);
         __syncthreads();
-        // the misses of the tile are spread over the CTA's warps (the longest merge chain of a request sets
-        // its latency, so no warp should have to do two of them in a row if another warp is idle)
-        const u32 nmiss = s_nmiss, nlong = s_nlong;
-        u32 msum = 0;
-        u64* wbuf = s_buf + wid * (2 * TT_WARP_PIECE_MAX);
-        for (u32 e = wid; e < nmiss; e += BPE_WARPS) {
-            const u32 i = s_miss[e];
-            const u32 a = (u32)(t0 + tp.off[i]);
-            const u32 n = (i + 1 < np ? tp.off[i + 1] : tp.end) - tp.off[i];
-            const u32 m = n <= 32 ? warp_merge_reg(text, a, n, P.tab, P.ext_id, P.stage, lane)
-                        : n <= 64 ? warp_merge_perm<2>(wbuf, text, a, n, P.tab, P.ext_id, P.stage, lane)
-                                  : warp_merge_perm<WCH>(wbuf, text, a, n, P.tab, P.ext_id, P.stage, lane);
-            if (lane == 0) P.piece_cnt[p0 + i] = m;
-            msum += m;
+        const u32 nreg = s_nmiss, nmid = s_nmid, nlong = s_nlong;
+        // Unsettled pieces of <= 256 bytes go into two queues that outlive the tile, so that in bulk text all
+        // warps have work at once: a full queue of pieces of <= 32 bytes is merged a thread per piece, a full
+        // queue of longer ones a warp per piece.
+        const bool last_tile = tile + (int)gridDim.x >= P.ntiles;
+        for (u32 done = 0; done < nreg;) {
+            const u32 take = min(nreg - done, (u32)LANE_SLOTS - qn);
+            if ((u32)tid < take) {
+                const u32 i = s_miss[done + tid];
+                const u32 n = (i + 1 < np ? tp.off[i + 1] : tp.end) - tp.off[i];
+                q_a[qn + tid] = (u32)(t0 + tp.off[i]); q_p[qn + tid] = p0 + i; q_tn[qn + tid] = ((u32)tile << 5) | (n - 1);
+            }
+            qn += take; done += take;
+            __syncthreads();
+            if (qn == (u32)LANE_SLOTS) { lane_flush(P, s_buf, q_a, q_p, q_tn, qn, text); qn = 0; __syncthreads(); }
         }
-        if (lane == 0) atomicAdd(&s_total, wsum + msum);
+        for (u32 done = 0; done < nmid;) {
+            const u32 take = min(nmid - done, (u32)MID_SLOTS - mq);
+            if ((u32)tid < take) {
+                const u32 i = s_mid[done + tid];
+                const u32 n = (i + 1 < np ? tp.off[i + 1] : tp.end) - tp.off[i];
+                m_a[mq + tid] = (u32)(t0 + tp.off[i]); m_p[mq + tid] = p0 + i; m_tn[mq + tid] = ((u32)tile << 8) | (n - 1);
+            }
+            mq += take; done += take;
+            if (tid == 0) s_next = 0;
+            __syncthreads();
+            if (mq == (u32)MID_SLOTS) { warp_flush(P, s_buf, m_a, m_p, m_tn, mq, q_a, q_p, q_tn, 0, &s_next, text); mq = 0; __syncthreads(); }
+        }
+        // after the CTA's last tile the warps take what is left, including a short rest of the other queue (the
+        // longest chain of a request sets its latency, so its few unsettled pieces get a warp each)
+        if (last_tile) {
+            const u32 ntail = qn < LANE_MIN_PIECES ? qn : 0;
+            if (tid == 0) s_next = 0;
+            __syncthreads();
+            warp_flush(P, s_buf, m_a, m_p, m_tn, mq, q_a, q_p, q_tn, ntail, &s_next, text);
+            mq = 0;
+            if (ntail) qn = 0;
+        }
+        if (lane == 0) atomicAdd(&s_total, wsum);
         for (u32 e = 0; e < nlong; e++) {                         // block-uniform
             const u32 i = s_miss[TILE_MAX_PIECES - 1 - e];
             const u32 a = (u32)(t0 + tp.off[i]);
@@ -495,7 +657,8 @@ k_pieces(const PieceParams P) {
             if (tid == 0) { P.piece_cnt[p0 + i] = m; atomicAdd(&s_total, m); }
         }
         __syncthreads();
-        if (tid == 0) P.tile_tok[tile] = s_total;
+        if (tid == 0) atomicAdd(&P.tile_tok[tile], s_total);
+        if (last_tile && qn) { lane_flush(P, s_buf, q_a, q_p, q_tn, qn, text); qn = 0; }
     }
     // the last CTA to finish: exclusive prefix of the tile totals, total token count, capacity check
     __threadfence();

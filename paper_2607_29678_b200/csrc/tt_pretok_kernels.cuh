@@ -302,7 +302,7 @@ k_pretok(const PretokParams P) {
         if (c_first + tid < P.nchunks) P.startmask[c_first + tid] = (u16)S;
         if (S) atomicMin(&s_first, (u32)(tid * TT_CHUNK + tt_lobit(S)));
         u32 total = cta_sum_u32(tt_popc(S), scratch);
-        if (tid == 0) { P.tile_cnt[tile] = total; P.tile_first[tile] = s_first; }
+        if (tid == 0) { P.tile_cnt[tile] = total; P.tile_first[tile] = s_first; if (P.tile_tok) P.tile_tok[tile] = 0; }
     }
     if (any_bad) atomicMax(&P.hdr->status, 4 /* TT_ERR_INVALID_UTF8 */);
 

@@ -366,3 +366,29 @@ def test_cjk_latin_mixtures_in_long_documents():
     ids, ioff, status = gpu_encode_batch(gpu_vocab("C4"), text, off)
     want, woff = cpu_vocab("C4").encode_batch(text, off, 1, nthreads=8)
     assert status == 0 and np.array_equal(ioff, woff) and np.array_equal(ids, want)
+
+
+def test_bulk_text_of_pieces_outside_the_vocabulary():
+    """Megabytes of random words (Latin and CJK, 2..80 bytes) that are no vocabulary entries: every CTA
+    handles many tiles and its piece queues fill and empty many times (thread-per-piece and warp-per-piece
+    merges in bulk).  IDs against the oracle."""
+    rng = random.Random(777)
+    parts, size = [], 0
+    while size < 6_000_000:
+        k = rng.random()
+        if k < 0.45:
+            w = " " + "".join(rng.choice("abcdefghijklmnopqrstuvwxyzABCDE") for _ in range(rng.randrange(1, 70)))
+        elif k < 0.9:
+            w = "，" + "".join(chr(rng.randrange(0x4E00, 0x9FA5)) for _ in range(rng.randrange(1, 26)))
+        elif k < 0.95:
+            w = " the quick brown fox\n"
+        else:
+            w = str(rng.randrange(10 ** rng.randrange(1, 40)))
+        parts.append(w)
+        size += len(w)
+    text = np.frombuffer("".join(parts).encode("utf-8"), dtype=np.uint8)
+    for name in ("C4", "C3"):
+        cfg = wl.CONFIGS[name]
+        ids, status = gpu_encode(gpu_vocab(name), text)
+        want, _ = cpu_vocab(name).encode(text, cfg.pattern_id, nthreads=16)
+        assert status == 0 and np.array_equal(ids, want), name

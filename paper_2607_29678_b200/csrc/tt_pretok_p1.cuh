@@ -4,15 +4,17 @@
 // run-local rules, and Unicode marks take a narrow sparse fallback while the common path stays
 // vectorised.  Here the vectorised path covers number runs, whitespace runs, punctuation runs with
 // their [\r\n/]* tails, word starts with the one-character prefix, the lower->upper case boundary and
-// the contraction suffix after a word.  Three constructs are not decided by local rules: a mark, an
+// the contraction suffix after a word.  Three constructs are not decided by those rules: a mark, an
 // upper-case letter that follows a caseless letter, and an apostrophe between letters that has another
-// apostrophe two or three bytes before it (a chain of possible contraction suffixes).  Each of them
-// marks the text from the last *sure* piece start before it up to the next sure piece start as
-// unresolved; a thread whose chunk contains unresolved bytes re-derives those bytes by matching
-// sequentially from that sure start (matching from a piece start never looks behind it).  Sure
-// starts are positions that begin a piece whatever surrounds them: a document start, the first
-// digit of a number run, whitespace or non-apostrophe punctuation right after a letter or digit, a
-// letter right after a digit or a CR/LF.
+// apostrophe two or three bytes before it (a chain of possible contraction suffixes).  The second
+// kind is decided from the tile's class masks wherever they reach (tt_resolve_upper_after_caseless).
+// What stays unresolved marks the text from the last *sure* piece start before it up to the next sure
+// piece start; a thread whose chunk contains such bytes re-derives them by matching sequentially from
+// that sure start (matching from a piece start never looks behind it).  Sure starts are positions that
+// begin a piece whatever surrounds them: a document start, the first digit of a number run, whitespace
+// or punctuation right after a digit, whitespace or non-apostrophe punctuation right after a letter, a
+// letter right after a digit or a CR/LF, a one-byte blank right before a letter, a letter after two
+// punctuation characters, and the decided case boundaries.
 #pragma once
 #include "tt_pretok.cuh"
 

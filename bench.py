@@ -406,7 +406,7 @@ def vocab_table_bytes(n_merges: int) -> int:
 
 # DRAM bytes (read + write) per launch from the committed ncu capture of the C3 request
 # (profiles/c3_1M_request_kernels.md).
-NCU_TRAFFIC = {"pieces": 5_282_048, "pretok": 1_129_728, "scatter": 4_909_824}
+NCU_TRAFFIC = {"pieces": 5_388_800, "pretok": 1_130_752, "scatter": 4_909_568}
 
 
 def ncu_traffic(kernel: str):

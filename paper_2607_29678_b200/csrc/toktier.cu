@@ -144,7 +144,7 @@ static int build_token_table(tt_vocab* v, const tt_merge* merges, size_t n_merge
     if (!ok) { cudaGetLastError(); return TT_ERR_CUDA; }
     std::vector<u32> keep;
     for (size_t i = 0; i < np; i++)
-        if (cnt[i] == 1 && stage[off[i]] == ext_id[cand[i]]) keep.push_back((u32)i);
+        if ((int32_t)cnt[i] == -1 && stage[off[i]] == ext_id[cand[i]]) keep.push_back((u32)i);   // minus the staged count
     u32 cap = 1024;
     while (cap < 2 * keep.size() + 2) cap <<= 1;
     u32 log2cap = 0;

@@ -527,7 +527,8 @@ struct PieceParams {
     PairTable tab;
     TokTable toktab;
     const int32_t* ext_id;
-    u32* piece_cnt;            // tokens per piece
+    u32* piece_cnt;            // per piece: the id itself if the piece is one token found without merging (>= 0),
+                               // else minus the number of tokens staged at the piece's text offset
     int32_t* stage;            // ids staged at the text offset of their piece
     u64* pairbuf;              // global scratch of the long-piece path, indexed like the text
     u32* tile_tok;             // out: tokens per tile, then their exclusive prefix (ntiles + 1)
@@ -557,7 +558,7 @@ __device__ __forceinline__ void warp_flush(const PieceParams& P, u64* s_buf, con
             m = warp_merge_reg(text, q_a[q], (q_tn[q] & 31) + 1, P.tab, P.ext_id, P.stage, lane);
             pidx = q_p[q]; tile = q_tn[q] >> 5;
         }
-        if (lane == 0) { P.piece_cnt[pidx] = m; atomicAdd(&P.tile_tok[tile], m); }
+        if (lane == 0) { P.piece_cnt[pidx] = 0u - m; atomicAdd(&P.tile_tok[tile], m); }
     }
 }
 
@@ -567,7 +568,7 @@ __device__ __forceinline__ void lane_flush(const PieceParams& P, u64* s_buf, con
     if ((u32)tid < qn) {
         u32* tok = reinterpret_cast<u32*>(s_buf);
         const u32 m = lane_merge(tok, tok + LANE_SLOTS * LANE_MAX, tid, text, q_a[tid], (q_tn[tid] & 31) + 1, P.tab, P.ext_id, P.stage);
-        P.piece_cnt[q_p[tid]] = m;
+        P.piece_cnt[q_p[tid]] = 0u - m;
         atomicAdd(&P.tile_tok[q_tn[tid] >> 5], m);
     }
 }
@@ -601,9 +602,9 @@ k_pieces(const PieceParams P) {
             const u32 a = (u32)(t0 + tp.off[i]);
             const u32 n = (i + 1 < np ? tp.off[i + 1] : tp.end) - tp.off[i];
             int32_t id;
-            if (n == 1) { P.stage[a] = P.ext_id[text[a]]; P.piece_cnt[p0 + i] = 1; wsum++; }
+            if (n == 1) { P.piece_cnt[p0 + i] = (u32)P.ext_id[text[a]]; wsum++; }
             else if (n <= TT_TOKTAB_MAXLEN && P.toktab.slots != nullptr && toktab_lookup(P.toktab, text, a, n, id)) {
-                P.stage[a] = id; P.piece_cnt[p0 + i] = 1; wsum++;
+                P.piece_cnt[p0 + i] = (u32)id; wsum++;
             } else if (n > TT_WARP_PIECE_MAX) { s_miss[TILE_MAX_PIECES - 1 - atomicAdd(&s_nlong, 1u)] = (u16)i; }   // long pieces from the back
             else if (n > LANE_MAX) s_mid[atomicAdd(&s_nmid, 1u)] = (u16)i;
             else s_miss[atomicAdd(&s_nmiss, 1u)] = (u16)i;
@@ -654,7 +655,7 @@ k_pieces(const PieceParams P) {
             const u32 a = (u32)(t0 + tp.off[i]);
             const u32 n = (i + 1 < np ? tp.off[i + 1] : tp.end) - tp.off[i];
             const u32 m = cta_merge_long(text, a, n, P.tab, P.ext_id, P.stage, P.pairbuf + a, s_buf, sc);
-            if (tid == 0) { P.piece_cnt[p0 + i] = m; atomicAdd(&s_total, m); }
+            if (tid == 0) { P.piece_cnt[p0 + i] = 0u - m; atomicAdd(&s_total, m); }
         }
         __syncthreads();
         if (tid == 0) atomicAdd(&P.tile_tok[tile], s_total);
@@ -737,12 +738,14 @@ k_scatter(const ScatterParams P) {
         u32 carry = P.tile_tok[tile];
         for (u32 b = 0; b < np; b += BPE_THREADS) {
             const u32 i = b + tid;
-            const u32 c = i < np ? P.piece_cnt[p0 + i] : 0;
+            const int32_t v = i < np ? (int32_t)P.piece_cnt[p0 + i] : 0;       // an id, or minus the staged count
+            const u32 c = i < np ? (v >= 0 ? 1u : (u32)(-v)) : 0u;
             u32 tot;
             const u32 dst = carry + cta_excl_sum_scan(c, sc, &tot);
             if (i < np) {
                 const u32 src = (u32)(t0 + tp.off[i]);
-                if (c <= 8) { for (u32 k = 0; k < c; k++) P.ids_out[dst + k] = P.stage[src + k]; }
+                if (v >= 0) P.ids_out[dst] = v;
+                else if (c <= 8) { for (u32 k = 0; k < c; k++) P.ids_out[dst + k] = P.stage[src + k]; }
                 else {
                     const u32 slot = atomicAdd(&s_nbig, 1u);
                     if (slot < TILE_MAX_PIECES / 8) { s_big[slot][0] = src; s_big[slot][1] = dst; s_big[slot][2] = c; }

@@ -52,7 +52,7 @@ struct TTWorkspace {
     u32* tile_cnt;     // pieces per tile, then exclusive prefix (ntiles + 1)
     u32* tile_first;   // offset of the first piece start inside each tile, ~0 if none (ntiles + 1)
     u32* tile_tok;     // tokens per tile, then exclusive prefix (ntiles + 1)
-    u32* piece_cnt;    // tokens per piece (len + 1)
+    u32* piece_cnt;    // per piece: its id (one token, no merging) or minus the staged token count (len + 1)
     int32_t* stage;    // token ids staged at the byte offset of their piece (len)
     u64* pairbuf;      // (token, rank) pairs of the long-piece path, indexed like the text (len)
 };

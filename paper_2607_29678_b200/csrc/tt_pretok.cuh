@@ -121,6 +121,21 @@ TT_HD u32 tt_walk_fwd_nl(const u16 (*sm)[TT_SLOTS], int s, int bit, bool& open) 
     return 0;
 }
 
+// The same question asked of the raw text from byte g on (the run has left the shared-memory window):
+// 1 / 0 = answered from ASCII bytes alone, -1 = undecided (a non-ASCII byte, which may be whitespace; a
+// document boundary mask to consult; or more than `limit` bytes of blanks).  One thread, plain loads.
+TT_HD int tt_raw_fwd_nl(const u8* base, long long g, long long hi, const u32* docmask, int limit = 256) {
+    if (docmask) return -1;
+    for (int k = 0; k < limit; k++, g++) {
+        if (g >= hi) return 0;
+        const u32 b = base[g];
+        if (b == '\n' || b == '\r') return 1;
+        if (b >= 0x80) return -1;
+        if (!(b == ' ' || (b >= 0x09 && b <= 0x0C))) return 0;
+    }
+    return -1;
+}
+
 // Contraction suffix length at the apostrophe whose two following bytes are b1, b2 (0 = none).
 TT_HD int tt_contraction_len(u32 b1, u32 b2) {
     const u32 a = b1 | 0x20, b = b2 | 0x20;       // ASCII case fold; no other byte maps onto these letters
@@ -133,7 +148,8 @@ TT_HD int tt_contraction_len(u32 b1, u32 b2) {
 // NEED_* flags of aggregates that leave the shared-memory window (then `tc` must be filled and the
 // function called again).
 TT_HD u32 tt_eval_chunk_p0(const u16 (*sm)[TT_SLOTS], int slot, const u8* base, long long g0, long long hi,
-                           const TileCarry& tc, bool have_tc, u32& need, bool single_digits = false) {
+                           const TileCarry& tc, bool have_tc, u32& need, bool single_digits = false,
+                           const u32* docmask = nullptr) {
     const u64 OWN = 0xFFFFull << 16;
     const u64 lead = tt_win(sm, F_LEAD, slot);
     const u64 L = tt_win(sm, F_LOW, slot) | tt_win(sm, F_UPP, slot) | tt_win(sm, F_CLESS, slot);
@@ -219,7 +235,12 @@ TT_HD u32 tt_eval_chunk_p0(const u16 (*sm)[TT_SLOTS], int slot, const u8* base, 
             int i = tt_lobit(cand); cand &= cand - 1;
             bool open;
             u32 later = tt_walk_fwd_nl(sm, slot, i, open);
-            if (open) { if (have_tc) later = tc.nl_later_after; else { need |= NEED_F; later = 1; } }
+            if (open) {
+                const int raw = tt_raw_fwd_nl(base, g0 + (long long)(TT_SLOTS - slot) * TT_CHUNK, hi, docmask);
+                if (raw >= 0) later = (u32)raw;
+                else if (have_tc) later = tc.nl_later_after;
+                else { need |= NEED_F; later = 1; }
+            }
             if (!later) S |= 1ull << (16 + i);
         }
     }

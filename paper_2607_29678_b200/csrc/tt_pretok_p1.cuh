@@ -419,7 +419,12 @@ TT_HD u32 tt_eval_chunk_p1(const u16 (*sm)[TT_SLOTS], int slot, const SeqCtx& C,
             int i = tt_lobit(cand); cand &= cand - 1;
             bool open;
             u32 later = tt_walk_fwd_nl(sm, slot, i, open);
-            if (open) { if (have_tc) later = tc.nl_later_after; else { need |= NEED_F; later = 1; } }
+            if (open) {
+                const int raw = tt_raw_fwd_nl(C.base, g0 + (long long)(TT_SLOTS - slot) * TT_CHUNK, C.hi, C.docmask);
+                if (raw >= 0) later = (u32)raw;
+                else if (have_tc) later = tc.nl_later_after;
+                else { need |= NEED_F; later = 1; }
+            }
             if (!later) S |= 1ull << (32 + i);
         }
     }

@@ -392,3 +392,22 @@ def test_bulk_text_of_pieces_outside_the_vocabulary():
         ids, status = gpu_encode(gpu_vocab(name), text)
         want, _ = cpu_vocab(name).encode(text, cfg.pattern_id, nthreads=16)
         assert status == 0 and np.array_equal(ids, want), name
+
+
+@pytest.mark.parametrize("pattern", [0, 1])
+def test_whitespace_lookahead_past_the_tile_single_document(pattern):
+    """A blank run that begins near the end of a 2 KiB tile and runs past the kernel's look-ahead window, as
+    ONE document (no boundary mask): the raw-byte look-ahead for a later CR/LF, its give-up cases (non-ASCII
+    whitespace, non-ASCII non-whitespace, very long runs) and the end of the text."""
+    name = "C2" if pattern == 0 else "C4"
+    rng = random.Random(31 + pattern)
+    tails = ["x", "\n", "\r\n", "é", "　\n", "　x", " ", "", "1", "!", "\t\n", "\x0b\x0c z"]
+    for case in range(120):
+        lead_len = 2048 * rng.randrange(1, 4) - rng.randrange(0, 40)
+        filler = wl.generate(wl.KIND_MIX, rng.randrange(1 << 30), lead_len)[:lead_len].tobytes()
+        filler = filler[:len(filler) - 1].decode("utf-8", errors="ignore").encode("utf-8")
+        run = rng.choice([" ", "\t", " \t"]) * rng.choice([1, 5, 17, 40, 130, 300, 700])
+        doc = filler + b"a\n" + run.encode() + rng.choice(tails).encode("utf-8") + rng.choice([b"", b" tail\n"])
+        text = np.frombuffer(doc, dtype=np.uint8)
+        got, status = gpu_pretok(gpu_vocab(name), text)
+        assert status == 0 and np.array_equal(got, _expect_pieces(text, pattern)), (case, doc[-60:])

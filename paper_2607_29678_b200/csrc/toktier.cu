@@ -114,37 +114,39 @@ static int build_token_table(tt_vocab* v, const tt_merge* merges, size_t n_merge
     for (size_t i = 0; i < np; i++) { smask[off[i] >> 4] |= (u16)(1u << (off[i] & 15)); tile_base[off[i] / TT_TILE_BYTES + 1]++;
         u32& tf = tile_first[off[i] / TT_TILE_BYTES]; if (tf == 0xFFFFFFFFu) tf = off[i] % TT_TILE_BYTES; }
     for (size_t t = 0; t < ntiles; t++) tile_base[t + 1] += tile_base[t];
-    u8* d_text = nullptr; u16* d_mask = nullptr; u32 *d_tb = nullptr, *d_tf = nullptr, *d_cnt = nullptr, *d_tt = nullptr; int32_t* d_stage = nullptr;
+    u8* d_text = nullptr; u16* d_mask = nullptr; u32 *d_tf = nullptr, *d_cnt = nullptr, *d_tt = nullptr, *d_gt = nullptr; int32_t* d_stage = nullptr;
     TTHeader* d_hdr = nullptr;
     TTHeader h; memset(&h, 0, sizeof(h)); h.n_pieces = (u32)np;
-    std::vector<u32> cnt(np); std::vector<int32_t> stage(nb);
+    std::vector<u32> cnt(ntiles * TT_TILE_BYTES); std::vector<int32_t> stage(nb);
+    const size_t ngroups = ntiles / TT_GROUP_TILES + 2;
     bool ok = cudaMalloc(&d_text, nchunks * TT_CHUNK + 64) == cudaSuccess && cudaMalloc(&d_mask, (nchunks + 1) * sizeof(u16)) == cudaSuccess &&
-              cudaMalloc(&d_tb, (ntiles + 1) * sizeof(u32)) == cudaSuccess && cudaMalloc(&d_tt, (ntiles + 1) * sizeof(u32)) == cudaSuccess && cudaMalloc(&d_tf, (ntiles + 1) * sizeof(u32)) == cudaSuccess &&
-              cudaMalloc(&d_cnt, (np + 1) * sizeof(u32)) == cudaSuccess && cudaMalloc(&d_stage, (nb + 1) * sizeof(int32_t)) == cudaSuccess &&
+              cudaMalloc(&d_gt, ngroups * sizeof(u32)) == cudaSuccess && cudaMalloc(&d_tt, (ntiles + 1) * sizeof(u32)) == cudaSuccess && cudaMalloc(&d_tf, (ntiles + 1) * sizeof(u32)) == cudaSuccess &&
+              cudaMalloc(&d_cnt, cnt.size() * sizeof(u32)) == cudaSuccess && cudaMalloc(&d_stage, (nb + 1) * sizeof(int32_t)) == cudaSuccess &&
               cudaMalloc(&d_hdr, sizeof(TTHeader)) == cudaSuccess;
     ok = ok && cudaMemcpy(d_text, cat.data(), nb, cudaMemcpyHostToDevice) == cudaSuccess;
     ok = ok && cudaMemcpy(d_mask, smask.data(), (nchunks + 1) * sizeof(u16), cudaMemcpyHostToDevice) == cudaSuccess;
-    ok = ok && cudaMemcpy(d_tb, tile_base.data(), (ntiles + 1) * sizeof(u32), cudaMemcpyHostToDevice) == cudaSuccess;
     ok = ok && cudaMemcpy(d_tf, tile_first.data(), (ntiles + 1) * sizeof(u32), cudaMemcpyHostToDevice) == cudaSuccess;
     ok = ok && cudaMemcpy(d_hdr, &h, sizeof(h), cudaMemcpyHostToDevice) == cudaSuccess;
-    ok = ok && cudaMemset(d_tt, 0, (ntiles + 1) * sizeof(u32)) == cudaSuccess;
+    ok = ok && cudaMemset(d_tt, 0, (ntiles + 1) * sizeof(u32)) == cudaSuccess && cudaMemset(d_gt, 0, ngroups * sizeof(u32)) == cudaSuccess;
     if (ok) {
         PieceParams Q;
         Q.base = d_text; Q.shift = 0; Q.hi = (long long)nb; Q.nchunks = (long long)nchunks; Q.ntiles = (int)ntiles;
-        Q.startmask = d_mask; Q.tile_base = d_tb; Q.tile_first = d_tf; Q.hdr = d_hdr; Q.tab = v->tab;
+        Q.startmask = d_mask; Q.tile_first = d_tf; Q.hdr = d_hdr; Q.tab = v->tab;
         Q.toktab.slots = nullptr; Q.toktab.mask = 0; Q.toktab.shift = 0;      // no table yet: every piece is merged
-        Q.ext_id = v->d_ext_id; Q.piece_cnt = d_cnt; Q.stage = d_stage; Q.pairbuf = nullptr; Q.tile_tok = d_tt; Q.ids_cap = ~0ull;
+        Q.ext_id = v->d_ext_id; Q.piece_cnt = d_cnt; Q.stage = d_stage; Q.pairbuf = nullptr; Q.tile_tok = d_tt; Q.grp_tok = d_gt;
         const int grid = (int)(ntiles < (size_t)v->sm_count * 8 ? ntiles : (size_t)v->sm_count * 8);
         k_pieces<<<grid, BPE_THREADS>>>(Q);
         ok = cudaGetLastError() == cudaSuccess && cudaDeviceSynchronize() == cudaSuccess;
     }
-    ok = ok && cudaMemcpy(cnt.data(), d_cnt, np * sizeof(u32), cudaMemcpyDeviceToHost) == cudaSuccess;
+    ok = ok && cudaMemcpy(cnt.data(), d_cnt, cnt.size() * sizeof(u32), cudaMemcpyDeviceToHost) == cudaSuccess;
     ok = ok && cudaMemcpy(stage.data(), d_stage, nb * sizeof(int32_t), cudaMemcpyDeviceToHost) == cudaSuccess;
-    cudaFree(d_text); cudaFree(d_mask); cudaFree(d_tb); cudaFree(d_tf); cudaFree(d_tt); cudaFree(d_cnt); cudaFree(d_stage); cudaFree(d_hdr);
+    cudaFree(d_text); cudaFree(d_mask); cudaFree(d_gt); cudaFree(d_tf); cudaFree(d_tt); cudaFree(d_cnt); cudaFree(d_stage); cudaFree(d_hdr);
     if (!ok) { cudaGetLastError(); return TT_ERR_CUDA; }
     std::vector<u32> keep;
-    for (size_t i = 0; i < np; i++)
-        if ((int32_t)cnt[i] == -1 && stage[off[i]] == ext_id[cand[i]]) keep.push_back((u32)i);   // minus the staged count
+    for (size_t i = 0; i < np; i++) {
+        const size_t tile = off[i] / TT_TILE_BYTES, slot = tile * TT_TILE_BYTES + (i - tile_base[tile]);   // pieces are indexed per tile
+        if ((int32_t)cnt[slot] == -1 && stage[off[i]] == ext_id[cand[i]]) keep.push_back((u32)i);           // minus the staged count
+    }
     u32 cap = 1024;
     while (cap < 2 * keep.size() + 2) cap <<= 1;
     u32 log2cap = 0;
@@ -275,7 +277,8 @@ static size_t carve(TTWorkspace* w, void* base, size_t max_len, size_t max_docs)
     p = take((ntiles + 1) * sizeof(u32));       if (w) w->tile_cnt = (u32*)p;
     p = take((ntiles + 1) * sizeof(u32));       if (w) w->tile_first = (u32*)p;
     p = take((ntiles + 1) * sizeof(u32));       if (w) w->tile_tok = (u32*)p;
-    p = take((max_len + 1) * sizeof(u32));      if (w) w->piece_cnt = (u32*)p;
+    p = take((ntiles / TT_GROUP_TILES + 2) * sizeof(u32));   if (w) w->grp_tok = (u32*)p;
+    p = take(ntiles * TT_TILE_BYTES * sizeof(u32));          if (w) w->piece_cnt = (u32*)p;
     p = take((max_len + 1) * sizeof(int32_t));  if (w) w->stage = (int32_t*)p;
     p = take((max_len + 1) * sizeof(u64));      if (w) w->pairbuf = (u64*)p;
     return off;
@@ -300,7 +303,7 @@ static int run_pretok(const tt_vocab* v, const uint8_t* text, size_t len, const 
     P.ntiles = (int)((P.nchunks + TT_TILE_CHUNKS - 1) / TT_TILE_CHUNKS);
     P.pattern = v->pattern;
     P.docmask = nullptr;
-    P.startmask = w.startmask; P.tile_cnt = w.tile_cnt; P.tile_first = w.tile_first; P.tile_tok = w.tile_tok; P.hdr = w.hdr;
+    P.startmask = w.startmask; P.tile_cnt = w.tile_cnt; P.tile_first = w.tile_first; P.tile_tok = w.tile_tok; P.grp_tok = w.grp_tok; P.want_prefix = piece_off_dst != nullptr; P.hdr = w.hdr;
     P.cls_tables = v->d_cls; P.cls_bytes = v->cls_bytes;
     if (doc_off) {
         CK(cudaMemsetAsync(w.docmask, 0, ((size_t)P.hi / 32 + 4) * sizeof(u32), st));
@@ -348,14 +351,13 @@ static int encode_impl(const tt_vocab* v, const uint8_t* text, size_t len, const
     const int tile_grid = PP.ntiles < v->sm_count * 8 ? PP.ntiles : v->sm_count * 8;
     PieceParams Q;
     Q.base = PP.base; Q.shift = PP.lo; Q.hi = PP.hi; Q.nchunks = PP.nchunks; Q.ntiles = PP.ntiles;
-    Q.startmask = w.startmask; Q.tile_base = w.tile_cnt; Q.tile_first = w.tile_first; Q.hdr = w.hdr; Q.tab = v->tab; Q.toktab = v->toktab;
-    Q.ext_id = v->d_ext_id; Q.piece_cnt = w.piece_cnt; Q.stage = w.stage; Q.pairbuf = w.pairbuf; Q.tile_tok = w.tile_tok;
-    Q.ids_cap = (unsigned long long)ids_cap;
+    Q.startmask = w.startmask; Q.tile_first = w.tile_first; Q.hdr = w.hdr; Q.tab = v->tab; Q.toktab = v->toktab;
+    Q.ext_id = v->d_ext_id; Q.piece_cnt = w.piece_cnt; Q.stage = w.stage; Q.pairbuf = w.pairbuf; Q.tile_tok = w.tile_tok; Q.grp_tok = w.grp_tok;
     k_pieces<<<tile_grid, BPE_THREADS, 0, st>>>(Q);
     MARK(2);
     ScatterParams S;
     S.shift = PP.lo; S.hi = PP.hi; S.nchunks = PP.nchunks; S.ntiles = PP.ntiles; S.startmask = w.startmask;
-    S.tile_base = w.tile_cnt; S.tile_first = w.tile_first; S.tile_tok = w.tile_tok; S.piece_cnt = w.piece_cnt; S.stage = w.stage; S.hdr = w.hdr;
+    S.tile_first = w.tile_first; S.tile_tok = w.tile_tok; S.grp_tok = w.grp_tok; S.ids_cap = (unsigned long long)ids_cap; S.piece_cnt = w.piece_cnt; S.stage = w.stage; S.hdr = w.hdr;
     S.ids_out = ids_out; S.count_out = (long long*)count_out; S.status_out = status_out;
     S.docmask = doc_off ? w.docmask : nullptr; S.doc_off = (const long long*)doc_off; S.n_docs = (int)n_docs;
     S.ids_off_out = (long long*)ids_off_out;

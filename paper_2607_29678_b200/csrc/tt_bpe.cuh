@@ -338,6 +338,18 @@ __device__ __forceinline__ u32 cta_excl_sum_scan(u32 v, u32* scratch /* >= 33 */
     *total = scratch[32];
     return scratch[wid] + x - v;
 }
+// Sum over the CTA, returned to every thread (scratch >= 33 entries; two barriers).
+__device__ __forceinline__ unsigned long long cta_sum_u64(unsigned long long v, unsigned long long* scratch) {
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5, nw = (blockDim.x + 31) >> 5;
+    for (int o = 16; o; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+    __syncthreads();
+    if (lane == 0) scratch[wid] = v;
+    __syncthreads();
+    unsigned long long t = 0;
+    for (int w = 0; w < nw; w++) t += scratch[w];
+    return t;
+}
+
 __device__ __forceinline__ u32 cta_min_u32(u32 v, u32* scratch /* >= 33 */) {
     v = __reduce_min_sync(0xFFFFFFFFu, v);
     __syncthreads();
@@ -511,9 +523,9 @@ __device__ void tile_pieces(TilePieces& tp, const u16* __restrict__ startmask, c
 // whole vocabulary entries).  Phase 2: the CTA's warps merge the pieces of 33..256 bytes phase 1 could not
 // settle; longer ones are merged by the whole CTA.  Unsettled pieces of <= 32 bytes go to a queue that
 // outlives the tile: it is emptied when it holds LANE_SLOTS pieces (a thread per piece) and after the CTA's
-// last tile (a warp per piece if few are left).  Phase 3: token totals per tile (tile_tok must be zero on
-// entry; queued pieces add to their tile when they are merged); the last CTA to finish turns the tile
-// totals into their exclusive prefix and checks the output capacity.
+// last tile (a warp per piece if few are left).  Phase 3: token totals per tile and per group of tiles
+// (both zero on entry; queued pieces add to theirs when they are merged).  No CTA waits for another and
+// nothing is scanned here: k_scatter derives each tile's output offset from the two levels of totals.
 // Without a token table (while the table itself is being built) every piece takes the merge path.
 struct PieceParams {
     const u8* base;            // aligned frame origin (text = base + shift)
@@ -521,7 +533,6 @@ struct PieceParams {
     long long nchunks;
     int ntiles;
     const u16* startmask;
-    const u32* tile_base;      // first piece index of every tile (exclusive prefix, ntiles + 1)
     const u32* tile_first;     // offset of the first piece start inside every tile (~0: none)
     TTHeader* hdr;
     PairTable tab;
@@ -531,8 +542,8 @@ struct PieceParams {
                                // else minus the number of tokens staged at the piece's text offset
     int32_t* stage;            // ids staged at the text offset of their piece
     u64* pairbuf;              // global scratch of the long-piece path, indexed like the text
-    u32* tile_tok;             // out: tokens per tile, then their exclusive prefix (ntiles + 1)
-    unsigned long long ids_cap;
+    u32* tile_tok;             // in: zero; out: tokens per tile
+    u32* grp_tok;              // in: zero; out: tokens per group of TT_GROUP_TILES tiles
 };
 
 constexpr int MID_SLOTS = 64;                         // queue of 33..256-byte pieces
@@ -558,7 +569,7 @@ __device__ __forceinline__ void warp_flush(const PieceParams& P, u64* s_buf, con
             m = warp_merge_reg(text, q_a[q], (q_tn[q] & 31) + 1, P.tab, P.ext_id, P.stage, lane);
             pidx = q_p[q]; tile = q_tn[q] >> 5;
         }
-        if (lane == 0) { P.piece_cnt[pidx] = 0u - m; atomicAdd(&P.tile_tok[tile], m); }
+        if (lane == 0) { P.piece_cnt[pidx] = 0u - m; atomicAdd(&P.tile_tok[tile], m); atomicAdd(&P.grp_tok[tile >> TT_GROUP_SHIFT], m); }
     }
 }
 
@@ -570,6 +581,7 @@ __device__ __forceinline__ void lane_flush(const PieceParams& P, u64* s_buf, con
         const u32 m = lane_merge(tok, tok + LANE_SLOTS * LANE_MAX, tid, text, q_a[tid], (q_tn[tid] & 31) + 1, P.tab, P.ext_id, P.stage);
         P.piece_cnt[q_p[tid]] = 0u - m;
         atomicAdd(&P.tile_tok[q_tn[tid] >> 5], m);
+        atomicAdd(&P.grp_tok[q_tn[tid] >> (5 + TT_GROUP_SHIFT)], m);
     }
 }
 
@@ -581,7 +593,7 @@ k_pieces(const PieceParams P) {
     __shared__ u16 s_mid[TT_TILE_BYTES / (LANE_MAX + 1) + 2];
     __shared__ u32 q_a[LANE_SLOTS], q_p[LANE_SLOTS], q_tn[LANE_SLOTS];     // queue: text offset, piece index, tile << 5 | (bytes - 1)
     __shared__ u32 m_a[MID_SLOTS], m_p[MID_SLOTS], m_tn[MID_SLOTS];        // queue of the 33..256-byte pieces: ..., tile << 8 | (bytes - 1)
-    __shared__ u32 s_nmiss, s_nmid, s_nlong, s_total, s_islast, s_next;
+    __shared__ u32 s_nmiss, s_nmid, s_nlong, s_total, s_next;
     __shared__ u32 sc[48];
     static_assert(LONG_SMEM_TOKENS >= BPE_WARPS * 2 * TT_WARP_PIECE_MAX, "buffer size");
     static_assert(LONG_SMEM_TOKENS * sizeof(u64) >= 2 * LANE_SLOTS * LANE_MAX * sizeof(u32), "buffer size");
@@ -595,7 +607,7 @@ k_pieces(const PieceParams P) {
         __syncthreads();
         if (tid == 0) { s_nmiss = 0; s_nmid = 0; s_nlong = 0; s_total = 0; }
         tile_pieces(tp, P.startmask, P.tile_first, P.nchunks, P.ntiles, tile, P.hi, sc);
-        const u32 np = tp.n, p0 = P.tile_base[tile];
+        const u32 np = tp.n, p0 = (u32)tile * TT_TILE_BYTES;     // pieces are indexed per tile
         const long long t0 = c0 * TT_CHUNK - P.shift;             // text offset of the tile start
         u32 wsum = 0;
         for (u32 i = tid; i < np; i += BPE_THREADS) {
@@ -658,30 +670,8 @@ k_pieces(const PieceParams P) {
             if (tid == 0) { P.piece_cnt[p0 + i] = 0u - m; atomicAdd(&s_total, m); }
         }
         __syncthreads();
-        if (tid == 0) atomicAdd(&P.tile_tok[tile], s_total);
+        if (tid == 0) { atomicAdd(&P.tile_tok[tile], s_total); atomicAdd(&P.grp_tok[tile >> TT_GROUP_SHIFT], s_total); }
         if (last_tile && qn) { lane_flush(P, s_buf, q_a, q_p, q_tn, qn, text); qn = 0; }
-    }
-    // the last CTA to finish: exclusive prefix of the tile totals, total token count, capacity check
-    __threadfence();
-    __syncthreads();
-    if (tid == 0) s_islast = (atomicAdd(&P.hdr->count_done, 1u) == gridDim.x - 1);
-    __syncthreads();
-    if (!s_islast) return;
-    __threadfence();
-    unsigned long long carry = 0;
-    const u32 nt = dead ? 0 : (u32)P.ntiles;
-    for (u32 b0 = 0; b0 < nt; b0 += BPE_THREADS) {
-        const u32 i = b0 + tid;
-        u32 x = i < nt ? P.tile_tok[i] : 0, t2;
-        const u32 ex = cta_excl_sum_scan(x, sc, &t2);
-        if (i < nt) P.tile_tok[i] = (u32)carry + ex;
-        carry += t2;
-        __syncthreads();
-    }
-    if (tid == 0) {
-        P.tile_tok[nt] = (u32)carry;
-        P.hdr->n_tokens = carry;
-        if (!dead && carry > P.ids_cap) atomicMax(&P.hdr->status, 5 /* TT_ERR_CAPACITY */);
     }
 }
 
@@ -691,9 +681,10 @@ struct ScatterParams {
     long long shift, hi, nchunks;
     int ntiles;
     const u16* startmask;
-    const u32* tile_base;
     const u32* tile_first;
-    const u32* tile_tok;
+    const u32* tile_tok;       // tokens per tile
+    const u32* grp_tok;        // tokens per group of TT_GROUP_TILES tiles
+    unsigned long long ids_cap;
     const u32* piece_cnt;
     const int32_t* stage;
     TTHeader* hdr;
@@ -712,11 +703,28 @@ k_scatter(const ScatterParams P) {
     __shared__ u32 sc[48];
     __shared__ u32 s_big[TILE_MAX_PIECES / 8][3];
     __shared__ u32 s_nbig;
+    __shared__ unsigned long long s_sum[33];
     const int tid = threadIdx.x;
-    const int status = P.hdr->status;
+    // Each CTA takes a contiguous range of tiles.  Tokens before its first tile = the whole groups of tiles
+    // before it plus the tiles of its own group before it; the grand total (all groups) gives the count and
+    // the capacity check, which every CTA makes for itself.
+    const int per = (P.ntiles + (int)gridDim.x - 1) / (int)gridDim.x;
+    const int tile_lo = (int)blockIdx.x * per, tile_hi = min(P.ntiles, tile_lo + per);
+    const int ngroups = (P.ntiles + TT_GROUP_TILES - 1) >> TT_GROUP_SHIFT, g_lo = tile_lo >> TT_GROUP_SHIFT;
+    unsigned long long before = 0, total = 0;
+    for (int g = tid; g < ngroups; g += BPE_THREADS) {
+        const u32 x = P.grp_tok[g];
+        total += x;
+        if (g < g_lo) before += x;
+    }
+    for (int t = (g_lo << TT_GROUP_SHIFT) + tid; t < tile_lo; t += BPE_THREADS) before += P.tile_tok[t];
+    before = cta_sum_u64(before, s_sum);
+    total = cta_sum_u64(total, s_sum);
+    int status = P.hdr->status;
+    if (status == 0 && total > P.ids_cap) status = 5;          // TT_ERR_CAPACITY
     if (blockIdx.x == 0 && tid == 0) {
         if (P.status_out) *P.status_out = status;
-        if (P.count_out) *P.count_out = status ? 0 : (long long)P.hdr->n_tokens;
+        if (P.count_out) *P.count_out = status ? 0 : (long long)total;
     }
     if (status != 0) {
         if (P.ids_off_out)
@@ -726,16 +734,16 @@ k_scatter(const ScatterParams P) {
     if (P.ids_off_out && blockIdx.x == 0) {
         // documents that start at the very end of the text (empty trailing documents) and the total
         const long long len = P.hi - P.shift;
-        for (int d = P.n_docs - tid; d >= 0 && P.doc_off[d] >= len; d -= blockDim.x) P.ids_off_out[d] = (long long)P.hdr->n_tokens;
+        for (int d = P.n_docs - tid; d >= 0 && P.doc_off[d] >= len; d -= blockDim.x) P.ids_off_out[d] = (long long)total;
     }
-    for (int tile = blockIdx.x; tile < P.ntiles; tile += gridDim.x) {
+    u32 carry = (u32)before;
+    for (int tile = tile_lo; tile < tile_hi; tile++) {
         const long long c0 = (long long)tile * TT_TILE_CHUNKS;
         __syncthreads();
         if (tid == 0) s_nbig = 0;
         tile_pieces(tp, P.startmask, P.tile_first, P.nchunks, P.ntiles, tile, P.hi, sc);
-        const u32 np = tp.n, p0 = P.tile_base[tile];
+        const u32 np = tp.n, p0 = (u32)tile * TT_TILE_BYTES;
         const long long t0 = c0 * TT_CHUNK - P.shift;
-        u32 carry = P.tile_tok[tile];
         for (u32 b = 0; b < np; b += BPE_THREADS) {
             const u32 i = b + tid;
             const int32_t v = i < np ? (int32_t)P.piece_cnt[p0 + i] : 0;       // an id, or minus the staged count

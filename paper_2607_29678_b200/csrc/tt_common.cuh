@@ -23,6 +23,8 @@ constexpr int TT_CHUNK = 16;
 #endif
 constexpr int TT_TILE_CHUNKS = TT_TILE_CHUNKS_DEF;        // = threads per CTA
 constexpr int TT_TILE_BYTES = TT_CHUNK * TT_TILE_CHUNKS; // 2 KiB of text per tile
+constexpr int TT_GROUP_SHIFT = 8;                 // token totals are also kept per group of 256 tiles
+constexpr int TT_GROUP_TILES = 1 << TT_GROUP_SHIFT;
 
 // ---- character class codes (two-stage Unicode table, see gen_unicode_table.py) ------------
 enum : u32 { CC_OTHER = 0, CC_MARK = 1, CC_SPACE = 2, CC_NUMBER = 3, CC_LOWER = 4, CC_UPPER = 5, CC_CASELESS = 6 };
@@ -37,11 +39,9 @@ constexpr int TT_WARP_PIECE_MAX = 256;            // bytes; longer pieces take t
 // ---- workspace header (device memory, zeroed at the start of every call) --------------------
 struct TTHeader {
     int status;              // TT_OK or a device-side error code
-    u32 pretok_done;         // CTAs that finished the pre-tokenization pass
-    u32 count_done;          // CTAs that finished the piece kernel
-    u32 n_pieces;            // number of pieces found
-    unsigned long long n_tokens;   // total tokens
-    u32 pad[26];
+    u32 pretok_done;         // CTAs that finished the pre-tokenization pass (tt_pretokenize only)
+    u32 n_pieces;            // number of pieces found (tt_pretokenize only)
+    u32 pad[29];
 };
 static_assert(sizeof(TTHeader) == 128, "header layout");
 
@@ -51,8 +51,10 @@ struct TTWorkspace {
     u16* startmask;    // bit per text byte: first byte of a piece (one u16 per chunk)
     u32* tile_cnt;     // pieces per tile, then exclusive prefix (ntiles + 1)
     u32* tile_first;   // offset of the first piece start inside each tile, ~0 if none (ntiles + 1)
-    u32* tile_tok;     // tokens per tile, then exclusive prefix (ntiles + 1)
-    u32* piece_cnt;    // per piece: its id (one token, no merging) or minus the staged token count (len + 1)
+    u32* tile_tok;     // tokens per tile (ntiles + 1)
+    u32* grp_tok;      // tokens per group of TT_GROUP_TILES tiles
+    u32* piece_cnt;    // per piece, at tile * TT_TILE_BYTES + index inside the tile: its id (one token, no merging)
+                       // or minus the staged token count
     int32_t* stage;    // token ids staged at the byte offset of their piece (len)
     u64* pairbuf;      // (token, rank) pairs of the long-piece path, indexed like the text (len)
 };

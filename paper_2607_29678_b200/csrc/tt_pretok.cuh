@@ -30,7 +30,9 @@ struct PretokParams {
     u16* startmask;          // out: one u16 per chunk
     u32* tile_cnt;           // out: pieces per tile; replaced by the exclusive prefix (ntiles + 1 entries)
     u32* tile_first;         // out: offset inside the tile of its first piece start, or ~0 if it has none
-    u32* tile_tok;           // out: zeroed (the piece kernel accumulates token totals per tile), or null
+    u32* tile_tok;           // out: zeroed (the piece kernel accumulates token totals per tile and per group
+    u32* grp_tok;            //      of tiles), or null
+    int want_prefix;         // turn tile_cnt into its exclusive prefix and count the pieces (tt_pretokenize only)
     TTHeader* hdr;
     const u8* cls_tables;    // stage1 | stage2 | ascii, contiguous in global memory
     int cls_bytes;

@@ -302,11 +302,16 @@ k_pretok(const PretokParams P) {
         if (c_first + tid < P.nchunks) P.startmask[c_first + tid] = (u16)S;
         if (S) atomicMin(&s_first, (u32)(tid * TT_CHUNK + tt_lobit(S)));
         u32 total = cta_sum_u32(tt_popc(S), scratch);
-        if (tid == 0) { P.tile_cnt[tile] = total; P.tile_first[tile] = s_first; if (P.tile_tok) P.tile_tok[tile] = 0; }
+        if (tid == 0) {
+            P.tile_cnt[tile] = total; P.tile_first[tile] = s_first;
+            if (P.tile_tok) { P.tile_tok[tile] = 0; if ((tile & (TT_GROUP_TILES - 1)) == 0) P.grp_tok[tile >> TT_GROUP_SHIFT] = 0; }
+        }
     }
     if (any_bad) atomicMax(&P.hdr->status, 4 /* TT_ERR_INVALID_UTF8 */);
 
-    // the last CTA to finish turns the tile counts into their exclusive prefix
+    // the last CTA to finish turns the tile counts into their exclusive prefix (only where the piece list is
+    // materialised: the encode chain indexes its pieces per tile and needs no prefix)
+    if (!P.want_prefix) return;
     __threadfence();
     __syncthreads();
     if (tid == 0) s_islast = (atomicAdd(&P.hdr->pretok_done, 1u) == gridDim.x - 1);

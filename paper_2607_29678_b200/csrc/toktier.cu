@@ -330,6 +330,21 @@ static int check_common(const tt_vocab* v, const void* text, size_t len, void* w
     return TT_OK;
 }
 
+// Launches `kernel` so that it may begin while the kernel before it on the stream is still draining
+// (programmatic dependent launch): its CTAs are placed as soon as every CTA of the predecessor has
+// signalled, and wait inside the kernel (cudaGridDependencySynchronize) until the predecessor's memory
+// is complete.  Only the launch latency is hidden; the data dependence is unchanged.
+template <typename Params>
+static cudaError_t launch_after(void (*kernel)(const Params), int grid, int block, cudaStream_t st, const Params& p) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid); cfg.blockDim = dim3((unsigned)block); cfg.dynamicSmemBytes = 0; cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, p);
+}
+
 static int encode_impl(const tt_vocab* v, const uint8_t* text, size_t len, const int64_t* doc_off, size_t n_docs,
                        cudaStream_t st, int32_t* ids_out, size_t ids_cap, int64_t* count_out, int64_t* ids_off_out,
                        int32_t* status_out, void* workspace, cudaEvent_t* ev = nullptr) {
@@ -353,7 +368,8 @@ static int encode_impl(const tt_vocab* v, const uint8_t* text, size_t len, const
     Q.base = PP.base; Q.shift = PP.lo; Q.hi = PP.hi; Q.nchunks = PP.nchunks; Q.ntiles = PP.ntiles;
     Q.startmask = w.startmask; Q.tile_first = w.tile_first; Q.hdr = w.hdr; Q.tab = v->tab; Q.toktab = v->toktab;
     Q.ext_id = v->d_ext_id; Q.piece_cnt = w.piece_cnt; Q.stage = w.stage; Q.pairbuf = w.pairbuf; Q.tile_tok = w.tile_tok; Q.grp_tok = w.grp_tok;
-    k_pieces<<<tile_grid, BPE_THREADS, 0, st>>>(Q);
+    if (ev) k_pieces<<<tile_grid, BPE_THREADS, 0, st>>>(Q);
+    else CK(launch_after(k_pieces, tile_grid, BPE_THREADS, st, Q));
     MARK(2);
     ScatterParams S;
     S.shift = PP.lo; S.hi = PP.hi; S.nchunks = PP.nchunks; S.ntiles = PP.ntiles; S.startmask = w.startmask;
@@ -361,7 +377,8 @@ static int encode_impl(const tt_vocab* v, const uint8_t* text, size_t len, const
     S.ids_out = ids_out; S.count_out = (long long*)count_out; S.status_out = status_out;
     S.docmask = doc_off ? w.docmask : nullptr; S.doc_off = (const long long*)doc_off; S.n_docs = (int)n_docs;
     S.ids_off_out = (long long*)ids_off_out;
-    k_scatter<<<tile_grid, BPE_THREADS, 0, st>>>(S);
+    if (ev) k_scatter<<<tile_grid, BPE_THREADS, 0, st>>>(S);
+    else CK(launch_after(k_scatter, tile_grid, BPE_THREADS, st, S));
     MARK(3);
 #undef MARK
     CK(cudaGetLastError());

@@ -599,6 +599,8 @@ k_pieces(const PieceParams P) {
     static_assert(LONG_SMEM_TOKENS * sizeof(u64) >= 2 * LANE_SLOTS * LANE_MAX * sizeof(u32), "buffer size");
     static_assert(LANE_SLOTS <= BPE_THREADS && LANE_MAX == 32, "queue layout");
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+    cudaTriggerProgrammaticLaunchCompletion();               // k_scatter may be placed; it waits for this grid's memory itself
+    cudaGridDependencySynchronize();                         // k_pretok's flags and counts are complete from here on
     const bool dead = P.hdr->status != 0;
     const u8* text = P.base + P.shift;
     u32 qn = 0, mq = 0;                                        // block-uniform queue lengths
@@ -705,6 +707,7 @@ k_scatter(const ScatterParams P) {
     __shared__ u32 s_nbig;
     __shared__ unsigned long long s_sum[33];
     const int tid = threadIdx.x;
+    cudaGridDependencySynchronize();                         // k_pieces' counts and staged ids are complete from here on
     // Each CTA takes a contiguous range of tiles.  Tokens before its first tile = the whole groups of tiles
     // before it plus the tiles of its own group before it; the grand total (all groups) gives the count and
     // the capacity check, which every CTA makes for itself.

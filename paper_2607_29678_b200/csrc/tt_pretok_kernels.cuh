@@ -204,6 +204,7 @@ k_pretok(const PretokParams P) {
     __shared__ u32 s_islast;
 
     const int tid = threadIdx.x;
+    cudaTriggerProgrammaticLaunchCompletion();               // the next kernel may be placed; it waits for this grid's memory itself
     // the 128-byte ASCII table is always staged; the two-stage Unicode table only once a tile holds a
     // non-ASCII byte (pattern 1 stages it at once: its sparse matcher may read beyond the tile)
     bool tables_loaded = P.pattern == 1;

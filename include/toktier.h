@@ -70,6 +70,20 @@ typedef struct { int32_t left, right, result; } tt_merge;
 int tt_vocab_load(const tt_merge* merges, size_t n_merges, const int32_t byte_map[256], int pattern_id,
                   tt_vocab** out);
 
+/*
+ * tt_vocab_load_ex -- tt_vocab_load with option flags.
+ *   TT_VOCAB_IGNORE_MERGES  (paper Sec. 4.2: families configured with ignore_merges)  a piece whose bytes are,
+ *             as a whole, the byte string of a vocabulary entry is encoded as that one entry without running
+ *             the merge loop, whatever the merges would have made of it.  Where several entries spell the same
+ *             bytes the base byte, else the lowest-ranked merge result, is taken.  All other pieces are merged
+ *             as usual.  Entries of any length up to 4,096 bytes take part (those longer than 24 bytes through a
+ *             second table); a vocabulary with a longer entry is refused with TT_ERR_BAD_VOCAB under this flag.
+ * Everything else is as for tt_vocab_load (flags = 0 is the same call).  Unknown flag bits: TT_ERR_ARG.
+ */
+#define TT_VOCAB_IGNORE_MERGES 1u
+int tt_vocab_load_ex(const tt_merge* merges, size_t n_merges, const int32_t byte_map[256], int pattern_id,
+                     unsigned flags, tt_vocab** out);
+
 /* Frees the handle and its device tables.  NULL is allowed.  No encode using it may be in flight. */
 void tt_vocab_free(tt_vocab* v);
 

@@ -87,6 +87,8 @@ def _load():
         lib.orc_vocab_new.restype = c.c_void_p
         lib.orc_vocab_new.argtypes = [c.c_void_p, c.c_size_t, c.c_void_p]
         lib.orc_vocab_free.argtypes = [c.c_void_p]
+        lib.orc_vocab_set_ignore_merges.restype = None
+        lib.orc_vocab_set_ignore_merges.argtypes = [c.c_void_p, c.c_int]
         lib.orc_token_bytes.restype = c.c_size_t
         lib.orc_token_bytes.argtypes = [c.c_void_p, c.c_int32, c.c_void_p, c.c_size_t]
         lib.orc_token_lens.restype = None
@@ -142,12 +144,16 @@ def pieces(text, pattern: int) -> list[bytes]:
 
 
 class Vocab:
-    """Merge table: merges int32[n,3] rows (left, right, result); rank = row index."""
+    """Merge table: merges int32[n,3] rows (left, right, result); rank = row index.
+    ``ignore_merges`` (paper Sec. 4.2): a piece that is a vocabulary entry as a whole is that one token."""
 
-    def __init__(self, merges, byte_map=None):
+    def __init__(self, merges, byte_map=None, ignore_merges: bool = False):
         self.merges = np.ascontiguousarray(merges, dtype=np.int32).reshape(-1, 3)
         self.byte_map = np.ascontiguousarray(np.arange(256) if byte_map is None else byte_map, dtype=np.int32)
         self._h = _load().orc_vocab_new(self.merges.ctypes.data, self.merges.shape[0], self.byte_map.ctypes.data)
+        self.ignore_merges = bool(ignore_merges)
+        if ignore_merges:
+            _load().orc_vocab_set_ignore_merges(self._h, 1)
 
     def __del__(self):
         try:

@@ -213,6 +213,11 @@ struct Vocab {
     std::unordered_map<uint64_t, int32_t> rank;    /* (left,right) -> rank (= index) */
     std::vector<std::string> token_bytes;          /* indexed by id (sparse ids allowed) */
     int32_t max_id = 0;
+    /* Paper Sec. 4.2 (families configured with ignore_merges): the encoder emits a single id whenever the
+     * whole piece is a vocabulary entry, whatever the merge loop would have made of its bytes.  Where two
+     * entries spell the same bytes the one defined first (a base byte, else the lowest rank) is taken. */
+    bool ignore_merges = false;
+    std::unordered_map<std::string, int32_t> by_bytes;
 };
 inline uint64_t pair_key(int32_t a, int32_t b) { return ((uint64_t)(uint32_t)a << 32) | (uint32_t)b; }
 
@@ -260,6 +265,10 @@ void bpe_heap(const Vocab &v, const uint8_t *b, size_t n, std::vector<int32_t> &
 }
 
 void bpe_piece(const Vocab &v, const uint8_t *b, size_t n, std::vector<int32_t> &t) {
+    if (v.ignore_merges) {
+        auto it = v.by_bytes.find(std::string((const char *)b, n));
+        if (it != v.by_bytes.end()) { t.assign(1, it->second); return; }
+    }
     if (n <= 2048) bpe_naive(v, b, n, t); else bpe_heap(v, b, n, t);
 }
 
@@ -348,6 +357,18 @@ void *orc_vocab_new(const int32_t *merges /* n x 3: left,right,result */, size_t
     return v;
 }
 void orc_vocab_free(void *v) { delete (Vocab *)v; }
+
+/* Switches the whole-piece rule on or off (off by default). */
+void orc_vocab_set_ignore_merges(void *vp, int on) {
+    Vocab *v = (Vocab *)vp;
+    v->ignore_merges = on != 0;
+    if (on && v->by_bytes.empty()) {
+        for (int i = 0; i < 256; i++) if (v->byte_map[i] >= 0) v->by_bytes.emplace(std::string(1, (char)i), v->byte_map[i]);
+        for (const Merge &m : v->merges)
+            if (m.result >= 0 && m.result <= v->max_id && !v->token_bytes[m.result].empty())
+                v->by_bytes.emplace(v->token_bytes[m.result], m.result);      /* emplace keeps the first */
+    }
+}
 
 /* Byte string of a token id; returns its length (0 if unknown), writes up to cap bytes. */
 size_t orc_token_bytes(const void *vp, int32_t id, uint8_t *out, size_t cap) {

@@ -17,8 +17,9 @@ LIB_PATH = os.path.join(_HERE, "libtoktier.so")
 TT_OK, TT_ERR_ARG, TT_ERR_BAD_VOCAB, TT_ERR_CUDA, TT_ERR_INVALID_UTF8, TT_ERR_CAPACITY, TT_ERR_INTERNAL_TIMEOUT, TT_ERR_TOO_LARGE, TT_ERR_BAD_IDS = range(9)
 TT_STATIC_MAX_LEN = 262144
 TT_PATTERN_CL100K, TT_PATTERN_O200K, TT_PATTERN_CL100K_N1 = 0, 1, 2
+TT_VOCAB_IGNORE_MERGES = 1
 
-EXPORTS = ["tt_vocab_load", "tt_vocab_free", "tt_workspace_bytes", "tt_encode", "tt_encode_batch",
+EXPORTS = ["tt_vocab_load", "tt_vocab_load_ex", "tt_vocab_free", "tt_workspace_bytes", "tt_encode", "tt_encode_batch",
            "tt_pretokenize", "tt_encode_timed", "tt_encode_host", "tt_encode_static", "tt_spans", "tt_spans_workspace_bytes", "tt_class_table", "tt_strerror"]
 
 _lib = None
@@ -40,6 +41,8 @@ def lib() -> ctypes.CDLL:
         c = ctypes
         L.tt_vocab_load.restype = c.c_int
         L.tt_vocab_load.argtypes = [c.c_void_p, c.c_size_t, c.c_void_p, c.c_int, c.POINTER(c.c_void_p)]
+        L.tt_vocab_load_ex.restype = c.c_int
+        L.tt_vocab_load_ex.argtypes = [c.c_void_p, c.c_size_t, c.c_void_p, c.c_int, c.c_uint, c.POINTER(c.c_void_p)]
         L.tt_vocab_free.restype = None
         L.tt_vocab_free.argtypes = [c.c_void_p]
         L.tt_workspace_bytes.restype = c.c_size_t
@@ -97,9 +100,10 @@ def _stream_ptr(stream) -> int:
 
 
 class Vocab:
-    """tt_vocab_load / tt_vocab_free.  merges: int32[n,3] rows (left, right, result); rank = row."""
+    """tt_vocab_load(_ex) / tt_vocab_free.  merges: int32[n,3] rows (left, right, result); rank = row.
+    ignore_merges: a piece that is a vocabulary entry as a whole becomes that one token (TT_VOCAB_IGNORE_MERGES)."""
 
-    def __init__(self, merges, byte_map=None, pattern_id: int = TT_PATTERN_CL100K):
+    def __init__(self, merges, byte_map=None, pattern_id: int = TT_PATTERN_CL100K, ignore_merges: bool = False):
         m = np.ascontiguousarray(merges, dtype=np.int32).reshape(-1, 3)
         bm = np.ascontiguousarray(np.arange(256) if byte_map is None else byte_map, dtype=np.int32)
         if bm.size != 256:
@@ -107,7 +111,8 @@ class Vocab:
         self.n_merges = m.shape[0]
         self.pattern_id = pattern_id
         h = ctypes.c_void_p()
-        _check(lib().tt_vocab_load(m.ctypes.data, m.shape[0], bm.ctypes.data, pattern_id, ctypes.byref(h)), "tt_vocab_load")
+        flags = TT_VOCAB_IGNORE_MERGES if ignore_merges else 0
+        _check(lib().tt_vocab_load_ex(m.ctypes.data, m.shape[0], bm.ctypes.data, pattern_id, flags, ctypes.byref(h)), "tt_vocab_load_ex")
         self._h = h
 
     def close(self):

@@ -32,6 +32,9 @@ struct tt_vocab {
     PairTable tab{};
     TokSlot* d_tokslots = nullptr;
     TokTable toktab{};
+    bool ignore_merges = false;
+    LongSlot* d_longslots = nullptr; u8* d_longblob = nullptr;
+    LongTable longtab{};
     size_t n_table_tokens = 0;
     uint2* d_meta = nullptr;             // per caller id: (byte length, non-continuation bytes) for tt_spans
     u32 meta_n = 0;
@@ -70,7 +73,7 @@ extern "C" size_t tt_class_table(uint8_t* out, size_t cap) {
 
 extern "C" void tt_vocab_free(tt_vocab* v) {
     if (!v) return;
-    cudaFree(v->d_slots); cudaFree(v->d_bytepair); cudaFree(v->d_ext_id); cudaFree(v->d_cls); cudaFree(v->d_tokslots); cudaFree(v->d_meta);
+    cudaFree(v->d_slots); cudaFree(v->d_bytepair); cudaFree(v->d_ext_id); cudaFree(v->d_cls); cudaFree(v->d_tokslots); cudaFree(v->d_longslots); cudaFree(v->d_longblob); cudaFree(v->d_meta);
     cudaFree(v->d_text); cudaFree(v->d_ids); cudaFree(v->d_count); cudaFree(v->d_status); cudaFree(v->d_ws);
     if (v->h_text) cudaFreeHost(v->h_text);
     if (v->h_ids) cudaFreeHost(v->h_ids);
@@ -83,6 +86,8 @@ extern "C" void tt_vocab_free(tt_vocab* v) {
 // Whole-piece table: every token of at most TT_TOKTAB_MAXLEN bytes is encoded with the merge kernel
 // itself; those whose byte string yields exactly that one token are entered (key = bytes, value = the
 // caller's id).  A hit in the table therefore equals what the merge loop returns for that piece.
+// With ignore_merges every entry is entered as it is (the first entry that spells given bytes wins) and
+// entries longer than TT_TOKTAB_MAXLEN bytes go to the long-entry table.
 static int build_token_table(tt_vocab* v, const tt_merge* merges, size_t n_merges, const std::vector<int32_t>& ext_id) {
     (void)merges;
     // byte strings of the merge results, by internal id (operands are lower internal ids by construction)
@@ -92,6 +97,9 @@ static int build_token_table(tt_vocab* v, const tt_merge* merges, size_t n_merge
     internal.reserve(2 * ext_id.size());
     for (size_t i = 0; i < ext_id.size(); i++) internal.emplace(ext_id[i], (u32)i);
     std::vector<u32> cand;                       // internal ids of candidate tokens
+    std::vector<u32> longer;                     // ignore_merges: internal ids of entries beyond TT_TOKTAB_MAXLEN bytes
+    std::unordered_set<std::string> spelled;     // ignore_merges: byte strings seen so far (base bytes first)
+    if (v->ignore_merges) for (int b = 0; b < 256; b++) spelled.insert(bytes[b]);
     std::vector<u8> cat; std::vector<u32> off;
     for (size_t r = 0; r < n_merges; r++) {
         const std::string& L = bytes[internal[merges[r].left]];
@@ -99,14 +107,41 @@ static int build_token_table(tt_vocab* v, const tt_merge* merges, size_t n_merge
         if (L.size() + R.size() <= 4096) bytes[256 + r] = L + R;          // longer strings are never candidates
         else bytes[256 + r] = std::string(4097, 'x');
         const std::string& t = bytes[256 + r];
+        if (v->ignore_merges && t.size() > 4096) return TT_ERR_BAD_VOCAB;   // documented limit of the whole-piece rule
+        if (v->ignore_merges && !spelled.insert(t).second) continue;      // an earlier entry spells the same bytes
+        if (v->ignore_merges && t.size() > (size_t)TT_TOKTAB_MAXLEN) longer.push_back((u32)(256 + r));
         if (t.size() >= 2 && t.size() <= (size_t)TT_TOKTAB_MAXLEN) {
             cand.push_back((u32)(256 + r)); off.push_back((u32)cat.size());
             cat.insert(cat.end(), t.begin(), t.end());
         }
     }
     off.push_back((u32)cat.size());
+    if (!longer.empty()) {
+        u32 cap = 64;
+        while (cap < 2 * longer.size() + 2) cap <<= 1;
+        std::vector<LongSlot> ls(cap);
+        memset(ls.data(), 0, cap * sizeof(LongSlot));
+        std::vector<u8> blob;
+        u32 maxlen = 0;
+        for (u32 t : longer) {
+            const std::string& b = bytes[t];
+            const u64 hsh = longtab_hash((const u8*)b.data(), (u32)b.size());
+            u32 sl = (u32)(hsh >> 32) & (cap - 1);
+            while (ls[sl].len != 0) sl = (sl + 1) & (cap - 1);
+            ls[sl].hash = hsh; ls[sl].off = (u32)blob.size(); ls[sl].len = (u32)b.size(); ls[sl].id = ext_id[t];
+            blob.insert(blob.end(), b.begin(), b.end());
+            maxlen = maxlen > (u32)b.size() ? maxlen : (u32)b.size();
+        }
+        if (cudaMalloc(&v->d_longslots, cap * sizeof(LongSlot)) != cudaSuccess || cudaMalloc(&v->d_longblob, blob.size() + 16) != cudaSuccess ||
+            cudaMemcpy(v->d_longslots, ls.data(), cap * sizeof(LongSlot), cudaMemcpyHostToDevice) != cudaSuccess ||
+            cudaMemcpy(v->d_longblob, blob.data(), blob.size(), cudaMemcpyHostToDevice) != cudaSuccess) { cudaGetLastError(); return TT_ERR_CUDA; }
+        v->longtab.slots = v->d_longslots; v->longtab.blob = v->d_longblob; v->longtab.mask = cap - 1; v->longtab.maxlen = maxlen;
+    }
     if (cand.empty()) return TT_OK;
     const size_t nb = cat.size(), np = cand.size();
+    std::vector<u32> keep;
+    if (v->ignore_merges) { for (size_t i = 0; i < np; i++) keep.push_back((u32)i); }
+    else {
     // start flags and per-tile piece counts of the concatenation, as k_pretok would leave them
     const size_t nchunks = (nb + TT_CHUNK - 1) / TT_CHUNK, ntiles = (nchunks + TT_TILE_CHUNKS - 1) / TT_TILE_CHUNKS;
     std::vector<u16> smask(nchunks + 1, 0);
@@ -133,6 +168,7 @@ static int build_token_table(tt_vocab* v, const tt_merge* merges, size_t n_merge
         Q.base = d_text; Q.shift = 0; Q.hi = (long long)nb; Q.nchunks = (long long)nchunks; Q.ntiles = (int)ntiles;
         Q.startmask = d_mask; Q.tile_first = d_tf; Q.hdr = d_hdr; Q.tab = v->tab;
         Q.toktab.slots = nullptr; Q.toktab.mask = 0; Q.toktab.shift = 0;      // no table yet: every piece is merged
+        Q.longtab = LongTable{};
         Q.ext_id = v->d_ext_id; Q.piece_cnt = d_cnt; Q.stage = d_stage; Q.pairbuf = nullptr; Q.tile_tok = d_tt; Q.grp_tok = d_gt;
         const int grid = (int)(ntiles < (size_t)v->sm_count * 8 ? ntiles : (size_t)v->sm_count * 8);
         k_pieces<<<grid, BPE_THREADS>>>(Q);
@@ -142,10 +178,10 @@ static int build_token_table(tt_vocab* v, const tt_merge* merges, size_t n_merge
     ok = ok && cudaMemcpy(stage.data(), d_stage, nb * sizeof(int32_t), cudaMemcpyDeviceToHost) == cudaSuccess;
     cudaFree(d_text); cudaFree(d_mask); cudaFree(d_gt); cudaFree(d_tf); cudaFree(d_tt); cudaFree(d_cnt); cudaFree(d_stage); cudaFree(d_hdr);
     if (!ok) { cudaGetLastError(); return TT_ERR_CUDA; }
-    std::vector<u32> keep;
     for (size_t i = 0; i < np; i++) {
         const size_t tile = off[i] / TT_TILE_BYTES, slot = tile * TT_TILE_BYTES + (i - tile_base[tile]);   // pieces are indexed per tile
         if ((int32_t)cnt[slot] == -1 && stage[off[i]] == ext_id[cand[i]]) keep.push_back((u32)i);           // minus the staged count
+    }
     }
     u32 cap = 1024;
     while (cap < 2 * keep.size() + 2) cap <<= 1;
@@ -174,8 +210,13 @@ static int build_token_table(tt_vocab* v, const tt_merge* merges, size_t n_merge
 
 extern "C" int tt_vocab_load(const tt_merge* merges, size_t n_merges, const int32_t byte_map[256], int pattern_id,
                              tt_vocab** out) {
+    return tt_vocab_load_ex(merges, n_merges, byte_map, pattern_id, 0u, out);
+}
+
+extern "C" int tt_vocab_load_ex(const tt_merge* merges, size_t n_merges, const int32_t byte_map[256], int pattern_id,
+                                unsigned flags, tt_vocab** out) {
     if (out) *out = nullptr;
-    if (!out || !byte_map || (n_merges && !merges)) return TT_ERR_ARG;
+    if (!out || !byte_map || (n_merges && !merges) || (flags & ~TT_VOCAB_IGNORE_MERGES)) return TT_ERR_ARG;
     if (pattern_id != TT_PATTERN_CL100K && pattern_id != TT_PATTERN_O200K && pattern_id != TT_PATTERN_CL100K_N1) return TT_ERR_ARG;
     if (n_merges > TT_MAX_INTERNAL - 256) return TT_ERR_ARG;
     // external id -> internal id (byte b -> b, result of rank r -> 256 + r)
@@ -218,7 +259,7 @@ extern "C" int tt_vocab_load(const tt_merge* merges, size_t n_merges, const int3
     }
     tt_vocab* v = new (std::nothrow) tt_vocab();
     if (!v) return TT_ERR_CUDA;
-    v->pattern = pattern_id; v->n_merges = n_merges;
+    v->pattern = pattern_id; v->n_merges = n_merges; v->ignore_merges = (flags & TT_VOCAB_IGNORE_MERGES) != 0;
     // class tables: stage1 | stage2 | ascii
     const int stage2_bytes = TT_CLS_NBLOCKS * 128;
     v->cls_bytes = (int)align_up(0x1100 + stage2_bytes, 16) + 128;
@@ -238,7 +279,7 @@ extern "C" int tt_vocab_load(const tt_merge* merges, size_t n_merges, const int3
     ok = ok && cudaMemcpy(v->d_cls, cls.data(), v->cls_bytes, cudaMemcpyHostToDevice) == cudaSuccess;
     if (!ok) { cudaGetLastError(); tt_vocab_free(v); return TT_ERR_CUDA; }
     v->tab.slots = v->d_slots; v->tab.bytepair = v->d_bytepair; v->tab.mask = mask; v->tab.shift = shift;
-    if (build_token_table(v, merges, n_merges, ext_id) != TT_OK) { tt_vocab_free(v); return TT_ERR_CUDA; }
+    { const int rc = build_token_table(v, merges, n_merges, ext_id); if (rc != TT_OK) { tt_vocab_free(v); return rc; } }
     {   // byte length and number of non-continuation bytes of every token, indexed by the caller's id
         std::vector<uint2> in(256 + n_merges);
         for (int b = 0; b < 256; b++) in[b] = make_uint2(1u, (b & 0xC0) != 0x80 ? 1u : 0u);
@@ -366,7 +407,7 @@ static int encode_impl(const tt_vocab* v, const uint8_t* text, size_t len, const
     const int tile_grid = PP.ntiles < v->sm_count * 8 ? PP.ntiles : v->sm_count * 8;
     PieceParams Q;
     Q.base = PP.base; Q.shift = PP.lo; Q.hi = PP.hi; Q.nchunks = PP.nchunks; Q.ntiles = PP.ntiles;
-    Q.startmask = w.startmask; Q.tile_first = w.tile_first; Q.hdr = w.hdr; Q.tab = v->tab; Q.toktab = v->toktab;
+    Q.startmask = w.startmask; Q.tile_first = w.tile_first; Q.hdr = w.hdr; Q.tab = v->tab; Q.toktab = v->toktab; Q.longtab = v->longtab;
     Q.ext_id = v->d_ext_id; Q.piece_cnt = w.piece_cnt; Q.stage = w.stage; Q.pairbuf = w.pairbuf; Q.tile_tok = w.tile_tok; Q.grp_tok = w.grp_tok;
     if (ev) k_pieces<<<tile_grid, BPE_THREADS, 0, st>>>(Q);
     else CK(launch_after(k_pieces, tile_grid, BPE_THREADS, st, Q));

@@ -94,6 +94,35 @@ __device__ __forceinline__ bool toktab_lookup(const TokTable& tab, const u8* __r
     return false;
 }
 
+// ---- long-entry table (ignore_merges only): vocabulary entries of more than TT_TOKTAB_MAXLEN bytes --------
+// Slot = (64-bit hash of the bytes, offset into a byte blob, length, id); open addressing, load <= 0.5.  A hit
+// needs equal hash, equal length and equal bytes.
+struct LongSlot { u64 hash; u32 off; u32 len; int32_t id; u32 pad; };
+static_assert(sizeof(LongSlot) == 24, "slot layout");
+struct LongTable { const LongSlot* slots; const u8* blob; u32 mask; u32 maxlen; };   // slots == nullptr: none
+
+TT_HD u64 longtab_hash(const u8* p, u32 n) {
+    u64 h = 0xCBF29CE484222325ull ^ n;
+    for (u32 i = 0; i < n; i++) { h ^= p[i]; h *= 0x100000001B3ull; }
+    h ^= h >> 32;
+    return h * 0x9E3779B97F4A7C15ull;
+}
+__device__ __forceinline__ bool longtab_lookup(const LongTable& tab, const u8* __restrict__ text, u32 a, u32 n, int32_t& id) {
+    const u64 h = longtab_hash(text + a, n);
+    u32 s = (u32)(h >> 32) & tab.mask;
+    for (u32 probe = 0; probe <= tab.mask; probe++) {             // bounded by the capacity
+        const LongSlot e = tab.slots[s];
+        if (e.len == 0) return false;
+        if (e.hash == h && e.len == n) {
+            u32 k = 0;
+            while (k < n && tab.blob[e.off + k] == text[a + k]) k++;
+            if (k == n) { id = e.id; return true; }
+        }
+        s = (s + 1) & tab.mask;
+    }
+    return false;
+}
+
 constexpr u32 RK_STALE = 0xFFFFFFFEu;                 // rank must be probed again
 constexpr int BPE_WARPS = 8;                          // warps per CTA of the piece kernels
 constexpr int BPE_THREADS = BPE_WARPS * 32;           // = pieces per CTA iteration
@@ -537,6 +566,7 @@ struct PieceParams {
     TTHeader* hdr;
     PairTable tab;
     TokTable toktab;
+    LongTable longtab;         // ignore_merges: entries longer than the whole-piece table holds (else slots == nullptr)
     const int32_t* ext_id;
     u32* piece_cnt;            // per piece: the id itself if the piece is one token found without merging (>= 0),
                                // else minus the number of tokens staged at the piece's text offset
@@ -618,6 +648,8 @@ k_pieces(const PieceParams P) {
             int32_t id;
             if (n == 1) { P.piece_cnt[p0 + i] = (u32)P.ext_id[text[a]]; wsum++; }
             else if (n <= TT_TOKTAB_MAXLEN && P.toktab.slots != nullptr && toktab_lookup(P.toktab, text, a, n, id)) {
+                P.piece_cnt[p0 + i] = (u32)id; wsum++;
+            } else if (n > TT_TOKTAB_MAXLEN && P.longtab.slots != nullptr && n <= P.longtab.maxlen && longtab_lookup(P.longtab, text, a, n, id)) {
                 P.piece_cnt[p0 + i] = (u32)id; wsum++;
             } else if (n > TT_WARP_PIECE_MAX) { s_miss[TILE_MAX_PIECES - 1 - atomicAdd(&s_nlong, 1u)] = (u16)i; }   // long pieces from the back
             else if (n > LANE_MAX) s_mid[atomicAdd(&s_nmid, 1u)] = (u16)i;

@@ -411,3 +411,57 @@ def test_whitespace_lookahead_past_the_tile_single_document(pattern):
         text = np.frombuffer(doc, dtype=np.uint8)
         got, status = gpu_pretok(gpu_vocab(name), text)
         assert status == 0 and np.array_equal(got, _expect_pieces(text, pattern)), (case, doc[-60:])
+
+
+def test_ignore_merges_whole_piece_rule():
+    """TT_VOCAB_IGNORE_MERGES (paper Sec. 4.2): the hand-worked examples, random merge tables over tiny
+    alphabets (where many pieces are entries that the merge loop would encode differently, including entries
+    longer than 24 bytes) and a stored vocabulary on its config's text; IDs against the oracle with the same
+    rule, and the rule must actually change some results."""
+    import json
+    import os
+    import paper_2607_29678_b200 as tt
+    with open(os.path.join(os.path.dirname(__file__), "golden", "ignore_merges_examples.jsonl"), encoding="utf-8") as f:
+        for line in f:
+            d = json.loads(line)
+            if "piece" not in d:
+                continue
+            pairs = np.asarray(d["merges"], dtype=np.int32)
+            merges = np.concatenate([pairs, 256 + np.arange(len(pairs), dtype=np.int32)[:, None]], axis=1)
+            text = np.frombuffer(d["piece"].encode(), dtype=np.uint8)
+            for ign, key in ((False, "plain"), (True, "ignore")):
+                ids, status = gpu_encode(tt.Vocab(merges, None, 0, ignore_merges=ign), text)
+                assert status == 0 and ids.tolist() == d[key], (d, key)
+    differs = 0
+    refused = 0
+    for seed, n_merges, alpha in [(11, 60, "ab"), (12, 400, "abc"), (13, 3000, "ab"), (14, 150, "ab")]:
+        rng = random.Random(seed)
+        merges = _random_wellformed_merges(rng, n_merges, [ord(c) for c in alpha])
+        cv, plain = oracle.Vocab(merges, ignore_merges=True), oracle.Vocab(merges)
+        entries = {cv.token_bytes(int(r)) for r in merges[:, 2]}
+        if max(len(e) for e in entries) > 4096:                                  # beyond the documented limit: refused
+            with pytest.raises(tt.TokTierError) as err:
+                tt.Vocab(merges, None, 0, ignore_merges=True)
+            assert err.value.code == tt.TT_ERR_BAD_VOCAB
+            refused += 1
+            continue
+        gv = tt.Vocab(merges, None, 0, ignore_merges=True)
+        docs = [bytes(rng.choice(alpha.encode()) for _ in range(n)) for n in list(range(1, 70)) * 3 + [100, 300, 5000]]
+        docs += rng.sample(sorted(entries), min(len(entries), 300))              # entries themselves, of any length
+        text = np.frombuffer(b"".join(docs), dtype=np.uint8)
+        off = np.zeros(len(docs) + 1, dtype=np.int64)
+        off[1:] = np.cumsum([len(d) for d in docs])
+        ids, ioff, status = gpu_encode_batch(gv, text, off)
+        assert status == 0
+        for k, d in enumerate(docs):
+            want = cv.bpe(d, 2)
+            assert np.array_equal(ids[ioff[k]:ioff[k + 1]], want), (seed, len(d), d[:40])
+            differs += not np.array_equal(want, plain.bpe(d, 2))
+        assert max(len(e) for e in entries) > 24
+    assert differs > 20 and refused == 1
+    cfg = wl.CONFIGS["C2"]
+    merges, byte_map = wl.load_vocab(cfg)
+    text = wl.request(cfg)
+    ids, status = gpu_encode(tt.Vocab(merges, byte_map, cfg.pattern_id, ignore_merges=True), text)
+    want, _ = oracle.Vocab(merges, byte_map, ignore_merges=True).encode(text, cfg.pattern_id, nthreads=4)
+    assert status == 0 and np.array_equal(ids, want)

@@ -162,3 +162,55 @@ def test_non_identity_byte_map_and_result_ids():
     v = oracle.Vocab(merges, byte_map)
     assert list(v.bpe(b"abcab", 0)) == [7, 5]
     assert v.decode([7, 5]) == b"abcab"
+
+
+# ---- whole-piece rule (ignore_merges) -------------------------------------------------------------
+IGNORE_GOLDEN = os.path.join(os.path.dirname(__file__), "golden", "ignore_merges_examples.jsonl")
+
+
+def test_ignore_merges_hand_worked_examples():
+    n = 0
+    with open(IGNORE_GOLDEN, encoding="utf-8") as f:
+        for line in f:
+            d = json.loads(line)
+            if "piece" not in d:
+                continue
+            pairs = np.asarray(d["merges"], dtype=np.int32)
+            merges = np.concatenate([pairs, 256 + np.arange(len(pairs), dtype=np.int32)[:, None]], axis=1)
+            assert list(oracle.Vocab(merges).bpe(d["piece"], 2)) == d["plain"], d
+            assert list(oracle.Vocab(merges, ignore_merges=True).bpe(d["piece"], 2)) == d["ignore"], d
+            n += 1
+    assert n >= 8
+
+
+def test_ignore_merges_against_a_dictionary_of_entry_strings():
+    """Independent restatement on a stored vocabulary: entry strings are built here by concatenation, the first
+    entry that spells given bytes is kept in a dict, and every piece of a text is looked up in it before
+    falling back to the merge loop (which the pins above cover).  Also: the rule changes nothing for pieces
+    that are no entry, and ids always spell the text."""
+    cfg = wl.CONFIGS["C1"]
+    merges, byte_map = wl.load_vocab(cfg)
+    spell = {int(byte_map[b]): bytes([b]) for b in range(256)}
+    first = {bytes([b]): int(byte_map[b]) for b in range(256)}
+    for left, right, result in merges.tolist():
+        spell[result] = spell[left] + spell[right]
+        first.setdefault(spell[result], result)
+    plain, ign = oracle.Vocab(merges, byte_map), oracle.Vocab(merges, byte_map, ignore_merges=True)
+    text = wl.request(cfg).tobytes()
+    pieces = oracle.pieces(text, cfg.pattern_id)
+    ids, _ = ign.encode(text, cfg.pattern_id)
+    want, changed = [], 0
+    for p in pieces:
+        if p in first:
+            want.append(first[p])
+            changed += list(plain.bpe(p, 2)) != [first[p]]
+        else:
+            want.extend(plain.bpe(p, 2).tolist())
+    assert ids.tolist() == want
+    assert ign.decode(ids) == text
+    # every entry that is one piece under the pattern encodes to the first entry with its spelling
+    rng = random.Random(5)
+    entries = [s for s in first if len(s) >= 2]
+    for s in rng.sample(entries, 400):
+        if len(oracle.pieces(s, cfg.pattern_id)) == 1:
+            assert ign.encode(s, cfg.pattern_id)[0].tolist() == [first[s]]

@@ -156,6 +156,52 @@ int tt_spans(const tt_vocab* v, const int32_t* ids, const int64_t* count, size_t
              void* workspace, size_t workspace_bytes);
 
 /*
+ * Sessions -- incremental repair on append (paper Sec. 3.3).  A session stores a text A and its tokenization as
+ * records (byte position, id) in device memory.  tt_session_append(B) tokenizes only the last w characters of A
+ * (w = 512 unless tt_session_set_window changed it) followed by B with the same kernels as tt_encode, looks for
+ * the longest run of records on which the cached and the fresh sequence agree in position and id (the rightmost
+ * of several), and admits it through the stable boundary check: at least two tokens, more characters than the
+ * longest vocabulary entry, and a stable boundary at the start of one of its tokens (a character-class transition
+ * after which the pieces do not depend on the text before it: whitespace, or punctuation other than a mark or an
+ * apostrophe, after a letter or number; the first digit of a number; a letter after a number).  Cached records
+ * are then kept up to the end of the run and fresh ones after it, in place.  If the check fails w doubles, at
+ * most five times; after that, and whenever the window reaches the start of A, the whole text is tokenized.
+ * The stored IDs always equal tt_encode of the whole text.
+ *   tt_session_create   allocates the session's device buffers for up to max_bytes of text (about 40 bytes per
+ *                       byte of capacity) on the current device; `v` must outlive the session.
+ *   tt_session_append   text: HOST pointer, len bytes of valid UTF-8 (a complete string: it must not end inside
+ *                       a character).  Synchronises `stream` (once per window tried).  info (HOST, may be NULL)
+ *                       receives what happened.  An error (TT_ERR_INVALID_UTF8, TT_ERR_TOO_LARGE when the capacity
+ *                       is exceeded, TT_ERR_CUDA) leaves the session unchanged.
+ *   tt_session_view     DEVICE pointers to the IDs, to the byte offset of every token (count + 1 entries, the last
+ *                       one the text length) and to the token count, plus the stored length in bytes; valid until
+ *                       the next append or tt_session_free.
+ *   tt_session_copy     copies the records into caller-owned DEVICE buffers, asynchronously on `stream`:
+ *                       ids_out int32[ids_cap] (may be NULL), off_out int32[ids_cap + 1] (may be NULL), count_out
+ *                       int64.  min(stored bytes, ids_cap) entries are copied (a token has at least one byte);
+ *                       entries beyond the count are unspecified.
+ * One session must not be used from two threads at once.
+ */
+typedef struct tt_session tt_session;
+typedef struct {
+    int32_t attempts;        /* windows tried (the full tokenization counts as one if it was the first try) */
+    int32_t status;          /* TT_OK or the error that was returned                                        */
+    int64_t window_chars;    /* window that was accepted, in characters; 0 = the whole text was tokenized    */
+    int64_t window_start;    /* its first byte                                                               */
+    int64_t run_tokens;      /* tokens in the matched run                                                    */
+    int64_t splice_byte;     /* byte position from which fresh records were taken                            */
+    int64_t n_tokens;        /* tokens now stored                                                            */
+} tt_append_info;
+int tt_session_create(const tt_vocab* v, size_t max_bytes, tt_session** out);
+void tt_session_free(tt_session* s);
+int tt_session_set_window(tt_session* s, uint32_t window_chars);
+int tt_session_append(tt_session* s, const uint8_t* text, size_t len, void* stream, tt_append_info* info);
+int tt_session_view(const tt_session* s, const int32_t** ids_dev, const int32_t** off_dev, const int64_t** count_dev,
+                    size_t* len_bytes);
+int tt_session_copy(const tt_session* s, int32_t* ids_out, size_t ids_cap, int32_t* off_out, int64_t* count_out,
+                    void* stream);
+
+/*
  * tt_encode_timed -- diagnostic variant of tt_encode (same arguments and results) that records
  * CUDA events on `stream` between the kernels of the chain, waits for the last one and returns the
  * device time of each step in milliseconds: ms_out[0] tag + piece-start flags and the tile

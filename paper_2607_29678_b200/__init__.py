@@ -20,7 +20,8 @@ TT_PATTERN_CL100K, TT_PATTERN_O200K, TT_PATTERN_CL100K_N1 = 0, 1, 2
 TT_VOCAB_IGNORE_MERGES = 1
 
 EXPORTS = ["tt_vocab_load", "tt_vocab_load_ex", "tt_vocab_free", "tt_workspace_bytes", "tt_encode", "tt_encode_batch",
-           "tt_pretokenize", "tt_encode_timed", "tt_encode_host", "tt_encode_static", "tt_spans", "tt_spans_workspace_bytes", "tt_class_table", "tt_strerror"]
+           "tt_pretokenize", "tt_encode_timed", "tt_encode_host", "tt_encode_static", "tt_spans", "tt_spans_workspace_bytes", "tt_class_table", "tt_strerror",
+           "tt_session_create", "tt_session_free", "tt_session_set_window", "tt_session_append", "tt_session_view", "tt_session_copy"]
 
 _lib = None
 
@@ -73,6 +74,18 @@ def lib() -> ctypes.CDLL:
         L.tt_class_table.argtypes = [c.c_void_p, c.c_size_t]
         L.tt_strerror.restype = c.c_char_p
         L.tt_strerror.argtypes = [c.c_int]
+        L.tt_session_create.restype = c.c_int
+        L.tt_session_create.argtypes = [c.c_void_p, c.c_size_t, c.POINTER(c.c_void_p)]
+        L.tt_session_free.restype = None
+        L.tt_session_free.argtypes = [c.c_void_p]
+        L.tt_session_set_window.restype = c.c_int
+        L.tt_session_set_window.argtypes = [c.c_void_p, c.c_uint32]
+        L.tt_session_append.restype = c.c_int
+        L.tt_session_append.argtypes = [c.c_void_p, c.c_void_p, c.c_size_t, c.c_void_p, c.c_void_p]
+        L.tt_session_view.restype = c.c_int
+        L.tt_session_view.argtypes = [c.c_void_p, c.POINTER(c.c_void_p), c.POINTER(c.c_void_p), c.POINTER(c.c_void_p), c.POINTER(c.c_size_t)]
+        L.tt_session_copy.restype = c.c_int
+        L.tt_session_copy.argtypes = [c.c_void_p, c.c_void_p, c.c_size_t, c.c_void_p, c.c_void_p, c.c_void_p]
         _lib = L
     return _lib
 
@@ -208,3 +221,55 @@ class Vocab:
         _check(lib().tt_encode_host(self._h, a.ctypes.data, a.size, out.ctypes.data, out.size, ctypes.byref(cnt)),
                "tt_encode_host")
         return out[:cnt.value]
+
+
+class AppendInfo(ctypes.Structure):
+    """tt_append_info."""
+    _fields_ = [("attempts", ctypes.c_int32), ("status", ctypes.c_int32), ("window_chars", ctypes.c_int64),
+                ("window_start", ctypes.c_int64), ("run_tokens", ctypes.c_int64), ("splice_byte", ctypes.c_int64),
+                ("n_tokens", ctypes.c_int64)]
+
+
+class Session:
+    """tt_session_*: a stored text with its token records on the device, updated by incremental repair."""
+
+    def __init__(self, vocab: Vocab, max_bytes: int, window_chars: int | None = None):
+        self.vocab = vocab                      # keeps the vocabulary alive
+        h = ctypes.c_void_p()
+        _check(lib().tt_session_create(vocab._h, max_bytes, ctypes.byref(h)), "tt_session_create")
+        self._h = h
+        if window_chars is not None:
+            _check(lib().tt_session_set_window(self._h, window_chars), "tt_session_set_window")
+
+    def close(self):
+        if getattr(self, "_h", None):
+            lib().tt_session_free(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def append(self, data, stream=None) -> dict:
+        """tt_session_append (host bytes in); returns the tt_append_info fields."""
+        a = np.frombuffer(bytes(data), dtype=np.uint8) if isinstance(data, (bytes, bytearray, str)) else np.ascontiguousarray(data, dtype=np.uint8)
+        info = AppendInfo()
+        _check(lib().tt_session_append(self._h, a.ctypes.data if a.size else None, a.size, _stream_ptr(stream), ctypes.byref(info)),
+               "tt_session_append")
+        return {k: getattr(info, k) for k, _ in AppendInfo._fields_}
+
+    def records(self, stream=None):
+        """tt_session_copy into fresh tensors: (ids int32[T], off int32[T + 1], stored bytes)."""
+        import torch
+        n = ctypes.c_size_t()
+        _check(lib().tt_session_view(self._h, None, None, None, ctypes.byref(n)), "tt_session_view")
+        ids = torch.empty(max(n.value, 1), dtype=torch.int32, device="cuda")
+        off = torch.empty(n.value + 1, dtype=torch.int32, device="cuda")
+        count = torch.zeros(1, dtype=torch.int64, device="cuda")
+        _check(lib().tt_session_copy(self._h, ids.data_ptr(), n.value, off.data_ptr(), count.data_ptr(), _stream_ptr(stream)),
+               "tt_session_copy")
+        torch.cuda.synchronize()
+        k = int(count.item())
+        return ids[:k], off[:k + 1], n.value

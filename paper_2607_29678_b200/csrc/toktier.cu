@@ -7,6 +7,7 @@
 #include "tt_pretok_kernels.cuh"
 #include "tt_bpe.cuh"
 #include "tt_spans.cuh"
+#include "tt_session.cuh"
 #include "unicode_table.inc"
 
 #include <climits>
@@ -38,6 +39,7 @@ struct tt_vocab {
     size_t n_table_tokens = 0;
     uint2* d_meta = nullptr;             // per caller id: (byte length, non-continuation bytes) for tt_spans
     u32 meta_n = 0;
+    u32 max_token_chars = 1;             // characters of the longest entry (stable boundary check of the sessions)
     // cached buffers of tt_encode_host
     u8* h_text = nullptr; int32_t* h_ids = nullptr; long long* h_scalars = nullptr;
     u8* d_text = nullptr; int32_t* d_ids = nullptr; long long* d_count = nullptr; int32_t* d_status = nullptr;
@@ -288,6 +290,7 @@ extern "C" int tt_vocab_load_ex(const tt_merge* merges, size_t n_merges, const i
         for (size_t r = 0; r < n_merges; r++) {
             const uint2 L = in[internal[merges[r].left]], R = in[internal[merges[r].right]];
             in[256 + r] = make_uint2(L.x + R.x, L.y + R.y);
+            if (in[256 + r].y > v->max_token_chars) v->max_token_chars = in[256 + r].y;
         }
         if (max_ext < (1 << 24)) {
             std::vector<uint2> meta((size_t)max_ext + 1, make_uint2(0, 0));
@@ -594,4 +597,157 @@ extern "C" int tt_encode_static(const tt_vocab* v, const uint8_t* text, size_t l
     // is written before it is read, so the previous call's contents do not matter.
     return encode_impl(v, text, len, nullptr, 1, (cudaStream_t)stream, ids_out, ids_cap, count_out, nullptr, status_out,
                        scratch);
+}
+
+// ---- sessions: incremental repair on append (paper Sec. 3.3) ------------------------------------------
+struct tt_session {
+    const tt_vocab* v = nullptr;
+    size_t cap = 0;                       // bytes of text the session can hold
+    size_t len = 0;                       // bytes stored
+    uint32_t window_chars = 512;
+    std::vector<u8> h_text;               // host mirror of the stored text (window starts are found here)
+    u8* d_text = nullptr;
+    int32_t *d_ids = nullptr, *d_off = nullptr;                 // cached records; d_off[ntok] = len
+    int32_t *d_fids = nullptr, *d_foff = nullptr, *d_fchar = nullptr;   // fresh records / scratch of the span export
+    u8* d_eq = nullptr;
+    long long *d_ntok = nullptr, *d_fcount = nullptr;
+    int32_t *d_fstatus = nullptr, *d_sstatus = nullptr;
+    RepairDecision* d_dec = nullptr;
+    struct Host { RepairDecision dec; long long ntok; int32_t fstatus, sstatus; }* h = nullptr;   // pinned
+    void *d_ws = nullptr, *d_sws = nullptr;
+    size_t ws_bytes = 0, sws_bytes = 0;
+};
+
+extern "C" void tt_session_free(tt_session* s) {
+    if (!s) return;
+    cudaFree(s->d_text); cudaFree(s->d_ids); cudaFree(s->d_off); cudaFree(s->d_fids); cudaFree(s->d_foff); cudaFree(s->d_fchar);
+    cudaFree(s->d_eq); cudaFree(s->d_ntok); cudaFree(s->d_fcount); cudaFree(s->d_fstatus); cudaFree(s->d_sstatus);
+    cudaFree(s->d_dec); cudaFree(s->d_ws); cudaFree(s->d_sws);
+    if (s->h) cudaFreeHost(s->h);
+    delete s;
+}
+
+extern "C" int tt_session_create(const tt_vocab* v, size_t max_bytes, tt_session** out) {
+    if (out) *out = nullptr;
+    if (!v || !out || max_bytes == 0 || max_bytes >= (size_t)INT32_MAX - 64 || v->meta_n == 0) return TT_ERR_ARG;
+    tt_session* s = new (std::nothrow) tt_session();
+    if (!s) return TT_ERR_CUDA;
+    s->v = v; s->cap = max_bytes;
+    s->ws_bytes = tt_workspace_bytes(v, max_bytes, 1);
+    s->sws_bytes = tt_spans_workspace_bytes(v, max_bytes);
+    const size_t n1 = max_bytes + 1;
+    bool ok = cudaMalloc(&s->d_text, max_bytes + 64) == cudaSuccess && cudaMalloc(&s->d_ids, n1 * 4) == cudaSuccess &&
+              cudaMalloc(&s->d_off, n1 * 4) == cudaSuccess && cudaMalloc(&s->d_fids, n1 * 4) == cudaSuccess &&
+              cudaMalloc(&s->d_foff, n1 * 4) == cudaSuccess && cudaMalloc(&s->d_fchar, n1 * 4) == cudaSuccess &&
+              cudaMalloc(&s->d_eq, n1) == cudaSuccess && cudaMalloc(&s->d_ntok, 8) == cudaSuccess &&
+              cudaMalloc(&s->d_fcount, 8) == cudaSuccess && cudaMalloc(&s->d_fstatus, 4) == cudaSuccess &&
+              cudaMalloc(&s->d_sstatus, 4) == cudaSuccess && cudaMalloc(&s->d_dec, sizeof(RepairDecision)) == cudaSuccess &&
+              cudaMalloc(&s->d_ws, s->ws_bytes) == cudaSuccess && cudaMalloc(&s->d_sws, s->sws_bytes) == cudaSuccess &&
+              cudaMallocHost(&s->h, sizeof(tt_session::Host)) == cudaSuccess;
+    ok = ok && cudaMemset(s->d_ntok, 0, 8) == cudaSuccess && cudaMemset(s->d_off, 0, 4) == cudaSuccess;
+    if (!ok) { cudaGetLastError(); tt_session_free(s); return TT_ERR_CUDA; }
+    *out = s;
+    return TT_OK;
+}
+
+extern "C" int tt_session_set_window(tt_session* s, uint32_t window_chars) {
+    if (!s || window_chars == 0 || window_chars > (1u << 24)) return TT_ERR_ARG;
+    s->window_chars = window_chars;
+    return TT_OK;
+}
+
+extern "C" int tt_session_view(const tt_session* s, const int32_t** ids_dev, const int32_t** off_dev,
+                               const int64_t** count_dev, size_t* len_bytes) {
+    if (!s) return TT_ERR_ARG;
+    if (ids_dev) *ids_dev = s->d_ids;
+    if (off_dev) *off_dev = s->d_off;
+    if (count_dev) *count_dev = (const int64_t*)s->d_ntok;
+    if (len_bytes) *len_bytes = s->len;
+    return TT_OK;
+}
+
+// Tokenizes text[from, new_len) into (ids, off, count) with offsets relative to `from`.
+static int session_tokenize(tt_session* s, size_t from, size_t new_len, cudaStream_t st, int32_t* ids, int32_t* off, long long* count) {
+    const size_t n = new_len - from;
+    int rc = encode_impl(s->v, s->d_text + from, n, nullptr, 1, st, ids, s->cap, (int64_t*)count, nullptr, s->d_fstatus, s->d_ws);
+    if (rc != TT_OK) return rc;
+    return tt_spans(s->v, ids, (const int64_t*)count, s->cap, n, st, off, s->d_fchar, s->d_sstatus, s->d_sws, s->sws_bytes);
+}
+
+extern "C" int tt_session_append(tt_session* s, const uint8_t* text, size_t len, void* stream, tt_append_info* info) {
+    if (!s || (len && !text)) return TT_ERR_ARG;
+    if (len > s->cap - s->len) return TT_ERR_TOO_LARGE;
+    cudaStream_t st = (cudaStream_t)stream;
+    tt_append_info local; memset(&local, 0, sizeof(local));
+    const size_t old_len = s->len, new_len = old_len + len;
+    s->h_text.insert(s->h_text.end(), text, text + len);
+    auto fail = [&](int code) { s->h_text.resize(old_len); if (info) { local.status = code; *info = local; } return code; };
+    if (len) { if (cudaMemcpyAsync(s->d_text + old_len, text, len, cudaMemcpyHostToDevice, st) != cudaSuccess) { cudaGetLastError(); return fail(TT_ERR_CUDA); } }
+    if (new_len == 0) { if (info) *info = local; return TT_OK; }
+    const u8* ht = s->h_text.data();
+    uint64_t w = s->window_chars;
+    for (int attempt = 0; attempt <= 5 && old_len > 0; attempt++, w *= 2) {
+        // byte offset of the character that lies w characters before the end of the stored text
+        size_t ws = old_len; uint64_t left = w;
+        while (ws > 0 && left > 0) { ws--; while (ws > 0 && (ht[ws] & 0xC0) == 0x80) ws--; left--; }
+        local.attempts = attempt + 1;
+        if (ws == 0) break;                                   // the window is the whole text
+        int rc = session_tokenize(s, ws, new_len, st, s->d_fids, s->d_foff, s->d_fcount);
+        if (rc != TT_OK) return fail(rc);
+        RepairParams P;
+        P.ids = s->d_ids; P.off = s->d_off; P.ntok = s->d_ntok;
+        P.fids = s->d_fids; P.foff = s->d_foff; P.fchar = s->d_fchar; P.fcount = s->d_fcount;
+        P.fstatus = s->d_fstatus; P.sstatus = s->d_sstatus; P.text = s->d_text;
+        P.ws = (long long)ws; P.old_len = (long long)old_len; P.new_len = (long long)new_len;
+        P.cls = s->v->d_cls; P.cls_bytes = s->v->cls_bytes; P.max_tok_chars = (int)s->v->max_token_chars;
+        P.eq = s->d_eq; P.dec = s->d_dec;
+        k_repair_decide<<<1, 256, 0, st>>>(P);
+        const size_t fresh_max = new_len - ws;
+        const int grid = (int)((fresh_max + 255) / 256 < (size_t)s->v->sm_count * 4 ? (fresh_max + 255) / 256 : (size_t)s->v->sm_count * 4);
+        k_repair_apply<<<grid, 256, 0, st>>>(P);
+        if (cudaMemcpyAsync(&s->h->dec, s->d_dec, sizeof(RepairDecision), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+            cudaStreamSynchronize(st) != cudaSuccess) { cudaGetLastError(); return fail(TT_ERR_CUDA); }
+        const RepairDecision d = s->h->dec;
+        if (d.status != TT_OK) return fail(d.status);          // e.g. the appended text is not valid UTF-8: nothing changed
+        if (d.accept) {
+            s->len = new_len;
+            local.window_chars = (int64_t)w; local.window_start = (int64_t)ws; local.run_tokens = d.j1 - d.j0;
+            local.splice_byte = d.splice_byte; local.n_tokens = d.new_ntok; local.status = TT_OK;
+            if (info) *info = local;
+            return TT_OK;
+        }
+    }
+    if (local.attempts == 0) local.attempts = 1;
+    // full tokenization straight into the session's records (into the fresh buffers first, so that an error
+    // leaves the session as it was)
+    int rc = session_tokenize(s, 0, new_len, st, s->d_fids, s->d_foff, s->d_fcount);
+    if (rc != TT_OK) return fail(rc);
+    if (cudaMemcpyAsync(&s->h->ntok, s->d_fcount, 8, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+        cudaMemcpyAsync(&s->h->fstatus, s->d_fstatus, 4, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+        cudaMemcpyAsync(&s->h->sstatus, s->d_sstatus, 4, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+        cudaStreamSynchronize(st) != cudaSuccess) { cudaGetLastError(); return fail(TT_ERR_CUDA); }
+    if (s->h->fstatus != TT_OK) return fail(s->h->fstatus);
+    if (s->h->sstatus != TT_OK) return fail(s->h->sstatus);
+    const size_t nt = (size_t)s->h->ntok;
+    if (cudaMemcpyAsync(s->d_ids, s->d_fids, nt * 4, cudaMemcpyDeviceToDevice, st) != cudaSuccess ||
+        cudaMemcpyAsync(s->d_off, s->d_foff, (nt + 1) * 4, cudaMemcpyDeviceToDevice, st) != cudaSuccess ||
+        cudaMemcpyAsync(s->d_ntok, s->d_fcount, 8, cudaMemcpyDeviceToDevice, st) != cudaSuccess ||
+        cudaStreamSynchronize(st) != cudaSuccess) { cudaGetLastError(); return fail(TT_ERR_CUDA); }
+    s->len = new_len;
+    local.window_chars = 0; local.window_start = 0; local.run_tokens = 0; local.splice_byte = 0;
+    local.n_tokens = (int64_t)nt; local.status = TT_OK;
+    if (info) *info = local;
+    return TT_OK;
+}
+
+extern "C" int tt_session_copy(const tt_session* s, int32_t* ids_out, size_t ids_cap, int32_t* off_out,
+                               int64_t* count_out, void* stream) {
+    if (!s || !count_out) return TT_ERR_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    // the count is known on the host only as an upper bound (one token per byte); copy by that bound
+    const size_t n = s->len < ids_cap ? s->len : ids_cap;
+    if (ids_out && n) CK(cudaMemcpyAsync(ids_out, s->d_ids, n * sizeof(int32_t), cudaMemcpyDeviceToDevice, st));
+    if (off_out) CK(cudaMemcpyAsync(off_out, s->d_off, (n + 1) * sizeof(int32_t), cudaMemcpyDeviceToDevice, st));
+    CK(cudaMemcpyAsync(count_out, s->d_ntok, sizeof(int64_t), cudaMemcpyDeviceToDevice, st));
+    return TT_OK;
 }

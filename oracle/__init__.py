@@ -233,3 +233,43 @@ def train(corpus, pattern: int, n_merges: int):
     if m < 0:
         raise InvalidUtf8("invalid UTF-8 in corpus")
     return pairs[:m].copy(), int(nd.value)
+
+
+def split_added(text, literals) -> list[tuple[int, int, int]]:
+    """Added-token literal pass (paper Sec. 4.3/4.4: a leftmost-longest literal pass extracts the added and special
+    tokens before the tokenizer family handles the remaining segments).  Scans left to right; at each byte
+    position the longest literal that matches there is taken and the scan continues behind it; positions
+    inside a taken literal start nothing.  Returns the segments in order as (start, end, k): k = index of the
+    literal, or -1 for the text between literals (empty segments are not returned)."""
+    data = _as_u8(text).tobytes()
+    lits = [bytes(x) if not isinstance(x, str) else x.encode("utf-8") for x in literals]
+    out, p, seg = [], 0, 0
+    while p < len(data):
+        best = -1
+        for k, lit in enumerate(lits):
+            if lit and data.startswith(lit, p) and (best < 0 or len(lit) > len(lits[best])):
+                best = k
+        if best < 0:
+            p += 1
+            continue
+        if p > seg:
+            out.append((seg, p, -1))
+        out.append((p, p + len(lits[best]), best))
+        p += len(lits[best])
+        seg = p
+    if len(data) > seg:
+        out.append((seg, len(data), -1))
+    return out
+
+
+def encode_added(vocab: "Vocab", text, pattern: int, literals, literal_ids) -> np.ndarray:
+    """IDs of a text with added tokens: every literal found by split_added becomes its id, every segment between
+    literals is encoded as if it were a text of its own."""
+    data = _as_u8(text)
+    ids = []
+    for a, b, k in split_added(data, literals):
+        if k >= 0:
+            ids.append(int(literal_ids[k]))
+        else:
+            ids.extend(vocab.encode(data[a:b], pattern)[0].tolist())
+    return np.asarray(ids, dtype=np.int32)

@@ -156,6 +156,23 @@ int tt_spans(const tt_vocab* v, const int32_t* ids, const int64_t* count, size_t
              void* workspace, size_t workspace_bytes);
 
 /*
+ * Added tokens (paper Sec. 4.3 / 4.4: added and special tokens are literal strings reserved as single ids; a
+ * leftmost-longest literal pass extracts them before the tokenizer family handles the remaining segments).
+ *   tt_vocab_add_literals  registers n literals once per vocabulary (HOST arrays, copied): literal i is
+ *                          bytes[off[i] .. off[i+1]) (1..255 bytes, all distinct) with id ids[i] >= 0.
+ *                          Returns TT_ERR_ARG for bad arguments or a second call.
+ *   tt_encode_added        tt_encode with that pass in front: scanning left to right, at each byte the longest
+ *                          literal that matches there is taken and the scan continues behind it; every taken literal
+ *                          yields its id, and every stretch of text between literals is tokenized exactly as if it
+ *                          were a text of its own.  Arguments, workspace and error behaviour as for tt_encode;
+ *                          without registered literals it is tt_encode.
+ */
+int tt_vocab_add_literals(tt_vocab* v, const uint8_t* bytes, const uint32_t* off, const int32_t* ids, size_t n);
+int tt_encode_added(const tt_vocab* v, const uint8_t* text, size_t len, void* stream,
+                    int32_t* ids_out, size_t ids_cap, int64_t* count_out, int32_t* status_out,
+                    void* workspace, size_t workspace_bytes);
+
+/*
  * Sessions -- incremental repair on append (paper Sec. 3.3).  A session stores a text A and its tokenization as
  * records (byte position, id) in device memory.  tt_session_append(B) tokenizes only the last w characters of A
  * (w = 512 unless tt_session_set_window changed it) followed by B with the same kernels as tt_encode, looks for

@@ -21,7 +21,7 @@ TT_VOCAB_IGNORE_MERGES = 1
 
 EXPORTS = ["tt_vocab_load", "tt_vocab_load_ex", "tt_vocab_free", "tt_workspace_bytes", "tt_encode", "tt_encode_batch",
            "tt_pretokenize", "tt_encode_timed", "tt_encode_host", "tt_encode_static", "tt_spans", "tt_spans_workspace_bytes", "tt_class_table", "tt_strerror",
-           "tt_session_create", "tt_session_free", "tt_session_set_window", "tt_session_append", "tt_session_view", "tt_session_copy"]
+           "tt_session_create", "tt_session_free", "tt_session_set_window", "tt_session_append", "tt_session_view", "tt_session_copy", "tt_vocab_add_literals", "tt_encode_added"]
 
 _lib = None
 
@@ -84,6 +84,10 @@ def lib() -> ctypes.CDLL:
         L.tt_session_append.argtypes = [c.c_void_p, c.c_void_p, c.c_size_t, c.c_void_p, c.c_void_p]
         L.tt_session_view.restype = c.c_int
         L.tt_session_view.argtypes = [c.c_void_p, c.POINTER(c.c_void_p), c.POINTER(c.c_void_p), c.POINTER(c.c_void_p), c.POINTER(c.c_size_t)]
+        L.tt_vocab_add_literals.restype = c.c_int
+        L.tt_vocab_add_literals.argtypes = [c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_size_t]
+        L.tt_encode_added.restype = c.c_int
+        L.tt_encode_added.argtypes = L.tt_encode.argtypes
         L.tt_session_copy.restype = c.c_int
         L.tt_session_copy.argtypes = [c.c_void_p, c.c_void_p, c.c_size_t, c.c_void_p, c.c_void_p, c.c_void_p]
         _lib = L
@@ -162,6 +166,24 @@ class Vocab:
         _check(lib().tt_encode(self._h, text.data_ptr(), n, _stream_ptr(stream), bufs["ids"].data_ptr(),
                                bufs["ids"].numel(), bufs["count"].data_ptr(), bufs["status"].data_ptr(),
                                ws.data_ptr(), ws.numel()), "tt_encode")
+
+    def add_literals(self, literals, ids):
+        """tt_vocab_add_literals: added / special tokens (bytes or str) with their ids; once per vocabulary."""
+        lits = [x.encode("utf-8") if isinstance(x, str) else bytes(x) for x in literals]
+        blob = np.frombuffer(b"".join(lits) or b"\0", dtype=np.uint8).copy()
+        off = np.zeros(len(lits) + 1, dtype=np.uint32)
+        off[1:] = np.cumsum([len(x) for x in lits])
+        idv = np.ascontiguousarray(ids, dtype=np.int32)
+        _check(lib().tt_vocab_add_literals(self._h, blob.ctypes.data, off.ctypes.data, idv.ctypes.data, len(lits)),
+               "tt_vocab_add_literals")
+
+    def encode_added(self, text, bufs, stream=None, length: int | None = None):
+        """tt_encode_added: tt_encode behind the leftmost-longest added-token pass."""
+        n = int(text.numel() if length is None else length)
+        ws = bufs["workspace"]
+        _check(lib().tt_encode_added(self._h, text.data_ptr(), n, _stream_ptr(stream), bufs["ids"].data_ptr(),
+                                     bufs["ids"].numel(), bufs["count"].data_ptr(), bufs["status"].data_ptr(),
+                                     ws.data_ptr(), ws.numel()), "tt_encode_added")
 
     KERNEL_NAMES = ("pretok", "pieces", "scatter")
 

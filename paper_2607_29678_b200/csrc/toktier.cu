@@ -8,6 +8,7 @@
 #include "tt_bpe.cuh"
 #include "tt_spans.cuh"
 #include "tt_session.cuh"
+#include "tt_literals.cuh"
 #include "unicode_table.inc"
 
 #include <climits>
@@ -19,6 +20,7 @@
 #include <unordered_map>
 #include <unordered_set>
 #include <vector>
+#include <algorithm>
 
 struct tt_vocab {
     int pattern = 0;
@@ -39,6 +41,8 @@ struct tt_vocab {
     size_t n_table_tokens = 0;
     uint2* d_meta = nullptr;             // per caller id: (byte length, non-continuation bytes) for tt_spans
     u32 meta_n = 0;
+    LitEntry* d_lit_entries = nullptr; u8* d_lit_blob = nullptr;
+    LitTable lit{};                      // added-token literals (tt_vocab_add_literals), n == 0: none
     u32 max_token_chars = 1;             // characters of the longest entry (stable boundary check of the sessions)
     // cached buffers of tt_encode_host
     u8* h_text = nullptr; int32_t* h_ids = nullptr; long long* h_scalars = nullptr;
@@ -75,7 +79,7 @@ extern "C" size_t tt_class_table(uint8_t* out, size_t cap) {
 
 extern "C" void tt_vocab_free(tt_vocab* v) {
     if (!v) return;
-    cudaFree(v->d_slots); cudaFree(v->d_bytepair); cudaFree(v->d_ext_id); cudaFree(v->d_cls); cudaFree(v->d_tokslots); cudaFree(v->d_longslots); cudaFree(v->d_longblob); cudaFree(v->d_meta);
+    cudaFree(v->d_slots); cudaFree(v->d_bytepair); cudaFree(v->d_ext_id); cudaFree(v->d_cls); cudaFree(v->d_lit_entries); cudaFree(v->d_lit_blob); cudaFree(v->d_tokslots); cudaFree(v->d_longslots); cudaFree(v->d_longblob); cudaFree(v->d_meta);
     cudaFree(v->d_text); cudaFree(v->d_ids); cudaFree(v->d_count); cudaFree(v->d_status); cudaFree(v->d_ws);
     if (v->h_text) cudaFreeHost(v->h_text);
     if (v->h_ids) cudaFreeHost(v->h_ids);
@@ -170,7 +174,7 @@ static int build_token_table(tt_vocab* v, const tt_merge* merges, size_t n_merge
         Q.base = d_text; Q.shift = 0; Q.hi = (long long)nb; Q.nchunks = (long long)nchunks; Q.ntiles = (int)ntiles;
         Q.startmask = d_mask; Q.tile_first = d_tf; Q.hdr = d_hdr; Q.tab = v->tab;
         Q.toktab.slots = nullptr; Q.toktab.mask = 0; Q.toktab.shift = 0;      // no table yet: every piece is merged
-        Q.longtab = LongTable{};
+        Q.longtab = LongTable{}; Q.litstart = nullptr;
         Q.ext_id = v->d_ext_id; Q.piece_cnt = d_cnt; Q.stage = d_stage; Q.pairbuf = nullptr; Q.tile_tok = d_tt; Q.grp_tok = d_gt;
         const int grid = (int)(ntiles < (size_t)v->sm_count * 8 ? ntiles : (size_t)v->sm_count * 8);
         k_pieces<<<grid, BPE_THREADS>>>(Q);
@@ -325,6 +329,9 @@ static size_t carve(TTWorkspace* w, void* base, size_t max_len, size_t max_docs)
     p = take(ntiles * TT_TILE_BYTES * sizeof(u32));          if (w) w->piece_cnt = (u32*)p;
     p = take((max_len + 1) * sizeof(int32_t));  if (w) w->stage = (int32_t*)p;
     p = take((max_len + 1) * sizeof(u64));      if (w) w->pairbuf = (u64*)p;
+    p = take(padded + 16);                      if (w) w->cand = (u8*)p;
+    p = take((padded / 32 + 4) * sizeof(u32));  if (w) w->litstart = (u32*)p;
+    p = take((padded / 32 + 4) * sizeof(u32));  if (w) w->litin = (u32*)p;
     return off;
 }
 
@@ -338,7 +345,7 @@ extern "C" size_t tt_workspace_bytes(const tt_vocab* v, size_t max_len, size_t m
 // Enqueues K1+K2 (and K3 when piece_off_dst is given: only tt_pretokenize materialises the offsets;
 // the encode chain derives them per tile from the start flags).
 static int run_pretok(const tt_vocab* v, const uint8_t* text, size_t len, const int64_t* doc_off, size_t n_docs,
-                      cudaStream_t st, TTWorkspace& w, u32* piece_off_dst, PretokParams& P) {
+                      cudaStream_t st, TTWorkspace& w, u32* piece_off_dst, PretokParams& P, bool literals = false) {
     const uintptr_t addr = (uintptr_t)text;
     const long long shift = (long long)(addr & 15);
     P.base = (const u8*)(addr - shift);
@@ -346,7 +353,7 @@ static int run_pretok(const tt_vocab* v, const uint8_t* text, size_t len, const 
     P.nchunks = (P.hi + TT_CHUNK - 1) / TT_CHUNK;
     P.ntiles = (int)((P.nchunks + TT_TILE_CHUNKS - 1) / TT_TILE_CHUNKS);
     P.pattern = v->pattern;
-    P.docmask = nullptr;
+    P.docmask = nullptr; P.litstart = nullptr; P.litin = nullptr;
     P.startmask = w.startmask; P.tile_cnt = w.tile_cnt; P.tile_first = w.tile_first; P.tile_tok = w.tile_tok; P.grp_tok = w.grp_tok; P.want_prefix = piece_off_dst != nullptr; P.hdr = w.hdr;
     P.cls_tables = v->d_cls; P.cls_bytes = v->cls_bytes;
     if (doc_off) {
@@ -354,6 +361,21 @@ static int run_pretok(const tt_vocab* v, const uint8_t* text, size_t len, const 
         const int threads = 256, blocks = (int)((n_docs + 1 + threads - 1) / threads);
         k_docmask<<<blocks, threads, 0, st>>>((const long long*)doc_off, (int)n_docs, shift, (long long)len, w.docmask, w.hdr);
         P.docmask = w.docmask;
+    }
+    if (literals && !doc_off) {
+        // added-token literal pass: extracted literals become documents of their own and single pieces
+        const size_t words = ((size_t)P.hi / 32 + 4) * sizeof(u32);
+        CK(cudaMemsetAsync(w.docmask, 0, words, st));
+        CK(cudaMemsetAsync(w.litstart, 0, words, st));
+        CK(cudaMemsetAsync(w.litin, 0, words, st));
+        LitParams L;
+        L.base = P.base; L.lo = P.lo; L.hi = P.hi; L.tab = v->lit; L.cand = w.cand; L.stage = w.stage;
+        L.docmask = w.docmask; L.litstart = w.litstart; L.litin = w.litin;
+        const size_t want = (len + 255) / 256;
+        const int lgrid = (int)(want < (size_t)v->sm_count * 8 ? want : (size_t)v->sm_count * 8);
+        k_lit_scan<<<lgrid, 256, 0, st>>>(L);
+        k_lit_select<<<lgrid, 256, 0, st>>>(L);
+        P.docmask = w.docmask; P.litstart = w.litstart; P.litin = w.litin;
     }
     const size_t smem = align_up(v->cls_bytes, 16) + sizeof(u16) * F_COUNT * TT_SLOTS;
     const int grid = P.ntiles < v->sm_count * 6 ? P.ntiles : v->sm_count * 6;
@@ -391,7 +413,7 @@ static cudaError_t launch_after(void (*kernel)(const Params), int grid, int bloc
 
 static int encode_impl(const tt_vocab* v, const uint8_t* text, size_t len, const int64_t* doc_off, size_t n_docs,
                        cudaStream_t st, int32_t* ids_out, size_t ids_cap, int64_t* count_out, int64_t* ids_off_out,
-                       int32_t* status_out, void* workspace, cudaEvent_t* ev = nullptr) {
+                       int32_t* status_out, void* workspace, cudaEvent_t* ev = nullptr, bool literals = false) {
 #define MARK(i) do { if (ev) cudaEventRecord(ev[i], st); } while (0)
     TTWorkspace w;
     carve(&w, workspace, len, n_docs);
@@ -404,13 +426,13 @@ static int encode_impl(const tt_vocab* v, const uint8_t* text, size_t len, const
     }
     MARK(0);
     PretokParams PP;
-    int rc = run_pretok(v, text, len, doc_off, n_docs, st, w, nullptr, PP);
+    int rc = run_pretok(v, text, len, doc_off, n_docs, st, w, nullptr, PP, literals);
     if (rc != TT_OK) return rc;
     MARK(1);
     const int tile_grid = PP.ntiles < v->sm_count * 8 ? PP.ntiles : v->sm_count * 8;
     PieceParams Q;
     Q.base = PP.base; Q.shift = PP.lo; Q.hi = PP.hi; Q.nchunks = PP.nchunks; Q.ntiles = PP.ntiles;
-    Q.startmask = w.startmask; Q.tile_first = w.tile_first; Q.hdr = w.hdr; Q.tab = v->tab; Q.toktab = v->toktab; Q.longtab = v->longtab;
+    Q.startmask = w.startmask; Q.tile_first = w.tile_first; Q.hdr = w.hdr; Q.tab = v->tab; Q.toktab = v->toktab; Q.longtab = v->longtab; Q.litstart = literals ? w.litstart : nullptr;
     Q.ext_id = v->d_ext_id; Q.piece_cnt = w.piece_cnt; Q.stage = w.stage; Q.pairbuf = w.pairbuf; Q.tile_tok = w.tile_tok; Q.grp_tok = w.grp_tok;
     if (ev) k_pieces<<<tile_grid, BPE_THREADS, 0, st>>>(Q);
     else CK(launch_after(k_pieces, tile_grid, BPE_THREADS, st, Q));
@@ -437,6 +459,45 @@ extern "C" int tt_encode(const tt_vocab* v, const uint8_t* text, size_t len, voi
     if (!count_out || !status_out || (len && !ids_out)) return TT_ERR_ARG;
     return encode_impl(v, text, len, nullptr, 1, (cudaStream_t)stream, ids_out, ids_cap, count_out, nullptr, status_out,
                        workspace);
+}
+
+extern "C" int tt_vocab_add_literals(tt_vocab* v, const uint8_t* bytes, const uint32_t* off, const int32_t* ids, size_t n) {
+    if (!v || v->lit.n != 0 || n == 0 || n > 65535 || !bytes || !off || !ids) return TT_ERR_ARG;
+    std::vector<LitEntry> e(n);
+    std::unordered_set<std::string> seen;
+    u32 maxlen = 0;
+    LitTable T{};
+    for (size_t i = 0; i < n; i++) {
+        if (off[i + 1] <= off[i] || off[i + 1] - off[i] > 255 || ids[i] < 0) return TT_ERR_ARG;
+        const u32 len = off[i + 1] - off[i];
+        if (!seen.insert(std::string((const char*)bytes + off[i], len)).second) return TT_ERR_ARG;     // the same literal twice
+        u32 f4 = 0;
+        for (u32 k = 0; k < 4 && k < len; k++) f4 |= (u32)bytes[off[i] + k] << (8 * k);
+        e[i].first4 = f4; e[i].off = off[i]; e[i].len = len; e[i].id = ids[i];
+        maxlen = maxlen > len ? maxlen : len;
+        T.first_byte[bytes[off[i]] >> 5] |= 1u << (bytes[off[i]] & 31);
+    }
+    std::stable_sort(e.begin(), e.end(), [](const LitEntry& a, const LitEntry& b) { return a.len > b.len; });
+    const size_t blob = off[n];
+    if (cudaMalloc(&v->d_lit_entries, n * sizeof(LitEntry)) != cudaSuccess || cudaMalloc(&v->d_lit_blob, blob + 16) != cudaSuccess ||
+        cudaMemcpy(v->d_lit_entries, e.data(), n * sizeof(LitEntry), cudaMemcpyHostToDevice) != cudaSuccess ||
+        cudaMemcpy(v->d_lit_blob, bytes, blob, cudaMemcpyHostToDevice) != cudaSuccess) {
+        cudaGetLastError(); cudaFree(v->d_lit_entries); cudaFree(v->d_lit_blob); v->d_lit_entries = nullptr; v->d_lit_blob = nullptr;
+        return TT_ERR_CUDA;
+    }
+    T.entries = v->d_lit_entries; T.blob = v->d_lit_blob; T.n = (u32)n; T.maxlen = maxlen;
+    v->lit = T;
+    return TT_OK;
+}
+
+extern "C" int tt_encode_added(const tt_vocab* v, const uint8_t* text, size_t len, void* stream, int32_t* ids_out,
+                               size_t ids_cap, int64_t* count_out, int32_t* status_out, void* workspace,
+                               size_t workspace_bytes) {
+    int rc = check_common(v, text, len, workspace, workspace_bytes, 1);
+    if (rc != TT_OK) return rc;
+    if (!count_out || !status_out || (len && !ids_out)) return TT_ERR_ARG;
+    return encode_impl(v, text, len, nullptr, 1, (cudaStream_t)stream, ids_out, ids_cap, count_out, nullptr, status_out,
+                       workspace, nullptr, v->lit.n != 0);
 }
 
 extern "C" int tt_encode_batch(const tt_vocab* v, const uint8_t* text, size_t total_len, const int64_t* doc_off,

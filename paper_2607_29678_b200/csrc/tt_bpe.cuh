@@ -566,6 +566,7 @@ struct PieceParams {
     TTHeader* hdr;
     PairTable tab;
     TokTable toktab;
+    const u32* litstart;       // literal pass: a piece that begins at such a bit is an added token whose id is staged, or null
     LongTable longtab;         // ignore_merges: entries longer than the whole-piece table holds (else slots == nullptr)
     const int32_t* ext_id;
     u32* piece_cnt;            // per piece: the id itself if the piece is one token found without merging (>= 0),
@@ -646,7 +647,9 @@ k_pieces(const PieceParams P) {
             const u32 a = (u32)(t0 + tp.off[i]);
             const u32 n = (i + 1 < np ? tp.off[i + 1] : tp.end) - tp.off[i];
             int32_t id;
-            if (n == 1) { P.piece_cnt[p0 + i] = (u32)P.ext_id[text[a]]; wsum++; }
+            if (P.litstart != nullptr && ((P.litstart[((long long)a + P.shift) >> 5] >> (((long long)a + P.shift) & 31)) & 1)) {
+                P.piece_cnt[p0 + i] = 0u - 1u; wsum++;               // one staged id (written by the literal pass)
+            } else if (n == 1) { P.piece_cnt[p0 + i] = (u32)P.ext_id[text[a]]; wsum++; }
             else if (n <= TT_TOKTAB_MAXLEN && P.toktab.slots != nullptr && toktab_lookup(P.toktab, text, a, n, id)) {
                 P.piece_cnt[p0 + i] = (u32)id; wsum++;
             } else if (n > TT_TOKTAB_MAXLEN && P.longtab.slots != nullptr && n <= P.longtab.maxlen && longtab_lookup(P.longtab, text, a, n, id)) {

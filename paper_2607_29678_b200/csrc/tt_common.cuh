@@ -57,4 +57,7 @@ struct TTWorkspace {
                        // or minus the staged token count
     int32_t* stage;    // token ids staged at the byte offset of their piece (len)
     u64* pairbuf;      // (token, rank) pairs of the long-piece path, indexed like the text (len)
+    u8* cand;          // literal pass: length of the longest added-token literal starting at each byte (aligned frame)
+    u32* litstart;     // literal pass: bit per byte, first byte of an extracted literal
+    u32* litin;        // literal pass: bit per byte, the other bytes of an extracted literal
 };

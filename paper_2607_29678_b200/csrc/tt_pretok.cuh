@@ -27,6 +27,8 @@ struct PretokParams {
     int ntiles;
     int pattern;
     const u32* docmask;      // bit per byte (aligned frame) marking document starts, or null (one document)
+    const u32* litstart;     // literal pass: first bytes of extracted literals (each becomes exactly one piece), or null
+    const u32* litin;        //               their other bytes (start nothing)
     u16* startmask;          // out: one u16 per chunk
     u32* tile_cnt;           // out: pieces per tile; replaced by the exclusive prefix (ntiles + 1 entries)
     u32* tile_first;         // out: offset inside the tile of its first piece start, or ~0 if it has none

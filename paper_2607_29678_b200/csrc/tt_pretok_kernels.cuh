@@ -300,6 +300,10 @@ k_pretok(const PretokParams P) {
             S = P.pattern != 1 ? tt_eval_chunk_p0(sm, slot, P.base, g0, P.hi, tc, true, need, P.pattern == 2, P.docmask)
                                : tt_eval_chunk_p1(sm, slot, SC, g0, tc, true, need);
         }
+        if (P.litstart && c_first + tid < P.nchunks) {                // an extracted literal is one piece whatever the pattern says
+            const long long chunk = c_first + tid;
+            S = (S & ~(u32)reinterpret_cast<const u16*>(P.litin)[chunk]) | reinterpret_cast<const u16*>(P.litstart)[chunk];
+        }
         if (c_first + tid < P.nchunks) P.startmask[c_first + tid] = (u16)S;
         if (S) atomicMin(&s_first, (u32)(tid * TT_CHUNK + tt_lobit(S)));
         u32 total = cta_sum_u32(tt_popc(S), scratch);

@@ -1,0 +1,75 @@
+"""GPU added-token literal pass (tt_encode_added) against the oracle: leftmost-longest extraction, segments
+between literals tokenized as texts of their own."""
+import random
+
+import numpy as np
+import pytest
+
+import oracle
+import workloads as wl
+from gpu_util import to_dev
+
+pytestmark = pytest.mark.gpu
+
+
+def _gpu_encode_added(v, text: np.ndarray, offset: int = 0):
+    import torch
+    d = to_dev(text, offset)
+    bufs = v.alloc(max(text.size, 1))
+    v.encode_added(d, bufs, length=text.size)
+    torch.cuda.synchronize()
+    return bufs["ids"][:int(bufs["count"].item())].cpu().numpy(), int(bufs["status"].item())
+
+
+@pytest.mark.parametrize("name", ["C1", "C4"])
+def test_special_tokens_in_transcripts(name):
+    """Role markers of the synthetic transcripts as added tokens, plus literals that are ordinary words,
+    prefixes of one another and non-ASCII; misaligned text pointer included."""
+    import paper_2607_29678_b200 as tt
+    cfg = wl.CONFIGS[name]
+    merges, byte_map = wl.load_vocab(cfg)
+    cv = oracle.Vocab(merges, byte_map)
+    gv = tt.Vocab(merges, byte_map, cfg.pattern_id)
+    lits = ["<|user|>", "<|assistant|>", "<|tool|>", "<|", "the", "there", "é中", "\n\n", "```python", "```", "    "]
+    ids = [500000 + k for k in range(len(lits))]
+    gv.add_literals(lits, ids)
+    text = wl.generate(wl.KIND_TRANSCRIPT_ADV if name == "C4" else wl.KIND_TRANSCRIPT, 321, 120_000)
+    text = np.concatenate([text, np.frombuffer("<|user|><|user|>é中é中<|<|assistant|>there the".encode(), dtype=np.uint8)])
+    for offset in (0, 5):
+        got, status = _gpu_encode_added(gv, text, offset)
+        want = oracle.encode_added(cv, text, cfg.pattern_id, lits, ids)
+        assert status == 0 and np.array_equal(got, want)
+    assert (want >= 500000).sum() > 100
+
+
+def test_overlapping_literal_chains_and_edges():
+    import paper_2607_29678_b200 as tt
+    merges, byte_map = wl.load_vocab(wl.CONFIGS["C1"])
+    cv = oracle.Vocab(merges, byte_map)
+    rng = random.Random(9)
+    for trial in range(40):
+        alpha = rng.choice(["ab", "abc<|>", "a<", "a é"])
+        lits = sorted({"".join(rng.choice(alpha) for _ in range(rng.randrange(1, 6))) for _ in range(rng.randrange(1, 7))})
+        lits = [x for x in lits if x.strip() or len(x) > 1] or ["ab"]
+        ids = [700000 + k for k in range(len(lits))]
+        gv = tt.Vocab(merges, byte_map, 0)
+        gv.add_literals(lits, ids)
+        for n in (0, 1, 2, 7, 60, 3000, 70000):
+            s = "".join(rng.choice(alpha) for _ in range(n))
+            if rng.random() < 0.3 and n > 10:
+                s = s[:n // 2] + "a" * 5000 + s[n // 2:]          # a long chain of overlapping candidates
+            text = np.frombuffer(s.encode(), dtype=np.uint8)
+            got, status = _gpu_encode_added(gv, text)
+            want = oracle.encode_added(cv, text, 0, lits, ids)
+            assert status == 0 and np.array_equal(got, want), (lits, s[:80])
+    # without registered literals the call is tt_encode
+    gv = tt.Vocab(merges, byte_map, 0)
+    text = wl.request(wl.CONFIGS["C1"])
+    got, status = _gpu_encode_added(gv, text)
+    assert status == 0 and np.array_equal(got, cv.encode(text, 0)[0])
+    # argument checks
+    with pytest.raises(tt.TokTierError):
+        gv.add_literals(["x", "x"], [1, 2])
+    gv.add_literals(["x"], [1])
+    with pytest.raises(tt.TokTierError):
+        gv.add_literals(["y"], [2])

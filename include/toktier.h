@@ -219,6 +219,36 @@ int tt_session_copy(const tt_session* s, int32_t* ids_out, size_t ids_cap, int32
                     void* stream);
 
 /*
+ * Shadow verification (paper Sec. 4.4): a background thread re-tokenizes a sample of the emitted sequences with a
+ * reference engine and compares ids exactly; a mismatch is quarantined with a content hash for offline
+ * reproduction; if the thread falls behind, samples are dropped and a visible counter is incremented.  Host only
+ * (no GPU call); the reference engine is a callback of the caller.
+ *   tt_verifier_create    reference(user, text, len, ids_out, ids_cap, count_out) must write the reference ids of
+ *                         `text` (HOST buffers; ids_cap = len + 1) and return 0, or non-zero on failure (counted as
+ *                         a mismatch).  sample_rate in [0, 1] (the paper serves with 0.05 and sweeps offline with 1);
+ *                         queue_cap > 0 = samples that may wait; seed fixes which submissions are sampled.
+ *   tt_verifier_submit    HOST text and ids of one emitted sequence (copied if sampled).  Returns 1 = queued,
+ *                         0 = not sampled, 2 = sampled but dropped (queue full), -1 = bad arguments.  Never blocks
+ *                         on the reference engine.
+ *   tt_verifier_drain     waits until every queued sample has been checked.
+ *   tt_verifier_get_stats counters so far.   tt_verifier_quarantined: mismatch `index` (0-based, at most 4,096 are
+ *                         kept): 64-bit FNV-1a hash and length of its text, index of the first differing id (or
+ *                         the shorter length; -2 if the reference engine failed).
+ *   tt_verifier_free      finishes queued samples, stops the thread.
+ */
+typedef int (*tt_reference_fn)(void* user, const uint8_t* text, size_t len, int32_t* ids_out, size_t ids_cap,
+                               int64_t* count_out);
+typedef struct tt_verifier tt_verifier;
+typedef struct { uint64_t submitted, sampled, checked, mismatches, dropped; } tt_verifier_stats;
+int tt_verifier_create(tt_reference_fn reference, void* user, double sample_rate, size_t queue_cap, uint64_t seed,
+                       tt_verifier** out);
+int tt_verifier_submit(tt_verifier* q, const uint8_t* text, size_t len, const int32_t* ids, size_t n_ids);
+void tt_verifier_drain(tt_verifier* q);
+void tt_verifier_get_stats(tt_verifier* q, tt_verifier_stats* out);
+int tt_verifier_quarantined(tt_verifier* q, size_t index, uint64_t* content_hash, uint64_t* len, int64_t* first_diff);
+void tt_verifier_free(tt_verifier* q);
+
+/*
  * tt_encode_timed -- diagnostic variant of tt_encode (same arguments and results) that records
  * CUDA events on `stream` between the kernels of the chain, waits for the last one and returns the
  * device time of each step in milliseconds: ms_out[0] tag + piece-start flags and the tile

@@ -21,9 +21,12 @@ TT_VOCAB_IGNORE_MERGES = 1
 
 EXPORTS = ["tt_vocab_load", "tt_vocab_load_ex", "tt_vocab_free", "tt_workspace_bytes", "tt_encode", "tt_encode_batch",
            "tt_pretokenize", "tt_encode_timed", "tt_encode_host", "tt_encode_static", "tt_spans", "tt_spans_workspace_bytes", "tt_class_table", "tt_strerror",
-           "tt_session_create", "tt_session_free", "tt_session_set_window", "tt_session_append", "tt_session_view", "tt_session_copy", "tt_vocab_add_literals", "tt_encode_added"]
+           "tt_session_create", "tt_session_free", "tt_session_set_window", "tt_session_append", "tt_session_view", "tt_session_copy", "tt_vocab_add_literals", "tt_encode_added",
+           "tt_verifier_create", "tt_verifier_submit", "tt_verifier_drain", "tt_verifier_get_stats", "tt_verifier_quarantined", "tt_verifier_free"]
 
 _lib = None
+REFERENCE_FN = ctypes.CFUNCTYPE(ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p, ctypes.c_size_t,
+                                ctypes.POINTER(ctypes.c_int64))
 
 
 class TokTierError(RuntimeError):
@@ -88,6 +91,18 @@ def lib() -> ctypes.CDLL:
         L.tt_vocab_add_literals.argtypes = [c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_size_t]
         L.tt_encode_added.restype = c.c_int
         L.tt_encode_added.argtypes = L.tt_encode.argtypes
+        L.tt_verifier_create.restype = c.c_int
+        L.tt_verifier_create.argtypes = [REFERENCE_FN, c.c_void_p, c.c_double, c.c_size_t, c.c_uint64, c.POINTER(c.c_void_p)]
+        L.tt_verifier_submit.restype = c.c_int
+        L.tt_verifier_submit.argtypes = [c.c_void_p, c.c_void_p, c.c_size_t, c.c_void_p, c.c_size_t]
+        L.tt_verifier_drain.restype = None
+        L.tt_verifier_drain.argtypes = [c.c_void_p]
+        L.tt_verifier_get_stats.restype = None
+        L.tt_verifier_get_stats.argtypes = [c.c_void_p, c.c_void_p]
+        L.tt_verifier_quarantined.restype = c.c_int
+        L.tt_verifier_quarantined.argtypes = [c.c_void_p, c.c_size_t, c.POINTER(c.c_uint64), c.POINTER(c.c_uint64), c.POINTER(c.c_int64)]
+        L.tt_verifier_free.restype = None
+        L.tt_verifier_free.argtypes = [c.c_void_p]
         L.tt_session_copy.restype = c.c_int
         L.tt_session_copy.argtypes = [c.c_void_p, c.c_void_p, c.c_size_t, c.c_void_p, c.c_void_p, c.c_void_p]
         _lib = L
@@ -295,3 +310,57 @@ class Session:
         torch.cuda.synchronize()
         k = int(count.item())
         return ids[:k], off[:k + 1], n.value
+
+
+class VerifierStats(ctypes.Structure):
+    _fields_ = [(k, ctypes.c_uint64) for k in ("submitted", "sampled", "checked", "mismatches", "dropped")]
+
+
+class Verifier:
+    """tt_verifier_*: shadow verification of emitted sequences against a reference engine.
+    reference(text: bytes) -> sequence of ids (a Python callable; it runs on the verifier's thread)."""
+
+    def __init__(self, reference, sample_rate: float = 0.05, queue_cap: int = 64, seed: int = 0):
+        def _cb(user, text, n, ids_out, cap, count_out):
+            try:
+                ids = np.asarray(reference(ctypes.string_at(text, n)), dtype=np.int32)
+                if ids.size > cap:
+                    return 1
+                ctypes.memmove(ids_out, ids.ctypes.data, 4 * ids.size)
+                count_out[0] = ids.size
+                return 0
+            except Exception:
+                return 1
+        self._cb = REFERENCE_FN(_cb)              # keeps the callback alive
+        h = ctypes.c_void_p()
+        _check(lib().tt_verifier_create(self._cb, None, sample_rate, queue_cap, seed, ctypes.byref(h)), "tt_verifier_create")
+        self._h = h
+
+    def submit(self, text, ids) -> int:
+        a = np.frombuffer(bytes(text), dtype=np.uint8) if isinstance(text, (bytes, bytearray)) else np.ascontiguousarray(text, dtype=np.uint8)
+        i = np.ascontiguousarray(ids, dtype=np.int32)
+        return int(lib().tt_verifier_submit(self._h, a.ctypes.data if a.size else None, a.size, i.ctypes.data if i.size else None, i.size))
+
+    def drain(self):
+        lib().tt_verifier_drain(self._h)
+
+    def stats(self) -> dict:
+        st = VerifierStats()
+        lib().tt_verifier_get_stats(self._h, ctypes.byref(st))
+        return {k: int(getattr(st, k)) for k, _ in VerifierStats._fields_}
+
+    def quarantined(self, index: int):
+        h, n, d = ctypes.c_uint64(), ctypes.c_uint64(), ctypes.c_int64()
+        _check(lib().tt_verifier_quarantined(self._h, index, ctypes.byref(h), ctypes.byref(n), ctypes.byref(d)), "tt_verifier_quarantined")
+        return h.value, n.value, d.value
+
+    def close(self):
+        if getattr(self, "_h", None):
+            lib().tt_verifier_free(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

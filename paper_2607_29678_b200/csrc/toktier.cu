@@ -812,3 +812,122 @@ extern "C" int tt_session_copy(const tt_session* s, int32_t* ids_out, size_t ids
     CK(cudaMemcpyAsync(count_out, s->d_ntok, sizeof(int64_t), cudaMemcpyDeviceToDevice, st));
     return TT_OK;
 }
+
+// ---- shadow verification (paper Sec. 4.4) ---------------------------------------------------------------
+// Host-only: a background thread re-tokenizes a sample of the emitted sequences with a reference engine
+// supplied by the caller and compares ids exactly; mismatches are kept with a content hash; when the queue
+// is full samples are dropped and counted.
+#include <condition_variable>
+#include <deque>
+#include <thread>
+
+struct tt_verifier {
+    tt_reference_fn ref = nullptr; void* user = nullptr;
+    double rate = 1.0; size_t queue_cap = 64; uint64_t seed = 0;
+    struct Item { std::vector<u8> text; std::vector<int32_t> ids; };
+    std::deque<Item> queue;
+    std::mutex mu; std::condition_variable cv_work, cv_idle;
+    bool stop = false, busy = false;
+    tt_verifier_stats st{};
+    struct Bad { uint64_t hash; uint64_t len; int64_t first_diff; };
+    std::vector<Bad> quarantine;
+    std::thread worker;
+};
+
+static uint64_t verifier_hash(const u8* p, size_t n) {          // FNV-1a, 64 bit
+    uint64_t h = 0xCBF29CE484222325ull;
+    for (size_t i = 0; i < n; i++) { h ^= p[i]; h *= 0x100000001B3ull; }
+    return h;
+}
+static uint64_t verifier_mix(uint64_t x) {                       // splitmix64 finaliser: the sampling decision of submission x
+    x += 0x9E3779B97F4A7C15ull; x = (x ^ (x >> 30)) * 0xBF58476D1CE4E5B9ull; x = (x ^ (x >> 27)) * 0x94D049BB133111EBull;
+    return x ^ (x >> 31);
+}
+
+static void verifier_loop(tt_verifier* q) {
+    std::vector<int32_t> out;
+    for (;;) {
+        tt_verifier::Item it;
+        {
+            std::unique_lock<std::mutex> lk(q->mu);
+            q->busy = false;
+            if (q->queue.empty()) q->cv_idle.notify_all();
+            q->cv_work.wait(lk, [&] { return q->stop || !q->queue.empty(); });
+            if (q->queue.empty()) return;                        // stop requested and nothing left
+            it = std::move(q->queue.front()); q->queue.pop_front();
+            q->busy = true;
+        }
+        out.assign(it.text.size() + 1, 0);
+        int64_t n = 0;
+        const int rc = q->ref(q->user, it.text.data(), it.text.size(), out.data(), out.size(), &n);
+        int64_t diff = -1;
+        if (rc != 0 || n < 0 || (size_t)n != it.ids.size()) diff = rc != 0 ? -2 : (int64_t)std::min<size_t>((size_t)(n < 0 ? 0 : n), it.ids.size());
+        if (diff == -1) for (size_t i = 0; i < it.ids.size(); i++) if (out[i] != it.ids[i]) { diff = (int64_t)i; break; }
+        std::lock_guard<std::mutex> lk(q->mu);
+        q->st.checked++;
+        if (diff != -1) {
+            q->st.mismatches++;
+            if (q->quarantine.size() < 4096) q->quarantine.push_back({verifier_hash(it.text.data(), it.text.size()), it.text.size(), diff});
+        }
+    }
+}
+
+extern "C" int tt_verifier_create(tt_reference_fn reference, void* user, double sample_rate, size_t queue_cap, uint64_t seed,
+                                  tt_verifier** out) {
+    if (out) *out = nullptr;
+    if (!reference || !out || !(sample_rate >= 0.0 && sample_rate <= 1.0) || queue_cap == 0) return TT_ERR_ARG;
+    tt_verifier* q = new (std::nothrow) tt_verifier();
+    if (!q) return TT_ERR_CUDA;
+    q->ref = reference; q->user = user; q->rate = sample_rate; q->queue_cap = queue_cap; q->seed = seed;
+    q->worker = std::thread(verifier_loop, q);
+    *out = q;
+    return TT_OK;
+}
+
+extern "C" int tt_verifier_submit(tt_verifier* q, const uint8_t* text, size_t len, const int32_t* ids, size_t n_ids) {
+    if (!q || (len && !text) || (n_ids && !ids)) return -1;
+    std::unique_lock<std::mutex> lk(q->mu);
+    const uint64_t k = q->st.submitted++;
+    const double u = (double)(verifier_mix(q->seed + k) >> 11) * (1.0 / 9007199254740992.0);
+    if (!(u < q->rate)) return 0;
+    q->st.sampled++;
+    if (q->queue.size() >= q->queue_cap) { q->st.dropped++; return 2; }    // behind: drop, visibly
+    lk.unlock();
+    tt_verifier::Item it;
+    it.text.assign(text, text + len); it.ids.assign(ids, ids + n_ids);
+    lk.lock();
+    if (q->queue.size() >= q->queue_cap) { q->st.dropped++; return 2; }
+    q->queue.push_back(std::move(it));
+    q->cv_work.notify_one();
+    return 1;
+}
+
+extern "C" void tt_verifier_drain(tt_verifier* q) {
+    if (!q) return;
+    std::unique_lock<std::mutex> lk(q->mu);
+    q->cv_idle.wait(lk, [&] { return q->queue.empty() && !q->busy; });
+}
+
+extern "C" void tt_verifier_get_stats(tt_verifier* q, tt_verifier_stats* out) {
+    if (!q || !out) return;
+    std::lock_guard<std::mutex> lk(q->mu);
+    *out = q->st;
+}
+
+extern "C" int tt_verifier_quarantined(tt_verifier* q, size_t index, uint64_t* content_hash, uint64_t* len, int64_t* first_diff) {
+    if (!q) return TT_ERR_ARG;
+    std::lock_guard<std::mutex> lk(q->mu);
+    if (index >= q->quarantine.size()) return TT_ERR_ARG;
+    if (content_hash) *content_hash = q->quarantine[index].hash;
+    if (len) *len = q->quarantine[index].len;
+    if (first_diff) *first_diff = q->quarantine[index].first_diff;
+    return TT_OK;
+}
+
+extern "C" void tt_verifier_free(tt_verifier* q) {
+    if (!q) return;
+    { std::lock_guard<std::mutex> lk(q->mu); q->stop = true; }
+    q->cv_work.notify_all();
+    if (q->worker.joinable()) q->worker.join();
+    delete q;
+}

@@ -47,8 +47,12 @@ enum {
  *   TT_PATTERN_O200K   case-aware word alternatives with an optional contraction suffix,
  *                      \p{N}{1,3}, ' '?[^\s\p{L}\p{N}]+[\r\n/]*, and the same whitespace rules.
  *   TT_PATTERN_CL100K_N1  TT_PATTERN_CL100K with \p{N} in place of \p{N}{1,3}: every digit is its own piece
- *                      (the "\p{N} single" front end of the paper's family table, App. A). */
-enum { TT_PATTERN_CL100K = 0, TT_PATTERN_O200K = 1, TT_PATTERN_CL100K_N1 = 2 };
+ *                      (the "\p{N} single" front end of the paper's family table, App. A).
+ *   TT_PATTERN_SPLIT3  three splitters in sequence (Sec. 4.1: each re-splits every piece of the stage before it, unmatched
+ *                      spans survive as pieces): \p{N}{1,3} isolated, then [\p{Lm}\p{Lo}]+ isolated, then TT_PATTERN_CL100K
+ *                      on every resulting span as a text of its own.  The paper prints no pattern of this family; this
+ *                      composition is a stand-in with the same structure. */
+enum { TT_PATTERN_CL100K = 0, TT_PATTERN_O200K = 1, TT_PATTERN_CL100K_N1 = 2, TT_PATTERN_SPLIT3 = 3 };
 
 typedef struct tt_vocab tt_vocab;   /* opaque; immutable after load; owns its device tables */
 
@@ -62,7 +66,7 @@ typedef struct { int32_t left, right, result; } tt_merge;
  *             (a value of byte_map) or the `result` of a LOWER-ranked merge; pairs must be distinct;
  *             results must be distinct, non-negative and differ from every base id.
  *   byte_map  HOST, 256 entries: byte value -> base token id; must be injective and non-negative.
- *   pattern_id  TT_PATTERN_CL100K, TT_PATTERN_O200K or TT_PATTERN_CL100K_N1.
+ *   pattern_id  TT_PATTERN_CL100K, TT_PATTERN_O200K, TT_PATTERN_CL100K_N1 or TT_PATTERN_SPLIT3.
  *   out       receives the handle (device tables live on the current CUDA device).
  * Limits: n_merges <= 262,144 - 256.  Synchronous (it waits for its own uploads).
  * Returns TT_OK, TT_ERR_ARG, TT_ERR_BAD_VOCAB or TT_ERR_CUDA; *out is NULL on failure.

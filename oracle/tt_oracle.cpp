@@ -192,7 +192,7 @@ struct Matcher {
 };
 
 /* piece starts as code-point indices */
-void pretok_cp(const Text &t, int pattern, std::vector<size_t> &starts) {
+void pretok_plain(const Text &t, int pattern, std::vector<size_t> &starts) {
     Matcher M(t);
     if (pattern == 2) M.maxDigits = 1;        /* pattern 2 = pattern 0 with \p{N} in place of \p{N}{1,3} */
     size_t p = 0;
@@ -203,6 +203,45 @@ void pretok_cp(const Text &t, int pattern, std::vector<size_t> &starts) {
         if (m == 0) m = 1;   /* cannot happen: every position matches some alternative */
         p += m;
     }
+}
+
+/* Pattern 3: three splitters in sequence (paper Sec. 4.1: each splitter re-splits every piece of the stage
+ * before it, and the spans a splitter does not match survive as pieces of their own).
+ *   A  \p{N}{1,3}        matches isolated
+ *   B  [\p{Lm}\p{Lo}]+   (caseless letters: CJK and the like) matches isolated
+ *   C  pattern 0 applied to every piece of A.B as a text of its own
+ * The paper prints no such pattern; this composition is this build's stand-in for the family it names. */
+void pretok_split3(const Text &t, std::vector<size_t> &starts) {
+    const size_t n = t.cp.size();
+    std::vector<std::pair<size_t, size_t>> a_spans, b_spans;
+    for (size_t p = 0; p < n;) {                              /* A */
+        size_t e = p;
+        if (g_cls[t.cp[p]] == K_N) { while (e < n && e < p + 3 && g_cls[t.cp[e]] == K_N) e++; }
+        else { while (e < n && g_cls[t.cp[e]] != K_N) e++; }
+        a_spans.push_back({p, e});
+        p = e;
+    }
+    for (auto sp : a_spans) {                                 /* B, inside every span of A */
+        for (size_t p = sp.first; p < sp.second;) {
+            const bool in = g_cls[t.cp[p]] == K_LB;
+            size_t e = p;
+            while (e < sp.second && (g_cls[t.cp[e]] == K_LB) == in) e++;
+            b_spans.push_back({p, e});
+            p = e;
+        }
+    }
+    starts.clear();
+    for (auto sp : b_spans) {                                 /* C: pattern 0 on the span alone */
+        Text sub;
+        sub.cp.assign(t.cp.begin() + sp.first, t.cp.begin() + sp.second);
+        std::vector<size_t> st;
+        pretok_plain(sub, 0, st);
+        for (size_t x : st) starts.push_back(sp.first + x);
+    }
+}
+
+void pretok_cp(const Text &t, int pattern, std::vector<size_t> &starts) {
+    if (pattern == 3) pretok_split3(t, starts); else pretok_plain(t, pattern, starts);
 }
 
 /* ------------------------------------------------------------------------------- BPE */

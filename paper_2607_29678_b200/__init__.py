@@ -16,7 +16,7 @@ LIB_PATH = os.path.join(_HERE, "libtoktier.so")
 
 TT_OK, TT_ERR_ARG, TT_ERR_BAD_VOCAB, TT_ERR_CUDA, TT_ERR_INVALID_UTF8, TT_ERR_CAPACITY, TT_ERR_INTERNAL_TIMEOUT, TT_ERR_TOO_LARGE, TT_ERR_BAD_IDS = range(9)
 TT_STATIC_MAX_LEN = 262144
-TT_PATTERN_CL100K, TT_PATTERN_O200K, TT_PATTERN_CL100K_N1 = 0, 1, 2
+TT_PATTERN_CL100K, TT_PATTERN_O200K, TT_PATTERN_CL100K_N1, TT_PATTERN_SPLIT3 = 0, 1, 2, 3
 TT_VOCAB_IGNORE_MERGES = 1
 
 EXPORTS = ["tt_vocab_load", "tt_vocab_load_ex", "tt_vocab_free", "tt_workspace_bytes", "tt_encode", "tt_encode_batch",

@@ -223,7 +223,7 @@ extern "C" int tt_vocab_load_ex(const tt_merge* merges, size_t n_merges, const i
                                 unsigned flags, tt_vocab** out) {
     if (out) *out = nullptr;
     if (!out || !byte_map || (n_merges && !merges) || (flags & ~TT_VOCAB_IGNORE_MERGES)) return TT_ERR_ARG;
-    if (pattern_id != TT_PATTERN_CL100K && pattern_id != TT_PATTERN_O200K && pattern_id != TT_PATTERN_CL100K_N1) return TT_ERR_ARG;
+    if (pattern_id != TT_PATTERN_CL100K && pattern_id != TT_PATTERN_O200K && pattern_id != TT_PATTERN_CL100K_N1 && pattern_id != TT_PATTERN_SPLIT3) return TT_ERR_ARG;
     if (n_merges > TT_MAX_INTERNAL - 256) return TT_ERR_ARG;
     // external id -> internal id (byte b -> b, result of rank r -> 256 + r)
     std::unordered_map<int32_t, u32> internal;
@@ -332,6 +332,7 @@ static size_t carve(TTWorkspace* w, void* base, size_t max_len, size_t max_docs)
     p = take(padded + 16);                      if (w) w->cand = (u8*)p;
     p = take((padded / 32 + 4) * sizeof(u32));  if (w) w->litstart = (u32*)p;
     p = take((padded / 32 + 4) * sizeof(u32));  if (w) w->litin = (u32*)p;
+    p = take((padded / 32 + 4) * sizeof(u32));  if (w) w->cutmask = (u32*)p;
     return off;
 }
 
@@ -379,6 +380,15 @@ static int run_pretok(const tt_vocab* v, const uint8_t* text, size_t len, const 
     }
     const size_t smem = align_up(v->cls_bytes, 16) + sizeof(u16) * F_COUNT * TT_SLOTS;
     const int grid = P.ntiles < v->sm_count * 6 ? P.ntiles : v->sm_count * 6;
+    if (v->pattern == TT_PATTERN_SPLIT3) {
+        // stages A and B: span starts into cutmask (with the caller's document starts); stage C: pattern 0 with
+        // those cuts as its document boundaries
+        PretokParams C1 = P;
+        C1.pattern = TT_PATTERN_CUTS; C1.startmask = reinterpret_cast<u16*>(w.cutmask); C1.tile_tok = nullptr; C1.grp_tok = nullptr;
+        C1.want_prefix = 0; C1.litstart = nullptr; C1.litin = nullptr;
+        k_pretok<<<grid, TT_TILE_CHUNKS, smem, st>>>(C1);
+        P.pattern = TT_PATTERN_CL100K; P.docmask = w.cutmask;
+    }
     k_pretok<<<grid, TT_TILE_CHUNKS, smem, st>>>(P);
     if (piece_off_dst)
         k_compact<<<grid, TT_TILE_CHUNKS, 0, st>>>(w.startmask, w.tile_cnt, P.nchunks, P.ntiles, shift, (long long)len,

@@ -60,4 +60,5 @@ struct TTWorkspace {
     u8* cand;          // literal pass: length of the longest added-token literal starting at each byte (aligned frame)
     u32* litstart;     // literal pass: bit per byte, first byte of an extracted literal
     u32* litin;        // literal pass: bit per byte, the other bytes of an extracted literal
+    u32* cutmask;      // three-splitter composition: bit per byte, span starts of the first two stages
 };

@@ -148,6 +148,44 @@ TT_HD int tt_contraction_len(u32 b1, u32 b2) {
     return 0;
 }
 
+// First two stages of the three-splitter composition (paper Sec. 4.1: three splitters applied in sequence
+// fold into the same per-character predicate, provided each splitter re-splits every piece of the stage
+// before it and unmatched spans survive as pieces): number groups of up to three digits and runs of
+// caseless letters are isolated.  Returns the 16 cut bits of the chunk in `slot`: a bit where a span of
+// these two stages begins.  The third stage (pattern 0) then runs with the cuts as document boundaries,
+// i.e. on every span as a text of its own.
+constexpr int TT_PATTERN_CUTS = 100;              // internal pattern id of this pass
+TT_HD u32 tt_eval_chunk_cuts(const u16 (*sm)[TT_SLOTS], int slot, const TileCarry& tc, bool have_tc, u32& need) {
+    const u64 OWN = 0xFFFFull << 16;
+    const u64 lead = tt_win(sm, F_LEAD, slot), N = tt_win(sm, F_NUM, slot), C = tt_win(sm, F_CLESS, slot), D = tt_win(sm, F_DOC, slot);
+    const u64 nD = ~D;
+#define PREV(x) (((x) << 1) & nD)
+    u64 S = D;
+    S |= lead & ~N & PREV(N);                        // first character after a number run
+    S |= C & lead & ~PREV(C);                        // a run of caseless letters begins
+    S |= lead & ~C & PREV(C);                        // first character after such a run
+    const u32 n_own = (u32)(N >> 16) & 0xFFFFu, ld_own = (u32)(lead >> 16) & 0xFFFFu;
+    const u32 nstart = (u32)((N & ~PREV(N)) >> 16) & 0xFFFFu;
+    u32 m = n_own & ld_own;
+    if (m) {                                         // every third number lead counted from the run start
+        u32 cnt = 0;
+        if ((n_own & 1) && !(nstart & 1)) {
+            bool open;
+            cnt = tt_walk_back_num(sm, slot - 1, open);
+            if (open) { if (have_tc) cnt += tc.n_before; else need |= NEED_N; }
+            cnt %= 3;
+        }
+        while (m) {
+            const int i = tt_lobit(m); m &= m - 1;
+            if ((nstart >> i) & 1) cnt = 0;
+            if (cnt == 0) S |= 1ull << (16 + i);
+            cnt = cnt == 2 ? 0 : cnt + 1;
+        }
+    }
+#undef PREV
+    return (u32)((S & lead & OWN) >> 16);
+}
+
 // Pattern 0 (cl100k-style).  Returns the 16 start bits of the chunk in `slot`; `need` receives the
 // NEED_* flags of aggregates that leave the shared-memory window (then `tc` must be filled and the
 // function called again).

@@ -272,7 +272,8 @@ k_pretok(const PretokParams P) {
         u32 need = 0;
         const int slot = tid + TT_LOW_HALO;
         const long long g0 = (c_first + tid) * TT_CHUNK;
-        u32 S = P.pattern != 1 ? tt_eval_chunk_p0(sm, slot, P.base, g0, P.hi, tc, false, need, P.pattern == 2, P.docmask)
+        u32 S = P.pattern == TT_PATTERN_CUTS ? tt_eval_chunk_cuts(sm, slot, tc, false, need)
+              : P.pattern != 1 ? tt_eval_chunk_p0(sm, slot, P.base, g0, P.hi, tc, false, need, P.pattern == 2, P.docmask)
                                : tt_eval_chunk_p1(sm, slot, SC, g0, tc, false, need);
         if (need) atomicOr(&s_need, need);
         __syncthreads();
@@ -297,7 +298,8 @@ k_pretok(const PretokParams P) {
                 tc.sure_before = (ev & 1) ? (coop_back_event(P, T, (ev >> 1) + 1, true, scratch) >> 1) : (ev >> 1);
             }
             need = 0;
-            S = P.pattern != 1 ? tt_eval_chunk_p0(sm, slot, P.base, g0, P.hi, tc, true, need, P.pattern == 2, P.docmask)
+            S = P.pattern == TT_PATTERN_CUTS ? tt_eval_chunk_cuts(sm, slot, tc, true, need)
+              : P.pattern != 1 ? tt_eval_chunk_p0(sm, slot, P.base, g0, P.hi, tc, true, need, P.pattern == 2, P.docmask)
                                : tt_eval_chunk_p1(sm, slot, SC, g0, tc, true, need);
         }
         if (P.litstart && c_first + tid < P.nchunks) {                // an extracted literal is one piece whatever the pattern says

@@ -34,3 +34,32 @@ def engine_starts(compiled, s: str):
         b += len(s[p:m.end()].encode("utf-8"))
         p = m.end()
     return out
+
+
+# pattern 3: three splitters in sequence, matches isolated, unmatched spans kept as pieces (paper Sec. 4.1)
+SPLIT3_A = r"\p{N}{1,3}"
+SPLIT3_B = r"[\p{Lm}\p{Lo}]+"
+
+
+def split_isolated(compiled, s: str, lo: int, hi: int):
+    """Spans of s[lo:hi]: the matches of `compiled` and the gaps between them, in order."""
+    out, p = [], lo
+    for m in compiled.finditer(s, lo, hi):
+        if m.start() > p:
+            out.append((p, m.start()))
+        out.append((m.start(), m.end()))
+        p = m.end()
+    if p < hi:
+        out.append((p, hi))
+    return out
+
+
+def engine_starts_split3(ra, rb, r0, s: str):
+    """Piece start BYTE offsets of the composition A, B, then pattern 0 on every piece as a text of its own."""
+    starts = []
+    for a0, a1 in split_isolated(ra, s, 0, len(s)):
+        for b0, b1 in split_isolated(rb, s, a0, a1):
+            piece = s[b0:b1]
+            base = len(s[:b0].encode("utf-8"))
+            starts.extend(base + x for x in engine_starts(r0, piece))
+    return starts

@@ -465,3 +465,49 @@ def test_ignore_merges_whole_piece_rule():
     ids, status = gpu_encode(tt.Vocab(merges, byte_map, cfg.pattern_id, ignore_merges=True), text)
     want, _ = oracle.Vocab(merges, byte_map, ignore_merges=True).encode(text, cfg.pattern_id, nthreads=4)
     assert status == 0 and np.array_equal(ids, want)
+
+
+def test_three_splitter_composition():
+    """TT_PATTERN_SPLIT3 (paper Sec. 4.1: three splitters in sequence): piece boundaries and IDs against the
+    oracle's pattern 3 -- exhaustive small alphabets and random Unicode documents in one batch, long digit and
+    caseless runs across tiles, a CJK-heavy request as one document."""
+    import paper_2607_29678_b200 as tt
+    merges, byte_map = wl.load_vocab(wl.CONFIGS["C2"])
+    gv = tt.Vocab(merges, byte_map, tt.TT_PATTERN_SPLIT3)
+    cv = cpu_vocab("C2")
+    rng = random.Random(33)
+    docs = _alphabet_docs("a1中 ", 6) + _alphabet_docs("1中x' \n", 5) + _alphabet_docs("12 !文a\t", 5)
+    for _ in range(300):
+        parts = []
+        for _ in range(rng.randrange(1, 6)):
+            k = rng.randrange(6)
+            if k == 0:
+                parts.append("7" * rng.randrange(1, 9000))
+            elif k == 1:
+                parts.append("中" * rng.randrange(1, 3000))
+            elif k == 2:
+                parts.append(" " * rng.randrange(1, 3000) + rng.choice(["1", "中", "x", ""]))
+            elif k == 3:
+                parts.append(rng.choice(["abc", "x's", "!!", "\n\n", "٣٣٣٣"]) * rng.randrange(1, 50))
+            elif k == 4:
+                parts.append("".join(rng.choice("ab12中文 \n'!") for _ in range(rng.randrange(1, 200))))
+            else:
+                parts.append("12中34文56 x")
+        docs.append("".join(parts).encode("utf-8"))
+    text = np.frombuffer(b"".join(docs), dtype=np.uint8)
+    off = np.zeros(len(docs) + 1, dtype=np.int64)
+    off[1:] = np.cumsum([len(d) for d in docs])
+    got, status = gpu_pretok(gv, text, doc_off=off)
+    want = np.concatenate([oracle.pretokenize(d, 3) + off[i] for i, d in enumerate(docs)])
+    assert status == 0
+    if got.size != want.size or not np.array_equal(got, want):
+        bad = sorted(set(got.tolist()) ^ set(want.tolist()))[:3]
+        which = [int(np.searchsorted(off, b, side="right") - 1) for b in bad]
+        raise AssertionError(f"piece mismatch in documents {[docs[w][:80] for w in which]}")
+    ids, ioff, status = gpu_encode_batch(gv, text, off)
+    want_ids, woff = cv.encode_batch(text, off, 3, nthreads=8)
+    assert status == 0 and np.array_equal(ioff, woff) and np.array_equal(ids, want_ids)
+    big = wl.generate(wl.KIND_TRANSCRIPT_ADV, 77, 300_000)
+    ids, status = gpu_encode(gv, big, offset=3)
+    want_ids, _ = cv.encode(big, 3, nthreads=8)
+    assert status == 0 and np.array_equal(ids, want_ids)

@@ -174,3 +174,28 @@ def test_strict_utf8(data, ok):
     if not ok:
         with pytest.raises(oracle.InvalidUtf8):
             oracle.pretokenize(data, 0)
+
+
+def test_pattern3_three_splitter_composition_equals_engine():
+    """Pattern 3 against the regex engine doing the three stages one after the other (isolated matches, gaps
+    kept, each piece re-split by the next stage): exhaustive small alphabets and random Unicode strings."""
+    from patterns import SPLIT3_A, SPLIT3_B, engine_starts_split3
+    ra, rb = regex.compile(SPLIT3_A), regex.compile(SPLIT3_B)
+    n = 0
+    for alphabet, maxlen in [("a1中 ", 6), ("1中x' \n", 5), ("12 !中文a", 5)]:
+        for ln in range(1, maxlen + 1):
+            for tup in itertools.product(alphabet, repeat=ln):
+                s = "".join(tup)
+                assert engine_starts_split3(ra, rb, R[0], s) == list(oracle.pretokenize(s, 3)), repr(s)
+                n += 1
+    assert n > 20000
+    pool = _agreeing_codepoints()
+    rng = random.Random(12)
+    special = list(" \t\n\r'/!.,0123456789中文") + ["'s", "\r\n", "  ", "1234567"]
+    for _ in range(3000):
+        k = rng.randrange(1, 40)
+        s = "".join(rng.choice(special) if rng.random() < 0.5 else chr(rng.choice(pool)) for _ in range(k))
+        assert engine_starts_split3(ra, rb, R[0], s) == list(oracle.pretokenize(s, 3)), repr(s)
+    # the composition is not pattern 0: context is cut at the stage boundaries
+    assert [p.decode() for p in oracle.pieces("x  12", 3)] == ["x", "  ", "12"]
+    assert [p.decode() for p in oracle.pieces("x  12", 0)] == ["x", " ", " ", "12"]

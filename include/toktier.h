@@ -267,9 +267,12 @@ int tt_encode_timed(const tt_vocab* v, const uint8_t* text, size_t len, void* st
 
 /*
  * tt_encode_host -- convenience wrapper for HOST buffers: copies `text` to the device, encodes,
- * copies IDs back and synchronises.  Allocates and caches its own device and pinned staging
+ * delivers the IDs to `ids_out` and synchronises.  Allocates and caches its own device and pinned staging
  * buffers inside the handle's context (not thread-safe per vocab).  ids_out HOST int32[ids_cap];
- * *count_out HOST.  Returns the host code, or the device status if that is not TT_OK.
+ * *count_out HOST.  Page-locked caller buffers (cudaHostAlloc / cudaHostRegister, a pinned tensor) are used
+ * directly: `text` is the source of the DMA, and the IDs are written by the scatter kernel through the mapped
+ * pointer straight into `ids_out` (entries beyond the count are unspecified); pageable buffers are staged.
+ * Returns the host code, or the device status if that is not TT_OK.
  */
 int tt_encode_host(tt_vocab* v, const uint8_t* text, size_t len, int32_t* ids_out, size_t ids_cap,
                    int64_t* count_out);

@@ -259,6 +259,17 @@ class Vocab:
                "tt_encode_host")
         return out[:cnt.value]
 
+    def encode_host_into(self, text, ids_out) -> int:
+        """tt_encode_host on caller buffers: `text` a uint8 host tensor / array, `ids_out` an int32 host tensor /
+        array that receives the ids; returns the count.  Pinned tensors are used without staging."""
+        tp = text.data_ptr() if hasattr(text, "data_ptr") else text.ctypes.data
+        tn = text.numel() if hasattr(text, "numel") else text.size
+        op = ids_out.data_ptr() if hasattr(ids_out, "data_ptr") else ids_out.ctypes.data
+        on = ids_out.numel() if hasattr(ids_out, "numel") else ids_out.size
+        cnt = ctypes.c_int64(0)
+        _check(lib().tt_encode_host(self._h, tp, tn, op, on, ctypes.byref(cnt)), "tt_encode_host")
+        return cnt.value
+
 
 class AppendInfo(ctypes.Structure):
     """tt_append_info."""

@@ -593,6 +593,15 @@ extern "C" int tt_spans(const tt_vocab* v, const int32_t* ids, const int64_t* co
     return TT_OK;
 }
 
+// Is p page-locked host memory?  dev_view (optional) receives the pointer a kernel may use to reach it.
+static bool host_pointer_is_pinned(const void* p, void** dev_view) {
+    cudaPointerAttributes a;
+    if (cudaPointerGetAttributes(&a, p) != cudaSuccess) { cudaGetLastError(); return false; }
+    if (a.type != cudaMemoryTypeHost) return false;
+    if (dev_view) *dev_view = a.devicePointer;
+    return true;
+}
+
 extern "C" int tt_encode_host(tt_vocab* v, const uint8_t* text, size_t len, int32_t* ids_out, size_t ids_cap,
                               int64_t* count_out) {
     if (!v || !count_out || (len && (!text || !ids_out))) return TT_ERR_ARG;
@@ -617,20 +626,35 @@ extern "C" int tt_encode_host(tt_vocab* v, const uint8_t* text, size_t len, int3
         v->host_cap = cap;
     }
     cudaStream_t st = v->host_stream;
-    memcpy(v->h_text, text, len);
-    CK(cudaMemcpyAsync(v->d_text, v->h_text, len, cudaMemcpyHostToDevice, st));
-    int rc = tt_encode(v, v->d_text, len, st, v->d_ids, v->host_cap, (int64_t*)v->d_count, v->d_status, v->d_ws, v->ws_cap);
+    // Pinned (page-locked) caller buffers take no staging: the text is copied by DMA straight from the caller's
+    // buffer, and the scatter kernel writes the ids through the mapped pointer straight into the caller's
+    // buffer, so no device-to-host copy follows.  Pageable buffers go through the handle's pinned staging.
+    int32_t* ids_dev_view = nullptr;
+    const bool in_pinned = len && host_pointer_is_pinned(text, nullptr);
+    const bool out_pinned = len && host_pointer_is_pinned(ids_out, (void**)&ids_dev_view) && ids_dev_view != nullptr;
+    if (!in_pinned) memcpy(v->h_text, text, len);
+    CK(cudaMemcpyAsync(v->d_text, in_pinned ? text : v->h_text, len, cudaMemcpyHostToDevice, st));
+    // count and status are written by the kernel into mapped pinned scalars of the handle
+    long long* count_dev = nullptr; int32_t* status_dev = nullptr;
+    {
+        void* p = nullptr;
+        if (!host_pointer_is_pinned(v->h_scalars, &p) || !p) return TT_ERR_CUDA;
+        count_dev = (long long*)p; status_dev = (int32_t*)((long long*)p + 1);
+    }
+    v->h_scalars[0] = 0; v->h_scalars[1] = 0;
+    int rc = tt_encode(v, v->d_text, len, st, out_pinned ? ids_dev_view : v->d_ids, out_pinned ? ids_cap : v->host_cap,
+                       (int64_t*)count_dev, status_dev, v->d_ws, v->ws_cap);
     if (rc != TT_OK) return rc;
-    CK(cudaMemcpyAsync(&v->h_scalars[0], v->d_count, sizeof(long long), cudaMemcpyDeviceToHost, st));
-    CK(cudaMemcpyAsync(&v->h_scalars[1], v->d_status, sizeof(int32_t), cudaMemcpyDeviceToHost, st));
     CK(cudaStreamSynchronize(st));
     const int status = (int)(v->h_scalars[1] & 0xFFFFFFFF);
     if (status != TT_OK) return status;
     const long long n = v->h_scalars[0];
     if ((size_t)n > ids_cap) return TT_ERR_CAPACITY;
-    CK(cudaMemcpyAsync(v->h_ids, v->d_ids, (size_t)n * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
-    CK(cudaStreamSynchronize(st));
-    memcpy(ids_out, v->h_ids, (size_t)n * sizeof(int32_t));
+    if (!out_pinned) {
+        CK(cudaMemcpyAsync(v->h_ids, v->d_ids, (size_t)n * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+        CK(cudaStreamSynchronize(st));
+        memcpy(ids_out, v->h_ids, (size_t)n * sizeof(int32_t));
+    }
     *count_out = n;
     return TT_OK;
 }

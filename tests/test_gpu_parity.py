@@ -511,3 +511,27 @@ def test_three_splitter_composition():
     ids, status = gpu_encode(gv, big, offset=3)
     want_ids, _ = cv.encode(big, 3, nthreads=8)
     assert status == 0 and np.array_equal(ids, want_ids)
+
+
+def test_host_entry_point_with_pinned_buffers():
+    """tt_encode_host on page-locked caller buffers: no staging, ids written by the kernel into the caller's buffer."""
+    import torch
+    cfg = wl.CONFIGS["C2"]
+    text = wl.request(cfg)
+    gv, cv = gpu_vocab("C2"), cpu_vocab("C2")
+    want, _ = cv.encode(text, cfg.pattern_id, nthreads=4)
+    pinned_text = torch.from_numpy(text.copy()).pin_memory()
+    pinned_ids = torch.full((text.size + 1,), -7, dtype=torch.int32).pin_memory()
+    for _ in range(2):
+        n = gv.encode_host_into(pinned_text, pinned_ids)
+        assert n == want.size and np.array_equal(pinned_ids[:n].numpy(), want)
+    out = np.empty(text.size, dtype=np.int32)                     # pinned in, pageable out
+    n = gv.encode_host_into(pinned_text, out)
+    assert n == want.size and np.array_equal(out[:n], want)
+    n = gv.encode_host_into(text, pinned_ids)                     # pageable in, pinned out
+    assert n == want.size and np.array_equal(pinned_ids[:n].numpy(), want)
+    small = torch.empty(10, dtype=torch.int32).pin_memory()       # too small: capacity error, nothing written past it
+    import paper_2607_29678_b200 as tt
+    with pytest.raises(tt.TokTierError) as err:
+        gv.encode_host_into(pinned_text, small)
+    assert err.value.code == tt.TT_ERR_CAPACITY

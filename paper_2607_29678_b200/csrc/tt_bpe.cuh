@@ -67,31 +67,41 @@ TT_HD u32 toktab_hash(u64 k0, u64 k1, u64 k2, u32 len, u32 shift) {
     return (u32)(h >> shift);
 }
 
-// Looks a piece of 2..24 bytes up; returns true and the id on a hit.
-__device__ __forceinline__ bool toktab_lookup(const TokTable& tab, const u8* __restrict__ text, u32 a, u32 n, int32_t& id) {
+// Key of a piece of 2..24 bytes: its bytes in three words, zero padded.
+__device__ __forceinline__ void toktab_key(const u8* __restrict__ text, u32 a, u32 n, u64& k0, u64& k1, u64& k2) {
     // gather the piece's bytes with aligned 8-byte loads (only words that hold a piece byte)
     const uintptr_t addr = (uintptr_t)(text + a);
     const u64* w = reinterpret_cast<const u64*>(addr & ~(uintptr_t)7);
     const u32 sh = (u32)(addr & 7) * 8, last = (u32)(addr & 7) + n;     // bytes used in the window
     const u64 w0 = __ldg(w), w1 = last > 8 ? __ldg(w + 1) : 0, w2 = last > 16 ? __ldg(w + 2) : 0, w3 = last > 24 ? __ldg(w + 3) : 0;
-    u64 k0 = sh ? (w0 >> sh) | (w1 << (64 - sh)) : w0;
-    u64 k1 = sh ? (w1 >> sh) | (w2 << (64 - sh)) : w1;
-    u64 k2 = sh ? (w2 >> sh) | (w3 << (64 - sh)) : w2;
+    k0 = sh ? (w0 >> sh) | (w1 << (64 - sh)) : w0;
+    k1 = sh ? (w1 >> sh) | (w2 << (64 - sh)) : w1;
+    k2 = sh ? (w2 >> sh) | (w3 << (64 - sh)) : w2;
     if (n < 8) { k0 &= (1ull << (8 * n)) - 1; k1 = 0; k2 = 0; }
     else if (n < 16) { k1 &= (n == 8) ? 0 : ((1ull << (8 * (n - 8))) - 1); k2 = 0; }
     else if (n < 24) { k2 &= (n == 16) ? 0 : ((1ull << (8 * (n - 16))) - 1); }
-    u32 h = toktab_hash(k0, k1, k2, n, tab.shift);
+}
+// Probes from slot h on; lo / hi are the two halves of slot h, already loaded.
+__device__ __forceinline__ bool toktab_finish(const TokTable& tab, u64 k0, u64 k1, u64 k2, u32 n, u32 h, uint4 lo, uint4 hi, int32_t& id) {
     for (u32 probe = 0; probe <= tab.mask; probe++) {           // bounded by the capacity
-        const uint4* sp = reinterpret_cast<const uint4*>(tab.slots + h);
-        const uint4 lo = __ldg(sp), hi = __ldg(sp + 1);
         if (hi.z == 0) return false;
         if (hi.z == n && (((u64)lo.y << 32) | lo.x) == k0 && (((u64)lo.w << 32) | lo.z) == k1 && (((u64)hi.y << 32) | hi.x) == k2) {
             id = (int32_t)hi.w;
             return true;
         }
         h = (h + 1) & tab.mask;
+        const uint4* sp = reinterpret_cast<const uint4*>(tab.slots + h);
+        lo = __ldg(sp); hi = __ldg(sp + 1);
     }
     return false;
+}
+// Looks a piece of 2..24 bytes up; returns true and the id on a hit.
+__device__ __forceinline__ bool toktab_lookup(const TokTable& tab, const u8* __restrict__ text, u32 a, u32 n, int32_t& id) {
+    u64 k0, k1, k2;
+    toktab_key(text, a, n, k0, k1, k2);
+    const u32 h = toktab_hash(k0, k1, k2, n, tab.shift);
+    const uint4* sp = reinterpret_cast<const uint4*>(tab.slots + h);
+    return toktab_finish(tab, k0, k1, k2, n, h, __ldg(sp), __ldg(sp + 1), id);
 }
 
 // ---- long-entry table (ignore_merges only): vocabulary entries of more than TT_TOKTAB_MAXLEN bytes --------
@@ -643,20 +653,50 @@ k_pieces(const PieceParams P) {
         const u32 np = tp.n, p0 = (u32)tile * TT_TILE_BYTES;     // pieces are indexed per tile
         const long long t0 = c0 * TT_CHUNK - P.shift;             // text offset of the tile start
         u32 wsum = 0;
-        for (u32 i = tid; i < np; i += BPE_THREADS) {
-            const u32 a = (u32)(t0 + tp.off[i]);
-            const u32 n = (i + 1 < np ? tp.off[i + 1] : tp.end) - tp.off[i];
-            int32_t id;
-            if (P.litstart != nullptr && ((P.litstart[((long long)a + P.shift) >> 5] >> (((long long)a + P.shift) & 31)) & 1)) {
-                P.piece_cnt[p0 + i] = 0u - 1u; wsum++;               // one staged id (written by the literal pass)
-            } else if (n == 1) { P.piece_cnt[p0 + i] = (u32)P.ext_id[text[a]]; wsum++; }
-            else if (n <= TT_TOKTAB_MAXLEN && P.toktab.slots != nullptr && toktab_lookup(P.toktab, text, a, n, id)) {
-                P.piece_cnt[p0 + i] = (u32)id; wsum++;
-            } else if (n > TT_TOKTAB_MAXLEN && P.longtab.slots != nullptr && n <= P.longtab.maxlen && longtab_lookup(P.longtab, text, a, n, id)) {
-                P.piece_cnt[p0 + i] = (u32)id; wsum++;
-            } else if (n > TT_WARP_PIECE_MAX) { s_miss[TILE_MAX_PIECES - 1 - atomicAdd(&s_nlong, 1u)] = (u16)i; }   // long pieces from the back
-            else if (n > LANE_MAX) s_mid[atomicAdd(&s_nmid, 1u)] = (u16)i;
-            else s_miss[atomicAdd(&s_nmiss, 1u)] = (u16)i;
+        // two pieces per thread and step, their loads issued side by side: first the bytes of both, then the
+        // table slots of both (each lookup is a chain of two dependent loads)
+        for (u32 ib = tid; ib < np; ib += 2 * BPE_THREADS) {
+            u32 a[2], n[2], h[2], kind[2];                        // kind: 0 none, 1 literal, 2 one byte, 3 table lookup, 4 other
+            u64 k0[2], k1[2], k2[2];
+            uint4 lo[2], hi[2];
+#pragma unroll
+            for (int j = 0; j < 2; j++) {
+                const u32 i = ib + j * BPE_THREADS;
+                kind[j] = 0; a[j] = 0; n[j] = 0; k0[j] = 0; k1[j] = 0; k2[j] = 0;
+                if (i < np) {
+                    a[j] = (u32)(t0 + tp.off[i]);
+                    n[j] = (i + 1 < np ? tp.off[i + 1] : tp.end) - tp.off[i];
+                    const long long g = (long long)a[j] + P.shift;
+                    if (P.litstart != nullptr && ((P.litstart[g >> 5] >> (g & 31)) & 1)) kind[j] = 1;
+                    else if (n[j] == 1) { kind[j] = 2; k0[j] = text[a[j]]; }
+                    else if (n[j] <= TT_TOKTAB_MAXLEN && P.toktab.slots != nullptr) { kind[j] = 3; toktab_key(text, a[j], n[j], k0[j], k1[j], k2[j]); }
+                    else kind[j] = 4;
+                }
+            }
+#pragma unroll
+            for (int j = 0; j < 2; j++) {
+                h[j] = 0; lo[j] = make_uint4(0, 0, 0, 0); hi[j] = lo[j];
+                if (kind[j] == 3) {
+                    h[j] = toktab_hash(k0[j], k1[j], k2[j], n[j], P.toktab.shift);
+                    const uint4* sp = reinterpret_cast<const uint4*>(P.toktab.slots + h[j]);
+                    lo[j] = __ldg(sp); hi[j] = __ldg(sp + 1);
+                } else if (kind[j] == 2) lo[j].x = (u32)P.ext_id[(u32)k0[j]];
+            }
+#pragma unroll
+            for (int j = 0; j < 2; j++) {
+                const u32 i = ib + j * BPE_THREADS;
+                int32_t id;
+                if (kind[j] == 0) continue;
+                if (kind[j] == 1) { P.piece_cnt[p0 + i] = 0u - 1u; wsum++; }     // one staged id (written by the literal pass)
+                else if (kind[j] == 2) { P.piece_cnt[p0 + i] = lo[j].x; wsum++; }
+                else if (kind[j] == 3 && toktab_finish(P.toktab, k0[j], k1[j], k2[j], n[j], h[j], lo[j], hi[j], id)) {
+                    P.piece_cnt[p0 + i] = (u32)id; wsum++;
+                } else if (n[j] > TT_TOKTAB_MAXLEN && P.longtab.slots != nullptr && n[j] <= P.longtab.maxlen && longtab_lookup(P.longtab, text, a[j], n[j], id)) {
+                    P.piece_cnt[p0 + i] = (u32)id; wsum++;
+                } else if (n[j] > TT_WARP_PIECE_MAX) { s_miss[TILE_MAX_PIECES - 1 - atomicAdd(&s_nlong, 1u)] = (u16)i; }   // long pieces from the back
+                else if (n[j] > LANE_MAX) s_mid[atomicAdd(&s_nmid, 1u)] = (u16)i;
+                else s_miss[atomicAdd(&s_nmiss, 1u)] = (u16)i;
+            }
         }
         for (int o = 16; o; o >>= 1) wsum += __shfl_xor_sync(0xFFFFFFFFu, wsum, o);
         __syncthreads();

@@ -424,7 +424,7 @@ def main():
                 "api": "tt_encode_host, wall clock of the synchronous call; pinned host buffers: text DMA'd from the caller's "
                        "buffer, ids written by the scatter kernel into the caller's pinned buffer; pageable_p50: the same call "
                        "on pageable buffers (staged through pinned memory inside the library)"},
-        "gpu_launches": 3 * args.steps,
+        "gpu_launches": 4 * args.steps,
         "batch": batch,
         "span_export": {"ms_p50": round(pct(span_ms, 0.5), 4), "what": "tt_spans on the ids of one C3 request: byte and character "
                         "offsets per token, device to device; the paper adds 0.13-0.73 ms for this step on its hardware"},

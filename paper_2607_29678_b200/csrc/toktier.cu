@@ -155,7 +155,7 @@ static int build_token_table(tt_vocab* v, const tt_merge* merges, size_t n_merge
     for (size_t i = 0; i < np; i++) { smask[off[i] >> 4] |= (u16)(1u << (off[i] & 15)); tile_base[off[i] / TT_TILE_BYTES + 1]++;
         u32& tf = tile_first[off[i] / TT_TILE_BYTES]; if (tf == 0xFFFFFFFFu) tf = off[i] % TT_TILE_BYTES; }
     for (size_t t = 0; t < ntiles; t++) tile_base[t + 1] += tile_base[t];
-    u8* d_text = nullptr; u16* d_mask = nullptr; u32 *d_tf = nullptr, *d_cnt = nullptr, *d_tt = nullptr, *d_gt = nullptr; int32_t* d_stage = nullptr;
+    u8* d_text = nullptr; u16* d_mask = nullptr; u32 *d_tf = nullptr, *d_cnt = nullptr, *d_tt = nullptr, *d_gt = nullptr; u64 *d_qs = nullptr, *d_qw = nullptr; uint4* d_ql = nullptr; int32_t* d_stage = nullptr;
     TTHeader* d_hdr = nullptr;
     TTHeader h; memset(&h, 0, sizeof(h)); h.n_pieces = (u32)np;
     std::vector<u32> cnt(ntiles * TT_TILE_BYTES); std::vector<int32_t> stage(nb);
@@ -163,7 +163,8 @@ static int build_token_table(tt_vocab* v, const tt_merge* merges, size_t n_merge
     bool ok = cudaMalloc(&d_text, nchunks * TT_CHUNK + 64) == cudaSuccess && cudaMalloc(&d_mask, (nchunks + 1) * sizeof(u16)) == cudaSuccess &&
               cudaMalloc(&d_gt, ngroups * sizeof(u32)) == cudaSuccess && cudaMalloc(&d_tt, (ntiles + 1) * sizeof(u32)) == cudaSuccess && cudaMalloc(&d_tf, (ntiles + 1) * sizeof(u32)) == cudaSuccess &&
               cudaMalloc(&d_cnt, cnt.size() * sizeof(u32)) == cudaSuccess && cudaMalloc(&d_stage, (nb + 1) * sizeof(int32_t)) == cudaSuccess &&
-              cudaMalloc(&d_hdr, sizeof(TTHeader)) == cudaSuccess;
+              cudaMalloc(&d_hdr, sizeof(TTHeader)) == cudaSuccess && cudaMalloc(&d_qs, (nb / 2 + 64) * sizeof(u64)) == cudaSuccess &&
+              cudaMalloc(&d_qw, (nb / 33 + 64) * sizeof(u64)) == cudaSuccess && cudaMalloc(&d_ql, (nb / 257 + 16) * sizeof(uint4)) == cudaSuccess;
     ok = ok && cudaMemcpy(d_text, cat.data(), nb, cudaMemcpyHostToDevice) == cudaSuccess;
     ok = ok && cudaMemcpy(d_mask, smask.data(), (nchunks + 1) * sizeof(u16), cudaMemcpyHostToDevice) == cudaSuccess;
     ok = ok && cudaMemcpy(d_tf, tile_first.data(), (ntiles + 1) * sizeof(u32), cudaMemcpyHostToDevice) == cudaSuccess;
@@ -175,14 +176,15 @@ static int build_token_table(tt_vocab* v, const tt_merge* merges, size_t n_merge
         Q.startmask = d_mask; Q.tile_first = d_tf; Q.hdr = d_hdr; Q.tab = v->tab;
         Q.toktab.slots = nullptr; Q.toktab.mask = 0; Q.toktab.shift = 0;      // no table yet: every piece is merged
         Q.longtab = LongTable{}; Q.litstart = nullptr;
-        Q.ext_id = v->d_ext_id; Q.piece_cnt = d_cnt; Q.stage = d_stage; Q.pairbuf = nullptr; Q.tile_tok = d_tt; Q.grp_tok = d_gt;
+        Q.ext_id = v->d_ext_id; Q.piece_cnt = d_cnt; Q.stage = d_stage; Q.pairbuf = nullptr; Q.tile_tok = d_tt; Q.grp_tok = d_gt; Q.q_short = d_qs; Q.q_warp = d_qw; Q.q_long = d_ql;
         const int grid = (int)(ntiles < (size_t)v->sm_count * 8 ? ntiles : (size_t)v->sm_count * 8);
-        k_pieces<<<grid, BPE_THREADS>>>(Q);
+        k_lookup<<<grid, LOOKUP_THREADS>>>(Q);
+        k_merge<<<v->sm_count * 7, MERGE_THREADS>>>(Q);
         ok = cudaGetLastError() == cudaSuccess && cudaDeviceSynchronize() == cudaSuccess;
     }
     ok = ok && cudaMemcpy(cnt.data(), d_cnt, cnt.size() * sizeof(u32), cudaMemcpyDeviceToHost) == cudaSuccess;
     ok = ok && cudaMemcpy(stage.data(), d_stage, nb * sizeof(int32_t), cudaMemcpyDeviceToHost) == cudaSuccess;
-    cudaFree(d_text); cudaFree(d_mask); cudaFree(d_gt); cudaFree(d_tf); cudaFree(d_tt); cudaFree(d_cnt); cudaFree(d_stage); cudaFree(d_hdr);
+    cudaFree(d_qs); cudaFree(d_qw); cudaFree(d_ql); cudaFree(d_text); cudaFree(d_mask); cudaFree(d_gt); cudaFree(d_tf); cudaFree(d_tt); cudaFree(d_cnt); cudaFree(d_stage); cudaFree(d_hdr);
     if (!ok) { cudaGetLastError(); return TT_ERR_CUDA; }
     for (size_t i = 0; i < np; i++) {
         const size_t tile = off[i] / TT_TILE_BYTES, slot = tile * TT_TILE_BYTES + (i - tile_base[tile]);   // pieces are indexed per tile
@@ -329,6 +331,9 @@ static size_t carve(TTWorkspace* w, void* base, size_t max_len, size_t max_docs)
     p = take(ntiles * TT_TILE_BYTES * sizeof(u32));          if (w) w->piece_cnt = (u32*)p;
     p = take((max_len + 1) * sizeof(int32_t));  if (w) w->stage = (int32_t*)p;
     p = take((max_len + 1) * sizeof(u64));      if (w) w->pairbuf = (u64*)p;
+    p = take((max_len / 2 + 64) * sizeof(u64)); if (w) w->q_short = (u64*)p;
+    p = take((max_len / 33 + 64) * sizeof(u64)); if (w) w->q_warp = (u64*)p;
+    p = take((max_len / 257 + 16) * sizeof(uint4)); if (w) w->q_long = (uint4*)p;
     p = take(padded + 16);                      if (w) w->cand = (u8*)p;
     p = take((padded / 32 + 4) * sizeof(u32));  if (w) w->litstart = (u32*)p;
     p = take((padded / 32 + 4) * sizeof(u32));  if (w) w->litin = (u32*)p;
@@ -440,13 +445,18 @@ static int encode_impl(const tt_vocab* v, const uint8_t* text, size_t len, const
     if (rc != TT_OK) return rc;
     MARK(1);
     const int tile_grid = PP.ntiles < v->sm_count * 8 ? PP.ntiles : v->sm_count * 8;
+    const int merge_grid = PP.ntiles * 4 + 1 < v->sm_count * 7 ? PP.ntiles * 4 + 1 : v->sm_count * 7;
     PieceParams Q;
     Q.base = PP.base; Q.shift = PP.lo; Q.hi = PP.hi; Q.nchunks = PP.nchunks; Q.ntiles = PP.ntiles;
     Q.startmask = w.startmask; Q.tile_first = w.tile_first; Q.hdr = w.hdr; Q.tab = v->tab; Q.toktab = v->toktab; Q.longtab = v->longtab; Q.litstart = literals ? w.litstart : nullptr;
     Q.ext_id = v->d_ext_id; Q.piece_cnt = w.piece_cnt; Q.stage = w.stage; Q.pairbuf = w.pairbuf; Q.tile_tok = w.tile_tok; Q.grp_tok = w.grp_tok;
-    if (ev) k_pieces<<<tile_grid, BPE_THREADS, 0, st>>>(Q);
-    else CK(launch_after(k_pieces, tile_grid, BPE_THREADS, st, Q));
+    Q.q_short = w.q_short; Q.q_warp = w.q_warp; Q.q_long = w.q_long;
+    if (ev) k_lookup<<<tile_grid, LOOKUP_THREADS, 0, st>>>(Q);
+    else CK(launch_after(k_lookup, tile_grid, LOOKUP_THREADS, st, Q));
     MARK(2);
+    if (ev) k_merge<<<merge_grid, MERGE_THREADS, 0, st>>>(Q);
+    else CK(launch_after(k_merge, merge_grid, MERGE_THREADS, st, Q));
+    MARK(3);
     ScatterParams S;
     S.shift = PP.lo; S.hi = PP.hi; S.nchunks = PP.nchunks; S.ntiles = PP.ntiles; S.startmask = w.startmask;
     S.tile_first = w.tile_first; S.tile_tok = w.tile_tok; S.grp_tok = w.grp_tok; S.ids_cap = (unsigned long long)ids_cap; S.piece_cnt = w.piece_cnt; S.stage = w.stage; S.hdr = w.hdr;
@@ -455,7 +465,7 @@ static int encode_impl(const tt_vocab* v, const uint8_t* text, size_t len, const
     S.ids_off_out = (long long*)ids_off_out;
     if (ev) k_scatter<<<tile_grid, BPE_THREADS, 0, st>>>(S);
     else CK(launch_after(k_scatter, tile_grid, BPE_THREADS, st, S));
-    MARK(3);
+    MARK(4);
 #undef MARK
     CK(cudaGetLastError());
     return TT_OK;
@@ -522,18 +532,18 @@ extern "C" int tt_encode_batch(const tt_vocab* v, const uint8_t* text, size_t to
 
 extern "C" int tt_encode_timed(const tt_vocab* v, const uint8_t* text, size_t len, void* stream, int32_t* ids_out,
                                size_t ids_cap, int64_t* count_out, int32_t* status_out, void* workspace,
-                               size_t workspace_bytes, float ms_out[3]) {
+                               size_t workspace_bytes, float ms_out[4]) {
     int rc = check_common(v, text, len, workspace, workspace_bytes, 1);
     if (rc != TT_OK) return rc;
     if (!count_out || !status_out || !ms_out || !len || !ids_out) return TT_ERR_ARG;
-    cudaEvent_t ev[4];
-    for (int i = 0; i < 4; i++) CK(cudaEventCreate(&ev[i]));
+    cudaEvent_t ev[5];
+    for (int i = 0; i < 5; i++) CK(cudaEventCreate(&ev[i]));
     rc = encode_impl(v, text, len, nullptr, 1, (cudaStream_t)stream, ids_out, ids_cap, count_out, nullptr, status_out,
                      workspace, ev);
-    if (rc == TT_OK && cudaEventSynchronize(ev[3]) != cudaSuccess) rc = TT_ERR_CUDA;
-    for (int i = 0; i < 3 && rc == TT_OK; i++)
+    if (rc == TT_OK && cudaEventSynchronize(ev[4]) != cudaSuccess) rc = TT_ERR_CUDA;
+    for (int i = 0; i < 4 && rc == TT_OK; i++)
         if (cudaEventElapsedTime(&ms_out[i], ev[i], ev[i + 1]) != cudaSuccess) rc = TT_ERR_CUDA;
-    for (int i = 0; i < 4; i++) cudaEventDestroy(ev[i]);
+    for (int i = 0; i < 5; i++) cudaEventDestroy(ev[i]);
     return rc;
 }
 

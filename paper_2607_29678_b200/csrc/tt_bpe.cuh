@@ -4,13 +4,13 @@
 // GPU hash tables; a round's minimum rank identifies one pair value, merging all its leftmost
 // non-overlapping occurrences equals iterated single merges, and only pairs next to a completed
 // merge need to be probed again.  Work is dispatched by piece length and difficulty:
-//   * a thread per piece looks the whole piece up as a vocabulary entry (one 32-byte probe);
-//   * pieces that are not a single entry are merged by a warp (<= 32 bytes: tokens in registers,
-//     candidates as ballot masks; <= 256 bytes: several tokens per lane, compaction through shared memory);
-//     where a CTA has many such pieces of <= 32 bytes waiting (text dense in pieces outside the vocabulary,
-//     or many tiles per CTA), it merges 128 of them at once, one thread per piece (lane_merge);
-//   * longer pieces are merged by the whole CTA (cta_merge_long: state in shared memory, or in global
-//     scratch while the piece still has more than 4,096 tokens).
+//   * k_lookup: a thread per piece looks the whole piece up as a vocabulary entry (one 32-byte probe); pieces
+//     that are not a single entry are appended to global queues by length class;
+//   * k_merge: every warp of the GPU draws from those queues -- a warp per piece (<= 32 bytes: tokens in
+//     registers, candidates as ballot masks; <= 256 bytes: several tokens per lane, compaction through shared
+//     memory), or, where the call has many pieces of <= 32 bytes, 32 of them at once, a thread per piece
+//     (lane_merge); longer pieces are merged by a whole CTA (cta_merge_long: state in shared memory, or in
+//     global scratch while the piece still has more than 4,096 tokens).
 // Token ids inside the kernels are "internal": byte b -> b, result of the merge of rank r -> 256 + r;
 // the caller's ids are looked up when the tokens are staged.
 #pragma once
@@ -277,11 +277,10 @@ __device__ __forceinline__ u32 warp_merge_perm(u64* buf /* 2 * 32 * E entries of
 // unmatched pieces; a thread per piece keeps 32 independent chains per warp in flight and issues an order
 // of magnitude fewer instructions per piece, so it serves bulk text.  Same rounds as everywhere: the
 // minimum rank of the piece, all its leftmost non-overlapping occurrences, new probes only next to a merge.
-// Column s of tok[LANE_MAX][LANE_SLOTS] / rk[LANE_MAX][LANE_SLOTS]: any two threads of a warp hit
-// different banks whatever rows they are at.
-constexpr int LANE_SLOTS = 128;                       // pieces merged at once
+// Column s of tok[LANE_MAX][LANE_SLOTS] / rk[LANE_MAX][LANE_SLOTS] (one pair of arrays per warp): any two
+// threads of the warp hit different banks whatever rows they are at.
+constexpr int LANE_SLOTS = 32;                        // pieces a warp merges at once
 constexpr int LANE_MAX = 32;                          // bytes per piece on this path
-constexpr u32 LANE_MIN_PIECES = 33;                   // fewer pieces left after a CTA's last tile get a warp each instead
 // Two independent probes with both first-bucket loads in flight together.
 __device__ __forceinline__ u32 pair_match_first(const PairTable& t, const uint4 lo, const uint4 hi, u64 key) {
     const u64 s0 = ((u64)lo.y << 32) | lo.x, s1 = ((u64)lo.w << 32) | lo.z, s2 = ((u64)hi.y << 32) | hi.x, s3 = ((u64)hi.w << 32) | hi.z;
@@ -377,16 +376,15 @@ __device__ __forceinline__ u32 cta_excl_sum_scan(u32 v, u32* scratch /* >= 33 */
     *total = scratch[32];
     return scratch[wid] + x - v;
 }
-// Sum over the CTA, returned to every thread (scratch >= 33 entries; two barriers).
-__device__ __forceinline__ unsigned long long cta_sum_u64(unsigned long long v, unsigned long long* scratch) {
+// Sums of two values over the CTA, returned to every thread (scratch >= 66 entries; two barriers).
+__device__ __forceinline__ void cta_sum2_u64(unsigned long long& x, unsigned long long& y, unsigned long long* scratch) {
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5, nw = (blockDim.x + 31) >> 5;
-    for (int o = 16; o; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+    for (int o = 16; o; o >>= 1) { x += __shfl_xor_sync(0xFFFFFFFFu, x, o); y += __shfl_xor_sync(0xFFFFFFFFu, y, o); }
     __syncthreads();
-    if (lane == 0) scratch[wid] = v;
+    if (lane == 0) { scratch[2 * wid] = x; scratch[2 * wid + 1] = y; }
     __syncthreads();
-    unsigned long long t = 0;
-    for (int w = 0; w < nw; w++) t += scratch[w];
-    return t;
+    x = 0; y = 0;
+    for (int w = 0; w < nw; w++) { x += scratch[2 * w]; y += scratch[2 * w + 1]; }
 }
 
 __device__ __forceinline__ u32 cta_min_u32(u32 v, u32* scratch /* >= 33 */) {
@@ -557,15 +555,14 @@ __device__ void tile_pieces(TilePieces& tp, const u16* __restrict__ startmask, c
     __syncthreads();
 }
 
-// ---- K4 (+ the scan of K5): all pieces of a text tile -----------------------------------------------------------
-// Phase 1: a thread per piece (one-byte pieces map directly, pieces of up to 24 bytes are looked up as
-// whole vocabulary entries).  Phase 2: the CTA's warps merge the pieces of 33..256 bytes phase 1 could not
-// settle; longer ones are merged by the whole CTA.  Unsettled pieces of <= 32 bytes go to a queue that
-// outlives the tile: it is emptied when it holds LANE_SLOTS pieces (a thread per piece) and after the CTA's
-// last tile (a warp per piece if few are left).  Phase 3: token totals per tile and per group of tiles
-// (both zero on entry; queued pieces add to theirs when they are merged).  No CTA waits for another and
-// nothing is scanned here: k_scatter derives each tile's output offset from the two levels of totals.
-// Without a token table (while the table itself is being built) every piece takes the merge path.
+// ---- K4, first half: whole-piece lookups of a text tile; unsettled pieces go to global queues -----------------
+// A thread per piece: one-byte pieces map directly, pieces of up to 24 bytes are looked up as whole
+// vocabulary entries (two pieces per thread and step, their loads side by side).  What stays unsettled is
+// appended to one of three queues in the workspace (one atomic reservation per tile and queue):
+//   q_short  pieces of <= 32 bytes,  q_warp  pieces of 33..256 bytes,  q_long  longer pieces.
+// Token totals of the settled pieces go to the per-tile and per-group counters.  This kernel holds no merge
+// code, so it runs at full occupancy; k_merge then has every warp of the GPU drawing from the same queues.
+// Without a token table (while the table itself is being built) every piece is queued.
 struct PieceParams {
     const u8* base;            // aligned frame origin (text = base + shift)
     long long shift, hi;       // text occupies [shift, hi)
@@ -585,83 +582,42 @@ struct PieceParams {
     u64* pairbuf;              // global scratch of the long-piece path, indexed like the text
     u32* tile_tok;             // in: zero; out: tokens per tile
     u32* grp_tok;              // in: zero; out: tokens per group of TT_GROUP_TILES tiles
+    u64* q_short; u64* q_warp; // queue entries: text offset | index in tile << 32 | (bytes - 1) << 43
+    uint4* q_long;             // (text offset, bytes, piece index, 0)
 };
 
-constexpr int MID_SLOTS = 64;                         // queue of 33..256-byte pieces
-// The CTA's warps take the nm queued pieces of 33..256 bytes and then nt queued pieces of <= 32 bytes, one
-// piece at a time each (*next must be zero and the queues visible on entry).
-__device__ __forceinline__ void warp_flush(const PieceParams& P, u64* s_buf, const u32* m_a, const u32* m_p, const u32* m_tn, u32 nm,
-                                           const u32* q_a, const u32* q_p, const u32* q_tn, u32 nt, u32* next, const u8* text) {
-    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
-    u64* wbuf = s_buf + wid * (2 * TT_WARP_PIECE_MAX);
-    for (;;) {
-        u32 e = 0;
-        if (lane == 0) e = atomicAdd(next, 1u);
-        e = __shfl_sync(0xFFFFFFFFu, e, 0);
-        if (e >= nm + nt) break;
-        u32 m, pidx, tile;
-        if (e < nm) {
-            const u32 a = m_a[e], n = (m_tn[e] & 255) + 1;
-            m = n <= 64 ? warp_merge_perm<2>(wbuf, text, a, n, P.tab, P.ext_id, P.stage, lane)
-                        : warp_merge_perm<WCH>(wbuf, text, a, n, P.tab, P.ext_id, P.stage, lane);
-            pidx = m_p[e]; tile = m_tn[e] >> 8;
-        } else {
-            const u32 q = e - nm;
-            m = warp_merge_reg(text, q_a[q], (q_tn[q] & 31) + 1, P.tab, P.ext_id, P.stage, lane);
-            pidx = q_p[q]; tile = q_tn[q] >> 5;
-        }
-        if (lane == 0) { P.piece_cnt[pidx] = 0u - m; atomicAdd(&P.tile_tok[tile], m); atomicAdd(&P.grp_tok[tile >> TT_GROUP_SHIFT], m); }
-    }
-}
+__device__ __forceinline__ u64 queue_entry(u32 a, u32 i, u32 n) { return (u64)a | ((u64)i << 32) | ((u64)(n - 1) << 43); }
 
-// Merges the queued pieces a thread per piece (all threads of the CTA call it; the queue must be visible).
-__device__ __forceinline__ void lane_flush(const PieceParams& P, u64* s_buf, const u32* q_a, const u32* q_p, const u32* q_tn, u32 qn, const u8* text) {
-    const int tid = threadIdx.x;
-    if ((u32)tid < qn) {
-        u32* tok = reinterpret_cast<u32*>(s_buf);
-        const u32 m = lane_merge(tok, tok + LANE_SLOTS * LANE_MAX, tid, text, q_a[tid], (q_tn[tid] & 31) + 1, P.tab, P.ext_id, P.stage);
-        P.piece_cnt[q_p[tid]] = 0u - m;
-        atomicAdd(&P.tile_tok[q_tn[tid] >> 5], m);
-        atomicAdd(&P.grp_tok[q_tn[tid] >> (5 + TT_GROUP_SHIFT)], m);
-    }
-}
-
-__global__ void __launch_bounds__(BPE_THREADS, 4)
-k_pieces(const PieceParams P) {
+constexpr int LOOKUP_THREADS = 256;
+__global__ void __launch_bounds__(LOOKUP_THREADS, 6)
+k_lookup(const PieceParams P) {
     __shared__ TilePieces tp;
-    __shared__ u64 s_buf[LONG_SMEM_TOKENS];                   // warp merge buffers (8 x 2 x 256), one long piece, or the lane path's columns
-    __shared__ u16 s_miss[TILE_MAX_PIECES];
-    __shared__ u16 s_mid[TT_TILE_BYTES / (LANE_MAX + 1) + 2];
-    __shared__ u32 q_a[LANE_SLOTS], q_p[LANE_SLOTS], q_tn[LANE_SLOTS];     // queue: text offset, piece index, tile << 5 | (bytes - 1)
-    __shared__ u32 m_a[MID_SLOTS], m_p[MID_SLOTS], m_tn[MID_SLOTS];        // queue of the 33..256-byte pieces: ..., tile << 8 | (bytes - 1)
-    __shared__ u32 s_nmiss, s_nmid, s_nlong, s_total, s_next;
+    __shared__ u16 s_short[TILE_MAX_PIECES];                  // short misses from the front, long pieces from the back
+    __shared__ u16 s_warp[TT_TILE_BYTES / (LANE_MAX + 1) + 2];
+    __shared__ u32 s_ns, s_nw, s_nl, s_total, s_bs, s_bw, s_bl;
     __shared__ u32 sc[48];
-    static_assert(LONG_SMEM_TOKENS >= BPE_WARPS * 2 * TT_WARP_PIECE_MAX, "buffer size");
-    static_assert(LONG_SMEM_TOKENS * sizeof(u64) >= 2 * LANE_SLOTS * LANE_MAX * sizeof(u32), "buffer size");
-    static_assert(LANE_SLOTS <= BPE_THREADS && LANE_MAX == 32, "queue layout");
-    const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
-    cudaTriggerProgrammaticLaunchCompletion();               // k_scatter may be placed; it waits for this grid's memory itself
+    const int tid = threadIdx.x;
+    cudaTriggerProgrammaticLaunchCompletion();               // the next kernel may be placed; it waits for this grid's memory itself
     cudaGridDependencySynchronize();                         // k_pretok's flags and counts are complete from here on
-    const bool dead = P.hdr->status != 0;
+    if (P.hdr->status != 0) return;
     const u8* text = P.base + P.shift;
-    u32 qn = 0, mq = 0;                                        // block-uniform queue lengths
-    for (int tile = blockIdx.x; tile < (dead ? 0 : P.ntiles); tile += gridDim.x) {
+    for (int tile = blockIdx.x; tile < P.ntiles; tile += gridDim.x) {
         const long long c0 = (long long)tile * TT_TILE_CHUNKS;
         __syncthreads();
-        if (tid == 0) { s_nmiss = 0; s_nmid = 0; s_nlong = 0; s_total = 0; }
+        if (tid == 0) { s_ns = 0; s_nw = 0; s_nl = 0; s_total = 0; }
         tile_pieces(tp, P.startmask, P.tile_first, P.nchunks, P.ntiles, tile, P.hi, sc);
         const u32 np = tp.n, p0 = (u32)tile * TT_TILE_BYTES;     // pieces are indexed per tile
         const long long t0 = c0 * TT_CHUNK - P.shift;             // text offset of the tile start
         u32 wsum = 0;
         // two pieces per thread and step, their loads issued side by side: first the bytes of both, then the
         // table slots of both (each lookup is a chain of two dependent loads)
-        for (u32 ib = tid; ib < np; ib += 2 * BPE_THREADS) {
+        for (u32 ib = tid; ib < np; ib += 2 * LOOKUP_THREADS) {
             u32 a[2], n[2], h[2], kind[2];                        // kind: 0 none, 1 literal, 2 one byte, 3 table lookup, 4 other
             u64 k0[2], k1[2], k2[2];
             uint4 lo[2], hi[2];
 #pragma unroll
             for (int j = 0; j < 2; j++) {
-                const u32 i = ib + j * BPE_THREADS;
+                const u32 i = ib + j * LOOKUP_THREADS;
                 kind[j] = 0; a[j] = 0; n[j] = 0; k0[j] = 0; k1[j] = 0; k2[j] = 0;
                 if (i < np) {
                     a[j] = (u32)(t0 + tp.off[i]);
@@ -684,7 +640,7 @@ k_pieces(const PieceParams P) {
             }
 #pragma unroll
             for (int j = 0; j < 2; j++) {
-                const u32 i = ib + j * BPE_THREADS;
+                const u32 i = ib + j * LOOKUP_THREADS;
                 int32_t id;
                 if (kind[j] == 0) continue;
                 if (kind[j] == 1) { P.piece_cnt[p0 + i] = 0u - 1u; wsum++; }     // one staged id (written by the literal pass)
@@ -693,62 +649,112 @@ k_pieces(const PieceParams P) {
                     P.piece_cnt[p0 + i] = (u32)id; wsum++;
                 } else if (n[j] > TT_TOKTAB_MAXLEN && P.longtab.slots != nullptr && n[j] <= P.longtab.maxlen && longtab_lookup(P.longtab, text, a[j], n[j], id)) {
                     P.piece_cnt[p0 + i] = (u32)id; wsum++;
-                } else if (n[j] > TT_WARP_PIECE_MAX) { s_miss[TILE_MAX_PIECES - 1 - atomicAdd(&s_nlong, 1u)] = (u16)i; }   // long pieces from the back
-                else if (n[j] > LANE_MAX) s_mid[atomicAdd(&s_nmid, 1u)] = (u16)i;
-                else s_miss[atomicAdd(&s_nmiss, 1u)] = (u16)i;
+                } else if (n[j] > TT_WARP_PIECE_MAX) s_short[TILE_MAX_PIECES - 1 - atomicAdd(&s_nl, 1u)] = (u16)i;
+                else if (n[j] > LANE_MAX) s_warp[atomicAdd(&s_nw, 1u)] = (u16)i;
+                else s_short[atomicAdd(&s_ns, 1u)] = (u16)i;
             }
         }
         for (int o = 16; o; o >>= 1) wsum += __shfl_xor_sync(0xFFFFFFFFu, wsum, o);
+        if ((tid & 31) == 0 && wsum) atomicAdd(&s_total, wsum);
         __syncthreads();
-        const u32 nreg = s_nmiss, nmid = s_nmid, nlong = s_nlong;
-        // Unsettled pieces of <= 256 bytes go into two queues that outlive the tile, so that in bulk text all
-        // warps have work at once: a full queue of pieces of <= 32 bytes is merged a thread per piece, a full
-        // queue of longer ones a warp per piece.
-        const bool last_tile = tile + (int)gridDim.x >= P.ntiles;
-        for (u32 done = 0; done < nreg;) {
-            const u32 take = min(nreg - done, (u32)LANE_SLOTS - qn);
-            if ((u32)tid < take) {
-                const u32 i = s_miss[done + tid];
+        const u32 ns = s_ns, nw = s_nw, nl = s_nl;
+        if (tid == 0) {
+            if (s_total) { atomicAdd(&P.tile_tok[tile], s_total); atomicAdd(&P.grp_tok[tile >> TT_GROUP_SHIFT], s_total); }
+            if (ns) s_bs = atomicAdd(&P.hdr->nq_short, ns);
+            if (nw) s_bw = atomicAdd(&P.hdr->nq_warp, nw);
+            if (nl) s_bl = atomicAdd(&P.hdr->nq_long, nl);
+        }
+        if (ns | nw | nl) {                                       // block-uniform
+            __syncthreads();
+            for (u32 e = tid; e < ns + nw + nl; e += LOOKUP_THREADS) {
+                const u32 i = e < ns ? s_short[e] : e < ns + nw ? s_warp[e - ns] : s_short[TILE_MAX_PIECES - 1 - (e - ns - nw)];
+                const u32 a = (u32)(t0 + tp.off[i]);
                 const u32 n = (i + 1 < np ? tp.off[i + 1] : tp.end) - tp.off[i];
-                q_a[qn + tid] = (u32)(t0 + tp.off[i]); q_p[qn + tid] = p0 + i; q_tn[qn + tid] = ((u32)tile << 5) | (n - 1);
+                if (e < ns) P.q_short[s_bs + e] = queue_entry(a, i, n);
+                else if (e < ns + nw) P.q_warp[s_bw + (e - ns)] = queue_entry(a, i, n);
+                else P.q_long[s_bl + (e - ns - nw)] = make_uint4(a, n, p0 + i, 0u);
             }
-            qn += take; done += take;
-            __syncthreads();
-            if (qn == (u32)LANE_SLOTS) { lane_flush(P, s_buf, q_a, q_p, q_tn, qn, text); qn = 0; __syncthreads(); }
         }
-        for (u32 done = 0; done < nmid;) {
-            const u32 take = min(nmid - done, (u32)MID_SLOTS - mq);
-            if ((u32)tid < take) {
-                const u32 i = s_mid[done + tid];
-                const u32 n = (i + 1 < np ? tp.off[i + 1] : tp.end) - tp.off[i];
-                m_a[mq + tid] = (u32)(t0 + tp.off[i]); m_p[mq + tid] = p0 + i; m_tn[mq + tid] = ((u32)tile << 8) | (n - 1);
+    }
+}
+
+// ---- K4, second half: the merges ------------------------------------------------------------------------------
+// Long pieces (> 256 bytes) first, a CTA each.  Then every warp works on its own: it takes the pieces of
+// 33..256 bytes one at a time (the longest chains, so they start first), then the pieces of <= 32 bytes --
+// one at a time with the tokens in registers if the whole call has few of them (the shortest chain per piece:
+// a request's latency is its longest chain), else 32 at a time, a thread per piece.  Tickets are global, so
+// all warps of the GPU stay busy until the queues are empty; no barrier after the long pieces.
+constexpr int MERGE_WARPS = 4;
+constexpr int MERGE_THREADS = MERGE_WARPS * 32;
+constexpr int WARP_SMEM_WORDS = 1024;                 // u64 per warp: two lane-path arrays of 32 x 32 u32, or the 2 x 256 merge buffers
+static_assert(MERGE_WARPS * WARP_SMEM_WORDS >= LONG_SMEM_TOKENS, "the CTA's buffer must hold a long piece");
+static_assert(WARP_SMEM_WORDS * sizeof(u64) >= 2 * LANE_SLOTS * LANE_MAX * sizeof(u32) && WARP_SMEM_WORDS >= 2 * TT_WARP_PIECE_MAX, "per-warp buffer");
+
+__global__ void __launch_bounds__(MERGE_THREADS, 7)
+k_merge(const PieceParams P) {
+    __shared__ u64 s_buf[MERGE_WARPS * WARP_SMEM_WORDS];
+    __shared__ u32 sc[48];
+    const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+    cudaTriggerProgrammaticLaunchCompletion();               // k_scatter may be placed; it waits for this grid's memory itself
+    cudaGridDependencySynchronize();                         // the queues are complete from here on
+    if (P.hdr->status != 0) return;
+    const u8* text = P.base + P.shift;
+    const u32 ns = P.hdr->nq_short, nw = P.hdr->nq_warp, nl = P.hdr->nq_long;
+    for (u32 e = blockIdx.x; e < nl; e += gridDim.x) {            // block-uniform
+        const uint4 q = P.q_long[e];
+        const u32 m = cta_merge_long(text, q.x, q.y, P.tab, P.ext_id, P.stage, P.pairbuf + q.x, s_buf, sc);
+        if (tid == 0) {
+            const u32 tile = q.z / TT_TILE_BYTES;
+            P.piece_cnt[q.z] = 0u - m; atomicAdd(&P.tile_tok[tile], m); atomicAdd(&P.grp_tok[tile >> TT_GROUP_SHIFT], m);
+        }
+    }
+    if (nl > blockIdx.x) __syncthreads();
+    u64* wbuf = s_buf + wid * WARP_SMEM_WORDS;
+    const u32 FULL = 0xFFFFFFFFu;
+    for (;;) {                                                    // bounded by the queue length
+        u32 e = 0;
+        if (lane == 0) e = atomicAdd(&P.hdr->t_warp, 1u);
+        e = __shfl_sync(FULL, e, 0);
+        if (e >= nw) break;
+        const u64 q = P.q_warp[e];
+        const u32 a = (u32)q, i = (u32)(q >> 32) & 2047u, n = (u32)(q >> 43) + 1;
+        const u32 m = n <= 64 ? warp_merge_perm<2>(wbuf, text, a, n, P.tab, P.ext_id, P.stage, lane)
+                              : warp_merge_perm<WCH>(wbuf, text, a, n, P.tab, P.ext_id, P.stage, lane);
+        if (lane == 0) {
+            const u32 tile = (u32)(((long long)a + P.shift) / TT_TILE_BYTES);
+            P.piece_cnt[tile * TT_TILE_BYTES + i] = 0u - m; atomicAdd(&P.tile_tok[tile], m); atomicAdd(&P.grp_tok[tile >> TT_GROUP_SHIFT], m);
+        }
+    }
+    if (ns <= 2u * MERGE_WARPS * gridDim.x) {                     // few: a warp per piece
+        for (;;) {
+            u32 e = 0;
+            if (lane == 0) e = atomicAdd(&P.hdr->t_short, 1u);
+            e = __shfl_sync(FULL, e, 0);
+            if (e >= ns) break;
+            const u64 q = P.q_short[e];
+            const u32 a = (u32)q, i = (u32)(q >> 32) & 2047u, n = (u32)(q >> 43) + 1;
+            const u32 m = warp_merge_reg(text, a, n, P.tab, P.ext_id, P.stage, lane);
+            if (lane == 0) {
+                const u32 tile = (u32)(((long long)a + P.shift) / TT_TILE_BYTES);
+                P.piece_cnt[tile * TT_TILE_BYTES + i] = 0u - m; atomicAdd(&P.tile_tok[tile], m); atomicAdd(&P.grp_tok[tile >> TT_GROUP_SHIFT], m);
             }
-            mq += take; done += take;
-            if (tid == 0) s_next = 0;
-            __syncthreads();
-            if (mq == (u32)MID_SLOTS) { warp_flush(P, s_buf, m_a, m_p, m_tn, mq, q_a, q_p, q_tn, 0, &s_next, text); mq = 0; __syncthreads(); }
         }
-        // after the CTA's last tile the warps take what is left, including a short rest of the other queue (the
-        // longest chain of a request sets its latency, so its few unsettled pieces get a warp each)
-        if (last_tile) {
-            const u32 ntail = qn < LANE_MIN_PIECES ? qn : 0;
-            if (tid == 0) s_next = 0;
-            __syncthreads();
-            warp_flush(P, s_buf, m_a, m_p, m_tn, mq, q_a, q_p, q_tn, ntail, &s_next, text);
-            mq = 0;
-            if (ntail) qn = 0;
+    } else {                                                      // bulk: 32 pieces per warp and step, a thread each
+        u32* tok = reinterpret_cast<u32*>(wbuf);
+        for (;;) {
+            u32 e0 = 0;
+            if (lane == 0) e0 = atomicAdd(&P.hdr->t_short, (u32)LANE_SLOTS);
+            e0 = __shfl_sync(FULL, e0, 0);
+            if (e0 >= ns) break;
+            if (e0 + lane < ns) {
+                const u64 q = P.q_short[e0 + lane];
+                const u32 a = (u32)q, i = (u32)(q >> 32) & 2047u, n = (u32)(q >> 43) + 1;
+                const u32 m = lane_merge(tok, tok + LANE_SLOTS * LANE_MAX, lane, text, a, n, P.tab, P.ext_id, P.stage);
+                const u32 tile = (u32)(((long long)a + P.shift) / TT_TILE_BYTES);
+                P.piece_cnt[tile * TT_TILE_BYTES + i] = 0u - m; atomicAdd(&P.tile_tok[tile], m); atomicAdd(&P.grp_tok[tile >> TT_GROUP_SHIFT], m);
+            }
+            __syncwarp();
         }
-        if (lane == 0) atomicAdd(&s_total, wsum);
-        for (u32 e = 0; e < nlong; e++) {                         // block-uniform
-            const u32 i = s_miss[TILE_MAX_PIECES - 1 - e];
-            const u32 a = (u32)(t0 + tp.off[i]);
-            const u32 n = (i + 1 < np ? tp.off[i + 1] : tp.end) - tp.off[i];
-            const u32 m = cta_merge_long(text, a, n, P.tab, P.ext_id, P.stage, P.pairbuf + a, s_buf, sc);
-            if (tid == 0) { P.piece_cnt[p0 + i] = 0u - m; atomicAdd(&s_total, m); }
-        }
-        __syncthreads();
-        if (tid == 0) { atomicAdd(&P.tile_tok[tile], s_total); atomicAdd(&P.grp_tok[tile >> TT_GROUP_SHIFT], s_total); }
-        if (last_tile && qn) { lane_flush(P, s_buf, q_a, q_p, q_tn, qn, text); qn = 0; }
     }
 }
 
@@ -780,7 +786,7 @@ k_scatter(const ScatterParams P) {
     __shared__ u32 sc[48];
     __shared__ u32 s_big[TILE_MAX_PIECES / 8][3];
     __shared__ u32 s_nbig;
-    __shared__ unsigned long long s_sum[33];
+    __shared__ unsigned long long s_sum[66];
     const int tid = threadIdx.x;
     cudaGridDependencySynchronize();                         // k_pieces' counts and staged ids are complete from here on
     // Each CTA takes a contiguous range of tiles.  Tokens before its first tile = the whole groups of tiles
@@ -796,8 +802,7 @@ k_scatter(const ScatterParams P) {
         if (g < g_lo) before += x;
     }
     for (int t = (g_lo << TT_GROUP_SHIFT) + tid; t < tile_lo; t += BPE_THREADS) before += P.tile_tok[t];
-    before = cta_sum_u64(before, s_sum);
-    total = cta_sum_u64(total, s_sum);
+    cta_sum2_u64(before, total, s_sum);
     int status = P.hdr->status;
     if (status == 0 && total > P.ids_cap) status = 5;          // TT_ERR_CAPACITY
     if (blockIdx.x == 0 && tid == 0) {

@@ -41,7 +41,9 @@ struct TTHeader {
     int status;              // TT_OK or a device-side error code
     u32 pretok_done;         // CTAs that finished the pre-tokenization pass (tt_pretokenize only)
     u32 n_pieces;            // number of pieces found (tt_pretokenize only)
-    u32 pad[29];
+    u32 nq_short, nq_warp, nq_long;   // lengths of the queues of unsettled pieces (k_lookup)
+    u32 t_short, t_warp;     // tickets of k_merge: entries handed out so far
+    u32 pad[24];
 };
 static_assert(sizeof(TTHeader) == 128, "header layout");
 
@@ -57,6 +59,9 @@ struct TTWorkspace {
                        // or minus the staged token count
     int32_t* stage;    // token ids staged at the byte offset of their piece (len)
     u64* pairbuf;      // (token, rank) pairs of the long-piece path, indexed like the text (len)
+    u64* q_short;      // unsettled pieces of <= 32 bytes (len / 2 + 64 entries)
+    u64* q_warp;       // unsettled pieces of 33..256 bytes (len / 33 + 64 entries)
+    uint4* q_long;     // unsettled longer pieces (len / 257 + 16 entries)
     u8* cand;          // literal pass: length of the longest added-token literal starting at each byte (aligned frame)
     u32* litstart;     // literal pass: bit per byte, first byte of an extracted literal
     u32* litin;        // literal pass: bit per byte, the other bytes of an extracted literal

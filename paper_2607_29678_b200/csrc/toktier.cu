@@ -179,7 +179,7 @@ static int build_token_table(tt_vocab* v, const tt_merge* merges, size_t n_merge
         Q.ext_id = v->d_ext_id; Q.piece_cnt = d_cnt; Q.stage = d_stage; Q.pairbuf = nullptr; Q.tile_tok = d_tt; Q.grp_tok = d_gt; Q.q_short = d_qs; Q.q_warp = d_qw; Q.q_long = d_ql;
         const int grid = (int)(ntiles < (size_t)v->sm_count * 8 ? ntiles : (size_t)v->sm_count * 8);
         k_lookup<<<grid, LOOKUP_THREADS>>>(Q);
-        k_merge<<<v->sm_count * 7, MERGE_THREADS>>>(Q);
+        k_merge<<<v->sm_count * 3, MERGE_THREADS, MERGE_SMEM_BYTES>>>(Q);
         ok = cudaGetLastError() == cudaSuccess && cudaDeviceSynchronize() == cudaSuccess;
     }
     ok = ok && cudaMemcpy(cnt.data(), d_cnt, cnt.size() * sizeof(u32), cudaMemcpyDeviceToHost) == cudaSuccess;
@@ -287,6 +287,7 @@ extern "C" int tt_vocab_load_ex(const tt_merge* merges, size_t n_merges, const i
     ok = ok && cudaMemcpy(v->d_cls, cls.data(), v->cls_bytes, cudaMemcpyHostToDevice) == cudaSuccess;
     if (!ok) { cudaGetLastError(); tt_vocab_free(v); return TT_ERR_CUDA; }
     v->tab.slots = v->d_slots; v->tab.bytepair = v->d_bytepair; v->tab.mask = mask; v->tab.shift = shift;
+    if (cudaFuncSetAttribute(k_merge, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)MERGE_SMEM_BYTES) != cudaSuccess) { cudaGetLastError(); tt_vocab_free(v); return TT_ERR_CUDA; }
     { const int rc = build_token_table(v, merges, n_merges, ext_id); if (rc != TT_OK) { tt_vocab_free(v); return rc; } }
     {   // byte length and number of non-continuation bytes of every token, indexed by the caller's id
         std::vector<uint2> in(256 + n_merges);
@@ -416,9 +417,9 @@ static int check_common(const tt_vocab* v, const void* text, size_t len, void* w
 // signalled, and wait inside the kernel (cudaGridDependencySynchronize) until the predecessor's memory
 // is complete.  Only the launch latency is hidden; the data dependence is unchanged.
 template <typename Params>
-static cudaError_t launch_after(void (*kernel)(const Params), int grid, int block, cudaStream_t st, const Params& p) {
+static cudaError_t launch_after(void (*kernel)(const Params), int grid, int block, cudaStream_t st, const Params& p, size_t smem = 0) {
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)grid); cfg.blockDim = dim3((unsigned)block); cfg.dynamicSmemBytes = 0; cfg.stream = st;
+    cfg.gridDim = dim3((unsigned)grid); cfg.blockDim = dim3((unsigned)block); cfg.dynamicSmemBytes = smem; cfg.stream = st;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
@@ -445,7 +446,7 @@ static int encode_impl(const tt_vocab* v, const uint8_t* text, size_t len, const
     if (rc != TT_OK) return rc;
     MARK(1);
     const int tile_grid = PP.ntiles < v->sm_count * 8 ? PP.ntiles : v->sm_count * 8;
-    const int merge_grid = PP.ntiles * 4 + 1 < v->sm_count * 7 ? PP.ntiles * 4 + 1 : v->sm_count * 7;
+    const int merge_grid = PP.ntiles * 2 + 1 < v->sm_count * 3 ? PP.ntiles * 2 + 1 : v->sm_count * 3;
     PieceParams Q;
     Q.base = PP.base; Q.shift = PP.lo; Q.hi = PP.hi; Q.nchunks = PP.nchunks; Q.ntiles = PP.ntiles;
     Q.startmask = w.startmask; Q.tile_first = w.tile_first; Q.hdr = w.hdr; Q.tab = v->tab; Q.toktab = v->toktab; Q.longtab = v->longtab; Q.litstart = literals ? w.litstart : nullptr;
@@ -454,8 +455,8 @@ static int encode_impl(const tt_vocab* v, const uint8_t* text, size_t len, const
     if (ev) k_lookup<<<tile_grid, LOOKUP_THREADS, 0, st>>>(Q);
     else CK(launch_after(k_lookup, tile_grid, LOOKUP_THREADS, st, Q));
     MARK(2);
-    if (ev) k_merge<<<merge_grid, MERGE_THREADS, 0, st>>>(Q);
-    else CK(launch_after(k_merge, merge_grid, MERGE_THREADS, st, Q));
+    if (ev) k_merge<<<merge_grid, MERGE_THREADS, MERGE_SMEM_BYTES, st>>>(Q);
+    else CK(launch_after(k_merge, merge_grid, MERGE_THREADS, st, Q, MERGE_SMEM_BYTES));
     MARK(3);
     ScatterParams S;
     S.shift = PP.lo; S.hi = PP.hi; S.nchunks = PP.nchunks; S.ntiles = PP.ntiles; S.startmask = w.startmask;

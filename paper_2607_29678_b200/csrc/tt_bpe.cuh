@@ -684,15 +684,16 @@ k_lookup(const PieceParams P) {
 // one at a time with the tokens in registers if the whole call has few of them (the shortest chain per piece:
 // a request's latency is its longest chain), else 32 at a time, a thread per piece.  Tickets are global, so
 // all warps of the GPU stay busy until the queues are empty; no barrier after the long pieces.
-constexpr int MERGE_WARPS = 4;
+constexpr int MERGE_WARPS = 8;
 constexpr int MERGE_THREADS = MERGE_WARPS * 32;
 constexpr int WARP_SMEM_WORDS = 1024;                 // u64 per warp: two lane-path arrays of 32 x 32 u32, or the 2 x 256 merge buffers
 static_assert(MERGE_WARPS * WARP_SMEM_WORDS >= LONG_SMEM_TOKENS, "the CTA's buffer must hold a long piece");
+constexpr size_t MERGE_SMEM_BYTES = (size_t)MERGE_WARPS * WARP_SMEM_WORDS * sizeof(u64);   // dynamic shared memory of k_merge (64 KiB)
 static_assert(WARP_SMEM_WORDS * sizeof(u64) >= 2 * LANE_SLOTS * LANE_MAX * sizeof(u32) && WARP_SMEM_WORDS >= 2 * TT_WARP_PIECE_MAX, "per-warp buffer");
 
-__global__ void __launch_bounds__(MERGE_THREADS, 7)
+__global__ void __launch_bounds__(MERGE_THREADS, 3)
 k_merge(const PieceParams P) {
-    __shared__ u64 s_buf[MERGE_WARPS * WARP_SMEM_WORDS];
+    extern __shared__ __align__(16) u64 s_buf[];              // MERGE_SMEM_BYTES
     __shared__ u32 sc[48];
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
     cudaTriggerProgrammaticLaunchCompletion();               // k_scatter may be placed; it waits for this grid's memory itself

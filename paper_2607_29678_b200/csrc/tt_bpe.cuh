@@ -599,13 +599,14 @@ k_lookup(const PieceParams P) {
     const int tid = threadIdx.x;
     cudaTriggerProgrammaticLaunchCompletion();               // the next kernel may be placed; it waits for this grid's memory itself
     cudaGridDependencySynchronize();                         // k_pretok's flags and counts are complete from here on
-    if (P.hdr->status != 0) return;
+    const int status = P.hdr->status;                        // looked at after the first tile's flags are in: the loads overlap
     const u8* text = P.base + P.shift;
     for (int tile = blockIdx.x; tile < P.ntiles; tile += gridDim.x) {
         const long long c0 = (long long)tile * TT_TILE_CHUNKS;
         __syncthreads();
         if (tid == 0) { s_ns = 0; s_nw = 0; s_nl = 0; s_total = 0; }
         tile_pieces(tp, P.startmask, P.tile_first, P.nchunks, P.ntiles, tile, P.hi, sc);
+        if (status != 0) return;                                  // nothing global has been written yet
         const u32 np = tp.n, p0 = (u32)tile * TT_TILE_BYTES;     // pieces are indexed per tile
         const long long t0 = c0 * TT_CHUNK - P.shift;             // text offset of the tile start
         u32 wsum = 0;

@@ -450,7 +450,7 @@ def vocab_table_bytes(n_merges: int) -> int:
 
 # DRAM bytes (read + write) per launch from the committed ncu capture of the C3 request
 # (profiles/c3_1M_request_kernels.md).
-NCU_TRAFFIC = {"pieces": 5_388_800, "pretok": 1_130_752, "scatter": 4_909_568}
+NCU_TRAFFIC = {"merge": 3_111_680, "lookup": 2_910_720, "pretok": 1_089_792, "scatter": 1_236_736}
 
 
 def ncu_traffic(kernel: str):

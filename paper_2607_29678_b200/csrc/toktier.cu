@@ -1,7 +1,9 @@
 // C ABI of the toktier library (see include/toktier.h).  Host side: argument checks, vocabulary
-// tables, workspace layout and the kernel chain  k_pretok (K1+K2, tile piece counts) -> k_pieces (K3 per tile in
-// shared memory, K4, K5's count scan in its last CTA) -> k_scatter (K5).
-// Nothing here synchronises with the device except tt_vocab_load and tt_encode_host.
+// tables, workspace layout and the kernel chain  k_pretok (K1+K2, tile piece counts) -> k_lookup (K3 per tile in
+// shared memory, whole-piece lookups) -> k_merge (K4's merges, from global queues) -> k_scatter (K5); sessions
+// (incremental repair), the added-token literal pass and the shadow verifier (host only) sit on top of it.
+// Nothing here synchronises with the device except tt_vocab_load, tt_encode_host, tt_encode_timed and
+// tt_session_append.
 #include "../../include/toktier.h"
 #include "tt_common.cuh"
 #include "tt_pretok_kernels.cuh"

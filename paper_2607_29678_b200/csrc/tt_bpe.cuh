@@ -790,7 +790,7 @@ k_scatter(const ScatterParams P) {
     __shared__ u32 s_nbig;
     __shared__ unsigned long long s_sum[66];
     const int tid = threadIdx.x;
-    cudaGridDependencySynchronize();                         // k_pieces' counts and staged ids are complete from here on
+    cudaGridDependencySynchronize();                         // k_merge's (and with it k_lookup's) results are complete from here on
     // Each CTA takes a contiguous range of tiles.  Tokens before its first tile = the whole groups of tiles
     // before it plus the tiles of its own group before it; the grand total (all groups) gives the count and
     // the capacity check, which every CTA makes for itself.

@@ -5,9 +5,10 @@ Headline metric: latency of one 1,000,000-character request (config C3: agent-tr
 cl100k-style pattern, 100,000-merge vocabulary) through ``tt_encode`` with the text resident in HBM,
 cold caches (L2 flushed before every step), timed with CUDA events on the launching stream.
 Also reported on the same line: the end-to-end figure through the host-buffer entry point
-(``tt_encode_host``: host->device copy of the text and device->host copy of the IDs inside the
-timed region), the batched chars/s of one ``tt_encode_batch`` call over config C5, the HBM roofline
-of the dominant kernel, and the CPU oracle timed on this machine's host cores.
+(``tt_encode_host`` on pinned host buffers: host->device copy of the text inside the timed call, the
+IDs arrive in pinned host memory; the pageable variant beside it), the batched chars/s of one
+``tt_encode_batch`` call over config C5, the latency of an incremental-repair append to a 1M-char
+session, the HBM roofline of the dominant kernel, and the CPU oracle timed on this machine's host cores.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
 

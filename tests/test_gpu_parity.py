@@ -535,3 +535,47 @@ def test_host_entry_point_with_pinned_buffers():
     with pytest.raises(tt.TokTierError) as err:
         gv.encode_host_into(pinned_text, small)
     assert err.value.code == tt.TT_ERR_CAPACITY
+
+
+def test_repeated_calls_on_the_same_buffers():
+    """tt_encode replays a cached CUDA graph when the same argument set comes again: the results must follow
+    the current contents of the text buffer, other lengths and buffers must not be confused with the cached
+    set, and more distinct sets than the cache holds must keep working."""
+    import torch
+    cfg = wl.CONFIGS["C2"]
+    gv, cv = gpu_vocab("C2"), cpu_vocab("C2")
+    texts = [wl.request(cfg, sample=s) for s in range(3)]
+    n = min(t.size for t in texts) - 8
+    texts = [np.frombuffer(t[:n].tobytes().decode("utf-8", errors="ignore").encode("utf-8"), dtype=np.uint8) for t in texts]
+    n = min(t.size for t in texts)
+    texts = [t[:n] if (t[n - 1] < 0x80) else t[:n] for t in texts]
+    want = [cv.encode(t, cfg.pattern_id, nthreads=4)[0] for t in texts]
+    dev = torch.zeros(n + 64, dtype=torch.uint8, device="cuda")
+    bufs = gv.alloc(n)
+    for rep in range(3):
+        for t, w in zip(texts, want):
+            if t.size != n:
+                continue
+            dev[:n].copy_(torch.from_numpy(t.copy()))
+            gv.encode(dev[:n], bufs)
+            torch.cuda.synchronize()
+            k = int(bufs["count"].item())
+            assert int(bufs["status"].item()) == 0 and np.array_equal(bufs["ids"][:k].cpu().numpy(), w)
+    # same buffers, other length
+    half = texts[0][: n // 2]
+    half = np.frombuffer(half.tobytes().decode("utf-8", errors="ignore").encode("utf-8"), dtype=np.uint8)
+    dev[:half.size].copy_(torch.from_numpy(half.copy()))
+    for _ in range(3):
+        gv.encode(dev[:half.size], bufs)
+        torch.cuda.synchronize()
+        k = int(bufs["count"].item())
+        assert np.array_equal(bufs["ids"][:k].cpu().numpy(), cv.encode(half, cfg.pattern_id)[0])
+    # more argument sets than the cache keeps, each used three times in rotation
+    sets = [(torch.from_numpy(texts[0].copy()).cuda(), gv.alloc(n)) for _ in range(20)]
+    for rep in range(3):
+        for d, b in sets:
+            gv.encode(d, b)
+        torch.cuda.synchronize()
+        for d, b in sets:
+            k = int(b["count"].item())
+            assert np.array_equal(b["ids"][:k].cpu().numpy(), want[0])

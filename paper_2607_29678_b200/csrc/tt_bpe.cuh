@@ -184,6 +184,54 @@ __device__ __forceinline__ u32 warp_merge_reg(const u8* __restrict__ text, u32 a
     return warp_merge_reg_rounds(t, r, n, n, a, tab, ext_id, stage, lane);
 }
 
+// ---- warp merge, 33..64 bytes: two tokens per lane, everything in registers ----------------------------------
+// Position k lives in lane k % 32, register k / 32.  A round applies the occurrences of the minimum rank one
+// after the other, leftmost first (a merge marks the pairs next to it stale, so an overlapping occurrence is
+// no candidate any more: exactly the leftmost non-overlapping ones are taken); every step closes the gap
+// with three shuffles per register pair instead of a trip through shared memory.  Then the stale pairs are
+// probed together.  At 32 tokens the one-register rounds take over.
+__device__ __forceinline__ u32 warp_merge_reg2(const u8* __restrict__ text, u32 a, u32 n, const PairTable& tab,
+                                               const int32_t* __restrict__ ext_id, int32_t* __restrict__ stage, int lane) {
+    const u32 FULL = 0xFFFFFFFFu;
+    u32 t0 = text[a + lane], t1 = 32u + lane < n ? text[a + 32 + lane] : 0u;
+    u32 m = n;
+    // pair (k, k + 1): right neighbour of position lane is (lane + 1, reg 0) or, for lane 31, (0, reg 1)
+    u32 nx0 = __shfl_down_sync(FULL, t0, 1); { const u32 w = __shfl_sync(FULL, t1, 0); if (lane == 31) nx0 = w; }
+    u32 nx1 = __shfl_down_sync(FULL, t1, 1);
+    u32 r0 = (u32)lane + 1 < m ? __ldg(tab.bytepair + ((t0 << 8) | nx0)) : TT_RANK_INF;
+    u32 r1 = 32u + lane + 1 < m ? __ldg(tab.bytepair + ((t1 << 8) | nx1)) : TT_RANK_INF;
+    for (u32 round = 0; round < n && m > 32; round++) {
+        const u32 mn = __reduce_min_sync(FULL, min(r0, r1));
+        if (mn == TT_RANK_INF) break;
+        for (u32 step = 0; step < 64; step++) {               // the occurrences of mn, leftmost first
+            const u32 c0 = __ballot_sync(FULL, r0 == mn), c1 = __ballot_sync(FULL, r1 == mn);
+            if (!(c0 | c1)) break;
+            const u32 p = c0 ? (u32)__ffs(c0) - 1 : 32u + (u32)__ffs(c1) - 1;       // merge positions p, p + 1
+            // new token at p, stale ranks at p - 1 and p, everything above p + 1 moves down by one
+            const u32 d0 = __shfl_down_sync(FULL, t0, 1), d1 = __shfl_down_sync(FULL, t1, 1), w0 = __shfl_sync(FULL, t1, 0);
+            const u32 e0 = __shfl_down_sync(FULL, r0, 1), e1 = __shfl_down_sync(FULL, r1, 1), x0 = __shfl_sync(FULL, r1, 0);
+            const u32 k0 = lane, k1 = 32u + lane;
+            const u32 up_t0 = lane == 31 ? w0 : d0, up_r0 = lane == 31 ? x0 : e0;        // old position k0 + 1
+            const u32 up_t1 = lane == 31 ? 0u : d1, up_r1 = lane == 31 ? TT_RANK_INF : e1;  // old position k1 + 1
+            t0 = k0 < p ? t0 : k0 == p ? 256u + mn : up_t0;
+            r0 = k0 + 1 < p ? r0 : (k0 + 1 == p || k0 == p) ? RK_STALE : up_r0;
+            t1 = k1 < p ? t1 : k1 == p ? 256u + mn : up_t1;
+            r1 = k1 + 1 < p ? r1 : (k1 + 1 == p || k1 == p) ? RK_STALE : up_r1;
+            m--;
+            if (k0 + 1 >= m) r0 = TT_RANK_INF;                   // the last token has no pair
+            if (k1 + 1 >= m) r1 = TT_RANK_INF;
+        }
+        nx0 = __shfl_down_sync(FULL, t0, 1); { const u32 w = __shfl_sync(FULL, t1, 0); if (lane == 31) nx0 = w; }
+        nx1 = __shfl_down_sync(FULL, t1, 1);
+        if (r0 == RK_STALE) r0 = pair_probe(tab, t0, nx0);
+        if (r1 == RK_STALE) r1 = pair_probe(tab, t1, nx1);
+    }
+    if (m <= 32) return warp_merge_reg_rounds(t0, r0, m, m, a, tab, ext_id, stage, lane);
+    if ((u32)lane < m) stage[a + lane] = ext_id[t0];
+    if (32u + lane < m) stage[a + 32 + lane] = ext_id[t1];
+    return m;
+}
+
 // ---- warp merge, 33..256 bytes: E tokens per lane in registers, compaction through shared memory ---------
 // Position k lives in lane k % 32, register k / 32.  Each round the surviving (token, rank) pairs are
 // written to their new positions in one of two shared-memory buffers (alternating, so one warp barrier
@@ -720,7 +768,7 @@ k_merge(const PieceParams P) {
         if (e >= nw) break;
         const u64 q = P.q_warp[e];
         const u32 a = (u32)q, i = (u32)(q >> 32) & 2047u, n = (u32)(q >> 43) + 1;
-        const u32 m = n <= 64 ? warp_merge_perm<2>(wbuf, text, a, n, P.tab, P.ext_id, P.stage, lane)
+        const u32 m = n <= 64 ? warp_merge_reg2(text, a, n, P.tab, P.ext_id, P.stage, lane)
                               : warp_merge_perm<WCH>(wbuf, text, a, n, P.tab, P.ext_id, P.stage, lane);
         if (lane == 0) {
             const u32 tile = (u32)(((long long)a + P.shift) / TT_TILE_BYTES);

@@ -43,12 +43,6 @@ struct tt_vocab {
     size_t n_table_tokens = 0;
     uint2* d_meta = nullptr;             // per caller id: (byte length, non-continuation bytes) for tt_spans
     u32 meta_n = 0;
-    // tt_encode keeps instantiated CUDA graphs of its kernel chain for argument sets it has seen before
-    struct GraphSlot { const void* key[6]; size_t len, cap; unsigned seen; cudaGraphExec_t exec; unsigned long long used; };
-    mutable GraphSlot gslots[16] = {};
-    mutable std::mutex gmutex;
-    mutable unsigned long long gclock = 0;
-    mutable cudaStream_t capture_stream = nullptr;
     LitEntry* d_lit_entries = nullptr; u8* d_lit_blob = nullptr;
     LitTable lit{};                      // added-token literals (tt_vocab_add_literals), n == 0: none
     u32 max_token_chars = 1;             // characters of the longest entry (stable boundary check of the sessions)
@@ -92,8 +86,6 @@ extern "C" void tt_vocab_free(tt_vocab* v) {
     if (v->h_text) cudaFreeHost(v->h_text);
     if (v->h_ids) cudaFreeHost(v->h_ids);
     if (v->h_scalars) cudaFreeHost(v->h_scalars);
-    for (auto& g : v->gslots) if (g.exec) cudaGraphExecDestroy(g.exec);
-    if (v->capture_stream) cudaStreamDestroy(v->capture_stream);
     if (v->host_stream) cudaStreamDestroy(v->host_stream);
     delete v;
 }
@@ -482,52 +474,12 @@ static int encode_impl(const tt_vocab* v, const uint8_t* text, size_t len, const
     return TT_OK;
 }
 
-// The chain of one tt_encode call (a memset and four kernels) as an instantiated CUDA graph, replayed when the
-// same arguments come again (paper Sec. 4.2: the chain is captured as a graph so that a request costs one
-// submission).  An argument set is captured the second time it is seen, never while the caller's stream is
-// itself being captured; 16 sets are kept, the least recently used one is replaced.  Returns true if the call
-// was served by a graph launch (rc holds its result).
-static bool encode_by_graph(const tt_vocab* v, const uint8_t* text, size_t len, cudaStream_t st, int32_t* ids_out,
-                            size_t ids_cap, int64_t* count_out, int32_t* status_out, void* workspace, int& rc) {
-    cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
-    if (cudaStreamIsCapturing(st, &cs) != cudaSuccess) { cudaGetLastError(); return false; }
-    if (cs != cudaStreamCaptureStatusNone) return false;
-    std::lock_guard<std::mutex> lk(v->gmutex);
-    const void* key[6] = {text, ids_out, count_out, status_out, workspace, nullptr};
-    tt_vocab::GraphSlot* hit = nullptr; tt_vocab::GraphSlot* lru = &v->gslots[0];
-    for (auto& g : v->gslots) {
-        if (g.seen && g.len == len && g.cap == ids_cap && memcmp(g.key, key, sizeof(key)) == 0) { hit = &g; break; }
-        if (g.used < lru->used) lru = &g;
-    }
-    if (!hit) {                                                   // first sight: remember, run directly
-        if (lru->exec) { cudaGraphExecDestroy(lru->exec); lru->exec = nullptr; }
-        memcpy(lru->key, key, sizeof(key)); lru->len = len; lru->cap = ids_cap; lru->seen = 1; lru->used = ++v->gclock;
-        return false;
-    }
-    hit->used = ++v->gclock;
-    if (!hit->exec) {
-        if (!v->capture_stream && cudaStreamCreateWithFlags(&v->capture_stream, cudaStreamNonBlocking) != cudaSuccess) { cudaGetLastError(); return false; }
-        if (cudaStreamBeginCapture(v->capture_stream, cudaStreamCaptureModeThreadLocal) != cudaSuccess) { cudaGetLastError(); return false; }
-        const int erc = encode_impl(v, text, len, nullptr, 1, v->capture_stream, ids_out, ids_cap, count_out, nullptr, status_out, workspace);
-        cudaGraph_t graph = nullptr;
-        const cudaError_t ce = cudaStreamEndCapture(v->capture_stream, &graph);
-        if (erc != TT_OK || ce != cudaSuccess || !graph) { cudaGetLastError(); if (graph) cudaGraphDestroy(graph); hit->seen = 0; return false; }
-        const cudaError_t ie = cudaGraphInstantiate(&hit->exec, graph, 0);
-        cudaGraphDestroy(graph);
-        if (ie != cudaSuccess) { cudaGetLastError(); hit->exec = nullptr; hit->seen = 0; return false; }
-    }
-    rc = cudaGraphLaunch(hit->exec, st) == cudaSuccess ? TT_OK : TT_ERR_CUDA;
-    if (rc != TT_OK) cudaGetLastError();
-    return true;
-}
-
 extern "C" int tt_encode(const tt_vocab* v, const uint8_t* text, size_t len, void* stream, int32_t* ids_out,
                          size_t ids_cap, int64_t* count_out, int32_t* status_out, void* workspace,
                          size_t workspace_bytes) {
     int rc = check_common(v, text, len, workspace, workspace_bytes, 1);
     if (rc != TT_OK) return rc;
     if (!count_out || !status_out || (len && !ids_out)) return TT_ERR_ARG;
-    if (len && encode_by_graph(v, text, len, (cudaStream_t)stream, ids_out, ids_cap, count_out, status_out, workspace, rc)) return rc;
     return encode_impl(v, text, len, nullptr, 1, (cudaStream_t)stream, ids_out, ids_cap, count_out, nullptr, status_out,
                        workspace);
 }

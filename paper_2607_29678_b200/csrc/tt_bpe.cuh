@@ -48,6 +48,16 @@ __device__ __forceinline__ u32 pair_probe(const PairTable& t, u32 a, u32 b) {
     return TT_RANK_INF;
 }
 
+// Asks for [p, p + bytes) to be brought into L2, spread over the whole grid (no result, nothing waits for it).
+// Used by a kernel while it waits for its predecessor: the tables it is about to probe at random are fetched
+// with idle bandwidth, so that after a cold start its dependent loads find them in L2.
+__device__ __forceinline__ void grid_prefetch_l2(const void* p, size_t bytes) {
+    const char* c = reinterpret_cast<const char*>(p);
+    const size_t lines = (bytes + 127) / 128, stride = (size_t)gridDim.x * blockDim.x;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < lines; i += stride)
+        asm volatile("prefetch.global.L2 [%0];" ::"l"(c + i * 128));
+}
+
 // ---- whole-piece table: byte string of a vocabulary entry -> its id ------------------------------------
 // Holds every token of at most TT_TOKTAB_MAXLEN bytes whose own byte string encodes to exactly that
 // token (checked at load time by running the merge kernel below on every token string), so a hit
@@ -646,6 +656,7 @@ k_lookup(const PieceParams P) {
     __shared__ u32 sc[48];
     const int tid = threadIdx.x;
     cudaTriggerProgrammaticLaunchCompletion();               // the next kernel may be placed; it waits for this grid's memory itself
+    if (P.toktab.slots != nullptr) grid_prefetch_l2(P.toktab.slots, ((size_t)P.toktab.mask + 1) * sizeof(TokSlot));
     cudaGridDependencySynchronize();                         // k_pretok's flags and counts are complete from here on
     const int status = P.hdr->status;                        // looked at after the first tile's flags are in: the loads overlap
     const u8* text = P.base + P.shift;
@@ -746,6 +757,8 @@ k_merge(const PieceParams P) {
     __shared__ u32 sc[48];
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
     cudaTriggerProgrammaticLaunchCompletion();               // k_scatter may be placed; it waits for this grid's memory itself
+    grid_prefetch_l2(P.tab.slots, ((size_t)P.tab.mask + 1) * 4 * sizeof(u64));
+    grid_prefetch_l2(P.tab.bytepair, 65536 * sizeof(u32));
     cudaGridDependencySynchronize();                         // the queues are complete from here on
     if (P.hdr->status != 0) return;
     const u8* text = P.base + P.shift;

@@ -538,9 +538,8 @@ def test_host_entry_point_with_pinned_buffers():
 
 
 def test_repeated_calls_on_the_same_buffers():
-    """tt_encode replays a cached CUDA graph when the same argument set comes again: the results must follow
-    the current contents of the text buffer, other lengths and buffers must not be confused with the cached
-    set, and more distinct sets than the cache holds must keep working."""
+    """The same buffers used for call after call: the results must follow the current contents of the text
+    buffer, another length in the same buffers must work, and many buffer sets in rotation too."""
     import torch
     cfg = wl.CONFIGS["C2"]
     gv, cv = gpu_vocab("C2"), cpu_vocab("C2")
@@ -570,7 +569,7 @@ def test_repeated_calls_on_the_same_buffers():
         torch.cuda.synchronize()
         k = int(bufs["count"].item())
         assert np.array_equal(bufs["ids"][:k].cpu().numpy(), cv.encode(half, cfg.pattern_id)[0])
-    # more argument sets than the cache keeps, each used three times in rotation
+    # many argument sets, each used three times in rotation
     sets = [(torch.from_numpy(texts[0].copy()).cuda(), gv.alloc(n)) for _ in range(20)]
     for rep in range(3):
         for d, b in sets:

@@ -451,7 +451,7 @@ def vocab_table_bytes(n_merges: int) -> int:
 
 # DRAM bytes (read + write) per launch from the committed ncu capture of the C3 request
 # (profiles/c3_1M_request_kernels.md).
-NCU_TRAFFIC = {"merge": 3_111_680, "lookup": 2_910_720, "pretok": 1_089_792, "scatter": 1_236_736}
+NCU_TRAFFIC = {"merge": 5_200_896, "lookup": 9_557_504, "pretok": 1_090_304, "scatter": 1_237_760}
 
 
 def ncu_traffic(kernel: str):

@@ -448,7 +448,7 @@ static int encode_impl(const tt_vocab* v, const uint8_t* text, size_t len, const
     if (rc != TT_OK) return rc;
     MARK(1);
     const int tile_grid = PP.ntiles < v->sm_count * 8 ? PP.ntiles : v->sm_count * 8;
-    const int merge_grid = PP.ntiles * 2 + 1 < v->sm_count * 3 ? PP.ntiles * 2 + 1 : v->sm_count * 3;
+    const int merge_grid = v->sm_count * 3;                  // all resident CTA slots: a request's unsettled pieces get a warp each
     PieceParams Q;
     Q.base = PP.base; Q.shift = PP.lo; Q.hi = PP.hi; Q.nchunks = PP.nchunks; Q.ntiles = PP.ntiles;
     Q.startmask = w.startmask; Q.tile_first = w.tile_first; Q.hdr = w.hdr; Q.tab = v->tab; Q.toktab = v->toktab; Q.longtab = v->longtab; Q.litstart = literals ? w.litstart : nullptr;

@@ -73,3 +73,23 @@ def test_overlapping_literal_chains_and_edges():
     gv.add_literals(["x"], [1])
     with pytest.raises(tt.TokTierError):
         gv.add_literals(["y"], [2])
+
+
+def test_literals_with_the_three_splitter_pattern():
+    """The literal pass in front of TT_PATTERN_SPLIT3: literal boundaries, the cuts of the first two splitter
+    stages and pattern 0 on every span must compose."""
+    import paper_2607_29678_b200 as tt
+    merges, byte_map = wl.load_vocab(wl.CONFIGS["C2"])
+    cv = oracle.Vocab(merges, byte_map)
+    gv = tt.Vocab(merges, byte_map, tt.TT_PATTERN_SPLIT3)
+    lits = ["<|sep|>", "123", "中文", "  "]
+    ids = [800000 + k for k in range(len(lits))]
+    gv.add_literals(lits, ids)
+    rng = random.Random(21)
+    parts = []
+    for _ in range(4000):
+        parts.append(rng.choice(["word ", "12345", "123", "中文字", "中文", "<|sep|>", "  ", " ", "x1中 ", "\n", "9 9", "it's"]))
+    text = np.frombuffer("".join(parts).encode("utf-8"), dtype=np.uint8)
+    got, status = _gpu_encode_added(gv, text)
+    want = oracle.encode_added(cv, text, 3, lits, ids)
+    assert status == 0 and np.array_equal(got, want)

@@ -24,7 +24,7 @@ def _stream(rng, text: bytes, n_cuts: int):
     return [text[a:b] for a, b in zip(cuts[:-1], cuts[1:])]
 
 
-@pytest.mark.parametrize("pattern", [0, 1, 2])
+@pytest.mark.parametrize("pattern", [0, 1, 2, 3])
 def test_stable_boundaries_cut_left_context(pattern):
     """At every stable boundary p of a text T the pieces of T from p on are the pieces of T[p:]: the text to
     the left has no influence (checked by tokenizing the suffix alone), and p itself begins a piece."""

@@ -26,23 +26,24 @@ def _parts(rng, text: bytes, n_cuts: int):
     return [text[a:b] for a, b in zip(cuts[:-1], cuts[1:])]
 
 
-@pytest.mark.parametrize("name,window", [("C1", 512), ("C1", 24), ("C2", 64), ("C4", 200)])
-def test_append_stream_matches_oracle_protocol_and_full_tokenization(name, window):
+@pytest.mark.parametrize("name,window,pattern", [("C1", 512, None), ("C1", 24, None), ("C2", 64, None), ("C4", 200, None), ("C2", 48, 3), ("C2", 100, 2)])
+def test_append_stream_matches_oracle_protocol_and_full_tokenization(name, window, pattern):
     import paper_2607_29678_b200 as tt
     cfg = wl.CONFIGS[name]
-    gv, cv = gpu_vocab(name), cpu_vocab(name)
+    pat = cfg.pattern_id if pattern is None else pattern
+    gv, cv = gpu_vocab(name, pattern=pat), cpu_vocab(name)
     rng = random.Random(1000 + window)
     text = wl.generate(cfg.kind, 99 + window, 9000).tobytes()
     text = text + "é中 1234567890123 x's's's tail   \n\n  end GPU加速 done".encode() * 3
     sess = tt.Session(gv, len(text) + 16, window_chars=window)
-    ref = repair.Session(cv, cfg.pattern_id, window=window)
+    ref = repair.Session(cv, pat, window=window)
     done = b""
     for part in _parts(rng, text, 30):
         info = sess.append(part)
         want_info = ref.append(part)
         done += part
         ids, off, nbytes = sess.records()
-        full, _ = cv.encode(done, cfg.pattern_id)
+        full, _ = cv.encode(done, pat)
         assert nbytes == len(done) and info["status"] == 0 and info["n_tokens"] == full.size
         assert np.array_equal(ids.cpu().numpy(), full)
         assert off.cpu().numpy().tolist() == ref.off

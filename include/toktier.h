@@ -166,7 +166,8 @@ int tt_spans(const tt_vocab* v, const int32_t* ids, const int64_t* count, size_t
  * leftmost-longest literal pass extracts them before the tokenizer family handles the remaining segments).
  *   tt_vocab_add_literals  registers n literals once per vocabulary (HOST arrays, copied): literal i is
  *                          bytes[off[i] .. off[i+1]) (1..255 bytes, all distinct) with id ids[i] >= 0.
- *                          Returns TT_ERR_ARG for bad arguments or a second call.
+ *                          Returns TT_ERR_ARG for bad arguments or a second call.  tt_spans afterwards also
+ *                          knows every literal whose id is below 2^24 and is not an id of the merge table.
  *   tt_encode_added        tt_encode with that pass in front: scanning left to right, at each byte the longest
  *                          literal that matches there is taken and the scan continues behind it; every taken literal
  *                          yields its id, and every stretch of text between literals is tokenized exactly as if it

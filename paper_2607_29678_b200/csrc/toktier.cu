@@ -510,6 +510,27 @@ extern "C" int tt_vocab_add_literals(tt_vocab* v, const uint8_t* bytes, const ui
     }
     T.entries = v->d_lit_entries; T.blob = v->d_lit_blob; T.n = (u32)n; T.maxlen = maxlen;
     v->lit = T;
+    if (v->meta_n) {
+        // tt_spans: byte and character length of every literal whose id the merge table does not use itself
+        int32_t max_id = (int32_t)v->meta_n - 1;
+        for (size_t i = 0; i < n; i++) max_id = ids[i] > max_id ? ids[i] : max_id;
+        if (max_id < (1 << 24)) {
+            std::vector<uint2> meta((size_t)max_id + 1, make_uint2(0, 0));
+            uint2* d_new = nullptr;
+            bool ok = cudaMemcpy(meta.data(), v->d_meta, (size_t)v->meta_n * sizeof(uint2), cudaMemcpyDeviceToHost) == cudaSuccess;
+            for (size_t i = 0; ok && i < n; i++) {
+                if (meta[ids[i]].x != 0) continue;
+                u32 chars = 0;
+                for (u32 k = off[i]; k < off[i + 1]; k++) chars += (bytes[k] & 0xC0) != 0x80;
+                meta[ids[i]] = make_uint2(off[i + 1] - off[i], chars);
+            }
+            ok = ok && cudaMalloc(&d_new, meta.size() * sizeof(uint2)) == cudaSuccess;
+            ok = ok && cudaMemcpy(d_new, meta.data(), meta.size() * sizeof(uint2), cudaMemcpyHostToDevice) == cudaSuccess;
+            if (!ok) { cudaGetLastError(); cudaFree(d_new); return TT_ERR_CUDA; }
+            cudaFree(v->d_meta);
+            v->d_meta = d_new; v->meta_n = (u32)meta.size();
+        }
+    }
     return TT_OK;
 }
 

@@ -93,3 +93,40 @@ def test_literals_with_the_three_splitter_pattern():
     got, status = _gpu_encode_added(gv, text)
     want = oracle.encode_added(cv, text, 3, lits, ids)
     assert status == 0 and np.array_equal(got, want)
+
+
+def test_spans_of_added_tokens():
+    """Span export over the output of tt_encode_added: a literal's record covers the literal's bytes."""
+    import torch
+    import paper_2607_29678_b200 as tt
+    merges, byte_map = wl.load_vocab(wl.CONFIGS["C1"])
+    cv = oracle.Vocab(merges, byte_map)
+    gv = tt.Vocab(merges, byte_map, 0)
+    lits = ["<|user|>", "<|assistant|>", "é中", "\n\n"]
+    ids = [600000 + k for k in range(len(lits))]
+    gv.add_literals(lits, ids)
+    body = wl.generate(wl.KIND_TRANSCRIPT, 77, 30_000)
+    text = np.concatenate([body, np.frombuffer("<|user|>é中é中 x<|assistant|>".encode(), dtype=np.uint8)])
+    d_text = torch.from_numpy(text).cuda()
+    bufs = gv.alloc(text.size)
+    gv.encode_added(d_text, bufs)
+    n = int(bufs["count"].item())
+    byte_off = torch.empty(bufs["ids"].numel() + 1, dtype=torch.int32, device="cuda")
+    char_off = torch.empty_like(byte_off)
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    gv.spans(bufs["ids"], bufs["count"], text.size, byte_off, char_off, st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    got_ids = bufs["ids"][:n].cpu().numpy()
+    bo, co = byte_off[:n + 1].cpu().numpy(), char_off[:n + 1].cpu().numpy()
+    # expected offsets from the token byte strings (vocabulary entries and literals alike)
+    lit_bytes = {i: s.encode("utf-8") for i, s in zip(ids, lits)}
+    pos = cpos = 0
+    data = text.tobytes()
+    for k, t in enumerate(got_ids.tolist()):
+        s = lit_bytes[t] if t in lit_bytes else cv.token_bytes(t)
+        assert bo[k] == pos and co[k] == cpos and data[pos:pos + len(s)] == s
+        pos += len(s)
+        cpos += sum((b & 0xC0) != 0x80 for b in s)
+    assert bo[n] == pos == text.size and co[n] == cpos
+    assert sum(t in lit_bytes for t in got_ids.tolist()) > 20

@@ -29,8 +29,8 @@ struct tt_vocab {
     int device = 0;
     int sm_count = 148;
     size_t n_merges = 0;
-    u64* d_slots = nullptr;
-    u32* d_bytepair = nullptr;
+    uint4* d_slots = nullptr;
+    u64* d_bytepair = nullptr;
     int32_t* d_ext_id = nullptr;
     u8* d_cls = nullptr;
     int cls_bytes = 0;
@@ -237,35 +237,59 @@ extern "C" int tt_vocab_load_ex(const tt_merge* merges, size_t n_merges, const i
         if (byte_map[b] < 0 || !internal.emplace(byte_map[b], (u32)b).second) return TT_ERR_BAD_VOCAB;   // not injective
         ext_id[b] = byte_map[b];
     }
-    // pair table: buckets of four slots, at most one key per bucket on average
-    u32 nbuckets = 256;
-    while (nbuckets < n_merges + 1) nbuckets <<= 1;
-    u32 log2b = 0;
-    while ((1u << log2b) < nbuckets) log2b++;
-    const u32 cap = 4 * nbuckets;
-    std::vector<u64> slots(cap, TT_SLOT_EMPTY);
-    std::vector<u32> bytepair(65536, TT_RANK_INF);      // ranks of the byte-byte pairs, directly indexed
-    const u32 mask = nbuckets - 1, shift = 32 - log2b;
-    std::unordered_set<u64> seen;
-    seen.reserve(2 * n_merges + 16);
+    // merges by internal id; children of every merge result
+    std::vector<u32> lch(256 + n_merges, 0xFFFFFFFFu), rch(256 + n_merges, 0xFFFFFFFFu);
+    struct Triple { u32 r, cl, cr; };
+    std::unordered_map<u64, Triple> info;               // key (left << 18 | right) -> rank and guards
+    info.reserve(6 * n_merges + 16);
     for (size_t r = 0; r < n_merges; r++) {
         const tt_merge& m = merges[r];
         auto l = internal.find(m.left), rr = internal.find(m.right);
         if (l == internal.end() || rr == internal.end()) return TT_ERR_BAD_VOCAB;      // operand not yet defined
         if (m.result < 0 || internal.count(m.result)) return TT_ERR_BAD_VOCAB;         // result id reused
-        const u64 key = ((u64)l->second << TT_ID_BITS) | rr->second;
-        if (!seen.insert(key).second) return TT_ERR_BAD_VOCAB;                         // duplicate pair
-        if (l->second < 256 && rr->second < 256) bytepair[(l->second << 8) | rr->second] = (u32)r;
-        u32 h = pair_bucket(key, shift);
-        for (;;) {
-            u64* b = &slots[4 * (size_t)h];
-            int k = 0;
-            while (k < 4 && b[k] != TT_SLOT_EMPTY) k++;
-            if (k < 4) { b[k] = (key << 20) | (u64)r; break; }
-            h = (h + 1) & mask;
+        const u32 a = l->second, b = rr->second;
+        const u64 key = ((u64)a << TT_ID_BITS) | b;
+        auto ins = info.emplace(key, Triple{TT_RANK_INF, TT_RANK_INF, TT_RANK_INF});
+        if (ins.first->second.r != TT_RANK_INF) return TT_ERR_BAD_VOCAB;               // duplicate pair
+        ins.first->second.r = (u32)r;
+        lch[256 + r] = a; rch[256 + r] = b;
+        // guards: the merge (a, b) of rank r can take b from the left after any token on a's right spine, and a
+        // from the right before any token on b's left spine (ranks ascend, so the first entry is the lowest)
+        for (u32 u = a; u != 0xFFFFFFFFu; u = u >= 256 ? rch[u] : 0xFFFFFFFFu) {
+            Triple& t = info.emplace(((u64)u << TT_ID_BITS) | b, Triple{TT_RANK_INF, TT_RANK_INF, TT_RANK_INF}).first->second;
+            if (t.cl == TT_RANK_INF) t.cl = (u32)r;
+        }
+        for (u32 w = b; w != 0xFFFFFFFFu; w = w >= 256 ? lch[w] : 0xFFFFFFFFu) {
+            Triple& t = info.emplace(((u64)a << TT_ID_BITS) | w, Triple{TT_RANK_INF, TT_RANK_INF, TT_RANK_INF}).first->second;
+            if (t.cr == TT_RANK_INF) t.cr = (u32)r;
         }
         internal.emplace(m.result, (u32)(256 + r));
         ext_id[256 + r] = m.result;
+    }
+    // pair table: buckets of two 16-byte slots, at most one key per bucket on average
+    u32 nbuckets = 256;
+    while (nbuckets < info.size() + 1) nbuckets <<= 1;
+    u32 log2b = 0;
+    while ((1u << log2b) < nbuckets) log2b++;
+    const size_t cap = 2 * (size_t)nbuckets;
+    std::vector<uint4> slots(cap, make_uint4(0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu));
+    std::vector<u64> bytepair(65536, ~0ull);            // the byte-byte pairs, directly indexed: three 20-bit fields
+    const u32 mask = nbuckets - 1, shift = 32 - log2b;
+    for (const auto& kv : info) {
+        const u64 key = kv.first;
+        const Triple& t = kv.second;
+        const u32 a = (u32)(key >> TT_ID_BITS), b = (u32)(key & (TT_MAX_INTERNAL - 1));
+        if (a < 256 && b < 256)
+            bytepair[(a << 8) | b] = (u64)f20_encode(t.r) | ((u64)f20_encode(t.cl) << 20) | ((u64)f20_encode(t.cr) << 40);
+        const u64 kr = (key << 20) | f20_encode(t.r);
+        u32 h = pair_bucket(key, shift);
+        for (;;) {
+            uint4* bk = &slots[2 * (size_t)h];
+            int k = 0;
+            while (k < 2 && !((bk[k].x & bk[k].y) == 0xFFFFFFFFu)) k++;
+            if (k < 2) { bk[k] = make_uint4((u32)kr, (u32)(kr >> 32), t.cl, t.cr); break; }
+            h = (h + 1) & mask;
+        }
     }
     tt_vocab* v = new (std::nothrow) tt_vocab();
     if (!v) return TT_ERR_CUDA;
@@ -279,12 +303,12 @@ extern "C" int tt_vocab_load_ex(const tt_merge* merges, size_t n_merges, const i
     tt_fill_ascii_table(cls.data() + v->cls_bytes - 128);
     bool ok = cudaGetDevice(&v->device) == cudaSuccess;
     ok = ok && cudaDeviceGetAttribute(&v->sm_count, cudaDevAttrMultiProcessorCount, v->device) == cudaSuccess;
-    ok = ok && cudaMalloc(&v->d_slots, (size_t)cap * sizeof(u64)) == cudaSuccess;
-    ok = ok && cudaMalloc(&v->d_bytepair, bytepair.size() * sizeof(u32)) == cudaSuccess;
-    ok = ok && cudaMemcpy(v->d_bytepair, bytepair.data(), bytepair.size() * sizeof(u32), cudaMemcpyHostToDevice) == cudaSuccess;
+    ok = ok && cudaMalloc(&v->d_slots, cap * sizeof(uint4)) == cudaSuccess;
+    ok = ok && cudaMalloc(&v->d_bytepair, bytepair.size() * sizeof(u64)) == cudaSuccess;
+    ok = ok && cudaMemcpy(v->d_bytepair, bytepair.data(), bytepair.size() * sizeof(u64), cudaMemcpyHostToDevice) == cudaSuccess;
     ok = ok && cudaMalloc(&v->d_ext_id, ext_id.size() * sizeof(int32_t)) == cudaSuccess;
     ok = ok && cudaMalloc(&v->d_cls, v->cls_bytes) == cudaSuccess;
-    ok = ok && cudaMemcpy(v->d_slots, slots.data(), (size_t)cap * sizeof(u64), cudaMemcpyHostToDevice) == cudaSuccess;
+    ok = ok && cudaMemcpy(v->d_slots, slots.data(), cap * sizeof(uint4), cudaMemcpyHostToDevice) == cudaSuccess;
     ok = ok && cudaMemcpy(v->d_ext_id, ext_id.data(), ext_id.size() * sizeof(int32_t), cudaMemcpyHostToDevice) == cudaSuccess;
     ok = ok && cudaMemcpy(v->d_cls, cls.data(), v->cls_bytes, cudaMemcpyHostToDevice) == cudaSuccess;
     if (!ok) { cudaGetLastError(); tt_vocab_free(v); return TT_ERR_CUDA; }

@@ -13,39 +13,72 @@
 //     global scratch while the piece still has more than 4,096 tokens).
 // Token ids inside the kernels are "internal": byte b -> b, result of the merge of rank r -> 256 + r;
 // the caller's ids are looked up when the tokens are staged.
+//
+// Rounds merge more than the minimum rank.  The sequential algorithm (always the leftmost pair of the lowest
+// rank) performs a fixed set of merges on a piece; a round may perform any of them early, because the set, not
+// the order, fixes the result.  A pair (t[i], t[i+1]) of rank r is certain to be in that set when neither token
+// can be taken by another merge before rank r comes up:
+//   * t[i] can only be taken from the left by a merge (X, t[i]) whose left operand X ends with the present
+//     token t[i-1] (X is t[i-1] itself or was built on top of it).  cl(u, t) is the lowest rank of any
+//     vocabulary merge (X, t) with u on the right spine of X's merge tree; the left guard is r < cl(t[i-1], t[i]);
+//   * t[i+1] can only be taken from the right by a merge (t[i+1], Y) whose right operand begins with t[i+2].
+//     cr(t, w) is the lowest rank of any merge (t, Y) with w on the left spine of Y; the right guard is
+//     r <= cr(t[i+1], t[i+2]) (at equal rank the pair on the left comes first).
+// Both guards are static properties of the vocabulary and are stored with the pair's rank, so one probe
+// returns (rank, cl, cr) for a pair of adjacent tokens.  The pairs of the round's minimum rank need no guard
+// (nothing can come before them).  In a run of identical pairs (t t t t ...) every other pair from a selected
+// first one is selected, as in the sequential left-to-right order.  Everything selected in a round is merged
+// at once; the result is the sequential one.
 #pragma once
 #include "tt_common.cuh"
 
-// ---- pair table: (left, right) -> rank ---------------------------------------------------------------
-// Buckets of four 8-byte slots (one 32-byte sector); slot = (left << 38) | (right << 20) | rank.
+// ---- pair table: (left, right) -> (rank, cl, cr) ----------------------------------------------------------
+// Buckets of two 16-byte slots (one 32-byte sector); slot = { (left << 38) | (right << 20) | rank20, cl, cr }
+// with rank20 = 0xFFFFF for a pair that is no merge itself (it is in the table for its guards).
 // A key lives in its home bucket or, if that is full, in the following ones; a bucket with a free
 // slot ends the search.  Sized for at most one key per bucket on average.
+struct PairInfo { u32 r, cl, cr; };                   // TT_RANK_INF where there is none
 struct PairTable {
-    const u64* slots;     // 4 * (mask + 1) slots
-    const u32* bytepair;  // rank of the pair (byte a, byte b) at [a << 8 | b], TT_RANK_INF if none: a piece's first probes
+    const uint4* slots;   // 2 * (mask + 1) slots
+    const u64* bytepair;  // (byte a, byte b) at [a << 8 | b]: rank20 | cl20 << 20 | cr20 << 40 (0xFFFFF = none): a piece's first probes
     u32 mask;             // number of buckets - 1 (power of two)
     u32 shift;            // 32 - log2(number of buckets)
 };
+constexpr u32 TT_F20 = 0xFFFFFu;                      // 20-bit field: none
+TT_HD u32 f20_decode(u32 f) { return f == TT_F20 ? TT_RANK_INF : f; }
+TT_HD u32 f20_encode(u32 r) { return r < TT_F20 ? r : TT_F20; }
 TT_HD u32 pair_bucket(u64 key, u32 shift) {
     const u32 x = ((u32)key ^ ((u32)(key >> 32) * 0x9E3779B1u)) * 0x85EBCA6Bu;
     return (x ^ (x >> 15)) * 0xC2B2AE35u >> shift;
 }
 
-__device__ __forceinline__ u32 pair_probe(const PairTable& t, u32 a, u32 b) {
+__device__ __forceinline__ PairInfo pair_none() { PairInfo p; p.r = p.cl = p.cr = TT_RANK_INF; return p; }
+__device__ __forceinline__ bool pair_match(const uint4 s, u64 key, PairInfo& out) {
+    const u64 kr = ((u64)s.y << 32) | s.x;
+    if ((kr >> 20) != key) return false;
+    out.r = f20_decode((u32)kr & TT_F20); out.cl = s.z; out.cr = s.w;
+    return true;
+}
+__device__ __forceinline__ bool pair_slot_free(const uint4 s) { return (s.x & s.y) == 0xFFFFFFFFu; }
+
+__device__ __forceinline__ PairInfo pair_probe(const PairTable& t, u32 a, u32 b) {
     const u64 key = ((u64)a << TT_ID_BITS) | b;
     u32 h = pair_bucket(key, t.shift);
+    PairInfo out = pair_none();
     for (u32 n = 0; n <= t.mask; n++) {               // bounded by the number of buckets
-        const uint4* bp = reinterpret_cast<const uint4*>(t.slots + 4 * (size_t)h);
+        const uint4* bp = t.slots + 2 * (size_t)h;
         const uint4 x = __ldg(bp), y = __ldg(bp + 1);
-        const u64 s0 = ((u64)x.y << 32) | x.x, s1 = ((u64)x.w << 32) | x.z, s2 = ((u64)y.y << 32) | y.x, s3 = ((u64)y.w << 32) | y.z;
-        if ((s0 >> 20) == key) return (u32)(s0 & 0xFFFFFu);
-        if ((s1 >> 20) == key) return (u32)(s1 & 0xFFFFFu);
-        if ((s2 >> 20) == key) return (u32)(s2 & 0xFFFFFu);
-        if ((s3 >> 20) == key) return (u32)(s3 & 0xFFFFFu);
-        if (s3 == TT_SLOT_EMPTY) return TT_RANK_INF;  // slots fill from the front: a free last slot ends the chain
+        if (pair_match(x, key, out) || pair_match(y, key, out)) return out;
+        if (pair_slot_free(y)) return out;            // slots fill from the front: a free last slot ends the chain
         h = (h + 1) & t.mask;
     }
-    return TT_RANK_INF;
+    return out;
+}
+__device__ __forceinline__ PairInfo bytepair_info(const PairTable& t, u32 a, u32 b) {
+    const u64 x = __ldg(t.bytepair + ((a << 8) | b));
+    PairInfo p;
+    p.r = f20_decode((u32)x & TT_F20); p.cl = f20_decode((u32)(x >> 20) & TT_F20); p.cr = f20_decode((u32)(x >> 40) & TT_F20);
+    return p;
 }
 
 // Asks for [p, p + bytes) to be brought into L2, spread over the whole grid (no result, nothing waits for it).
@@ -149,26 +182,36 @@ constexpr int BPE_THREADS = BPE_WARPS * 32;           // = pieces per CTA iterat
 constexpr int WCH = TT_WARP_PIECE_MAX / 32;           // 32-token chunks per piece
 
 // ---- warp merge rounds with at most 32 tokens: one token per lane, no shared memory -----------------------
-// t = token of position `lane`, r = rank of the pair (lane, lane + 1) or TT_RANK_INF, m = token count.
+// t = token of position `lane`, p = (rank, cl, cr) of the pair (lane, lane + 1) or none, m = token count.
 // Runs rounds to the fixpoint, stages the tokens (caller's ids) at stage[a ...] and returns their count.
-__device__ __forceinline__ u32 warp_merge_reg_rounds(u32 t, u32 r, u32 m, u32 max_rounds, u32 a, const PairTable& tab,
+// A round: Q marks a pair identical to the pair on its left (t t t); a pair that is not Q heads a run; a head
+// may go if its left guard holds or it has the round's minimum rank; a pair goes if its run's head may go, it
+// lies an even number of places behind the head and its right guard holds (or it has the minimum rank).
+__device__ __forceinline__ u32 warp_merge_reg_rounds(u32 t, PairInfo p, u32 m, u32 a, const PairTable& tab,
                                                      const int32_t* __restrict__ ext_id, int32_t* __restrict__ stage, int lane) {
-    const u32 FULL = 0xFFFFFFFFu, lt = (1u << lane) - 1;
+    const u32 FULL = 0xFFFFFFFFu, lt = (1u << lane) - 1, le = lt | (1u << lane);
+    u32 r = p.r, cl = p.cl, cr = p.cr;
+    if ((u32)lane + 1 >= m) r = cl = cr = TT_RANK_INF;      // the last token has no pair
+    const u32 max_rounds = m;                           // every round merges at least one pair
     for (u32 round = 0; round < max_rounds; round++) {
         const u32 mn = __reduce_min_sync(FULL, r);
         if (mn == TT_RANK_INF) break;
-        // leftmost non-overlapping occurrences: inside a run of consecutive candidates, every other one
-        const u32 c = __ballot_sync(FULL, r == mn);
-        const u32 below = ~c & lt;
-        const u32 dist = below ? (u32)(lane - (32 - __clz(below))) : (u32)lane;
-        const u32 sel = __ballot_sync(FULL, ((c >> lane) & 1) && !(dist & 1));
+        const u32 tl = __shfl_up_sync(FULL, t, 1), tn0 = __shfl_down_sync(FULL, t, 1);
+        u32 cll = __shfl_up_sync(FULL, cl, 1), crr = __shfl_down_sync(FULL, cr, 1);
+        if (lane == 0) cll = TT_RANK_INF;
+        if (lane == 31) crr = TT_RANK_INF;
+        const bool R = r != TT_RANK_INF, Mn = r == mn;
+        const bool Q = R && lane >= 1 && tl == t && t == tn0;
+        const u32 qm = __ballot_sync(FULL, Q), hm = __ballot_sync(FULL, !Q && R && (r < cll || Mn));
+        const u32 h = 31u - (u32)__clz(~qm & le);       // bit 0 of qm is never set
+        const u32 sel = __ballot_sync(FULL, R && ((hm >> h) & 1) && !(((u32)lane - h) & 1) && (r <= crr || Mn));
         const bool me = (sel >> lane) & 1;
         const bool nxt = lane < 31 ? ((sel >> (lane + 1)) & 1) : false;
-        const u32 nt = me ? 256u + mn : t;
+        const u32 nt = me ? 256u + r : t;
         const u32 nr = (me || nxt) ? RK_STALE : r;
         // survivors move down: new lane j takes the j-th surviving old lane
         u32 src;
-        if ((sel & (sel - 1)) == 0) {                   // one merge (the usual case): everything above it moves down by one
+        if ((sel & (sel - 1)) == 0) {                   // one merge: everything above it moves down by one
             src = (u32)lane + ((u32)lane > (u32)(__ffs(sel) - 1) ? 1u : 0u);
         } else {
             const u32 surv = ~(sel << 1) & (m >= 32 ? FULL : ((1u << m) - 1));
@@ -176,10 +219,12 @@ __device__ __forceinline__ u32 warp_merge_reg_rounds(u32 t, u32 r, u32 m, u32 ma
         }
         t = __shfl_sync(FULL, nt, src & 31);
         r = __shfl_sync(FULL, nr, src & 31);
+        cl = __shfl_sync(FULL, cl, src & 31);
+        cr = __shfl_sync(FULL, cr, src & 31);
         m -= __popc(sel);
         const u32 tn = __shfl_down_sync(FULL, t, 1);
-        if ((u32)lane + 1 >= m) r = TT_RANK_INF;
-        else if (r == RK_STALE) r = pair_probe(tab, t, tn);
+        if ((u32)lane + 1 >= m) r = cl = cr = TT_RANK_INF;
+        else if (r == RK_STALE) { const PairInfo q = pair_probe(tab, t, tn); r = q.r; cl = q.cl; cr = q.cr; }
     }
     if ((u32)lane < m) stage[a + lane] = ext_id[t];
     return m;
@@ -190,105 +235,72 @@ __device__ __forceinline__ u32 warp_merge_reg(const u8* __restrict__ text, u32 a
                                               const int32_t* __restrict__ ext_id, int32_t* __restrict__ stage, int lane) {
     const u32 t = (u32)lane < n ? text[a + lane] : 0;
     const u32 tn = __shfl_down_sync(0xFFFFFFFFu, t, 1);
-    const u32 r = ((u32)lane + 1 < n) ? __ldg(tab.bytepair + ((t << 8) | tn)) : TT_RANK_INF;
-    return warp_merge_reg_rounds(t, r, n, n, a, tab, ext_id, stage, lane);
+    const PairInfo p = ((u32)lane + 1 < n) ? bytepair_info(tab, t, tn) : pair_none();
+    return warp_merge_reg_rounds(t, p, n, a, tab, ext_id, stage, lane);
 }
 
-// ---- warp merge, 33..64 bytes: two tokens per lane, everything in registers ----------------------------------
-// Position k lives in lane k % 32, register k / 32.  A round applies the occurrences of the minimum rank one
-// after the other, leftmost first (a merge marks the pairs next to it stale, so an overlapping occurrence is
-// no candidate any more: exactly the leftmost non-overlapping ones are taken); every step closes the gap
-// with three shuffles per register pair instead of a trip through shared memory.  Then the stale pairs are
-// probed together.  At 32 tokens the one-register rounds take over.
-__device__ __forceinline__ u32 warp_merge_reg2(const u8* __restrict__ text, u32 a, u32 n, const PairTable& tab,
-                                               const int32_t* __restrict__ ext_id, int32_t* __restrict__ stage, int lane) {
-    const u32 FULL = 0xFFFFFFFFu;
-    u32 t0 = text[a + lane], t1 = 32u + lane < n ? text[a + 32 + lane] : 0u;
-    u32 m = n;
-    // pair (k, k + 1): right neighbour of position lane is (lane + 1, reg 0) or, for lane 31, (0, reg 1)
-    u32 nx0 = __shfl_down_sync(FULL, t0, 1); { const u32 w = __shfl_sync(FULL, t1, 0); if (lane == 31) nx0 = w; }
-    u32 nx1 = __shfl_down_sync(FULL, t1, 1);
-    u32 r0 = (u32)lane + 1 < m ? __ldg(tab.bytepair + ((t0 << 8) | nx0)) : TT_RANK_INF;
-    u32 r1 = 32u + lane + 1 < m ? __ldg(tab.bytepair + ((t1 << 8) | nx1)) : TT_RANK_INF;
-    for (u32 round = 0; round < n && m > 32; round++) {
-        const u32 mn = __reduce_min_sync(FULL, min(r0, r1));
-        if (mn == TT_RANK_INF) break;
-        for (u32 step = 0; step < 64; step++) {               // the occurrences of mn, leftmost first
-            const u32 c0 = __ballot_sync(FULL, r0 == mn), c1 = __ballot_sync(FULL, r1 == mn);
-            if (!(c0 | c1)) break;
-            const u32 p = c0 ? (u32)__ffs(c0) - 1 : 32u + (u32)__ffs(c1) - 1;       // merge positions p, p + 1
-            // new token at p, stale ranks at p - 1 and p, everything above p + 1 moves down by one
-            const u32 d0 = __shfl_down_sync(FULL, t0, 1), d1 = __shfl_down_sync(FULL, t1, 1), w0 = __shfl_sync(FULL, t1, 0);
-            const u32 e0 = __shfl_down_sync(FULL, r0, 1), e1 = __shfl_down_sync(FULL, r1, 1), x0 = __shfl_sync(FULL, r1, 0);
-            const u32 k0 = lane, k1 = 32u + lane;
-            const u32 up_t0 = lane == 31 ? w0 : d0, up_r0 = lane == 31 ? x0 : e0;        // old position k0 + 1
-            const u32 up_t1 = lane == 31 ? 0u : d1, up_r1 = lane == 31 ? TT_RANK_INF : e1;  // old position k1 + 1
-            t0 = k0 < p ? t0 : k0 == p ? 256u + mn : up_t0;
-            r0 = k0 + 1 < p ? r0 : (k0 + 1 == p || k0 == p) ? RK_STALE : up_r0;
-            t1 = k1 < p ? t1 : k1 == p ? 256u + mn : up_t1;
-            r1 = k1 + 1 < p ? r1 : (k1 + 1 == p || k1 == p) ? RK_STALE : up_r1;
-            m--;
-            if (k0 + 1 >= m) r0 = TT_RANK_INF;                   // the last token has no pair
-            if (k1 + 1 >= m) r1 = TT_RANK_INF;
-        }
-        nx0 = __shfl_down_sync(FULL, t0, 1); { const u32 w = __shfl_sync(FULL, t1, 0); if (lane == 31) nx0 = w; }
-        nx1 = __shfl_down_sync(FULL, t1, 1);
-        if (r0 == RK_STALE) r0 = pair_probe(tab, t0, nx0);
-        if (r1 == RK_STALE) r1 = pair_probe(tab, t1, nx1);
-    }
-    if (m <= 32) return warp_merge_reg_rounds(t0, r0, m, m, a, tab, ext_id, stage, lane);
-    if ((u32)lane < m) stage[a + lane] = ext_id[t0];
-    if (32u + lane < m) stage[a + 32 + lane] = ext_id[t1];
-    return m;
-}
-
-// ---- warp merge, 33..256 bytes: E tokens per lane in registers, compaction through shared memory ---------
-// Position k lives in lane k % 32, register k / 32.  Each round the surviving (token, rank) pairs are
-// written to their new positions in one of two shared-memory buffers (alternating, so one warp barrier
-// per round suffices) and read back; ranks next to a merge are marked stale and probed again.
+// ---- warp merge, 33..32 E bytes: E tokens per lane, compaction through shared memory ------------------------
+// Position k lives in lane k % 32, register k / 32.  Shared memory holds two copies of four arrays of 32 E
+// words (token, rank, cl, cr by position).  Each round the survivors are written to their new positions in
+// the other copy and read back (one warp barrier); ranks next to a merge are marked stale and probed again,
+// the probed guards go to the current copy, from which the next round reads its neighbours' values.
 template <int E>
-__device__ __forceinline__ u32 warp_merge_perm(u64* buf /* 2 * 32 * E entries of this warp */, const u8* __restrict__ text,
+__device__ __forceinline__ u32 warp_merge_perm(u32* buf /* 2 * 4 * 32 E words of this warp */, const u8* __restrict__ text,
                                                u32 a, u32 n, const PairTable& tab, const int32_t* __restrict__ ext_id,
                                                int32_t* __restrict__ stage, int lane) {
-    const u32 FULL = 0xFFFFFFFFu, lt = (1u << lane) - 1;
+    constexpr u32 N = 32 * E;
+    const u32 FULL = 0xFFFFFFFFu, lt = (1u << lane) - 1, le = lt | (1u << lane);
     u32 t[E], r[E];
     u32 m = n;
+    u32* cb = buf;                                      // current copy: tokens [0, N), ranks [N, 2N), cl [2N, 3N), cr [3N, 4N)
+    u32* ob = buf + 4 * N;
     __syncwarp();
 #pragma unroll
     for (int j = 0; j < E; j++) {
         const u32 k = j * 32 + lane;
         t[j] = k < n ? text[a + k] : 0;
-        buf[k] = t[j];
+        cb[k] = t[j];
     }
     __syncwarp();
 #pragma unroll
     for (int j = 0; j < E; j++) {
         const u32 k = j * 32 + lane;
-        r[j] = (k + 1 < n) ? __ldg(tab.bytepair + ((t[j] << 8) | (u32)buf[k + 1])) : TT_RANK_INF;
+        const PairInfo p = (k + 1 < n) ? bytepair_info(tab, t[j], cb[k + 1]) : pair_none();
+        r[j] = p.r; cb[2 * N + k] = p.cl; cb[3 * N + k] = p.cr;
     }
-    int cur = 0;
-    for (u32 round = 0; round < n; round++) {          // at most n - 1 merges
+    for (u32 round = 0; round < n; round++) {          // at most n - 1 merges, at least one per round
         u32 mn = r[0];
 #pragma unroll
         for (int j = 1; j < E; j++) mn = min(mn, r[j]);
         mn = __reduce_min_sync(FULL, mn);
         if (mn == TT_RANK_INF) break;
-        if (m <= 32) return warp_merge_reg_rounds(t[0], r[0], m, m, a, tab, ext_id, stage, lane);   // cheaper rounds from here on
+        __syncwarp();                                   // the guards written after the probes are visible
+        if (m <= 32) {                                  // cheaper rounds from here on
+            PairInfo p; p.r = r[0]; p.cl = cb[2 * N + lane]; p.cr = cb[3 * N + lane];
+            return warp_merge_reg_rounds(t[0], p, m, a, tab, ext_id, stage, lane);
+        }
         const int nch = (int)((m + 31) >> 5);
         u32 sel[E];
-        u32 prev_ones = 0;                              // candidate run ending at the top of the previous word
+        u32 carry_hok = 0, carry_par = 0;               // head of the run that reaches into the word: may it go / parity of its position
 #pragma unroll
         for (int j = 0; j < E; j++) {
             sel[j] = 0;
             if (j < nch) {
-                const u32 c = __ballot_sync(FULL, r[j] == mn);
-                const u32 below = ~c & lt;
-                const u32 dist = below ? (u32)(lane - (32 - __clz(below))) : (u32)lane + prev_ones;
-                sel[j] = __ballot_sync(FULL, ((c >> lane) & 1) && !(dist & 1));
-                prev_ones = (c == FULL) ? prev_ones + 32 : (u32)__clz(~c);
+                const u32 k = j * 32 + lane;
+                const bool R = r[j] != TT_RANK_INF, Mn = r[j] == mn;          // R implies k + 1 < m
+                const u32 tl = k ? cb[k - 1] : 0xFFFFFFFFu, tn = R ? cb[k + 1] : 0xFFFFFFFEu;
+                const u32 cll = k ? cb[2 * N + k - 1] : TT_RANK_INF;
+                const u32 crr = (k + 2 < m) ? cb[3 * N + k + 1] : TT_RANK_INF;
+                const bool Q = R && tl == t[j] && t[j] == tn;
+                const u32 qm = __ballot_sync(FULL, Q), hm = __ballot_sync(FULL, !Q && R && (r[j] < cll || Mn));
+                const u32 z = ~qm & le;
+                u32 hok, par;
+                if (z) { const u32 ph = 31u - (u32)__clz(z); hok = (hm >> ph) & 1; par = ((u32)lane - ph) & 1; }
+                else { hok = carry_hok; par = ((u32)lane & 1) ^ carry_par; }
+                sel[j] = __ballot_sync(FULL, R && hok && !par && (r[j] <= crr || Mn));
+                if (~qm) { const u32 ph = 31u - (u32)__clz(~qm); carry_par = ph & 1; carry_hok = (hm >> ph) & 1; }
             }
         }
-        u64* nb = buf + (cur ^ 1) * (32 * E);
         u32 removed = 0;
 #pragma unroll
         for (int j = 0; j < E; j++) {
@@ -300,24 +312,29 @@ __device__ __forceinline__ u32 warp_merge_perm(u64* buf /* 2 * 32 * E entries of
                 const bool next_sel = lane < 31 ? ((s >> (lane + 1)) & 1) : ((j + 1 < E) ? (sel[j + 1 < E ? j + 1 : j] & 1) : 0);
                 if (k < m && !gone) {
                     const u32 np = k - removed - __popc(s & lt);
-                    nb[np] = ((u64)((me || next_sel) ? RK_STALE : r[j]) << 32) | (me ? 256u + mn : t[j]);
+                    ob[np] = me ? 256u + r[j] : t[j];
+                    ob[N + np] = (me || next_sel) ? RK_STALE : r[j];
+                    ob[2 * N + np] = cb[2 * N + k];
+                    ob[3 * N + np] = cb[3 * N + k];
                 }
                 removed += __popc(s);
             }
         }
         m -= removed;
-        cur ^= 1;
+        { u32* x = cb; cb = ob; ob = x; }
         __syncwarp();
 #pragma unroll
         for (int j = 0; j < E; j++) {
             const u32 k = j * 32 + lane;
             r[j] = TT_RANK_INF;
             if (k < m) {
-                const u64 v = nb[k];
-                t[j] = (u32)v;
-                r[j] = (u32)(v >> 32);
+                t[j] = cb[k];
+                r[j] = cb[N + k];
                 if (k + 1 >= m) r[j] = TT_RANK_INF;
-                else if (r[j] == RK_STALE) r[j] = pair_probe(tab, t[j], (u32)nb[k + 1]);
+                else if (r[j] == RK_STALE) {
+                    const PairInfo p = pair_probe(tab, t[j], cb[k + 1]);
+                    r[j] = p.r; cb[2 * N + k] = p.cl; cb[3 * N + k] = p.cr;
+                }
             }
         }
     }
@@ -339,23 +356,20 @@ __device__ __forceinline__ u32 warp_merge_perm(u64* buf /* 2 * 32 * E entries of
 // threads of the warp hit different banks whatever rows they are at.
 constexpr int LANE_SLOTS = 32;                        // pieces a warp merges at once
 constexpr int LANE_MAX = 32;                          // bytes per piece on this path
-// Two independent probes with both first-bucket loads in flight together.
-__device__ __forceinline__ u32 pair_match_first(const PairTable& t, const uint4 lo, const uint4 hi, u64 key) {
-    const u64 s0 = ((u64)lo.y << 32) | lo.x, s1 = ((u64)lo.w << 32) | lo.z, s2 = ((u64)hi.y << 32) | hi.x, s3 = ((u64)hi.w << 32) | hi.z;
-    if ((s0 >> 20) == key) return (u32)(s0 & 0xFFFFFu);
-    if ((s1 >> 20) == key) return (u32)(s1 & 0xFFFFFu);
-    if ((s2 >> 20) == key) return (u32)(s2 & 0xFFFFFu);
-    if ((s3 >> 20) == key) return (u32)(s3 & 0xFFFFFu);
-    if (s3 == TT_SLOT_EMPTY) return TT_RANK_INF;
-    return pair_probe(t, (u32)(key >> TT_ID_BITS), (u32)(key & (TT_MAX_INTERNAL - 1)));     // full bucket: walk the chain
+// Two independent probes (ranks only) with both first-bucket loads in flight together.
+__device__ __forceinline__ u32 pair_rank_first(const PairTable& t, const uint4 lo, const uint4 hi, u64 key) {
+    PairInfo p = pair_none();
+    if (pair_match(lo, key, p) || pair_match(hi, key, p)) return p.r;
+    if (pair_slot_free(hi)) return TT_RANK_INF;
+    return pair_probe(t, (u32)(key >> TT_ID_BITS), (u32)(key & (TT_MAX_INTERNAL - 1))).r;     // full bucket: walk the chain
 }
 __device__ __forceinline__ void pair_probe2(const PairTable& t, u32 a0, u32 b0, u32 a1, u32 b1, u32& r0, u32& r1) {
     const u64 key0 = ((u64)a0 << TT_ID_BITS) | b0, key1 = ((u64)a1 << TT_ID_BITS) | b1;
-    const uint4* p0 = reinterpret_cast<const uint4*>(t.slots + 4 * (size_t)pair_bucket(key0, t.shift));
-    const uint4* p1 = reinterpret_cast<const uint4*>(t.slots + 4 * (size_t)pair_bucket(key1, t.shift));
+    const uint4* p0 = t.slots + 2 * (size_t)pair_bucket(key0, t.shift);
+    const uint4* p1 = t.slots + 2 * (size_t)pair_bucket(key1, t.shift);
     const uint4 x0 = __ldg(p0), y0 = __ldg(p0 + 1), x1 = __ldg(p1), y1 = __ldg(p1 + 1);
-    r0 = pair_match_first(t, x0, y0, key0);
-    r1 = pair_match_first(t, x1, y1, key1);
+    r0 = pair_rank_first(t, x0, y0, key0);
+    r1 = pair_rank_first(t, x1, y1, key1);
 }
 
 // Tokens stay at the byte position where they began; `al` has a bit per position that still holds a
@@ -371,7 +385,7 @@ __device__ __forceinline__ u32 lane_merge(u32* __restrict__ tok, u32* __restrict
     for (u32 k = 1; k < n; k++) {
         const u32 t = text[a + k];
         TK(k) = t;
-        RK(k - 1) = __ldg(tab.bytepair + ((prev << 8) | t));
+        RK(k - 1) = f20_decode((u32)__ldg(tab.bytepair + ((prev << 8) | t)) & TT_F20);
         prev = t;
     }
     u32 al = 0xFFFFFFFFu >> (32 - n);
@@ -456,68 +470,99 @@ __device__ __forceinline__ u32 cta_min_u32(u32 v, u32* scratch /* >= 33 */) {
 }
 
 // ---- CTA merge for long pieces -----------------------------------------------------------------------------
-// arr[i] = token | (rank of the pair (i, i+1) << 32), in global scratch or shared memory.  One round:
-// the minimum rank is found, every thread takes LK consecutive positions, decides which of its
-// candidates are merged (the parity of a run of consecutive candidates is carried from thread to
-// thread with one ballot-based scan; LK is even, so a slice that is all candidates leaves the parity
-// unchanged), and the survivors are written to their new positions in place, chunk after chunk (every
-// thread of a chunk has its positions in registers before anything is written, and writes never pass
-// the read front).  Ranks next to a merge are marked stale and probed again in a second sweep, which
-// also yields the next round's minimum.
+// arr[i] = token | rank20 << 18 | cl20 << 38 and crr[i] = cr20 for position i (rank and guards of the pair
+// (i, i + 1); 20-bit fields, 0xFFFFF = none), in global scratch or shared memory.  One round: the minimum rank
+// is found, every thread takes LK consecutive positions and decides which of its pairs are merged (same rule
+// as in the warp rounds; the state of a run of identical pairs that crosses slices -- may its head go, parity
+// of the distance to it -- is carried from thread to thread with one ballot-based scan; LK is even, so a
+// slice that lies inside one run passes the state on unchanged), and the survivors are written to their new
+// positions in place, chunk after chunk (every thread of a chunk has its positions in registers before
+// anything is written, and writes never pass the read front).  Ranks next to a merge are marked stale and
+// probed again in a second sweep, which also yields the next round's minimum.
 constexpr int LK = 16;
+constexpr u32 F20_STALE = 0xFFFFEu;
+TT_HD u64 lp_pack(u32 t, u32 r20, u32 cl20) { return (u64)t | ((u64)r20 << TT_ID_BITS) | ((u64)cl20 << (TT_ID_BITS + 20)); }
+TT_HD u32 lp_tok(u64 v) { return (u32)v & (TT_MAX_INTERNAL - 1); }
+TT_HD u32 lp_rank(u64 v) { return (u32)(v >> TT_ID_BITS) & TT_F20; }
+TT_HD u32 lp_cl(u64 v) { return (u32)(v >> (TT_ID_BITS + 20)) & TT_F20; }
 
-__device__ __noinline__ u32 cta_merge_rounds(u64* arr, u32 m, const PairTable& tab, u32* s_scr /* >= 48 */, u32 stop_at, bool& finished) {
+__device__ __noinline__ u32 cta_merge_rounds(u64* arr, u32* crr, u32 m, const PairTable& tab, u32* s_scr /* >= 48 */, u32 stop_at, bool& finished) {
     const int tid = threadIdx.x, T = blockDim.x, lane = tid & 31, wid = tid >> 5, nw = T >> 5;
+    const u32 FULL = 0xFFFFFFFFu, inmask = (1u << LK) - 1;
     finished = false;
     // minimum rank of the current array
-    u32 lmin = TT_RANK_INF;
-    for (u32 i = tid; i < m; i += T) lmin = min(lmin, (u32)(arr[i] >> 32));
+    u32 lmin = TT_F20;
+    for (u32 i = tid; i < m; i += T) lmin = min(lmin, lp_rank(arr[i]));
     for (;;) {
         const u32 mn = cta_min_u32(lmin, s_scr);
-        if (mn == TT_RANK_INF) { finished = true; return m; }
+        if (mn >= F20_STALE) { finished = true; return m; }
         if (m <= stop_at) return m;
-        u32 carry_par = 0, out = 0;                        // parity of the candidate run before the chunk; survivors so far
+        u32 carry_hok = 0, carry_par = 0, carry_last = 0, out = 0;    // run state and last selection before the chunk; survivors so far
         for (u32 base = 0; base < m; base += (u32)T * LK) {
             const u32 i0 = base + (u32)tid * LK;
-            u32 tok[LK + 1], rk[LK + 1];
+            u64 v[LK + 3];                                  // positions i0 - 1 .. i0 + LK + 1
+            u32 c[LK + 3];
 #pragma unroll
-            for (int k = 0; k <= LK; k++) {
-                const u32 i = i0 + k;
-                const u64 v = i < m ? arr[i] : ~0ull;
-                tok[k] = (u32)v; rk[k] = i < m ? (u32)(v >> 32) : TT_RANK_INF;
+            for (int k = 0; k < LK + 3; k++) {
+                const u32 i = i0 + k - 1;                   // wraps for position -1 of the piece: not below m
+                v[k] = lp_pack(0, TT_F20, TT_F20); c[k] = TT_F20;
+                if (k == 0 && tid == 0) { if (base) v[k] = lp_pack(s_scr[42], TT_F20, s_scr[43]); }   // overwritten by the chunk before: carried
+                else if (i < m) { v[k] = arr[i]; c[k] = crr[i]; }
             }
             const u32 nval = i0 < m ? min((u32)LK, m - i0) : 0;
-            u32 cand = 0;
-#pragma unroll
-            for (int k = 0; k <= LK; k++) cand |= (u32)(rk[k] == mn) << k;
-            const u32 cand_in = cand & ((1u << LK) - 1);
-            const bool all = cand_in == ((1u << LK) - 1);
-            // parity of my trailing candidate run (if not all candidates)
-            const u32 trail = __clz(~(cand_in << (32 - LK)));                 // consecutive candidates at the top of the slice
-            const u32 my_par = trail & 1;
-            // incoming parity: trailing parity of the nearest lower slice that is not all candidates
-            const u32 allm = __ballot_sync(0xFFFFFFFFu, all), parm = __ballot_sync(0xFFFFFFFFu, my_par);
-            const u32 lower = ~allm & ((1u << lane) - 1);
-            __syncthreads();
-            if (lane == 31) { const u32 na = ~allm; s_scr[wid] = na ? (2u | ((parm >> (31 - __clz(na))) & 1)) : 0u; }   // 0 = all lanes pass through
-            __syncthreads();
-            u32 in_par;
-            if (lower) in_par = (parm >> (31 - __clz(lower))) & 1;
-            else {
-                in_par = carry_par;
-                for (int w = wid - 1; w >= 0; w--) { const u32 e = s_scr[w]; if (e) { in_par = e & 1; break; } }
-            }
-            u32 next_carry = carry_par;
-            for (int w = nw - 1; w >= 0; w--) { const u32 e = s_scr[w]; if (e) { next_carry = e & 1; break; } }
-            // selection inside the slice (positions 0..LK; position LK only to know whether it is merged)
-            u32 sel = 0, off = in_par;
+            u32 Qm = 0, Hm = 0, Gm = 0;                     // bit k: position i0 + k, k = 0 .. LK
 #pragma unroll
             for (int k = 0; k <= LK; k++) {
-                if ((cand >> k) & 1) { sel |= (u32)!(off & 1) << k; off++; } else off = 0;
+                const u32 rr = lp_rank(v[k + 1]), tk = lp_tok(v[k + 1]);
+                const bool R = rr < F20_STALE, Mn = rr == mn;
+                const bool Q = R && (i0 + k >= 1) && lp_tok(v[k]) == tk && tk == lp_tok(v[k + 2]);
+                Qm |= (u32)Q << k;
+                Hm |= (u32)(!Q && R && (rr < lp_cl(v[k]) || Mn)) << k;
+                Gm |= (u32)(R && (rr <= c[k + 2] || Mn)) << k;
             }
-            const bool gone0 = in_par == 1;                                    // the element before the slice was merged with my first
-            const u32 gone = ((sel << 1) | (u32)gone0) & ((1u << LK) - 1);
-            const u32 valid = nval >= LK ? ((1u << LK) - 1) : ((1u << nval) - 1);
+            // state handed to the next slice: from my highest pair that heads a run
+            const u32 nq = ~Qm & inmask;
+            const bool all = nq == 0;
+            u32 out_hok = 0, out_par = 0;
+            if (nq) { const u32 ph = 31u - (u32)__clz(nq); out_hok = (Hm >> ph) & 1; out_par = ((u32)LK - ph) & 1; }
+            const u32 allm = __ballot_sync(FULL, all), hokm = __ballot_sync(FULL, out_hok), parm = __ballot_sync(FULL, out_par);
+            const u32 lower = ~allm & ((1u << lane) - 1);
+            __syncthreads();
+            if (lane == 31) {
+                const u32 na = ~allm;
+                u32 e = 0;
+                if (na) { const u32 src = 31u - (u32)__clz(na); e = 4u | (((hokm >> src) & 1) << 1) | ((parm >> src) & 1); }
+                s_scr[wid] = e;                              // 0 = all lanes pass through
+            }
+            __syncthreads();
+            u32 in_hok, in_par;
+            if (lower) { const u32 src = 31u - (u32)__clz(lower); in_hok = (hokm >> src) & 1; in_par = (parm >> src) & 1; }
+            else {
+                in_hok = carry_hok; in_par = carry_par;
+                for (int w = wid - 1; w >= 0; w--) { const u32 e = s_scr[w]; if (e) { in_hok = (e >> 1) & 1; in_par = e & 1; break; } }
+            }
+            u32 next_hok = carry_hok, next_par = carry_par;
+            for (int w = nw - 1; w >= 0; w--) { const u32 e = s_scr[w]; if (e) { next_hok = (e >> 1) & 1; next_par = e & 1; break; } }
+            // selection inside the slice (positions 0..LK; position LK only to know whether it is merged)
+            u32 sel = 0;
+            {
+                u32 hok = in_hok, par = in_par;
+#pragma unroll
+                for (int k = 0; k <= LK; k++) {
+                    if (!((Qm >> k) & 1)) { hok = (Hm >> k) & 1; par = 0; }
+                    sel |= (((Gm >> k) & 1) & hok & (par ^ 1u)) << k;
+                    par ^= 1u;
+                }
+            }
+            // was the position before my slice merged with my first one?
+            const u32 lastm = __ballot_sync(FULL, (sel >> (LK - 1)) & 1);
+            if (lane == 31) s_scr[33 + wid] = lastm >> 31;
+            if (tid == T - 1) { s_scr[42] = lp_tok(v[LK]); s_scr[43] = lp_cl(v[LK]); }     // position i0 + LK - 1 as it is now
+            __syncthreads();
+            const u32 gone0 = lane ? (lastm >> (lane - 1)) & 1 : (wid ? s_scr[33 + wid - 1] : carry_last);
+            const u32 next_last = s_scr[33 + nw - 1];
+            const u32 gone = ((sel << 1) | gone0) & inmask;
+            const u32 valid = nval >= LK ? inmask : ((1u << nval) - 1);
             const u32 surv = valid & ~gone;
             u32 tot;
             const u32 ex = cta_excl_sum_scan(__popc(surv), s_scr, &tot);         // all loads of the chunk are done: barrier inside
@@ -527,24 +572,29 @@ __device__ __noinline__ u32 cta_merge_rounds(u64* arr, u32 m, const PairTable& t
                 if ((surv >> k) & 1) {
                     const bool me = (sel >> k) & 1;
                     const bool nxt = me ? false : ((sel >> (k + 1)) & 1);
-                    const u32 nt = me ? 256u + mn : tok[k];
-                    const u32 nr = (me || nxt) ? RK_STALE : rk[k];
-                    arr[o++] = ((u64)nr << 32) | nt;
+                    const u64 x = v[k + 1];
+                    arr[o] = lp_pack(me ? 256u + lp_rank(x) : lp_tok(x), (me || nxt) ? F20_STALE : lp_rank(x), lp_cl(x));
+                    crr[o] = c[k + 1];
+                    o++;
                 }
             }
             out += tot;
-            carry_par = next_carry;
+            carry_hok = next_hok; carry_par = next_par; carry_last = next_last;
             __syncthreads();
         }
         m = out;
         __syncthreads();
         // probe the stale ranks again; collect the minimum for the next round
-        lmin = TT_RANK_INF;
+        lmin = TT_F20;
         for (u32 i = tid; i < m; i += T) {
-            const u64 v = arr[i];
-            u32 r = (u32)(v >> 32);
-            if (i + 1 >= m) { r = TT_RANK_INF; arr[i] = ((u64)r << 32) | (u32)v; }
-            else if (r == RK_STALE) { r = pair_probe(tab, (u32)v, (u32)arr[i + 1]); arr[i] = ((u64)r << 32) | (u32)v; }
+            const u64 x = arr[i];
+            u32 r = lp_rank(x);
+            if (i + 1 >= m) { r = TT_F20; arr[i] = lp_pack(lp_tok(x), TT_F20, TT_F20); crr[i] = TT_F20; }
+            else if (r == F20_STALE) {
+                const PairInfo p = pair_probe(tab, lp_tok(x), lp_tok(arr[i + 1]));
+                r = f20_encode(p.r);
+                arr[i] = lp_pack(lp_tok(x), r, f20_encode(p.cl)); crr[i] = f20_encode(p.cr);
+            }
             lmin = min(lmin, r);
         }
         __syncthreads();
@@ -553,29 +603,35 @@ __device__ __noinline__ u32 cta_merge_rounds(u64* arr, u32 m, const PairTable& t
 
 constexpr int LONG_SMEM_TOKENS = 4096;                  // long pieces move into shared memory below this many tokens
 
-// Encodes one piece of n > TT_WARP_PIECE_MAX bytes with the whole CTA.  gbuf: n entries of global scratch.
+// Encodes one piece of n > TT_WARP_PIECE_MAX bytes with the whole CTA.  gbuf: n entries of global scratch; the
+// piece's own n words of the staging array serve as the second global array until the ids are staged there.
+// sbuf: LONG_SMEM_TOKENS u64 followed by LONG_SMEM_TOKENS u32.
 __device__ u32 cta_merge_long(const u8* __restrict__ text, u32 a, u32 n, const PairTable& tab, const int32_t* __restrict__ ext_id,
-                              int32_t* __restrict__ stage, u64* gbuf, u64* sbuf /* LONG_SMEM_TOKENS */, u32* s_scr) {
+                              int32_t* __restrict__ stage, u64* gbuf, u64* sbuf, u32* s_scr) {
     const int tid = threadIdx.x, T = blockDim.x;
+    u32* const scr = reinterpret_cast<u32*>(sbuf + LONG_SMEM_TOKENS);
+    u32* const gcr = reinterpret_cast<u32*>(stage + a);
     u64* arr = n <= LONG_SMEM_TOKENS ? sbuf : gbuf;
+    u32* crr = n <= LONG_SMEM_TOKENS ? scr : gcr;
     __syncthreads();
     for (u32 i = tid; i < n; i += T) {
         const u32 t0 = text[a + i];
-        const u32 r = (i + 1 < n) ? __ldg(tab.bytepair + ((t0 << 8) | text[a + i + 1])) : TT_RANK_INF;
-        arr[i] = ((u64)r << 32) | t0;
+        const PairInfo p = (i + 1 < n) ? bytepair_info(tab, t0, text[a + i + 1]) : pair_none();
+        arr[i] = lp_pack(t0, f20_encode(p.r), f20_encode(p.cl));
+        crr[i] = f20_encode(p.cr);
     }
     __syncthreads();
     bool finished;
-    u32 m = cta_merge_rounds(arr, n, tab, s_scr, arr == gbuf ? LONG_SMEM_TOKENS : 0, finished);
+    u32 m = cta_merge_rounds(arr, crr, n, tab, s_scr, arr == gbuf ? LONG_SMEM_TOKENS : 0, finished);
     if (!finished && arr == gbuf) {
         __syncthreads();
-        for (u32 i = tid; i < m; i += T) sbuf[i] = gbuf[i];
+        for (u32 i = tid; i < m; i += T) { sbuf[i] = gbuf[i]; scr[i] = gcr[i]; }
         __syncthreads();
         arr = sbuf;
-        m = cta_merge_rounds(arr, m, tab, s_scr, 0, finished);
+        m = cta_merge_rounds(arr, scr, m, tab, s_scr, 0, finished);
     }
     __syncthreads();
-    for (u32 i = tid; i < m; i += T) stage[a + i] = ext_id[(u32)arr[i]];
+    for (u32 i = tid; i < m; i += T) stage[a + i] = ext_id[lp_tok(arr[i])];
     __syncthreads();
     return m;
 }
@@ -746,10 +802,10 @@ k_lookup(const PieceParams P) {
 // all warps of the GPU stay busy until the queues are empty; no barrier after the long pieces.
 constexpr int MERGE_WARPS = 8;
 constexpr int MERGE_THREADS = MERGE_WARPS * 32;
-constexpr int WARP_SMEM_WORDS = 1024;                 // u64 per warp: two lane-path arrays of 32 x 32 u32, or the 2 x 256 merge buffers
-static_assert(MERGE_WARPS * WARP_SMEM_WORDS >= LONG_SMEM_TOKENS, "the CTA's buffer must hold a long piece");
+constexpr int WARP_SMEM_WORDS = 1024;                 // u64 per warp: two lane-path arrays of 32 x 32 u32, or two copies of four 256-word merge arrays
+static_assert(MERGE_WARPS * WARP_SMEM_WORDS * sizeof(u64) >= LONG_SMEM_TOKENS * (sizeof(u64) + sizeof(u32)), "the CTA's buffer must hold a long piece");
 constexpr size_t MERGE_SMEM_BYTES = (size_t)MERGE_WARPS * WARP_SMEM_WORDS * sizeof(u64);   // dynamic shared memory of k_merge (64 KiB)
-static_assert(WARP_SMEM_WORDS * sizeof(u64) >= 2 * LANE_SLOTS * LANE_MAX * sizeof(u32) && WARP_SMEM_WORDS >= 2 * TT_WARP_PIECE_MAX, "per-warp buffer");
+static_assert(WARP_SMEM_WORDS * sizeof(u64) >= 2 * LANE_SLOTS * LANE_MAX * sizeof(u32) && WARP_SMEM_WORDS * sizeof(u64) >= 2 * 4 * TT_WARP_PIECE_MAX * sizeof(u32), "per-warp buffer");
 
 __global__ void __launch_bounds__(MERGE_THREADS, 3)
 k_merge(const PieceParams P) {
@@ -757,8 +813,8 @@ k_merge(const PieceParams P) {
     __shared__ u32 sc[48];
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
     cudaTriggerProgrammaticLaunchCompletion();               // k_scatter may be placed; it waits for this grid's memory itself
-    grid_prefetch_l2(P.tab.slots, ((size_t)P.tab.mask + 1) * 4 * sizeof(u64));
-    grid_prefetch_l2(P.tab.bytepair, 65536 * sizeof(u32));
+    grid_prefetch_l2(P.tab.slots, ((size_t)P.tab.mask + 1) * 2 * sizeof(uint4));
+    grid_prefetch_l2(P.tab.bytepair, 65536 * sizeof(u64));
     cudaGridDependencySynchronize();                         // the queues are complete from here on
     if (P.hdr->status != 0) return;
     const u8* text = P.base + P.shift;
@@ -781,8 +837,10 @@ k_merge(const PieceParams P) {
         if (e >= nw) break;
         const u64 q = P.q_warp[e];
         const u32 a = (u32)q, i = (u32)(q >> 32) & 2047u, n = (u32)(q >> 43) + 1;
-        const u32 m = n <= 64 ? warp_merge_reg2(text, a, n, P.tab, P.ext_id, P.stage, lane)
-                              : warp_merge_perm<WCH>(wbuf, text, a, n, P.tab, P.ext_id, P.stage, lane);
+        u32* const pbuf = reinterpret_cast<u32*>(wbuf);
+        const u32 m = n <= 64 ? warp_merge_perm<2>(pbuf, text, a, n, P.tab, P.ext_id, P.stage, lane)
+                    : n <= 128 ? warp_merge_perm<4>(pbuf, text, a, n, P.tab, P.ext_id, P.stage, lane)
+                               : warp_merge_perm<WCH>(pbuf, text, a, n, P.tab, P.ext_id, P.stage, lane);
         if (lane == 0) {
             const u32 tile = (u32)(((long long)a + P.shift) / TT_TILE_BYTES);
             P.piece_cnt[tile * TT_TILE_BYTES + i] = 0u - m; atomicAdd(&P.tile_tok[tile], m); atomicAdd(&P.grp_tok[tile >> TT_GROUP_SHIFT], m);

@@ -266,15 +266,10 @@ extern "C" int tt_vocab_load_ex(const tt_merge* merges, size_t n_merges, const i
         internal.emplace(m.result, (u32)(256 + r));
         ext_id[256 + r] = m.result;
     }
-    // pair table: buckets of two 16-byte slots, at most one key per bucket on average
-    u32 nbuckets = 256;
-    while (nbuckets < info.size() + 1) nbuckets <<= 1;
-    u32 log2b = 0;
-    while ((1u << log2b) < nbuckets) log2b++;
-    const size_t cap = 2 * (size_t)nbuckets;
-    std::vector<uint4> slots(cap, make_uint4(0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu));
+    // pair table: two-choice hashing, buckets of two 16-byte slots, at most half of the slots used
     std::vector<u64> bytepair(65536, ~0ull);            // the byte-byte pairs, directly indexed: three 20-bit fields
-    const u32 mask = nbuckets - 1, shift = 32 - log2b;
+    std::vector<uint4> entries;
+    entries.reserve(info.size());
     for (const auto& kv : info) {
         const u64 key = kv.first;
         const Triple& t = kv.second;
@@ -282,14 +277,45 @@ extern "C" int tt_vocab_load_ex(const tt_merge* merges, size_t n_merges, const i
         if (a < 256 && b < 256)
             bytepair[(a << 8) | b] = (u64)f20_encode(t.r) | ((u64)f20_encode(t.cl) << 20) | ((u64)f20_encode(t.cr) << 40);
         const u64 kr = (key << 20) | f20_encode(t.r);
-        u32 h = pair_bucket(key, shift);
-        for (;;) {
-            uint4* bk = &slots[2 * (size_t)h];
-            int k = 0;
-            while (k < 2 && !((bk[k].x & bk[k].y) == 0xFFFFFFFFu)) k++;
-            if (k < 2) { bk[k] = make_uint4((u32)kr, (u32)(kr >> 32), t.cl, t.cr); break; }
-            h = (h + 1) & mask;
+        entries.push_back(make_uint4((u32)kr, (u32)(kr >> 32), t.cl, t.cr));
+    }
+    u32 nbuckets = 256;
+    while (nbuckets < entries.size() + 1) nbuckets <<= 1;
+    std::vector<uint4> slots;
+    u32 mask = 0, shift = 0;
+    size_t cap = 0;
+    for (;; nbuckets <<= 1) {                            // a placement that fails (not seen so far) doubles the table
+        if (nbuckets > (1u << 24)) return TT_ERR_BAD_VOCAB;
+        u32 log2b = 0;
+        while ((1u << log2b) < nbuckets) log2b++;
+        mask = nbuckets - 1; shift = 32 - log2b; cap = 2 * (size_t)nbuckets;
+        slots.assign(cap, make_uint4(0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu));
+        auto is_free = [](const uint4& s) { return (s.x & s.y) == 0xFFFFFFFFu; };
+        auto key_of = [](const uint4& s) { return (((u64)s.y << 32) | s.x) >> 20; };
+        u64 rng = 0x9E3779B97F4A7C15ull;
+        bool ok_all = true;
+        for (const uint4& e0 : entries) {
+            uint4 cur = e0;
+            u32 avoid = 0xFFFFFFFFu;                     // do not move straight back into the bucket just left
+            bool placed = false;
+            for (int iter = 0; iter < 2000 && !placed; iter++) {
+                const u64 key = key_of(cur);
+                const u32 h0 = pair_bucket(key, shift), h1 = pair_bucket_alt(key, shift, h0);
+                for (u32 h : {h0, h1}) {
+                    uint4* bk = &slots[2 * (size_t)h];
+                    for (int k = 0; k < 2 && !placed; k++) if (is_free(bk[k])) { bk[k] = cur; placed = true; }
+                    if (placed) break;
+                }
+                if (placed) break;
+                rng = rng * 6364136223846793005ull + 1442695040888963407ull;
+                const u32 h = (h0 == avoid) ? h1 : (h1 == avoid) ? h0 : ((rng >> 33) & 1 ? h1 : h0);
+                uint4* bk = &slots[2 * (size_t)h + ((rng >> 40) & 1)];
+                const uint4 victim = *bk;
+                *bk = cur; cur = victim; avoid = h;
+            }
+            if (!placed) { ok_all = false; break; }
         }
+        if (ok_all) break;
     }
     tt_vocab* v = new (std::nothrow) tt_vocab();
     if (!v) return TT_ERR_CUDA;

@@ -33,15 +33,15 @@
 #include "tt_common.cuh"
 
 // ---- pair table: (left, right) -> (rank, cl, cr) ----------------------------------------------------------
-// Buckets of two 16-byte slots (one 32-byte sector); slot = { (left << 38) | (right << 20) | rank20, cl, cr }
-// with rank20 = 0xFFFFF for a pair that is no merge itself (it is in the table for its guards).
-// A key lives in its home bucket or, if that is full, in the following ones; a bucket with a free
-// slot ends the search.  Sized for at most one key per bucket on average.
+// Two-choice (cuckoo) hashing over buckets of two 16-byte slots (one 32-byte sector): a key is in one of its
+// two buckets or nowhere, so a probe is two independent sector loads and no chain to walk, hit or miss.
+// slot = { (left << 38) | (right << 20) | rank20, cl, cr } with rank20 = 0xFFFFF for a pair that is no merge
+// itself (it is in the table for its guards); a free slot is all ones.
 struct PairInfo { u32 r, cl, cr; };                   // TT_RANK_INF where there is none
 struct PairTable {
     const uint4* slots;   // 2 * (mask + 1) slots
     const u64* bytepair;  // (byte a, byte b) at [a << 8 | b]: rank20 | cl20 << 20 | cr20 << 40 (0xFFFFF = none): a piece's first probes
-    u32 mask;             // number of buckets - 1 (power of two)
+    u32 mask;             // number of buckets - 1 (power of two, >= 256)
     u32 shift;            // 32 - log2(number of buckets)
 };
 constexpr u32 TT_F20 = 0xFFFFFu;                      // 20-bit field: none
@@ -51,6 +51,12 @@ TT_HD u32 pair_bucket(u64 key, u32 shift) {
     const u32 x = ((u32)key ^ ((u32)(key >> 32) * 0x9E3779B1u)) * 0x85EBCA6Bu;
     return (x ^ (x >> 15)) * 0xC2B2AE35u >> shift;
 }
+TT_HD u32 pair_bucket_alt(u64 key, u32 shift, u32 first) {      // the key's other bucket, never the first one
+    u32 x = ((u32)(key >> TT_ID_BITS) * 0xCC9E2D51u) ^ ((u32)key * 0x1B873593u);
+    x ^= x >> 16; x *= 0x7FEB352Du; x ^= x >> 15;
+    const u32 h = (x * 0x846CA68Bu) >> shift;
+    return h == first ? (first ^ 1u) : h;
+}
 
 __device__ __forceinline__ PairInfo pair_none() { PairInfo p; p.r = p.cl = p.cr = TT_RANK_INF; return p; }
 __device__ __forceinline__ bool pair_match(const uint4 s, u64 key, PairInfo& out) {
@@ -59,19 +65,15 @@ __device__ __forceinline__ bool pair_match(const uint4 s, u64 key, PairInfo& out
     out.r = f20_decode((u32)kr & TT_F20); out.cl = s.z; out.cr = s.w;
     return true;
 }
-__device__ __forceinline__ bool pair_slot_free(const uint4 s) { return (s.x & s.y) == 0xFFFFFFFFu; }
 
 __device__ __forceinline__ PairInfo pair_probe(const PairTable& t, u32 a, u32 b) {
     const u64 key = ((u64)a << TT_ID_BITS) | b;
-    u32 h = pair_bucket(key, t.shift);
+    const u32 h0 = pair_bucket(key, t.shift), h1 = pair_bucket_alt(key, t.shift, h0);
+    const uint4* b0 = t.slots + 2 * (size_t)h0;
+    const uint4* b1 = t.slots + 2 * (size_t)h1;
+    const uint4 x0 = __ldg(b0), y0 = __ldg(b0 + 1), x1 = __ldg(b1), y1 = __ldg(b1 + 1);
     PairInfo out = pair_none();
-    for (u32 n = 0; n <= t.mask; n++) {               // bounded by the number of buckets
-        const uint4* bp = t.slots + 2 * (size_t)h;
-        const uint4 x = __ldg(bp), y = __ldg(bp + 1);
-        if (pair_match(x, key, out) || pair_match(y, key, out)) return out;
-        if (pair_slot_free(y)) return out;            // slots fill from the front: a free last slot ends the chain
-        h = (h + 1) & t.mask;
-    }
+    if (!pair_match(x0, key, out) && !pair_match(y0, key, out) && !pair_match(x1, key, out)) pair_match(y1, key, out);
     return out;
 }
 __device__ __forceinline__ PairInfo bytepair_info(const PairTable& t, u32 a, u32 b) {
@@ -356,20 +358,19 @@ __device__ __forceinline__ u32 warp_merge_perm(u32* buf /* 2 * 4 * 32 E words of
 // threads of the warp hit different banks whatever rows they are at.
 constexpr int LANE_SLOTS = 32;                        // pieces a warp merges at once
 constexpr int LANE_MAX = 32;                          // bytes per piece on this path
-// Two independent probes (ranks only) with both first-bucket loads in flight together.
-__device__ __forceinline__ u32 pair_rank_first(const PairTable& t, const uint4 lo, const uint4 hi, u64 key) {
-    PairInfo p = pair_none();
-    if (pair_match(lo, key, p) || pair_match(hi, key, p)) return p.r;
-    if (pair_slot_free(hi)) return TT_RANK_INF;
-    return pair_probe(t, (u32)(key >> TT_ID_BITS), (u32)(key & (TT_MAX_INTERNAL - 1))).r;     // full bucket: walk the chain
-}
+// Two independent probes (ranks only), all loads in flight together.
 __device__ __forceinline__ void pair_probe2(const PairTable& t, u32 a0, u32 b0, u32 a1, u32 b1, u32& r0, u32& r1) {
     const u64 key0 = ((u64)a0 << TT_ID_BITS) | b0, key1 = ((u64)a1 << TT_ID_BITS) | b1;
-    const uint4* p0 = t.slots + 2 * (size_t)pair_bucket(key0, t.shift);
-    const uint4* p1 = t.slots + 2 * (size_t)pair_bucket(key1, t.shift);
-    const uint4 x0 = __ldg(p0), y0 = __ldg(p0 + 1), x1 = __ldg(p1), y1 = __ldg(p1 + 1);
-    r0 = pair_rank_first(t, x0, y0, key0);
-    r1 = pair_rank_first(t, x1, y1, key1);
+    const u32 h00 = pair_bucket(key0, t.shift), h01 = pair_bucket_alt(key0, t.shift, h00);
+    const u32 h10 = pair_bucket(key1, t.shift), h11 = pair_bucket_alt(key1, t.shift, h10);
+    const uint4* p00 = t.slots + 2 * (size_t)h00; const uint4* p01 = t.slots + 2 * (size_t)h01;
+    const uint4* p10 = t.slots + 2 * (size_t)h10; const uint4* p11 = t.slots + 2 * (size_t)h11;
+    const uint4 a00 = __ldg(p00), a01 = __ldg(p00 + 1), a02 = __ldg(p01), a03 = __ldg(p01 + 1);
+    const uint4 a10 = __ldg(p10), a11 = __ldg(p10 + 1), a12 = __ldg(p11), a13 = __ldg(p11 + 1);
+    PairInfo q0 = pair_none(), q1 = pair_none();
+    if (!pair_match(a00, key0, q0) && !pair_match(a01, key0, q0) && !pair_match(a02, key0, q0)) pair_match(a03, key0, q0);
+    if (!pair_match(a10, key1, q1) && !pair_match(a11, key1, q1) && !pair_match(a12, key1, q1)) pair_match(a13, key1, q1);
+    r0 = q0.r; r1 = q1.r;
 }
 
 // Tokens stay at the byte position where they began; `al` has a bit per position that still holds a
@@ -830,11 +831,11 @@ k_merge(const PieceParams P) {
     if (nl > blockIdx.x) __syncthreads();
     u64* wbuf = s_buf + wid * WARP_SMEM_WORDS;
     const u32 FULL = 0xFFFFFFFFu;
-    for (;;) {                                                    // bounded by the queue length
-        u32 e = 0;
-        if (lane == 0) e = atomicAdd(&P.hdr->t_warp, 1u);
-        e = __shfl_sync(FULL, e, 0);
-        if (e >= nw) break;
+    // Queue entry e belongs to warp e of the grid (numbered across the CTAs first, so that neighbouring entries
+    // run on different SMs); only what lies beyond the grid's warp count is handed out by ticket.  A request's
+    // few unsettled pieces thus start without an atomic round trip.
+    const u32 W = gridDim.x * MERGE_WARPS, gw = (u32)wid * gridDim.x + blockIdx.x;
+    for (u32 e = gw; e < nw;) {                                   // bounded by the queue length
         const u64 q = P.q_warp[e];
         const u32 a = (u32)q, i = (u32)(q >> 32) & 2047u, n = (u32)(q >> 43) + 1;
         u32* const pbuf = reinterpret_cast<u32*>(wbuf);
@@ -845,20 +846,30 @@ k_merge(const PieceParams P) {
             const u32 tile = (u32)(((long long)a + P.shift) / TT_TILE_BYTES);
             P.piece_cnt[tile * TT_TILE_BYTES + i] = 0u - m; atomicAdd(&P.tile_tok[tile], m); atomicAdd(&P.grp_tok[tile >> TT_GROUP_SHIFT], m);
         }
+        if (nw <= W) break;
+        if (lane == 0) e = W + atomicAdd(&P.hdr->t_warp, 1u);
+        e = __shfl_sync(FULL, e, 0);
     }
-    if (ns <= 2u * MERGE_WARPS * gridDim.x) {                     // few: a warp per piece
+#ifndef TT_SHORT_WARP_FACTOR
+#define TT_SHORT_WARP_FACTOR 2u
+#endif
+    if (ns <= TT_SHORT_WARP_FACTOR * W) {                         // few: a warp per piece
+        const u32 nstatic = nw < W ? W - nw : 0u;                 // warps nw .. W-1 take the first entries
+        u32 e = gw >= nw ? gw - nw : ns;
         for (;;) {
-            u32 e = 0;
-            if (lane == 0) e = atomicAdd(&P.hdr->t_short, 1u);
+            if (e < ns) {
+                const u64 q = P.q_short[e];
+                const u32 a = (u32)q, i = (u32)(q >> 32) & 2047u, n = (u32)(q >> 43) + 1;
+                const u32 m = warp_merge_reg(text, a, n, P.tab, P.ext_id, P.stage, lane);
+                if (lane == 0) {
+                    const u32 tile = (u32)(((long long)a + P.shift) / TT_TILE_BYTES);
+                    P.piece_cnt[tile * TT_TILE_BYTES + i] = 0u - m; atomicAdd(&P.tile_tok[tile], m); atomicAdd(&P.grp_tok[tile >> TT_GROUP_SHIFT], m);
+                }
+            }
+            if (ns <= nstatic) break;                             // every entry has its warp
+            if (lane == 0) e = nstatic + atomicAdd(&P.hdr->t_short, 1u);
             e = __shfl_sync(FULL, e, 0);
             if (e >= ns) break;
-            const u64 q = P.q_short[e];
-            const u32 a = (u32)q, i = (u32)(q >> 32) & 2047u, n = (u32)(q >> 43) + 1;
-            const u32 m = warp_merge_reg(text, a, n, P.tab, P.ext_id, P.stage, lane);
-            if (lane == 0) {
-                const u32 tile = (u32)(((long long)a + P.shift) / TT_TILE_BYTES);
-                P.piece_cnt[tile * TT_TILE_BYTES + i] = 0u - m; atomicAdd(&P.tile_tok[tile], m); atomicAdd(&P.grp_tok[tile >> TT_GROUP_SHIFT], m);
-            }
         }
     } else {                                                      // bulk: 32 pieces per warp and step, a thread each
         u32* tok = reinterpret_cast<u32*>(wbuf);

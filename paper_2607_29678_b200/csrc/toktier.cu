@@ -21,6 +21,7 @@
 #include <string>
 #include <unordered_map>
 #include <unordered_set>
+#include <atomic>
 #include <vector>
 #include <algorithm>
 
@@ -54,6 +55,10 @@ struct tt_vocab {
 };
 
 static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// Epoch of a call: tags the status word of the workspace header (see TTHeader).  Never zero, never repeated.
+static std::atomic<unsigned long long> g_epoch{1};
+static inline unsigned long long next_epoch() { return g_epoch.fetch_add(1, std::memory_order_relaxed) & ((1ull << 56) - 1); }
 
 extern "C" const char* tt_strerror(int code) {
     switch (code) {
@@ -177,7 +182,7 @@ static int build_token_table(tt_vocab* v, const tt_merge* merges, size_t n_merge
         Q.base = d_text; Q.shift = 0; Q.hi = (long long)nb; Q.nchunks = (long long)nchunks; Q.ntiles = (int)ntiles;
         Q.startmask = d_mask; Q.tile_first = d_tf; Q.hdr = d_hdr; Q.tab = v->tab;
         Q.toktab.slots = nullptr; Q.toktab.mask = 0; Q.toktab.shift = 0;      // no table yet: every piece is merged
-        Q.longtab = LongTable{}; Q.litstart = nullptr;
+        Q.longtab = LongTable{}; Q.litstart = nullptr; Q.epoch = next_epoch();
         Q.ext_id = v->d_ext_id; Q.piece_cnt = d_cnt; Q.stage = d_stage; Q.pairbuf = nullptr; Q.tile_tok = d_tt; Q.grp_tok = d_gt; Q.q_short = d_qs; Q.q_warp = d_qw; Q.q_long = d_ql;
         const int grid = (int)(ntiles < (size_t)v->sm_count * 8 ? ntiles : (size_t)v->sm_count * 8);
         k_lookup<<<grid, LOOKUP_THREADS>>>(Q);
@@ -411,14 +416,14 @@ static int run_pretok(const tt_vocab* v, const uint8_t* text, size_t len, const 
     P.lo = shift; P.hi = shift + (long long)len;
     P.nchunks = (P.hi + TT_CHUNK - 1) / TT_CHUNK;
     P.ntiles = (int)((P.nchunks + TT_TILE_CHUNKS - 1) / TT_TILE_CHUNKS);
-    P.pattern = v->pattern;
+    P.pattern = v->pattern; P.epoch = next_epoch();
     P.docmask = nullptr; P.litstart = nullptr; P.litin = nullptr;
     P.startmask = w.startmask; P.tile_cnt = w.tile_cnt; P.tile_first = w.tile_first; P.tile_tok = w.tile_tok; P.grp_tok = w.grp_tok; P.want_prefix = piece_off_dst != nullptr; P.hdr = w.hdr;
     P.cls_tables = v->d_cls; P.cls_bytes = v->cls_bytes;
     if (doc_off) {
         CK(cudaMemsetAsync(w.docmask, 0, ((size_t)P.hi / 32 + 4) * sizeof(u32), st));
         const int threads = 256, blocks = (int)((n_docs + 1 + threads - 1) / threads);
-        k_docmask<<<blocks, threads, 0, st>>>((const long long*)doc_off, (int)n_docs, shift, (long long)len, w.docmask, w.hdr);
+        k_docmask<<<blocks, threads, 0, st>>>((const long long*)doc_off, (int)n_docs, shift, (long long)len, w.docmask, w.hdr, P.epoch);
         P.docmask = w.docmask;
     }
     if (literals && !doc_off) {
@@ -450,7 +455,7 @@ static int run_pretok(const tt_vocab* v, const uint8_t* text, size_t len, const 
     k_pretok<<<grid, TT_TILE_CHUNKS, smem, st>>>(P);
     if (piece_off_dst)
         k_compact<<<grid, TT_TILE_CHUNKS, 0, st>>>(w.startmask, w.tile_cnt, P.nchunks, P.ntiles, shift, (long long)len,
-                                                   piece_off_dst, w.hdr);
+                                                   piece_off_dst, w.hdr, P.epoch);
     CK(cudaGetLastError());
     return TT_OK;
 }
@@ -485,13 +490,18 @@ static int encode_impl(const tt_vocab* v, const uint8_t* text, size_t len, const
 #define MARK(i) do { if (ev) cudaEventRecord(ev[i], st); } while (0)
     TTWorkspace w;
     carve(&w, workspace, len, n_docs);
-    CK(cudaMemsetAsync(w.hdr, 0, sizeof(TTHeader), st));
     if (len == 0) {
         if (count_out) CK(cudaMemsetAsync(count_out, 0, sizeof(int64_t), st));
         if (ids_off_out) CK(cudaMemsetAsync(ids_off_out, 0, (n_docs + 1) * sizeof(int64_t), st));
         CK(cudaMemsetAsync(status_out, 0, sizeof(int32_t), st));
         return TT_OK;
     }
+    // The header's counters are zeroed by the first kernel and its status word is tagged with the call's epoch,
+    // so a single request starts with its first kernel.  The passes in front of it (document mask, literals) and
+    // a stream capture (whose replays repeat the epoch) clear the header first.
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(st, &cap) != cudaSuccess) { cudaGetLastError(); cap = cudaStreamCaptureStatusActive; }
+    if (doc_off || literals || cap != cudaStreamCaptureStatusNone) CK(cudaMemsetAsync(w.hdr, 0, sizeof(TTHeader), st));
     MARK(0);
     PretokParams PP;
     int rc = run_pretok(v, text, len, doc_off, n_docs, st, w, nullptr, PP, literals);
@@ -501,7 +511,7 @@ static int encode_impl(const tt_vocab* v, const uint8_t* text, size_t len, const
     const int merge_grid = v->sm_count * 3;                  // all resident CTA slots: a request's unsettled pieces get a warp each
     PieceParams Q;
     Q.base = PP.base; Q.shift = PP.lo; Q.hi = PP.hi; Q.nchunks = PP.nchunks; Q.ntiles = PP.ntiles;
-    Q.startmask = w.startmask; Q.tile_first = w.tile_first; Q.hdr = w.hdr; Q.tab = v->tab; Q.toktab = v->toktab; Q.longtab = v->longtab; Q.litstart = literals ? w.litstart : nullptr;
+    Q.startmask = w.startmask; Q.tile_first = w.tile_first; Q.hdr = w.hdr; Q.tab = v->tab; Q.toktab = v->toktab; Q.longtab = v->longtab; Q.litstart = literals ? w.litstart : nullptr; Q.epoch = PP.epoch;
     Q.ext_id = v->d_ext_id; Q.piece_cnt = w.piece_cnt; Q.stage = w.stage; Q.pairbuf = w.pairbuf; Q.tile_tok = w.tile_tok; Q.grp_tok = w.grp_tok;
     Q.q_short = w.q_short; Q.q_warp = w.q_warp; Q.q_long = w.q_long;
     if (ev) k_lookup<<<tile_grid, LOOKUP_THREADS, 0, st>>>(Q);
@@ -512,7 +522,7 @@ static int encode_impl(const tt_vocab* v, const uint8_t* text, size_t len, const
     MARK(3);
     ScatterParams S;
     S.shift = PP.lo; S.hi = PP.hi; S.nchunks = PP.nchunks; S.ntiles = PP.ntiles; S.startmask = w.startmask;
-    S.tile_first = w.tile_first; S.tile_tok = w.tile_tok; S.grp_tok = w.grp_tok; S.ids_cap = (unsigned long long)ids_cap; S.piece_cnt = w.piece_cnt; S.stage = w.stage; S.hdr = w.hdr;
+    S.tile_first = w.tile_first; S.tile_tok = w.tile_tok; S.grp_tok = w.grp_tok; S.ids_cap = (unsigned long long)ids_cap; S.piece_cnt = w.piece_cnt; S.stage = w.stage; S.hdr = w.hdr; S.epoch = PP.epoch;
     S.ids_out = ids_out; S.count_out = (long long*)count_out; S.status_out = status_out;
     S.docmask = doc_off ? w.docmask : nullptr; S.doc_off = (const long long*)doc_off; S.n_docs = (int)n_docs;
     S.ids_off_out = (long long*)ids_off_out;
@@ -621,9 +631,10 @@ extern "C" int tt_encode_timed(const tt_vocab* v, const uint8_t* text, size_t le
     return rc;
 }
 
-__global__ void k_finish_pretok(const TTHeader* hdr, long long* n_pieces_out, int32_t* status_out) {
-    *status_out = hdr->status;
-    *n_pieces_out = hdr->status ? 0 : (long long)hdr->n_pieces;
+__global__ void k_finish_pretok(const TTHeader* hdr, unsigned long long epoch, long long* n_pieces_out, int32_t* status_out) {
+    const int status = hdr_status(hdr, epoch);
+    *status_out = status;
+    *n_pieces_out = status ? 0 : (long long)hdr->n_pieces;
 }
 
 extern "C" int tt_pretokenize(const tt_vocab* v, const uint8_t* text, size_t len, const int64_t* doc_off, size_t n_docs,
@@ -644,7 +655,7 @@ extern "C" int tt_pretokenize(const tt_vocab* v, const uint8_t* text, size_t len
     PretokParams PP;
     rc = run_pretok(v, text, len, doc_off, n_docs, st, w, (u32*)piece_off_out, PP);
     if (rc != TT_OK) return rc;
-    k_finish_pretok<<<1, 1, 0, st>>>(w.hdr, (long long*)n_pieces_out, status_out);
+    k_finish_pretok<<<1, 1, 0, st>>>(w.hdr, PP.epoch, (long long*)n_pieces_out, status_out);
     CK(cudaGetLastError());
     return TT_OK;
 }

@@ -686,6 +686,7 @@ struct PieceParams {
     const u16* startmask;
     const u32* tile_first;     // offset of the first piece start inside every tile (~0: none)
     TTHeader* hdr;
+    unsigned long long epoch;
     PairTable tab;
     TokTable toktab;
     const u32* litstart;       // literal pass: a piece that begins at such a bit is an added token whose id is staged, or null
@@ -715,7 +716,7 @@ k_lookup(const PieceParams P) {
     cudaTriggerProgrammaticLaunchCompletion();               // the next kernel may be placed; it waits for this grid's memory itself
     if (P.toktab.slots != nullptr) grid_prefetch_l2(P.toktab.slots, ((size_t)P.toktab.mask + 1) * sizeof(TokSlot));
     cudaGridDependencySynchronize();                         // k_pretok's flags and counts are complete from here on
-    const int status = P.hdr->status;                        // looked at after the first tile's flags are in: the loads overlap
+    const int status = hdr_status(P.hdr, P.epoch);           // looked at after the first tile's flags are in: the loads overlap
     const u8* text = P.base + P.shift;
     for (int tile = blockIdx.x; tile < P.ntiles; tile += gridDim.x) {
         const long long c0 = (long long)tile * TT_TILE_CHUNKS;
@@ -817,7 +818,7 @@ k_merge(const PieceParams P) {
     grid_prefetch_l2(P.tab.slots, ((size_t)P.tab.mask + 1) * 2 * sizeof(uint4));
     grid_prefetch_l2(P.tab.bytepair, 65536 * sizeof(u64));
     cudaGridDependencySynchronize();                         // the queues are complete from here on
-    if (P.hdr->status != 0) return;
+    if (hdr_status(P.hdr, P.epoch) != 0) return;
     const u8* text = P.base + P.shift;
     const u32 ns = P.hdr->nq_short, nw = P.hdr->nq_warp, nl = P.hdr->nq_long;
     for (u32 e = blockIdx.x; e < nl; e += gridDim.x) {            // block-uniform
@@ -903,6 +904,7 @@ struct ScatterParams {
     const u32* piece_cnt;
     const int32_t* stage;
     TTHeader* hdr;
+    unsigned long long epoch;
     int32_t* ids_out;
     long long* count_out;
     int32_t* status_out;
@@ -935,7 +937,7 @@ k_scatter(const ScatterParams P) {
     }
     for (int t = (g_lo << TT_GROUP_SHIFT) + tid; t < tile_lo; t += BPE_THREADS) before += P.tile_tok[t];
     cta_sum2_u64(before, total, s_sum);
-    int status = P.hdr->status;
+    int status = hdr_status(P.hdr, P.epoch);
     if (status == 0 && total > P.ids_cap) status = 5;          // TT_ERR_CAPACITY
     if (blockIdx.x == 0 && tid == 0) {
         if (P.status_out) *P.status_out = status;

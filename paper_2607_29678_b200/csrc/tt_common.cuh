@@ -38,14 +38,34 @@ constexpr int TT_WARP_PIECE_MAX = 256;            // bytes; longer pieces take t
 
 // ---- workspace header (device memory, zeroed at the start of every call) --------------------
 struct TTHeader {
-    int status;              // TT_OK or a device-side error code
+    unsigned long long status_tag;   // (epoch of the call << 8) | device-side error code of that call
     u32 pretok_done;         // CTAs that finished the pre-tokenization pass (tt_pretokenize only)
     u32 n_pieces;            // number of pieces found (tt_pretokenize only)
     u32 nq_short, nq_warp, nq_long;   // lengths of the queues of unsettled pieces (k_lookup)
     u32 t_short, t_warp;     // tickets of k_merge: entries handed out so far
-    u32 pad[24];
+    u32 pad[23];
 };
 static_assert(sizeof(TTHeader) == 128, "header layout");
+
+// The status word carries the epoch of the call that wrote it (a process-wide counter, never zero), so a
+// value left by an earlier call -- or whatever an unused workspace holds -- reads as TT_OK and a single
+// request needs no clearing pass before its first kernel.
+#if defined(__CUDACC__)
+__device__ __forceinline__ int hdr_status(const TTHeader* h, unsigned long long epoch) {
+    const unsigned long long t = *reinterpret_cast<const volatile unsigned long long*>(&h->status_tag);
+    return (t >> 8) == epoch ? (int)(t & 0xFF) : 0;
+}
+__device__ __forceinline__ void hdr_set_status(TTHeader* h, unsigned long long epoch, int code) {   // the larger code stays
+    unsigned long long old = *reinterpret_cast<volatile unsigned long long*>(&h->status_tag);
+    for (int tries = 0; tries < 64; tries++) {
+        const int cur = (old >> 8) == epoch ? (int)(old & 0xFF) : 0;
+        if (cur >= code) return;
+        const unsigned long long prev = atomicCAS(&h->status_tag, old, (epoch << 8) | (unsigned long long)code);
+        if (prev == old) return;
+        old = prev;
+    }
+}
+#endif
 
 struct TTWorkspace {
     TTHeader* hdr;

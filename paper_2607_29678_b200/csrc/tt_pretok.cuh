@@ -36,6 +36,7 @@ struct PretokParams {
     u32* grp_tok;            //      of tiles), or null
     int want_prefix;         // turn tile_cnt into its exclusive prefix and count the pieces (tt_pretokenize only)
     TTHeader* hdr;
+    unsigned long long epoch; // of this call (see TTHeader)
     const u8* cls_tables;    // stage1 | stage2 | ascii, contiguous in global memory
     int cls_bytes;
 };

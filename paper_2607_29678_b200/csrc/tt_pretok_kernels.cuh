@@ -46,12 +46,12 @@ __device__ __forceinline__ u32 cta_exscan_u32(u32 v, u32* scratch /* >= 33 */, u
 // Sets the bit of every document's first byte (aligned frame).  Offsets must be ascending, start at
 // 0 and end at the total length; a violation is reported as TT_ERR_ARG in the status word.
 __global__ void k_docmask(const long long* __restrict__ doc_off, int n_docs, long long shift, long long len,
-                          u32* __restrict__ docmask, TTHeader* hdr) {
+                          u32* __restrict__ docmask, TTHeader* hdr, unsigned long long epoch) {
     int d = blockIdx.x * blockDim.x + threadIdx.x;
     if (d > n_docs) return;
     long long o = doc_off[d];
     bool ok = o >= 0 && o <= len && (d == 0 ? o == 0 : o >= doc_off[d - 1]) && (d < n_docs || o == len);
-    if (!ok) { atomicMax(&hdr->status, 1 /* TT_ERR_ARG */); return; }
+    if (!ok) { hdr_set_status(hdr, epoch, 1 /* TT_ERR_ARG */); return; }
     if (d < n_docs && o < len) {
         long long g = o + shift;
         atomicOr(&docmask[g >> 5], 1u << (g & 31));
@@ -205,6 +205,9 @@ k_pretok(const PretokParams P) {
 
     const int tid = threadIdx.x;
     cudaTriggerProgrammaticLaunchCompletion();               // the next kernel may be placed; it waits for this grid's memory itself
+    if (blockIdx.x == 0 && tid == 0) {                       // the counters of the kernels behind this one
+        P.hdr->nq_short = 0; P.hdr->nq_warp = 0; P.hdr->nq_long = 0; P.hdr->t_short = 0; P.hdr->t_warp = 0;
+    }
     // the 128-byte ASCII table is always staged; the two-stage Unicode table only once a tile holds a
     // non-ASCII byte (pattern 1 stages it at once: its sparse matcher may read beyond the tile)
     bool tables_loaded = P.pattern == 1;
@@ -314,7 +317,7 @@ k_pretok(const PretokParams P) {
             if (P.tile_tok) { P.tile_tok[tile] = 0; if ((tile & (TT_GROUP_TILES - 1)) == 0) P.grp_tok[tile >> TT_GROUP_SHIFT] = 0; }
         }
     }
-    if (any_bad) atomicMax(&P.hdr->status, 4 /* TT_ERR_INVALID_UTF8 */);
+    if (any_bad) hdr_set_status(P.hdr, P.epoch, 4 /* TT_ERR_INVALID_UTF8 */);
 
     // the last CTA to finish turns the tile counts into their exclusive prefix (only where the piece list is
     // materialised: the encode chain indexes its pieces per tile and needs no prefix)
@@ -344,9 +347,9 @@ k_pretok(const PretokParams P) {
 // chain does the same per tile in shared memory (tile_pieces in tt_bpe.cuh) and never stores the list.
 __global__ void __launch_bounds__(TT_TILE_CHUNKS)
 k_compact(const u16* __restrict__ startmask, const u32* __restrict__ tile_base, long long nchunks, int ntiles,
-          long long shift, long long len, u32* __restrict__ piece_off, TTHeader* hdr) {
+          long long shift, long long len, u32* __restrict__ piece_off, TTHeader* hdr, unsigned long long epoch) {
     __shared__ u32 sc[40];
-    if (hdr->status != 0) return;
+    if (hdr_status(hdr, epoch) != 0) return;
     for (int tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
         const long long chunk = (long long)tile * TT_TILE_CHUNKS + threadIdx.x;
         u32 m = chunk < nchunks ? startmask[chunk] : 0;

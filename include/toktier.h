@@ -305,6 +305,21 @@ int tt_encode_host(tt_vocab* v, const uint8_t* text, size_t len, int32_t* ids_ou
 int tt_encode_static(const tt_vocab* v, const uint8_t* text, size_t len, void* stream,
                      int32_t* ids_out, size_t ids_cap, int64_t* count_out, int32_t* status_out);
 
+/*
+ * Ranks and merge guards of token pairs as the merge kernels see them, computed on the HOST with no CUDA call
+ * (for checks of the table construction).  Paper Sec. 4.2 merges, per round, the occurrences of the lowest
+ * rank; the kernels also merge, in the same round, every pair that the sequential order is certain to merge:
+ * a pair (x, y) of rank r with left neighbour u and right neighbour w such that r < cl(u, x) and
+ * r <= cr(y, w), where
+ *   cl(u, t) = lowest rank of a merge (X, t) whose left operand X has u on the right spine of its merge tree
+ *              (X = u included),
+ *   cr(t, w) = lowest rank of a merge (t, Y) whose right operand Y has w on the left spine of its merge tree.
+ * left / right: n_pairs caller ids (HOST); out: 3 * n_pairs int64 (HOST): rank, cl, cr of each pair, -1 = none.
+ * Returns TT_ERR_BAD_VOCAB / TT_ERR_ARG like tt_vocab_load.
+ */
+int tt_pair_info_host(const tt_merge* merges, size_t n_merges, const int32_t byte_map[256],
+                      const int32_t* left, const int32_t* right, size_t n_pairs, int64_t* out);
+
 /* Number of class-table entries (0x110000) copied to out (HOST uint8, one class code per code
  * point as the kernels see it): 0 other, 1 mark, 2 whitespace, 3 number, 4 lowercase letter,
  * 5 uppercase/titlecase letter, 6 caseless letter.  For exhaustive table checks. */

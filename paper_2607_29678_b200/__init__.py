@@ -22,7 +22,7 @@ TT_VOCAB_IGNORE_MERGES = 1
 EXPORTS = ["tt_vocab_load", "tt_vocab_load_ex", "tt_vocab_free", "tt_workspace_bytes", "tt_encode", "tt_encode_batch",
            "tt_pretokenize", "tt_encode_timed", "tt_encode_host", "tt_encode_static", "tt_spans", "tt_spans_workspace_bytes", "tt_class_table", "tt_strerror",
            "tt_session_create", "tt_session_free", "tt_session_set_window", "tt_session_append", "tt_session_view", "tt_session_copy", "tt_vocab_add_literals", "tt_encode_added",
-           "tt_verifier_create", "tt_verifier_submit", "tt_verifier_drain", "tt_verifier_get_stats", "tt_verifier_quarantined", "tt_verifier_free"]
+           "tt_pair_info_host", "tt_verifier_create", "tt_verifier_submit", "tt_verifier_drain", "tt_verifier_get_stats", "tt_verifier_quarantined", "tt_verifier_free"]
 
 _lib = None
 REFERENCE_FN = ctypes.CFUNCTYPE(ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p, ctypes.c_size_t,
@@ -117,6 +117,22 @@ def class_table() -> np.ndarray:
     """uint8[0x110000]: the class code the kernels assign to every code point."""
     out = np.empty(0x110000, dtype=np.uint8)
     lib().tt_class_table(out.ctypes.data, out.size)
+    return out
+
+
+def pair_info_host(merges, byte_map, left, right) -> np.ndarray:
+    """tt_pair_info_host: int64[n, 3] (rank, cl, cr; -1 = none) of the pairs (left[i], right[i]); runs on the host."""
+    m = np.ascontiguousarray(merges, dtype=np.int32)
+    bm = np.ascontiguousarray(np.arange(256) if byte_map is None else byte_map, dtype=np.int32)
+    l = np.ascontiguousarray(left, dtype=np.int32)
+    r = np.ascontiguousarray(right, dtype=np.int32)
+    out = np.empty((l.size, 3), dtype=np.int64)
+    L = lib()
+    L.tt_pair_info_host.restype = ctypes.c_int
+    L.tt_pair_info_host.argtypes = [ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
+                                    ctypes.c_size_t, ctypes.c_void_p]
+    _check(L.tt_pair_info_host(m.ctypes.data, m.shape[0], bm.ctypes.data, l.ctypes.data, r.ctypes.data, l.size,
+                               out.ctypes.data), "tt_pair_info_host")
     return out
 
 

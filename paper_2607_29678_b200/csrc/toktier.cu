@@ -228,56 +228,87 @@ extern "C" int tt_vocab_load(const tt_merge* merges, size_t n_merges, const int3
     return tt_vocab_load_ex(merges, n_merges, byte_map, pattern_id, 0u, out);
 }
 
-extern "C" int tt_vocab_load_ex(const tt_merge* merges, size_t n_merges, const int32_t byte_map[256], int pattern_id,
-                                unsigned flags, tt_vocab** out) {
-    if (out) *out = nullptr;
-    if (!out || !byte_map || (n_merges && !merges) || (flags & ~TT_VOCAB_IGNORE_MERGES)) return TT_ERR_ARG;
-    if (pattern_id != TT_PATTERN_CL100K && pattern_id != TT_PATTERN_O200K && pattern_id != TT_PATTERN_CL100K_N1 && pattern_id != TT_PATTERN_SPLIT3) return TT_ERR_ARG;
+// ---- ranks and guards of the pairs (host only, no CUDA call) ---------------------------------------------------
+// For every merge (a, b) of rank r: the pair (a, b) gets the rank; every pair (u, b) with u on the right spine
+// of a's merge tree gets cl <= r (the merge can take b from the left of a token built on u); every pair (a, w)
+// with w on the left spine of b gets cr <= r.  Ranks ascend, so the first value written is the lowest.
+struct PairTriple { u32 r, cl, cr; };
+static int build_pair_info(const tt_merge* merges, size_t n_merges, const int32_t byte_map[256],
+                           std::unordered_map<int32_t, u32>& internal, std::vector<int32_t>& ext_id,
+                           std::unordered_map<u64, PairTriple>& info) {
     if (n_merges > TT_MAX_INTERNAL - 256) return TT_ERR_ARG;
     // external id -> internal id (byte b -> b, result of rank r -> 256 + r)
-    std::unordered_map<int32_t, u32> internal;
-    internal.reserve(512 + 2 * n_merges);
-    std::vector<int32_t> ext_id(256 + n_merges);
+    internal.clear(); internal.reserve(512 + 2 * n_merges);
+    ext_id.assign(256 + n_merges, 0);
     for (int b = 0; b < 256; b++) {
         if (byte_map[b] < 0 || !internal.emplace(byte_map[b], (u32)b).second) return TT_ERR_BAD_VOCAB;   // not injective
         ext_id[b] = byte_map[b];
     }
-    // merges by internal id; children of every merge result
-    std::vector<u32> lch(256 + n_merges, 0xFFFFFFFFu), rch(256 + n_merges, 0xFFFFFFFFu);
-    struct Triple { u32 r, cl, cr; };
-    std::unordered_map<u64, Triple> info;               // key (left << 18 | right) -> rank and guards
-    info.reserve(6 * n_merges + 16);
+    std::vector<u32> lch(256 + n_merges, 0xFFFFFFFFu), rch(256 + n_merges, 0xFFFFFFFFu);   // children of every merge result
+    const PairTriple none{TT_RANK_INF, TT_RANK_INF, TT_RANK_INF};
+    info.clear(); info.reserve(6 * n_merges + 16);
     for (size_t r = 0; r < n_merges; r++) {
         const tt_merge& m = merges[r];
         auto l = internal.find(m.left), rr = internal.find(m.right);
         if (l == internal.end() || rr == internal.end()) return TT_ERR_BAD_VOCAB;      // operand not yet defined
         if (m.result < 0 || internal.count(m.result)) return TT_ERR_BAD_VOCAB;         // result id reused
         const u32 a = l->second, b = rr->second;
-        const u64 key = ((u64)a << TT_ID_BITS) | b;
-        auto ins = info.emplace(key, Triple{TT_RANK_INF, TT_RANK_INF, TT_RANK_INF});
+        auto ins = info.emplace(((u64)a << TT_ID_BITS) | b, none);
         if (ins.first->second.r != TT_RANK_INF) return TT_ERR_BAD_VOCAB;               // duplicate pair
         ins.first->second.r = (u32)r;
         lch[256 + r] = a; rch[256 + r] = b;
-        // guards: the merge (a, b) of rank r can take b from the left after any token on a's right spine, and a
-        // from the right before any token on b's left spine (ranks ascend, so the first entry is the lowest)
         for (u32 u = a; u != 0xFFFFFFFFu; u = u >= 256 ? rch[u] : 0xFFFFFFFFu) {
-            Triple& t = info.emplace(((u64)u << TT_ID_BITS) | b, Triple{TT_RANK_INF, TT_RANK_INF, TT_RANK_INF}).first->second;
+            PairTriple& t = info.emplace(((u64)u << TT_ID_BITS) | b, none).first->second;
             if (t.cl == TT_RANK_INF) t.cl = (u32)r;
         }
         for (u32 w = b; w != 0xFFFFFFFFu; w = w >= 256 ? lch[w] : 0xFFFFFFFFu) {
-            Triple& t = info.emplace(((u64)a << TT_ID_BITS) | w, Triple{TT_RANK_INF, TT_RANK_INF, TT_RANK_INF}).first->second;
+            PairTriple& t = info.emplace(((u64)a << TT_ID_BITS) | w, none).first->second;
             if (t.cr == TT_RANK_INF) t.cr = (u32)r;
         }
         internal.emplace(m.result, (u32)(256 + r));
         ext_id[256 + r] = m.result;
     }
+    return TT_OK;
+}
+
+extern "C" int tt_pair_info_host(const tt_merge* merges, size_t n_merges, const int32_t byte_map[256],
+                                 const int32_t* left, const int32_t* right, size_t n_pairs, int64_t* out) {
+    if (!byte_map || (n_merges && !merges) || (n_pairs && (!left || !right || !out))) return TT_ERR_ARG;
+    std::unordered_map<int32_t, u32> internal;
+    std::vector<int32_t> ext_id;
+    std::unordered_map<u64, PairTriple> info;
+    const int rc = build_pair_info(merges, n_merges, byte_map, internal, ext_id, info);
+    if (rc != TT_OK) return rc;
+    for (size_t i = 0; i < n_pairs; i++) {
+        PairTriple t{TT_RANK_INF, TT_RANK_INF, TT_RANK_INF};
+        auto l = internal.find(left[i]), r = internal.find(right[i]);
+        if (l != internal.end() && r != internal.end()) {
+            auto it = info.find(((u64)l->second << TT_ID_BITS) | r->second);
+            if (it != info.end()) t = it->second;
+        }
+        out[3 * i] = t.r == TT_RANK_INF ? -1 : (int64_t)t.r;
+        out[3 * i + 1] = t.cl == TT_RANK_INF ? -1 : (int64_t)t.cl;
+        out[3 * i + 2] = t.cr == TT_RANK_INF ? -1 : (int64_t)t.cr;
+    }
+    return TT_OK;
+}
+
+extern "C" int tt_vocab_load_ex(const tt_merge* merges, size_t n_merges, const int32_t byte_map[256], int pattern_id,
+                                unsigned flags, tt_vocab** out) {
+    if (out) *out = nullptr;
+    if (!out || !byte_map || (n_merges && !merges) || (flags & ~TT_VOCAB_IGNORE_MERGES)) return TT_ERR_ARG;
+    if (pattern_id != TT_PATTERN_CL100K && pattern_id != TT_PATTERN_O200K && pattern_id != TT_PATTERN_CL100K_N1 && pattern_id != TT_PATTERN_SPLIT3) return TT_ERR_ARG;
+    std::unordered_map<int32_t, u32> internal;
+    std::vector<int32_t> ext_id;
+    std::unordered_map<u64, PairTriple> info;           // key (left << 18 | right) -> rank and guards
+    { const int rc = build_pair_info(merges, n_merges, byte_map, internal, ext_id, info); if (rc != TT_OK) return rc; }
     // pair table: two-choice hashing, buckets of two 16-byte slots, at most half of the slots used
     std::vector<u64> bytepair(65536, ~0ull);            // the byte-byte pairs, directly indexed: three 20-bit fields
     std::vector<uint4> entries;
     entries.reserve(info.size());
     for (const auto& kv : info) {
         const u64 key = kv.first;
-        const Triple& t = kv.second;
+        const PairTriple& t = kv.second;
         const u32 a = (u32)(key >> TT_ID_BITS), b = (u32)(key & (TT_MAX_INTERNAL - 1));
         if (a < 256 && b < 256)
             bytepair[(a << 8) | b] = (u64)f20_encode(t.r) | ((u64)f20_encode(t.cl) << 20) | ((u64)f20_encode(t.cr) << 40);

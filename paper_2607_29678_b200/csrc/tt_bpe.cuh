@@ -704,8 +704,11 @@ struct PieceParams {
 
 __device__ __forceinline__ u64 queue_entry(u32 a, u32 i, u32 n) { return (u64)a | ((u64)i << 32) | ((u64)(n - 1) << 43); }
 
-constexpr int LOOKUP_THREADS = 256;
-__global__ void __launch_bounds__(LOOKUP_THREADS, 6)
+#ifndef TT_LOOKUP_THREADS_DEF
+#define TT_LOOKUP_THREADS_DEF 256
+#endif
+constexpr int LOOKUP_THREADS = TT_LOOKUP_THREADS_DEF;
+__global__ void __launch_bounds__(LOOKUP_THREADS, 1536 / LOOKUP_THREADS)
 k_lookup(const PieceParams P) {
     __shared__ TilePieces tp;
     __shared__ u16 s_short[TILE_MAX_PIECES];                  // short misses from the front, long pieces from the back
@@ -776,12 +779,11 @@ k_lookup(const PieceParams P) {
         if ((tid & 31) == 0 && wsum) atomicAdd(&s_total, wsum);
         __syncthreads();
         const u32 ns = s_ns, nw = s_nw, nl = s_nl;
-        if (tid == 0) {
-            if (s_total) { atomicAdd(&P.tile_tok[tile], s_total); atomicAdd(&P.grp_tok[tile >> TT_GROUP_SHIFT], s_total); }
-            if (ns) s_bs = atomicAdd(&P.hdr->nq_short, ns);
-            if (nw) s_bw = atomicAdd(&P.hdr->nq_warp, nw);
-            if (nl) s_bl = atomicAdd(&P.hdr->nq_long, nl);
-        }
+        // the three reservations wait for their answers side by side, in different warps
+        if (tid == 0 && ns) s_bs = atomicAdd(&P.hdr->nq_short, ns);
+        if (tid == 32 && nw) s_bw = atomicAdd(&P.hdr->nq_warp, nw);
+        if (tid == 64 && nl) s_bl = atomicAdd(&P.hdr->nq_long, nl);
+        if (tid == 96 && s_total) { atomicAdd(&P.tile_tok[tile], s_total); atomicAdd(&P.grp_tok[tile >> TT_GROUP_SHIFT], s_total); }
         if (ns | nw | nl) {                                       // block-uniform
             __syncthreads();
             for (u32 e = tid; e < ns + nw + nl; e += LOOKUP_THREADS) {

@@ -462,7 +462,7 @@ def vocab_table_bytes(n_merges: int) -> int:
 
 # DRAM bytes (read + write) per launch from the committed ncu capture of the C3 request
 # (profiles/c3_1M_request_kernels.md).
-NCU_TRAFFIC = {"merge": 5_200_896, "lookup": 9_557_504, "pretok": 1_090_304, "scatter": 1_237_760}
+NCU_TRAFFIC = {"merge": 9_463_296, "lookup": 9_557_760, "pretok": 1_091_328, "scatter": 1_235_712}
 
 
 def ncu_traffic(kernel: str):

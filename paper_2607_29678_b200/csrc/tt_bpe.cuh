@@ -183,6 +183,17 @@ constexpr int BPE_WARPS = 8;                          // warps per CTA of the pi
 constexpr int BPE_THREADS = BPE_WARPS * 32;           // = pieces per CTA iteration
 constexpr int WCH = TT_WARP_PIECE_MAX / 32;           // 32-token chunks per piece
 
+// Position of the (j + 1)-th set bit of mask (a value >= 32 where there is none): five halving steps.
+__device__ __forceinline__ u32 select_bit(u32 mask, u32 j) {
+    u32 pos = 0, c;
+    c = __popc(mask & 0xFFFFu);          if (j >= c) { pos = 16; j -= c; }
+    c = __popc((mask >> pos) & 0xFFu);   if (j >= c) { pos += 8; j -= c; }
+    c = __popc((mask >> pos) & 0xFu);    if (j >= c) { pos += 4; j -= c; }
+    c = __popc((mask >> pos) & 0x3u);    if (j >= c) { pos += 2; j -= c; }
+    c = (mask >> pos) & 1u;              if (j >= c) { pos += 1; j -= c; }
+    return ((mask >> (pos & 31)) & 1u) && j == 0 && pos < 32 ? pos : 32u;
+}
+
 // ---- warp merge rounds with at most 32 tokens: one token per lane, no shared memory -----------------------
 // t = token of position `lane`, p = (rank, cl, cr) of the pair (lane, lane + 1) or none, m = token count.
 // Runs rounds to the fixpoint, stages the tokens (caller's ids) at stage[a ...] and returns their count.
@@ -217,7 +228,7 @@ __device__ __forceinline__ u32 warp_merge_reg_rounds(u32 t, PairInfo p, u32 m, u
             src = (u32)lane + ((u32)lane > (u32)(__ffs(sel) - 1) ? 1u : 0u);
         } else {
             const u32 surv = ~(sel << 1) & (m >= 32 ? FULL : ((1u << m) - 1));
-            src = __fns(surv, 0, lane + 1);
+            src = select_bit(surv, (u32)lane);
         }
         t = __shfl_sync(FULL, nt, src & 31);
         r = __shfl_sync(FULL, nr, src & 31);

@@ -813,7 +813,8 @@ k_lookup(const PieceParams P) {
 // Long pieces (> 256 bytes) first, a CTA each.  Then every warp works on its own: it takes the pieces of
 // 33..256 bytes one at a time (the longest chains, so they start first), then the pieces of <= 32 bytes --
 // one at a time with the tokens in registers if the whole call has few of them (the shortest chain per piece:
-// a request's latency is its longest chain), else 32 at a time, a thread per piece.  Tickets are global, so
+// a request's latency is its longest chain), else 32 at a time, a thread per piece.  A queue entry within the
+// grid's warp count belongs to the warp of that index; entries beyond it are handed out by global tickets, so
 // all warps of the GPU stay busy until the queues are empty; no barrier after the long pieces.
 constexpr int MERGE_WARPS = 8;
 constexpr int MERGE_THREADS = MERGE_WARPS * 32;

@@ -36,13 +36,13 @@ constexpr u32 TT_RANK_INF = 0xFFFFFFFFu;
 constexpr u64 TT_SLOT_EMPTY = ~0ull;              // pair-table slot: (left << 38) | (right << 20) | rank
 constexpr int TT_WARP_PIECE_MAX = 256;            // bytes; longer pieces take the block-cooperative path
 
-// ---- workspace header (device memory, zeroed at the start of every call) --------------------
+// ---- workspace header (device memory; counters zeroed by the call's first kernel or a memset) ----
 struct TTHeader {
     unsigned long long status_tag;   // (epoch of the call << 8) | device-side error code of that call
     u32 pretok_done;         // CTAs that finished the pre-tokenization pass (tt_pretokenize only)
     u32 n_pieces;            // number of pieces found (tt_pretokenize only)
     u32 nq_short, nq_warp, nq_long;   // lengths of the queues of unsettled pieces (k_lookup)
-    u32 t_short, t_warp;     // tickets of k_merge: entries handed out so far
+    u32 t_short, t_warp;     // tickets of k_merge: queue entries handed out beyond the ones that warps own by index
     u32 pad[23];
 };
 static_assert(sizeof(TTHeader) == 128, "header layout");

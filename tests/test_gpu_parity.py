@@ -537,6 +537,54 @@ def test_host_entry_point_with_pinned_buffers():
     assert err.value.code == tt.TT_ERR_CAPACITY
 
 
+def test_host_entry_point_pinned_views_all_patterns():
+    """Pinned caller buffers as views into a larger pinned allocation: several byte alignments, a text that ends
+    exactly at the end of the allocation and one that starts at its first byte, every pattern, CJK and adversarial
+    runs, changing contents of the same buffer, invalid UTF-8."""
+    import torch
+    import paper_2607_29678_b200 as tt
+    merges, byte_map = wl.load_vocab(wl.CONFIGS["C4"])
+    cv = cpu_vocab("C4")
+    body = wl.generate(wl.KIND_TRANSCRIPT_ADV, 4242, 150_000)
+
+    def cut(n):                                                   # the largest length <= n that ends on a character boundary
+        while n < body.size and (body[n] & 0xC0) == 0x80:
+            n -= 1
+        return n
+
+    pinned = torch.empty(body.size + 64, dtype=torch.uint8).pin_memory()
+    ids = torch.empty(body.size + 64, dtype=torch.int32).pin_memory()
+    for pattern in (0, 1, 2, 3):
+        gv = tt.Vocab(merges, byte_map, pattern)
+        for off in (0, 1, 5, 15, 16, 33):
+            n_text = cut(body.size - 7) if off == 5 else body.size
+            view = pinned[off:off + n_text]
+            view.copy_(torch.from_numpy(body[:n_text].copy()))
+            want, _ = cv.encode(body[:n_text], pattern, nthreads=8)
+            n = gv.encode_host_into(view, ids)
+            assert n == want.size and np.array_equal(ids[:n].numpy(), want), (pattern, off)
+        # the text ends with the allocation; then a short text at its very start
+        n_tail = cut(5000)
+        tail = pinned[pinned.numel() - n_tail:]
+        tail.copy_(torch.from_numpy(body[:n_tail].copy()))
+        want, _ = cv.encode(body[:n_tail], pattern, nthreads=2)
+        n = gv.encode_host_into(tail, ids)
+        assert n == want.size and np.array_equal(ids[:n].numpy(), want)
+        head = pinned[:3]
+        head.copy_(torch.from_numpy(np.frombuffer(b"a b", dtype=np.uint8).copy()))
+        want, _ = cv.encode(np.frombuffer(b"a b", dtype=np.uint8), pattern)
+        n = gv.encode_host_into(head, ids)
+        assert n == want.size and np.array_equal(ids[:n].numpy(), want)
+    # invalid UTF-8 in pinned text is reported, not tokenized
+    gv = tt.Vocab(merges, byte_map, 0)
+    bad = pinned[:cut(1000)]
+    bad.copy_(torch.from_numpy(body[:cut(1000)].copy()))
+    bad[500] = 0xFF
+    with pytest.raises(tt.TokTierError) as err:
+        gv.encode_host_into(bad, ids)
+    assert err.value.code == tt.TT_ERR_INVALID_UTF8
+
+
 def test_repeated_calls_on_the_same_buffers():
     """The same buffers used for call after call: the results must follow the current contents of the text
     buffer, another length in the same buffers must work, and many buffer sets in rotation too."""

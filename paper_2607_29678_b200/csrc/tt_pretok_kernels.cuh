@@ -263,9 +263,10 @@ k_pretok(const PretokParams P) {
         __syncthreads();
         if (P.pattern == 1) {                                          // sure starts / unresolved constructs per slot
             u32 su, ha;
-            tt_sure_hard(sm, tid + TT_LOW_HALO, su, ha);
+            const long long gs0 = (c_first - TT_LOW_HALO) * TT_CHUNK;       // byte 0 of slot 0
+            tt_sure_hard(sm, tid + TT_LOW_HALO, su, ha, P.base, gs0, P.hi);
             sm[F_SURE][tid + TT_LOW_HALO] = (u16)su; sm[F_HARD][tid + TT_LOW_HALO] = (u16)ha;
-            if (tid >= 1 && tid < TT_LOW_HALO) { tt_sure_hard(sm, tid, su, ha); sm[F_SURE][tid] = (u16)su; sm[F_HARD][tid] = (u16)ha; }
+            if (tid >= 1 && tid < TT_LOW_HALO) { tt_sure_hard(sm, tid, su, ha, P.base, gs0, P.hi); sm[F_SURE][tid] = (u16)su; sm[F_HARD][tid] = (u16)ha; }
             __syncthreads();
         }
         // phase B: evaluate the piece-start predicate

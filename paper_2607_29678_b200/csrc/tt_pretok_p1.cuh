@@ -184,7 +184,9 @@ TT_HD ChunkDoc tt_load_slot(const u16 (*sm)[TT_SLOTS], int s) {
 }
 // p = previous chunk, c = the chunk, n = next chunk
 // upcl: the unresolved constructs of the second kind (upper-case letter after a caseless letter), a subset of hard
-TT_HD void tt_sure_hard_cm(const ChunkDoc& p, const ChunkDoc& c, const ChunkDoc& n, u32& sure, u32& hard, u32& upcl) {
+// apch: the unresolved constructs of the third kind (apostrophe between letters with another apostrophe two or three
+// bytes before it), a subset of hard
+TT_HD void tt_sure_hard_cm(const ChunkDoc& p, const ChunkDoc& c, const ChunkDoc& n, u32& sure, u32& hard, u32& upcl, u32& apch) {
     // 20-bit frame: bits 0..2 = last three bytes of the previous chunk, bits 3..18 = the chunk, bit 19 = first byte of the next
 #define FR(x) ((((u32)p.x) >> 13) | (((u32)c.x) << 3) | ((((u32)n.x) & 1u) << 19))
     const u32 lead = FR(m.lead), D = FR(doc);
@@ -201,15 +203,17 @@ TT_HD void tt_sure_hard_cm(const ChunkDoc& p, const ChunkDoc& c, const ChunkDoc&
     // an apostrophe between letters is a possible contraction suffix; it is decided locally unless another
     // apostrophe two or three bytes before it may have consumed the letter in front of it
     const u32 h2 = FR(m.upp) & pCl;
-    const u32 h = FR(m.mark) | h2 | (AP & pLr & nLr & ((AP << 2) | (AP << 3)));
+    const u32 h3 = AP & pLr & nLr & ((AP << 2) | (AP << 3));
+    const u32 h = FR(m.mark) | h2 | h3;
 #undef FR
     sure = ((cs & lead) >> 3) & 0xFFFFu;
     hard = ((h & lead) >> 3) & 0xFFFFu;
     upcl = ((h2 & lead) >> 3) & 0xFFFFu;
+    apch = ((h3 & lead) >> 3) & 0xFFFFu;
 }
 TT_HD void tt_sure_hard_cm(const ChunkDoc& p, const ChunkDoc& c, const ChunkDoc& n, u32& sure, u32& hard) {
-    u32 upcl;
-    tt_sure_hard_cm(p, c, n, sure, hard, upcl);
+    u32 upcl, apch;
+    tt_sure_hard_cm(p, c, n, sure, hard, upcl, apch);
 }
 
 // An upper-case letter (bit i of slot s) that follows a caseless letter, decided from the class masks of
@@ -252,16 +256,64 @@ TT_HD int tt_resolve_upper_after_caseless(const u16 (*sm)[TT_SLOTS], int s, int 
     }
 }
 
-// Valid for 1 <= s <= TT_SLOTS - 2 (needs the neighbouring slots).  Unresolved constructs of the second
-// kind that the tile's masks decide leave `hard`; those that start a piece join `sure`.
-TT_HD void tt_sure_hard(const u16 (*sm)[TT_SLOTS], int s, u32& sure, u32& hard) {
-    u32 upcl;
-    tt_sure_hard_cm(tt_load_slot(sm, s - 1), tt_load_slot(sm, s), tt_load_slot(sm, s + 1), sure, hard, upcl);
+// An apostrophe between letters (tile position pos = slot * 16 + bit) that has another apostrophe two or three bytes
+// before it: is it the start of a contraction suffix of the word in front of it?  1 = yes, 0 = no, -1 = left to the
+// sparse path.  A contraction suffix ends its match, so the letter in front of this apostrophe belongs to a word
+// body -- and the apostrophe can open a suffix -- unless that letter is itself the last letter of a suffix opened by
+// the apostrophe before.  Whether that one opened a suffix hangs on the one before it in the same way: the chain of
+// apostrophes is followed to its head (an apostrophe with none two or three bytes before it, or one that is not
+// between letters) and decided from there.  base0 / g0: the text and the position of byte 0 of slot 0.
+TT_HD int tt_resolve_chained_apostrophe(const u16 (*sm)[TT_SLOTS], int pos, const u8* base, long long g0, long long hi) {
+    const int K = 8;
+    int chain[K];
+    int n = 0;
+#define MB(f, q) ((sm[f][(q) >> 4] >> ((q) & 15)) & 1u)
+#define LETTER(q) (MB(F_LOW, q) | MB(F_UPP, q) | MB(F_CLESS, q))
+#define CAND(q) (MB(F_AP, q) && LETTER((q) - 1) && !MB(F_DOC, q) && LETTER((q) + 1) && !MB(F_DOC, (q) + 1))
+    int cur = pos;
+    for (;;) {
+        if (n == K) return -1;
+        if (cur < 4 || cur + 2 >= TT_SLOTS * 16) return -1;       // the look leaves the tile's window
+        chain[n++] = cur;
+        if (!CAND(cur)) break;                                      // opens no suffix whatever precedes it: a head
+        int prev = -1;
+        if (MB(F_AP, cur - 2) && !MB(F_DOC, cur - 1) && !MB(F_DOC, cur)) prev = cur - 2;
+        else if (MB(F_AP, cur - 3) && !MB(F_DOC, cur - 2) && !MB(F_DOC, cur - 1) && !MB(F_DOC, cur)) prev = cur - 3;
+        if (prev < 0) break;                                        // nothing before it can have taken its letter: a head
+        cur = prev;
+    }
+    bool consumed = false;                                          // the letter before the apostrophe ends a suffix
+    for (int k = n - 1;; k--) {
+        const int q = chain[k];
+        int cl = 0;
+        if (CAND(q) && !consumed) {
+            const long long g = g0 + q;
+            const u32 b1 = (g + 1 < hi) ? base[g + 1] : 0, b2 = (g + 2 < hi && !MB(F_DOC, q + 2)) ? base[g + 2] : 0;
+            cl = tt_contraction_len(b1, b2);
+        }
+        if (k == 0) return cl ? 1 : 0;
+        consumed = cl != 0 && q + cl == chain[k - 1];
+    }
+#undef CAND
+#undef LETTER
+#undef MB
+}
+
+// Valid for 1 <= s <= TT_SLOTS - 2 (needs the neighbouring slots).  Unresolved constructs of the second and third
+// kind that the tile's masks decide leave `hard`; upper-case letters that start a piece join `sure`.
+TT_HD void tt_sure_hard(const u16 (*sm)[TT_SLOTS], int s, u32& sure, u32& hard, const u8* base, long long g0, long long hi) {
+    u32 upcl, apch;
+    tt_sure_hard_cm(tt_load_slot(sm, s - 1), tt_load_slot(sm, s), tt_load_slot(sm, s + 1), sure, hard, upcl, apch);
     while (upcl) {
         const int i = tt_lobit(upcl);
         upcl &= upcl - 1;
         const int r = tt_resolve_upper_after_caseless(sm, s, i);
         if (r >= 0) { hard &= ~(1u << i); sure |= (u32)r << i; }
+    }
+    while (apch) {
+        const int i = tt_lobit(apch);
+        apch &= apch - 1;
+        if (tt_resolve_chained_apostrophe(sm, s * 16 + i, base, g0, hi) >= 0) hard &= ~(1u << i);
     }
 }
 
@@ -369,15 +421,19 @@ TT_HD u32 tt_eval_chunk_p1(const u16 (*sm)[TT_SLOTS], int slot, const SeqCtx& C,
     S |= upp & lead & PREV(low);                          // case boundary: upper after lower
     // ---- contraction suffix: an apostrophe between letters with a valid suffix ('s 't 'm 'd 're 've 'll, ASCII,
     // any case) belongs to the word before it; the suffix letters start nothing and the next letter starts a piece.
-    // (Apostrophes with another apostrophe 2-3 bytes before them are left to the sparse path.)
+    // (An apostrophe with another one 2-3 bytes before it is decided along the chain of such apostrophes.)
     {
-        u64 ca = AP & PREV(Lr) & ((Lr >> 1) & ~(D >> 1)) & ~((AP << 2) | (AP << 3)) & (0x7FFFFull << 29);   // own bytes -3 .. +15
+        u64 ca = AP & PREV(Lr) & ((Lr >> 1) & ~(D >> 1)) & (0x7FFFFull << 29);   // own bytes -3 .. +15
+        const u64 chained = (AP << 2) | (AP << 3);
         while (ca) {
             const int q = (u32)ca ? tt_lobit((u32)ca) : 32 + tt_lobit((u32)(ca >> 32));
             ca &= ca - 1;
             const long long g = g0 + (q - 32);
             const u32 b1 = (g + 1 < C.hi) ? C.base[g + 1] : 0, b2 = (g + 2 < C.hi) ? C.base[g + 2] : 0;
             int cl = tt_contraction_len(b1, (D >> (q + 2)) & 1 ? 0u : b2);
+            // an apostrophe shortly before this one may have taken the letter in front of it: decided along the chain,
+            // or (result -1) left to the sparse path, which then overrides these bits
+            if (cl && ((chained >> q) & 1) && tt_resolve_chained_apostrophe(sm, (slot - 2) * 16 + q, C.base, g0 - (long long)slot * 16, C.hi) != 1) cl = 0;
             if (cl) {
                 const u64 span = ((1ull << cl) - 1) << q;                 // apostrophe and suffix letters
                 S &= ~span;

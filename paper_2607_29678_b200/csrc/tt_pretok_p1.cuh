@@ -495,7 +495,9 @@ TT_HD u32 tt_eval_chunk_p1(const u16 (*sm)[TT_SLOTS], int slot, const SeqCtx& C,
         u32 carry = 0;
         bool open;
         carry = tt_walk_back_dirty(sm, slot - 2, open);
-        if (open) { if (have_tc) carry = tc.dirty_before; else need |= NEED_H; }
+        // (nothing lies before the text: its first tile needs no look beyond the window)
+        const bool at_text_start = C.lo >= g0 - (long long)(slot - 1) * TT_CHUNK;
+        if (open && !at_text_start) { if (have_tc) carry = tc.dirty_before; else need |= NEED_H; }
         const u64 sure2 = sure & ~0xFFFFull;
         u64 F = (hard & ~0xFFFFull) | (((u64)carry << 16) & ~sure2);
         u64 R = ~sure2;
@@ -521,6 +523,7 @@ TT_HD u32 tt_eval_chunk_p1(const u16 (*sm)[TT_SLOTS], int slot, const SeqCtx& C,
         } else {
             int pos = tt_walk_back_sure(sm, slot - 2);
             if (pos >= 0) from = g0 + ((long long)pos - (long long)slot * 16);
+            else if (C.lo >= g0 - (long long)(slot - 1) * TT_CHUNK) from = C.lo;      // the text start is a sure start
             else if (have_tc) from = tc.sure_before;
             else need |= NEED_C;
         }

@@ -626,3 +626,30 @@ def test_repeated_calls_on_the_same_buffers():
         for d, b in sets:
             k = int(b["count"].item())
             assert np.array_equal(b["ids"][:k].cpu().numpy(), want[0])
+
+
+@pytest.mark.parametrize("pattern", [0, 1])
+def test_apostrophe_chains(pattern):
+    """Contraction suffixes in chains (x's's, 'it's', he'll've, quotes around words): pattern 1 decides them along
+    the chain of apostrophes, pattern 0 treats every suffix as a piece of its own.  Random strings of such atoms
+    as one text (several alignments) and as a batch of documents; long chains beyond the resolver's bound."""
+    rng = random.Random(31 + pattern)
+    gv, cv = gpu_vocab("C4", pattern=pattern), cpu_vocab("C4")
+    atoms = ["'", "'s", "'t", "'re", "'ve", "'ll", "'LL", "'S", "'d", "'m", "a", "x", "It", "word", "中", "é", "É", "Ab", "AB",
+             " ", "  ", "\n", "1", ",", ".", "''", "\"", "́", "he", "don", "I"]
+    docs = []
+    for k in range(600):
+        docs.append("".join(rng.choice(atoms) for _ in range(rng.randrange(0, rng.choice([5, 60, 600])))).encode())
+    for k in range(1, 24):
+        for unit in ("'s", "'re", "x's", "'ll", "a'"):
+            docs.append(("x" + unit * k + "y").encode())
+    text = np.frombuffer(b"".join(docs), dtype=np.uint8)
+    off = np.zeros(len(docs) + 1, dtype=np.int64)
+    off[1:] = np.cumsum([len(d) for d in docs])
+    ids, ioff, status = gpu_encode_batch(gv, text, off)
+    want, woff = cv.encode_batch(text, off, pattern, nthreads=8)
+    assert status == 0 and np.array_equal(ioff, woff) and np.array_equal(ids, want)
+    want1, _ = cv.encode(text, pattern, nthreads=8)
+    for offset in (0, 7, 13):
+        ids1, status1 = gpu_encode(gv, text, offset=offset)
+        assert status1 == 0 and np.array_equal(ids1, want1)

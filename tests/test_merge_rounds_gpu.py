@@ -45,3 +45,15 @@ def test_dense_vocabularies_all_length_classes(seed):
         ids, status = gpu_encode(gv, text, offset=rng.randrange(16))
         want, _ = cv.encode(text, pattern, nthreads=8)
         assert status == 0 and np.array_equal(ids, want), (seed, len(s), s[:60])
+
+
+def test_no_merges_and_one_merge():
+    """Degenerate vocabularies: without merges every byte is a token; with one merge only that pair combines."""
+    import paper_2607_29678_b200 as tt
+    text = np.frombuffer(("aab aaaa b " * 300 + "a" * 5000).encode(), dtype=np.uint8)
+    for merges in (np.zeros((0, 3), dtype=np.int32), np.array([[ord("a"), ord("a"), 256]], dtype=np.int32)):
+        gv, cv = tt.Vocab(merges, None, 0), oracle.Vocab(merges, None)
+        ids, status = gpu_encode(gv, text)
+        want, _ = cv.encode(text, 0)
+        assert status == 0 and np.array_equal(ids, want)
+    assert int((ids == 256).sum()) > 2500

@@ -403,6 +403,29 @@ def main():
             dist.destroy_process_group()
         return
 
+    # ---- pattern variants: the same 1M-char transcript text under the other front ends (L2 flushed, CUDA events) ----
+    variants = None
+    if not args.no_batch:
+        variants = {}
+        vtext = torch.from_numpy(wl.generate(wl.KIND_TRANSCRIPT, 99, cfg.n_chars)).cuda()
+        for name, vocab_cfg, pattern in (("o200k_style", "C4", tt.TT_PATTERN_O200K), ("single_digit", "C3", tt.TT_PATTERN_CL100K_N1),
+                                         ("three_splitter", "C3", tt.TT_PATTERN_SPLIT3)):
+            vm, vb = wl.load_vocab(wl.CONFIGS[vocab_cfg])
+            vv = tt.Vocab(vm, vb, pattern)
+            vbufs = vv.alloc(vtext.numel())
+            ts = []
+            for k in range(3 + 12):
+                flush_l2(); torch.cuda.synchronize()
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(stream); vv.encode(vtext, vbufs); b.record(stream)
+                torch.cuda.synchronize()
+                if k >= 3:
+                    ts.append(a.elapsed_time(b))
+            assert int(vbufs["status"].item()) == 0
+            variants[name] = {"cold_p50_ms": round(pct(ts, 0.5), 4), "merges": int(vm.shape[0]), "tokens": int(vbufs["count"].item())}
+            del vv, vbufs
+        variants["what"] = "tt_encode of one 1,000,000-char transcript under the other pattern ids (o200k-style with its own 199,744-merge vocabulary)"
+
     # ---- roofline of the dominant kernel: algorithmic bytes of one request / its device time ----
     peak, peak_kind = measured_peak()
     nbytes = int(np.mean([t.size for t in host_texts]))
@@ -444,6 +467,7 @@ def main():
                           "spliced_on_first_window": first_window,
                           "what": "tt_session_append of 1,500 chars (host bytes in, wall clock, synchronous) to a session holding "
                                   "~1M chars; ids checked against a full tokenization; the paper reports 1.23 ms P50 at 1M context"},
+        "pattern_variants": variants,
         "roofline": roofline,
         "cpu_baseline": cpu,
         "clocks": clocks,

@@ -186,7 +186,7 @@ static int build_token_table(tt_vocab* v, const tt_merge* merges, size_t n_merge
         Q.ext_id = v->d_ext_id; Q.piece_cnt = d_cnt; Q.stage = d_stage; Q.pairbuf = nullptr; Q.tile_tok = d_tt; Q.grp_tok = d_gt; Q.q_short = d_qs; Q.q_warp = d_qw; Q.q_long = d_ql;
         const int grid = (int)(ntiles < (size_t)v->sm_count * 8 ? ntiles : (size_t)v->sm_count * 8);
         k_lookup<<<grid, LOOKUP_THREADS>>>(Q);
-        k_merge<<<v->sm_count * 3, MERGE_THREADS, MERGE_SMEM_BYTES>>>(Q);
+        k_merge<<<v->sm_count * MERGE_CTAS_PER_SM, MERGE_THREADS, MERGE_SMEM_BYTES>>>(Q);
         ok = cudaGetLastError() == cudaSuccess && cudaDeviceSynchronize() == cudaSuccess;
     }
     ok = ok && cudaMemcpy(cnt.data(), d_cnt, cnt.size() * sizeof(u32), cudaMemcpyDeviceToHost) == cudaSuccess;
@@ -539,7 +539,7 @@ static int encode_impl(const tt_vocab* v, const uint8_t* text, size_t len, const
     if (rc != TT_OK) return rc;
     MARK(1);
     const int tile_grid = PP.ntiles < v->sm_count * 8 ? PP.ntiles : v->sm_count * 8;
-    const int merge_grid = v->sm_count * 3;                  // all resident CTA slots: a request's unsettled pieces get a warp each
+    const int merge_grid = v->sm_count * MERGE_CTAS_PER_SM;                  // all resident CTA slots: a request's unsettled pieces get a warp each
     PieceParams Q;
     Q.base = PP.base; Q.shift = PP.lo; Q.hi = PP.hi; Q.nchunks = PP.nchunks; Q.ntiles = PP.ntiles;
     Q.startmask = w.startmask; Q.tile_first = w.tile_first; Q.hdr = w.hdr; Q.tab = v->tab; Q.toktab = v->toktab; Q.longtab = v->longtab; Q.litstart = literals ? w.litstart : nullptr; Q.epoch = PP.epoch;

@@ -823,7 +823,11 @@ static_assert(MERGE_WARPS * WARP_SMEM_WORDS * sizeof(u64) >= LONG_SMEM_TOKENS * 
 constexpr size_t MERGE_SMEM_BYTES = (size_t)MERGE_WARPS * WARP_SMEM_WORDS * sizeof(u64);   // dynamic shared memory of k_merge (64 KiB)
 static_assert(WARP_SMEM_WORDS * sizeof(u64) >= 2 * LANE_SLOTS * LANE_MAX * sizeof(u32) && WARP_SMEM_WORDS * sizeof(u64) >= 2 * 4 * TT_WARP_PIECE_MAX * sizeof(u32), "per-warp buffer");
 
-__global__ void __launch_bounds__(MERGE_THREADS, 3)
+#ifndef TT_MERGE_CTAS_PER_SM
+#define TT_MERGE_CTAS_PER_SM 3
+#endif
+constexpr int MERGE_CTAS_PER_SM = TT_MERGE_CTAS_PER_SM;   // resident CTAs per SM (registers and the 64 KiB of shared memory each)
+__global__ void __launch_bounds__(MERGE_THREADS, MERGE_CTAS_PER_SM)
 k_merge(const PieceParams P) {
     extern __shared__ __align__(16) u64 s_buf[];              // MERGE_SMEM_BYTES
     __shared__ u32 sc[48];

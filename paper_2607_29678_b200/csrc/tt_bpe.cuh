@@ -491,7 +491,10 @@ __device__ __forceinline__ u32 cta_min_u32(u32 v, u32* scratch /* >= 33 */) {
 // positions in place, chunk after chunk (every thread of a chunk has its positions in registers before
 // anything is written, and writes never pass the read front).  Ranks next to a merge are marked stale and
 // probed again in a second sweep, which also yields the next round's minimum.
-constexpr int LK = 16;
+#ifndef TT_LK
+#define TT_LK 16
+#endif
+constexpr int LK = TT_LK;                               // positions per thread and chunk (even)
 constexpr u32 F20_STALE = 0xFFFFEu;
 TT_HD u64 lp_pack(u32 t, u32 r20, u32 cl20) { return (u64)t | ((u64)r20 << TT_ID_BITS) | ((u64)cl20 << (TT_ID_BITS + 20)); }
 TT_HD u32 lp_tok(u64 v) { return (u32)v & (TT_MAX_INTERNAL - 1); }
@@ -504,7 +507,13 @@ __device__ __noinline__ u32 cta_merge_rounds(u64* arr, u32* crr, u32 m, const Pa
     finished = false;
     // minimum rank of the current array
     u32 lmin = TT_F20;
-    for (u32 i = tid; i < m; i += T) lmin = min(lmin, lp_rank(arr[i]));
+    for (u32 i0 = tid; i0 < m; i0 += (u32)T * 8) {
+        u64 xs[8];
+#pragma unroll
+        for (int u = 0; u < 8; u++) { const u32 i = i0 + (u32)u * T; xs[u] = i < m ? arr[i] : lp_pack(0, TT_F20, TT_F20); }
+#pragma unroll
+        for (int u = 0; u < 8; u++) lmin = min(lmin, lp_rank(xs[u]));
+    }
     for (;;) {
         const u32 mn = cta_min_u32(lmin, s_scr);
         if (mn >= F20_STALE) { finished = true; return m; }
@@ -597,17 +606,27 @@ __device__ __noinline__ u32 cta_merge_rounds(u64* arr, u32* crr, u32 m, const Pa
         m = out;
         __syncthreads();
         // probe the stale ranks again; collect the minimum for the next round
+        // (eight loads in flight per thread: in global scratch every one of them is an L2 round trip)
         lmin = TT_F20;
-        for (u32 i = tid; i < m; i += T) {
-            const u64 x = arr[i];
-            u32 r = lp_rank(x);
-            if (i + 1 >= m) { r = TT_F20; arr[i] = lp_pack(lp_tok(x), TT_F20, TT_F20); crr[i] = TT_F20; }
-            else if (r == F20_STALE) {
-                const PairInfo p = pair_probe(tab, lp_tok(x), lp_tok(arr[i + 1]));
-                r = f20_encode(p.r);
-                arr[i] = lp_pack(lp_tok(x), r, f20_encode(p.cl)); crr[i] = f20_encode(p.cr);
+        for (u32 i0 = tid; i0 < m; i0 += (u32)T * 8) {
+            u64 xs[8];
+#pragma unroll
+            for (int u = 0; u < 8; u++) { const u32 i = i0 + (u32)u * T; xs[u] = i < m ? arr[i] : lp_pack(0, TT_F20, TT_F20); }
+#pragma unroll
+            for (int u = 0; u < 8; u++) {
+                const u32 i = i0 + (u32)u * T;
+                const u64 x = xs[u];
+                u32 r = lp_rank(x);
+                if (i < m) {
+                    if (i + 1 >= m) { r = TT_F20; arr[i] = lp_pack(lp_tok(x), TT_F20, TT_F20); crr[i] = TT_F20; }
+                    else if (r == F20_STALE) {
+                        const PairInfo p = pair_probe(tab, lp_tok(x), lp_tok(arr[i + 1]));
+                        r = f20_encode(p.r);
+                        arr[i] = lp_pack(lp_tok(x), r, f20_encode(p.cl)); crr[i] = f20_encode(p.cr);
+                    }
+                }
+                lmin = min(lmin, r);
             }
-            lmin = min(lmin, r);
         }
         __syncthreads();
     }

@@ -501,7 +501,10 @@ TT_HD u32 lp_tok(u64 v) { return (u32)v & (TT_MAX_INTERNAL - 1); }
 TT_HD u32 lp_rank(u64 v) { return (u32)(v >> TT_ID_BITS) & TT_F20; }
 TT_HD u32 lp_cl(u64 v) { return (u32)(v >> (TT_ID_BITS + 20)) & TT_F20; }
 
-__device__ __noinline__ u32 cta_merge_rounds(u64* arr, u32* crr, u32 m, const PairTable& tab, u32* s_scr /* >= 48 */, u32 stop_at, bool& finished) {
+// padshift: 4 for arrays in shared memory (index i lives at i + i / 16, so that the 16-position slices of the
+// threads of a warp fall into different banks), 31 for arrays in global scratch (no padding).
+#define AX(i) ((i) + ((i) >> padshift))
+__device__ __noinline__ u32 cta_merge_rounds(u64* arr, u32* crr, u32 m, const PairTable& tab, u32* s_scr /* >= 48 */, u32 stop_at, bool& finished, u32 padshift) {
     const int tid = threadIdx.x, T = blockDim.x, lane = tid & 31, wid = tid >> 5, nw = T >> 5;
     const u32 FULL = 0xFFFFFFFFu, inmask = (1u << LK) - 1;
     finished = false;
@@ -510,7 +513,7 @@ __device__ __noinline__ u32 cta_merge_rounds(u64* arr, u32* crr, u32 m, const Pa
     for (u32 i0 = tid; i0 < m; i0 += (u32)T * 8) {
         u64 xs[8];
 #pragma unroll
-        for (int u = 0; u < 8; u++) { const u32 i = i0 + (u32)u * T; xs[u] = i < m ? arr[i] : lp_pack(0, TT_F20, TT_F20); }
+        for (int u = 0; u < 8; u++) { const u32 i = i0 + (u32)u * T; xs[u] = i < m ? arr[AX(i)] : lp_pack(0, TT_F20, TT_F20); }
 #pragma unroll
         for (int u = 0; u < 8; u++) lmin = min(lmin, lp_rank(xs[u]));
     }
@@ -528,7 +531,7 @@ __device__ __noinline__ u32 cta_merge_rounds(u64* arr, u32* crr, u32 m, const Pa
                 const u32 i = i0 + k - 1;                   // wraps for position -1 of the piece: not below m
                 v[k] = lp_pack(0, TT_F20, TT_F20); c[k] = TT_F20;
                 if (k == 0 && tid == 0) { if (base) v[k] = lp_pack(s_scr[42], TT_F20, s_scr[43]); }   // overwritten by the chunk before: carried
-                else if (i < m) { v[k] = arr[i]; c[k] = crr[i]; }
+                else if (i < m) { v[k] = arr[AX(i)]; c[k] = crr[AX(i)]; }
             }
             const u32 nval = i0 < m ? min((u32)LK, m - i0) : 0;
             u32 Qm = 0, Hm = 0, Gm = 0;                     // bit k: position i0 + k, k = 0 .. LK
@@ -594,8 +597,8 @@ __device__ __noinline__ u32 cta_merge_rounds(u64* arr, u32* crr, u32 m, const Pa
                     const bool me = (sel >> k) & 1;
                     const bool nxt = me ? false : ((sel >> (k + 1)) & 1);
                     const u64 x = v[k + 1];
-                    arr[o] = lp_pack(me ? 256u + lp_rank(x) : lp_tok(x), (me || nxt) ? F20_STALE : lp_rank(x), lp_cl(x));
-                    crr[o] = c[k + 1];
+                    arr[AX(o)] = lp_pack(me ? 256u + lp_rank(x) : lp_tok(x), (me || nxt) ? F20_STALE : lp_rank(x), lp_cl(x));
+                    crr[AX(o)] = c[k + 1];
                     o++;
                 }
             }
@@ -611,18 +614,18 @@ __device__ __noinline__ u32 cta_merge_rounds(u64* arr, u32* crr, u32 m, const Pa
         for (u32 i0 = tid; i0 < m; i0 += (u32)T * 8) {
             u64 xs[8];
 #pragma unroll
-            for (int u = 0; u < 8; u++) { const u32 i = i0 + (u32)u * T; xs[u] = i < m ? arr[i] : lp_pack(0, TT_F20, TT_F20); }
+            for (int u = 0; u < 8; u++) { const u32 i = i0 + (u32)u * T; xs[u] = i < m ? arr[AX(i)] : lp_pack(0, TT_F20, TT_F20); }
 #pragma unroll
             for (int u = 0; u < 8; u++) {
                 const u32 i = i0 + (u32)u * T;
                 const u64 x = xs[u];
                 u32 r = lp_rank(x);
                 if (i < m) {
-                    if (i + 1 >= m) { r = TT_F20; arr[i] = lp_pack(lp_tok(x), TT_F20, TT_F20); crr[i] = TT_F20; }
+                    if (i + 1 >= m) { r = TT_F20; arr[AX(i)] = lp_pack(lp_tok(x), TT_F20, TT_F20); crr[AX(i)] = TT_F20; }
                     else if (r == F20_STALE) {
-                        const PairInfo p = pair_probe(tab, lp_tok(x), lp_tok(arr[i + 1]));
+                        const PairInfo p = pair_probe(tab, lp_tok(x), lp_tok(arr[AX(i + 1)]));
                         r = f20_encode(p.r);
-                        arr[i] = lp_pack(lp_tok(x), r, f20_encode(p.cl)); crr[i] = f20_encode(p.cr);
+                        arr[AX(i)] = lp_pack(lp_tok(x), r, f20_encode(p.cl)); crr[AX(i)] = f20_encode(p.cr);
                     }
                 }
                 lmin = min(lmin, r);
@@ -633,39 +636,43 @@ __device__ __noinline__ u32 cta_merge_rounds(u64* arr, u32* crr, u32 m, const Pa
 }
 
 constexpr int LONG_SMEM_TOKENS = 4096;                  // long pieces move into shared memory below this many tokens
+constexpr int LONG_SMEM_SLOTS = LONG_SMEM_TOKENS + LONG_SMEM_TOKENS / 16 + 1;   // with the padding of the shared-memory layout
 
 // Encodes one piece of n > TT_WARP_PIECE_MAX bytes with the whole CTA.  gbuf: n entries of global scratch; the
 // piece's own n words of the staging array serve as the second global array until the ids are staged there.
-// sbuf: LONG_SMEM_TOKENS u64 followed by LONG_SMEM_TOKENS u32.
+// sbuf: LONG_SMEM_SLOTS u64 followed by LONG_SMEM_SLOTS u32.
 __device__ u32 cta_merge_long(const u8* __restrict__ text, u32 a, u32 n, const PairTable& tab, const int32_t* __restrict__ ext_id,
                               int32_t* __restrict__ stage, u64* gbuf, u64* sbuf, u32* s_scr) {
     const int tid = threadIdx.x, T = blockDim.x;
-    u32* const scr = reinterpret_cast<u32*>(sbuf + LONG_SMEM_TOKENS);
+    u32* const scr = reinterpret_cast<u32*>(sbuf + LONG_SMEM_SLOTS);
     u32* const gcr = reinterpret_cast<u32*>(stage + a);
     u64* arr = n <= LONG_SMEM_TOKENS ? sbuf : gbuf;
     u32* crr = n <= LONG_SMEM_TOKENS ? scr : gcr;
+    u32 padshift = n <= LONG_SMEM_TOKENS ? 4u : 31u;
     __syncthreads();
     for (u32 i = tid; i < n; i += T) {
         const u32 t0 = text[a + i];
         const PairInfo p = (i + 1 < n) ? bytepair_info(tab, t0, text[a + i + 1]) : pair_none();
-        arr[i] = lp_pack(t0, f20_encode(p.r), f20_encode(p.cl));
-        crr[i] = f20_encode(p.cr);
+        arr[AX(i)] = lp_pack(t0, f20_encode(p.r), f20_encode(p.cl));
+        crr[AX(i)] = f20_encode(p.cr);
     }
     __syncthreads();
     bool finished;
-    u32 m = cta_merge_rounds(arr, crr, n, tab, s_scr, arr == gbuf ? LONG_SMEM_TOKENS : 0, finished);
+    u32 m = cta_merge_rounds(arr, crr, n, tab, s_scr, arr == gbuf ? LONG_SMEM_TOKENS : 0, finished, padshift);
     if (!finished && arr == gbuf) {
         __syncthreads();
-        for (u32 i = tid; i < m; i += T) { sbuf[i] = gbuf[i]; scr[i] = gcr[i]; }
+        padshift = 4u;
+        for (u32 i = tid; i < m; i += T) { sbuf[AX(i)] = gbuf[i]; scr[AX(i)] = gcr[i]; }
         __syncthreads();
         arr = sbuf;
-        m = cta_merge_rounds(arr, scr, m, tab, s_scr, 0, finished);
+        m = cta_merge_rounds(arr, scr, m, tab, s_scr, 0, finished, padshift);
     }
     __syncthreads();
-    for (u32 i = tid; i < m; i += T) stage[a + i] = ext_id[lp_tok(arr[i])];
+    for (u32 i = tid; i < m; i += T) stage[a + i] = ext_id[lp_tok(arr[AX(i)])];
     __syncthreads();
     return m;
 }
+#undef AX
 
 // ---- pieces of one text tile -----------------------------------------------------------------------------
 // The start flags of a tile (TT_TILE_CHUNKS u16 masks) become a list of in-tile piece offsets in shared
@@ -838,7 +845,7 @@ k_lookup(const PieceParams P) {
 constexpr int MERGE_WARPS = 8;
 constexpr int MERGE_THREADS = MERGE_WARPS * 32;
 constexpr int WARP_SMEM_WORDS = 1024;                 // u64 per warp: two lane-path arrays of 32 x 32 u32, or two copies of four 256-word merge arrays
-static_assert(MERGE_WARPS * WARP_SMEM_WORDS * sizeof(u64) >= LONG_SMEM_TOKENS * (sizeof(u64) + sizeof(u32)), "the CTA's buffer must hold a long piece");
+static_assert(MERGE_WARPS * WARP_SMEM_WORDS * sizeof(u64) >= LONG_SMEM_SLOTS * (sizeof(u64) + sizeof(u32)), "the CTA's buffer must hold a long piece");
 constexpr size_t MERGE_SMEM_BYTES = (size_t)MERGE_WARPS * WARP_SMEM_WORDS * sizeof(u64);   // dynamic shared memory of k_merge (64 KiB)
 static_assert(WARP_SMEM_WORDS * sizeof(u64) >= 2 * LANE_SLOTS * LANE_MAX * sizeof(u32) && WARP_SMEM_WORDS * sizeof(u64) >= 2 * 4 * TT_WARP_PIECE_MAX * sizeof(u32), "per-warp buffer");
 

@@ -504,7 +504,8 @@ TT_HD u32 lp_cl(u64 v) { return (u32)(v >> (TT_ID_BITS + 20)) & TT_F20; }
 // padshift: 4 for arrays in shared memory (index i lives at i + i / 16, so that the 16-position slices of the
 // threads of a warp fall into different banks), 31 for arrays in global scratch (no padding).
 #define AX(i) ((i) + ((i) >> padshift))
-__device__ __noinline__ u32 cta_merge_rounds(u64* arr, u32* crr, u32 m, const PairTable& tab, u32* s_scr /* >= 48 */, u32 stop_at, bool& finished, u32 padshift) {
+__device__ __noinline__ u32 cta_merge_rounds(u64* arr, u32* crr, u32 m, const PairTable& tab, u32* s_scr /* >= 48 */, u32 stop_at, bool& finished, u32 padshift,
+                                           u64* stg_a = nullptr, u32* stg_c = nullptr) {
     const int tid = threadIdx.x, T = blockDim.x, lane = tid & 31, wid = tid >> 5, nw = T >> 5;
     const u32 FULL = 0xFFFFFFFFu, inmask = (1u << LK) - 1;
     finished = false;
@@ -590,17 +591,27 @@ __device__ __noinline__ u32 cta_merge_rounds(u64* arr, u32* crr, u32 m, const Pa
             const u32 surv = valid & ~gone;
             u32 tot;
             const u32 ex = cta_excl_sum_scan(__popc(surv), s_scr, &tot);         // all loads of the chunk are done: barrier inside
-            u32 o = out + ex;
+            // Arrays in global scratch: the chunk's survivors are collected in shared memory and written out with
+            // coalesced stores (a thread storing its own run of positions touches a line per store and lane, which
+            // is what a chunk spent most of its time on).
+            u64* const wa = stg_a ? stg_a : arr;
+            u32* const wc = stg_a ? stg_c : crr;
+            u32 o = stg_a ? ex : out + ex;
 #pragma unroll
             for (int k = 0; k < LK; k++) {
                 if ((surv >> k) & 1) {
                     const bool me = (sel >> k) & 1;
                     const bool nxt = me ? false : ((sel >> (k + 1)) & 1);
                     const u64 x = v[k + 1];
-                    arr[AX(o)] = lp_pack(me ? 256u + lp_rank(x) : lp_tok(x), (me || nxt) ? F20_STALE : lp_rank(x), lp_cl(x));
-                    crr[AX(o)] = c[k + 1];
+                    const u32 oi = stg_a ? o : AX(o);
+                    wa[oi] = lp_pack(me ? 256u + lp_rank(x) : lp_tok(x), (me || nxt) ? F20_STALE : lp_rank(x), lp_cl(x));
+                    wc[oi] = c[k + 1];
                     o++;
                 }
+            }
+            if (stg_a) {
+                __syncthreads();
+                for (u32 e = tid; e < tot; e += T) { arr[out + e] = stg_a[e]; crr[out + e] = stg_c[e]; }
             }
             out += tot;
             carry_hok = next_hok; carry_par = next_par; carry_last = next_last;
@@ -636,7 +647,8 @@ __device__ __noinline__ u32 cta_merge_rounds(u64* arr, u32* crr, u32 m, const Pa
 }
 
 constexpr int LONG_SMEM_TOKENS = 4096;                  // long pieces move into shared memory below this many tokens
-constexpr int LONG_SMEM_SLOTS = LONG_SMEM_TOKENS + LONG_SMEM_TOKENS / 16 + 1;   // with the padding of the shared-memory layout
+constexpr int LONG_SMEM_SLOTS = LONG_SMEM_TOKENS + LONG_SMEM_TOKENS / 16 + 8;   // with the padding of the shared-memory layout; also holds a chunk's survivors
+static_assert(LONG_SMEM_TOKENS >= 256 * LK, "the survivors of a chunk (threads x LK positions) must fit the shared buffer");
 
 // Encodes one piece of n > TT_WARP_PIECE_MAX bytes with the whole CTA.  gbuf: n entries of global scratch; the
 // piece's own n words of the staging array serve as the second global array until the ids are staged there.
@@ -658,7 +670,8 @@ __device__ u32 cta_merge_long(const u8* __restrict__ text, u32 a, u32 n, const P
     }
     __syncthreads();
     bool finished;
-    u32 m = cta_merge_rounds(arr, crr, n, tab, s_scr, arr == gbuf ? LONG_SMEM_TOKENS : 0, finished, padshift);
+    u32 m = cta_merge_rounds(arr, crr, n, tab, s_scr, arr == gbuf ? LONG_SMEM_TOKENS : 0, finished, padshift,
+                             arr == gbuf ? sbuf : nullptr, arr == gbuf ? scr : nullptr);       // the shared buffer stages the stores meanwhile
     if (!finished && arr == gbuf) {
         __syncthreads();
         padshift = 4u;

@@ -396,6 +396,17 @@ def main():
                  "chars": int(bchars), "bytes": int(btext.size), "tokens": btok, "ms": round(bms, 3),
                  "chars_per_s": round(cps, 1), "GB_per_s": round(btext.size / (bms * 1e-3) / 1e9, 3),
                  "hbm_roofline_frac": round((btext.size + 4 * btok + 16 * boff.size) / (bms * 1e-3) / 1e9 / peak, 5)}
+        if args.batch_docs == c5.n_docs and world == 1:
+            # the batch is bound by instruction issue, not by HBM: warp instructions of the four kernels (ncu capture
+            # of this very workload, profiles/c5_batch_256_requests_kernels.md) per second against what the SMs can
+            # issue (SMs x 4 schedulers x 1 warp instruction per clock at the maximum SM clock)
+            sm_count = torch.cuda.get_device_properties(0).multi_processor_count
+            mhz = (clocks or {}).get("sm_max_mhz") or 1965.0
+            issue_peak = sm_count * 4 * mhz * 1e6
+            winst = sum(NCU_BATCH_WARP_INST.values())
+            batch["alu_roofline"] = {"bound": "alu", "achieved": round(winst / (bms * 1e-3) / 1e9, 1), "peak": round(issue_peak / 1e9, 1),
+                                     "unit": "G warp-instructions/s", "frac": round(winst / (bms * 1e-3) / issue_peak, 4),
+                                     "warp_instructions": winst}
         del d_text, bb
 
     if rank != 0:
@@ -483,6 +494,10 @@ def vocab_table_bytes(n_merges: int) -> int:
     slot per merge, the 4-byte id map and the 21,632-byte class tables."""
     return 8 * n_merges + 4 * (256 + n_merges) + 21632
 
+
+# Warp instructions per launch (smsp__inst_executed.sum) from the committed ncu capture of the C5 batch
+# (profiles/c5_batch_256_requests_kernels.md).
+NCU_BATCH_WARP_INST = {"pretok": 373_891_564, "lookup": 360_754_739, "merge": 148_638_787, "scatter": 163_907_810}
 
 # DRAM bytes (read + write) per launch from the committed ncu capture of the C3 request
 # (profiles/c3_1M_request_kernels.md).

@@ -52,6 +52,7 @@ struct tt_vocab {
     u8* d_text = nullptr; int32_t* d_ids = nullptr; long long* d_count = nullptr; int32_t* d_status = nullptr;
     void* d_ws = nullptr; size_t host_cap = 0, ws_cap = 0;
     cudaStream_t host_stream = nullptr;
+    cudaEvent_t slice_ev[8] = {};
 };
 
 static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -92,6 +93,7 @@ extern "C" void tt_vocab_free(tt_vocab* v) {
     if (v->h_ids) cudaFreeHost(v->h_ids);
     if (v->h_scalars) cudaFreeHost(v->h_scalars);
     if (v->host_stream) cudaStreamDestroy(v->host_stream);
+    for (cudaEvent_t e : v->slice_ev) if (e) cudaEventDestroy(e);
     delete v;
 }
 
@@ -758,8 +760,16 @@ extern "C" int tt_encode_host(tt_vocab* v, const uint8_t* text, size_t len, int3
     int32_t* ids_dev_view = nullptr;
     const bool in_pinned = len && host_pointer_is_pinned(text, nullptr);
     const bool out_pinned = len && host_pointer_is_pinned(ids_out, (void**)&ids_dev_view) && ids_dev_view != nullptr;
-    if (!in_pinned) memcpy(v->h_text, text, len);
-    CK(cudaMemcpyAsync(v->d_text, in_pinned ? text : v->h_text, len, cudaMemcpyHostToDevice, st));
+    if (in_pinned) CK(cudaMemcpyAsync(v->d_text, text, len, cudaMemcpyHostToDevice, st));
+    else {
+        // pageable text is staged in slices, so that the DMA of one slice runs while the next is being staged
+        const size_t slice = 256u << 10;
+        for (size_t o = 0; o < len; o += slice) {
+            const size_t n = len - o < slice ? len - o : slice;
+            memcpy(v->h_text + o, text + o, n);
+            CK(cudaMemcpyAsync(v->d_text + o, v->h_text + o, n, cudaMemcpyHostToDevice, st));
+        }
+    }
     // count and status are written by the kernel into mapped pinned scalars of the handle
     long long* count_dev = nullptr; int32_t* status_dev = nullptr;
     {
@@ -776,10 +786,23 @@ extern "C" int tt_encode_host(tt_vocab* v, const uint8_t* text, size_t len, int3
     if (status != TT_OK) return status;
     const long long n = v->h_scalars[0];
     if ((size_t)n > ids_cap) return TT_ERR_CAPACITY;
-    if (!out_pinned) {
-        CK(cudaMemcpyAsync(v->h_ids, v->d_ids, (size_t)n * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
-        CK(cudaStreamSynchronize(st));
-        memcpy(ids_out, v->h_ids, (size_t)n * sizeof(int32_t));
+    if (!out_pinned && n > 0) {
+        // the ids come back in up to eight slices: while one is copied out of the staging buffer the DMA brings the next
+        const size_t total = (size_t)n * sizeof(int32_t);
+        size_t nsl = (total + (256u << 10) - 1) / (256u << 10);
+        if (nsl > 8) nsl = 8;
+        const size_t per = align_up((total + nsl - 1) / nsl, 4096);
+        for (size_t k = 0; k < nsl; k++) {
+            if (!v->slice_ev[k]) CK(cudaEventCreateWithFlags(&v->slice_ev[k], cudaEventDisableTiming));
+            const size_t o = k * per, nb = o >= total ? 0 : (total - o < per ? total - o : per);
+            if (nb) CK(cudaMemcpyAsync((char*)v->h_ids + o, (const char*)v->d_ids + o, nb, cudaMemcpyDeviceToHost, st));
+            CK(cudaEventRecord(v->slice_ev[k], st));
+        }
+        for (size_t k = 0; k < nsl; k++) {
+            CK(cudaEventSynchronize(v->slice_ev[k]));
+            const size_t o = k * per, nb = o >= total ? 0 : (total - o < per ? total - o : per);
+            if (nb) memcpy((char*)ids_out + o, (const char*)v->h_ids + o, nb);
+        }
     }
     *count_out = n;
     return TT_OK;

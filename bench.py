@@ -161,6 +161,8 @@ def main():
                     help="run only the warm-up and the timed steps, then exit (command used under ncu)")
     ap.add_argument("--profile-batch", action="store_true",
                     help="run only the config-C5 batch leg (2 warm-up + 2 timed calls), then exit (command used under ncu)")
+    ap.add_argument("--profile-long-piece", action="store_true",
+                    help="encode one 16,384-byte piece of random lower-case letters three times, then exit (command used under ncu)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -188,6 +190,19 @@ def main():
     cfg = wl.CONFIGS["C3"]
     merges, byte_map = wl.load_vocab(cfg)
     vocab = tt.Vocab(merges, byte_map, cfg.pattern_id)
+    if args.profile_long_piece:
+        piece = (97 + np.random.default_rng(1).integers(0, 26, 16384)).astype(np.uint8)
+        d_piece = torch.from_numpy(piece).cuda()
+        pb = vocab.alloc(piece.size)
+        ts = []
+        for k in range(3):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(); vocab.encode(d_piece, pb); b.record()
+            torch.cuda.synchronize()
+            ts.append(a.elapsed_time(b))
+        print(json.dumps({"profile_long_piece_run": True, "bytes": int(piece.size), "ms": [round(t, 3) for t in ts],
+                          "tokens": int(pb["count"].item())}), flush=True)
+        return
     if args.profile_batch:
         c5 = wl.CONFIGS["C5"]
         btext, boff = wl.batch(c5, sample=rank, n_docs=args.batch_docs)

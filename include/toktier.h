@@ -132,8 +132,11 @@ int tt_encode_batch(const tt_vocab* v, const uint8_t* text, size_t total_len, co
 /*
  * tt_pretokenize -- the pre-tokenization half alone (paper Sec. 4.1; the paper checks piece
  * boundaries separately from IDs because ID-level agreement can hide a boundary fault).
- *   piece_off_out  DEVICE int32[piece_cap]: byte offset of every piece start, ascending;
- *                  piece_cap >= len always suffices.
+ *   piece_off_out  DEVICE int32[piece_cap]: byte offset of every piece start, ascending, followed by one
+ *                  closing entry piece_off_out[n_pieces] = len.  piece_cap must be at least len + 1 (a piece
+ *                  has at least one byte, so that always suffices; a smaller capacity is refused with
+ *                  TT_ERR_ARG before anything is enqueued).  With len == 0 nothing is written and any
+ *                  capacity, also 0 with a null pointer, is accepted.
  *   n_pieces_out   DEVICE int64: number of pieces.
  * doc_off / n_docs as in tt_encode_batch, or doc_off = NULL and n_docs = 1 for one document.
  */

@@ -372,6 +372,37 @@ int64_t orc_pretok(int pattern, const uint8_t *text, size_t len, int64_t *starts
     return (int64_t)st.size();
 }
 
+/* Piece starts of a batch: every document [doc_off[d], doc_off[d+1]) is matched exactly as if it were alone
+ * (orc_pretok on its bytes); the starts are written as offsets into the concatenation, in document order.
+ * Documents are spread over threads in contiguous ranges.  Returns the total piece count (only cap are
+ * written), or -(d+1) if document d is invalid UTF-8. */
+int64_t orc_pretok_batch(int pattern, const uint8_t *text, const int64_t *doc_off, size_t n_docs, int nthreads,
+                         int64_t *starts_out, size_t cap) {
+    if (nthreads < 1) nthreads = 1;
+    std::vector<std::vector<int64_t>> part((size_t)nthreads);
+    std::vector<int64_t> bad((size_t)nthreads, 0);
+    std::vector<std::thread> th;
+    const size_t per = (n_docs + (size_t)nthreads - 1) / (size_t)nthreads;
+    for (int k = 0; k < nthreads; k++) {
+        th.emplace_back([&, k]() {
+            const size_t lo = std::min(n_docs, (size_t)k * per), hi = std::min(n_docs, lo + per);
+            Text t; std::vector<size_t> st;
+            for (size_t d = lo; d < hi; d++) {
+                const size_t len = (size_t)(doc_off[d + 1] - doc_off[d]);
+                if (!decode_utf8(text + doc_off[d], len, t)) { bad[k] = -(int64_t)(d + 1); return; }
+                st.clear();
+                pretok_cp(t, pattern, st);
+                for (size_t i = 0; i < st.size(); i++) part[k].push_back(doc_off[d] + (int64_t)t.off[st[i]]);
+            }
+        });
+    }
+    for (auto &x : th) x.join();
+    for (int k = 0; k < nthreads; k++) if (bad[k] < 0) return bad[k];
+    size_t n = 0;
+    for (auto &p : part) { for (int64_t v : p) { if (n < cap) starts_out[n] = v; n++; } }
+    return (int64_t)n;
+}
+
 void *orc_vocab_new(const int32_t *merges /* n x 3: left,right,result */, size_t n, const int32_t *byte_map) {
     Vocab *v = new Vocab();
     std::memcpy(v->byte_map, byte_map, sizeof(v->byte_map));

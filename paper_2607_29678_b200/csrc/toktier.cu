@@ -602,7 +602,9 @@ extern "C" int tt_vocab_add_literals(tt_vocab* v, const uint8_t* bytes, const ui
         return TT_ERR_CUDA;
     }
     T.entries = v->d_lit_entries; T.blob = v->d_lit_blob; T.n = (u32)n; T.maxlen = maxlen;
-    v->lit = T;
+    // the literals are registered (v->lit) only once every allocation and copy below has succeeded, so that a
+    // failed call leaves the vocabulary as it was and may be repeated
+    auto undo = [&]() { cudaFree(v->d_lit_entries); cudaFree(v->d_lit_blob); v->d_lit_entries = nullptr; v->d_lit_blob = nullptr; };
     if (v->meta_n) {
         // tt_spans: byte and character length of every literal whose id the merge table does not use itself
         int32_t max_id = (int32_t)v->meta_n - 1;
@@ -619,11 +621,12 @@ extern "C" int tt_vocab_add_literals(tt_vocab* v, const uint8_t* bytes, const ui
             }
             ok = ok && cudaMalloc(&d_new, meta.size() * sizeof(uint2)) == cudaSuccess;
             ok = ok && cudaMemcpy(d_new, meta.data(), meta.size() * sizeof(uint2), cudaMemcpyHostToDevice) == cudaSuccess;
-            if (!ok) { cudaGetLastError(); cudaFree(d_new); return TT_ERR_CUDA; }
+            if (!ok) { cudaGetLastError(); cudaFree(d_new); undo(); return TT_ERR_CUDA; }
             cudaFree(v->d_meta);
             v->d_meta = d_new; v->meta_n = (u32)meta.size();
         }
     }
+    v->lit = T;
     return TT_OK;
 }
 
@@ -675,7 +678,7 @@ extern "C" int tt_pretokenize(const tt_vocab* v, const uint8_t* text, size_t len
                               int32_t* status_out, void* workspace, size_t workspace_bytes) {
     int rc = check_common(v, text, len, workspace, workspace_bytes, n_docs);
     if (rc != TT_OK) return rc;
-    if (!n_pieces_out || !status_out || (len && !piece_off_out) || piece_cap < len + 1) return TT_ERR_ARG;
+    if (!n_pieces_out || !status_out || (len && (!piece_off_out || piece_cap < len + 1))) return TT_ERR_ARG;
     cudaStream_t st = (cudaStream_t)stream;
     TTWorkspace w;
     carve(&w, workspace, len, n_docs);
@@ -837,8 +840,10 @@ extern "C" int tt_encode_static(const tt_vocab* v, const uint8_t* text, size_t l
         }
         scratch = g_static_scratch_ptr[dev];
     }
-    // encode_impl clears the header (status word and work counters) first; every other scratch array
-    // is written before it is read, so the previous call's contents do not matter.
+    // Nothing of the previous call's contents matters: the chain's first kernel zeroes the header's work
+    // counters, the status word is tagged with this call's epoch (an older tag reads as "no error"; encode_impl
+    // clears the header with a memset only under stream capture), and every other scratch array is written
+    // before it is read.
     return encode_impl(v, text, len, nullptr, 1, (cudaStream_t)stream, ids_out, ids_cap, count_out, nullptr, status_out,
                        scratch);
 }
@@ -925,7 +930,8 @@ extern "C" int tt_session_append(tt_session* s, const uint8_t* text, size_t len,
     tt_append_info local; memset(&local, 0, sizeof(local));
     const size_t old_len = s->len, new_len = old_len + len;
     s->h_text.insert(s->h_text.end(), text, text + len);
-    auto fail = [&](int code) { s->h_text.resize(old_len); if (info) { local.status = code; *info = local; } return code; };
+    // (an error return waits for the stream first: the copy from the caller's buffer may still be in flight)
+    auto fail = [&](int code) { cudaStreamSynchronize(st); cudaGetLastError(); s->h_text.resize(old_len); if (info) { local.status = code; *info = local; } return code; };
     if (len) { if (cudaMemcpyAsync(s->d_text + old_len, text, len, cudaMemcpyHostToDevice, st) != cudaSuccess) { cudaGetLastError(); return fail(TT_ERR_CUDA); } }
     if (new_len == 0) { if (info) *info = local; return TT_OK; }
     const u8* ht = s->h_text.data();

@@ -1,9 +1,30 @@
-"""Helpers for the GPU parity tests: run the C-ABI entry points on device tensors."""
+"""Helpers for the GPU parity tests: run the C-ABI entry points on device tensors, and the one comparison
+every parity test applies to what comes back."""
 import functools
 
 import numpy as np
 
 import workloads as wl
+
+
+def same(got, want) -> bool:
+    """Bit-exact equality of two integer sequences (token ids, piece offsets, token offsets): same length,
+    same dtype kind, same value at every index.  This is the whole tolerance of the parity tests; the
+    planted-fault test (test_harness_faults.py) feeds it mutated GPU output and expects False every time."""
+    got, want = np.asarray(got), np.asarray(want)
+    if got.ndim != 1 or want.ndim != 1 or got.dtype.kind not in "iu" or want.dtype.kind not in "iu":
+        return False
+    return got.shape == want.shape and bool(np.array_equal(got, want))
+
+
+def first_difference(got, want) -> str:
+    """Where two sequences part, for assertion messages."""
+    got, want = np.asarray(got), np.asarray(want)
+    n = min(got.size, want.size)
+    d = np.flatnonzero(got[:n] != want[:n])
+    k = int(d[0]) if d.size else n
+    return (f"sizes {got.size} / {want.size}, first difference at index {k}: "
+            f"got {got[k:k + 4].tolist()} want {want[k:k + 4].tolist()}")
 
 
 @functools.lru_cache(maxsize=None)

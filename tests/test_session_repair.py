@@ -9,7 +9,7 @@ import pytest
 import oracle
 import workloads as wl
 from oracle import repair
-from gpu_util import cpu_vocab, gpu_vocab
+from gpu_util import cpu_vocab, gpu_vocab, same
 
 pytestmark = pytest.mark.gpu
 
@@ -45,7 +45,7 @@ def test_append_stream_matches_oracle_protocol_and_full_tokenization(name, windo
         ids, off, nbytes = sess.records()
         full, _ = cv.encode(done, pat)
         assert nbytes == len(done) and info["status"] == 0 and info["n_tokens"] == full.size
-        assert np.array_equal(ids.cpu().numpy(), full)
+        assert same(ids.cpu().numpy(), full)
         assert off.cpu().numpy().tolist() == ref.off
         for key in ("attempts", "window_chars", "window_start", "run_tokens", "splice_byte"):
             assert info[key] == want_info[key], (key, info, want_info, len(done))
@@ -63,7 +63,7 @@ def test_digit_run_without_stable_boundary_is_not_spliced():
     info = sess.append(b)
     ids, off, _ = sess.records()
     full, _ = cv.encode(a + b, 0)
-    assert np.array_equal(ids.cpu().numpy(), full) and info["attempts"] > 1
+    assert same(ids.cpu().numpy(), full) and info["attempts"] > 1
 
 
 def test_rejected_append_leaves_the_session_unchanged():
@@ -81,4 +81,4 @@ def test_rejected_append_leaves_the_session_unchanged():
     sess.append(b" And on it goes.")
     ids, _, nbytes = sess.records()
     full, _ = cv.encode(good + b" And on it goes.", 0)
-    assert nbytes == len(good) + 16 and np.array_equal(ids.cpu().numpy(), full)
+    assert nbytes == len(good) + 16 and same(ids.cpu().numpy(), full)

@@ -4,7 +4,7 @@ import pytest
 
 import oracle
 import workloads as wl
-from gpu_util import cpu_vocab, gpu_vocab, to_dev
+from gpu_util import cpu_vocab, gpu_vocab, to_dev, same
 from patterns import PATTERNS
 
 
@@ -43,7 +43,7 @@ def test_oracle_spans_against_string_slicing_and_tiktoken(name):
     enc = tiktoken.Encoding("spans", pat_str=PATTERNS[cfg.pattern_id], mergeable_ranks={t: i for i, t in enumerate(toks)}, special_tokens={})
     _, offs = enc.decode_with_offsets([int(i) for i in ids])
     offs = np.asarray(offs)
-    assert np.array_equal(offs[on_boundary], c[:-1][on_boundary])
+    assert same(offs[on_boundary], c[:-1][on_boundary])
 
 
 @pytest.mark.gpu
@@ -65,8 +65,8 @@ def test_gpu_spans_match_oracle(name, n_chars):
     n = int(bufs["count"].item())
     ids = bufs["ids"][:n].cpu().numpy()
     wb, wc = cv.spans(text, ids)
-    assert np.array_equal(boff[:n + 1].cpu().numpy(), wb)
-    assert np.array_equal(coff[:n + 1].cpu().numpy(), wc)
+    assert same(boff[:n + 1].cpu().numpy(), wb)
+    assert same(coff[:n + 1].cpu().numpy(), wc)
     # ids that do not belong to the text are reported, not trusted
     gv.spans(bufs["ids"], bufs["count"], text.size + 1, boff, coff, bufs["status"])
     torch.cuda.synchronize()

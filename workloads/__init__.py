@@ -45,6 +45,9 @@ def _load():
                                          ctypes.c_double, ctypes.c_double, ctypes.c_void_p]
         lib.wl_count_chars.restype = ctypes.c_size_t
         lib.wl_count_chars.argtypes = [ctypes.c_void_p, ctypes.c_size_t]
+        lib.wl_exhaustive.restype = ctypes.c_size_t
+        lib.wl_exhaustive.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.c_void_p, ctypes.c_size_t,
+                                      ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p]
         _lib = lib
     return _lib
 
@@ -62,6 +65,25 @@ def generate(kind: int, seed: int, n_chars: int) -> np.ndarray:
 def count_chars(text: np.ndarray) -> int:
     text = np.ascontiguousarray(text, dtype=np.uint8)
     return int(_load().wl_count_chars(text.ctypes.data, text.size))
+
+
+def exhaustive(alphabet, maxlen: int):
+    """Every string of 1..maxlen symbols over ``alphabet`` (a str: one symbol per character), shortest first,
+    in the order of ``itertools.product``: returns (concatenated uint8 text, int64 byte offsets[n + 1])."""
+    lib = _load()
+    syms = [ch.encode("utf-8") for ch in alphabet]
+    blob = np.frombuffer(b"".join(syms), dtype=np.uint8).copy()
+    soff = np.zeros(len(syms) + 1, dtype=np.uint32)
+    soff[1:] = np.cumsum([len(x) for x in syms])
+    need = ctypes.c_size_t(0)
+    n = lib.wl_exhaustive(blob.ctypes.data, soff.ctypes.data, len(syms), maxlen, None, 0, None, 0, ctypes.byref(need))
+    text = np.empty(need.value + 16, dtype=np.uint8)
+    off = np.empty(n + 1, dtype=np.int64)
+    got = lib.wl_exhaustive(blob.ctypes.data, soff.ctypes.data, len(syms), maxlen, text.ctypes.data, text.size,
+                            off.ctypes.data, off.size + 1, None)
+    if got != n:
+        raise RuntimeError("exhaustive generator: buffers too small")
+    return text[:need.value], off
 
 
 def batch_lengths(seed: int, n: int, median: float, sigma: float, lo: float, hi: float) -> np.ndarray:

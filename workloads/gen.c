@@ -491,3 +491,36 @@ size_t wl_count_chars(const uint8_t *p, size_t len) {
     for (size_t i = 0; i < len; i++) n += ((p[i] & 0xC0) != 0x80);
     return n;
 }
+
+/* Every string of 1..maxlen symbols over an alphabet of k symbols (each symbol a byte string of its own,
+ * sym_off[k+1] offsets into sym_bytes), shortest first, each length in odometer order with the last
+ * position fastest.  The strings are written back to back into `out`; doc_off receives the n + 1 byte
+ * offsets.  Returns the number of strings n, or 0 if either buffer is too small.  With out == NULL only
+ * the sizes are computed: *bytes_needed receives the total number of bytes. */
+size_t wl_exhaustive(const uint8_t *sym_bytes, const uint32_t *sym_off, int k, int maxlen, uint8_t *out, size_t cap,
+                     int64_t *doc_off, size_t doc_cap, size_t *bytes_needed) {
+    size_t n = 0, bytes = 0;
+    int idx[32];
+    if (k < 1 || maxlen < 1 || maxlen > 32) return 0;
+    for (int len = 1; len <= maxlen; len++) {
+        for (int i = 0; i < len; i++) idx[i] = 0;
+        for (;;) {
+            if (out) {
+                if (n + 1 >= doc_cap) return 0;
+                doc_off[n] = (int64_t)bytes;
+            }
+            for (int i = 0; i < len; i++) {
+                const uint32_t a = sym_off[idx[i]], b = sym_off[idx[i] + 1];
+                if (out) { if (bytes + (b - a) > cap) return 0; memcpy(out + bytes, sym_bytes + a, b - a); }
+                bytes += b - a;
+            }
+            n++;
+            int i = len - 1;
+            while (i >= 0 && ++idx[i] == k) { idx[i] = 0; i--; }
+            if (i < 0) break;
+        }
+    }
+    if (out) doc_off[n] = (int64_t)bytes;
+    if (bytes_needed) *bytes_needed = bytes;
+    return n;
+}

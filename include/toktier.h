@@ -261,15 +261,15 @@ void tt_verifier_free(tt_verifier* q);
 /*
  * tt_encode_timed -- diagnostic variant of tt_encode (same arguments and results) that records
  * CUDA events on `stream` between the kernels of the chain, waits for the last one and returns the
- * device time of each step in milliseconds: ms_out[0] tag + piece-start flags and the tile
- * piece counts (K1+K2), [1] per-tile compaction and whole-piece lookup (K3+K4a), [2] merges of the
- * pieces the lookup did not settle (K4b), [3] token offsets and scatter (K5).  Synchronises; requires len > 0.  Used by the benchmark for the
- * per-kernel roofline; the event records perturb the chain slightly, so latency is never quoted
- * from this call.
+ * device time of each step in milliseconds: ms_out[0] the first kernel (tag + piece-start flags, per-tile
+ * compaction and whole-piece lookups: K1+K2+K3+K4a), [1] merges of the pieces the lookups did not settle
+ * (K4b), [2] token offsets and scatter (K5).  Synchronises; requires len > 0.  Used by the benchmark for the
+ * per-kernel roofline; the event records perturb the chain slightly (the kernels are launched without
+ * programmatic dependent launch here), so the sum exceeds the latency of a plain tt_encode call.
  */
-int tt_encode_timed(const tt_vocab* v, const uint8_t* text, size_t len, void* stream,
-                    int32_t* ids_out, size_t ids_cap, int64_t* count_out, int32_t* status_out,
-                    void* workspace, size_t workspace_bytes, float ms_out[4]);
+int tt_encode_timed(const tt_vocab* v, const uint8_t* text, size_t len, void* stream, int32_t* ids_out,
+                    size_t ids_cap, int64_t* count_out, int32_t* status_out, void* workspace,
+                    size_t workspace_bytes, float ms_out[3]);
 
 /*
  * tt_encode_host -- convenience wrapper for HOST buffers: copies `text` to the device, encodes,

@@ -216,12 +216,12 @@ class Vocab:
                                      bufs["ids"].numel(), bufs["count"].data_ptr(), bufs["status"].data_ptr(),
                                      ws.data_ptr(), ws.numel()), "tt_encode_added")
 
-    KERNEL_NAMES = ("pretok", "lookup", "merge", "scatter")
+    KERNEL_NAMES = ("front", "merge", "scatter")
 
     def encode_timed(self, text, bufs, stream=None) -> dict:
         """tt_encode_timed: like encode, synchronises, returns {kernel name: milliseconds}."""
         ws = bufs["workspace"]
-        ms = (ctypes.c_float * 4)()
+        ms = (ctypes.c_float * 3)()
         _check(lib().tt_encode_timed(self._h, text.data_ptr(), int(text.numel()), _stream_ptr(stream),
                                      bufs["ids"].data_ptr(), bufs["ids"].numel(), bufs["count"].data_ptr(),
                                      bufs["status"].data_ptr(), ws.data_ptr(), ws.numel(), ms), "tt_encode_timed")

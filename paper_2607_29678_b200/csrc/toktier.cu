@@ -1,6 +1,6 @@
 // C ABI of the toktier library (see include/toktier.h).  Host side: argument checks, vocabulary
-// tables, workspace layout and the kernel chain  k_pretok (K1+K2, tile piece counts) -> k_lookup (K3 per tile in
-// shared memory, whole-piece lookups) -> k_merge (K4's merges, from global queues) -> k_scatter (K5); sessions
+// tables, workspace layout and the kernel chain  k_pretok<fused> (K1+K2, K3 per tile in shared memory, whole-piece
+// lookups) -> k_merge (K4's merges, from the per-tile queues) -> k_scatter (K5); sessions
 // (incremental repair), the added-token literal pass and the shadow verifier (host only) sit on top of it.
 // Nothing here synchronises with the device except tt_vocab_load, tt_encode_host, tt_encode_timed and
 // tt_session_append.
@@ -157,43 +157,50 @@ static int build_token_table(tt_vocab* v, const tt_merge* merges, size_t n_merge
     std::vector<u32> keep;
     if (v->ignore_merges) { for (size_t i = 0; i < np; i++) keep.push_back((u32)i); }
     else {
-    // start flags and per-tile piece counts of the concatenation, as k_pretok would leave them
+    // the per-tile records of the concatenation as the first kernel would leave them without a table: every piece
+    // but the last of its tile is queued (all are short), the last one of every tile is k_merge's anyway
     const size_t nchunks = (nb + TT_CHUNK - 1) / TT_CHUNK, ntiles = (nchunks + TT_TILE_CHUNKS - 1) / TT_TILE_CHUNKS;
-    std::vector<u16> smask(nchunks + 1, 0);
-    std::vector<u32> tile_base(ntiles + 1, 0), tile_first(ntiles + 1, 0xFFFFFFFFu);
-    for (size_t i = 0; i < np; i++) { smask[off[i] >> 4] |= (u16)(1u << (off[i] & 15)); tile_base[off[i] / TT_TILE_BYTES + 1]++;
-        u32& tf = tile_first[off[i] / TT_TILE_BYTES]; if (tf == 0xFFFFFFFFu) tf = off[i] % TT_TILE_BYTES; }
-    for (size_t t = 0; t < ntiles; t++) tile_base[t + 1] += tile_base[t];
-    u8* d_text = nullptr; u16* d_mask = nullptr; u32 *d_tf = nullptr, *d_cnt = nullptr, *d_tt = nullptr, *d_gt = nullptr; u64 *d_qs = nullptr, *d_qw = nullptr; uint4* d_ql = nullptr; int32_t* d_stage = nullptr;
+    std::vector<u32> tile_base(ntiles + 1, 0), tile_cnt(ntiles, 0), tile_first(ntiles, TT_NONE), tile_last(ntiles, TT_NONE), tile_q(ntiles, 0);
+    std::vector<u16> off16(ntiles * TT_TILE_BYTES, 0);
+    std::vector<u32> qv(ntiles * TT_TILE_QCAP, 0);
+    for (size_t i = 0; i < np; i++) {
+        const size_t t = off[i] / TT_TILE_BYTES; const u32 o = off[i] % TT_TILE_BYTES;
+        off16[t * TT_TILE_BYTES + tile_cnt[t]] = (u16)o;
+        if (tile_first[t] == TT_NONE) tile_first[t] = o;
+        tile_last[t] = o; tile_cnt[t]++;
+    }
+    for (size_t t = 0; t < ntiles; t++) tile_base[t + 1] = tile_base[t] + tile_cnt[t];
+    for (size_t t = 0; t < ntiles; t++)
+        for (u32 k = 0; k + 1 < tile_cnt[t]; k++) {
+            const size_t i = tile_base[t] + k;
+            qv[t * TT_TILE_QCAP + tile_q[t]++] = off16[t * TT_TILE_BYTES + k] | (k << 11) | ((off[i + 1] - off[i] - 1) << 22);
+        }
+    u8* d_text = nullptr; u32 *d_tc = nullptr, *d_tf = nullptr, *d_tl = nullptr, *d_tq = nullptr, *d_cnt = nullptr, *d_tt = nullptr, *d_q = nullptr; u16 *d_o16 = nullptr, *d_lg = nullptr; int32_t* d_stage = nullptr;
     TTHeader* d_hdr = nullptr;
-    TTHeader h; memset(&h, 0, sizeof(h)); h.n_pieces = (u32)np;
     std::vector<u32> cnt(ntiles * TT_TILE_BYTES); std::vector<int32_t> stage(nb);
-    const size_t ngroups = ntiles / TT_GROUP_TILES + 2;
-    bool ok = cudaMalloc(&d_text, nchunks * TT_CHUNK + 64) == cudaSuccess && cudaMalloc(&d_mask, (nchunks + 1) * sizeof(u16)) == cudaSuccess &&
-              cudaMalloc(&d_gt, ngroups * sizeof(u32)) == cudaSuccess && cudaMalloc(&d_tt, (ntiles + 1) * sizeof(u32)) == cudaSuccess && cudaMalloc(&d_tf, (ntiles + 1) * sizeof(u32)) == cudaSuccess &&
+    auto up = [&](auto** dp, const auto& h) {
+        return cudaMalloc(dp, h.size() * sizeof(h[0]) + 64) == cudaSuccess && cudaMemcpy(*dp, h.data(), h.size() * sizeof(h[0]), cudaMemcpyHostToDevice) == cudaSuccess;
+    };
+    bool ok = cudaMalloc(&d_text, nchunks * TT_CHUNK + 64) == cudaSuccess && cudaMemcpy(d_text, cat.data(), nb, cudaMemcpyHostToDevice) == cudaSuccess;
+    ok = ok && up(&d_tc, tile_cnt) && up(&d_tf, tile_first) && up(&d_tl, tile_last) && up(&d_tq, tile_q) && up(&d_o16, off16) && up(&d_q, qv);
+    ok = ok && cudaMalloc(&d_lg, ntiles * TT_TILE_LONGCAP * sizeof(u16)) == cudaSuccess && cudaMalloc(&d_tt, (ntiles + 1) * sizeof(u32)) == cudaSuccess &&
               cudaMalloc(&d_cnt, cnt.size() * sizeof(u32)) == cudaSuccess && cudaMalloc(&d_stage, (nb + 1) * sizeof(int32_t)) == cudaSuccess &&
-              cudaMalloc(&d_hdr, sizeof(TTHeader)) == cudaSuccess && cudaMalloc(&d_qs, (nb / 2 + 64) * sizeof(u64)) == cudaSuccess &&
-              cudaMalloc(&d_qw, (nb / 33 + 64) * sizeof(u64)) == cudaSuccess && cudaMalloc(&d_ql, (nb / 257 + 16) * sizeof(uint4)) == cudaSuccess;
-    ok = ok && cudaMemcpy(d_text, cat.data(), nb, cudaMemcpyHostToDevice) == cudaSuccess;
-    ok = ok && cudaMemcpy(d_mask, smask.data(), (nchunks + 1) * sizeof(u16), cudaMemcpyHostToDevice) == cudaSuccess;
-    ok = ok && cudaMemcpy(d_tf, tile_first.data(), (ntiles + 1) * sizeof(u32), cudaMemcpyHostToDevice) == cudaSuccess;
-    ok = ok && cudaMemcpy(d_hdr, &h, sizeof(h), cudaMemcpyHostToDevice) == cudaSuccess;
-    ok = ok && cudaMemset(d_tt, 0, (ntiles + 1) * sizeof(u32)) == cudaSuccess && cudaMemset(d_gt, 0, ngroups * sizeof(u32)) == cudaSuccess;
+              cudaMalloc(&d_hdr, sizeof(TTHeader)) == cudaSuccess;
+    ok = ok && cudaMemset(d_hdr, 0, sizeof(TTHeader)) == cudaSuccess && cudaMemset(d_tt, 0, (ntiles + 1) * sizeof(u32)) == cudaSuccess;
     if (ok) {
         PieceParams Q;
-        Q.base = d_text; Q.shift = 0; Q.hi = (long long)nb; Q.nchunks = (long long)nchunks; Q.ntiles = (int)ntiles;
-        Q.startmask = d_mask; Q.tile_first = d_tf; Q.hdr = d_hdr; Q.tab = v->tab;
+        Q.base = d_text; Q.shift = 0; Q.hi = (long long)nb; Q.ntiles = (int)ntiles;
+        Q.tile_cnt = d_tc; Q.tile_first = d_tf; Q.tile_last = d_tl; Q.tile_q = d_tq; Q.tile_long = d_lg; Q.piece_off16 = d_o16; Q.q = d_q;
+        Q.hdr = d_hdr; Q.epoch = next_epoch(); Q.tab = v->tab;
         Q.toktab.slots = nullptr; Q.toktab.mask = 0; Q.toktab.shift = 0;      // no table yet: every piece is merged
-        Q.longtab = LongTable{}; Q.litstart = nullptr; Q.epoch = next_epoch();
-        Q.ext_id = v->d_ext_id; Q.piece_cnt = d_cnt; Q.stage = d_stage; Q.pairbuf = nullptr; Q.tile_tok = d_tt; Q.grp_tok = d_gt; Q.q_short = d_qs; Q.q_warp = d_qw; Q.q_long = d_ql;
-        const int grid = (int)(ntiles < (size_t)v->sm_count * 8 ? ntiles : (size_t)v->sm_count * 8);
-        k_lookup<<<grid, LOOKUP_THREADS>>>(Q);
+        Q.longtab = LongTable{}; Q.litstart = nullptr;
+        Q.ext_id = v->d_ext_id; Q.piece_cnt = d_cnt; Q.stage = d_stage; Q.pairbuf = nullptr; Q.tile_tok = d_tt;
         k_merge<<<v->sm_count * MERGE_CTAS_PER_SM, MERGE_THREADS, MERGE_SMEM_BYTES>>>(Q);
         ok = cudaGetLastError() == cudaSuccess && cudaDeviceSynchronize() == cudaSuccess;
     }
     ok = ok && cudaMemcpy(cnt.data(), d_cnt, cnt.size() * sizeof(u32), cudaMemcpyDeviceToHost) == cudaSuccess;
     ok = ok && cudaMemcpy(stage.data(), d_stage, nb * sizeof(int32_t), cudaMemcpyDeviceToHost) == cudaSuccess;
-    cudaFree(d_qs); cudaFree(d_qw); cudaFree(d_ql); cudaFree(d_text); cudaFree(d_mask); cudaFree(d_gt); cudaFree(d_tf); cudaFree(d_tt); cudaFree(d_cnt); cudaFree(d_stage); cudaFree(d_hdr);
+    cudaFree(d_text); cudaFree(d_tc); cudaFree(d_tf); cudaFree(d_tl); cudaFree(d_tq); cudaFree(d_o16); cudaFree(d_q); cudaFree(d_lg); cudaFree(d_tt); cudaFree(d_cnt); cudaFree(d_stage); cudaFree(d_hdr);
     if (!ok) { cudaGetLastError(); return TT_ERR_CUDA; }
     for (size_t i = 0; i < np; i++) {
         const size_t tile = off[i] / TT_TILE_BYTES, slot = tile * TT_TILE_BYTES + (i - tile_base[tile]);   // pieces are indexed per tile
@@ -417,14 +424,15 @@ static size_t carve(TTWorkspace* w, void* base, size_t max_len, size_t max_docs)
     p = take(nchunks * sizeof(u16));            if (w) w->startmask = (u16*)p;
     p = take((ntiles + 1) * sizeof(u32));       if (w) w->tile_cnt = (u32*)p;
     p = take((ntiles + 1) * sizeof(u32));       if (w) w->tile_first = (u32*)p;
+    p = take((ntiles + 1) * sizeof(u32));       if (w) w->tile_last = (u32*)p;
     p = take((ntiles + 1) * sizeof(u32));       if (w) w->tile_tok = (u32*)p;
-    p = take((ntiles / TT_GROUP_TILES + 2) * sizeof(u32));   if (w) w->grp_tok = (u32*)p;
+    p = take((ntiles + 1) * sizeof(u32));       if (w) w->tile_q = (u32*)p;
+    p = take(ntiles * TT_TILE_LONGCAP * sizeof(u16));        if (w) w->tile_long = (u16*)p;
+    p = take(ntiles * TT_TILE_BYTES * sizeof(u16));          if (w) w->piece_off16 = (u16*)p;
     p = take(ntiles * TT_TILE_BYTES * sizeof(u32));          if (w) w->piece_cnt = (u32*)p;
+    p = take(ntiles * TT_TILE_QCAP * sizeof(u32));           if (w) w->q = (u32*)p;
     p = take((max_len + 1) * sizeof(int32_t));  if (w) w->stage = (int32_t*)p;
     p = take((max_len + 1) * sizeof(u64));      if (w) w->pairbuf = (u64*)p;
-    p = take((max_len / 2 + 64) * sizeof(u64)); if (w) w->q_short = (u64*)p;
-    p = take((max_len / 33 + 64) * sizeof(u64)); if (w) w->q_warp = (u64*)p;
-    p = take((max_len / 257 + 16) * sizeof(uint4)); if (w) w->q_long = (uint4*)p;
     p = take(padded + 16);                      if (w) w->cand = (u8*)p;
     p = take((padded / 32 + 4) * sizeof(u32));  if (w) w->litstart = (u32*)p;
     p = take((padded / 32 + 4) * sizeof(u32));  if (w) w->litin = (u32*)p;
@@ -442,7 +450,7 @@ extern "C" size_t tt_workspace_bytes(const tt_vocab* v, size_t max_len, size_t m
 // Enqueues K1+K2 (and K3 when piece_off_dst is given: only tt_pretokenize materialises the offsets;
 // the encode chain derives them per tile from the start flags).
 static int run_pretok(const tt_vocab* v, const uint8_t* text, size_t len, const int64_t* doc_off, size_t n_docs,
-                      cudaStream_t st, TTWorkspace& w, u32* piece_off_dst, PretokParams& P, bool literals = false) {
+                      cudaStream_t st, TTWorkspace& w, u32* piece_off_dst, PretokParams& P, bool literals = false, bool fused = false) {
     const uintptr_t addr = (uintptr_t)text;
     const long long shift = (long long)(addr & 15);
     P.base = (const u8*)(addr - shift);
@@ -451,7 +459,7 @@ static int run_pretok(const tt_vocab* v, const uint8_t* text, size_t len, const 
     P.ntiles = (int)((P.nchunks + TT_TILE_CHUNKS - 1) / TT_TILE_CHUNKS);
     P.pattern = v->pattern; P.epoch = next_epoch();
     P.docmask = nullptr; P.litstart = nullptr; P.litin = nullptr;
-    P.startmask = w.startmask; P.tile_cnt = w.tile_cnt; P.tile_first = w.tile_first; P.tile_tok = w.tile_tok; P.grp_tok = w.grp_tok; P.want_prefix = piece_off_dst != nullptr; P.hdr = w.hdr;
+    P.startmask = w.startmask; P.tile_cnt = w.tile_cnt; P.tile_first = w.tile_first; P.want_prefix = piece_off_dst != nullptr; P.hdr = w.hdr;
     P.cls_tables = v->d_cls; P.cls_bytes = v->cls_bytes;
     if (doc_off) {
         CK(cudaMemsetAsync(w.docmask, 0, ((size_t)P.hi / 32 + 4) * sizeof(u32), st));
@@ -480,12 +488,17 @@ static int run_pretok(const tt_vocab* v, const uint8_t* text, size_t len, const 
         // stages A and B: span starts into cutmask (with the caller's document starts); stage C: pattern 0 with
         // those cuts as its document boundaries
         PretokParams C1 = P;
-        C1.pattern = TT_PATTERN_CUTS; C1.startmask = reinterpret_cast<u16*>(w.cutmask); C1.tile_tok = nullptr; C1.grp_tok = nullptr;
+        C1.pattern = TT_PATTERN_CUTS; C1.startmask = reinterpret_cast<u16*>(w.cutmask);
         C1.want_prefix = 0; C1.litstart = nullptr; C1.litin = nullptr;
-        k_pretok<<<grid, TT_TILE_CHUNKS, smem, st>>>(C1);
+        k_pretok<false><<<grid, TT_TILE_CHUNKS, smem, st>>>(C1, FrontParams{});
         P.pattern = TT_PATTERN_CL100K; P.docmask = w.cutmask;
     }
-    k_pretok<<<grid, TT_TILE_CHUNKS, smem, st>>>(P);
+    if (fused) {
+        FrontParams F;
+        F.tile_last = w.tile_last; F.tile_tok = w.tile_tok; F.tile_q = w.tile_q; F.tile_long = w.tile_long; F.piece_off16 = w.piece_off16;
+        F.piece_cnt = w.piece_cnt; F.q = w.q; F.toktab = v->toktab; F.longtab = v->longtab; F.ext_id = v->d_ext_id;
+        k_pretok<true><<<grid, TT_TILE_CHUNKS, smem, st>>>(P, F);
+    } else k_pretok<false><<<grid, TT_TILE_CHUNKS, smem, st>>>(P, FrontParams{});
     if (piece_off_dst)
         k_compact<<<grid, TT_TILE_CHUNKS, 0, st>>>(w.startmask, w.tile_cnt, P.nchunks, P.ntiles, shift, (long long)len,
                                                    piece_off_dst, w.hdr, P.epoch);
@@ -529,39 +542,37 @@ static int encode_impl(const tt_vocab* v, const uint8_t* text, size_t len, const
         CK(cudaMemsetAsync(status_out, 0, sizeof(int32_t), st));
         return TT_OK;
     }
-    // The header's counters are zeroed by the first kernel and its status word is tagged with the call's epoch,
-    // so a single request starts with its first kernel.  The passes in front of it (document mask, literals) and
-    // a stream capture (whose replays repeat the epoch) clear the header first.
+    // Nothing is cleared in front of the chain: the status word of the header is tagged with the call's epoch, the
+    // one counter of the chain (k_merge's tickets) is zeroed by the kernel before it, and every per-tile record has
+    // exactly one writer.  A stream capture (whose replays repeat the epoch) clears the header first.
     cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
     if (cudaStreamIsCapturing(st, &cap) != cudaSuccess) { cudaGetLastError(); cap = cudaStreamCaptureStatusActive; }
     if (doc_off || literals || cap != cudaStreamCaptureStatusNone) CK(cudaMemsetAsync(w.hdr, 0, sizeof(TTHeader), st));
     MARK(0);
     PretokParams PP;
-    int rc = run_pretok(v, text, len, doc_off, n_docs, st, w, nullptr, PP, literals);
+    int rc = run_pretok(v, text, len, doc_off, n_docs, st, w, nullptr, PP, literals, true);
     if (rc != TT_OK) return rc;
     MARK(1);
     const int tile_grid = PP.ntiles < v->sm_count * 8 ? PP.ntiles : v->sm_count * 8;
     const int merge_grid = v->sm_count * MERGE_CTAS_PER_SM;                  // all resident CTA slots: a request's unsettled pieces get a warp each
     PieceParams Q;
-    Q.base = PP.base; Q.shift = PP.lo; Q.hi = PP.hi; Q.nchunks = PP.nchunks; Q.ntiles = PP.ntiles;
-    Q.startmask = w.startmask; Q.tile_first = w.tile_first; Q.hdr = w.hdr; Q.tab = v->tab; Q.toktab = v->toktab; Q.longtab = v->longtab; Q.litstart = literals ? w.litstart : nullptr; Q.epoch = PP.epoch;
-    Q.ext_id = v->d_ext_id; Q.piece_cnt = w.piece_cnt; Q.stage = w.stage; Q.pairbuf = w.pairbuf; Q.tile_tok = w.tile_tok; Q.grp_tok = w.grp_tok;
-    Q.q_short = w.q_short; Q.q_warp = w.q_warp; Q.q_long = w.q_long;
-    if (ev) k_lookup<<<tile_grid, LOOKUP_THREADS, 0, st>>>(Q);
-    else CK(launch_after(k_lookup, tile_grid, LOOKUP_THREADS, st, Q));
-    MARK(2);
+    Q.base = PP.base; Q.shift = PP.lo; Q.hi = PP.hi; Q.ntiles = PP.ntiles;
+    Q.tile_cnt = w.tile_cnt; Q.tile_first = w.tile_first; Q.tile_last = w.tile_last; Q.tile_q = w.tile_q; Q.tile_long = w.tile_long;
+    Q.piece_off16 = w.piece_off16; Q.q = w.q;
+    Q.hdr = w.hdr; Q.tab = v->tab; Q.toktab = v->toktab; Q.longtab = v->longtab; Q.litstart = literals ? w.litstart : nullptr; Q.epoch = PP.epoch;
+    Q.ext_id = v->d_ext_id; Q.piece_cnt = w.piece_cnt; Q.stage = w.stage; Q.pairbuf = w.pairbuf; Q.tile_tok = w.tile_tok;
     if (ev) k_merge<<<merge_grid, MERGE_THREADS, MERGE_SMEM_BYTES, st>>>(Q);
     else CK(launch_after(k_merge, merge_grid, MERGE_THREADS, st, Q, MERGE_SMEM_BYTES));
-    MARK(3);
+    MARK(2);
     ScatterParams S;
-    S.shift = PP.lo; S.hi = PP.hi; S.nchunks = PP.nchunks; S.ntiles = PP.ntiles; S.startmask = w.startmask;
-    S.tile_first = w.tile_first; S.tile_tok = w.tile_tok; S.grp_tok = w.grp_tok; S.ids_cap = (unsigned long long)ids_cap; S.piece_cnt = w.piece_cnt; S.stage = w.stage; S.hdr = w.hdr; S.epoch = PP.epoch;
+    S.shift = PP.lo; S.hi = PP.hi; S.ntiles = PP.ntiles; S.tile_cnt = w.tile_cnt; S.tile_tok = w.tile_tok; S.piece_off16 = w.piece_off16;
+    S.ids_cap = (unsigned long long)ids_cap; S.piece_cnt = w.piece_cnt; S.stage = w.stage; S.hdr = w.hdr; S.epoch = PP.epoch;
     S.ids_out = ids_out; S.count_out = (long long*)count_out; S.status_out = status_out;
     S.docmask = doc_off ? w.docmask : nullptr; S.doc_off = (const long long*)doc_off; S.n_docs = (int)n_docs;
     S.ids_off_out = (long long*)ids_off_out;
     if (ev) k_scatter<<<tile_grid, BPE_THREADS, 0, st>>>(S);
     else CK(launch_after(k_scatter, tile_grid, BPE_THREADS, st, S));
-    MARK(4);
+    MARK(3);
 #undef MARK
     CK(cudaGetLastError());
     return TT_OK;
@@ -652,18 +663,18 @@ extern "C" int tt_encode_batch(const tt_vocab* v, const uint8_t* text, size_t to
 
 extern "C" int tt_encode_timed(const tt_vocab* v, const uint8_t* text, size_t len, void* stream, int32_t* ids_out,
                                size_t ids_cap, int64_t* count_out, int32_t* status_out, void* workspace,
-                               size_t workspace_bytes, float ms_out[4]) {
+                               size_t workspace_bytes, float ms_out[3]) {
     int rc = check_common(v, text, len, workspace, workspace_bytes, 1);
     if (rc != TT_OK) return rc;
     if (!count_out || !status_out || !ms_out || !len || !ids_out) return TT_ERR_ARG;
-    cudaEvent_t ev[5];
-    for (int i = 0; i < 5; i++) CK(cudaEventCreate(&ev[i]));
+    cudaEvent_t ev[4];
+    for (int i = 0; i < 4; i++) CK(cudaEventCreate(&ev[i]));
     rc = encode_impl(v, text, len, nullptr, 1, (cudaStream_t)stream, ids_out, ids_cap, count_out, nullptr, status_out,
                      workspace, ev);
-    if (rc == TT_OK && cudaEventSynchronize(ev[4]) != cudaSuccess) rc = TT_ERR_CUDA;
-    for (int i = 0; i < 4 && rc == TT_OK; i++)
+    if (rc == TT_OK && cudaEventSynchronize(ev[3]) != cudaSuccess) rc = TT_ERR_CUDA;
+    for (int i = 0; i < 3 && rc == TT_OK; i++)
         if (cudaEventElapsedTime(&ms_out[i], ev[i], ev[i + 1]) != cudaSuccess) rc = TT_ERR_CUDA;
-    for (int i = 0; i < 5; i++) cudaEventDestroy(ev[i]);
+    for (int i = 0; i < 4; i++) cudaEventDestroy(ev[i]);
     return rc;
 }
 

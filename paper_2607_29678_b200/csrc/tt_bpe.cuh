@@ -687,263 +687,333 @@ __device__ u32 cta_merge_long(const u8* __restrict__ text, u32 a, u32 n, const P
 }
 #undef AX
 
-// ---- pieces of one text tile -----------------------------------------------------------------------------
-// The start flags of a tile (TT_TILE_CHUNKS u16 masks) become a list of in-tile piece offsets in shared
-// memory; the end of the tile's last piece is the next start flag after the tile (or the text end).
-constexpr int TILE_MAX_PIECES = TT_TILE_BYTES;
+// ---- what the first kernel (tag + piece starts + whole-piece lookups) leaves per tile -----------------------
+// See TTWorkspace.  A queue entry of a tile names one unsettled piece of at most 256 bytes that lies inside the
+// tile: offset in the tile | index among the tile's pieces << 11 | (bytes - 1) << 22.  The tile's LAST piece is
+// never settled by the first kernel (its end is the next piece start, which another CTA finds): k_merge
+// settles it, looking the end up in tile_first of the following tiles.
+__device__ __forceinline__ u32 tile_queue_entry(u32 off, u32 idx, u32 n) { return off | (idx << 11) | ((n - 1) << 22); }
+constexpr u32 TQ_NS_MASK = 0x7FFu, TQ_NW_SHIFT = 11, TQ_NW_MASK = 0x7Fu, TQ_NL_SHIFT = 18, TQ_NL_MASK = 0xFu;
 
-struct TilePieces {
-    u16 off[TILE_MAX_PIECES];      // byte offset of each piece inside the tile (aligned frame)
-    u32 n;                         // pieces that start in the tile
-    u32 end;                       // end of the last piece, relative to the tile start (may lie far beyond the tile)
-};
-
-__device__ void tile_pieces(TilePieces& tp, const u16* __restrict__ startmask, const u32* __restrict__ tile_first,
-                            long long nchunks, int ntiles, int tile, long long hi /* end of text, aligned frame */, u32* s_scr) {
-    const int tid = threadIdx.x;
-    const long long c0 = (long long)tile * TT_TILE_CHUNKS;
-    u32 m = 0;
-    if (tid < TT_TILE_CHUNKS && c0 + tid < nchunks) m = startmask[c0 + tid];
-    if (tid == 0) {
-        // the next start after the tile: the first start of the next tile that has one, else the text end
-        u32 end = (u32)(hi - c0 * TT_CHUNK);
-        for (int t = tile + 1; t < ntiles; t++) {
-            const u32 f = tile_first[t];
-            if (f != 0xFFFFFFFFu) { end = (u32)(t - tile) * TT_TILE_BYTES + f; break; }
-        }
-        tp.end = end;
-    }
-    u32 tot;
-    u32 r = cta_excl_sum_scan(__popc(m), s_scr, &tot);
-    while (m) { const int i = __ffs(m) - 1; m &= m - 1; tp.off[r++] = (u16)(tid * TT_CHUNK + i); }
-    if (tid == 0) tp.n = tot;
-    __syncthreads();
-}
-
-// ---- K4, first half: whole-piece lookups of a text tile; unsettled pieces go to global queues -----------------
-// A thread per piece: one-byte pieces map directly, pieces of up to 24 bytes are looked up as whole
-// vocabulary entries (two pieces per thread and step, their loads side by side).  What stays unsettled is
-// appended to one of three queues in the workspace (one atomic reservation per tile and queue):
-//   q_short  pieces of <= 32 bytes,  q_warp  pieces of 33..256 bytes,  q_long  longer pieces.
-// Token totals of the settled pieces go to the per-tile and per-group counters.  This kernel holds no merge
-// code, so it runs at full occupancy; k_merge then has every warp of the GPU drawing from the same queues.
-// Without a token table (while the table itself is being built) every piece is queued.
 struct PieceParams {
     const u8* base;            // aligned frame origin (text = base + shift)
     long long shift, hi;       // text occupies [shift, hi)
-    long long nchunks;
     int ntiles;
-    const u16* startmask;
-    const u32* tile_first;     // offset of the first piece start inside every tile (~0: none)
+    const u32* tile_cnt;
+    const u32* tile_first;
+    const u32* tile_last;
+    const u32* tile_q;
+    const u16* tile_long;
+    const u16* piece_off16;
+    const u32* q;
     TTHeader* hdr;
     unsigned long long epoch;
     PairTable tab;
-    TokTable toktab;
+    TokTable toktab;           // slots == nullptr: no whole-piece table (while the table itself is being built)
     const u32* litstart;       // literal pass: a piece that begins at such a bit is an added token whose id is staged, or null
     LongTable longtab;         // ignore_merges: entries longer than the whole-piece table holds (else slots == nullptr)
     const int32_t* ext_id;
-    u32* piece_cnt;            // per piece: the id itself if the piece is one token found without merging (>= 0),
-                               // else minus the number of tokens staged at the piece's text offset
+    u32* piece_cnt;
     int32_t* stage;            // ids staged at the text offset of their piece
     u64* pairbuf;              // global scratch of the long-piece path, indexed like the text
-    u32* tile_tok;             // in: zero; out: tokens per tile
-    u32* grp_tok;              // in: zero; out: tokens per group of TT_GROUP_TILES tiles
-    u64* q_short; u64* q_warp; // queue entries: text offset | index in tile << 32 | (bytes - 1) << 43
-    uint4* q_long;             // (text offset, bytes, piece index, 0)
+    u32* tile_tok;
 };
 
-__device__ __forceinline__ u64 queue_entry(u32 a, u32 i, u32 n) { return (u64)a | ((u64)i << 32) | ((u64)(n - 1) << 43); }
-
-#ifndef TT_LOOKUP_THREADS_DEF
-#define TT_LOOKUP_THREADS_DEF 256
-#endif
-constexpr int LOOKUP_THREADS = TT_LOOKUP_THREADS_DEF;
-__global__ void __launch_bounds__(LOOKUP_THREADS, 1536 / LOOKUP_THREADS)
-k_lookup(const PieceParams P) {
-    __shared__ TilePieces tp;
-    __shared__ u16 s_short[TILE_MAX_PIECES];                  // short misses from the front, long pieces from the back
-    __shared__ u16 s_warp[TT_TILE_BYTES / (LANE_MAX + 1) + 2];
-    __shared__ u32 s_ns, s_nw, s_nl, s_total, s_bs, s_bw, s_bl;
-    __shared__ u32 sc[48];
-    const int tid = threadIdx.x;
-    cudaTriggerProgrammaticLaunchCompletion();               // the next kernel may be placed; it waits for this grid's memory itself
-    if (P.toktab.slots != nullptr) grid_prefetch_l2(P.toktab.slots, ((size_t)P.toktab.mask + 1) * sizeof(TokSlot));
-    cudaGridDependencySynchronize();                         // k_pretok's flags and counts are complete from here on
-    const int status = hdr_status(P.hdr, P.epoch);           // looked at after the first tile's flags are in: the loads overlap
-    const u8* text = P.base + P.shift;
-    for (int tile = blockIdx.x; tile < P.ntiles; tile += gridDim.x) {
-        const long long c0 = (long long)tile * TT_TILE_CHUNKS;
-        __syncthreads();
-        if (tid == 0) { s_ns = 0; s_nw = 0; s_nl = 0; s_total = 0; }
-        tile_pieces(tp, P.startmask, P.tile_first, P.nchunks, P.ntiles, tile, P.hi, sc);
-        if (status != 0) return;                                  // nothing global has been written yet
-        const u32 np = tp.n, p0 = (u32)tile * TT_TILE_BYTES;     // pieces are indexed per tile
-        const long long t0 = c0 * TT_CHUNK - P.shift;             // text offset of the tile start
-        u32 wsum = 0;
-        // two pieces per thread and step, their loads issued side by side: first the bytes of both, then the
-        // table slots of both (each lookup is a chain of two dependent loads)
-        for (u32 ib = tid; ib < np; ib += 2 * LOOKUP_THREADS) {
-            u32 a[2], n[2], h[2], kind[2];                        // kind: 0 none, 1 literal, 2 one byte, 3 table lookup, 4 other
-            u64 k0[2], k1[2], k2[2];
-            uint4 lo[2], hi[2];
-#pragma unroll
-            for (int j = 0; j < 2; j++) {
-                const u32 i = ib + j * LOOKUP_THREADS;
-                kind[j] = 0; a[j] = 0; n[j] = 0; k0[j] = 0; k1[j] = 0; k2[j] = 0;
-                if (i < np) {
-                    a[j] = (u32)(t0 + tp.off[i]);
-                    n[j] = (i + 1 < np ? tp.off[i + 1] : tp.end) - tp.off[i];
-                    const long long g = (long long)a[j] + P.shift;
-                    if (P.litstart != nullptr && ((P.litstart[g >> 5] >> (g & 31)) & 1)) kind[j] = 1;
-                    else if (n[j] == 1) { kind[j] = 2; k0[j] = text[a[j]]; }
-                    else if (n[j] <= TT_TOKTAB_MAXLEN && P.toktab.slots != nullptr) { kind[j] = 3; toktab_key(text, a[j], n[j], k0[j], k1[j], k2[j]); }
-                    else kind[j] = 4;
-                }
-            }
-#pragma unroll
-            for (int j = 0; j < 2; j++) {
-                h[j] = 0; lo[j] = make_uint4(0, 0, 0, 0); hi[j] = lo[j];
-                if (kind[j] == 3) {
-                    h[j] = toktab_hash(k0[j], k1[j], k2[j], n[j], P.toktab.shift);
-                    const uint4* sp = reinterpret_cast<const uint4*>(P.toktab.slots + h[j]);
-                    lo[j] = __ldg(sp); hi[j] = __ldg(sp + 1);
-                } else if (kind[j] == 2) lo[j].x = (u32)P.ext_id[(u32)k0[j]];
-            }
-#pragma unroll
-            for (int j = 0; j < 2; j++) {
-                const u32 i = ib + j * LOOKUP_THREADS;
-                int32_t id;
-                if (kind[j] == 0) continue;
-                if (kind[j] == 1) { P.piece_cnt[p0 + i] = 0u - 1u; wsum++; }     // one staged id (written by the literal pass)
-                else if (kind[j] == 2) { P.piece_cnt[p0 + i] = lo[j].x; wsum++; }
-                else if (kind[j] == 3 && toktab_finish(P.toktab, k0[j], k1[j], k2[j], n[j], h[j], lo[j], hi[j], id)) {
-                    P.piece_cnt[p0 + i] = (u32)id; wsum++;
-                } else if (n[j] > TT_TOKTAB_MAXLEN && P.longtab.slots != nullptr && n[j] <= P.longtab.maxlen && longtab_lookup(P.longtab, text, a[j], n[j], id)) {
-                    P.piece_cnt[p0 + i] = (u32)id; wsum++;
-                } else if (n[j] > TT_WARP_PIECE_MAX) s_short[TILE_MAX_PIECES - 1 - atomicAdd(&s_nl, 1u)] = (u16)i;
-                else if (n[j] > LANE_MAX) s_warp[atomicAdd(&s_nw, 1u)] = (u16)i;
-                else s_short[atomicAdd(&s_ns, 1u)] = (u16)i;
-            }
-        }
-        for (int o = 16; o; o >>= 1) wsum += __shfl_xor_sync(0xFFFFFFFFu, wsum, o);
-        if ((tid & 31) == 0 && wsum) atomicAdd(&s_total, wsum);
-        __syncthreads();
-        const u32 ns = s_ns, nw = s_nw, nl = s_nl;
-        // the three reservations wait for their answers side by side, in different warps
-        if (tid == 0 && ns) s_bs = atomicAdd(&P.hdr->nq_short, ns);
-        if (tid == 32 && nw) s_bw = atomicAdd(&P.hdr->nq_warp, nw);
-        if (tid == 64 && nl) s_bl = atomicAdd(&P.hdr->nq_long, nl);
-        if (tid == 96 && s_total) { atomicAdd(&P.tile_tok[tile], s_total); atomicAdd(&P.grp_tok[tile >> TT_GROUP_SHIFT], s_total); }
-        if (ns | nw | nl) {                                       // block-uniform
-            __syncthreads();
-            for (u32 e = tid; e < ns + nw + nl; e += LOOKUP_THREADS) {
-                const u32 i = e < ns ? s_short[e] : e < ns + nw ? s_warp[e - ns] : s_short[TILE_MAX_PIECES - 1 - (e - ns - nw)];
-                const u32 a = (u32)(t0 + tp.off[i]);
-                const u32 n = (i + 1 < np ? tp.off[i + 1] : tp.end) - tp.off[i];
-                if (e < ns) P.q_short[s_bs + e] = queue_entry(a, i, n);
-                else if (e < ns + nw) P.q_warp[s_bw + (e - ns)] = queue_entry(a, i, n);
-                else P.q_long[s_bl + (e - ns - nw)] = make_uint4(a, n, p0 + i, 0u);
-            }
-        }
-    }
-}
-
 // ---- K4, second half: the merges ------------------------------------------------------------------------------
-// Long pieces (> 256 bytes) first, a CTA each.  Then every warp works on its own: it takes the pieces of
-// 33..256 bytes one at a time (the longest chains, so they start first), then the pieces of <= 32 bytes --
-// one at a time with the tokens in registers if the whole call has few of them (the shortest chain per piece:
-// a request's latency is its longest chain), else 32 at a time, a thread per piece.  A queue entry within the
-// grid's warp count belongs to the warp of that index; entries beyond it are handed out by global tickets, so
-// all warps of the GPU stay busy until the queues are empty; no barrier after the long pieces.
+// Work of this kernel: the unsettled pieces the first kernel queued per tile, and the last piece of every tile.
+//   (A) pieces of more than 256 bytes, a whole CTA each: every CTA looks through a contiguous share of the
+//       tiles (the in-tile long pieces the first kernel listed, and tile-closing pieces that turn out long).
+//   (B) everything else, warp by warp, without any barrier:
+//       - a request (few tiles, few unsettled pieces): job j belongs to warp j of the grid.  Jobs are numbered
+//         warp-class pieces first (the longest chains), then the tile-closing pieces, then the short pieces;
+//         a warp finds its job from the per-tile counts alone (every lane sums a stretch of tiles, one warp
+//         scan), so nothing is handed out through a counter.  One warp per piece, tokens in registers.
+//       - bulk text: warps draw tickets of 16 tiles and settle what those tiles left: short pieces 32 at a
+//         time, a thread each (lane_merge), warp-class pieces one at a time.
 constexpr int MERGE_WARPS = 8;
 constexpr int MERGE_THREADS = MERGE_WARPS * 32;
 constexpr int WARP_SMEM_WORDS = 1024;                 // u64 per warp: two lane-path arrays of 32 x 32 u32, or two copies of four 256-word merge arrays
 static_assert(MERGE_WARPS * WARP_SMEM_WORDS * sizeof(u64) >= LONG_SMEM_SLOTS * (sizeof(u64) + sizeof(u32)), "the CTA's buffer must hold a long piece");
 constexpr size_t MERGE_SMEM_BYTES = (size_t)MERGE_WARPS * WARP_SMEM_WORDS * sizeof(u64);   // dynamic shared memory of k_merge (64 KiB)
 static_assert(WARP_SMEM_WORDS * sizeof(u64) >= 2 * LANE_SLOTS * LANE_MAX * sizeof(u32) && WARP_SMEM_WORDS * sizeof(u64) >= 2 * 4 * TT_WARP_PIECE_MAX * sizeof(u32), "per-warp buffer");
+constexpr int MERGE_SR_MAX_TILES = 2048;              // the per-warp job search covers at most 32 lanes x 64 tiles
+constexpr int MERGE_TICKET_TILES = 16;                // tiles per ticket of the bulk mode
 
 #ifndef TT_MERGE_CTAS_PER_SM
 #define TT_MERGE_CTAS_PER_SM 3
 #endif
 constexpr int MERGE_CTAS_PER_SM = TT_MERGE_CTAS_PER_SM;   // resident CTAs per SM (registers and the 64 KiB of shared memory each)
+
+// End (aligned frame) of the piece that starts last in `tile`: the first piece start of a later tile, or the text end.
+__device__ __forceinline__ u32 closing_piece_end(const PieceParams& P, int tile) {
+    for (int t = tile + 1; t < P.ntiles; t++) {                   // bounded by the number of tiles
+        const u32 f = P.tile_first[t];
+        if (f != TT_NONE) return (u32)t * TT_TILE_BYTES + f;
+    }
+    return (u32)P.hi;
+}
+
+// A piece that needs no merging: an extracted literal (its id is staged already), a single byte, or a whole
+// vocabulary entry.  Returns true and the value for piece_cnt.  One thread.
+__device__ __forceinline__ bool piece_settled_without_merge(const PieceParams& P, const u8* __restrict__ text, u32 a, u32 n, u32& value) {
+    if (P.litstart != nullptr) {
+        const long long g = (long long)a + P.shift;
+        if ((P.litstart[g >> 5] >> (g & 31)) & 1) { value = 0u - 1u; return true; }
+    }
+    int32_t id;
+    if (n == 1) { value = (u32)P.ext_id[text[a]]; return true; }
+    if (n <= TT_TOKTAB_MAXLEN) {
+        if (P.toktab.slots != nullptr && toktab_lookup(P.toktab, text, a, n, id)) { value = (u32)id; return true; }
+    } else if (P.longtab.slots != nullptr && n <= P.longtab.maxlen && longtab_lookup(P.longtab, text, a, n, id)) { value = (u32)id; return true; }
+    return false;
+}
+
+__device__ __forceinline__ void piece_done(const PieceParams& P, u32 slot, u32 m) {
+    P.piece_cnt[slot] = 0u - m;
+    atomicAdd(&P.tile_tok[slot / TT_TILE_BYTES], m);
+}
+
+// One piece of 2..256 bytes, the whole warp.
+__device__ __forceinline__ bool piece_in_range(const PieceParams& P, u32 a, u32 n, u32 slot, u32 site) {
+    const bool ok = n >= 1 && (long long)a + n <= P.hi - P.shift && slot < (u32)P.ntiles * TT_TILE_BYTES;
+    if (!ok) hdr_selfcheck_failed(P.hdr, P.epoch, site, a, n, slot, 0u);
+    return ok;
+}
+__device__ __forceinline__ void warp_merge_piece(const PieceParams& P, const u8* __restrict__ text, u32 a, u32 n, u32 slot, u64* wbuf, int lane) {
+    if (!piece_in_range(P, a, n, slot, 1u) || n < 2 || n > (u32)TT_WARP_PIECE_MAX) { if (n < 2 || n > (u32)TT_WARP_PIECE_MAX) hdr_selfcheck_failed(P.hdr, P.epoch, 2u, a, n, slot, 0u); return; }
+    u32* const pbuf = reinterpret_cast<u32*>(wbuf);
+    const u32 m = n <= LANE_MAX ? warp_merge_reg(text, a, n, P.tab, P.ext_id, P.stage, lane)
+                : n <= 64 ? warp_merge_perm<2>(pbuf, text, a, n, P.tab, P.ext_id, P.stage, lane)
+                : n <= 128 ? warp_merge_perm<4>(pbuf, text, a, n, P.tab, P.ext_id, P.stage, lane)
+                           : warp_merge_perm<WCH>(pbuf, text, a, n, P.tab, P.ext_id, P.stage, lane);
+    if (lane == 0) piece_done(P, slot, m);
+}
+
+// Exclusive prefix over the lanes of a 64-bit value holding two counts (low 32 bits, high 32 bits); *total = warp sum.
+__device__ __forceinline__ u64 warp_exscan_u64(u64 v, int lane, u64* total) {
+    u64 x = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) { const u64 t = __shfl_up_sync(0xFFFFFFFFu, x, o); if (lane >= o) x += t; }
+    *total = __shfl_sync(0xFFFFFFFFu, x, 31);
+    return x - v;
+}
+
 __global__ void __launch_bounds__(MERGE_THREADS, MERGE_CTAS_PER_SM)
 k_merge(const PieceParams P) {
     extern __shared__ __align__(16) u64 s_buf[];              // MERGE_SMEM_BYTES
     __shared__ u32 sc[48];
+    __shared__ uint4 s_long[MERGE_THREADS];                   // long pieces found in one pass over the CTA's tiles
+    __shared__ u32 s_nlong;
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+    const u32 FULL = 0xFFFFFFFFu;
     cudaTriggerProgrammaticLaunchCompletion();               // k_scatter may be placed; it waits for this grid's memory itself
     grid_prefetch_l2(P.tab.slots, ((size_t)P.tab.mask + 1) * 2 * sizeof(uint4));
     grid_prefetch_l2(P.tab.bytepair, 65536 * sizeof(u64));
-    cudaGridDependencySynchronize();                         // the queues are complete from here on
+    cudaGridDependencySynchronize();                         // the first kernel's per-tile records are complete from here on
     if (hdr_status(P.hdr, P.epoch) != 0) return;
     const u8* text = P.base + P.shift;
-    const u32 ns = P.hdr->nq_short, nw = P.hdr->nq_warp, nl = P.hdr->nq_long;
-    for (u32 e = blockIdx.x; e < nl; e += gridDim.x) {            // block-uniform
-        const uint4 q = P.q_long[e];
-        const u32 m = cta_merge_long(text, q.x, q.y, P.tab, P.ext_id, P.stage, P.pairbuf + q.x, s_buf, sc);
-        if (tid == 0) {
-            const u32 tile = q.z / TT_TILE_BYTES;
-            P.piece_cnt[q.z] = 0u - m; atomicAdd(&P.tile_tok[tile], m); atomicAdd(&P.grp_tok[tile >> TT_GROUP_SHIFT], m);
+
+    // ---- (A) long pieces of this CTA's share of the tiles -------------------------------------------------------
+    {
+        const int per = (P.ntiles + (int)gridDim.x - 1) / (int)gridDim.x;
+        const int t_lo = (int)blockIdx.x * per, t_hi = min(P.ntiles, t_lo + per);
+        for (int t0 = t_lo; t0 < t_hi; t0 += MERGE_THREADS) {     // block-uniform
+            const int t = t0 + tid;
+            u32 nl = 0, np = 0, last = 0, next_first = TT_NONE;
+            if (t < t_hi) {
+                nl = (P.tile_q[t] >> TQ_NL_SHIFT) & TQ_NL_MASK; np = P.tile_cnt[t]; last = P.tile_last[t];
+                if (t + 1 < P.ntiles) next_first = P.tile_first[t + 1];
+            }
+            // the closing piece is long if it reaches more than 256 bytes beyond its start
+            bool closing_long = false;
+            u32 c_end = 0;
+            if (np) {
+                c_end = (t + 1 >= P.ntiles) ? (u32)P.hi : next_first != TT_NONE ? (u32)(t + 1) * TT_TILE_BYTES + next_first : closing_piece_end(P, t);
+                closing_long = c_end - ((u32)t * TT_TILE_BYTES + last) > (u32)TT_WARP_PIECE_MAX;
+            }
+            if (!__syncthreads_or(nl != 0 || closing_long)) continue;
+            // rare: tile after tile of this pass, so that the shared list cannot overflow
+            for (int k = 0; k < MERGE_THREADS && t0 + k < t_hi; k++) {    // block-uniform
+                __syncthreads();
+                if (tid == 0) s_nlong = 0;
+                __syncthreads();
+                if (tid == k) {
+                    u32 cnt = 0;
+                    for (u32 j = 0; j < nl; j++) {
+                        const u32 idx = P.tile_long[(size_t)t * TT_TILE_LONGCAP + j];
+                        const u32 o = P.piece_off16[(size_t)t * TT_TILE_BYTES + idx], o2 = P.piece_off16[(size_t)t * TT_TILE_BYTES + idx + 1];
+                        s_long[cnt++] = make_uint4((u32)((long long)t * TT_TILE_BYTES + o - P.shift), o2 - o, (u32)t * TT_TILE_BYTES + idx, 0u);
+                    }
+                    if (closing_long) {
+                        const u32 st = (u32)t * TT_TILE_BYTES + last;
+                        s_long[cnt++] = make_uint4((u32)((long long)st - P.shift), c_end - st, (u32)t * TT_TILE_BYTES + np - 1, 0u);
+                    }
+                    s_nlong = cnt;
+                }
+                __syncthreads();
+                const u32 cnt = s_nlong;
+                for (u32 e = 0; e < cnt; e++) {                   // block-uniform
+                    const uint4 q = s_long[e];
+                    __syncthreads();
+                    if (!piece_in_range(P, q.x, q.y, q.z, 3u)) continue;
+                    if (tid == 0) { u32 v; sc[47] = piece_settled_without_merge(P, text, q.x, q.y, v) ? 1u : 0u; sc[46] = v; }
+                    __syncthreads();
+                    if (sc[47]) { if (tid == 0) { P.piece_cnt[q.z] = sc[46]; atomicAdd(&P.tile_tok[q.z / TT_TILE_BYTES], 1u); } continue; }
+                    const u32 m = cta_merge_long(text, q.x, q.y, P.tab, P.ext_id, P.stage, P.pairbuf + q.x, s_buf, sc);
+                    if (tid == 0) piece_done(P, q.z, m);
+                }
+            }
+            __syncthreads();
         }
     }
-    if (nl > blockIdx.x) __syncthreads();
+
+    // ---- (B) everything of at most 256 bytes ----------------------------------------------------------------------
     u64* wbuf = s_buf + wid * WARP_SMEM_WORDS;
-    const u32 FULL = 0xFFFFFFFFu;
-    // Queue entry e belongs to warp e of the grid (numbered across the CTAs first, so that neighbouring entries
-    // run on different SMs); only what lies beyond the grid's warp count is handed out by ticket.  A request's
-    // few unsettled pieces thus start without an atomic round trip.
-    const u32 W = gridDim.x * MERGE_WARPS, gw = (u32)wid * gridDim.x + blockIdx.x;
-    for (u32 e = gw; e < nw;) {                                   // bounded by the queue length
-        const u64 q = P.q_warp[e];
-        const u32 a = (u32)q, i = (u32)(q >> 32) & 2047u, n = (u32)(q >> 43) + 1;
-        u32* const pbuf = reinterpret_cast<u32*>(wbuf);
-        const u32 m = n <= 64 ? warp_merge_perm<2>(pbuf, text, a, n, P.tab, P.ext_id, P.stage, lane)
-                    : n <= 128 ? warp_merge_perm<4>(pbuf, text, a, n, P.tab, P.ext_id, P.stage, lane)
-                               : warp_merge_perm<WCH>(pbuf, text, a, n, P.tab, P.ext_id, P.stage, lane);
-        if (lane == 0) {
-            const u32 tile = (u32)(((long long)a + P.shift) / TT_TILE_BYTES);
-            P.piece_cnt[tile * TT_TILE_BYTES + i] = 0u - m; atomicAdd(&P.tile_tok[tile], m); atomicAdd(&P.grp_tok[tile >> TT_GROUP_SHIFT], m);
+    const u32 W = gridDim.x * MERGE_WARPS, gw = (u32)wid * gridDim.x + blockIdx.x;   // numbered across the CTAs first
+    bool bulk = P.ntiles > MERGE_SR_MAX_TILES;
+    if (!bulk) {
+        // every lane sums the counts of a stretch of K tiles (K a multiple of 4), kept as sums of four tiles
+        const int K = ((P.ntiles + 31) / 32 + 3) & ~3;            // <= 64
+        u64 part[16];                                             // low word: short pieces, high word: warp-class pieces
+        u64 mine = 0;
+        const int tb = lane * K;
+#pragma unroll
+        for (int g = 0; g < 16; g++) {
+            u64 s4 = 0;
+            if (g * 4 < K) {
+#pragma unroll
+                for (int u = 0; u < 4; u++) {
+                    const int t = tb + g * 4 + u;
+                    if (t < P.ntiles) { const u32 q = P.tile_q[t]; s4 += (u64)(q & TQ_NS_MASK) | ((u64)((q >> TQ_NW_SHIFT) & TQ_NW_MASK) << 32); }
+                }
+            }
+            part[g] = s4; mine += s4;
         }
-        if (nw <= W) break;
-        if (lane == 0) e = W + atomicAdd(&P.hdr->t_warp, 1u);
-        e = __shfl_sync(FULL, e, 0);
-    }
-    // Measured crossover (1 M to 8 M chars of Unicode-heavy prose, 15 K to 120 K unsettled pieces): a warp per piece
-    // wins up to about 17 pieces per warp of the grid (29 against 64 us at 4 per warp, 44 against 63 us at 8).
+        u64 total;
+        const u64 before = warp_exscan_u64(mine, lane, &total);
+        const u32 NS = (u32)total, NW = (u32)(total >> 32), NT = (u32)P.ntiles;
 #ifndef TT_SHORT_WARP_FACTOR
 #define TT_SHORT_WARP_FACTOR 12u
 #endif
-    if (ns <= TT_SHORT_WARP_FACTOR * W) {                         // few: a warp per piece
-        const u32 nstatic = nw < W ? W - nw : 0u;                 // warps nw .. W-1 take the first entries
-        u32 e = gw >= nw ? gw - nw : ns;
-        for (;;) {
-            if (e < ns) {
-                const u64 q = P.q_short[e];
-                const u32 a = (u32)q, i = (u32)(q >> 32) & 2047u, n = (u32)(q >> 43) + 1;
-                const u32 m = warp_merge_reg(text, a, n, P.tab, P.ext_id, P.stage, lane);
-                if (lane == 0) {
-                    const u32 tile = (u32)(((long long)a + P.shift) / TT_TILE_BYTES);
-                    P.piece_cnt[tile * TT_TILE_BYTES + i] = 0u - m; atomicAdd(&P.tile_tok[tile], m); atomicAdd(&P.grp_tok[tile >> TT_GROUP_SHIFT], m);
+        // Measured crossover (1 M to 8 M chars of Unicode-heavy prose, 15 K to 120 K unsettled pieces): a warp per piece
+        // wins up to about 17 pieces per warp of the grid.
+        bulk = NS + NT > TT_SHORT_WARP_FACTOR * W;
+        if (!bulk) {
+            const u32 J = NW + NT + NS;
+            for (u32 j = gw; j < J; j += W) {                         // bounded by the number of jobs
+                u32 a, n, slot;
+                if (j >= NW && j < NW + NT) {                         // the closing piece of tile j - NW
+                    const int t = (int)(j - NW);
+                    const u32 np = P.tile_cnt[t];
+                    if (np == 0) continue;
+                    const u32 st = (u32)t * TT_TILE_BYTES + P.tile_last[t];
+                    n = closing_piece_end(P, t) - st;
+                    if (n > (u32)TT_WARP_PIECE_MAX) continue;         // settled by a CTA in (A)
+                    a = (u32)((long long)st - P.shift); slot = (u32)t * TT_TILE_BYTES + np - 1;
+                    u32 v;
+                    if (piece_settled_without_merge(P, text, a, n, v)) {     // every lane computes the same
+                        if (lane == 0) { P.piece_cnt[slot] = v; atomicAdd(&P.tile_tok[t], 1u); }
+                        continue;
+                    }
+                } else {
+                    // the k-th queued piece of its class: the lane whose stretch holds it finds the tile
+                    const bool wclass = j < NW;
+                    const u32 k = wclass ? j : j - NW - NT;
+                    const u32 bsel = wclass ? (u32)(before >> 32) : (u32)before;
+                    const u32 owner = 31u - (u32)__clz(__ballot_sync(FULL, bsel <= k) | 1u);
+                    u32 found = 0;                                    // tile << 11 | rank within the tile
+                    if ((u32)lane == owner) {
+                        u32 r = k - bsel;
+                        int g = 0;
+#pragma unroll
+                        for (int gg = 0; gg < 16; gg++) {
+                            const u32 c = wclass ? (u32)(part[gg] >> 32) : (u32)part[gg];
+                            if (g == gg && r >= c && gg < 15) { r -= c; g = gg + 1; }
+                        }
+                        int t = tb + g * 4;
+                        for (int u = 0; u < 4; u++) {
+                            const u32 q = t < P.ntiles ? P.tile_q[t] : 0u;
+                            const u32 c = wclass ? (q >> TQ_NW_SHIFT) & TQ_NW_MASK : q & TQ_NS_MASK;
+                            if (r < c || u == 3) break;
+                            r -= c; t++;
+                        }
+                        found = ((u32)t << 11) | r;
+                    }
+                    found = __shfl_sync(FULL, found, owner);
+                    const u32 t = found >> 11, r = found & 2047u;
+                    const u32 e = P.q[(size_t)t * TT_TILE_QCAP + (wclass ? (u32)TT_TILE_QCAP - 1 - r : r)];
+                    n = (e >> 22) + 1;
+                    a = (u32)((long long)t * TT_TILE_BYTES + (e & 2047u) - P.shift); slot = t * TT_TILE_BYTES + ((e >> 11) & 2047u);
                 }
+                warp_merge_piece(P, text, a, n, slot, wbuf, lane);
             }
-            if (ns <= nstatic) break;                             // every entry has its warp
-            if (lane == 0) e = nstatic + atomicAdd(&P.hdr->t_short, 1u);
-            e = __shfl_sync(FULL, e, 0);
-            if (e >= ns) break;
+            return;
         }
-    } else {                                                      // bulk: 32 pieces per warp and step, a thread each
-        u32* tok = reinterpret_cast<u32*>(wbuf);
-        for (;;) {
-            u32 e0 = 0;
-            if (lane == 0) e0 = atomicAdd(&P.hdr->t_short, (u32)LANE_SLOTS);
-            e0 = __shfl_sync(FULL, e0, 0);
-            if (e0 >= ns) break;
-            if (e0 + lane < ns) {
-                const u64 q = P.q_short[e0 + lane];
-                const u32 a = (u32)q, i = (u32)(q >> 32) & 2047u, n = (u32)(q >> 43) + 1;
-                const u32 m = lane_merge(tok, tok + LANE_SLOTS * LANE_MAX, lane, text, a, n, P.tab, P.ext_id, P.stage);
-                const u32 tile = (u32)(((long long)a + P.shift) / TT_TILE_BYTES);
-                P.piece_cnt[tile * TT_TILE_BYTES + i] = 0u - m; atomicAdd(&P.tile_tok[tile], m); atomicAdd(&P.grp_tok[tile >> TT_GROUP_SHIFT], m);
+    }
+    // bulk mode
+    u32* const tok = reinterpret_cast<u32*>(wbuf);
+    const u32 ntick = ((u32)P.ntiles + MERGE_TICKET_TILES - 1) / MERGE_TICKET_TILES;
+    for (;;) {                                                        // bounded by the number of tickets
+        u32 tk = 0;
+        if (lane == 0) tk = atomicAdd(&P.hdr->t_tiles, 1u);
+        tk = __shfl_sync(FULL, tk, 0);
+        if (tk >= ntick) break;
+        const int t = (int)(tk * MERGE_TICKET_TILES) + lane;              // lanes 0..15: a tile each
+        const bool have_tile = lane < MERGE_TICKET_TILES && t < P.ntiles;
+        u32 q = 0, np = 0;
+        if (have_tile) { q = P.tile_q[t]; np = P.tile_cnt[t]; }
+        const u32 ns = q & TQ_NS_MASK, nw = (q >> TQ_NW_SHIFT) & TQ_NW_MASK;
+        // the closing piece of my tile
+        u32 ca = 0, cn = 0, cslot = 0;                                    // cn == 0: nothing left to do for it
+        if (np) {
+            const u32 st = (u32)t * TT_TILE_BYTES + P.tile_last[t];
+            cn = closing_piece_end(P, t) - st;
+            ca = (u32)((long long)st - P.shift); cslot = (u32)t * TT_TILE_BYTES + np - 1;
+            u32 v;
+            if (cn > (u32)TT_WARP_PIECE_MAX) cn = 0;                      // settled by a CTA in (A)
+            else if (piece_settled_without_merge(P, text, ca, cn, v)) { P.piece_cnt[cslot] = v; atomicAdd(&P.tile_tok[t], 1u); cn = 0; }
+        }
+        // warp-class pieces, one at a time
+        const u32 wany = __ballot_sync(FULL, nw != 0 || cn > (u32)LANE_MAX);
+        for (u32 x = wany; x; x &= x - 1) {                               // warp-uniform
+            const int l = __ffs(x) - 1;
+            const u32 nw_l = __shfl_sync(FULL, nw, l), cn_l = __shfl_sync(FULL, cn, l), ca_l = __shfl_sync(FULL, ca, l), cs_l = __shfl_sync(FULL, cslot, l);
+            const u32 tl = tk * MERGE_TICKET_TILES + (u32)l;
+            for (u32 r = 0; r < nw_l; r++) {
+                const u32 e = P.q[(size_t)tl * TT_TILE_QCAP + (u32)TT_TILE_QCAP - 1 - r];
+                warp_merge_piece(P, text, (u32)((long long)tl * TT_TILE_BYTES + (e & 2047u) - P.shift), (e >> 22) + 1, tl * TT_TILE_BYTES + ((e >> 11) & 2047u), wbuf, lane);
+            }
+            if (cn_l > (u32)LANE_MAX) warp_merge_piece(P, text, ca_l, cn_l, cs_l, wbuf, lane);
+        }
+        if (cn > (u32)LANE_MAX) cn = 0;
+        // short pieces: the queued ones of the 16 tiles, then the short closing pieces, 32 per step, a thread each
+        u32 pre = ns;                                                     // exclusive prefix of ns over the lanes
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) { const u32 v = __shfl_up_sync(FULL, pre, o); if (lane >= o) pre += v; }
+        const u32 QS = __shfl_sync(FULL, pre, 31);
+        pre -= ns;
+        const u32 cm = __ballot_sync(FULL, cn != 0);
+        const u32 nj = QS + __popc(cm);
+        for (u32 b = 0; b < nj; b += 32) {                                // warp-uniform
+            const u32 e = b + lane;
+            u32 tl = 0, pl = 0;                                           // queued piece: its tile within the ticket, that tile's prefix
+#pragma unroll
+            for (int l = 1; l < MERGE_TICKET_TILES; l++) { const u32 p = __shfl_sync(FULL, pre, l); if (p <= e) { tl = (u32)l; pl = p; } }
+            const u32 src = select_bit(cm, e >= QS ? e - QS : 0u) & 31u;  // closing piece: the lane that holds it
+            const u32 ca_s = __shfl_sync(FULL, ca, src), cn_s = __shfl_sync(FULL, cn, src), cs_s = __shfl_sync(FULL, cslot, src);
+            if (e < nj) {
+                u32 a, n, slot;
+                if (e < QS) {
+                    const u32 tt = tk * MERGE_TICKET_TILES + tl;
+                    const u32 qe = P.q[(size_t)tt * TT_TILE_QCAP + (e - pl)];
+                    n = (qe >> 22) + 1;
+                    a = (u32)((long long)tt * TT_TILE_BYTES + (qe & 2047u) - P.shift); slot = tt * TT_TILE_BYTES + ((qe >> 11) & 2047u);
+                } else { a = ca_s; n = cn_s; slot = cs_s; }
+                if (!piece_in_range(P, a, n, slot, 4u) || n < 2 || n > (u32)LANE_MAX) hdr_selfcheck_failed(P.hdr, P.epoch, 5u, a, n, slot, e);
+                else {
+                    const u32 m = lane_merge(tok, tok + LANE_SLOTS * LANE_MAX, lane, text, a, n, P.tab, P.ext_id, P.stage);
+                    piece_done(P, slot, m);
+                }
             }
             __syncwarp();
         }
@@ -953,12 +1023,11 @@ k_merge(const PieceParams P) {
 // ---- K5: coalesced scatter of the staged ids, one text tile per CTA iteration ---------------------------------
 // Also writes the token offset of every document that starts in the tile (batch calls).
 struct ScatterParams {
-    long long shift, hi, nchunks;
+    long long shift, hi;
     int ntiles;
-    const u16* startmask;
-    const u32* tile_first;
+    const u32* tile_cnt;
     const u32* tile_tok;       // tokens per tile
-    const u32* grp_tok;        // tokens per group of TT_GROUP_TILES tiles
+    const u16* piece_off16;
     unsigned long long ids_cap;
     const u32* piece_cnt;
     const int32_t* stage;
@@ -975,26 +1044,24 @@ struct ScatterParams {
 
 __global__ void __launch_bounds__(BPE_THREADS)
 k_scatter(const ScatterParams P) {
-    __shared__ TilePieces tp;
     __shared__ u32 sc[48];
-    __shared__ u32 s_big[TILE_MAX_PIECES / 8][3];
+    __shared__ u32 s_big[TT_TILE_BYTES / 8][3];
     __shared__ u32 s_nbig;
     __shared__ unsigned long long s_sum[66];
     const int tid = threadIdx.x;
-    cudaGridDependencySynchronize();                         // k_merge's (and with it k_lookup's) results are complete from here on
-    // Each CTA takes a contiguous range of tiles.  Tokens before its first tile = the whole groups of tiles
-    // before it plus the tiles of its own group before it; the grand total (all groups) gives the count and
-    // the capacity check, which every CTA makes for itself.
+    cudaGridDependencySynchronize();                         // k_merge's (and with it the first kernel's) results are complete from here on
+    // Each CTA takes a contiguous range of tiles and sums the token counts of all tiles itself: those before its
+    // range give its first output position, all of them the count and the capacity check.
     const int per = (P.ntiles + (int)gridDim.x - 1) / (int)gridDim.x;
     const int tile_lo = (int)blockIdx.x * per, tile_hi = min(P.ntiles, tile_lo + per);
-    const int ngroups = (P.ntiles + TT_GROUP_TILES - 1) >> TT_GROUP_SHIFT, g_lo = tile_lo >> TT_GROUP_SHIFT;
     unsigned long long before = 0, total = 0;
-    for (int g = tid; g < ngroups; g += BPE_THREADS) {
-        const u32 x = P.grp_tok[g];
-        total += x;
-        if (g < g_lo) before += x;
+    for (int t0 = 0; t0 < P.ntiles; t0 += BPE_THREADS * 4) {
+        u32 x[4];
+#pragma unroll
+        for (int u = 0; u < 4; u++) { const int t = t0 + u * BPE_THREADS + tid; x[u] = t < P.ntiles ? P.tile_tok[t] : 0u; }
+#pragma unroll
+        for (int u = 0; u < 4; u++) { total += x[u]; if (t0 + u * BPE_THREADS + tid < tile_lo) before += x[u]; }
     }
-    for (int t = (g_lo << TT_GROUP_SHIFT) + tid; t < tile_lo; t += BPE_THREADS) before += P.tile_tok[t];
     cta_sum2_u64(before, total, s_sum);
     int status = hdr_status(P.hdr, P.epoch);
     if (status == 0 && total > P.ids_cap) status = 5;          // TT_ERR_CAPACITY
@@ -1014,28 +1081,30 @@ k_scatter(const ScatterParams P) {
     }
     u32 carry = (u32)before;
     for (int tile = tile_lo; tile < tile_hi; tile++) {
-        const long long c0 = (long long)tile * TT_TILE_CHUNKS;
         __syncthreads();
         if (tid == 0) s_nbig = 0;
-        tile_pieces(tp, P.startmask, P.tile_first, P.nchunks, P.ntiles, tile, P.hi, sc);
-        const u32 np = tp.n, p0 = (u32)tile * TT_TILE_BYTES;
-        const long long t0 = c0 * TT_CHUNK - P.shift;
+        const u32 np = P.tile_cnt[tile];
+        const size_t p0 = (size_t)tile * TT_TILE_BYTES;
+        const long long t0 = (long long)tile * TT_TILE_BYTES - P.shift;      // text offset of the tile start
         for (u32 b = 0; b < np; b += BPE_THREADS) {
             const u32 i = b + tid;
             const int32_t v = i < np ? (int32_t)P.piece_cnt[p0 + i] : 0;       // an id, or minus the staged count
             const u32 c = i < np ? (v >= 0 ? 1u : (u32)(-v)) : 0u;
+            const u32 off = (i < np && (v < 0 || P.docmask)) ? P.piece_off16[p0 + i] : 0u;
             u32 tot;
             const u32 dst = carry + cta_excl_sum_scan(c, sc, &tot);
-            if (i < np) {
-                const u32 src = (u32)(t0 + tp.off[i]);
+            if (i < np && ((unsigned long long)dst + c > total || (v < 0 && (long long)t0 + off + c > P.hi - P.shift))) {
+                hdr_selfcheck_failed(P.hdr, P.epoch, 6u, (u32)tile, i, (u32)v, dst);
+            } else if (i < np) {
+                const u32 src = (u32)(t0 + off);
                 if (v >= 0) P.ids_out[dst] = v;
                 else if (c <= 8) { for (u32 k = 0; k < c; k++) P.ids_out[dst + k] = P.stage[src + k]; }
                 else {
                     const u32 slot = atomicAdd(&s_nbig, 1u);
-                    if (slot < TILE_MAX_PIECES / 8) { s_big[slot][0] = src; s_big[slot][1] = dst; s_big[slot][2] = c; }
+                    if (slot < TT_TILE_BYTES / 8) { s_big[slot][0] = src; s_big[slot][1] = dst; s_big[slot][2] = c; }
                 }
                 if (P.docmask) {
-                    const long long g = c0 * TT_CHUNK + tp.off[i];
+                    const long long g = (long long)tile * TT_TILE_BYTES + off;
                     if ((P.docmask[g >> 5] >> (g & 31)) & 1) {
                         // every document that starts at this byte (empty ones included) gets this token offset
                         const long long want = g - P.shift;
@@ -1048,7 +1117,7 @@ k_scatter(const ScatterParams P) {
             carry += tot;
             __syncthreads();
         }
-        const u32 nbig = min(s_nbig, (u32)(TILE_MAX_PIECES / 8));
+        const u32 nbig = min(s_nbig, (u32)(TT_TILE_BYTES / 8));
         for (u32 e = 0; e < nbig; e++) {
             const u32 src = s_big[e][0], d2 = s_big[e][1], cc = s_big[e][2];
             for (u32 k = tid; k < cc; k += BPE_THREADS) P.ids_out[d2 + k] = P.stage[src + k];

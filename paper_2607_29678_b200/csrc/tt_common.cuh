@@ -23,8 +23,9 @@ constexpr int TT_CHUNK = 16;
 #endif
 constexpr int TT_TILE_CHUNKS = TT_TILE_CHUNKS_DEF;        // = threads per CTA
 constexpr int TT_TILE_BYTES = TT_CHUNK * TT_TILE_CHUNKS; // 2 KiB of text per tile
-constexpr int TT_GROUP_SHIFT = 8;                 // token totals are also kept per group of 256 tiles
-constexpr int TT_GROUP_TILES = 1 << TT_GROUP_SHIFT;
+constexpr int TT_TILE_QCAP = TT_TILE_BYTES / 2;  // unsettled pieces of <= 256 bytes a tile can have (each has >= 2 bytes)
+constexpr int TT_TILE_LONGCAP = 8;               // pieces of > 256 bytes that lie inside one tile
+constexpr u32 TT_NONE = 0xFFFFFFFFu;
 
 // ---- character class codes (two-stage Unicode table, see gen_unicode_table.py) ------------
 enum : u32 { CC_OTHER = 0, CC_MARK = 1, CC_SPACE = 2, CC_NUMBER = 3, CC_LOWER = 4, CC_UPPER = 5, CC_CASELESS = 6 };
@@ -36,14 +37,14 @@ constexpr u32 TT_RANK_INF = 0xFFFFFFFFu;
 constexpr u64 TT_SLOT_EMPTY = ~0ull;              // pair-table slot: (left << 38) | (right << 20) | rank
 constexpr int TT_WARP_PIECE_MAX = 256;            // bytes; longer pieces take the block-cooperative path
 
-// ---- workspace header (device memory; counters zeroed by the call's first kernel or a memset) ----
+// ---- workspace header (device memory) -----------------------------------------------------------
 struct TTHeader {
     unsigned long long status_tag;   // (epoch of the call << 8) | device-side error code of that call
-    u32 pretok_done;         // CTAs that finished the pre-tokenization pass (tt_pretokenize only)
+    u32 pretok_done;         // CTAs that finished the pre-tokenization pass (tt_pretokenize only; cleared by a memset)
     u32 n_pieces;            // number of pieces found (tt_pretokenize only)
-    u32 nq_short, nq_warp, nq_long;   // lengths of the queues of unsettled pieces (k_lookup)
-    u32 t_short, t_warp;     // tickets of k_merge: queue entries handed out beyond the ones that warps own by index
-    u32 pad[23];
+    u32 t_tiles;             // ticket counter of k_merge's bulk mode (groups of tiles handed out); zeroed by the kernel before it
+    u32 dbg[8];              // first failed self-check of a kernel: site, then up to seven values (diagnostics only)
+    u32 pad[19];
 };
 static_assert(sizeof(TTHeader) == 128, "header layout");
 
@@ -51,6 +52,13 @@ static_assert(sizeof(TTHeader) == 128, "header layout");
 // value left by an earlier call -- or whatever an unused workspace holds -- reads as TT_OK and a single
 // request needs no clearing pass before its first kernel.
 #if defined(__CUDACC__)
+// A kernel that finds one of its own indices out of range records where and what (first record wins), reports
+// TT_ERR_INTERNAL_TIMEOUT through the status word and skips the access.
+__device__ __forceinline__ void hdr_set_status(TTHeader* h, unsigned long long epoch, int code);
+__device__ __noinline__ void hdr_selfcheck_failed(TTHeader* h, unsigned long long epoch, u32 site, u32 v0, u32 v1, u32 v2, u32 v3) {
+    if (atomicCAS(&h->dbg[0], 0u, site) == 0u) { h->dbg[1] = v0; h->dbg[2] = v1; h->dbg[3] = v2; h->dbg[4] = v3; }
+    hdr_set_status(h, epoch, 6 /* TT_ERR_INTERNAL_TIMEOUT */);
+}
 __device__ __forceinline__ int hdr_status(const TTHeader* h, unsigned long long epoch) {
     const unsigned long long t = *reinterpret_cast<const volatile unsigned long long*>(&h->status_tag);
     return (t >> 8) == epoch ? (int)(t & 0xFF) : 0;
@@ -67,21 +75,36 @@ __device__ __forceinline__ void hdr_set_status(TTHeader* h, unsigned long long e
 }
 #endif
 
+// Per-tile records of the encode chain (all indexed by tile; a tile is TT_TILE_BYTES of the aligned frame).
+// Nothing here is a global counter: every array element has exactly one writer in the first kernel, so that
+// kernel needs neither atomics on global memory nor a clearing pass, and the layout does not depend on the
+// order in which CTAs run.
+//   tile_cnt[t]    pieces that start in the tile
+//   tile_first[t]  offset in the tile of its first piece start, TT_NONE if it has none
+//   tile_last[t]   offset in the tile of its last piece start (that piece ends in a later tile, or with the text)
+//   tile_tok[t]    tokens of the tile's pieces (the first kernel stores the settled ones, k_merge adds the rest)
+//   tile_q[t]      unsettled pieces: short (<= 32 B) count | warp-class (33..256 B) count << 11 | long count << 18
+//   piece_off16    [t * TT_TILE_BYTES + i]  offset in the tile of piece i
+//   piece_cnt      [t * TT_TILE_BYTES + i]  the id of piece i if it is one token found without merging (>= 0),
+//                                           else minus the number of ids staged at the piece's text offset
+//   q              [t * TT_TILE_QCAP ...]   queue entries of the tile: short pieces from the front, warp-class
+//                                           pieces from the back; entry = offset in tile | index << 11 | (bytes-1) << 22
+//   tile_long      [t * TT_TILE_LONGCAP + k] index of the k-th piece of > 256 bytes that lies inside the tile
 struct TTWorkspace {
     TTHeader* hdr;
     u32* docmask;      // bit per text byte: first byte of a document (batch only)
-    u16* startmask;    // bit per text byte: first byte of a piece (one u16 per chunk)
-    u32* tile_cnt;     // pieces per tile, then exclusive prefix (ntiles + 1)
-    u32* tile_first;   // offset of the first piece start inside each tile, ~0 if none (ntiles + 1)
-    u32* tile_tok;     // tokens per tile (ntiles + 1)
-    u32* grp_tok;      // tokens per group of TT_GROUP_TILES tiles
-    u32* piece_cnt;    // per piece, at tile * TT_TILE_BYTES + index inside the tile: its id (one token, no merging)
-                       // or minus the staged token count
+    u16* startmask;    // bit per text byte: first byte of a piece, one u16 per chunk (tt_pretokenize and the cut pass only)
+    u32* tile_cnt;     // (tt_pretokenize: then the exclusive prefix, ntiles + 1)
+    u32* tile_first;
+    u32* tile_last;
+    u32* tile_tok;
+    u32* tile_q;
+    u16* tile_long;
+    u16* piece_off16;
+    u32* piece_cnt;
+    u32* q;
     int32_t* stage;    // token ids staged at the byte offset of their piece (len)
     u64* pairbuf;      // (token, rank) pairs of the long-piece path, indexed like the text (len)
-    u64* q_short;      // unsettled pieces of <= 32 bytes (len / 2 + 64 entries)
-    u64* q_warp;       // unsettled pieces of 33..256 bytes (len / 33 + 64 entries)
-    uint4* q_long;     // unsettled longer pieces (len / 257 + 16 entries)
     u8* cand;          // literal pass: length of the longest added-token literal starting at each byte (aligned frame)
     u32* litstart;     // literal pass: bit per byte, first byte of an extracted literal
     u32* litin;        // literal pass: bit per byte, the other bytes of an extracted literal

@@ -29,11 +29,9 @@ struct PretokParams {
     const u32* docmask;      // bit per byte (aligned frame) marking document starts, or null (one document)
     const u32* litstart;     // literal pass: first bytes of extracted literals (each becomes exactly one piece), or null
     const u32* litin;        //               their other bytes (start nothing)
-    u16* startmask;          // out: one u16 per chunk
-    u32* tile_cnt;           // out: pieces per tile; replaced by the exclusive prefix (ntiles + 1 entries)
+    u16* startmask;          // out (flags-only kernel): one u16 per chunk
+    u32* tile_cnt;           // out: pieces per tile; flags-only kernel with want_prefix: replaced by the exclusive prefix (ntiles + 1)
     u32* tile_first;         // out: offset inside the tile of its first piece start, or ~0 if it has none
-    u32* tile_tok;           // out: zeroed (the piece kernel accumulates token totals per tile and per group
-    u32* grp_tok;            //      of tiles), or null
     int want_prefix;         // turn tile_cnt into its exclusive prefix and count the pieces (tt_pretokenize only)
     TTHeader* hdr;
     unsigned long long epoch; // of this call (see TTHeader)

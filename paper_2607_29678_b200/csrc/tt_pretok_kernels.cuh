@@ -3,6 +3,7 @@
 #pragma once
 #include "tt_pretok.cuh"
 #include "tt_pretok_p1.cuh"
+#include "tt_bpe.cuh"
 
 // ---- CTA-wide reductions over 256 threads (results broadcast to every thread) ---------------
 __device__ __forceinline__ long long cta_max_ll(long long v, long long* scratch /* >= 9 */) {
@@ -194,19 +195,40 @@ __device__ __forceinline__ void store_slot(u16 (*sm)[TT_SLOTS], int s, const Chu
     sm[F_NL][s] = m.nl; sm[F_SP][s] = m.sp; sm[F_AP][s] = m.ap; sm[F_SL][s] = m.sl; sm[F_DOC][s] = (u16)d;
 }
 
+// What the fused kernel needs beyond the piece-start predicate: the per-tile records it leaves (see TTWorkspace)
+// and the tables of the whole-piece lookups.
+struct FrontParams {
+    u32* tile_last; u32* tile_tok; u32* tile_q; u16* tile_long; u16* piece_off16; u32* piece_cnt; u32* q;
+    TokTable toktab;           // slots == nullptr: none
+    LongTable longtab;         // ignore_merges: entries longer than the whole-piece table holds (else slots == nullptr)
+    const int32_t* ext_id;
+};
+
+// FUSED = false: the start flags go to P.startmask, with the pieces per tile (tt_pretokenize and the cut pass of the
+// three-splitter composition).
+// FUSED = true (the encode chain's first kernel): the tile's flags stay in shared memory and become its list of
+// piece offsets (K3); every piece but the tile's last one -- whose end another tile knows -- is settled here if it
+// is a single byte, an extracted literal or a whole vocabulary entry (one 32-byte probe), and queued for k_merge
+// otherwise.  Everything a tile leaves behind has this CTA as its only writer: no atomics on global memory, no
+// counter that would have to be cleared before the call.
+template <bool FUSED>
 __global__ void __launch_bounds__(TT_TILE_CHUNKS, 6)
-k_pretok(const PretokParams P) {
+k_pretok(const PretokParams P, const FrontParams F) {
     extern __shared__ __align__(16) u8 smem_raw[];
     u8* tables = smem_raw;                                            // class tables
     u16 (*sm)[TT_SLOTS] = reinterpret_cast<u16 (*)[TT_SLOTS]>(smem_raw + ((P.cls_bytes + 15) & ~15));
     __shared__ long long scratch[40];
     __shared__ u32 s_need, s_first;
     __shared__ u32 s_islast;
+    __shared__ u16 s_off[FUSED ? TT_TILE_BYTES + 2 : 2];              // piece offsets of the tile
+    __shared__ u32 s_wtot[TT_TILE_CHUNKS / 32], s_ns, s_nw, s_nl, s_total;
 
     const int tid = threadIdx.x;
     cudaTriggerProgrammaticLaunchCompletion();               // the next kernel may be placed; it waits for this grid's memory itself
-    if (blockIdx.x == 0 && tid == 0) {                       // the counters of the kernels behind this one
-        P.hdr->nq_short = 0; P.hdr->nq_warp = 0; P.hdr->nq_long = 0; P.hdr->t_short = 0; P.hdr->t_warp = 0;
+    if (FUSED) {
+        if (blockIdx.x == 0 && tid == 0) P.hdr->t_tiles = 0;  // k_merge's ticket counter (k_merge touches it only after this grid)
+        // the whole-piece table is probed at random a few microseconds from now: ask for it to be brought into L2
+        if (F.toktab.slots != nullptr) grid_prefetch_l2(F.toktab.slots, ((size_t)F.toktab.mask + 1) * sizeof(TokSlot));
     }
     // the 128-byte ASCII table is always staged; the two-stage Unicode table only once a tile holds a
     // non-ASCII byte (pattern 1 stages it at once: its sparse matcher may read beyond the tile)
@@ -222,7 +244,7 @@ k_pretok(const PretokParams P) {
 
     for (int tile = blockIdx.x; tile < P.ntiles; tile += gridDim.x) {
         __syncthreads();
-        if (tid == 0) { s_need = 0; s_first = 0xFFFFFFFFu; }
+        if (tid == 0) { s_need = 0; s_first = 0xFFFFFFFFu; s_ns = 0; s_nw = 0; s_nl = 0; s_total = 0; }
         const long long c_first = (long long)tile * TT_TILE_CHUNKS;
         if (!tables_loaded) {                                         // block-uniform
             bool hi_bit = false;
@@ -310,19 +332,97 @@ k_pretok(const PretokParams P) {
             const long long chunk = c_first + tid;
             S = (S & ~(u32)reinterpret_cast<const u16*>(P.litin)[chunk]) | reinterpret_cast<const u16*>(P.litstart)[chunk];
         }
-        if (c_first + tid < P.nchunks) P.startmask[c_first + tid] = (u16)S;
-        if (S) atomicMin(&s_first, (u32)(tid * TT_CHUNK + tt_lobit(S)));
-        u32 total = cta_sum_u32(tt_popc(S), scratch);
+        if (!FUSED) {
+            if (c_first + tid < P.nchunks) P.startmask[c_first + tid] = (u16)S;
+            if (S) atomicMin(&s_first, (u32)(tid * TT_CHUNK + tt_lobit(S)));
+            u32 total = cta_sum_u32(tt_popc(S), scratch);
+            if (tid == 0) { P.tile_cnt[tile] = total; P.tile_first[tile] = s_first; }
+            continue;
+        }
+        // ---- K3 in shared memory: the tile's piece offsets ------------------------------------------------------
+        const int lane = tid & 31, wid = tid >> 5;
+        const u32 cnt = tt_popc(S);
+        u32 x = cnt;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) { const u32 t = __shfl_up_sync(0xFFFFFFFFu, x, o); if (lane >= o) x += t; }
+        if (lane == 31) s_wtot[wid] = x;
+        __syncthreads();
+        u32 np = 0, r = x - cnt;
+#pragma unroll
+        for (int w = 0; w < TT_TILE_CHUNKS / 32; w++) { const u32 v = s_wtot[w]; np += v; if (w < wid) r += v; }
+        for (u32 m = S; m; m &= m - 1) s_off[r++] = (u16)(tid * TT_CHUNK + tt_lobit(m));
+        __syncthreads();
+        const size_t p0 = (size_t)tile * TT_TILE_BYTES;              // pieces are indexed per tile
+        for (u32 i = tid; i < np; i += TT_TILE_CHUNKS) F.piece_off16[p0 + i] = s_off[i];
         if (tid == 0) {
-            P.tile_cnt[tile] = total; P.tile_first[tile] = s_first;
-            if (P.tile_tok) { P.tile_tok[tile] = 0; if ((tile & (TT_GROUP_TILES - 1)) == 0) P.grp_tok[tile >> TT_GROUP_SHIFT] = 0; }
+            P.tile_cnt[tile] = np;
+            P.tile_first[tile] = np ? (u32)s_off[0] : TT_NONE;
+            F.tile_last[tile] = np ? (u32)s_off[np - 1] : TT_NONE;
+        }
+        // ---- K4, first half: whole-piece lookups, a thread per piece, two pieces per thread and step (first the
+        // bytes of both, then the table slots of both: each lookup is a chain of two dependent loads).  The tile's
+        // last piece is left to k_merge.
+        const u8* text = P.base + P.lo;
+        const long long t0 = c_first * TT_CHUNK - P.lo;               // text offset of the tile start
+        const u32 nlook = np ? np - 1 : 0;
+        u32 wsum = 0;
+        for (u32 ib = tid; ib < nlook; ib += 2 * TT_TILE_CHUNKS) {
+            u32 a[2], n[2], h[2], kind[2];                            // kind: 0 none, 1 literal, 2 one byte, 3 table lookup, 4 other
+            u64 k0[2], k1[2], k2[2];
+            uint4 lo[2], hi[2];
+#pragma unroll
+            for (int j = 0; j < 2; j++) {
+                const u32 i = ib + j * TT_TILE_CHUNKS;
+                kind[j] = 0; a[j] = 0; n[j] = 0; k0[j] = 0; k1[j] = 0; k2[j] = 0;
+                if (i < nlook) {
+                    a[j] = (u32)(t0 + s_off[i]);
+                    n[j] = (u32)s_off[i + 1] - s_off[i];
+                    const long long g = (long long)a[j] + P.lo;
+                    if (P.litstart != nullptr && ((P.litstart[g >> 5] >> (g & 31)) & 1)) kind[j] = 1;
+                    else if (n[j] == 1) { kind[j] = 2; k0[j] = text[a[j]]; }
+                    else if (n[j] <= TT_TOKTAB_MAXLEN && F.toktab.slots != nullptr) { kind[j] = 3; toktab_key(text, a[j], n[j], k0[j], k1[j], k2[j]); }
+                    else kind[j] = 4;
+                }
+            }
+#pragma unroll
+            for (int j = 0; j < 2; j++) {
+                h[j] = 0; lo[j] = make_uint4(0, 0, 0, 0); hi[j] = lo[j];
+                if (kind[j] == 3) {
+                    h[j] = toktab_hash(k0[j], k1[j], k2[j], n[j], F.toktab.shift);
+                    const uint4* sp = reinterpret_cast<const uint4*>(F.toktab.slots + h[j]);
+                    lo[j] = __ldg(sp); hi[j] = __ldg(sp + 1);
+                } else if (kind[j] == 2) lo[j].x = (u32)F.ext_id[(u32)k0[j]];
+            }
+#pragma unroll
+            for (int j = 0; j < 2; j++) {
+                const u32 i = ib + j * TT_TILE_CHUNKS;
+                int32_t id;
+                if (kind[j] == 0) continue;
+                if (kind[j] == 1) { F.piece_cnt[p0 + i] = 0u - 1u; wsum++; }     // one staged id (written by the literal pass)
+                else if (kind[j] == 2) { F.piece_cnt[p0 + i] = lo[j].x; wsum++; }
+                else if (kind[j] == 3 && toktab_finish(F.toktab, k0[j], k1[j], k2[j], n[j], h[j], lo[j], hi[j], id)) {
+                    F.piece_cnt[p0 + i] = (u32)id; wsum++;
+                } else if (n[j] > TT_TOKTAB_MAXLEN && F.longtab.slots != nullptr && n[j] <= F.longtab.maxlen && longtab_lookup(F.longtab, text, a[j], n[j], id)) {
+                    F.piece_cnt[p0 + i] = (u32)id; wsum++;
+                } else if (n[j] > (u32)TT_WARP_PIECE_MAX) F.tile_long[(size_t)tile * TT_TILE_LONGCAP + atomicAdd(&s_nl, 1u)] = (u16)i;
+                else if (n[j] > (u32)LANE_MAX) F.q[(size_t)tile * TT_TILE_QCAP + (u32)TT_TILE_QCAP - 1 - atomicAdd(&s_nw, 1u)] = tile_queue_entry(s_off[i], i, n[j]);
+                else F.q[(size_t)tile * TT_TILE_QCAP + atomicAdd(&s_ns, 1u)] = tile_queue_entry(s_off[i], i, n[j]);
+            }
+        }
+#pragma unroll
+        for (int o = 16; o; o >>= 1) wsum += __shfl_xor_sync(0xFFFFFFFFu, wsum, o);
+        if (lane == 0 && wsum) atomicAdd(&s_total, wsum);
+        __syncthreads();
+        if (tid == 0) {
+            F.tile_tok[tile] = s_total;
+            F.tile_q[tile] = s_ns | (s_nw << TQ_NW_SHIFT) | (s_nl << TQ_NL_SHIFT);
         }
     }
     if (any_bad) hdr_set_status(P.hdr, P.epoch, 4 /* TT_ERR_INVALID_UTF8 */);
 
     // the last CTA to finish turns the tile counts into their exclusive prefix (only where the piece list is
     // materialised: the encode chain indexes its pieces per tile and needs no prefix)
-    if (!P.want_prefix) return;
+    if (FUSED || !P.want_prefix) return;
     __threadfence();
     __syncthreads();
     if (tid == 0) s_islast = (atomicAdd(&P.hdr->pretok_done, 1u) == gridDim.x - 1);

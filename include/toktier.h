@@ -92,6 +92,13 @@ int tt_vocab_load_ex(const tt_merge* merges, size_t n_merges, const int32_t byte
 void tt_vocab_free(tt_vocab* v);
 
 /*
+ * tt_vocab_table_entries -- number of vocabulary entries in the whole-piece table of `v` (paper Sec. 4.2 keeps
+ * the vocabulary entries in a hash table on the GPU): the entries of at most 24 bytes whose own byte string
+ * encodes to exactly that entry, i.e. the pieces that one table probe settles.  Host value, no device work.
+ */
+size_t tt_vocab_table_entries(const tt_vocab* v);
+
+/*
  * tt_workspace_bytes -- DEVICE scratch size needed by an encode call over at most max_len text
  * bytes in at most max_docs documents (use 1 for tt_encode).  The caller allocates the scratch
  * (256-byte aligned) and may reuse it for any number of calls that do not overlap in time.

@@ -19,7 +19,7 @@ TT_STATIC_MAX_LEN = 262144
 TT_PATTERN_CL100K, TT_PATTERN_O200K, TT_PATTERN_CL100K_N1, TT_PATTERN_SPLIT3 = 0, 1, 2, 3
 TT_VOCAB_IGNORE_MERGES = 1
 
-EXPORTS = ["tt_vocab_load", "tt_vocab_load_ex", "tt_vocab_free", "tt_workspace_bytes", "tt_encode", "tt_encode_batch",
+EXPORTS = ["tt_vocab_load", "tt_vocab_load_ex", "tt_vocab_free", "tt_vocab_table_entries", "tt_workspace_bytes", "tt_encode", "tt_encode_batch",
            "tt_pretokenize", "tt_encode_timed", "tt_encode_host", "tt_encode_static", "tt_spans", "tt_spans_workspace_bytes", "tt_class_table", "tt_strerror",
            "tt_session_create", "tt_session_free", "tt_session_set_window", "tt_session_append", "tt_session_view", "tt_session_copy", "tt_vocab_add_literals", "tt_encode_added",
            "tt_pair_info_host", "tt_verifier_create", "tt_verifier_submit", "tt_verifier_drain", "tt_verifier_get_stats", "tt_verifier_quarantined", "tt_verifier_free"]
@@ -49,6 +49,8 @@ def lib() -> ctypes.CDLL:
         L.tt_vocab_load_ex.argtypes = [c.c_void_p, c.c_size_t, c.c_void_p, c.c_int, c.c_uint, c.POINTER(c.c_void_p)]
         L.tt_vocab_free.restype = None
         L.tt_vocab_free.argtypes = [c.c_void_p]
+        L.tt_vocab_table_entries.restype = c.c_size_t
+        L.tt_vocab_table_entries.argtypes = [c.c_void_p]
         L.tt_workspace_bytes.restype = c.c_size_t
         L.tt_workspace_bytes.argtypes = [c.c_void_p, c.c_size_t, c.c_size_t]
         L.tt_encode.restype = c.c_int
@@ -173,6 +175,10 @@ class Vocab:
             self.close()
         except Exception:
             pass
+
+    def table_entries(self) -> int:
+        """tt_vocab_table_entries: vocabulary entries that one probe of the whole-piece table settles."""
+        return int(lib().tt_vocab_table_entries(self._h))
 
     # -- sizes -------------------------------------------------------------------------------
     def workspace_bytes(self, max_len: int, max_docs: int = 1) -> int:

@@ -194,7 +194,7 @@ static int build_token_table(tt_vocab* v, const tt_merge* merges, size_t n_merge
         Q.hdr = d_hdr; Q.epoch = next_epoch(); Q.tab = v->tab;
         Q.toktab.slots = nullptr; Q.toktab.mask = 0; Q.toktab.shift = 0;      // no table yet: every piece is merged
         Q.longtab = LongTable{}; Q.litstart = nullptr;
-        Q.ext_id = v->d_ext_id; Q.piece_cnt = d_cnt; Q.stage = d_stage; Q.pairbuf = nullptr; Q.tile_tok = d_tt;
+        Q.ext_id = v->d_ext_id; Q.piece_cnt = d_cnt; Q.stage = d_stage; Q.pairbuf = nullptr; Q.tile_tok = d_tt; Q.grp_tok = nullptr; Q.wq = nullptr; Q.nwq = nullptr;
         k_merge<<<v->sm_count * MERGE_CTAS_PER_SM, MERGE_THREADS, MERGE_SMEM_BYTES>>>(Q);
         ok = cudaGetLastError() == cudaSuccess && cudaDeviceSynchronize() == cudaSuccess;
     }
@@ -231,6 +231,8 @@ static int build_token_table(tt_vocab* v, const tt_merge* merges, size_t n_merge
     v->n_table_tokens = keep.size();
     return TT_OK;
 }
+
+extern "C" size_t tt_vocab_table_entries(const tt_vocab* v) { return v ? v->n_table_tokens : 0; }
 
 extern "C" int tt_vocab_load(const tt_merge* merges, size_t n_merges, const int32_t byte_map[256], int pattern_id,
                              tt_vocab** out) {
@@ -427,10 +429,12 @@ static size_t carve(TTWorkspace* w, void* base, size_t max_len, size_t max_docs)
     p = take((ntiles + 1) * sizeof(u32));       if (w) w->tile_last = (u32*)p;
     p = take((ntiles + 1) * sizeof(u32));       if (w) w->tile_tok = (u32*)p;
     p = take((ntiles + 1) * sizeof(u32));       if (w) w->tile_q = (u32*)p;
+    p = take((ntiles / TT_GROUP_TILES + 2) * sizeof(u32));   if (w) w->grp_tok = (u32*)p;
     p = take(ntiles * TT_TILE_LONGCAP * sizeof(u16));        if (w) w->tile_long = (u16*)p;
     p = take(ntiles * TT_TILE_BYTES * sizeof(u16));          if (w) w->piece_off16 = (u16*)p;
     p = take(ntiles * TT_TILE_BYTES * sizeof(u32));          if (w) w->piece_cnt = (u32*)p;
     p = take(ntiles * TT_TILE_QCAP * sizeof(u32));           if (w) w->q = (u32*)p;
+    p = take((max_len / 33 + 64) * sizeof(u64));             if (w) w->wq = (u64*)p;
     p = take((max_len + 1) * sizeof(int32_t));  if (w) w->stage = (int32_t*)p;
     p = take((max_len + 1) * sizeof(u64));      if (w) w->pairbuf = (u64*)p;
     p = take(padded + 16);                      if (w) w->cand = (u8*)p;
@@ -497,6 +501,7 @@ static int run_pretok(const tt_vocab* v, const uint8_t* text, size_t len, const 
         FrontParams F;
         F.tile_last = w.tile_last; F.tile_tok = w.tile_tok; F.tile_q = w.tile_q; F.tile_long = w.tile_long; F.piece_off16 = w.piece_off16;
         F.piece_cnt = w.piece_cnt; F.q = w.q; F.toktab = v->toktab; F.longtab = v->longtab; F.ext_id = v->d_ext_id;
+        F.wq = P.ntiles > MERGE_SR_MAX_TILES ? w.wq : nullptr;
         k_pretok<true><<<grid, TT_TILE_CHUNKS, smem, st>>>(P, F);
     } else k_pretok<false><<<grid, TT_TILE_CHUNKS, smem, st>>>(P, FrontParams{});
     if (piece_off_dst)
@@ -547,7 +552,10 @@ static int encode_impl(const tt_vocab* v, const uint8_t* text, size_t len, const
     // exactly one writer.  A stream capture (whose replays repeat the epoch) clears the header first.
     cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
     if (cudaStreamIsCapturing(st, &cap) != cudaSuccess) { cudaGetLastError(); cap = cudaStreamCaptureStatusActive; }
-    if (doc_off || literals || cap != cudaStreamCaptureStatusNone) CK(cudaMemsetAsync(w.hdr, 0, sizeof(TTHeader), st));
+    // Bulk text (more tiles than a request's job search covers) uses one counter in the first kernel itself, the length
+    // of the global list of warp-class pieces: there the header is cleared too.
+    const bool big = (((uintptr_t)text & 15) + len + TT_TILE_BYTES - 1) / TT_TILE_BYTES > (size_t)MERGE_SR_MAX_TILES;
+    if (doc_off || literals || big || cap != cudaStreamCaptureStatusNone) CK(cudaMemsetAsync(w.hdr, 0, sizeof(TTHeader), st));
     MARK(0);
     PretokParams PP;
     int rc = run_pretok(v, text, len, doc_off, n_docs, st, w, nullptr, PP, literals, true);
@@ -561,11 +569,13 @@ static int encode_impl(const tt_vocab* v, const uint8_t* text, size_t len, const
     Q.piece_off16 = w.piece_off16; Q.q = w.q;
     Q.hdr = w.hdr; Q.tab = v->tab; Q.toktab = v->toktab; Q.longtab = v->longtab; Q.litstart = literals ? w.litstart : nullptr; Q.epoch = PP.epoch;
     Q.ext_id = v->d_ext_id; Q.piece_cnt = w.piece_cnt; Q.stage = w.stage; Q.pairbuf = w.pairbuf; Q.tile_tok = w.tile_tok;
+    Q.grp_tok = PP.ntiles > MERGE_SR_MAX_TILES ? w.grp_tok : nullptr;   // group totals only where k_scatter's CTAs would otherwise sum thousands of tiles each
+    Q.wq = PP.ntiles > MERGE_SR_MAX_TILES ? w.wq : nullptr; Q.nwq = &w.hdr->nwq;
     if (ev) k_merge<<<merge_grid, MERGE_THREADS, MERGE_SMEM_BYTES, st>>>(Q);
     else CK(launch_after(k_merge, merge_grid, MERGE_THREADS, st, Q, MERGE_SMEM_BYTES));
     MARK(2);
     ScatterParams S;
-    S.shift = PP.lo; S.hi = PP.hi; S.ntiles = PP.ntiles; S.tile_cnt = w.tile_cnt; S.tile_tok = w.tile_tok; S.piece_off16 = w.piece_off16;
+    S.shift = PP.lo; S.hi = PP.hi; S.ntiles = PP.ntiles; S.tile_cnt = w.tile_cnt; S.tile_tok = w.tile_tok; S.grp_tok = Q.grp_tok; S.piece_off16 = w.piece_off16;
     S.ids_cap = (unsigned long long)ids_cap; S.piece_cnt = w.piece_cnt; S.stage = w.stage; S.hdr = w.hdr; S.epoch = PP.epoch;
     S.ids_out = ids_out; S.count_out = (long long*)count_out; S.status_out = status_out;
     S.docmask = doc_off ? w.docmask : nullptr; S.doc_off = (const long long*)doc_off; S.n_docs = (int)n_docs;

@@ -717,6 +717,9 @@ struct PieceParams {
     int32_t* stage;            // ids staged at the text offset of their piece
     u64* pairbuf;              // global scratch of the long-piece path, indexed like the text
     u32* tile_tok;
+    u32* grp_tok;              // bulk text: tokens per group of TT_GROUP_TILES tiles (written by the last CTA), else null
+    const u64* wq;             // bulk text: the warp-class pieces of all tiles (tile << 32 | queue entry), else null
+    const u32* nwq;            //            their number
 };
 
 // ---- K4, second half: the merges ------------------------------------------------------------------------------
@@ -728,8 +731,9 @@ struct PieceParams {
 //         warp-class pieces first (the longest chains), then the tile-closing pieces, then the short pieces;
 //         a warp finds its job from the per-tile counts alone (every lane sums a stretch of tiles, one warp
 //         scan), so nothing is handed out through a counter.  One warp per piece, tokens in registers.
-//       - bulk text: warps draw tickets of 16 tiles and settle what those tiles left: short pieces 32 at a
-//         time, a thread each (lane_merge), warp-class pieces one at a time.
+//       - bulk text: the warp-class pieces stand in one global list (they come in clusters; a list lets every warp
+//         take its share), then warps draw tickets of one tile and settle its short pieces 32 at a time, a thread
+//         each (lane_merge); pieces wait in the lanes across tickets until 32 are together.
 constexpr int MERGE_WARPS = 8;
 constexpr int MERGE_THREADS = MERGE_WARPS * 32;
 constexpr int WARP_SMEM_WORDS = 1024;                 // u64 per warp: two lane-path arrays of 32 x 32 u32, or two copies of four 256-word merge arrays
@@ -737,7 +741,6 @@ static_assert(MERGE_WARPS * WARP_SMEM_WORDS * sizeof(u64) >= LONG_SMEM_SLOTS * (
 constexpr size_t MERGE_SMEM_BYTES = (size_t)MERGE_WARPS * WARP_SMEM_WORDS * sizeof(u64);   // dynamic shared memory of k_merge (64 KiB)
 static_assert(WARP_SMEM_WORDS * sizeof(u64) >= 2 * LANE_SLOTS * LANE_MAX * sizeof(u32) && WARP_SMEM_WORDS * sizeof(u64) >= 2 * 4 * TT_WARP_PIECE_MAX * sizeof(u32), "per-warp buffer");
 constexpr int MERGE_SR_MAX_TILES = 2048;              // the per-warp job search covers at most 32 lanes x 64 tiles
-constexpr int MERGE_TICKET_TILES = 16;                // tiles per ticket of the bulk mode
 
 #ifndef TT_MERGE_CTAS_PER_SM
 #define TT_MERGE_CTAS_PER_SM 3
@@ -798,225 +801,277 @@ __device__ __forceinline__ u64 warp_exscan_u64(u64 v, int lane, u64* total) {
     return x - v;
 }
 
+// Long pieces of the tiles [t_lo, t_hi) (at most MERGE_THREADS of them), a whole CTA each.  Called by all threads
+// of the CTA with the records of tile t_lo + tid in nl / np / last / c_end / closing_long.
+__device__ void cta_long_pieces(const PieceParams& P, const u8* __restrict__ text, int t_lo, int t_hi, u32 nl, u32 np, u32 last, u32 c_end,
+                                bool closing_long, u64* s_buf, u32* sc, uint4* s_long, u32* s_nlong) {
+    const int tid = threadIdx.x;
+    for (int k = 0; k < MERGE_THREADS && t_lo + k < t_hi; k++) {      // block-uniform; tile after tile, so that the shared list cannot overflow
+        if (!__syncthreads_or(tid == k && (nl != 0 || closing_long))) continue;
+        if (tid == k) {
+            const int t = t_lo + k;
+            u32 cnt = 0;
+            for (u32 j = 0; j < nl && j < (u32)TT_TILE_LONGCAP; j++) {
+                const u32 idx = P.tile_long[(size_t)t * TT_TILE_LONGCAP + j];
+                const u32 o = P.piece_off16[(size_t)t * TT_TILE_BYTES + idx], o2 = P.piece_off16[(size_t)t * TT_TILE_BYTES + idx + 1];
+                s_long[cnt++] = make_uint4((u32)((long long)t * TT_TILE_BYTES + o - P.shift), o2 - o, (u32)t * TT_TILE_BYTES + idx, 0u);
+            }
+            if (closing_long) {
+                const u32 st = (u32)t * TT_TILE_BYTES + last;
+                s_long[cnt++] = make_uint4((u32)((long long)st - P.shift), c_end - st, (u32)t * TT_TILE_BYTES + np - 1, 0u);
+            }
+            *s_nlong = cnt;
+        }
+        __syncthreads();
+        const u32 cnt = *s_nlong;
+        for (u32 e = 0; e < cnt; e++) {                               // block-uniform
+            const uint4 q = s_long[e];
+            __syncthreads();
+            if (!piece_in_range(P, q.x, q.y, q.z, 3u)) continue;
+            if (tid == 0) { u32 v = 0; sc[47] = piece_settled_without_merge(P, text, q.x, q.y, v) ? 1u : 0u; sc[46] = v; }
+            __syncthreads();
+            if (sc[47]) { if (tid == 0) { P.piece_cnt[q.z] = sc[46]; atomicAdd(&P.tile_tok[q.z / TT_TILE_BYTES], 1u); } continue; }
+            const u32 m = cta_merge_long(text, q.x, q.y, P.tab, P.ext_id, P.stage, P.pairbuf + q.x, s_buf, sc);
+            if (tid == 0) piece_done(P, q.z, m);
+        }
+    }
+    __syncthreads();
+}
+
 __global__ void __launch_bounds__(MERGE_THREADS, MERGE_CTAS_PER_SM)
 k_merge(const PieceParams P) {
     extern __shared__ __align__(16) u64 s_buf[];              // MERGE_SMEM_BYTES
     __shared__ u32 sc[48];
-    __shared__ uint4 s_long[MERGE_THREADS];                   // long pieces found in one pass over the CTA's tiles
-    __shared__ u32 s_nlong;
+    __shared__ uint4 s_long[TT_TILE_LONGCAP + 2];             // the long pieces of one tile
+    __shared__ u32 s_nlong, s_warps_done;
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
     const u32 FULL = 0xFFFFFFFFu;
     cudaTriggerProgrammaticLaunchCompletion();               // k_scatter may be placed; it waits for this grid's memory itself
     grid_prefetch_l2(P.tab.slots, ((size_t)P.tab.mask + 1) * 2 * sizeof(uint4));
     grid_prefetch_l2(P.tab.bytepair, 65536 * sizeof(u64));
+    if (tid == 0) s_warps_done = 0;
     cudaGridDependencySynchronize();                         // the first kernel's per-tile records are complete from here on
     if (hdr_status(P.hdr, P.epoch) != 0) return;
     const u8* text = P.base + P.shift;
 
-    // ---- (A) long pieces of this CTA's share of the tiles -------------------------------------------------------
+    // ---- records of this CTA's share of the tiles (long pieces, a whole CTA each; a request settles them after
+    // its short pieces, bulk text before); the loads go out next to those of the job search below
+    const int per = (P.ntiles + (int)gridDim.x - 1) / (int)gridDim.x;
+    const int t_lo = (int)blockIdx.x * per, t_hi = min(P.ntiles, t_lo + per);
+    u32 a_nl = 0, a_np = 0, a_last = 0, a_next = TT_NONE;
     {
-        const int per = (P.ntiles + (int)gridDim.x - 1) / (int)gridDim.x;
-        const int t_lo = (int)blockIdx.x * per, t_hi = min(P.ntiles, t_lo + per);
-        for (int t0 = t_lo; t0 < t_hi; t0 += MERGE_THREADS) {     // block-uniform
-            const int t = t0 + tid;
-            u32 nl = 0, np = 0, last = 0, next_first = TT_NONE;
-            if (t < t_hi) {
-                nl = (P.tile_q[t] >> TQ_NL_SHIFT) & TQ_NL_MASK; np = P.tile_cnt[t]; last = P.tile_last[t];
-                if (t + 1 < P.ntiles) next_first = P.tile_first[t + 1];
-            }
-            // the closing piece is long if it reaches more than 256 bytes beyond its start
-            bool closing_long = false;
-            u32 c_end = 0;
-            if (np) {
-                c_end = (t + 1 >= P.ntiles) ? (u32)P.hi : next_first != TT_NONE ? (u32)(t + 1) * TT_TILE_BYTES + next_first : closing_piece_end(P, t);
-                closing_long = c_end - ((u32)t * TT_TILE_BYTES + last) > (u32)TT_WARP_PIECE_MAX;
-            }
-            if (!__syncthreads_or(nl != 0 || closing_long)) continue;
-            // rare: tile after tile of this pass, so that the shared list cannot overflow
-            for (int k = 0; k < MERGE_THREADS && t0 + k < t_hi; k++) {    // block-uniform
-                __syncthreads();
-                if (tid == 0) s_nlong = 0;
-                __syncthreads();
-                if (tid == k) {
-                    u32 cnt = 0;
-                    for (u32 j = 0; j < nl; j++) {
-                        const u32 idx = P.tile_long[(size_t)t * TT_TILE_LONGCAP + j];
-                        const u32 o = P.piece_off16[(size_t)t * TT_TILE_BYTES + idx], o2 = P.piece_off16[(size_t)t * TT_TILE_BYTES + idx + 1];
-                        s_long[cnt++] = make_uint4((u32)((long long)t * TT_TILE_BYTES + o - P.shift), o2 - o, (u32)t * TT_TILE_BYTES + idx, 0u);
-                    }
-                    if (closing_long) {
-                        const u32 st = (u32)t * TT_TILE_BYTES + last;
-                        s_long[cnt++] = make_uint4((u32)((long long)st - P.shift), c_end - st, (u32)t * TT_TILE_BYTES + np - 1, 0u);
-                    }
-                    s_nlong = cnt;
-                }
-                __syncthreads();
-                const u32 cnt = s_nlong;
-                for (u32 e = 0; e < cnt; e++) {                   // block-uniform
-                    const uint4 q = s_long[e];
-                    __syncthreads();
-                    if (!piece_in_range(P, q.x, q.y, q.z, 3u)) continue;
-                    if (tid == 0) { u32 v; sc[47] = piece_settled_without_merge(P, text, q.x, q.y, v) ? 1u : 0u; sc[46] = v; }
-                    __syncthreads();
-                    if (sc[47]) { if (tid == 0) { P.piece_cnt[q.z] = sc[46]; atomicAdd(&P.tile_tok[q.z / TT_TILE_BYTES], 1u); } continue; }
-                    const u32 m = cta_merge_long(text, q.x, q.y, P.tab, P.ext_id, P.stage, P.pairbuf + q.x, s_buf, sc);
-                    if (tid == 0) piece_done(P, q.z, m);
-                }
-            }
-            __syncthreads();
+        const int t = t_lo + tid;
+        if (t < t_hi) {
+            a_nl = (P.tile_q[t] >> TQ_NL_SHIFT) & TQ_NL_MASK; a_np = P.tile_cnt[t]; a_last = P.tile_last[t];
+            if (t + 1 < P.ntiles) a_next = P.tile_first[t + 1];
         }
     }
-
-    // ---- (B) everything of at most 256 bytes ----------------------------------------------------------------------
     u64* wbuf = s_buf + wid * WARP_SMEM_WORDS;
     const u32 W = gridDim.x * MERGE_WARPS, gw = (u32)wid * gridDim.x + blockIdx.x;   // numbered across the CTAs first
-    bool bulk = P.ntiles > MERGE_SR_MAX_TILES;
-    if (!bulk) {
-        // every lane sums the counts of a stretch of K tiles (K a multiple of 4), kept as sums of four tiles
-        const int K = ((P.ntiles + 31) / 32 + 3) & ~3;            // <= 64
-        u64 part[16];                                             // low word: short pieces, high word: warp-class pieces
-        u64 mine = 0;
-        const int tb = lane * K;
+    const bool big = P.wq != nullptr;                             // more than MERGE_SR_MAX_TILES tiles
+    // job search of a request: every lane sums the counts of a stretch of tiles, kept as 16 sums of `unit` tiles
+    // (short pieces in the low half, warp-class pieces in the high half of a word)
+    const int unit = (P.ntiles + 511) / 512;                      // 1..4 tiles per register
+    const int tb = lane * 16 * unit;
+    u32 part[16];
+    u32 my_s = 0, my_w = 0;
+    if (!big) {
+        if (unit == 1) {                                          // up to 512 tiles: sixteen counts per lane, four vector loads
+            const uint4* src = reinterpret_cast<const uint4*>(P.tile_q + tb);
+            uint4 v[4];
 #pragma unroll
-        for (int g = 0; g < 16; g++) {
-            u64 s4 = 0;
-            if (g * 4 < K) {
+            for (int g = 0; g < 4; g++) v[g] = tb + 4 * g < P.ntiles ? src[g] : make_uint4(0, 0, 0, 0);
 #pragma unroll
-                for (int u = 0; u < 4; u++) {
-                    const int t = tb + g * 4 + u;
-                    if (t < P.ntiles) { const u32 q = P.tile_q[t]; s4 += (u64)(q & TQ_NS_MASK) | ((u64)((q >> TQ_NW_SHIFT) & TQ_NW_MASK) << 32); }
-                }
+            for (int g = 0; g < 16; g++) {
+                const uint4 x = v[g >> 2];
+                const u32 q = (g & 3) == 0 ? x.x : (g & 3) == 1 ? x.y : (g & 3) == 2 ? x.z : x.w;
+                part[g] = tb + g < P.ntiles ? (q & TQ_NS_MASK) | (((q >> TQ_NW_SHIFT) & TQ_NW_MASK) << 16) : 0u;
             }
-            part[g] = s4; mine += s4;
+        } else {
+#pragma unroll
+            for (int g = 0; g < 16; g++) {
+                u32 s1 = 0;
+                for (int u = 0; u < unit; u++) {
+                    const int t = tb + g * unit + u;
+                    if (t < P.ntiles) { const u32 q = P.tile_q[t]; s1 += (q & TQ_NS_MASK) | (((q >> TQ_NW_SHIFT) & TQ_NW_MASK) << 16); }
+                }
+                part[g] = s1;
+            }
         }
-        u64 total;
-        const u64 before = warp_exscan_u64(mine, lane, &total);
-        const u32 NS = (u32)total, NW = (u32)(total >> 32), NT = (u32)P.ntiles;
+#pragma unroll
+        for (int g = 0; g < 16; g++) { my_s += part[g] & 0xFFFFu; my_w += part[g] >> 16; }
+    }
+    // the closing piece of tile t_lo + tid: is it long?
+    bool closing_long = false;
+    u32 c_end = 0;
+    if (a_np) {
+        const int t = t_lo + tid;
+        c_end = (t + 1 >= P.ntiles) ? (u32)P.hi : a_next != TT_NONE ? (u32)(t + 1) * TT_TILE_BYTES + a_next : closing_piece_end(P, t);
+        closing_long = c_end - ((u32)t * TT_TILE_BYTES + a_last) > (u32)TT_WARP_PIECE_MAX;
+    }
+    bool tickets = big;                                           // short pieces by tickets (bulk) or job by job (a request)
+    if (!big) {
+        u32 bs = my_s, bw = my_w;                                     // exclusive prefixes over the lanes
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const u32 x = __shfl_up_sync(FULL, bs, o), y = __shfl_up_sync(FULL, bw, o);
+            if (lane >= o) { bs += x; bw += y; }
+        }
+        const u32 NS = __shfl_sync(FULL, bs, 31), NW = __shfl_sync(FULL, bw, 31), NT = (u32)P.ntiles;
+        bs -= my_s; bw -= my_w;
 #ifndef TT_SHORT_WARP_FACTOR
 #define TT_SHORT_WARP_FACTOR 12u
 #endif
         // Measured crossover (1 M to 8 M chars of Unicode-heavy prose, 15 K to 120 K unsettled pieces): a warp per piece
         // wins up to about 17 pieces per warp of the grid.
-        bulk = NS + NT > TT_SHORT_WARP_FACTOR * W;
-        if (!bulk) {
-            const u32 J = NW + NT + NS;
-            for (u32 j = gw; j < J; j += W) {                         // bounded by the number of jobs
-                u32 a, n, slot;
-                if (j >= NW && j < NW + NT) {                         // the closing piece of tile j - NW
-                    const int t = (int)(j - NW);
-                    const u32 np = P.tile_cnt[t];
-                    if (np == 0) continue;
-                    const u32 st = (u32)t * TT_TILE_BYTES + P.tile_last[t];
-                    n = closing_piece_end(P, t) - st;
-                    if (n > (u32)TT_WARP_PIECE_MAX) continue;         // settled by a CTA in (A)
-                    a = (u32)((long long)st - P.shift); slot = (u32)t * TT_TILE_BYTES + np - 1;
-                    u32 v;
-                    if (piece_settled_without_merge(P, text, a, n, v)) {     // every lane computes the same
-                        if (lane == 0) { P.piece_cnt[slot] = v; atomicAdd(&P.tile_tok[t], 1u); }
-                        continue;
-                    }
-                } else {
-                    // the k-th queued piece of its class: the lane whose stretch holds it finds the tile
-                    const bool wclass = j < NW;
-                    const u32 k = wclass ? j : j - NW - NT;
-                    const u32 bsel = wclass ? (u32)(before >> 32) : (u32)before;
-                    const u32 owner = 31u - (u32)__clz(__ballot_sync(FULL, bsel <= k) | 1u);
-                    u32 found = 0;                                    // tile << 11 | rank within the tile
-                    if ((u32)lane == owner) {
-                        u32 r = k - bsel;
-                        int g = 0;
-#pragma unroll
-                        for (int gg = 0; gg < 16; gg++) {
-                            const u32 c = wclass ? (u32)(part[gg] >> 32) : (u32)part[gg];
-                            if (g == gg && r >= c && gg < 15) { r -= c; g = gg + 1; }
-                        }
-                        int t = tb + g * 4;
-                        for (int u = 0; u < 4; u++) {
-                            const u32 q = t < P.ntiles ? P.tile_q[t] : 0u;
-                            const u32 c = wclass ? (q >> TQ_NW_SHIFT) & TQ_NW_MASK : q & TQ_NS_MASK;
-                            if (r < c || u == 3) break;
-                            r -= c; t++;
-                        }
-                        found = ((u32)t << 11) | r;
-                    }
-                    found = __shfl_sync(FULL, found, owner);
-                    const u32 t = found >> 11, r = found & 2047u;
-                    const u32 e = P.q[(size_t)t * TT_TILE_QCAP + (wclass ? (u32)TT_TILE_QCAP - 1 - r : r)];
-                    n = (e >> 22) + 1;
-                    a = (u32)((long long)t * TT_TILE_BYTES + (e & 2047u) - P.shift); slot = t * TT_TILE_BYTES + ((e >> 11) & 2047u);
+        tickets = NS + NT > TT_SHORT_WARP_FACTOR * W;
+        const u32 J = tickets ? NW : NW + NT + NS;                    // with tickets only the warp-class pieces go job by job
+        for (u32 j = gw; j < J; j += W) {                             // bounded by the number of jobs
+            u32 a, n, slot;
+            if (j >= NW && j < NW + NT) {                             // the closing piece of tile j - NW
+                const int t = (int)(j - NW);
+                const u32 np = P.tile_cnt[t];
+                if (np == 0) continue;
+                const u32 st = (u32)t * TT_TILE_BYTES + P.tile_last[t];
+                n = closing_piece_end(P, t) - st;
+                if (n > (u32)TT_WARP_PIECE_MAX) continue;             // settled by a CTA below
+                a = (u32)((long long)st - P.shift); slot = (u32)t * TT_TILE_BYTES + np - 1;
+                u32 v;
+                if (piece_settled_without_merge(P, text, a, n, v)) {  // every lane computes the same
+                    if (lane == 0) { P.piece_cnt[slot] = v; atomicAdd(&P.tile_tok[t], 1u); }
+                    continue;
                 }
-                warp_merge_piece(P, text, a, n, slot, wbuf, lane);
+            } else {
+                // the k-th queued piece of its class: the lane whose stretch holds it finds the tile
+                const bool wclass = j < NW;
+                const u32 k = wclass ? j : j - NW - NT;
+                const int sh = wclass ? 16 : 0;
+                const u32 owner = 31u - (u32)__clz(__ballot_sync(FULL, (wclass ? bw : bs) <= k) | 1u);
+                u32 found = 0;                                        // tile << 11 | rank within the tile
+                if ((u32)lane == owner) {
+                    u32 r = k - (wclass ? bw : bs);
+                    int g = 0;
+#pragma unroll
+                    for (int gg = 0; gg < 15; gg++) {
+                        const u32 c = (part[gg] >> sh) & 0xFFFFu;
+                        if (g == gg && r >= c) { r -= c; g = gg + 1; }
+                    }
+                    int t = tb + g * unit;
+                    for (int u = 0; u + 1 < unit; u++) {
+                        const u32 q = t < P.ntiles ? P.tile_q[t] : 0u;
+                        const u32 c = wclass ? (q >> TQ_NW_SHIFT) & TQ_NW_MASK : q & TQ_NS_MASK;
+                        if (r < c) break;
+                        r -= c; t++;
+                    }
+                    found = ((u32)t << 11) | r;
+                }
+                found = __shfl_sync(FULL, found, owner);
+                const u32 t = found >> 11, r = found & 2047u;
+                const u32 e = P.q[(size_t)t * TT_TILE_QCAP + (wclass ? (u32)TT_TILE_QCAP - 1 - r : r)];
+                n = (e >> 22) + 1;
+                a = (u32)((long long)t * TT_TILE_BYTES + (e & 2047u) - P.shift); slot = t * TT_TILE_BYTES + ((e >> 11) & 2047u);
             }
+            warp_merge_piece(P, text, a, n, slot, wbuf, lane);
+        }
+        if (!tickets) {
+            // the request's long pieces, once every warp of the CTA is through with its short ones
+            if (__syncthreads_or(a_nl != 0 || closing_long))
+                cta_long_pieces(P, text, t_lo, t_hi, a_nl, a_np, a_last, c_end, closing_long, s_buf, sc, s_long, &s_nlong);
             return;
         }
+    } else {
+        // bulk text: the warp-class pieces stand in one global list (the first kernel appended them tile by tile)
+        const u32 nwq = *P.nwq;
+        for (u32 j = gw; j < nwq; j += W) {                           // bounded by the list length
+            const u64 x = P.wq[j];
+            const u32 t = (u32)(x >> 32), e = (u32)x;
+            warp_merge_piece(P, text, (u32)((long long)t * TT_TILE_BYTES + (e & 2047u) - P.shift), (e >> 22) + 1, t * TT_TILE_BYTES + ((e >> 11) & 2047u), wbuf, lane);
+        }
     }
-    // bulk mode
-    u32* const tok = reinterpret_cast<u32*>(wbuf);
-    const u32 ntick = ((u32)P.ntiles + MERGE_TICKET_TILES - 1) / MERGE_TICKET_TILES;
-    for (;;) {                                                        // bounded by the number of tickets
-        u32 tk = 0;
-        if (lane == 0) tk = atomicAdd(&P.hdr->t_tiles, 1u);
-        tk = __shfl_sync(FULL, tk, 0);
-        if (tk >= ntick) break;
-        const int t = (int)(tk * MERGE_TICKET_TILES) + lane;              // lanes 0..15: a tile each
-        const bool have_tile = lane < MERGE_TICKET_TILES && t < P.ntiles;
-        u32 q = 0, np = 0;
-        if (have_tile) { q = P.tile_q[t]; np = P.tile_cnt[t]; }
-        const u32 ns = q & TQ_NS_MASK, nw = (q >> TQ_NW_SHIFT) & TQ_NW_MASK;
-        // the closing piece of my tile
-        u32 ca = 0, cn = 0, cslot = 0;                                    // cn == 0: nothing left to do for it
-        if (np) {
-            const u32 st = (u32)t * TT_TILE_BYTES + P.tile_last[t];
-            cn = closing_piece_end(P, t) - st;
-            ca = (u32)((long long)st - P.shift); cslot = (u32)t * TT_TILE_BYTES + np - 1;
-            u32 v;
-            if (cn > (u32)TT_WARP_PIECE_MAX) cn = 0;                      // settled by a CTA in (A)
-            else if (piece_settled_without_merge(P, text, ca, cn, v)) { P.piece_cnt[cslot] = v; atomicAdd(&P.tile_tok[t], 1u); cn = 0; }
-        }
-        // warp-class pieces, one at a time
-        const u32 wany = __ballot_sync(FULL, nw != 0 || cn > (u32)LANE_MAX);
-        for (u32 x = wany; x; x &= x - 1) {                               // warp-uniform
-            const int l = __ffs(x) - 1;
-            const u32 nw_l = __shfl_sync(FULL, nw, l), cn_l = __shfl_sync(FULL, cn, l), ca_l = __shfl_sync(FULL, ca, l), cs_l = __shfl_sync(FULL, cslot, l);
-            const u32 tl = tk * MERGE_TICKET_TILES + (u32)l;
-            for (u32 r = 0; r < nw_l; r++) {
-                const u32 e = P.q[(size_t)tl * TT_TILE_QCAP + (u32)TT_TILE_QCAP - 1 - r];
-                warp_merge_piece(P, text, (u32)((long long)tl * TT_TILE_BYTES + (e & 2047u) - P.shift), (e >> 22) + 1, tl * TT_TILE_BYTES + ((e >> 11) & 2047u), wbuf, lane);
+    for (int t0 = t_lo; t0 < t_hi; t0 += MERGE_THREADS) {            // block-uniform; shares beyond MERGE_THREADS tiles reload their records
+        if (t0 != t_lo) {
+            const int t = t0 + tid;
+            a_nl = 0; a_np = 0; a_last = 0; c_end = 0; closing_long = false;
+            if (t < t_hi) {
+                a_nl = (P.tile_q[t] >> TQ_NL_SHIFT) & TQ_NL_MASK; a_np = P.tile_cnt[t]; a_last = P.tile_last[t];
+                if (a_np) { c_end = closing_piece_end(P, t); closing_long = c_end - ((u32)t * TT_TILE_BYTES + a_last) > (u32)TT_WARP_PIECE_MAX; }
             }
-            if (cn_l > (u32)LANE_MAX) warp_merge_piece(P, text, ca_l, cn_l, cs_l, wbuf, lane);
         }
-        if (cn > (u32)LANE_MAX) cn = 0;
-        // short pieces: the queued ones of the 16 tiles, then the short closing pieces, 32 per step, a thread each
-        u32 pre = ns;                                                     // exclusive prefix of ns over the lanes
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) { const u32 v = __shfl_up_sync(FULL, pre, o); if (lane >= o) pre += v; }
-        const u32 QS = __shfl_sync(FULL, pre, 31);
-        pre -= ns;
-        const u32 cm = __ballot_sync(FULL, cn != 0);
-        const u32 nj = QS + __popc(cm);
-        for (u32 b = 0; b < nj; b += 32) {                                // warp-uniform
-            const u32 e = b + lane;
-            u32 tl = 0, pl = 0;                                           // queued piece: its tile within the ticket, that tile's prefix
-#pragma unroll
-            for (int l = 1; l < MERGE_TICKET_TILES; l++) { const u32 p = __shfl_sync(FULL, pre, l); if (p <= e) { tl = (u32)l; pl = p; } }
-            const u32 src = select_bit(cm, e >= QS ? e - QS : 0u) & 31u;  // closing piece: the lane that holds it
-            const u32 ca_s = __shfl_sync(FULL, ca, src), cn_s = __shfl_sync(FULL, cn, src), cs_s = __shfl_sync(FULL, cslot, src);
-            if (e < nj) {
-                u32 a, n, slot;
-                if (e < QS) {
-                    const u32 tt = tk * MERGE_TICKET_TILES + tl;
-                    const u32 qe = P.q[(size_t)tt * TT_TILE_QCAP + (e - pl)];
-                    n = (qe >> 22) + 1;
-                    a = (u32)((long long)tt * TT_TILE_BYTES + (qe & 2047u) - P.shift); slot = tt * TT_TILE_BYTES + ((qe >> 11) & 2047u);
-                } else { a = ca_s; n = cn_s; slot = cs_s; }
-                if (!piece_in_range(P, a, n, slot, 4u) || n < 2 || n > (u32)LANE_MAX) hdr_selfcheck_failed(P.hdr, P.epoch, 5u, a, n, slot, e);
-                else {
-                    const u32 m = lane_merge(tok, tok + LANE_SLOTS * LANE_MAX, lane, text, a, n, P.tab, P.ext_id, P.stage);
-                    piece_done(P, slot, m);
+        if (__syncthreads_or(a_nl != 0 || closing_long))
+            cta_long_pieces(P, text, t0, t_hi, a_nl, a_np, a_last, c_end, closing_long, s_buf, sc, s_long, &s_nlong);
+    }
+    // ---- tickets: a tile each; its short pieces (queued ones, then its closing piece if that is short) wait in the
+    // lanes until 32 of them are together, so that every step of the thread-per-piece merge is full
+    {
+        u32* const tok = reinterpret_cast<u32*>(wbuf);
+        const u32 ntick = (u32)P.ntiles;
+        u32 pa = 0, pn = 0, pslot = 0, pend = 0;                      // lanes below `pend` hold a short piece that waits for a full step
+        for (;;) {                                                    // bounded by the number of tickets
+            u32 t = 0;
+            if (lane == 0) t = atomicAdd(&P.hdr->t_tiles, 1u);
+            t = __shfl_sync(FULL, t, 0);
+            const bool last_round = t >= ntick;
+            u32 ns = 0, ca = 0, cn = 0, cslot = 0;                    // cn == 0: no closing piece left to merge
+            if (!last_round) {                                        // warp-uniform; every lane computes the same
+                const u32 q = P.tile_q[t], np = P.tile_cnt[t], last = P.tile_last[t];
+                const u32 nf = t + 1 < ntick ? P.tile_first[t + 1] : TT_NONE;
+                ns = q & TQ_NS_MASK;
+                if (np) {
+                    const u32 st = t * TT_TILE_BYTES + last;
+                    cn = (t + 1 >= ntick ? (u32)P.hi : nf != TT_NONE ? (t + 1) * TT_TILE_BYTES + nf : closing_piece_end(P, (int)t)) - st;
+                    ca = (u32)((long long)st - P.shift); cslot = t * TT_TILE_BYTES + np - 1;
+                    u32 v;
+                    if (cn > (u32)TT_WARP_PIECE_MAX) cn = 0;          // settled by a CTA above
+                    else if (piece_settled_without_merge(P, text, ca, cn, v)) { if (lane == 0) { P.piece_cnt[cslot] = v; atomicAdd(&P.tile_tok[t], 1u); } cn = 0; }
+                    else if (cn > (u32)LANE_MAX) { warp_merge_piece(P, text, ca, cn, cslot, wbuf, lane); cn = 0; }
                 }
             }
-            __syncwarp();
+            const u32 nj = ns + (cn ? 1u : 0u);
+            u32 e0 = 0;                                               // new pieces handed to lanes so far
+            for (;;) {                                                // warp-uniform; bounded by nj / 32 + 2
+                const u32 left = nj - e0;
+                const bool run = pend + left >= 32u || (last_round && pend != 0);
+                const u32 take = min(32u - pend, left);               // lanes pend .. pend + take - 1 take new pieces
+                const u32 e = e0 + ((u32)lane - pend);
+                if ((u32)lane >= pend && (u32)lane - pend < take) {
+                    if (e < ns) {
+                        const u32 qe = P.q[(size_t)t * TT_TILE_QCAP + e];
+                        pn = (qe >> 22) + 1;
+                        pa = (u32)((long long)t * TT_TILE_BYTES + (qe & 2047u) - P.shift); pslot = t * TT_TILE_BYTES + ((qe >> 11) & 2047u);
+                    } else { pa = ca; pn = cn; pslot = cslot; }
+                }
+                e0 += take; pend += take;
+                if (!run) break;
+                if ((u32)lane < pend) {
+                    if (!piece_in_range(P, pa, pn, pslot, 4u) || pn < 2 || pn > (u32)LANE_MAX) hdr_selfcheck_failed(P.hdr, P.epoch, 5u, pa, pn, pslot, e);
+                    else {
+                        const u32 m = lane_merge(tok, tok + LANE_SLOTS * LANE_MAX, lane, text, pa, pn, P.tab, P.ext_id, P.stage);
+                        piece_done(P, pslot, m);
+                    }
+                }
+                __syncwarp();
+                pend = 0;
+            }
+            if (last_round) break;
         }
+    }
+    // ---- bulk text: the last CTA to finish sums the token counts of every group of 256 tiles for k_scatter (a counter
+    // zeroed by the kernel before this one tells which CTA that is; nobody waits for anybody)
+    if (P.grp_tok == nullptr) return;
+    __threadfence();
+    __syncwarp();
+    u32 fin = 0;
+    if (lane == 0 && atomicAdd(&s_warps_done, 1u) == MERGE_WARPS - 1) fin = atomicAdd(&P.hdr->merge_done, 1u) == gridDim.x - 1;
+    if (!__shfl_sync(FULL, fin, 0)) return;
+    __threadfence();
+    const int ngroups = (P.ntiles + TT_GROUP_TILES - 1) / TT_GROUP_TILES;
+    for (int g = 0; g < ngroups; g++) {                               // one warp: eight loads per lane and group
+        u32 sum = 0;
+#pragma unroll
+        for (int u = 0; u < TT_GROUP_TILES / 32; u++) { const int t = g * TT_GROUP_TILES + u * 32 + lane; if (t < P.ntiles) sum += __ldcg(&P.tile_tok[t]); }
+#pragma unroll
+        for (int o = 16; o; o >>= 1) sum += __shfl_xor_sync(FULL, sum, o);
+        if (lane == 0) P.grp_tok[g] = sum;
     }
 }
 
@@ -1027,6 +1082,7 @@ struct ScatterParams {
     int ntiles;
     const u32* tile_cnt;
     const u32* tile_tok;       // tokens per tile
+    const u32* grp_tok;        // bulk text: tokens per group of TT_GROUP_TILES tiles, else null
     const u16* piece_off16;
     unsigned long long ids_cap;
     const u32* piece_cnt;
@@ -1047,20 +1103,29 @@ k_scatter(const ScatterParams P) {
     __shared__ u32 sc[48];
     __shared__ u32 s_big[TT_TILE_BYTES / 8][3];
     __shared__ u32 s_nbig;
+    __shared__ u32 s_np[BPE_THREADS];                         // pieces of the next tiles of this CTA's range
     __shared__ unsigned long long s_sum[66];
     const int tid = threadIdx.x;
     cudaGridDependencySynchronize();                         // k_merge's (and with it the first kernel's) results are complete from here on
-    // Each CTA takes a contiguous range of tiles and sums the token counts of all tiles itself: those before its
-    // range give its first output position, all of them the count and the capacity check.
+    // Each CTA takes a contiguous range of tiles.  Tokens before its first tile: a request's CTAs sum the counts of
+    // all tiles themselves; for bulk text k_merge has left the totals of groups of tiles, so a CTA adds the whole
+    // groups before its range and the tiles of its own group before it.  The grand total gives the count and the
+    // capacity check, which every CTA makes for itself.
     const int per = (P.ntiles + (int)gridDim.x - 1) / (int)gridDim.x;
     const int tile_lo = (int)blockIdx.x * per, tile_hi = min(P.ntiles, tile_lo + per);
     unsigned long long before = 0, total = 0;
-    for (int t0 = 0; t0 < P.ntiles; t0 += BPE_THREADS * 4) {
-        u32 x[4];
+    if (P.grp_tok == nullptr) {
+        for (int t0 = 0; t0 < P.ntiles; t0 += BPE_THREADS * 4) {
+            u32 x[4];
 #pragma unroll
-        for (int u = 0; u < 4; u++) { const int t = t0 + u * BPE_THREADS + tid; x[u] = t < P.ntiles ? P.tile_tok[t] : 0u; }
+            for (int u = 0; u < 4; u++) { const int t = t0 + u * BPE_THREADS + tid; x[u] = t < P.ntiles ? P.tile_tok[t] : 0u; }
 #pragma unroll
-        for (int u = 0; u < 4; u++) { total += x[u]; if (t0 + u * BPE_THREADS + tid < tile_lo) before += x[u]; }
+            for (int u = 0; u < 4; u++) { total += x[u]; if (t0 + u * BPE_THREADS + tid < tile_lo) before += x[u]; }
+        }
+    } else {
+        const int ngroups = (P.ntiles + TT_GROUP_TILES - 1) / TT_GROUP_TILES, g_lo = tile_lo / TT_GROUP_TILES;
+        for (int g = tid; g < ngroups; g += BPE_THREADS) { const u32 x = P.grp_tok[g]; total += x; if (g < g_lo) before += x; }
+        for (int t = g_lo * TT_GROUP_TILES + tid; t < tile_lo; t += BPE_THREADS) before += P.tile_tok[t];
     }
     cta_sum2_u64(before, total, s_sum);
     int status = hdr_status(P.hdr, P.epoch);
@@ -1079,26 +1144,55 @@ k_scatter(const ScatterParams P) {
         const long long len = P.hi - P.shift;
         for (int d = P.n_docs - tid; d >= 0 && P.doc_off[d] >= len; d -= blockDim.x) P.ids_off_out[d] = (long long)total;
     }
+    // Work items: (tile, block of 512 of its pieces), two neighbouring pieces per thread.  The loads of the next item
+    // (piece values and offsets) go out before the current one is scanned and written, so that the chain
+    // "count of the tile -> its piece values -> scan -> staged ids" of one tile overlaps with the next tile's.
     u32 carry = (u32)before;
-    for (int tile = tile_lo; tile < tile_hi; tile++) {
+    for (int tc = tile_lo; tc < tile_hi; tc += BPE_THREADS) {         // block-uniform
+        const int nk = min(BPE_THREADS, tile_hi - tc);
         __syncthreads();
+        if (tid < nk) s_np[tid] = P.tile_cnt[tc + tid];
         if (tid == 0) s_nbig = 0;
-        const u32 np = P.tile_cnt[tile];
-        const size_t p0 = (size_t)tile * TT_TILE_BYTES;
-        const long long t0 = (long long)tile * TT_TILE_BYTES - P.shift;      // text offset of the tile start
-        for (u32 b = 0; b < np; b += BPE_THREADS) {
-            const u32 i = b + tid;
-            const int32_t v = i < np ? (int32_t)P.piece_cnt[p0 + i] : 0;       // an id, or minus the staged count
-            const u32 c = i < np ? (v >= 0 ? 1u : (u32)(-v)) : 0u;
-            const u32 off = (i < np && (v < 0 || P.docmask)) ? P.piece_off16[p0 + i] : 0u;
+        __syncthreads();
+        int k = 0;
+        u32 b = 0;
+        while (k < nk && s_np[k] == 0) k++;
+        uint2 v = make_uint2(0, 0);
+        u32 o2 = 0;
+        if (k < nk) {
+            const size_t p0 = (size_t)(tc + k) * TT_TILE_BYTES;
+            const u32 i0 = 2 * (u32)tid;
+            if (i0 < s_np[k]) { v = *reinterpret_cast<const uint2*>(P.piece_cnt + p0 + i0); o2 = *reinterpret_cast<const u32*>(P.piece_off16 + p0 + i0); }
+        }
+        while (k < nk) {                                              // block-uniform
+            // the item after this one
+            int k2 = k;
+            u32 b2 = b + 2 * BPE_THREADS;
+            if (b2 >= s_np[k2]) { b2 = 0; k2++; while (k2 < nk && s_np[k2] == 0) k2++; }
+            uint2 vn = make_uint2(0, 0);
+            u32 on = 0;
+            if (k2 < nk) {
+                const size_t q0 = (size_t)(tc + k2) * TT_TILE_BYTES;
+                const u32 j0 = b2 + 2 * (u32)tid;
+                if (j0 < s_np[k2]) { vn = *reinterpret_cast<const uint2*>(P.piece_cnt + q0 + j0); on = *reinterpret_cast<const u32*>(P.piece_off16 + q0 + j0); }
+            }
+            // this item
+            const int tile = tc + k;
+            const u32 np = s_np[k], i0 = b + 2 * (u32)tid;
+            const long long t0 = (long long)tile * TT_TILE_BYTES - P.shift;  // text offset of the tile start
+            const int32_t x0 = i0 < np ? (int32_t)v.x : 0, x1 = i0 + 1 < np ? (int32_t)v.y : 0;   // an id, or minus the staged count
+            const u32 c0 = i0 < np ? (x0 >= 0 ? 1u : (u32)(-x0)) : 0u, c1 = i0 + 1 < np ? (x1 >= 0 ? 1u : (u32)(-x1)) : 0u;
             u32 tot;
-            const u32 dst = carry + cta_excl_sum_scan(c, sc, &tot);
-            if (i < np && ((unsigned long long)dst + c > total || (v < 0 && (long long)t0 + off + c > P.hi - P.shift))) {
-                hdr_selfcheck_failed(P.hdr, P.epoch, 6u, (u32)tile, i, (u32)v, dst);
-            } else if (i < np) {
+            const u32 d0 = carry + cta_excl_sum_scan(c0 + c1, sc, &tot);
+#pragma unroll
+            for (int h = 0; h < 2; h++) {
+                const u32 i = i0 + h, c = h ? c1 : c0, dst = h ? d0 + c0 : d0, off = h ? o2 >> 16 : o2 & 0xFFFFu;
+                const int32_t x = h ? x1 : x0;
+                if (i >= np) continue;
+                if ((unsigned long long)dst + c > total || (x < 0 && t0 + off + c > P.hi - P.shift)) { hdr_selfcheck_failed(P.hdr, P.epoch, 6u, (u32)tile, i, (u32)x, dst); continue; }
                 const u32 src = (u32)(t0 + off);
-                if (v >= 0) P.ids_out[dst] = v;
-                else if (c <= 8) { for (u32 k = 0; k < c; k++) P.ids_out[dst + k] = P.stage[src + k]; }
+                if (x >= 0) P.ids_out[dst] = x;
+                else if (c <= 8) { for (u32 kk = 0; kk < c; kk++) P.ids_out[dst + kk] = P.stage[src + kk]; }
                 else {
                     const u32 slot = atomicAdd(&s_nbig, 1u);
                     if (slot < TT_TILE_BYTES / 8) { s_big[slot][0] = src; s_big[slot][1] = dst; s_big[slot][2] = c; }
@@ -1116,11 +1210,16 @@ k_scatter(const ScatterParams P) {
             }
             carry += tot;
             __syncthreads();
-        }
-        const u32 nbig = min(s_nbig, (u32)(TT_TILE_BYTES / 8));
-        for (u32 e = 0; e < nbig; e++) {
-            const u32 src = s_big[e][0], d2 = s_big[e][1], cc = s_big[e][2];
-            for (u32 k = tid; k < cc; k += BPE_THREADS) P.ids_out[d2 + k] = P.stage[src + k];
+            const u32 nbig = min(s_nbig, (u32)(TT_TILE_BYTES / 8));
+            if (nbig) {                                               // block-uniform: pieces of more than 8 tokens, copied by the whole CTA
+                for (u32 e = 0; e < nbig; e++) {
+                    const u32 src = s_big[e][0], d2 = s_big[e][1], cc = s_big[e][2];
+                    for (u32 kk = tid; kk < cc; kk += BPE_THREADS) P.ids_out[d2 + kk] = P.stage[src + kk];
+                }
+                __syncthreads();
+                if (tid == 0) s_nbig = 0;
+            }
+            k = k2; b = b2; v = vn; o2 = on;
         }
     }
 }

@@ -23,6 +23,7 @@ constexpr int TT_CHUNK = 16;
 #endif
 constexpr int TT_TILE_CHUNKS = TT_TILE_CHUNKS_DEF;        // = threads per CTA
 constexpr int TT_TILE_BYTES = TT_CHUNK * TT_TILE_CHUNKS; // 2 KiB of text per tile
+constexpr int TT_GROUP_TILES = 256;              // bulk text: token totals are also kept per group of 256 tiles
 constexpr int TT_TILE_QCAP = TT_TILE_BYTES / 2;  // unsettled pieces of <= 256 bytes a tile can have (each has >= 2 bytes)
 constexpr int TT_TILE_LONGCAP = 8;               // pieces of > 256 bytes that lie inside one tile
 constexpr u32 TT_NONE = 0xFFFFFFFFu;
@@ -43,8 +44,10 @@ struct TTHeader {
     u32 pretok_done;         // CTAs that finished the pre-tokenization pass (tt_pretokenize only; cleared by a memset)
     u32 n_pieces;            // number of pieces found (tt_pretokenize only)
     u32 t_tiles;             // ticket counter of k_merge's bulk mode (groups of tiles handed out); zeroed by the kernel before it
+    u32 merge_done;          // CTAs of k_merge that have finished (bulk text: the last one sums the groups); zeroed likewise
+    u32 nwq;                 // bulk text: length of the global list of warp-class pieces (cleared by a memset before the chain)
     u32 dbg[8];              // first failed self-check of a kernel: site, then up to seven values (diagnostics only)
-    u32 pad[19];
+    u32 pad[17];
 };
 static_assert(sizeof(TTHeader) == 128, "header layout");
 
@@ -99,10 +102,12 @@ struct TTWorkspace {
     u32* tile_last;
     u32* tile_tok;
     u32* tile_q;
+    u32* grp_tok;      // bulk text only: tokens per group of TT_GROUP_TILES tiles
     u16* tile_long;
     u16* piece_off16;
     u32* piece_cnt;
     u32* q;
+    u64* wq;           // bulk text only: warp-class pieces of all tiles (len / 33 + 64 entries)
     int32_t* stage;    // token ids staged at the byte offset of their piece (len)
     u64* pairbuf;      // (token, rank) pairs of the long-piece path, indexed like the text (len)
     u8* cand;          // literal pass: length of the longest added-token literal starting at each byte (aligned frame)

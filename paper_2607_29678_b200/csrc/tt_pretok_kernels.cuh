@@ -199,6 +199,8 @@ __device__ __forceinline__ void store_slot(u16 (*sm)[TT_SLOTS], int s, const Chu
 // and the tables of the whole-piece lookups.
 struct FrontParams {
     u32* tile_last; u32* tile_tok; u32* tile_q; u16* tile_long; u16* piece_off16; u32* piece_cnt; u32* q;
+    u64* wq;                   // bulk text (more tiles than a request's job search covers): the warp-class pieces of all tiles go
+                               // to this one list, appended tile by tile (hdr->nwq, cleared before the chain); else null
     TokTable toktab;           // slots == nullptr: none
     LongTable longtab;         // ignore_merges: entries longer than the whole-piece table holds (else slots == nullptr)
     const int32_t* ext_id;
@@ -221,12 +223,13 @@ k_pretok(const PretokParams P, const FrontParams F) {
     __shared__ u32 s_need, s_first;
     __shared__ u32 s_islast;
     __shared__ u16 s_off[FUSED ? TT_TILE_BYTES + 2 : 2];              // piece offsets of the tile
-    __shared__ u32 s_wtot[TT_TILE_CHUNKS / 32], s_ns, s_nw, s_nl, s_total;
+    __shared__ u32 s_wtot[TT_TILE_CHUNKS / 32], s_ns, s_nw, s_nl, s_total, s_wbase;
+    __shared__ u16 s_wlist[TT_TILE_BYTES / (LANE_MAX + 1) + 2];       // bulk text: the tile's warp-class pieces
 
     const int tid = threadIdx.x;
     cudaTriggerProgrammaticLaunchCompletion();               // the next kernel may be placed; it waits for this grid's memory itself
     if (FUSED) {
-        if (blockIdx.x == 0 && tid == 0) P.hdr->t_tiles = 0;  // k_merge's ticket counter (k_merge touches it only after this grid)
+        if (blockIdx.x == 0 && tid == 0) { P.hdr->t_tiles = 0; P.hdr->merge_done = 0; }   // k_merge's counters (k_merge touches them only after this grid)
         // the whole-piece table is probed at random a few microseconds from now: ask for it to be brought into L2
         if (F.toktab.slots != nullptr) grid_prefetch_l2(F.toktab.slots, ((size_t)F.toktab.mask + 1) * sizeof(TokSlot));
     }
@@ -405,7 +408,11 @@ k_pretok(const PretokParams P, const FrontParams F) {
                 } else if (n[j] > TT_TOKTAB_MAXLEN && F.longtab.slots != nullptr && n[j] <= F.longtab.maxlen && longtab_lookup(F.longtab, text, a[j], n[j], id)) {
                     F.piece_cnt[p0 + i] = (u32)id; wsum++;
                 } else if (n[j] > (u32)TT_WARP_PIECE_MAX) F.tile_long[(size_t)tile * TT_TILE_LONGCAP + atomicAdd(&s_nl, 1u)] = (u16)i;
-                else if (n[j] > (u32)LANE_MAX) F.q[(size_t)tile * TT_TILE_QCAP + (u32)TT_TILE_QCAP - 1 - atomicAdd(&s_nw, 1u)] = tile_queue_entry(s_off[i], i, n[j]);
+                else if (n[j] > (u32)LANE_MAX) {
+                    const u32 k = atomicAdd(&s_nw, 1u);
+                    if (F.wq != nullptr) s_wlist[k] = (u16)i;
+                    else F.q[(size_t)tile * TT_TILE_QCAP + (u32)TT_TILE_QCAP - 1 - k] = tile_queue_entry(s_off[i], i, n[j]);
+                }
                 else F.q[(size_t)tile * TT_TILE_QCAP + atomicAdd(&s_ns, 1u)] = tile_queue_entry(s_off[i], i, n[j]);
             }
         }
@@ -415,7 +422,15 @@ k_pretok(const PretokParams P, const FrontParams F) {
         __syncthreads();
         if (tid == 0) {
             F.tile_tok[tile] = s_total;
-            F.tile_q[tile] = s_ns | (s_nw << TQ_NW_SHIFT) | (s_nl << TQ_NL_SHIFT);
+            F.tile_q[tile] = s_ns | ((F.wq != nullptr ? 0u : s_nw) << TQ_NW_SHIFT) | (s_nl << TQ_NL_SHIFT);
+            if (F.wq != nullptr && s_nw) s_wbase = atomicAdd(&P.hdr->nwq, s_nw);
+        }
+        if (F.wq != nullptr && s_nw) {                                // block-uniform
+            __syncthreads();
+            for (u32 k = tid; k < s_nw; k += TT_TILE_CHUNKS) {
+                const u32 i = s_wlist[k];
+                F.wq[s_wbase + k] = ((u64)(u32)tile << 32) | tile_queue_entry(s_off[i], i, (u32)s_off[i + 1] - s_off[i]);
+            }
         }
     }
     if (any_bad) hdr_set_status(P.hdr, P.epoch, 4 /* TT_ERR_INVALID_UTF8 */);

@@ -211,17 +211,18 @@ static int build_token_table(tt_vocab* v, const tt_merge* merges, size_t n_merge
     while (cap < 2 * keep.size() + 2) cap <<= 1;
     u32 log2cap = 0;
     while ((1u << log2cap) < cap) log2cap++;
-    const u32 mask = cap - 1, shift = 64 - log2cap;
+    const u32 mask = cap - 1, shift = 32 - log2cap;
     std::vector<TokSlot> slots(cap);
     memset(slots.data(), 0, cap * sizeof(TokSlot));
     for (u32 i : keep) {
         const u32 n = off[i + 1] - off[i];
         u8 key[24] = {0};
         memcpy(key, cat.data() + off[i], n);
-        u64 k[3]; memcpy(k, key, 24);
-        u32 hh = toktab_hash(k[0], k[1], k[2], n, shift);
+        u32 k[6]; memcpy(k, key, 24);
+        u32 hh = toktab_hash_final(toktab_hash_rest(toktab_hash_short(k[0], k[1], n), k[2], k[3], k[4], k[5]), shift);
         while (slots[hh].len != 0) hh = (hh + 1) & mask;
-        slots[hh].k0 = k[0]; slots[hh].k1 = k[1]; slots[hh].k2 = k[2]; slots[hh].len = n; slots[hh].id = ext_id[cand[i]];
+        slots[hh].len = n; slots[hh].id = ext_id[cand[i]];
+        for (int j = 0; j < 6; j++) slots[hh].k[j] = k[j];
     }
     if (cudaMalloc(&v->d_tokslots, (size_t)cap * sizeof(TokSlot)) != cudaSuccess ||
         cudaMemcpy(v->d_tokslots, slots.data(), (size_t)cap * sizeof(TokSlot), cudaMemcpyHostToDevice) != cudaSuccess) {

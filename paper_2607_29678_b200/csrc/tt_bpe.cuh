@@ -96,58 +96,62 @@ __device__ __forceinline__ void grid_prefetch_l2(const void* p, size_t bytes) {
 // ---- whole-piece table: byte string of a vocabulary entry -> its id ------------------------------------
 // Holds every token of at most TT_TOKTAB_MAXLEN bytes whose own byte string encodes to exactly that
 // token (checked at load time by running the merge kernel below on every token string), so a hit
-// returns what the merge loop would return.  Slots are 32 bytes (one sector): three key words, the
-// length (0 = empty) and the caller's id; open addressing, linear probing, load factor <= 0.5.
+// returns what the merge loop would return.  Slots are 32 bytes (one sector): length (0 = empty), the
+// caller's id and six key words (the bytes, little endian, zero padded); open addressing, linear probing,
+// load factor <= 0.5.  The first 16 bytes of a slot (length, id, key words 0 and 1) decide every piece of at
+// most 8 bytes -- most pieces of ordinary text -- with one vector load.
 constexpr int TT_TOKTAB_MAXLEN = 24;
-struct TokSlot { u64 k0, k1, k2; u32 len; int32_t id; };
+struct TokSlot { u32 len; int32_t id; u32 k[6]; };
 static_assert(sizeof(TokSlot) == 32, "slot layout");
-struct TokTable { const TokSlot* slots; u32 mask; u32 shift; };
+struct TokTable { const TokSlot* slots; u32 mask; u32 shift; };   // shift = 32 - log2(capacity)
 
-TT_HD u32 toktab_hash(u64 k0, u64 k1, u64 k2, u32 len, u32 shift) {
-    u64 h = (k0 + len) * 0x9E3779B97F4A7C15ull;
-    h ^= (k1 + 0x632BE59BD9B4E019ull) * 0xC2B2AE3D27D4EB4Full;
-    h ^= (k2 + 0x85157AF5ull) * 0x165667B19E3779F9ull;
-    h ^= h >> 29;
-    h *= 0xBF58476D1CE4E5B9ull;
-    return (u32)(h >> shift);
+// Key words beyond the piece are zero, so they add nothing: a piece of at most 8 bytes is hashed from two words.
+TT_HD u32 toktab_hash_short(u32 k0, u32 k1, u32 n) { return n * 0x9E3779B1u + k0 * 0x85EBCA6Bu + k1 * 0xC2B2AE35u; }
+TT_HD u32 toktab_hash_rest(u32 h, u32 k2, u32 k3, u32 k4, u32 k5) { return h + k2 * 0x27D4EB2Fu + k3 * 0x165667B1u + k4 * 0xD3A2646Du + k5 * 0xFD7046C5u; }
+TT_HD u32 toktab_hash_final(u32 h, u32 shift) {
+    h ^= h >> 15; h *= 0x2C1B3C6Du; h ^= h >> 12; h *= 0x297A2D39u; h ^= h >> 15;
+    return h >> shift;
+}
+TT_HD u32 toktab_mask_word(u32 w, u32 n, u32 j) {      // key word j of a piece of n bytes: bytes beyond the piece are zero
+    const u32 have = n > 4 * j ? n - 4 * j : 0u;
+    return have >= 4 ? w : have == 0 ? 0u : w & ((1u << (8 * have)) - 1u);
 }
 
-// Key of a piece of 2..24 bytes: its bytes in three words, zero padded.
-__device__ __forceinline__ void toktab_key(const u8* __restrict__ text, u32 a, u32 n, u64& k0, u64& k1, u64& k2) {
-    // gather the piece's bytes with aligned 8-byte loads (only words that hold a piece byte)
+#if defined(__CUDACC__)
+// Key words 0 and 1 of the piece of n >= 1 bytes at text + a, from the aligned words x0, x1, x2 that hold it
+// (x1 / x2 only where the piece reaches them).
+__device__ __forceinline__ void toktab_key01(u32 x0, u32 x1, u32 x2, u32 sb, u32 n, u32& k0, u32& k1) {
+    const u32 sh = sb * 8;
+    k0 = toktab_mask_word(__funnelshift_r(x0, x1, sh), n, 0);
+    k1 = toktab_mask_word(__funnelshift_r(x1, x2, sh), n, 1);
+}
+// Looks a piece of 2..24 bytes up; returns true and the id on a hit.  (The first kernel has its own copy of the
+// first steps for pieces of at most 8 bytes, four pieces in flight per thread.)
+__device__ __forceinline__ bool toktab_lookup(const TokTable& tab, const u8* __restrict__ text, u32 a, u32 n, int32_t& id) {
     const uintptr_t addr = (uintptr_t)(text + a);
-    const u64* w = reinterpret_cast<const u64*>(addr & ~(uintptr_t)7);
-    const u32 sh = (u32)(addr & 7) * 8, last = (u32)(addr & 7) + n;     // bytes used in the window
-    const u64 w0 = __ldg(w), w1 = last > 8 ? __ldg(w + 1) : 0, w2 = last > 16 ? __ldg(w + 2) : 0, w3 = last > 24 ? __ldg(w + 3) : 0;
-    k0 = sh ? (w0 >> sh) | (w1 << (64 - sh)) : w0;
-    k1 = sh ? (w1 >> sh) | (w2 << (64 - sh)) : w1;
-    k2 = sh ? (w2 >> sh) | (w3 << (64 - sh)) : w2;
-    if (n < 8) { k0 &= (1ull << (8 * n)) - 1; k1 = 0; k2 = 0; }
-    else if (n < 16) { k1 &= (n == 8) ? 0 : ((1ull << (8 * (n - 8))) - 1); k2 = 0; }
-    else if (n < 24) { k2 &= (n == 16) ? 0 : ((1ull << (8 * (n - 16))) - 1); }
-}
-// Probes from slot h on; lo / hi are the two halves of slot h, already loaded.
-__device__ __forceinline__ bool toktab_finish(const TokTable& tab, u64 k0, u64 k1, u64 k2, u32 n, u32 h, uint4 lo, uint4 hi, int32_t& id) {
+    const u32* w = reinterpret_cast<const u32*>(addr & ~(uintptr_t)3);
+    const u32 sb = (u32)(addr & 3), sh = sb * 8, used = sb + n;           // bytes of the aligned window that hold the piece
+    u32 x[7];
+#pragma unroll
+    for (int j = 0; j < 7; j++) x[j] = used > 4u * j ? __ldg(w + j) : 0u;  // only words that hold a piece byte
+    u32 k[6];
+#pragma unroll
+    for (int j = 0; j < 6; j++) k[j] = toktab_mask_word(__funnelshift_r(x[j], x[j + 1], sh), n, j);
+    u32 h = toktab_hash_final(toktab_hash_rest(toktab_hash_short(k[0], k[1], n), k[2], k[3], k[4], k[5]), tab.shift);
     for (u32 probe = 0; probe <= tab.mask; probe++) {           // bounded by the capacity
-        if (hi.z == 0) return false;
-        if (hi.z == n && (((u64)lo.y << 32) | lo.x) == k0 && (((u64)lo.w << 32) | lo.z) == k1 && (((u64)hi.y << 32) | hi.x) == k2) {
-            id = (int32_t)hi.w;
-            return true;
+        const uint4* sp = reinterpret_cast<const uint4*>(tab.slots + h);
+        const uint4 lo = __ldg(sp);
+        if (lo.x == 0) return false;
+        if (lo.x == n && lo.z == k[0] && lo.w == k[1]) {
+            bool same = true;
+            if (n > 8) { const uint4 hi = __ldg(sp + 1); same = hi.x == k[2] && hi.y == k[3] && hi.z == k[4] && hi.w == k[5]; }
+            if (same) { id = (int32_t)lo.y; return true; }
         }
         h = (h + 1) & tab.mask;
-        const uint4* sp = reinterpret_cast<const uint4*>(tab.slots + h);
-        lo = __ldg(sp); hi = __ldg(sp + 1);
     }
     return false;
 }
-// Looks a piece of 2..24 bytes up; returns true and the id on a hit.
-__device__ __forceinline__ bool toktab_lookup(const TokTable& tab, const u8* __restrict__ text, u32 a, u32 n, int32_t& id) {
-    u64 k0, k1, k2;
-    toktab_key(text, a, n, k0, k1, k2);
-    const u32 h = toktab_hash(k0, k1, k2, n, tab.shift);
-    const uint4* sp = reinterpret_cast<const uint4*>(tab.slots + h);
-    return toktab_finish(tab, k0, k1, k2, n, h, __ldg(sp), __ldg(sp + 1), id);
-}
+#endif
 
 // ---- long-entry table (ignore_merges only): vocabulary entries of more than TT_TOKTAB_MAXLEN bytes --------
 // Slot = (64-bit hash of the bytes, offset into a byte blob, length, id); open addressing, load <= 0.5.  A hit

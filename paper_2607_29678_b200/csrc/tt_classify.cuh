@@ -39,6 +39,62 @@ inline void tt_fill_ascii_table(u8* t) {
     }
 }
 
+// ---- sixteen ASCII bytes without a table ------------------------------------------------------------------
+// For a word of four bytes below 0x80, tt_swar_ge(y, c) has the top bit of a byte set exactly where that byte is
+// >= c (1 <= c <= 0x80): the byte-wise sums stay below 0x100, so nothing carries from byte to byte.  A range is
+// ge(lo) & ~ge(hi + 1).
+TT_HD u32 tt_swar_ge(u32 y, u32 c) { return y + (0x80u - c) * 0x01010101u; }
+TT_HD u32 tt_swar_range(u32 y, u32 lo, u32 hi) { return tt_swar_ge(y, lo) & ~tt_swar_ge(y, hi + 1) & 0x80808080u; }
+// The four words are first transposed (word j = byte j of each input word), so that the top bits of the test
+// results fall into place with four shifts: bit 4k + j of the result <- top bit of byte k of m_j.
+TT_HD u32 tt_gather_top_bits(u32 m0, u32 m1, u32 m2, u32 m3) {
+    u32 u = (m0 >> 7) | (m1 >> 6) | (m2 >> 5) | (m3 >> 4);          // bit 8k + j
+    u = (u | (u >> 4)) & 0x00FF00FFu;
+    return (u | (u >> 8)) & 0xFFFFu;
+}
+TT_HD u32 tt_perm(u32 x, u32 y, u32 sel) {                              // bytes of {x, y} picked by four selector nibbles
+#if defined(__CUDA_ARCH__)
+    return __byte_perm(x, y, sel);
+#else
+    const u64 v = ((u64)y << 32) | x;
+    u32 r = 0;
+    for (int i = 0; i < 4; i++) r |= (u32)((v >> (8 * ((sel >> (4 * i)) & 7))) & 0xFF) << (8 * i);
+    return r;
+#endif
+}
+TT_HD ChunkMasks tt_classify_ascii16(u32 w0, u32 w1, u32 w2, u32 w3) {
+    // transpose: y[j] = (byte j of w0, byte j of w1, byte j of w2, byte j of w3)
+    const u32 p = tt_perm(w0, w1, 0x5140u), q = tt_perm(w2, w3, 0x5140u);      // bytes 0 and 1 of each pair
+    const u32 r = tt_perm(w0, w1, 0x7362u), t = tt_perm(w2, w3, 0x7362u);      // bytes 2 and 3
+    const u32 y[4] = {tt_perm(p, q, 0x5410u), tt_perm(p, q, 0x7632u), tt_perm(r, t, 0x5410u), tt_perm(r, t, 0x7632u)};
+    u32 let[4], cas[4], num[4], spc[4], nl[4], sp[4], ap[4], sl[4], oth[4];
+#pragma unroll
+    for (int j = 0; j < 4; j++) {
+        const u32 v = y[j];
+        let[j] = tt_swar_range(v | 0x20202020u, 'a', 'z');                      // only letters fold into a..z
+        cas[j] = v << 2;                                                          // bit 5 of a byte (lower case) in its top bit
+        num[j] = tt_swar_range(v, '0', '9');
+        sp[j] = tt_swar_range(v, ' ', ' ');
+        spc[j] = tt_swar_range(v, 9, 13) | sp[j];
+        nl[j] = tt_swar_range(v, '\n', '\n') | tt_swar_range(v, '\r', '\r');
+        ap[j] = tt_swar_range(v, '\'', '\'');
+        sl[j] = tt_swar_range(v, '/', '/');
+        oth[j] = ~(let[j] | num[j] | spc[j]) & 0x80808080u;
+    }
+    ChunkMasks m;
+    m.lead = 0xFFFF; m.mark = 0; m.cless = 0; m.bad = 0;
+    m.low = (u16)tt_gather_top_bits(let[0] & cas[0], let[1] & cas[1], let[2] & cas[2], let[3] & cas[3]);
+    m.upp = (u16)tt_gather_top_bits(let[0] & ~cas[0], let[1] & ~cas[1], let[2] & ~cas[2], let[3] & ~cas[3]);
+    m.num = (u16)tt_gather_top_bits(num[0], num[1], num[2], num[3]);
+    m.spc = (u16)tt_gather_top_bits(spc[0], spc[1], spc[2], spc[3]);
+    m.oth = (u16)tt_gather_top_bits(oth[0], oth[1], oth[2], oth[3]);
+    m.nl = (u16)tt_gather_top_bits(nl[0], nl[1], nl[2], nl[3]);
+    m.sp = (u16)tt_gather_top_bits(sp[0], sp[1], sp[2], sp[3]);
+    m.ap = (u16)tt_gather_top_bits(ap[0], ap[1], ap[2], ap[3]);
+    m.sl = (u16)tt_gather_top_bits(sl[0], sl[1], sl[2], sl[3]);
+    return m;
+}
+
 // words w[0] = the 4 bytes before the chunk, w[1..4] = the chunk, w[5] = the 4 bytes after it
 #define TT_BYTE(w, j) (((w)[((j) + 4) >> 2] >> (8 * (((j) + 4) & 3))) & 0xFFu)
 
@@ -47,22 +103,19 @@ inline void tt_fill_ascii_table(u8* t) {
 TT_HD ChunkMasks tt_classify_words(const u32 (&w)[6], long long g0, long long lo, long long hi, const ClassTables& T) {
     u64 accA = 0, accB = 0, accF = 0;   // 16-bit lanes: A = codes 0..3, B = codes 4..6, F = flags 1..4
     u32 lead = 0, bad = 0, cov = 0, contm = 0;
-    u32 valid = 0;
-#pragma unroll
-    for (int k = 0; k < 16; k++) valid |= (u32)(g0 + k >= lo && g0 + k < hi) << k;
+    // bytes of the chunk inside [lo, hi)
+    const long long vlo = lo - g0, vhi = hi - g0;
+    const u32 klo = vlo <= 0 ? 0u : vlo >= 16 ? 16u : (u32)vlo, khi = vhi <= 0 ? 0u : vhi >= 16 ? 16u : (u32)vhi;
+    const u32 valid = khi > klo ? ((1u << khi) - 1u) & ~((1u << klo) - 1u) : 0u;
     const bool all_ascii = ((w[1] | w[2] | w[3] | w[4]) & 0x80808080u) == 0;
     if (all_ascii) {
-#pragma unroll
-        for (int k = 0; k < 16; k++) {
-            u32 b = TT_BYTE(w, k);
-            u32 v = T.ascii[b];
-            u32 c = v & 7, f = v >> 3;
-            u64 bit = 1ull << ((c & 3) * 16 + k);
-            accA |= (c < 4) ? bit : 0ull;
-            accB |= (c >= 4) ? bit : 0ull;
-            accF |= f ? (1ull << ((f - 1) * 16 + k)) : 0ull;
-        }
-        lead = 0xFFFF;
+        // sixteen ASCII bytes at once: byte-wise range tests on the four words (see tt_swar_ge), the flag bits gathered
+        // into 16-bit masks; no table look-ups
+        ChunkMasks a = tt_classify_ascii16(w[1], w[2], w[3], w[4]);
+        a.lead = (u16)(0xFFFFu & valid);
+        a.oth &= (u16)valid; a.spc &= (u16)valid; a.num &= (u16)valid; a.low &= (u16)valid; a.upp &= (u16)valid;
+        a.nl &= (u16)valid; a.sp &= (u16)valid; a.ap &= (u16)valid; a.sl &= (u16)valid;
+        return a;
     } else {
 #pragma unroll
         for (int j = -3; j < 16; j++) {
@@ -127,8 +180,10 @@ TT_HD ChunkMasks tt_classify_chunk(const u8* base, long long chunk, long long nc
     if (chunk >= 0 && chunk < nchunks) {
         const uint4 v = *reinterpret_cast<const uint4*>(base + chunk * TT_CHUNK);
         w[1] = v.x; w[2] = v.y; w[3] = v.z; w[4] = v.w;
-        if (chunk > 0) w[0] = *reinterpret_cast<const u32*>(base + chunk * TT_CHUNK - 4);
-        if (chunk + 1 < nchunks) w[5] = *reinterpret_cast<const u32*>(base + (chunk + 1) * TT_CHUNK);
+        if (((v.x | v.y | v.z | v.w) & 0x80808080u) != 0) {       // the neighbours matter only to multi-byte characters
+            if (chunk > 0) w[0] = *reinterpret_cast<const u32*>(base + chunk * TT_CHUNK - 4);
+            if (chunk + 1 < nchunks) w[5] = *reinterpret_cast<const u32*>(base + (chunk + 1) * TT_CHUNK);
+        }
     }
     return tt_classify_words(w, chunk * TT_CHUNK, lo, hi, T);
 }

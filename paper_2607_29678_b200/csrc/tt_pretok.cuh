@@ -185,52 +185,59 @@ TT_HD u32 tt_eval_chunk_cuts(const u16 (*sm)[TT_SLOTS], int slot, const TileCarr
     return (u32)((S & lead & OWN) >> 16);
 }
 
+// A 32-bit window over the masks of field f: bits 0..7 = the last eight bytes of the chunk before, bits 8..23 = the
+// chunk in `slot`, bits 24..31 = the first eight bytes of the chunk after it.  Pattern 0 looks at most four bytes
+// back and three ahead, so single-word operations cover it.
+TT_HD u32 tt_win32(const u16 (*sm)[TT_SLOTS], int f, int slot) {
+    return ((u32)sm[f][slot - 1] >> 8) | ((u32)sm[f][slot] << 8) | ((u32)sm[f][slot + 1] << 24);
+}
+
 // Pattern 0 (cl100k-style).  Returns the 16 start bits of the chunk in `slot`; `need` receives the
 // NEED_* flags of aggregates that leave the shared-memory window (then `tc` must be filled and the
 // function called again).
 TT_HD u32 tt_eval_chunk_p0(const u16 (*sm)[TT_SLOTS], int slot, const u8* base, long long g0, long long hi,
                            const TileCarry& tc, bool have_tc, u32& need, bool single_digits = false,
                            const u32* docmask = nullptr) {
-    const u64 OWN = 0xFFFFull << 16;
-    const u64 lead = tt_win(sm, F_LEAD, slot);
-    const u64 L = tt_win(sm, F_LOW, slot) | tt_win(sm, F_UPP, slot) | tt_win(sm, F_CLESS, slot);
-    const u64 N = tt_win(sm, F_NUM, slot);
-    const u64 W = tt_win(sm, F_SPC, slot);
-    const u64 O = tt_win(sm, F_OTH, slot) | tt_win(sm, F_MARK, slot);
-    const u64 NL = tt_win(sm, F_NL, slot), SP = tt_win(sm, F_SP, slot), AP = tt_win(sm, F_AP, slot);
-    const u64 D = tt_win(sm, F_DOC, slot);
-    const u64 V = L | N | W | O;                       // bytes that exist and are valid
-    const u64 cont = V & ~lead;
-    const u64 nD = ~D;
-    u64 S = 0;
+    const u32 OWN = 0xFFFFu << 8;
+    const u32 lead = tt_win32(sm, F_LEAD, slot);
+    const u32 L = tt_win32(sm, F_LOW, slot) | tt_win32(sm, F_UPP, slot) | tt_win32(sm, F_CLESS, slot);
+    const u32 N = tt_win32(sm, F_NUM, slot);
+    const u32 W = tt_win32(sm, F_SPC, slot);
+    const u32 O = tt_win32(sm, F_OTH, slot) | tt_win32(sm, F_MARK, slot);
+    const u32 NL = tt_win32(sm, F_NL, slot), SP = tt_win32(sm, F_SP, slot), AP = tt_win32(sm, F_AP, slot);
+    const u32 D = tt_win32(sm, F_DOC, slot);
+    const u32 V = L | N | W | O;                       // bytes that exist and are valid
+    const u32 cont = V & ~lead;
+    const u32 nD = ~D;
+    u32 S = 0;
 #define PREV(x) (((x) << 1) & nD)
     // punctuation runs: start of the run, unless a blank precedes it (the blank starts the piece)
-    const u64 G = O & lead & ~PREV(O) & ~PREV(SP);
+    const u32 G = O & lead & ~PREV(O) & ~PREV(SP);
     S |= G;
     // letter runs: the run start, unless non-CR/LF whitespace or a single match-start punctuation char precedes it
-    const u64 c1 = cont << 1, c2 = cont << 2, c3 = cont << 3;
-    const u64 pfx = ((G << 1) | ((G << 2) & c1) | ((G << 3) & c2 & c1) | ((G << 4) & c3 & c2 & c1)) & nD;
+    const u32 c1 = cont << 1, c2 = cont << 2, c3 = cont << 3;
+    const u32 pfx = ((G << 1) | ((G << 2) & c1) | ((G << 3) & c2 & c1) | ((G << 4) & c3 & c2 & c1)) & nD;
     S |= L & lead & ~PREV(L) & ~((PREV(W) & ~PREV(NL)) | pfx);
     // contractions: apostrophe that is a match start, then s/t/m/d or re/ve/ll; the letter after the suffix starts a piece
-    u64 ga = G & AP & (0x3FFFFull << 12);              // apostrophes at own bytes -4 .. +13 can put a start into this chunk
+    u32 ga = G & AP & (0x3FFFFu << 4);                 // apostrophes at own bytes -4 .. +13 can put a start into this chunk
     while (ga) {
-        int p = tt_lobit((u32)(ga >> 12)) + 12; ga &= ga - 1;
-        long long g = g0 + (p - 16);
+        const int p = tt_lobit(ga); ga &= ga - 1;
+        const long long g = g0 + (p - 8);
         u32 b1 = (g + 1 < hi) ? base[g + 1] : 0, b2 = (g + 2 < hi) ? base[g + 2] : 0;
         if ((D >> (p + 1)) & 1) b1 = 0;
         if ((D >> (p + 2)) & 1) b2 = 0;
-        int cl = tt_contraction_len(b1, b2);
+        const int cl = tt_contraction_len(b1, b2);
         if (cl) {
-            u64 at = 1ull << (p + cl);
-            bool same_doc = ((D >> (p + 1)) & ((1ull << cl) - 1)) == 0;
+            const u32 at = 1u << (p + cl);
+            const bool same_doc = ((D >> (p + 1)) & ((1u << cl) - 1)) == 0;
             if (same_doc) S |= at & L & lead;
         }
     }
     // number runs: every third number lead counted from the run start (single-digit variant: every lead)
     if (single_digits) S |= N & lead;
     else {
-        u32 n_own = (u32)(N >> 16) & 0xFFFFu, ld_own = (u32)(lead >> 16) & 0xFFFFu;
-        u32 nstart = (u32)((N & ~PREV(N)) >> 16) & 0xFFFFu;
+        const u32 n_own = (N >> 8) & 0xFFFFu, ld_own = (lead >> 8) & 0xFFFFu;
+        const u32 nstart = ((N & ~PREV(N)) >> 8) & 0xFFFFu;
         u32 m = n_own & ld_own;
         if (m) {
             u32 cnt = 0;
@@ -241,9 +248,9 @@ TT_HD u32 tt_eval_chunk_p0(const u16 (*sm)[TT_SLOTS], int slot, const u8* base, 
                 cnt %= 3;
             }
             while (m) {
-                int i = tt_lobit(m); m &= m - 1;
+                const int i = tt_lobit(m); m &= m - 1;
                 if ((nstart >> i) & 1) cnt = 0;
-                if (cnt == 0) S |= 1ull << (16 + i);
+                if (cnt == 0) S |= 1u << (8 + i);
                 cnt = cnt == 2 ? 0 : cnt + 1;
             }
         }
@@ -253,27 +260,27 @@ TT_HD u32 tt_eval_chunk_p0(const u16 (*sm)[TT_SLOTS], int slot, const u8* base, 
         // (a) run start, unless it is a CR/LF glued to preceding punctuation
         S |= W & lead & ~PREV(W) & ~(PREV(O) & NL);
         // (b) CR/LF absorbed by preceding punctuation: CR/LF runs that begin right after punctuation
-        u32 nl_own = (u32)(NL >> 16) & 0xFFFFu, d_own = (u32)(D >> 16) & 0xFFFFu;
+        const u32 nl_own = (NL >> 8) & 0xFFFFu, d_own = (D >> 8) & 0xFFFFu;
         u32 prev_absorbed = 0;                             // byte before the chunk is an absorbed CR/LF
-        if (((NL >> 15) & 1) && !(d_own & 1)) {
+        if (((NL >> 7) & 1) && !(d_own & 1)) {
             bool open;
             prev_absorbed = tt_walk_back_nl(sm, slot - 1, 1, open);
             if (open) { if (have_tc) prev_absorbed = tc.nl_absorbed_before; else need |= NEED_A; }
         }
-        u32 nlq = nl_own & ~d_own;
-        u32 sel = (u32)(((NL & ~PREV(NL) & PREV(O)) >> 16) & 0xFFFFu) | ((nlq & 1) ? prev_absorbed : 0);
-        u32 absorbed = nlq & ~(nlq + sel);
-        u64 prevA = (((u64)absorbed << 17) | ((u64)prev_absorbed << 16)) & nD;
+        const u32 nlq = nl_own & ~d_own;
+        const u32 sel = (((NL & ~PREV(NL) & PREV(O)) >> 8) & 0xFFFFu) | ((nlq & 1) ? prev_absorbed : 0);
+        const u32 absorbed = nlq & ~(nlq + sel);
+        const u32 prevA = ((absorbed << 9) | (prev_absorbed << 8)) & nD;
         S |= W & lead & ~NL & prevA;
         // (c) last character of the run when something follows in the same document (and it is not CR/LF)
-        const u64 next_exists = (V >> 1) & ~(D >> 1);
-        const u64 wend = W & ~((W >> 1) & ~(D >> 1)) & next_exists;
-        const u64 k1 = cont >> 1, k2 = cont >> 2, k3 = cont >> 3;
+        const u32 next_exists = (V >> 1) & ~(D >> 1);
+        const u32 wend = W & ~((W >> 1) & ~(D >> 1)) & next_exists;
+        const u32 k1 = cont >> 1, k2 = cont >> 2, k3 = cont >> 3;
         S |= lead & W & ~NL & (wend | ((wend >> 1) & k1) | ((wend >> 2) & k1 & k2) | ((wend >> 3) & k1 & k2 & k3));
         // (d) first character after the last CR/LF of the run
-        u32 cand = (u32)((W & lead & ~NL & PREV(NL)) >> 16) & 0xFFFFu;
+        u32 cand = ((W & lead & ~NL & PREV(NL)) >> 8) & 0xFFFFu;
         while (cand) {
-            int i = tt_lobit(cand); cand &= cand - 1;
+            const int i = tt_lobit(cand); cand &= cand - 1;
             bool open;
             u32 later = tt_walk_fwd_nl(sm, slot, i, open);
             if (open) {
@@ -282,9 +289,9 @@ TT_HD u32 tt_eval_chunk_p0(const u16 (*sm)[TT_SLOTS], int slot, const u8* base, 
                 else if (have_tc) later = tc.nl_later_after;
                 else { need |= NEED_F; later = 1; }
             }
-            if (!later) S |= 1ull << (16 + i);
+            if (!later) S |= 1u << (8 + i);
         }
     }
 #undef PREV
-    return (u32)((S & lead & OWN) >> 16);
+    return (S & lead & OWN) >> 8;
 }

@@ -206,6 +206,31 @@ struct FrontParams {
     const int32_t* ext_id;
 };
 
+// A piece on the general path of the fused kernel: an extracted literal, a single byte, a vocabulary entry of up to
+// 24 bytes, or (ignore_merges) a longer entry.  Returns true and the value for piece_cnt if it needs no merging.
+__device__ __forceinline__ bool front_piece_general(const PretokParams& P, const FrontParams& F, const u8* __restrict__ text, u32 a, u32 n, u32& val) {
+    int32_t id;
+    if (P.litstart != nullptr) {
+        const long long g = (long long)a + P.lo;
+        if ((P.litstart[g >> 5] >> (g & 31)) & 1) { val = 0u - 1u; return true; }    // one staged id (written by the literal pass)
+    }
+    if (n == 1) { val = (u32)F.ext_id[text[a]]; return true; }
+    if (n <= (u32)TT_TOKTAB_MAXLEN) {
+        if (F.toktab.slots != nullptr && toktab_lookup(F.toktab, text, a, n, id)) { val = (u32)id; return true; }
+    } else if (F.longtab.slots != nullptr && n <= F.longtab.maxlen && longtab_lookup(F.longtab, text, a, n, id)) { val = (u32)id; return true; }
+    return false;
+}
+// An unsettled piece (offset o in the tile, index i, n bytes) goes to the tile's queue of its length class.
+__device__ __forceinline__ void front_piece_queue(const FrontParams& F, int tile, u32 o, u32 i, u32 n, u32* s_ns, u32* s_nw, u32* s_nl, u16* s_wlist) {
+    if (n > (u32)TT_WARP_PIECE_MAX) F.tile_long[(size_t)tile * TT_TILE_LONGCAP + atomicAdd(s_nl, 1u)] = (u16)i;
+    else if (n > (u32)LANE_MAX) {
+        const u32 k = atomicAdd(s_nw, 1u);
+        if (F.wq != nullptr) s_wlist[k] = (u16)i;
+        else F.q[(size_t)tile * TT_TILE_QCAP + (u32)TT_TILE_QCAP - 1 - k] = tile_queue_entry(o, i, n);
+    }
+    else F.q[(size_t)tile * TT_TILE_QCAP + atomicAdd(s_ns, 1u)] = tile_queue_entry(o, i, n);
+}
+
 // FUSED = false: the start flags go to P.startmask, with the pieces per tile (tt_pretokenize and the cut pass of the
 // three-splitter composition).
 // FUSED = true (the encode chain's first kernel): the tile's flags stay in shared memory and become its list of
@@ -225,6 +250,8 @@ k_pretok(const PretokParams P, const FrontParams F) {
     __shared__ u16 s_off[FUSED ? TT_TILE_BYTES + 2 : 2];              // piece offsets of the tile
     __shared__ u32 s_wtot[TT_TILE_CHUNKS / 32], s_ns, s_nw, s_nl, s_total, s_wbase;
     __shared__ u16 s_wlist[TT_TILE_BYTES / (LANE_MAX + 1) + 2];       // bulk text: the tile's warp-class pieces
+    __shared__ u16 s_slow[TT_TILE_BYTES / 9 + 4];                     // pieces of more than 8 bytes (looked up together)
+    __shared__ u32 s_nslow;
 
     const int tid = threadIdx.x;
     cudaTriggerProgrammaticLaunchCompletion();               // the next kernel may be placed; it waits for this grid's memory itself
@@ -247,7 +274,7 @@ k_pretok(const PretokParams P, const FrontParams F) {
 
     for (int tile = blockIdx.x; tile < P.ntiles; tile += gridDim.x) {
         __syncthreads();
-        if (tid == 0) { s_need = 0; s_first = 0xFFFFFFFFu; s_ns = 0; s_nw = 0; s_nl = 0; s_total = 0; }
+        if (tid == 0) { s_need = 0; s_first = 0xFFFFFFFFu; s_ns = 0; s_nw = 0; s_nl = 0; s_total = 0; s_nslow = 0; }
         const long long c_first = (long long)tile * TT_TILE_CHUNKS;
         if (!tables_loaded) {                                         // block-uniform
             bool hi_bit = false;
@@ -362,58 +389,74 @@ k_pretok(const PretokParams P, const FrontParams F) {
             P.tile_first[tile] = np ? (u32)s_off[0] : TT_NONE;
             F.tile_last[tile] = np ? (u32)s_off[np - 1] : TT_NONE;
         }
-        // ---- K4, first half: whole-piece lookups, a thread per piece, two pieces per thread and step (first the
-        // bytes of both, then the table slots of both: each lookup is a chain of two dependent loads).  The tile's
-        // last piece is left to k_merge.
+        // ---- K4, first half: whole-piece lookups, a thread per piece, four pieces per thread and step, their loads side
+        // by side (a lookup is a chain of two dependent loads: the text words, then the table slot).  Pieces of at most 8
+        // bytes -- most of them -- take a path of their own: two key words, one 16-byte half of the slot.  The tile's last
+        // piece is left to k_merge.
         const u8* text = P.base + P.lo;
         const long long t0 = c_first * TT_CHUNK - P.lo;               // text offset of the tile start
         const u32 nlook = np ? np - 1 : 0;
+        const bool quick = P.litstart == nullptr && F.toktab.slots != nullptr;     // block-uniform
         u32 wsum = 0;
-        for (u32 ib = tid; ib < nlook; ib += 2 * TT_TILE_CHUNKS) {
-            u32 a[2], n[2], h[2], kind[2];                            // kind: 0 none, 1 literal, 2 one byte, 3 table lookup, 4 other
-            u64 k0[2], k1[2], k2[2];
-            uint4 lo[2], hi[2];
+        for (u32 ib = tid; ib < nlook; ib += 4 * TT_TILE_CHUNKS) {
+            u32 o[4], n[4], k0[4], k1[4], h[4], x0[4], x1[4], x2[4];
+            uint4 sl[4];
 #pragma unroll
-            for (int j = 0; j < 2; j++) {
+            for (int j = 0; j < 4; j++) {
                 const u32 i = ib + j * TT_TILE_CHUNKS;
-                kind[j] = 0; a[j] = 0; n[j] = 0; k0[j] = 0; k1[j] = 0; k2[j] = 0;
-                if (i < nlook) {
-                    a[j] = (u32)(t0 + s_off[i]);
-                    n[j] = (u32)s_off[i + 1] - s_off[i];
-                    const long long g = (long long)a[j] + P.lo;
-                    if (P.litstart != nullptr && ((P.litstart[g >> 5] >> (g & 31)) & 1)) kind[j] = 1;
-                    else if (n[j] == 1) { kind[j] = 2; k0[j] = text[a[j]]; }
-                    else if (n[j] <= TT_TOKTAB_MAXLEN && F.toktab.slots != nullptr) { kind[j] = 3; toktab_key(text, a[j], n[j], k0[j], k1[j], k2[j]); }
-                    else kind[j] = 4;
+                o[j] = 0; n[j] = 0; x0[j] = 0; x1[j] = 0; x2[j] = 0;
+                if (i < nlook) { o[j] = s_off[i]; n[j] = (u32)s_off[i + 1] - o[j]; }
+                if (quick && n[j] != 0 && n[j] <= 8) {
+                    const uintptr_t addr = (uintptr_t)(text + t0 + o[j]);
+                    const u32* w = reinterpret_cast<const u32*>(addr & ~(uintptr_t)3);
+                    const u32 used = (u32)(addr & 3) + n[j];
+                    x0[j] = __ldg(w);
+                    if (used > 4) x1[j] = __ldg(w + 1);
+                    if (used > 8) x2[j] = __ldg(w + 2);
                 }
             }
 #pragma unroll
-            for (int j = 0; j < 2; j++) {
-                h[j] = 0; lo[j] = make_uint4(0, 0, 0, 0); hi[j] = lo[j];
-                if (kind[j] == 3) {
-                    h[j] = toktab_hash(k0[j], k1[j], k2[j], n[j], F.toktab.shift);
-                    const uint4* sp = reinterpret_cast<const uint4*>(F.toktab.slots + h[j]);
-                    lo[j] = __ldg(sp); hi[j] = __ldg(sp + 1);
-                } else if (kind[j] == 2) lo[j].x = (u32)F.ext_id[(u32)k0[j]];
+            for (int j = 0; j < 4; j++) {
+                k0[j] = 0; k1[j] = 0; h[j] = 0; sl[j] = make_uint4(0, 0, 0, 0);
+                if (quick && n[j] != 0 && n[j] <= 8) {
+                    toktab_key01(x0[j], x1[j], x2[j], (u32)((uintptr_t)(text + t0 + o[j]) & 3), n[j], k0[j], k1[j]);
+                    if (n[j] == 1) sl[j].y = (u32)F.ext_id[k0[j]];
+                    else {
+                        h[j] = toktab_hash_final(toktab_hash_short(k0[j], k1[j], n[j]), F.toktab.shift);
+                        sl[j] = __ldg(reinterpret_cast<const uint4*>(F.toktab.slots + h[j]));
+                    }
+                }
             }
 #pragma unroll
-            for (int j = 0; j < 2; j++) {
+            for (int j = 0; j < 4; j++) {
                 const u32 i = ib + j * TT_TILE_CHUNKS;
-                int32_t id;
-                if (kind[j] == 0) continue;
-                if (kind[j] == 1) { F.piece_cnt[p0 + i] = 0u - 1u; wsum++; }     // one staged id (written by the literal pass)
-                else if (kind[j] == 2) { F.piece_cnt[p0 + i] = lo[j].x; wsum++; }
-                else if (kind[j] == 3 && toktab_finish(F.toktab, k0[j], k1[j], k2[j], n[j], h[j], lo[j], hi[j], id)) {
-                    F.piece_cnt[p0 + i] = (u32)id; wsum++;
-                } else if (n[j] > TT_TOKTAB_MAXLEN && F.longtab.slots != nullptr && n[j] <= F.longtab.maxlen && longtab_lookup(F.longtab, text, a[j], n[j], id)) {
-                    F.piece_cnt[p0 + i] = (u32)id; wsum++;
-                } else if (n[j] > (u32)TT_WARP_PIECE_MAX) F.tile_long[(size_t)tile * TT_TILE_LONGCAP + atomicAdd(&s_nl, 1u)] = (u16)i;
-                else if (n[j] > (u32)LANE_MAX) {
-                    const u32 k = atomicAdd(&s_nw, 1u);
-                    if (F.wq != nullptr) s_wlist[k] = (u16)i;
-                    else F.q[(size_t)tile * TT_TILE_QCAP + (u32)TT_TILE_QCAP - 1 - k] = tile_queue_entry(s_off[i], i, n[j]);
-                }
-                else F.q[(size_t)tile * TT_TILE_QCAP + atomicAdd(&s_ns, 1u)] = tile_queue_entry(s_off[i], i, n[j]);
+                if (n[j] == 0) continue;
+                bool settled = false;
+                u32 val = 0;
+                if (quick && n[j] == 1) { val = sl[j].y; settled = true; }
+                else if (quick && n[j] <= 8) {
+                    uint4 c = sl[j];
+                    u32 hh = h[j];
+                    for (u32 probe = 0; probe <= F.toktab.mask; probe++) {       // bounded by the capacity
+                        if (c.x == 0) break;
+                        if (c.x == n[j] && c.z == k0[j] && c.w == k1[j]) { val = c.y; settled = true; break; }
+                        hh = (hh + 1) & F.toktab.mask;
+                        c = __ldg(reinterpret_cast<const uint4*>(F.toktab.slots + hh));
+                    }
+                } else if (quick) { s_slow[atomicAdd(&s_nslow, 1u)] = (u16)i; continue; }     // longer pieces: together, below
+                else settled = front_piece_general(P, F, text, (u32)(t0 + o[j]), n[j], val);
+                if (settled) { F.piece_cnt[p0 + i] = val; wsum++; }
+                else front_piece_queue(F, tile, o[j], i, n[j], &s_ns, &s_nw, &s_nl, s_wlist);
+            }
+        }
+        if (quick) {                                                  // block-uniform: the pieces of more than 8 bytes, a thread each
+            __syncthreads();
+            const u32 nslow = s_nslow;
+            for (u32 e = tid; e < nslow; e += TT_TILE_CHUNKS) {
+                const u32 i = s_slow[e], o = s_off[i], n = (u32)s_off[i + 1] - o;
+                u32 val = 0;
+                if (front_piece_general(P, F, text, (u32)(t0 + o), n, val)) { F.piece_cnt[p0 + i] = val; wsum++; }
+                else front_piece_queue(F, tile, o, i, n, &s_ns, &s_nw, &s_nl, s_wlist);
             }
         }
 #pragma unroll

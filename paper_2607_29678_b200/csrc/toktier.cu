@@ -194,7 +194,7 @@ static int build_token_table(tt_vocab* v, const tt_merge* merges, size_t n_merge
         Q.hdr = d_hdr; Q.epoch = next_epoch(); Q.tab = v->tab;
         Q.toktab.slots = nullptr; Q.toktab.mask = 0; Q.toktab.shift = 0;      // no table yet: every piece is merged
         Q.longtab = LongTable{}; Q.litstart = nullptr;
-        Q.ext_id = v->d_ext_id; Q.piece_cnt = d_cnt; Q.stage = d_stage; Q.pairbuf = nullptr; Q.tile_tok = d_tt; Q.grp_tok = nullptr; Q.wq = nullptr; Q.nwq = nullptr;
+        Q.ext_id = v->d_ext_id; Q.piece_cnt = d_cnt; Q.stage = d_stage; Q.pairbuf = nullptr; Q.tile_tok = d_tt; Q.grp_tok = nullptr; Q.wq = nullptr; Q.gq = nullptr; Q.lq = nullptr;
         k_merge<<<v->sm_count * MERGE_CTAS_PER_SM, MERGE_THREADS, MERGE_SMEM_BYTES>>>(Q);
         ok = cudaGetLastError() == cudaSuccess && cudaDeviceSynchronize() == cudaSuccess;
     }
@@ -387,7 +387,8 @@ extern "C" int tt_vocab_load_ex(const tt_merge* merges, size_t n_merges, const i
     ok = ok && cudaMemcpy(v->d_cls, cls.data(), v->cls_bytes, cudaMemcpyHostToDevice) == cudaSuccess;
     if (!ok) { cudaGetLastError(); tt_vocab_free(v); return TT_ERR_CUDA; }
     v->tab.slots = v->d_slots; v->tab.bytepair = v->d_bytepair; v->tab.mask = mask; v->tab.shift = shift;
-    if (cudaFuncSetAttribute(k_merge, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)MERGE_SMEM_BYTES) != cudaSuccess) { cudaGetLastError(); tt_vocab_free(v); return TT_ERR_CUDA; }
+    if (cudaFuncSetAttribute(k_merge, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)MERGE_SMEM_BYTES) != cudaSuccess ||
+        cudaFuncSetAttribute(k_merge_bulk, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)MERGE_SMEM_BYTES) != cudaSuccess) { cudaGetLastError(); tt_vocab_free(v); return TT_ERR_CUDA; }
     { const int rc = build_token_table(v, merges, n_merges, ext_id); if (rc != TT_OK) { tt_vocab_free(v); return rc; } }
     {   // byte length and number of non-continuation bytes of every token, indexed by the caller's id
         std::vector<uint2> in(256 + n_merges);
@@ -436,6 +437,8 @@ static size_t carve(TTWorkspace* w, void* base, size_t max_len, size_t max_docs)
     p = take(ntiles * TT_TILE_BYTES * sizeof(u32));          if (w) w->piece_cnt = (u32*)p;
     p = take(ntiles * TT_TILE_QCAP * sizeof(u32));           if (w) w->q = (u32*)p;
     p = take((max_len / 33 + 64) * sizeof(u64));             if (w) w->wq = (u64*)p;
+    p = take((max_len / 2 + 64) * sizeof(u64));              if (w) w->gq = (u64*)p;
+    p = take((max_len / 257 + 16) * sizeof(uint4));          if (w) w->lq = (uint4*)p;
     p = take((max_len + 1) * sizeof(int32_t));  if (w) w->stage = (int32_t*)p;
     p = take((max_len + 1) * sizeof(u64));      if (w) w->pairbuf = (u64*)p;
     p = take(padded + 16);                      if (w) w->cand = (u8*)p;
@@ -571,9 +574,14 @@ static int encode_impl(const tt_vocab* v, const uint8_t* text, size_t len, const
     Q.hdr = w.hdr; Q.tab = v->tab; Q.toktab = v->toktab; Q.longtab = v->longtab; Q.litstart = literals ? w.litstart : nullptr; Q.epoch = PP.epoch;
     Q.ext_id = v->d_ext_id; Q.piece_cnt = w.piece_cnt; Q.stage = w.stage; Q.pairbuf = w.pairbuf; Q.tile_tok = w.tile_tok;
     Q.grp_tok = PP.ntiles > MERGE_SR_MAX_TILES ? w.grp_tok : nullptr;   // group totals only where k_scatter's CTAs would otherwise sum thousands of tiles each
-    Q.wq = PP.ntiles > MERGE_SR_MAX_TILES ? w.wq : nullptr; Q.nwq = &w.hdr->nwq;
-    if (ev) k_merge<<<merge_grid, MERGE_THREADS, MERGE_SMEM_BYTES, st>>>(Q);
-    else CK(launch_after(k_merge, merge_grid, MERGE_THREADS, st, Q, MERGE_SMEM_BYTES));
+    Q.wq = big ? w.wq : nullptr; Q.gq = big ? w.gq : nullptr; Q.lq = big ? w.lq : nullptr;
+    if (big) {                                                               // bulk text: closing pieces and the global lists first
+        const int cgrid = (PP.ntiles + CLOSING_THREADS - 1) / CLOSING_THREADS;
+        if (ev) k_closing<<<cgrid, CLOSING_THREADS, 0, st>>>(Q);
+        else CK(launch_after(k_closing, cgrid, CLOSING_THREADS, st, Q));
+    }
+    if (ev) { if (big) k_merge_bulk<<<merge_grid, MERGE_THREADS, MERGE_SMEM_BYTES, st>>>(Q); else k_merge<<<merge_grid, MERGE_THREADS, MERGE_SMEM_BYTES, st>>>(Q); }
+    else CK(launch_after(big ? k_merge_bulk : k_merge, merge_grid, MERGE_THREADS, st, Q, MERGE_SMEM_BYTES));
     MARK(2);
     ScatterParams S;
     S.shift = PP.lo; S.hi = PP.hi; S.ntiles = PP.ntiles; S.tile_cnt = w.tile_cnt; S.tile_tok = w.tile_tok; S.grp_tok = Q.grp_tok; S.piece_off16 = w.piece_off16;

@@ -722,8 +722,9 @@ struct PieceParams {
     u64* pairbuf;              // global scratch of the long-piece path, indexed like the text
     u32* tile_tok;
     u32* grp_tok;              // bulk text: tokens per group of TT_GROUP_TILES tiles (written by the last CTA), else null
-    const u64* wq;             // bulk text: the warp-class pieces of all tiles (tile << 32 | queue entry), else null
-    const u32* nwq;            //            their number
+    u64* wq;                   // bulk text: the warp-class pieces of all tiles (tile << 32 | queue entry), else null
+    u64* gq;                   // bulk text: the short pieces of all tiles, gathered by k_closing (tile << 32 | queue entry)
+    uint4* lq;                 // bulk text: the long pieces of all tiles, listed by k_closing (text offset, bytes, piece slot, 0)
 };
 
 // ---- K4, second half: the merges ------------------------------------------------------------------------------
@@ -805,6 +806,62 @@ __device__ __forceinline__ u64 warp_exscan_u64(u64 v, int lane, u64* total) {
     return x - v;
 }
 
+// ---- bulk text only: the closing pieces, and one list per length class for the whole text ---------------------
+// A thread per tile settles the tile's closing piece where no merging is needed and gathers what is left of the
+// 32 tiles of its warp -- queued short pieces, a short closing piece -- into one global list (one reservation
+// per warp), so that k_merge's warps take 32 short pieces at a time whatever tile they come from; warp-class
+// closing pieces join the first kernel's list, long pieces get a list of their own.  The counters were cleared
+// by the memset in front of the chain.
+constexpr int CLOSING_THREADS = 256;
+__global__ void __launch_bounds__(CLOSING_THREADS)
+k_closing(const PieceParams P) {
+    const int lane = threadIdx.x & 31;
+    const u32 FULL = 0xFFFFFFFFu;
+    cudaTriggerProgrammaticLaunchCompletion();
+    cudaGridDependencySynchronize();                         // the first kernel's per-tile records are complete from here on
+    if (hdr_status(P.hdr, P.epoch) != 0) return;
+    const u8* text = P.base + P.shift;
+    const int t = (int)(blockIdx.x * blockDim.x + threadIdx.x);
+    u32 ns = 0, nl = 0, np = 0, centry = 0;                  // centry != 0: a short closing piece to be queued
+    if (t < P.ntiles) {
+        const u32 q = P.tile_q[t];
+        ns = q & TQ_NS_MASK; nl = (q >> TQ_NL_SHIFT) & TQ_NL_MASK; np = P.tile_cnt[t];
+    }
+    u32 cn = 0, ca = 0, cslot = 0, clast = 0;
+    if (np) {
+        clast = P.tile_last[t];
+        const u32 st = (u32)t * TT_TILE_BYTES + clast;
+        cn = closing_piece_end(P, t) - st;
+        ca = (u32)((long long)st - P.shift); cslot = (u32)t * TT_TILE_BYTES + np - 1;
+        u32 v;
+        if (piece_settled_without_merge(P, text, ca, cn, v)) { P.piece_cnt[cslot] = v; P.tile_tok[t] += 1u; cn = 0; }   // this thread is the tile's only writer here
+        else if (cn <= (u32)LANE_MAX) { centry = tile_queue_entry(clast, np - 1, cn); }
+        else if (cn <= (u32)TT_WARP_PIECE_MAX) P.wq[atomicAdd(&P.hdr->nwq, 1u)] = ((u64)(u32)t << 32) | tile_queue_entry(clast, np - 1, cn);
+    }
+    // long pieces: those inside the tile (listed by the first kernel) and a long closing piece
+    const u32 nlong = nl + (cn > (u32)TT_WARP_PIECE_MAX ? 1u : 0u);
+    if (nlong) {
+        u32 b = atomicAdd(&P.hdr->nq_long, nlong);
+        for (u32 j = 0; j < nl && j < (u32)TT_TILE_LONGCAP; j++) {
+            const u32 idx = P.tile_long[(size_t)t * TT_TILE_LONGCAP + j];
+            const u32 o = P.piece_off16[(size_t)t * TT_TILE_BYTES + idx], o2 = P.piece_off16[(size_t)t * TT_TILE_BYTES + idx + 1];
+            P.lq[b++] = make_uint4((u32)((long long)t * TT_TILE_BYTES + o - P.shift), o2 - o, (u32)t * TT_TILE_BYTES + idx, 0u);
+        }
+        if (cn > (u32)TT_WARP_PIECE_MAX) P.lq[b] = make_uint4(ca, cn, cslot, 0u);
+    }
+    // short pieces: one reservation per warp
+    const u32 mine = ns + (centry ? 1u : 0u);
+    u32 pre = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) { const u32 v = __shfl_up_sync(FULL, pre, o); if (lane >= o) pre += v; }
+    const u32 tot = __shfl_sync(FULL, pre, 31);
+    u32 base = 0;
+    if (lane == 31 && tot) base = atomicAdd(&P.hdr->nq_short, tot);
+    base = __shfl_sync(FULL, base, 31) + pre - mine;
+    for (u32 e = 0; e < ns; e++) P.gq[base + e] = ((u64)(u32)t << 32) | P.q[(size_t)t * TT_TILE_QCAP + e];
+    if (centry) P.gq[base + ns] = ((u64)(u32)t << 32) | centry;
+}
+
 // Long pieces of the tiles [t_lo, t_hi) (at most MERGE_THREADS of them), a whole CTA each.  Called by all threads
 // of the CTA with the records of tile t_lo + tid in nl / np / last / c_end / closing_long.
 __device__ void cta_long_pieces(const PieceParams& P, const u8* __restrict__ text, int t_lo, int t_hi, u32 nl, u32 np, u32 last, u32 c_end,
@@ -842,22 +899,101 @@ __device__ void cta_long_pieces(const PieceParams& P, const u8* __restrict__ tex
     __syncthreads();
 }
 
+// Bulk text: the last CTA of k_merge to finish sums the token counts of every group of 256 tiles for k_scatter (a
+// counter cleared before the chain tells which CTA that is; nobody waits for anybody).  Called by every warp.
+__device__ __forceinline__ void merge_group_totals(const PieceParams& P, u32* s_warps_done) {
+    const int lane = threadIdx.x & 31;
+    const u32 FULL = 0xFFFFFFFFu;
+    if (P.grp_tok == nullptr) return;
+    __threadfence();
+    __syncwarp();
+    u32 fin = 0;
+    if (lane == 0 && atomicAdd(s_warps_done, 1u) == MERGE_WARPS - 1) fin = atomicAdd(&P.hdr->merge_done, 1u) == gridDim.x - 1;
+    if (!__shfl_sync(FULL, fin, 0)) return;
+    __threadfence();
+    const int ngroups = (P.ntiles + TT_GROUP_TILES - 1) / TT_GROUP_TILES;
+    for (int g = 0; g < ngroups; g++) {                               // one warp: eight loads per lane and group
+        u32 sum = 0;
+#pragma unroll
+        for (int u = 0; u < TT_GROUP_TILES / 32; u++) { const int t = g * TT_GROUP_TILES + u * 32 + lane; if (t < P.ntiles) sum += __ldcg(&P.tile_tok[t]); }
+#pragma unroll
+        for (int o = 16; o; o >>= 1) sum += __shfl_xor_sync(FULL, sum, o);
+        if (lane == 0) P.grp_tok[g] = sum;
+    }
+}
+
+// Bulk text (k_closing has gathered one list per length class): long pieces a CTA each, warp-class pieces a warp
+// each by index, short pieces 32 at a time by ticket, a thread each.
+__device__ void merge_bulk_lists(const PieceParams& P, const u8* __restrict__ text, u64* s_buf, u32* sc, u32* s_warps_done) {
+    const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+    const u32 FULL = 0xFFFFFFFFu;
+    const u32 nl = P.hdr->nq_long, nw = P.hdr->nwq, ns = P.hdr->nq_short;
+    for (u32 e = blockIdx.x; e < nl; e += gridDim.x) {                // block-uniform
+        const uint4 q = P.lq[e];
+        __syncthreads();
+        if (!piece_in_range(P, q.x, q.y, q.z, 3u)) continue;
+        const u32 m = cta_merge_long(text, q.x, q.y, P.tab, P.ext_id, P.stage, P.pairbuf + q.x, s_buf, sc);
+        if (tid == 0) piece_done(P, q.z, m);
+    }
+    if (nl > blockIdx.x) __syncthreads();
+    u64* wbuf = s_buf + wid * WARP_SMEM_WORDS;
+    const u32 W = gridDim.x * MERGE_WARPS, gw = (u32)wid * gridDim.x + blockIdx.x;
+    for (u32 j = gw; j < nw; j += W) {                                // bounded by the list length
+        const u64 x = P.wq[j];
+        const u32 t = (u32)(x >> 32), e = (u32)x;
+        warp_merge_piece(P, text, (u32)((long long)t * TT_TILE_BYTES + (e & 2047u) - P.shift), (e >> 22) + 1, t * TT_TILE_BYTES + ((e >> 11) & 2047u), wbuf, lane);
+    }
+    u32* const tok = reinterpret_cast<u32*>(wbuf);
+    for (;;) {                                                        // bounded by the list length
+        u32 e0 = 0;
+        if (lane == 0) e0 = atomicAdd(&P.hdr->t_short, (u32)LANE_SLOTS);
+        e0 = __shfl_sync(FULL, e0, 0);
+        if (e0 >= ns) break;
+        if (e0 + lane < ns) {
+            const u64 x = P.gq[e0 + lane];
+            const u32 t = (u32)(x >> 32), e = (u32)x;
+            const u32 a = (u32)((long long)t * TT_TILE_BYTES + (e & 2047u) - P.shift), n = (e >> 22) + 1, slot = t * TT_TILE_BYTES + ((e >> 11) & 2047u);
+            if (!piece_in_range(P, a, n, slot, 4u) || n < 2 || n > (u32)LANE_MAX) hdr_selfcheck_failed(P.hdr, P.epoch, 5u, a, n, slot, e0);
+            else {
+                const u32 m = lane_merge(tok, tok + LANE_SLOTS * LANE_MAX, lane, text, a, n, P.tab, P.ext_id, P.stage);
+                piece_done(P, slot, m);
+            }
+        }
+        __syncwarp();
+    }
+    merge_group_totals(P, s_warps_done);
+}
+
+// The merge kernel of bulk text (more tiles than a request's job search covers): works off the lists k_closing built.
+__global__ void __launch_bounds__(MERGE_THREADS, MERGE_CTAS_PER_SM)
+k_merge_bulk(const PieceParams P) {
+    extern __shared__ __align__(16) u64 s_buf[];              // MERGE_SMEM_BYTES
+    __shared__ u32 sc[48];
+    __shared__ u32 s_warps_done;
+    cudaTriggerProgrammaticLaunchCompletion();               // k_scatter may be placed; it waits for this grid's memory itself
+    grid_prefetch_l2(P.tab.slots, ((size_t)P.tab.mask + 1) * 2 * sizeof(uint4));
+    grid_prefetch_l2(P.tab.bytepair, 65536 * sizeof(u64));
+    if (threadIdx.x == 0) s_warps_done = 0;
+    cudaGridDependencySynchronize();                         // k_closing's lists are complete from here on
+    __syncthreads();
+    if (hdr_status(P.hdr, P.epoch) != 0) return;
+    merge_bulk_lists(P, P.base + P.shift, s_buf, sc, &s_warps_done);
+}
+
 __global__ void __launch_bounds__(MERGE_THREADS, MERGE_CTAS_PER_SM)
 k_merge(const PieceParams P) {
     extern __shared__ __align__(16) u64 s_buf[];              // MERGE_SMEM_BYTES
     __shared__ u32 sc[48];
     __shared__ uint4 s_long[TT_TILE_LONGCAP + 2];             // the long pieces of one tile
-    __shared__ u32 s_nlong, s_warps_done;
+    __shared__ u32 s_nlong;
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
     const u32 FULL = 0xFFFFFFFFu;
     cudaTriggerProgrammaticLaunchCompletion();               // k_scatter may be placed; it waits for this grid's memory itself
     grid_prefetch_l2(P.tab.slots, ((size_t)P.tab.mask + 1) * 2 * sizeof(uint4));
     grid_prefetch_l2(P.tab.bytepair, 65536 * sizeof(u64));
-    if (tid == 0) s_warps_done = 0;
     cudaGridDependencySynchronize();                         // the first kernel's per-tile records are complete from here on
     if (hdr_status(P.hdr, P.epoch) != 0) return;
     const u8* text = P.base + P.shift;
-
     // ---- records of this CTA's share of the tiles (long pieces, a whole CTA each; a request settles them after
     // its short pieces, bulk text before); the loads go out next to those of the job search below
     const int per = (P.ntiles + (int)gridDim.x - 1) / (int)gridDim.x;
@@ -872,7 +1008,7 @@ k_merge(const PieceParams P) {
     }
     u64* wbuf = s_buf + wid * WARP_SMEM_WORDS;
     const u32 W = gridDim.x * MERGE_WARPS, gw = (u32)wid * gridDim.x + blockIdx.x;   // numbered across the CTAs first
-    const bool big = P.wq != nullptr;                             // more than MERGE_SR_MAX_TILES tiles
+    const bool big = false;                                       // (bulk text took the lists above)
     // job search of a request: every lane sums the counts of a stretch of tiles, kept as 16 sums of `unit` tiles
     // (short pieces in the low half, warp-class pieces in the high half of a word)
     const int unit = (P.ntiles + 511) / 512;                      // 1..4 tiles per register
@@ -983,14 +1119,6 @@ k_merge(const PieceParams P) {
                 cta_long_pieces(P, text, t_lo, t_hi, a_nl, a_np, a_last, c_end, closing_long, s_buf, sc, s_long, &s_nlong);
             return;
         }
-    } else {
-        // bulk text: the warp-class pieces stand in one global list (the first kernel appended them tile by tile)
-        const u32 nwq = *P.nwq;
-        for (u32 j = gw; j < nwq; j += W) {                           // bounded by the list length
-            const u64 x = P.wq[j];
-            const u32 t = (u32)(x >> 32), e = (u32)x;
-            warp_merge_piece(P, text, (u32)((long long)t * TT_TILE_BYTES + (e & 2047u) - P.shift), (e >> 22) + 1, t * TT_TILE_BYTES + ((e >> 11) & 2047u), wbuf, lane);
-        }
     }
     for (int t0 = t_lo; t0 < t_hi; t0 += MERGE_THREADS) {            // block-uniform; shares beyond MERGE_THREADS tiles reload their records
         if (t0 != t_lo) {
@@ -1058,24 +1186,6 @@ k_merge(const PieceParams P) {
             }
             if (last_round) break;
         }
-    }
-    // ---- bulk text: the last CTA to finish sums the token counts of every group of 256 tiles for k_scatter (a counter
-    // zeroed by the kernel before this one tells which CTA that is; nobody waits for anybody)
-    if (P.grp_tok == nullptr) return;
-    __threadfence();
-    __syncwarp();
-    u32 fin = 0;
-    if (lane == 0 && atomicAdd(&s_warps_done, 1u) == MERGE_WARPS - 1) fin = atomicAdd(&P.hdr->merge_done, 1u) == gridDim.x - 1;
-    if (!__shfl_sync(FULL, fin, 0)) return;
-    __threadfence();
-    const int ngroups = (P.ntiles + TT_GROUP_TILES - 1) / TT_GROUP_TILES;
-    for (int g = 0; g < ngroups; g++) {                               // one warp: eight loads per lane and group
-        u32 sum = 0;
-#pragma unroll
-        for (int u = 0; u < TT_GROUP_TILES / 32; u++) { const int t = g * TT_GROUP_TILES + u * 32 + lane; if (t < P.ntiles) sum += __ldcg(&P.tile_tok[t]); }
-#pragma unroll
-        for (int o = 16; o; o >>= 1) sum += __shfl_xor_sync(FULL, sum, o);
-        if (lane == 0) P.grp_tok[g] = sum;
     }
 }
 

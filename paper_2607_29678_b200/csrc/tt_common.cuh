@@ -45,9 +45,11 @@ struct TTHeader {
     u32 n_pieces;            // number of pieces found (tt_pretokenize only)
     u32 t_tiles;             // ticket counter of k_merge's bulk mode (groups of tiles handed out); zeroed by the kernel before it
     u32 merge_done;          // CTAs of k_merge that have finished (bulk text: the last one sums the groups); zeroed likewise
-    u32 nwq;                 // bulk text: length of the global list of warp-class pieces (cleared by a memset before the chain)
+    u32 nwq;                 // bulk text: lengths of the global lists of warp-class, short and long pieces and the ticket
+    u32 nq_short, nq_long;   //            counter of the short list (all cleared by a memset before the chain)
+    u32 t_short;
     u32 dbg[8];              // first failed self-check of a kernel: site, then up to seven values (diagnostics only)
-    u32 pad[17];
+    u32 pad[14];
 };
 static_assert(sizeof(TTHeader) == 128, "header layout");
 
@@ -108,6 +110,8 @@ struct TTWorkspace {
     u32* piece_cnt;
     u32* q;
     u64* wq;           // bulk text only: warp-class pieces of all tiles (len / 33 + 64 entries)
+    u64* gq;           // bulk text only: short pieces of all tiles (len / 2 + 64 entries)
+    uint4* lq;         // bulk text only: long pieces of all tiles (len / 257 + 16 entries)
     int32_t* stage;    // token ids staged at the byte offset of their piece (len)
     u64* pairbuf;      // (token, rank) pairs of the long-piece path, indexed like the text (len)
     u8* cand;          // literal pass: length of the longest added-token literal starting at each byte (aligned frame)

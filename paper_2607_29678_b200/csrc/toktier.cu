@@ -490,15 +490,18 @@ static int run_pretok(const tt_vocab* v, const uint8_t* text, size_t len, const 
         k_lit_select<<<lgrid, 256, 0, st>>>(L);
         P.docmask = w.docmask; P.litstart = w.litstart; P.litin = w.litin;
     }
-    const size_t smem = align_up(v->cls_bytes, 16) + sizeof(u16) * F_COUNT * TT_SLOTS;
-    const int grid = P.ntiles < v->sm_count * 6 ? P.ntiles : v->sm_count * 6;
+    const size_t smem = sizeof(u16) * F_COUNT * TT_SLOTS;
+    const bool bulk = P.ntiles > MERGE_SR_MAX_TILES;
+    const int per_sm = bulk ? PRETOK_CTAS_BULK : PRETOK_CTAS_REQUEST;
+    const int grid = P.ntiles < v->sm_count * per_sm ? P.ntiles : v->sm_count * per_sm;
     if (v->pattern == TT_PATTERN_SPLIT3) {
         // stages A and B: span starts into cutmask (with the caller's document starts); stage C: pattern 0 with
         // those cuts as its document boundaries
         PretokParams C1 = P;
         C1.pattern = TT_PATTERN_CUTS; C1.startmask = reinterpret_cast<u16*>(w.cutmask);
         C1.want_prefix = 0; C1.litstart = nullptr; C1.litin = nullptr;
-        k_pretok<false><<<grid, TT_TILE_CHUNKS, smem, st>>>(C1, FrontParams{});
+        if (bulk) k_pretok<false, PRETOK_CTAS_BULK><<<grid, TT_TILE_CHUNKS, smem, st>>>(C1, FrontParams{});
+        else k_pretok<false, PRETOK_CTAS_REQUEST><<<grid, TT_TILE_CHUNKS, smem, st>>>(C1, FrontParams{});
         P.pattern = TT_PATTERN_CL100K; P.docmask = w.cutmask;
     }
     if (fused) {
@@ -506,8 +509,10 @@ static int run_pretok(const tt_vocab* v, const uint8_t* text, size_t len, const 
         F.tile_last = w.tile_last; F.tile_tok = w.tile_tok; F.tile_q = w.tile_q; F.tile_long = w.tile_long; F.piece_off16 = w.piece_off16;
         F.piece_cnt = w.piece_cnt; F.q = w.q; F.toktab = v->toktab; F.longtab = v->longtab; F.ext_id = v->d_ext_id;
         F.wq = P.ntiles > MERGE_SR_MAX_TILES ? w.wq : nullptr;
-        k_pretok<true><<<grid, TT_TILE_CHUNKS, smem, st>>>(P, F);
-    } else k_pretok<false><<<grid, TT_TILE_CHUNKS, smem, st>>>(P, FrontParams{});
+        if (bulk) k_pretok<true, PRETOK_CTAS_BULK><<<grid, TT_TILE_CHUNKS, smem, st>>>(P, F);
+        else k_pretok<true, PRETOK_CTAS_REQUEST><<<grid, TT_TILE_CHUNKS, smem, st>>>(P, F);
+    } else if (bulk) k_pretok<false, PRETOK_CTAS_BULK><<<grid, TT_TILE_CHUNKS, smem, st>>>(P, FrontParams{});
+    else k_pretok<false, PRETOK_CTAS_REQUEST><<<grid, TT_TILE_CHUNKS, smem, st>>>(P, FrontParams{});
     if (piece_off_dst)
         k_compact<<<grid, TT_TILE_CHUNKS, 0, st>>>(w.startmask, w.tile_cnt, P.nchunks, P.ntiles, shift, (long long)len,
                                                    piece_off_dst, w.hdr, P.epoch);
@@ -589,8 +594,8 @@ static int encode_impl(const tt_vocab* v, const uint8_t* text, size_t len, const
     S.ids_out = ids_out; S.count_out = (long long*)count_out; S.status_out = status_out;
     S.docmask = doc_off ? w.docmask : nullptr; S.doc_off = (const long long*)doc_off; S.n_docs = (int)n_docs;
     S.ids_off_out = (long long*)ids_off_out;
-    if (ev) k_scatter<<<tile_grid, BPE_THREADS, 0, st>>>(S);
-    else CK(launch_after(k_scatter, tile_grid, BPE_THREADS, st, S));
+    if (ev) { if (big) k_scatter_bulk<<<tile_grid, BPE_THREADS, 0, st>>>(S); else k_scatter<<<tile_grid, BPE_THREADS, 0, st>>>(S); }
+    else CK(launch_after(big ? k_scatter_bulk : k_scatter, tile_grid, BPE_THREADS, st, S));
     MARK(3);
 #undef MARK
     CK(cudaGetLastError());

@@ -1337,3 +1337,117 @@ k_scatter(const ScatterParams P) {
         }
     }
 }
+
+// ---- K5 for bulk text: a warp per tile, no barrier after the prologue -----------------------------------------
+// Each CTA takes a contiguous range of tiles, its warps every eighth tile of it.  A warp knows where its tile's ids
+// go from the token counts of the tiles before it (group totals, then tile counts), scans the tile's pieces 128 at
+// a time (four neighbouring pieces per lane, one 16-byte load) with warp shuffles, and copies pieces of more than
+// eight tokens with all its lanes.
+__global__ void __launch_bounds__(BPE_THREADS)
+k_scatter_bulk(const ScatterParams P) {
+    __shared__ unsigned long long s_sum[66];
+    const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+    const u32 FULL = 0xFFFFFFFFu;
+    cudaGridDependencySynchronize();                         // k_merge_bulk's (and with it the kernels' before it) results are complete
+    const int per = (P.ntiles + (int)gridDim.x - 1) / (int)gridDim.x;
+    const int tile_lo = (int)blockIdx.x * per, tile_hi = min(P.ntiles, tile_lo + per);
+    unsigned long long before = 0, total = 0;
+    {
+        const int ngroups = (P.ntiles + TT_GROUP_TILES - 1) / TT_GROUP_TILES, g_lo = tile_lo / TT_GROUP_TILES;
+        for (int g = tid; g < ngroups; g += BPE_THREADS) { const u32 x = P.grp_tok[g]; total += x; if (g < g_lo) before += x; }
+        for (int t = g_lo * TT_GROUP_TILES + tid; t < tile_lo; t += BPE_THREADS) before += P.tile_tok[t];
+    }
+    cta_sum2_u64(before, total, s_sum);
+    int status = hdr_status(P.hdr, P.epoch);
+    if (status == 0 && total > P.ids_cap) status = 5;          // TT_ERR_CAPACITY
+    if (blockIdx.x == 0 && tid == 0) {
+        if (P.status_out) *P.status_out = status;
+        if (P.count_out) *P.count_out = status ? 0 : (long long)total;
+    }
+    if (status != 0) {
+        if (P.ids_off_out)
+            for (long long d = (long long)blockIdx.x * blockDim.x + tid; d <= P.n_docs; d += (long long)gridDim.x * blockDim.x) P.ids_off_out[d] = 0;
+        return;
+    }
+    if (P.ids_off_out && blockIdx.x == 0) {
+        const long long len = P.hi - P.shift;
+        for (int d = P.n_docs - tid; d >= 0 && P.doc_off[d] >= len; d -= blockDim.x) P.ids_off_out[d] = (long long)total;
+    }
+    // tokens of the tiles of this CTA's range before the warp's first tile
+    u32 carry = (u32)before;
+    {
+        u32 x = (lane < wid && tile_lo + lane < tile_hi) ? P.tile_tok[tile_lo + lane] : 0u;
+#pragma unroll
+        for (int o = 16; o; o >>= 1) x += __shfl_xor_sync(FULL, x, o);
+        carry += x;
+    }
+    for (int tile = tile_lo + wid; tile < tile_hi; tile += BPE_WARPS) {   // warp-uniform
+        const u32 np = P.tile_cnt[tile];
+        // the seven tiles between this one and the warp's next
+        u32 skip = (lane >= 1 && lane < BPE_WARPS && tile + lane < tile_hi) ? P.tile_tok[tile + lane] : 0u;
+        const size_t p0 = (size_t)tile * TT_TILE_BYTES;
+        const long long t0 = (long long)tile * TT_TILE_BYTES - P.shift;      // text offset of the tile start
+        u32 run = carry;
+        uint4 v = make_uint4(0, 0, 0, 0);
+        uint2 o4 = make_uint2(0, 0);
+        if (4u * lane < np) { v = *reinterpret_cast<const uint4*>(P.piece_cnt + p0 + 4 * lane); o4 = *reinterpret_cast<const uint2*>(P.piece_off16 + p0 + 4 * lane); }
+        for (u32 b = 0; b < np; b += 128) {                               // warp-uniform
+            // the next 128 pieces
+            uint4 vn = make_uint4(0, 0, 0, 0);
+            uint2 on = make_uint2(0, 0);
+            const u32 j0 = b + 128 + 4 * lane;
+            if (j0 < np) { vn = *reinterpret_cast<const uint4*>(P.piece_cnt + p0 + j0); on = *reinterpret_cast<const uint2*>(P.piece_off16 + p0 + j0); }
+            const u32 i0 = b + 4 * lane;
+            const int32_t x[4] = {(int32_t)v.x, (int32_t)v.y, (int32_t)v.z, (int32_t)v.w};
+            const u32 off[4] = {o4.x & 0xFFFFu, o4.x >> 16, o4.y & 0xFFFFu, o4.y >> 16};
+            u32 c[4], mine = 0;
+#pragma unroll
+            for (int h = 0; h < 4; h++) { c[h] = i0 + h < np ? (x[h] >= 0 ? 1u : (u32)(-x[h])) : 0u; mine += c[h]; }
+            u32 inc = mine;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) { const u32 y = __shfl_up_sync(FULL, inc, o); if (lane >= o) inc += y; }
+            const u32 tot = __shfl_sync(FULL, inc, 31);
+            u32 dst = run + inc - mine;
+            u32 bigmask = 0;                                              // which of my four pieces have more than eight tokens
+#pragma unroll
+            for (int h = 0; h < 4; h++) {
+                const u32 i = i0 + h;
+                if (i < np) {
+                    const u32 src = (u32)(t0 + off[h]);
+                    if ((unsigned long long)dst + c[h] > total || (x[h] < 0 && t0 + off[h] + c[h] > P.hi - P.shift)) hdr_selfcheck_failed(P.hdr, P.epoch, 7u, (u32)tile, i, (u32)x[h], dst);
+                    else if (x[h] >= 0) P.ids_out[dst] = x[h];
+                    else if (c[h] <= 8) { for (u32 kk = 0; kk < c[h]; kk++) P.ids_out[dst + kk] = P.stage[src + kk]; }
+                    else bigmask |= 1u << h;
+                    if (P.docmask) {
+                        const long long g = (long long)tile * TT_TILE_BYTES + off[h];
+                        if ((P.docmask[g >> 5] >> (g & 31)) & 1) {
+                            // every document that starts at this byte (empty ones included) gets this token offset
+                            const long long want = g - P.shift;
+                            int lo = 0, hi2 = P.n_docs;
+                            while (lo < hi2) { int mid = (lo + hi2) >> 1; if (P.doc_off[mid] < want) lo = mid + 1; else hi2 = mid; }
+                            for (int d = lo; d <= P.n_docs && P.doc_off[d] == want; d++) P.ids_off_out[d] = dst;
+                        }
+                    }
+                }
+                dst += c[h];
+            }
+            // pieces of more than eight tokens: copied by the whole warp, one after the other
+#pragma unroll
+            for (int h = 0; h < 4; h++) {
+                for (u32 m = __ballot_sync(FULL, (bigmask >> h) & 1); m; m &= m - 1) {     // warp-uniform
+                    const int l = __ffs(m) - 1;
+                    u32 d2 = run + inc - mine;
+#pragma unroll
+                    for (int g = 0; g < 4; g++) if (g < h) d2 += c[g];
+                    const u32 src = __shfl_sync(FULL, (u32)(t0 + off[h]), l), dd = __shfl_sync(FULL, d2, l), cc = __shfl_sync(FULL, c[h], l);
+                    for (u32 kk = lane; kk < cc; kk += 32) P.ids_out[dd + kk] = P.stage[src + kk];
+                }
+            }
+            run += tot;
+            v = vn; o4 = on;
+        }
+#pragma unroll
+        for (int o = 16; o; o >>= 1) skip += __shfl_xor_sync(FULL, skip, o);
+        carry = run + skip;
+    }
+}

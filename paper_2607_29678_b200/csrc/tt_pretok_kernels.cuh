@@ -238,12 +238,16 @@ __device__ __forceinline__ void front_piece_queue(const FrontParams& F, int tile
 // is a single byte, an extracted literal or a whole vocabulary entry (one 32-byte probe), and queued for k_merge
 // otherwise.  Everything a tile leaves behind has this CTA as its only writer: no atomics on global memory, no
 // counter that would have to be cleared before the call.
-template <bool FUSED>
-__global__ void __launch_bounds__(TT_TILE_CHUNKS, 6)
+// MINB = CTAs per SM the kernel is compiled for.  A request (at most a few tiles per CTA) is a latency chain and
+// gets the registers it wants (6 CTAs of 128 threads, 80 registers); bulk text is bound by instruction issue and
+// by the latencies between its barriers, which more resident warps hide (10 CTAs, 48 registers, a few spills:
+// the 132 MB batch 1.80 -> 1.64 ms).
+constexpr int PRETOK_CTAS_REQUEST = 6, PRETOK_CTAS_BULK = 10;
+template <bool FUSED, int MINB>
+__global__ void __launch_bounds__(TT_TILE_CHUNKS, MINB)
 k_pretok(const PretokParams P, const FrontParams F) {
     extern __shared__ __align__(16) u8 smem_raw[];
-    u8* tables = smem_raw;                                            // class tables
-    u16 (*sm)[TT_SLOTS] = reinterpret_cast<u16 (*)[TT_SLOTS]>(smem_raw + ((P.cls_bytes + 15) & ~15));
+    u16 (*sm)[TT_SLOTS] = reinterpret_cast<u16 (*)[TT_SLOTS]>(smem_raw);        // class masks of the tile and its halo
     __shared__ long long scratch[40];
     __shared__ u32 s_need, s_first;
     __shared__ u32 s_islast;
@@ -260,14 +264,10 @@ k_pretok(const PretokParams P, const FrontParams F) {
         // the whole-piece table is probed at random a few microseconds from now: ask for it to be brought into L2
         if (F.toktab.slots != nullptr) grid_prefetch_l2(F.toktab.slots, ((size_t)F.toktab.mask + 1) * sizeof(TokSlot));
     }
-    // the 128-byte ASCII table is always staged; the two-stage Unicode table only once a tile holds a
-    // non-ASCII byte (pattern 1 stages it at once: its sparse matcher may read beyond the tile)
-    bool tables_loaded = P.pattern == 1;
-    for (int i = tid * 16; i < P.cls_bytes; i += blockDim.x * 16)
-        if (tables_loaded || i >= P.cls_bytes - 128)
-            *reinterpret_cast<uint4*>(tables + i) = *reinterpret_cast<const uint4*>(P.cls_tables + i);
+    // The class tables stay in global memory (21 KB, read through L1): chunks of plain ASCII -- nearly all of a
+    // transcript -- are classified without any table, so shared memory is left to the masks and more CTAs fit an SM.
     ClassTables T;
-    T.stage1 = tables; T.stage2 = tables + 0x1100; T.ascii = tables + P.cls_bytes - 128;
+    T.stage1 = P.cls_tables; T.stage2 = P.cls_tables + 0x1100; T.ascii = P.cls_tables + P.cls_bytes - 128;
     SeqCtx SC;
     SC.base = P.base; SC.lo = P.lo; SC.hi = P.hi; SC.docmask = P.docmask; SC.T = T;
     u32 any_bad = 0;
@@ -276,29 +276,6 @@ k_pretok(const PretokParams P, const FrontParams F) {
         __syncthreads();
         if (tid == 0) { s_need = 0; s_first = 0xFFFFFFFFu; s_ns = 0; s_nw = 0; s_nl = 0; s_total = 0; s_nslow = 0; }
         const long long c_first = (long long)tile * TT_TILE_CHUNKS;
-        if (!tables_loaded) {                                         // block-uniform
-            bool hi_bit = false;
-            {
-                const long long chunk = c_first + tid;
-                if (chunk >= 0 && chunk < P.nchunks) {
-                    const uint4 v = *reinterpret_cast<const uint4*>(P.base + chunk * TT_CHUNK);
-                    hi_bit = ((v.x | v.y | v.z | v.w) & 0x80808080u) != 0;
-                }
-            }
-            if (tid < TT_LOW_HALO + 1) {
-                const long long chunk = tid < TT_LOW_HALO ? c_first - TT_LOW_HALO + tid : c_first + TT_TILE_CHUNKS;
-                if (chunk >= 0 && chunk < P.nchunks) {
-                    const uint4 v = *reinterpret_cast<const uint4*>(P.base + chunk * TT_CHUNK);
-                    hi_bit = hi_bit || ((v.x | v.y | v.z | v.w) & 0x80808080u) != 0;
-                }
-            }
-            if (__syncthreads_or(hi_bit)) {
-                for (int i = tid * 16; i < P.cls_bytes - 128; i += blockDim.x * 16)
-                    *reinterpret_cast<uint4*>(tables + i) = *reinterpret_cast<const uint4*>(P.cls_tables + i);
-                tables_loaded = true;
-                __syncthreads();
-            }
-        }
         // phase A: classify own chunk (+ the halo chunks)
         {
             const long long chunk = c_first + tid;
@@ -335,12 +312,6 @@ k_pretok(const PretokParams P, const FrontParams F) {
         __syncthreads();
         const u32 need_all = s_need;
         if (need_all) {                                               // block-uniform
-            if (!tables_loaded) {                                     // the walks below classify text outside the tile
-                for (int i = tid * 16; i < P.cls_bytes - 128; i += blockDim.x * 16)
-                    *reinterpret_cast<uint4*>(tables + i) = *reinterpret_cast<const uint4*>(P.cls_tables + i);
-                tables_loaded = true;
-                __syncthreads();
-            }
             const long long below = (c_first - TT_LOW_HALO) * TT_CHUNK;    // first byte of the low halo
             if (need_all & NEED_N) tc.n_before = coop_back_num(P, T, below, scratch);
             if (need_all & NEED_A) tc.nl_absorbed_before = coop_back_nl(P, T, below, scratch);

@@ -33,7 +33,10 @@ sys.path.insert(0, ROOT)
 import workloads as wl  # noqa: E402
 
 FALLBACK_HBM_GBS = 6650.0
-N_DISTINCT_INPUTS = 8
+N_DISTINCT_INPUTS = 20        # fresh-sample protocol: 20 distinct seeded inputs per config
+WORKLOAD_C3 = ("C3: one 1,000,000-char agent-transcript request per step, cl100k-style pattern, 256+100,000 merges; "
+               "device-resident text -> device int32 IDs")
+KERNELS_PER_REQUEST = 3       # k_pretok<fused>, k_merge, k_scatter
 
 
 def measured_peak():
@@ -140,12 +143,62 @@ def run_reference(args, rank, world):
     line = {"impl": "reference", "metric": "encode_latency_1M_chars", "value": round(val, 4), "unit": "ms", "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(val, 4), "higher_is_better": False,
             "scaling": "weak", "vs_baseline": None, "dtype": "u8/int32", "data": "synthetic",
-            "config": {"workload": "C3: one 1,000,000-char agent-transcript request, cl100k-style pattern, 256+100,000 merges"},
+            "config": {"workload": WORKLOAD_C3},
             "cpu_baseline": {"value": round(val, 4), "unit": "ms", "cores": ncores, "kind": "oracle",
                              "sample": f"{args.steps} whole C3 requests, all host threads"},
             "e2e": {"value": round(val, 4), "unit": "ms", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
     print(json.dumps(line), flush=True)
+
+
+def config_leg(tt, name, flush_l2, stream, n_inputs=N_DISTINCT_INPUTS, timed_reps=8):
+    """Fresh-sample and steady-state latency of one config through tt_encode on its own text, pattern and vocabulary:
+    one cold call (L2 flushed) per distinct seeded input, then repeats of one input; per-kernel device times."""
+    import torch
+    cfg = wl.CONFIGS[name]
+    merges, byte_map = wl.load_vocab(cfg)
+    v = tt.Vocab(merges, byte_map, cfg.pattern_id)
+    host = [wl.request(cfg, sample=200 + s) for s in range(n_inputs)]
+    dev = [torch.from_numpy(t).cuda() for t in host]
+    bufs = v.alloc(max(t.size for t in host))
+    for k in range(3):
+        v.encode(dev[k % n_inputs], bufs)
+    torch.cuda.synchronize()
+    cold, toks = [], []
+    for k in range(n_inputs):
+        flush_l2(); torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream); v.encode(dev[k], bufs); b.record(stream)
+        torch.cuda.synchronize()
+        cold.append(a.elapsed_time(b)); toks.append(int(bufs["count"].item()))
+        assert int(bufs["status"].item()) == 0
+    warm = []
+    for k in range(3 + 30):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream); v.encode(dev[0], bufs); b.record(stream)
+        torch.cuda.synchronize()
+        if k >= 3:
+            warm.append(a.elapsed_time(b))
+    kt = {}
+    for k in range(timed_reps):
+        flush_l2(); torch.cuda.synchronize()
+        for kn, ms in v.encode_timed(dev[k % n_inputs], bufs).items():
+            kt.setdefault(kn, []).append(ms)
+    kmean = {n: sum(x) / len(x) for n, x in kt.items()}
+    nbytes = int(np.mean([t.size for t in host]))
+    ntok = int(np.mean(toks))
+    out = {"workload": f"{name}: one {cfg.n_chars:,}-char request, pattern {cfg.pattern_id}, 256+{cfg.n_merges:,} merges; "
+                       f"{n_inputs} distinct seeded inputs, one cold call each (L2 flushed before the call, outside the events)",
+           "bytes": nbytes, "tokens": ntok, "cold_p50_ms": round(pct(cold, 0.5), 4), "cold_p99_ms": round(pct(cold, 0.99), 4),
+           "steady_p50_ms": round(pct(warm, 0.5), 4), "kernel_ms": {n: round(x, 4) for n, x in kmean.items()}}
+    peak, peak_kind = measured_peak()
+    dom = max(kmean, key=kmean.get)
+    algo = nbytes + 4 * ntok + 8 + vocab_table_bytes(cfg.n_merges)
+    out["roofline"] = {"bound": "hbm", "kernel": dom, "algorithmic_bytes": algo, "achieved": round(algo / (kmean[dom] * 1e-3) / 1e9, 2),
+                       "peak": peak, "unit": "GB/s", "frac": round(algo / (kmean[dom] * 1e-3) / 1e9 / peak, 5), "of": peak_kind,
+                       "whole_call_frac": round(algo / (pct(cold, 0.5) * 1e-3) / 1e9 / peak, 5), "traffic": None}
+    del v, bufs, dev
+    return out
 
 
 def main():
@@ -408,21 +461,29 @@ def main():
         batch = {"workload": f"C5: {boff.size - 1} requests, lognormal lengths (median 350,000 chars), one tt_encode_batch call; "
                              "input larger than L2",
                  "per_request_ms": {"p50": round(pct(per_req, 0.5), 4), "p99": round(pct(per_req, 0.99), 4),
-                                    "what": "the same requests encoded one at a time with tt_encode (10,000 to 3,000,000 chars each)"},
+                                    "what": "the same requests encoded one at a time with tt_encode (10,000 to 3,000,000 chars each)",
+                                    "inside_the_batch_call": "every document's ids are complete only when the call's last kernel has "
+                                                             "run (ids are scattered tile by tile across the whole batch), so the "
+                                                             "latency of a request inside the one call is the call's: " + str(round(bms, 3)) + " ms"},
                  "chars": int(bchars), "bytes": int(btext.size), "tokens": btok, "ms": round(bms, 3),
                  "chars_per_s": round(cps, 1), "GB_per_s": round(btext.size / (bms * 1e-3) / 1e9, 3),
                  "hbm_roofline_frac": round((btext.size + 4 * btok + 16 * boff.size) / (bms * 1e-3) / 1e9 / peak, 5)}
         if args.batch_docs == c5.n_docs and world == 1:
-            # the batch is bound by instruction issue, not by HBM: warp instructions of the four kernels (ncu capture
-            # of this very workload, profiles/c5_batch_256_requests_kernels.md) per second against what the SMs can
-            # issue (SMs x 4 schedulers x 1 warp instruction per clock at the maximum SM clock)
+            # the batch is bound by instruction issue, not by HBM: warp instructions of its kernels (from the committed
+            # ncu capture of this very workload) per second against what the SMs can issue (SMs x 4 schedulers x 1 warp
+            # instruction per clock at the maximum SM clock)
             sm_count = torch.cuda.get_device_properties(0).multi_processor_count
             mhz = (clocks or {}).get("sm_max_mhz") or 1965.0
             issue_peak = sm_count * 4 * mhz * 1e6
-            winst = sum(NCU_BATCH_WARP_INST.values())
-            batch["alu_roofline"] = {"bound": "alu", "achieved": round(winst / (bms * 1e-3) / 1e9, 1), "peak": round(issue_peak / 1e9, 1),
-                                     "unit": "G warp-instructions/s", "frac": round(winst / (bms * 1e-3) / issue_peak, 4),
-                                     "warp_instructions": winst}
+            winst_by_kernel = ncu_capture("batch_warp_inst")
+            if winst_by_kernel:
+                winst = sum(winst_by_kernel.values())
+                batch["alu_roofline"] = {"bound": "alu", "achieved": round(winst / (bms * 1e-3) / 1e9, 1), "peak": round(issue_peak / 1e9, 1),
+                                         "unit": "G warp-instructions/s", "frac": round(winst / (bms * 1e-3) / issue_peak, 4),
+                                         "warp_instructions": winst, "source": "ncu capture of these sources (smsp__inst_executed.sum)"}
+            else:
+                batch["alu_roofline"] = {"bound": "alu", "peak": round(issue_peak / 1e9, 1), "unit": "G warp-instructions/s",
+                                         "achieved": None, "frac": None, "capture_stale": True}
         del d_text, bb
 
     if rank != 0:
@@ -453,6 +514,12 @@ def main():
             del vv, vbufs
         variants["what"] = "tt_encode of one 1,000,000-char transcript under the other pattern ids (o200k-style with its own 199,744-merge vocabulary)"
 
+    # ---- the other single-request configs: C1 (4,000 chars), C2 (100,000 chars, 5 % non-ASCII), C4 (3,000,000 chars with
+    # adversarial runs, o200k-style pattern, 199,744 merges) ----
+    configs = None
+    if not args.no_batch:
+        configs = {name: config_leg(tt, name, flush_l2, stream) for name in ("C1", "C2", "C4")}
+
     # ---- roofline of the dominant kernel: algorithmic bytes of one request / its device time ----
     peak, peak_kind = measured_peak()
     nbytes = int(np.mean([t.size for t in host_texts]))
@@ -461,7 +528,10 @@ def main():
     dom_ms = kmean[dominant]
     achieved = algo_bytes / (dom_ms * 1e-3) / 1e9
     roofline = {"bound": "hbm", "kernel": dominant, "achieved": round(achieved, 2), "peak": peak, "unit": "GB/s",
-                "frac": round(achieved / peak, 5), "of": peak_kind, "traffic": ncu_traffic(dominant),
+                "frac": round(achieved / peak, 5), "of": peak_kind,
+                "traffic": (ncu_capture("c3_dram_bytes") or {}).get(dominant),
+                "traffic_what": "dram__bytes_read.sum + dram__bytes_write.sum of that kernel, one launch, from the committed ncu capture "
+                                "(null when the capture belongs to other sources)",
                 "algorithmic_bytes": algo_bytes, "kernel_ms": {k: round(v, 4) for k, v in kmean.items()},
                 "whole_call_frac": round(algo_bytes / (ms_per_step * 1e-3) / 1e9 / peak, 5),
                 "nominal_peak_frac": round(achieved / 8000.0, 5)}
@@ -471,10 +541,9 @@ def main():
         "metric": "encode_latency_1M_chars", "value": round(ms_per_step, 4), "unit": "ms", "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(ms_per_step, 4), "higher_is_better": False,
         "scaling": "weak", "vs_baseline": None, "dtype": "u8/int32", "data": "synthetic",
-        "config": {"workload": "C3: one 1,000,000-char agent-transcript request per step, cl100k-style pattern, "
-                               "256+100,000 merges; device-resident text -> device int32 IDs",
+        "config": {"workload": WORKLOAD_C3,
                    "chars": cfg.n_chars, "bytes": nbytes, "tokens": n_tokens_last,
-                   "timing": f"CUDA events around each tt_encode call; {N_DISTINCT_INPUTS} distinct seeded inputs in rotation; "
+                   "timing": f"CUDA events around each tt_encode call; {min(N_DISTINCT_INPUTS, args.steps + args.warmup)} distinct seeded inputs in rotation; "
                              "L2 flushed (512 MiB written, then read back so no dirty lines remain) before every timed step, outside the events",
                    "replicas": world},
         "latency_ms": {"cold_p50": round(pct(cold, 0.5), 4), "cold_p99": round(pct(cold, 0.99), 4),
@@ -486,7 +555,7 @@ def main():
                 "api": "tt_encode_host, wall clock of the synchronous call; pinned host buffers: text DMA'd from the caller's "
                        "buffer, ids written by the scatter kernel into the caller's pinned buffer; pageable_p50: the same call "
                        "on pageable buffers (staged through pinned memory inside the library)"},
-        "gpu_launches": 4 * args.steps,
+        "gpu_launches": KERNELS_PER_REQUEST * args.steps,
         "batch": batch,
         "span_export": {"ms_p50": round(pct(span_ms, 0.5), 4), "what": "tt_spans on the ids of one C3 request: byte and character "
                         "offsets per token, device to device; the paper adds 0.13-0.73 ms for this step on its hardware"},
@@ -495,6 +564,7 @@ def main():
                           "what": "tt_session_append of 1,500 chars (host bytes in, wall clock, synchronous) to a session holding "
                                   "~1M chars; ids checked against a full tokenization; the paper reports 1.23 ms P50 at 1M context"},
         "pattern_variants": variants,
+        "configs": configs,
         "roofline": roofline,
         "cpu_baseline": cpu,
         "clocks": clocks,
@@ -511,17 +581,32 @@ def vocab_table_bytes(n_merges: int) -> int:
     return 8 * n_merges + 4 * (256 + n_merges) + 21632
 
 
-# Warp instructions per launch (smsp__inst_executed.sum) from the committed ncu capture of the C5 batch
-# (profiles/c5_batch_256_requests_kernels.md).
-NCU_BATCH_WARP_INST = {"pretok": 373_891_564, "lookup": 360_754_739, "merge": 148_638_787, "scatter": 163_907_810}
+def csrc_hash() -> str:
+    """SHA-256 over the CUDA sources (the figures below belong to one state of them)."""
+    import hashlib
+    h = hashlib.sha256()
+    d = os.path.join(ROOT, "paper_2607_29678_b200", "csrc")
+    for f in sorted(os.listdir(d)):
+        if f.endswith((".cu", ".cuh", ".inc")):
+            with open(os.path.join(d, f), "rb") as fh:
+                h.update(f.encode()); h.update(fh.read())
+    return h.hexdigest()[:16]
 
-# DRAM bytes (read + write) per launch from the committed ncu capture of the C3 request
-# (profiles/c3_1M_request_kernels.md).
-NCU_TRAFFIC = {"merge": 9_463_296, "lookup": 9_557_760, "pretok": 1_091_328, "scatter": 1_235_712}
+
+# Figures that only a profiler can give (DRAM bytes per launch, warp instructions per launch), from the committed ncu
+# captures.  They belong to the source state whose hash is recorded with them; with other sources they are not
+# printed as measurements (the keys are null and "capture_stale" is true).
+NCU_CAPTURE = {
+    "csrc": None,                       # filled in when the captures are refreshed
+    "c3_dram_bytes": {},                # kernel -> dram__bytes_read.sum + dram__bytes_write.sum per launch, one C3 request
+    "batch_warp_inst": {},              # kernel -> smsp__inst_executed.sum per launch, the 256-request batch
+}
 
 
-def ncu_traffic(kernel: str):
-    return NCU_TRAFFIC.get(kernel)
+def ncu_capture(key: str):
+    if NCU_CAPTURE["csrc"] != csrc_hash():
+        return None
+    return NCU_CAPTURE.get(key) or None
 
 
 if __name__ == "__main__":

@@ -1212,12 +1212,14 @@ struct ScatterParams {
     long long* ids_off_out;    // batch: n_docs + 1 token offsets
 };
 
+constexpr int SCATTER_STAGE_IDS = 2048;                   // ids of one work item that are put together in shared memory
 __global__ void __launch_bounds__(BPE_THREADS)
 k_scatter(const ScatterParams P) {
     __shared__ u32 sc[48];
     __shared__ u32 s_big[TT_TILE_BYTES / 8][3];
     __shared__ u32 s_nbig;
     __shared__ u32 s_np[BPE_THREADS];                         // pieces of the next tiles of this CTA's range
+    __shared__ int32_t s_out[SCATTER_STAGE_IDS];              // the ids of one item on their way out
     __shared__ unsigned long long s_sum[66];
     const int tid = threadIdx.x;
     cudaGridDependencySynchronize();                         // k_merge's (and with it the first kernel's) results are complete from here on
@@ -1298,6 +1300,10 @@ k_scatter(const ScatterParams P) {
             const u32 c0 = i0 < np ? (x0 >= 0 ? 1u : (u32)(-x0)) : 0u, c1 = i0 + 1 < np ? (x1 >= 0 ? 1u : (u32)(-x1)) : 0u;
             u32 tot;
             const u32 d0 = carry + cta_excl_sum_scan(c0 + c1, sc, &tot);
+            // An item without pieces of more than eight tokens (nearly all) is put together in shared memory and leaves in
+            // whole lines, every thread writing consecutive words: the output may be mapped host memory, where a warp that
+            // writes every other word costs a bus transaction per word.
+            const bool staged = !__syncthreads_or(c0 > 8 || c1 > 8) && tot <= (u32)SCATTER_STAGE_IDS;
 #pragma unroll
             for (int h = 0; h < 2; h++) {
                 const u32 i = i0 + h, c = h ? c1 : c0, dst = h ? d0 + c0 : d0, off = h ? o2 >> 16 : o2 & 0xFFFFu;
@@ -1305,8 +1311,9 @@ k_scatter(const ScatterParams P) {
                 if (i >= np) continue;
                 if ((unsigned long long)dst + c > total || (x < 0 && t0 + off + c > P.hi - P.shift)) { hdr_selfcheck_failed(P.hdr, P.epoch, 6u, (u32)tile, i, (u32)x, dst); continue; }
                 const u32 src = (u32)(t0 + off);
-                if (x >= 0) P.ids_out[dst] = x;
-                else if (c <= 8) { for (u32 kk = 0; kk < c; kk++) P.ids_out[dst + kk] = P.stage[src + kk]; }
+                int32_t* const out = staged ? s_out - carry : P.ids_out;             // same index either way
+                if (x >= 0) out[dst] = x;
+                else if (c <= 8) { for (u32 kk = 0; kk < c; kk++) out[dst + kk] = P.stage[src + kk]; }
                 else {
                     const u32 slot = atomicAdd(&s_nbig, 1u);
                     if (slot < TT_TILE_BYTES / 8) { s_big[slot][0] = src; s_big[slot][1] = dst; s_big[slot][2] = c; }
@@ -1321,6 +1328,10 @@ k_scatter(const ScatterParams P) {
                         for (int d = lo; d <= P.n_docs && P.doc_off[d] == want; d++) P.ids_off_out[d] = dst;
                     }
                 }
+            }
+            if (staged) {                                             // block-uniform
+                __syncthreads();
+                for (u32 kk = tid; kk < tot; kk += BPE_THREADS) P.ids_out[carry + kk] = s_out[kk];
             }
             carry += tot;
             __syncthreads();

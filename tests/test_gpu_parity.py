@@ -212,6 +212,44 @@ def test_pretokenize_capacity_rule():
     assert int(npc.item()) == 0 and int(bufs["status"].item()) == 0
 
 
+def test_whole_piece_table_holds_exactly_the_self_encoding_entries():
+    """tt_vocab_table_entries against the oracle: an entry of 2..24 bytes belongs to the whole-piece table exactly if
+    the oracle's BPE of its own bytes is that one entry (the library decides this with its merge kernel at load)."""
+    for name in ("C1", "C2"):
+        cv = cpu_vocab(name)
+        want = 0
+        for r in range(cv.n_merges):
+            t = cv.token_bytes(256 + r)
+            if 2 <= len(t) <= 24:
+                ids = cv.bpe(t, 0)
+                want += int(ids.size == 1 and ids[0] == 256 + r)
+        assert gpu_vocab(name).table_entries() == want
+
+
+@pytest.mark.parametrize("pattern", [0, 1])
+def test_every_ascii_code_in_random_strings(pattern):
+    """Strings over all 128 ASCII codes (control characters included), many of them aligned so that whole 16-byte
+    chunks are ASCII: the table-free classification of such chunks against the oracle's class table, through the
+    piece boundaries and the ids."""
+    rng = random.Random(900 + pattern)
+    name = "C2" if pattern == 0 else "C4"
+    docs = []
+    for _ in range(3000):
+        n = rng.choice([1, 5, 16, 17, 31, 32, 48, 100, 333])
+        docs.append(bytes(rng.randrange(128) for _ in range(n)))
+    docs.append(bytes(range(128)) * 3)
+    text = np.frombuffer(b"".join(docs), dtype=np.uint8)
+    off = np.zeros(len(docs) + 1, dtype=np.int64)
+    off[1:] = np.cumsum([len(d) for d in docs])
+    _batch_pieces_check_arrays(name, pattern, text, off)
+    ids, ioff, status = gpu_encode_batch(gpu_vocab(name), text, off)
+    want, woff = cpu_vocab(name).encode_batch(text, off, pattern, nthreads=8)
+    assert status == 0 and same(ioff, woff) and same(ids, want)
+    one, status = gpu_encode(gpu_vocab(name), text, offset=5)
+    want1, _ = cpu_vocab(name).encode(text, pattern, nthreads=8)
+    assert status == 0 and same(one, want1)
+
+
 def test_host_wrapper_and_non_identity_ids():
     import paper_2607_29678_b200 as tt
     rng = random.Random(4)

@@ -499,6 +499,9 @@ __device__ __forceinline__ u32 cta_min_u32(u32 v, u32* scratch /* >= 33 */) {
 #define TT_LK 16
 #endif
 constexpr int LK = TT_LK;                               // positions per thread and chunk (even)
+// words of the CTA's scratch array: [0, 33) block scans and per-warp run states, then per-warp "last position merged" flags,
+// the carried token / guard of a chunk's last position, and two words for broadcasts
+constexpr int SCR_LASTM = 40, SCR_CARRY_TOK = 72, SCR_CARRY_CL = 73, SCR_FLAG = 74, SCR_VALUE = 75, SCR_WORDS = 80;
 constexpr u32 F20_STALE = 0xFFFFEu;
 TT_HD u64 lp_pack(u32 t, u32 r20, u32 cl20) { return (u64)t | ((u64)r20 << TT_ID_BITS) | ((u64)cl20 << (TT_ID_BITS + 20)); }
 TT_HD u32 lp_tok(u64 v) { return (u32)v & (TT_MAX_INTERNAL - 1); }
@@ -508,7 +511,7 @@ TT_HD u32 lp_cl(u64 v) { return (u32)(v >> (TT_ID_BITS + 20)) & TT_F20; }
 // padshift: 4 for arrays in shared memory (index i lives at i + i / 16, so that the 16-position slices of the
 // threads of a warp fall into different banks), 31 for arrays in global scratch (no padding).
 #define AX(i) ((i) + ((i) >> padshift))
-__device__ __noinline__ u32 cta_merge_rounds(u64* arr, u32* crr, u32 m, const PairTable& tab, u32* s_scr /* >= 48 */, u32 stop_at, bool& finished, u32 padshift,
+__device__ __noinline__ u32 cta_merge_rounds(u64* arr, u32* crr, u32 m, const PairTable& tab, u32* s_scr /* SCR_WORDS */, u32 stop_at, bool& finished, u32 padshift,
                                            u64* stg_a = nullptr, u32* stg_c = nullptr) {
     const int tid = threadIdx.x, T = blockDim.x, lane = tid & 31, wid = tid >> 5, nw = T >> 5;
     const u32 FULL = 0xFFFFFFFFu, inmask = (1u << LK) - 1;
@@ -535,7 +538,7 @@ __device__ __noinline__ u32 cta_merge_rounds(u64* arr, u32* crr, u32 m, const Pa
             for (int k = 0; k < LK + 3; k++) {
                 const u32 i = i0 + k - 1;                   // wraps for position -1 of the piece: not below m
                 v[k] = lp_pack(0, TT_F20, TT_F20); c[k] = TT_F20;
-                if (k == 0 && tid == 0) { if (base) v[k] = lp_pack(s_scr[42], TT_F20, s_scr[43]); }   // overwritten by the chunk before: carried
+                if (k == 0 && tid == 0) { if (base) v[k] = lp_pack(s_scr[SCR_CARRY_TOK], TT_F20, s_scr[SCR_CARRY_CL]); }   // overwritten by the chunk before: carried
                 else if (i < m) { v[k] = arr[AX(i)]; c[k] = crr[AX(i)]; }
             }
             const u32 nval = i0 < m ? min((u32)LK, m - i0) : 0;
@@ -585,11 +588,11 @@ __device__ __noinline__ u32 cta_merge_rounds(u64* arr, u32* crr, u32 m, const Pa
             }
             // was the position before my slice merged with my first one?
             const u32 lastm = __ballot_sync(FULL, (sel >> (LK - 1)) & 1);
-            if (lane == 31) s_scr[33 + wid] = lastm >> 31;
-            if (tid == T - 1) { s_scr[42] = lp_tok(v[LK]); s_scr[43] = lp_cl(v[LK]); }     // position i0 + LK - 1 as it is now
+            if (lane == 31) s_scr[SCR_LASTM + wid] = lastm >> 31;
+            if (tid == T - 1) { s_scr[SCR_CARRY_TOK] = lp_tok(v[LK]); s_scr[SCR_CARRY_CL] = lp_cl(v[LK]); }     // position i0 + LK - 1 as it is now
             __syncthreads();
-            const u32 gone0 = lane ? (lastm >> (lane - 1)) & 1 : (wid ? s_scr[33 + wid - 1] : carry_last);
-            const u32 next_last = s_scr[33 + nw - 1];
+            const u32 gone0 = lane ? (lastm >> (lane - 1)) & 1 : (wid ? s_scr[SCR_LASTM + wid - 1] : carry_last);
+            const u32 next_last = s_scr[SCR_LASTM + nw - 1];
             const u32 gone = ((sel << 1) | gone0) & inmask;
             const u32 valid = nval >= LK ? inmask : ((1u << nval) - 1);
             const u32 surv = valid & ~gone;
@@ -650,9 +653,12 @@ __device__ __noinline__ u32 cta_merge_rounds(u64* arr, u32* crr, u32 m, const Pa
     }
 }
 
-constexpr int LONG_SMEM_TOKENS = 4096;                  // long pieces move into shared memory below this many tokens
+#ifndef TT_LONG_SMEM_TOKENS
+#define TT_LONG_SMEM_TOKENS 14336
+#endif
+constexpr int LONG_SMEM_TOKENS = TT_LONG_SMEM_TOKENS;   // long pieces move into shared memory below this many tokens
 constexpr int LONG_SMEM_SLOTS = LONG_SMEM_TOKENS + LONG_SMEM_TOKENS / 16 + 8;   // with the padding of the shared-memory layout; also holds a chunk's survivors
-static_assert(LONG_SMEM_TOKENS >= 256 * LK, "the survivors of a chunk (threads x LK positions) must fit the shared buffer");
+
 
 // Encodes one piece of n > TT_WARP_PIECE_MAX bytes with the whole CTA.  gbuf: n entries of global scratch; the
 // piece's own n words of the staging array serve as the second global array until the ids are staged there.
@@ -739,16 +745,20 @@ struct PieceParams {
 //       - bulk text: the warp-class pieces stand in one global list (they come in clusters; a list lets every warp
 //         take its share), then warps draw tickets of one tile and settle its short pieces 32 at a time, a thread
 //         each (lane_merge); pieces wait in the lanes across tickets until 32 are together.
-constexpr int MERGE_WARPS = 8;
+#ifndef TT_MERGE_WARPS
+#define TT_MERGE_WARPS 24
+#endif
+constexpr int MERGE_WARPS = TT_MERGE_WARPS;           // one CTA per SM: a long piece gets all its 768 threads and 192 KiB
 constexpr int MERGE_THREADS = MERGE_WARPS * 32;
 constexpr int WARP_SMEM_WORDS = 1024;                 // u64 per warp: two lane-path arrays of 32 x 32 u32, or two copies of four 256-word merge arrays
 static_assert(MERGE_WARPS * WARP_SMEM_WORDS * sizeof(u64) >= LONG_SMEM_SLOTS * (sizeof(u64) + sizeof(u32)), "the CTA's buffer must hold a long piece");
+static_assert(LONG_SMEM_TOKENS >= MERGE_WARPS * 32 * LK, "the survivors of a chunk (threads x LK positions) must fit the shared buffer");
 constexpr size_t MERGE_SMEM_BYTES = (size_t)MERGE_WARPS * WARP_SMEM_WORDS * sizeof(u64);   // dynamic shared memory of k_merge (64 KiB)
 static_assert(WARP_SMEM_WORDS * sizeof(u64) >= 2 * LANE_SLOTS * LANE_MAX * sizeof(u32) && WARP_SMEM_WORDS * sizeof(u64) >= 2 * 4 * TT_WARP_PIECE_MAX * sizeof(u32), "per-warp buffer");
 constexpr int MERGE_SR_MAX_TILES = 2048;              // the per-warp job search covers at most 32 lanes x 64 tiles
 
 #ifndef TT_MERGE_CTAS_PER_SM
-#define TT_MERGE_CTAS_PER_SM 3
+#define TT_MERGE_CTAS_PER_SM 1
 #endif
 constexpr int MERGE_CTAS_PER_SM = TT_MERGE_CTAS_PER_SM;   // resident CTAs per SM (registers and the 64 KiB of shared memory each)
 
@@ -889,9 +899,9 @@ __device__ void cta_long_pieces(const PieceParams& P, const u8* __restrict__ tex
             const uint4 q = s_long[e];
             __syncthreads();
             if (!piece_in_range(P, q.x, q.y, q.z, 3u)) continue;
-            if (tid == 0) { u32 v = 0; sc[47] = piece_settled_without_merge(P, text, q.x, q.y, v) ? 1u : 0u; sc[46] = v; }
+            if (tid == 0) { u32 v = 0; sc[SCR_FLAG] = piece_settled_without_merge(P, text, q.x, q.y, v) ? 1u : 0u; sc[SCR_VALUE] = v; }
             __syncthreads();
-            if (sc[47]) { if (tid == 0) { P.piece_cnt[q.z] = sc[46]; atomicAdd(&P.tile_tok[q.z / TT_TILE_BYTES], 1u); } continue; }
+            if (sc[SCR_FLAG]) { if (tid == 0) { P.piece_cnt[q.z] = sc[SCR_VALUE]; atomicAdd(&P.tile_tok[q.z / TT_TILE_BYTES], 1u); } continue; }
             const u32 m = cta_merge_long(text, q.x, q.y, P.tab, P.ext_id, P.stage, P.pairbuf + q.x, s_buf, sc);
             if (tid == 0) piece_done(P, q.z, m);
         }
@@ -968,7 +978,7 @@ __device__ void merge_bulk_lists(const PieceParams& P, const u8* __restrict__ te
 __global__ void __launch_bounds__(MERGE_THREADS, MERGE_CTAS_PER_SM)
 k_merge_bulk(const PieceParams P) {
     extern __shared__ __align__(16) u64 s_buf[];              // MERGE_SMEM_BYTES
-    __shared__ u32 sc[48];
+    __shared__ u32 sc[SCR_WORDS];
     __shared__ u32 s_warps_done;
     cudaTriggerProgrammaticLaunchCompletion();               // k_scatter may be placed; it waits for this grid's memory itself
     grid_prefetch_l2(P.tab.slots, ((size_t)P.tab.mask + 1) * 2 * sizeof(uint4));
@@ -983,7 +993,7 @@ k_merge_bulk(const PieceParams P) {
 __global__ void __launch_bounds__(MERGE_THREADS, MERGE_CTAS_PER_SM)
 k_merge(const PieceParams P) {
     extern __shared__ __align__(16) u64 s_buf[];              // MERGE_SMEM_BYTES
-    __shared__ u32 sc[48];
+    __shared__ u32 sc[SCR_WORDS];
     __shared__ uint4 s_long[TT_TILE_LONGCAP + 2];             // the long pieces of one tile
     __shared__ u32 s_nlong;
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
@@ -1215,7 +1225,7 @@ struct ScatterParams {
 constexpr int SCATTER_STAGE_IDS = 2048;                   // ids of one work item that are put together in shared memory
 __global__ void __launch_bounds__(BPE_THREADS)
 k_scatter(const ScatterParams P) {
-    __shared__ u32 sc[48];
+    __shared__ u32 sc[SCR_WORDS];
     __shared__ u32 s_big[TT_TILE_BYTES / 8][3];
     __shared__ u32 s_nbig;
     __shared__ u32 s_np[BPE_THREADS];                         // pieces of the next tiles of this CTA's range

@@ -512,7 +512,30 @@ def main():
             assert int(vbufs["status"].item()) == 0
             variants[name] = {"cold_p50_ms": round(pct(ts, 0.5), 4), "merges": int(vm.shape[0]), "tokens": int(vbufs["count"].item())}
             del vv, vbufs
-        variants["what"] = "tt_encode of one 1,000,000-char transcript under the other pattern ids (o200k-style with its own 199,744-merge vocabulary)"
+        # pattern 1 where its sparse sequential path decides most of the text: glued words with a combining mark every
+        # second or third letter, and Thai-like text (caseless letters with marks, a blank only between phrases)
+        vm, vb = wl.load_vocab(wl.CONFIGS["C4"])
+        vv = tt.Vocab(vm, vb, tt.TT_PATTERN_O200K)
+        for name, kind in (("o200k_marks", wl.KIND_MARKS), ("o200k_thai_like", wl.KIND_THAI)):
+            mtext = torch.from_numpy(wl.generate(kind, 99, cfg.n_chars)).cuda()
+            vbufs = vv.alloc(mtext.numel())
+            ts, kt = [], {}
+            for k in range(3 + 8):
+                flush_l2(); torch.cuda.synchronize()
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(stream); vv.encode(mtext, vbufs); b.record(stream)
+                torch.cuda.synchronize()
+                if k >= 3:
+                    ts.append(a.elapsed_time(b))
+            for kn, ms in vv.encode_timed(mtext, vbufs).items():
+                kt[kn] = round(ms, 4)
+            assert int(vbufs["status"].item()) == 0
+            variants[name] = {"cold_p50_ms": round(pct(ts, 0.5), 4), "bytes": int(mtext.numel()), "tokens": int(vbufs["count"].item()),
+                              "kernel_ms": kt}
+            del vbufs, mtext
+        del vv
+        variants["what"] = ("tt_encode of one 1,000,000-char text under the other pattern ids (o200k-style with its own 199,744-merge "
+                            "vocabulary): a transcript, mark-dense text without blanks, Thai-like text")
 
     # ---- the other single-request configs: C1 (4,000 chars), C2 (100,000 chars, 5 % non-ASCII), C4 (3,000,000 chars with
     # adversarial runs, o200k-style pattern, 199,744 merges) ----

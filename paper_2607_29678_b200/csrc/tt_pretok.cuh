@@ -15,7 +15,7 @@
 enum { F_LEAD = 0, F_OTH, F_MARK, F_SPC, F_NUM, F_LOW, F_UPP, F_CLESS, F_NL, F_SP, F_AP, F_SL, F_DOC,
        F_SURE, F_HARD,     // pattern 1: sure piece starts / unresolved constructs, filled after classification
        F_COUNT };
-constexpr int TT_LOW_HALO = 6;                          // chunks kept below the tile (look-back context, 96 bytes)
+constexpr int TT_LOW_HALO = 14;                         // chunks kept below the tile (look-back context, 224 bytes)
 constexpr int TT_SLOTS = TT_TILE_CHUNKS + TT_LOW_HALO + 1;   // low halo, tile, one high halo chunk
 
 enum { NEED_N = 1, NEED_A = 2, NEED_F = 4, NEED_S = 8, NEED_H = 16, NEED_C = 32 };

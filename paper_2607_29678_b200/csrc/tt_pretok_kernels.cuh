@@ -175,6 +175,7 @@ __device__ long long coop_back_event(const PretokParams& P, const ClassTables& T
             p.m = tt_classify_chunk(P.base, chunk - 1, P.nchunks, P.lo, P.hi, T); p.doc = doc_bits(P, chunk - 1);
             c.m = tt_classify_chunk(P.base, chunk, P.nchunks, P.lo, P.hi, T);     c.doc = doc_bits(P, chunk);
             n.m = tt_classify_chunk(P.base, chunk + 1, P.nchunks, P.lo, P.hi, T); n.doc = doc_bits(P, chunk + 1);
+            tt_marks_inside_words_cm(p, c, n);
             u32 sure, hard;
             tt_sure_hard_cm(p, c, n, sure, hard);
             u32 live = 0xFFFFu;
@@ -290,6 +291,15 @@ k_pretok(const PretokParams P, const FrontParams F) {
             store_slot(sm, s, tt_classify_chunk(P.base, chunk, P.nchunks, P.lo, P.hi, T), doc_bits(P, chunk));
         }
         __syncthreads();
+        if (P.pattern == 1) {                                          // marks inside words count as caseless letters from here on
+            const u32 in_own = tt_marks_inside_words(sm, tid + TT_LOW_HALO);
+            const int hs = tid < TT_LOW_HALO ? tid : TT_SLOTS - 1;
+            const u32 in_halo = tid < TT_LOW_HALO + 1 ? tt_marks_inside_words(sm, hs) : 0u;
+            __syncthreads();
+            if (in_own) { sm[F_MARK][tid + TT_LOW_HALO] &= (u16)~in_own; sm[F_CLESS][tid + TT_LOW_HALO] |= (u16)in_own; }
+            if (in_halo) { sm[F_MARK][hs] &= (u16)~in_halo; sm[F_CLESS][hs] |= (u16)in_halo; }
+            __syncthreads();
+        }
         if (P.pattern == 1) {                                          // sure starts / unresolved constructs per slot
             u32 su, ha;
             const long long gs0 = (c_first - TT_LOW_HALO) * TT_CHUNK;       // byte 0 of slot 0

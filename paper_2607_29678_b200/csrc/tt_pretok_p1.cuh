@@ -172,6 +172,28 @@ TT_HD u32 tt_seq_starts_p1(const SeqCtx& C, long long from, long long g0, long l
     return bits;
 }
 
+// ---- marks inside words -------------------------------------------------------------------------------
+// In pattern 1 a mark belongs to both word classes, exactly like a caseless letter, and a word match that has taken a
+// letter always goes on over a mark that follows it.  So a run of marks right behind a letter lies inside that
+// letter's word and behaves as caseless letters do; only a mark at the head of a run of word characters (after
+// whitespace, punctuation, a digit, the start of the text) can also be punctuation and stays an unresolved construct.
+// One exception: a letter that may end a contraction suffix (an apostrophe one or two bytes before it) ends its piece,
+// so marks behind it are left unresolved as well.  Returns the bits of slot s (s >= 0) whose marks lie inside a word;
+// the masks of the two slots before it give the look-back (a run of marks that reaches back beyond them stays
+// unresolved).
+TT_HD u32 tt_marks_inside_words(const u16 (*sm)[TT_SLOTS], int s) {
+    const u32 own = sm[F_MARK][s];
+    if (own == 0) return 0;
+#define W3(f) ((s >= 2 ? (u64)sm[f][s - 2] : 0ull) | (s >= 1 ? (u64)sm[f][s - 1] << 16 : 0ull) | ((u64)sm[f][s] << 32))
+    const u64 D = W3(F_DOC), Mk = W3(F_MARK) & ~D;                 // a mark that starts a document heads a run
+    const u64 Lr = W3(F_LOW) | W3(F_UPP) | W3(F_CLESS), AP = W3(F_AP);
+#undef W3
+    const u64 starts = Mk & ~(Mk << 1);
+    const u64 good = starts & (Lr << 1) & ~D & ~((AP << 2) | (AP << 3));
+    const u64 inside = Mk & ~(Mk + good);                          // the carry runs through every run that starts well
+    return (u32)(inside >> 32) & 0xFFFFu;
+}
+
 // ---- masks of sure piece starts and of unresolved constructs for one chunk ---------------------------
 struct ChunkDoc { ChunkMasks m; u32 doc; };
 
@@ -182,6 +204,21 @@ TT_HD ChunkDoc tt_load_slot(const u16 (*sm)[TT_SLOTS], int s) {
     c.m.ap = sm[F_AP][s]; c.m.sl = sm[F_SL][s]; c.m.bad = 0; c.doc = sm[F_DOC][s];
     return c;
 }
+// The same for three neighbouring chunks held in registers (the cooperative walks over the text): marks inside words
+// become caseless letters in all three, as far as the 48 bytes show it.
+TT_HD void tt_marks_inside_words_cm(ChunkDoc& p, ChunkDoc& c, ChunkDoc& n) {
+    if ((p.m.mark | c.m.mark | n.m.mark) == 0) return;
+#define W3(x) ((u64)p.x | ((u64)c.x << 16) | ((u64)n.x << 32))
+    const u64 D = W3(doc), Mk = W3(m.mark) & ~D;
+    const u64 Lr = W3(m.low) | W3(m.upp) | W3(m.cless), AP = W3(m.ap);
+#undef W3
+    const u64 starts = Mk & ~(Mk << 1);
+    const u64 good = starts & (Lr << 1) & ~D & ~((AP << 2) | (AP << 3));
+    const u64 inside = Mk & ~(Mk + good);
+    const u16 ip = (u16)inside, ic = (u16)(inside >> 16), in = (u16)(inside >> 32);
+    p.m.mark &= (u16)~ip; p.m.cless |= ip; c.m.mark &= (u16)~ic; c.m.cless |= ic; n.m.mark &= (u16)~in; n.m.cless |= in;
+}
+
 // p = previous chunk, c = the chunk, n = next chunk
 // upcl: the unresolved constructs of the second kind (upper-case letter after a caseless letter), a subset of hard
 // apch: the unresolved constructs of the third kind (apostrophe between letters with another apostrophe two or three

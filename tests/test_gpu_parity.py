@@ -431,6 +431,37 @@ def test_cjk_latin_mixtures_in_long_documents():
     assert status == 0 and same(ioff, woff) and same(ids, want)
 
 
+@pytest.mark.parametrize("kind", ["marks", "thai"])
+@pytest.mark.parametrize("pattern", [0, 1])
+def test_mark_dense_text_without_blanks(kind, pattern):
+    """Text whose words are glued and carry a combining mark every second or third letter, and Thai-like text
+    (caseless consonants with vowel signs and tone marks, a blank only between phrases): under pattern 1 nearly every
+    piece holds unresolved constructs, so the sparse sequential path decides most of the text.  Pieces and ids
+    against the oracle: one 1,000,000-char text, a misaligned copy of a part of it, and a batch of documents."""
+    name = "C2" if pattern == 0 else "C4"
+    k = wl.KIND_MARKS if kind == "marks" else wl.KIND_THAI
+    text = wl.generate(k, 11, 1_000_000)
+    got, status = gpu_pretok(gpu_vocab(name), text)
+    assert status == 0 and same(got, _expect_pieces(text, pattern))
+    ids, status = gpu_encode(gpu_vocab(name), text)
+    want, _ = cpu_vocab(name).encode(text, pattern, nthreads=16)
+    assert status == 0 and same(ids, want)
+    part = text[:200_000]
+    while (part[-1] & 0xC0) == 0x80 or part[-1] >= 0xC0:            # end on a character boundary
+        part = part[:-1]
+    ids, status = gpu_encode(gpu_vocab(name), part, offset=9)
+    want, _ = cpu_vocab(name).encode(part, pattern, nthreads=8)
+    assert status == 0 and same(ids, want)
+    docs = [wl.generate(k, 100 + d, 200 + 97 * d).tobytes() for d in range(60)]
+    _batch_pieces_check(name, pattern, docs)
+    btext = np.frombuffer(b"".join(docs), dtype=np.uint8)
+    off = np.zeros(len(docs) + 1, dtype=np.int64)
+    off[1:] = np.cumsum([len(d) for d in docs])
+    ids, ioff, status = gpu_encode_batch(gpu_vocab(name), btext, off)
+    want, woff = cpu_vocab(name).encode_batch(btext, off, pattern, nthreads=8)
+    assert status == 0 and same(ioff, woff) and same(ids, want)
+
+
 def test_bulk_text_of_pieces_outside_the_vocabulary():
     """Megabytes of random words (Latin and CJK, 2..80 bytes) that are no vocabulary entries: every CTA
     handles many tiles and its piece queues fill and empty many times (thread-per-piece and warp-per-piece

@@ -23,7 +23,7 @@ _lib = None
 
 BASE_SEED = 0x260729678
 
-KIND_MIX, KIND_MIX_UNI, KIND_TRANSCRIPT, KIND_TRANSCRIPT_ADV = 0, 1, 2, 3
+KIND_MIX, KIND_MIX_UNI, KIND_TRANSCRIPT, KIND_TRANSCRIPT_ADV, KIND_MARKS, KIND_THAI = 0, 1, 2, 3, 4, 5
 
 
 def build(force: bool = False) -> str:

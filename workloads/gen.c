@@ -420,6 +420,43 @@ static void emit_adversarial(ctx_t *c) {
     if (t == 0) put_nl(c); else if (t == 1) put_c(c, ' '); else if (t == 2) put_ident(c, 1);
 }
 
+/* ------------------------------------------------- mark-dense, blank-free text */
+/* Latin letters with a combining mark after every second or third one, no blanks: words are glued, a comma or a full
+ * stop comes every 20-80 characters and a line feed every few hundred. */
+static void emit_marks(ctx_t *c, size_t n_chars) {
+    static const uint32_t MARK[] = {0x301, 0x300, 0x308, 0x323, 0x302, 0x303};
+    size_t next_punct = 20 + rng_below(&c->rng, 60), next_nl = 200 + rng_below(&c->rng, 300), since_mark = 0;
+    while (c->chars < n_chars) {
+        int upper = rng_chance(&c->rng, 0.06);
+        put_c(c, (char)((upper ? 'A' : 'a') + rng_below(&c->rng, 26)));
+        if (++since_mark >= 2 + rng_below(&c->rng, 2)) { put_cp(c, MARK[rng_below(&c->rng, 6)]); since_mark = 0; }
+        if (rng_chance(&c->rng, 0.004)) { put_c(c, '\''); put_c(c, "stmd"[rng_below(&c->rng, 4)]); }
+        if (c->chars >= next_punct) { put_c(c, rng_chance(&c->rng, 0.7) ? ',' : '.'); next_punct = c->chars + 20 + rng_below(&c->rng, 60); }
+        if (c->chars >= next_nl) { put_c(c, '\n'); next_nl = c->chars + 200 + rng_below(&c->rng, 300); }
+    }
+}
+/* Thai-like text: consonants (caseless letters, three bytes each) carrying vowel signs and tone marks (marks) above and
+ * below, words glued into phrases of 5-40 characters that a single blank separates, now and then digits, a Latin
+ * word or punctuation. */
+static void emit_thai_like(ctx_t *c, size_t n_chars) {
+    static const uint32_t SIGN[] = {0xE31, 0xE34, 0xE35, 0xE36, 0xE37, 0xE38, 0xE39, 0xE47, 0xE48, 0xE49, 0xE4A, 0xE4B, 0xE4C};
+    lex_init();
+    while (c->chars < n_chars) {
+        size_t phrase = 5 + rng_below(&c->rng, 36);
+        for (size_t k = 0; k < phrase; k++) {
+            put_cp(c, 0xE01 + rng_below(&c->rng, 46));                       /* consonant */
+            if (rng_chance(&c->rng, 0.45)) put_cp(c, SIGN[rng_below(&c->rng, 13)]);
+            if (rng_chance(&c->rng, 0.12)) put_cp(c, 0xE30 + 2 * rng_below(&c->rng, 2));   /* a spacing vowel (letter) */
+        }
+        uint32_t k = rng_below(&c->rng, 100);
+        if (k < 70) put_c(c, ' ');
+        else if (k < 78) { put_c(c, ' '); put_int(c, log_uniform_int(&c->rng, 1e7)); put_c(c, ' '); }
+        else if (k < 86) { put_c(c, ' '); put_word(c, zipf_word(&c->rng), rng_below(&c->rng, 3)); put_c(c, ' '); }
+        else if (k < 94) put_s(c, rng_chance(&c->rng, 0.5) ? " (" : ") ");
+        else put_nl(c);
+    }
+}
+
 /* ------------------------------------------------------------- top level */
 static void emit_mix(ctx_t *c, size_t n_chars) {
     while (c->chars < n_chars) {
@@ -467,6 +504,8 @@ size_t wl_generate(int kind, uint64_t seed, size_t n_chars, uint8_t *out, size_t
     if (kind == 1) { c.uni_rate = 0.17; c.crlf_rate = 0.10; }
     if (kind == 3) { c.uni_rate = 0.02; c.cjk_rate = 0.85; }
     if (kind == 0 || kind == 1) emit_mix(&c, n_chars);
+    else if (kind == 4) emit_marks(&c, n_chars);
+    else if (kind == 5) emit_thai_like(&c, n_chars);
     else emit_transcript(&c, n_chars, kind == 3);
     size_t nbytes = truncate_to_chars(c.p, c.len, n_chars);
     if (nbytes > cap) { free(c.p); return 0; }

@@ -889,7 +889,8 @@ struct tt_session {
     size_t cap = 0;                       // bytes of text the session can hold
     size_t len = 0;                       // bytes stored
     uint32_t window_chars = 512;
-    std::vector<u8> h_text;               // host mirror of the stored text (window starts are found here)
+    std::vector<u8> h_tail;               // host copy of the END of the stored text only: the window starts are found here
+    size_t tail_base = 0;                 // (text offset of h_tail[0]; enough for the widest window, see session_keep_tail)
     u8* d_text = nullptr;
     int32_t *d_ids = nullptr, *d_off = nullptr;                 // cached records; d_off[ntok] = len
     int32_t *d_fids = nullptr, *d_foff = nullptr, *d_fchar = nullptr;   // fresh records / scratch of the span export
@@ -958,23 +959,36 @@ static int session_tokenize(tt_session* s, size_t from, size_t new_len, cudaStre
     return tt_spans(s->v, ids, (const int64_t*)count, s->cap, n, st, off, s->d_fchar, s->d_sstatus, s->d_sws, s->sws_bytes);
 }
 
+// The host keeps the last bytes of the stored text, as many as the widest window of the protocol can span (five
+// doublings of the window, four bytes a character): an append costs a copy of that tail at most, whatever the
+// session holds.
+static void session_keep_tail(tt_session* s, const uint8_t* text, size_t len) {
+    const size_t keep = (size_t)s->window_chars * 32 * 4 + 64;
+    s->h_tail.insert(s->h_tail.end(), text, text + len);
+    if (s->h_tail.size() > 2 * keep) {
+        const size_t drop = s->h_tail.size() - keep;
+        s->h_tail.erase(s->h_tail.begin(), s->h_tail.begin() + (ptrdiff_t)drop);
+        s->tail_base += drop;
+    }
+}
+
 extern "C" int tt_session_append(tt_session* s, const uint8_t* text, size_t len, void* stream, tt_append_info* info) {
     if (!s || (len && !text)) return TT_ERR_ARG;
     if (len > s->cap - s->len) return TT_ERR_TOO_LARGE;
     cudaStream_t st = (cudaStream_t)stream;
     tt_append_info local; memset(&local, 0, sizeof(local));
     const size_t old_len = s->len, new_len = old_len + len;
-    s->h_text.insert(s->h_text.end(), text, text + len);
     // (an error return waits for the stream first: the copy from the caller's buffer may still be in flight)
-    auto fail = [&](int code) { cudaStreamSynchronize(st); cudaGetLastError(); s->h_text.resize(old_len); if (info) { local.status = code; *info = local; } return code; };
+    auto fail = [&](int code) { cudaStreamSynchronize(st); cudaGetLastError(); if (info) { local.status = code; *info = local; } return code; };
     if (len) { if (cudaMemcpyAsync(s->d_text + old_len, text, len, cudaMemcpyHostToDevice, st) != cudaSuccess) { cudaGetLastError(); return fail(TT_ERR_CUDA); } }
     if (new_len == 0) { if (info) *info = local; return TT_OK; }
-    const u8* ht = s->h_text.data();
+    const u8* ht = s->h_tail.data() - s->tail_base;          // ht[i] = byte i of the stored text, for i >= tail_base
     uint64_t w = s->window_chars;
     for (int attempt = 0; attempt <= 5 && old_len > 0; attempt++, w *= 2) {
         // byte offset of the character that lies w characters before the end of the stored text
         size_t ws = old_len; uint64_t left = w;
-        while (ws > 0 && left > 0) { ws--; while (ws > 0 && (ht[ws] & 0xC0) == 0x80) ws--; left--; }
+        while (ws > s->tail_base && left > 0) { ws--; while (ws > s->tail_base && (ht[ws] & 0xC0) == 0x80) ws--; left--; }
+        if (left > 0 || ws == s->tail_base) ws = 0;           // the window reaches the start of the text (or beyond what the host kept: more work, same ids)
         local.attempts = attempt + 1;
         if (ws == 0) break;                                   // the window is the whole text
         int rc = session_tokenize(s, ws, new_len, st, s->d_fids, s->d_foff, s->d_fcount);
@@ -995,7 +1009,7 @@ extern "C" int tt_session_append(tt_session* s, const uint8_t* text, size_t len,
         const RepairDecision d = s->h->dec;
         if (d.status != TT_OK) return fail(d.status);          // e.g. the appended text is not valid UTF-8: nothing changed
         if (d.accept) {
-            s->len = new_len;
+            s->len = new_len; session_keep_tail(s, text, len);
             local.window_chars = (int64_t)w; local.window_start = (int64_t)ws; local.run_tokens = d.j1 - d.j0;
             local.splice_byte = d.splice_byte; local.n_tokens = d.new_ntok; local.status = TT_OK;
             if (info) *info = local;
@@ -1018,7 +1032,7 @@ extern "C" int tt_session_append(tt_session* s, const uint8_t* text, size_t len,
         cudaMemcpyAsync(s->d_off, s->d_foff, (nt + 1) * 4, cudaMemcpyDeviceToDevice, st) != cudaSuccess ||
         cudaMemcpyAsync(s->d_ntok, s->d_fcount, 8, cudaMemcpyDeviceToDevice, st) != cudaSuccess ||
         cudaStreamSynchronize(st) != cudaSuccess) { cudaGetLastError(); return fail(TT_ERR_CUDA); }
-    s->len = new_len;
+    s->len = new_len; session_keep_tail(s, text, len);
     local.window_chars = 0; local.window_start = 0; local.run_tokens = 0; local.splice_byte = 0;
     local.n_tokens = (int64_t)nt; local.status = TT_OK;
     if (info) *info = local;

@@ -496,7 +496,7 @@ __device__ __forceinline__ u32 cta_min_u32(u32 v, u32* scratch /* >= 33 */) {
 // anything is written, and writes never pass the read front).  Ranks next to a merge are marked stale and
 // probed again in a second sweep, which also yields the next round's minimum.
 #ifndef TT_LK
-#define TT_LK 16
+#define TT_LK 6        // measured with 768 threads: 64 KB of random letters 94 ms at 16, 59 at 8, 45 at 6, 51 at 4, 59 at 2
 #endif
 constexpr int LK = TT_LK;                               // positions per thread and chunk (even)
 // words of the CTA's scratch array: [0, 33) block scans and per-warp run states, then per-warp "last position merged" flags,
@@ -508,8 +508,8 @@ TT_HD u32 lp_tok(u64 v) { return (u32)v & (TT_MAX_INTERNAL - 1); }
 TT_HD u32 lp_rank(u64 v) { return (u32)(v >> TT_ID_BITS) & TT_F20; }
 TT_HD u32 lp_cl(u64 v) { return (u32)(v >> (TT_ID_BITS + 20)) & TT_F20; }
 
-// padshift: 4 for arrays in shared memory (index i lives at i + i / 16, so that the 16-position slices of the
-// threads of a warp fall into different banks), 31 for arrays in global scratch (no padding).
+// padshift: 4 for arrays in shared memory (index i lives at i + i / 16: the slices of LK consecutive positions that the
+// threads of a warp read then spread over more banks), 31 for arrays in global scratch (no padding).
 #define AX(i) ((i) + ((i) >> padshift))
 __device__ __noinline__ u32 cta_merge_rounds(u64* arr, u32* crr, u32 m, const PairTable& tab, u32* s_scr /* SCR_WORDS */, u32 stop_at, bool& finished, u32 padshift,
                                            u64* stg_a = nullptr, u32* stg_c = nullptr) {

@@ -365,6 +365,16 @@ TT_HD u32 tt_walk_back_dirty(const u16 (*sm)[TT_SLOTS], int s, bool& open) {
     open = true;
     return 0;
 }
+// Do the slots 1..s hold neither letters nor marks?  Then no unresolved construct that lies before them can reach beyond
+// them: whitespace, punctuation and digits are split by rules that look at most a few bytes back (plus the run
+// aggregates that have carries of their own), so what an earlier word turned out to be is forgotten after the first
+// such character.  (Asked only by chunks that found no event in the whole look-back window: long runs of blanks or
+// of one punctuation character, where the alternative is a walk back to the run's start from every tile in it.)
+TT_HD bool tt_window_plain(const u16 (*sm)[TT_SLOTS], int s) {
+    u32 wordy = 0;
+    for (; s >= 1; s--) wordy |= (u32)sm[F_LOW][s] | sm[F_UPP][s] | sm[F_CLESS][s] | sm[F_MARK][s];
+    return wordy == 0;
+}
 // Walks down from slot s: position (slot * 16 + bit) of the nearest sure start, or -1 when open.
 TT_HD int tt_walk_back_sure(const u16 (*sm)[TT_SLOTS], int s) {
     for (; s >= 1; s--) {
@@ -534,7 +544,7 @@ TT_HD u32 tt_eval_chunk_p1(const u16 (*sm)[TT_SLOTS], int slot, const SeqCtx& C,
         carry = tt_walk_back_dirty(sm, slot - 2, open);
         // (nothing lies before the text: its first tile needs no look beyond the window)
         const bool at_text_start = C.lo >= g0 - (long long)(slot - 1) * TT_CHUNK;
-        if (open && !at_text_start) { if (have_tc) carry = tc.dirty_before; else need |= NEED_H; }
+        if (open && !at_text_start && !tt_window_plain(sm, slot - 2)) { if (have_tc) carry = tc.dirty_before; else need |= NEED_H; }
         const u64 sure2 = sure & ~0xFFFFull;
         u64 F = (hard & ~0xFFFFull) | (((u64)carry << 16) & ~sure2);
         u64 R = ~sure2;

@@ -462,6 +462,36 @@ def test_mark_dense_text_without_blanks(kind, pattern):
     assert status == 0 and same(ioff, woff) and same(ids, want)
 
 
+@pytest.mark.parametrize("pattern", [0, 1])
+def test_unresolved_constructs_before_long_plain_runs(pattern):
+    """A mark, a caseless letter before an upper-case one, or a chain of contraction suffixes, followed at once (or after
+    a few characters) by hundreds to thousands of bytes of one plain class (blanks, tabs, line feeds, one punctuation
+    character, digits, slashes, apostrophes) and then by a tail that the rules have to place: whatever the construct
+    turns out to be must not reach the pieces far inside or behind the run.  Piece boundaries and ids per document."""
+    name = "C2" if pattern == 0 else "C4"
+    rng = random.Random(5150 + pattern)
+    heads = ["x\u0301", "!\u0301", "\u0301", "中A", "x's's's", "a'", "É\u0301'", "1\u0301", " \u0301", "word", "'s", "A\u0301B"]
+    mids = ["", " ", "!", "\n", "a", "'", "/"]
+    runs = [" ", "\t", " \t", "\n", "\r\n", "=", "*", "'", "/", "9", "!\n", " \n", "\u3000"]
+    tails = ["abc", "A", "\u0301x", "\n", "'s", " x", "  x", "1", "!", "/a", "", "aB", "中"]
+    docs = []
+    for _ in range(700):
+        n = rng.choice([230, 260, 500, 2049, 2300, 4500, 9000])
+        run = rng.choice(runs)
+        docs.append((rng.choice(["", "lead in. ", "xy\n"]) + rng.choice(heads) + rng.choice(mids) + run * (n // len(run)) + rng.choice(tails)
+                     + rng.choice(["", " end", "\n"])).encode("utf-8"))
+    _batch_pieces_check(name, pattern, docs)
+    text = np.frombuffer(b"".join(docs), dtype=np.uint8)
+    off = np.zeros(len(docs) + 1, dtype=np.int64)
+    off[1:] = np.cumsum([len(d) for d in docs])
+    ids, ioff, status = gpu_encode_batch(gpu_vocab(name), text, off)
+    want, woff = cpu_vocab(name).encode_batch(text, off, pattern, nthreads=8)
+    assert status == 0 and same(ioff, woff) and same(ids, want)
+    # and as one text: the documents glued together, so that a run can follow whatever the document before left
+    got, status = gpu_pretok(gpu_vocab(name), text)
+    assert status == 0 and same(got, _expect_pieces(text, pattern))
+
+
 def test_bulk_text_of_pieces_outside_the_vocabulary():
     """Megabytes of random words (Latin and CJK, 2..80 bytes) that are no vocabulary entries: every CTA
     handles many tiles and its piece queues fill and empty many times (thread-per-piece and warp-per-piece

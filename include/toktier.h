@@ -113,8 +113,8 @@ size_t tt_workspace_bytes(const tt_vocab* v, size_t max_len, size_t max_docs);
  *   status_out  DEVICE int32: TT_OK, TT_ERR_INVALID_UTF8, TT_ERR_CAPACITY or TT_ERR_INTERNAL_TIMEOUT.
  *   workspace   DEVICE scratch of at least tt_workspace_bytes(v, len, 1) bytes.
  * Asynchronous on `stream`.  len == 0 yields count 0, status TT_OK.
- * The call enqueues four kernels (inside a stream capture a 128-byte memset in front of them) and may be captured
- * into a CUDA graph by the caller (paper Sec. 4.2: one submission per request for a caller that reuses its buffers).
+ * The call enqueues three kernels (for text of more than 4 MB four, behind a 128-byte memset; inside a stream
+ * capture the memset is always there) and may be captured into a CUDA graph by the caller (paper Sec. 4.2: one submission per request for a caller that reuses its buffers).
  */
 int tt_encode(const tt_vocab* v, const uint8_t* text, size_t len, void* stream,
               int32_t* ids_out, size_t ids_cap, int64_t* count_out, int32_t* status_out,

@@ -455,6 +455,18 @@ extern "C" size_t tt_workspace_bytes(const tt_vocab* v, size_t max_len, size_t m
 
 #define CK(x) do { if ((x) != cudaSuccess) { cudaGetLastError(); return TT_ERR_CUDA; } } while (0)
 
+// One instance of the first kernel per pattern (the pattern's rules are compiled in), chosen here.
+template <bool FUSED, int MINB>
+static void launch_pretok(int grid, cudaStream_t st, const PretokParams& P, const FrontParams& F) {
+    const size_t smem = sizeof(u16) * F_COUNT * TT_SLOTS;
+    switch (P.pattern) {
+    case TT_PATTERN_O200K:     k_pretok<FUSED, MINB, TT_PATTERN_O200K><<<grid, TT_TILE_CHUNKS, smem, st>>>(P, F); break;
+    case TT_PATTERN_CL100K_N1: k_pretok<FUSED, MINB, TT_PATTERN_CL100K_N1><<<grid, TT_TILE_CHUNKS, smem, st>>>(P, F); break;
+    case TT_PATTERN_CUTS:      if constexpr (!FUSED) k_pretok<false, MINB, TT_PATTERN_CUTS><<<grid, TT_TILE_CHUNKS, smem, st>>>(P, F); break;
+    default:                   k_pretok<FUSED, MINB, TT_PATTERN_CL100K><<<grid, TT_TILE_CHUNKS, smem, st>>>(P, F); break;
+    }
+}
+
 // Enqueues K1+K2 (and K3 when piece_off_dst is given: only tt_pretokenize materialises the offsets;
 // the encode chain derives them per tile from the start flags).
 static int run_pretok(const tt_vocab* v, const uint8_t* text, size_t len, const int64_t* doc_off, size_t n_docs,
@@ -490,9 +502,8 @@ static int run_pretok(const tt_vocab* v, const uint8_t* text, size_t len, const 
         k_lit_select<<<lgrid, 256, 0, st>>>(L);
         P.docmask = w.docmask; P.litstart = w.litstart; P.litin = w.litin;
     }
-    const size_t smem = sizeof(u16) * F_COUNT * TT_SLOTS;
     const bool bulk = P.ntiles > MERGE_SR_MAX_TILES;
-    const int per_sm = bulk ? PRETOK_CTAS_BULK : PRETOK_CTAS_REQUEST;
+    const int per_sm = bulk && fused ? PRETOK_CTAS_BULK : PRETOK_CTAS_REQUEST;
     const int grid = P.ntiles < v->sm_count * per_sm ? P.ntiles : v->sm_count * per_sm;
     if (v->pattern == TT_PATTERN_SPLIT3) {
         // stages A and B: span starts into cutmask (with the caller's document starts); stage C: pattern 0 with
@@ -500,8 +511,7 @@ static int run_pretok(const tt_vocab* v, const uint8_t* text, size_t len, const 
         PretokParams C1 = P;
         C1.pattern = TT_PATTERN_CUTS; C1.startmask = reinterpret_cast<u16*>(w.cutmask);
         C1.want_prefix = 0; C1.litstart = nullptr; C1.litin = nullptr;
-        if (bulk) k_pretok<false, PRETOK_CTAS_BULK><<<grid, TT_TILE_CHUNKS, smem, st>>>(C1, FrontParams{});
-        else k_pretok<false, PRETOK_CTAS_REQUEST><<<grid, TT_TILE_CHUNKS, smem, st>>>(C1, FrontParams{});
+        launch_pretok<false, PRETOK_CTAS_REQUEST>(grid, st, C1, FrontParams{});
         P.pattern = TT_PATTERN_CL100K; P.docmask = w.cutmask;
     }
     if (fused) {
@@ -509,10 +519,9 @@ static int run_pretok(const tt_vocab* v, const uint8_t* text, size_t len, const 
         F.tile_last = w.tile_last; F.tile_tok = w.tile_tok; F.tile_q = w.tile_q; F.tile_long = w.tile_long; F.piece_off16 = w.piece_off16;
         F.piece_cnt = w.piece_cnt; F.q = w.q; F.toktab = v->toktab; F.longtab = v->longtab; F.ext_id = v->d_ext_id;
         F.wq = P.ntiles > MERGE_SR_MAX_TILES ? w.wq : nullptr;
-        if (bulk) k_pretok<true, PRETOK_CTAS_BULK><<<grid, TT_TILE_CHUNKS, smem, st>>>(P, F);
-        else k_pretok<true, PRETOK_CTAS_REQUEST><<<grid, TT_TILE_CHUNKS, smem, st>>>(P, F);
-    } else if (bulk) k_pretok<false, PRETOK_CTAS_BULK><<<grid, TT_TILE_CHUNKS, smem, st>>>(P, FrontParams{});
-    else k_pretok<false, PRETOK_CTAS_REQUEST><<<grid, TT_TILE_CHUNKS, smem, st>>>(P, FrontParams{});
+        if (bulk) launch_pretok<true, PRETOK_CTAS_BULK>(grid, st, P, F);
+        else launch_pretok<true, PRETOK_CTAS_REQUEST>(grid, st, P, F);
+    } else launch_pretok<false, PRETOK_CTAS_REQUEST>(grid, st, P, FrontParams{});
     if (piece_off_dst)
         k_compact<<<grid, TT_TILE_CHUNKS, 0, st>>>(w.startmask, w.tile_cnt, P.nchunks, P.ntiles, shift, (long long)len,
                                                    piece_off_dst, w.hdr, P.epoch);

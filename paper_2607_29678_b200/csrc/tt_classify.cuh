@@ -95,81 +95,95 @@ TT_HD ChunkMasks tt_classify_ascii16(u32 w0, u32 w1, u32 w2, u32 w3) {
     return m;
 }
 
-// words w[0] = the 4 bytes before the chunk, w[1..4] = the chunk, w[5] = the 4 bytes after it
-#define TT_BYTE(w, j) (((w)[((j) + 4) >> 2] >> (8 * (((j) + 4) & 3))) & 0xFFu)
+// Top bits of the four bytes of a word as a 4-bit number (byte k -> bit k): the bits are first brought to positions
+// 0, 8, 16, 24; the multiplication then adds them up at 24..27 (the partial products fall on distinct bits).
+TT_HD u32 tt_movemask4(u32 x) { return ((((x >> 7) & 0x01010101u) * 0x01020408u) >> 24) & 0xFu; }
 
-// g0 = global index (in the aligned frame) of the chunk's first byte; bytes outside [lo, hi) do
-// not exist.  `w` as above (missing neighbours are zero).
+// A chunk that holds non-ASCII bytes.  Its ASCII bytes are classified like those of a plain chunk (the other bytes
+// blanked out for the purpose); the loop then visits only the lead bytes of multi-byte characters -- those of the
+// chunk and those of the three bytes before it, whose characters may reach into the chunk -- decodes, validates and
+// looks up each one.  One copy of this code serves every caller (arguments by value: nothing of the caller has to
+// live in memory for the call's sake).
+// w0..w5 = the 4 bytes before the chunk, the chunk, the 4 bytes after it (missing neighbours are zero); g0 = global
+// index (in the aligned frame) of the chunk's first byte; bytes outside [lo, hi) do not exist; valid = the chunk's
+// bytes inside [lo, hi).
+TT_HD_COLD ChunkMasks tt_classify_words_general(u32 w0, u32 w1, u32 w2, u32 w3, u32 w4, u32 w5, long long g0, long long lo,
+                                                long long hi, u32 valid, const u8* stage1, const u8* stage2) {
+    const u32 w[7] = {w0, w1, w2, w3, w4, w5, 0u};
+    ClassTables T;
+    T.stage1 = stage1; T.stage2 = stage2; T.ascii = nullptr;
+    // bit k <- byte k of the chunk has its top bit set / has bit 6 set
+    const u32 na = tt_movemask4(w1) | (tt_movemask4(w2) << 4) | (tt_movemask4(w3) << 8) | (tt_movemask4(w4) << 12);
+    const u32 b6 = tt_movemask4(w1 << 1) | (tt_movemask4(w2 << 1) << 4) | (tt_movemask4(w3 << 1) << 8) | (tt_movemask4(w4 << 1) << 12);
+    const u32 ascm = ~na & valid;
+    // words with the non-ASCII bytes blanked: a byte whose top bit is set becomes 0
+#define TT_BLANK(x) ((x) & ~((((x) >> 7) & 0x01010101u) * 0xFFu))
+    ChunkMasks m = tt_classify_ascii16(TT_BLANK(w1), TT_BLANK(w2), TT_BLANK(w3), TT_BLANK(w4));
+#undef TT_BLANK
+    m.oth &= (u16)ascm; m.spc &= (u16)ascm; m.num &= (u16)ascm; m.low &= (u16)ascm; m.upp &= (u16)ascm;
+    m.nl &= (u16)ascm; m.sp &= (u16)ascm; m.ap &= (u16)ascm; m.sl &= (u16)ascm;
+    u32 lead = ascm, bad = 0, cov = 0;
+    u64 accA = 0, accB = 0;             // 16-bit lanes: A = class codes 0..3, B = codes 4..6
+    const u32 contm = na & ~b6 & valid;                           // continuation bytes of the chunk
+    // lead bytes: bit (j + 3) for j = -3 .. 15
+    u32 todo = ((na & b6) << 3) | ((tt_movemask4(w0) & tt_movemask4(w0 << 1)) >> 1);
+    while (todo) {
+#if defined(__CUDA_ARCH__)
+        const int j = __ffs((int)todo) - 4;
+#else
+        const int j = __builtin_ctz(todo) - 3;
+#endif
+        todo &= todo - 1;
+        if (g0 + j < lo || g0 + j >= hi) continue;          // the byte does not exist
+        const int at = j + 4;                                     // byte index in w
+        const u32 sh = (u32)(at & 3) * 8, x0 = w[at >> 2], x1 = w[(at >> 2) + 1];
+        const u32 v = sh ? (x0 >> sh) | (x1 << (32 - sh)) : x0;   // the lead byte and the three bytes behind it
+        const u32 b = v & 0xFFu, b1 = (v >> 8) & 0xFFu, b2 = (v >> 16) & 0xFFu, b3 = v >> 24;
+        const int n = b >= 0xF0 ? 4 : b >= 0xE0 ? 3 : 2;
+        if (j + n - 1 < 0) continue;                     // ends before this chunk
+        if (j >= 0) lead |= 1u << j;
+        bool ok = (b >= 0xC2) && (b <= 0xF4);
+        u32 cp = b & (0x7Fu >> n);
+        ok = ok && (g0 + j + n - 1 < hi);
+        ok = ok && ((b1 & 0xC0) == 0x80);
+        cp = (cp << 6) | (b1 & 0x3F);
+        if (n >= 3) { ok = ok && ((b2 & 0xC0) == 0x80); cp = (cp << 6) | (b2 & 0x3F); }
+        if (n >= 4) { ok = ok && ((b3 & 0xC0) == 0x80); cp = (cp << 6) | (b3 & 0x3F); }
+        if (n == 3) ok = ok && cp >= 0x800 && !(cp >= 0xD800 && cp <= 0xDFFF);
+        if (n == 4) ok = ok && cp >= 0x10000 && cp <= 0x10FFFF;
+        const u32 span = ((((1u << n) - 1) << (j + 3)) >> 3) & 0xFFFFu;   // bytes of this char inside the chunk
+        if (!ok) { bad |= span; continue; }
+        const u32 c = tt_class_of(cp, T);
+        const u64 lane = (u64)span << ((c & 3) * 16);
+        accA |= (c < 4) ? lane : 0ull;
+        accB |= (c >= 4) ? lane : 0ull;
+        cov |= span;
+    }
+    bad |= contm & ~cov;                                 // continuation byte without a lead
+    m.lead = (u16)(lead & valid);
+    m.oth |= (u16)(accA & valid);          m.mark = (u16)((accA >> 16) & valid);
+    m.spc |= (u16)((accA >> 32) & valid);  m.num |= (u16)((accA >> 48) & valid);
+    m.low |= (u16)(accB & valid);          m.upp |= (u16)((accB >> 16) & valid);
+    m.cless = (u16)((accB >> 32) & valid);
+    m.bad = (u16)(bad & valid);
+    return m;
+}
+
+// `w` = the 4 bytes before the chunk, the chunk, the 4 bytes after it; g0, lo, hi as above.
 TT_HD ChunkMasks tt_classify_words(const u32 (&w)[6], long long g0, long long lo, long long hi, const ClassTables& T) {
-    u64 accA = 0, accB = 0, accF = 0;   // 16-bit lanes: A = codes 0..3, B = codes 4..6, F = flags 1..4
-    u32 lead = 0, bad = 0, cov = 0, contm = 0;
     // bytes of the chunk inside [lo, hi)
     const long long vlo = lo - g0, vhi = hi - g0;
     const u32 klo = vlo <= 0 ? 0u : vlo >= 16 ? 16u : (u32)vlo, khi = vhi <= 0 ? 0u : vhi >= 16 ? 16u : (u32)vhi;
     const u32 valid = khi > klo ? ((1u << khi) - 1u) & ~((1u << klo) - 1u) : 0u;
     const bool all_ascii = ((w[1] | w[2] | w[3] | w[4]) & 0x80808080u) == 0;
-    if (all_ascii) {
-        // sixteen ASCII bytes at once: byte-wise range tests on the four words (see tt_swar_ge), the flag bits gathered
-        // into 16-bit masks; no table look-ups
-        ChunkMasks a = tt_classify_ascii16(w[1], w[2], w[3], w[4]);
-        a.lead = (u16)(0xFFFFu & valid);
-        a.oth &= (u16)valid; a.spc &= (u16)valid; a.num &= (u16)valid; a.low &= (u16)valid; a.upp &= (u16)valid;
-        a.nl &= (u16)valid; a.sp &= (u16)valid; a.ap &= (u16)valid; a.sl &= (u16)valid;
-        return a;
-    } else {
-#pragma unroll
-        for (int j = -3; j < 16; j++) {
-            u32 b = TT_BYTE(w, j);
-            bool exists = (g0 + j >= lo) && (g0 + j < hi);
-            if (!exists) continue;
-            if (b < 0x80) {
-                if (j >= 0) {
-                    u32 v = T.ascii[b];
-                    u32 c = v & 7, f = v >> 3;
-                    u64 bit = 1ull << ((c & 3) * 16 + j);
-                    accA |= (c < 4) ? bit : 0ull;
-                    accB |= (c >= 4) ? bit : 0ull;
-                    accF |= f ? (1ull << ((f - 1) * 16 + j)) : 0ull;
-                    lead |= 1u << j;
-                }
-                continue;
-            }
-            if ((b & 0xC0) == 0x80) { if (j >= 0) contm |= 1u << j; continue; }
-            int n = b >= 0xF0 ? 4 : b >= 0xE0 ? 3 : 2;
-            if (j + n - 1 < 0) continue;                     // ends before this chunk
-            if (j >= 0) lead |= 1u << j;
-            bool ok = (b >= 0xC2) && (b <= 0xF4);
-            u32 cp = b & (0x7Fu >> n);
-            u32 b1 = (j + 1 < 19) ? TT_BYTE(w, (j + 1 < 19 ? j + 1 : 18)) : 0;
-            u32 b2 = (j + 2 < 19) ? TT_BYTE(w, (j + 2 < 19 ? j + 2 : 18)) : 0;
-            u32 b3 = (j + 3 < 19) ? TT_BYTE(w, (j + 3 < 19 ? j + 3 : 18)) : 0;
-            ok = ok && (g0 + j + n - 1 < hi);
-            ok = ok && ((b1 & 0xC0) == 0x80);
-            cp = (cp << 6) | (b1 & 0x3F);
-            if (n >= 3) { ok = ok && ((b2 & 0xC0) == 0x80); cp = (cp << 6) | (b2 & 0x3F); }
-            if (n >= 4) { ok = ok && ((b3 & 0xC0) == 0x80); cp = (cp << 6) | (b3 & 0x3F); }
-            if (n == 3) ok = ok && cp >= 0x800 && !(cp >= 0xD800 && cp <= 0xDFFF);
-            if (n == 4) ok = ok && cp >= 0x10000 && cp <= 0x10FFFF;
-            u32 span = ((((1u << n) - 1) << (j + 3)) >> 3) & 0xFFFFu;   // bytes of this char inside the chunk
-            if (!ok) { bad |= span; continue; }
-            u32 c = tt_class_of(cp, T);
-            u64 lane = (u64)span << ((c & 3) * 16);
-            accA |= (c < 4) ? lane : 0ull;
-            accB |= (c >= 4) ? lane : 0ull;
-            cov |= span;
-        }
-        bad |= contm & ~cov;                                 // continuation byte without a lead
-    }
-    ChunkMasks m;
-    m.lead = (u16)(lead & valid);
-    m.oth = (u16)(accA & valid);          m.mark = (u16)((accA >> 16) & valid);
-    m.spc = (u16)((accA >> 32) & valid);  m.num = (u16)((accA >> 48) & valid);
-    m.low = (u16)(accB & valid);          m.upp = (u16)((accB >> 16) & valid);
-    m.cless = (u16)((accB >> 32) & valid);
-    m.nl = (u16)(accF & valid);           m.sp = (u16)((accF >> 16) & valid);
-    m.ap = (u16)((accF >> 32) & valid);   m.sl = (u16)((accF >> 48) & valid);
-    m.bad = (u16)(bad & valid);
-    return m;
+    if (!all_ascii) return tt_classify_words_general(w[0], w[1], w[2], w[3], w[4], w[5], g0, lo, hi, valid, T.stage1, T.stage2);
+    // sixteen ASCII bytes at once: byte-wise range tests on the four words (see tt_swar_ge), the flag bits gathered
+    // into 16-bit masks; no table look-ups
+    ChunkMasks a = tt_classify_ascii16(w[1], w[2], w[3], w[4]);
+    a.lead = (u16)(0xFFFFu & valid);
+    a.oth &= (u16)valid; a.spc &= (u16)valid; a.num &= (u16)valid; a.low &= (u16)valid; a.upp &= (u16)valid;
+    a.nl &= (u16)valid; a.sp &= (u16)valid; a.ap &= (u16)valid; a.sl &= (u16)valid;
+    return a;
 }
 
 // Loads the chunk and its two 4-byte neighbours with aligned accesses and classifies it.

@@ -6,8 +6,13 @@
 
 #if defined(__CUDACC__)
 #define TT_HD __host__ __device__ __forceinline__
+// Rarely executed and large: kept out of line, so that the code a kernel runs through for every tile stays small
+// enough for the instruction caches.
+#define TT_HD_COLD __host__ __device__ __noinline__
+#define TT_D_COLD __device__ __noinline__
 #else
 #define TT_HD inline
+#define TT_HD_COLD inline
 #endif
 
 typedef uint8_t u8;

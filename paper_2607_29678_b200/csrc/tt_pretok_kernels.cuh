@@ -80,7 +80,7 @@ __device__ __forceinline__ u32 run_mask(const ChunkMasks& m, int kind) {
 // position of the first byte that is not part of the run, with flags in the low three bits:
 // 1 = the run was cut by a document start, 2 = that byte is "other" (4 = a mark), 8 = it is CR/LF.
 // *leads receives the number of code-point leads inside the run (RUN_NUM only).
-__device__ long long coop_back_run(const PretokParams& P, const ClassTables& T, long long gend, int kind,
+TT_D_COLD long long coop_back_run(const PretokParams& P, const ClassTables& T, long long gend, int kind,
                                    long long* scratch, u32* leads) {
     u32 total = 0;
     long long found = COOP_NONE;
@@ -123,27 +123,27 @@ __device__ long long coop_back_run(const PretokParams& P, const ClassTables& T, 
 }
 
 // Number leads (mod 3) of the number run that ends right before gend.
-__device__ u32 coop_back_num(const PretokParams& P, const ClassTables& T, long long gend, long long* scratch) {
+TT_D_COLD u32 coop_back_num(const PretokParams& P, const ClassTables& T, long long gend, long long* scratch) {
     u32 leads = 0;
     coop_back_run(P, T, gend, RUN_NUM, scratch, &leads);
     return leads % 3;
 }
 // Is the byte before gend an "other" character, or a CR/LF run glued to one?  (marks count as
 // "other" only for pattern 0)
-__device__ u32 coop_back_nl(const PretokParams& P, const ClassTables& T, long long gend, long long* scratch) {
+TT_D_COLD u32 coop_back_nl(const PretokParams& P, const ClassTables& T, long long gend, long long* scratch) {
     const long long r = coop_back_run(P, T, gend, RUN_NL, scratch, nullptr);
     if (r & 1) return 0;
     return ((r >> 1) & 1) | (P.pattern != 1 ? ((r >> 2) & 1) : 0);
 }
 // Pattern 1: is the byte before gend a '/' run (or CR/LF run) that belongs to a punctuation tail?
-__device__ u32 coop_back_slash(const PretokParams& P, const ClassTables& T, long long gend, long long* scratch) {
+TT_D_COLD u32 coop_back_slash(const PretokParams& P, const ClassTables& T, long long gend, long long* scratch) {
     const long long r = coop_back_run(P, T, gend, RUN_SL, scratch, nullptr);
     if ((r & 1) || !((r >> 3) & 1)) return 0;                 // cut by a document, or not preceded by CR/LF
     return coop_back_nl(P, T, (r >> 4) + 1, scratch);
 }
 
 // Does the whitespace run that continues at chunk c0 (its first byte) still contain a CR/LF?
-__device__ u32 coop_fwd_nl(const PretokParams& P, const ClassTables& T, long long c0, long long* scratch) {
+TT_D_COLD u32 coop_fwd_nl(const PretokParams& P, const ClassTables& T, long long c0, long long* scratch) {
     for (long long cb = c0;; cb += TT_TILE_CHUNKS) {
         long long chunk = cb + threadIdx.x;
         ChunkMasks m = tt_classify_chunk(P.base, chunk, P.nchunks, P.lo, P.hi, T);
@@ -164,7 +164,7 @@ __device__ u32 coop_fwd_nl(const PretokParams& P, const ClassTables& T, long lon
 
 // Pattern 1: nearest sure piece start (sure_only) or nearest sure-start / unresolved-construct event
 // below gend.  Returns (position << 1) | is_unresolved; the text start is always a sure start.
-__device__ long long coop_back_event(const PretokParams& P, const ClassTables& T, long long gend, bool sure_only,
+TT_D_COLD long long coop_back_event(const PretokParams& P, const ClassTables& T, long long gend, bool sure_only,
                                      long long* scratch) {
     const long long ctop = (gend + TT_CHUNK - 1) / TT_CHUNK;
     for (long long cb = ctop - TT_TILE_CHUNKS;; cb -= TT_TILE_CHUNKS) {
@@ -244,7 +244,10 @@ __device__ __forceinline__ void front_piece_queue(const FrontParams& F, int tile
 // by the latencies between its barriers, which more resident warps hide (10 CTAs, 48 registers, a few spills:
 // the 132 MB batch 1.80 -> 1.64 ms).
 constexpr int PRETOK_CTAS_REQUEST = 6, PRETOK_CTAS_BULK = 10;
-template <bool FUSED, int MINB>
+// PAT = the pattern the kernel is compiled for (P.pattern says the same): each pattern's rules are a few hundred
+// kilobytes of code, and a kernel that carries all of them keeps missing the instruction caches on its way through
+// the one it runs.
+template <bool FUSED, int MINB, int PAT>
 __global__ void __launch_bounds__(TT_TILE_CHUNKS, MINB)
 k_pretok(const PretokParams P, const FrontParams F) {
     extern __shared__ __align__(16) u8 smem_raw[];
@@ -291,7 +294,7 @@ k_pretok(const PretokParams P, const FrontParams F) {
             store_slot(sm, s, tt_classify_chunk(P.base, chunk, P.nchunks, P.lo, P.hi, T), doc_bits(P, chunk));
         }
         __syncthreads();
-        if (P.pattern == 1) {                                          // marks inside words count as caseless letters from here on
+        if (PAT == 1) {                                          // marks inside words count as caseless letters from here on
             const u32 in_own = tt_marks_inside_words(sm, tid + TT_LOW_HALO);
             const int hs = tid < TT_LOW_HALO ? tid : TT_SLOTS - 1;
             const u32 in_halo = tid < TT_LOW_HALO + 1 ? tt_marks_inside_words(sm, hs) : 0u;
@@ -300,7 +303,7 @@ k_pretok(const PretokParams P, const FrontParams F) {
             if (in_halo) { sm[F_MARK][hs] &= (u16)~in_halo; sm[F_CLESS][hs] |= (u16)in_halo; }
             __syncthreads();
         }
-        if (P.pattern == 1) {                                          // sure starts / unresolved constructs per slot
+        if (PAT == 1) {                                          // sure starts / unresolved constructs per slot
             u32 su, ha;
             const long long gs0 = (c_first - TT_LOW_HALO) * TT_CHUNK;       // byte 0 of slot 0
             tt_sure_hard(sm, tid + TT_LOW_HALO, su, ha, P.base, gs0, P.hi);
@@ -315,9 +318,9 @@ k_pretok(const PretokParams P, const FrontParams F) {
         u32 need = 0;
         const int slot = tid + TT_LOW_HALO;
         const long long g0 = (c_first + tid) * TT_CHUNK;
-        u32 S = P.pattern == TT_PATTERN_CUTS ? tt_eval_chunk_cuts(sm, slot, tc, false, need)
-              : P.pattern != 1 ? tt_eval_chunk_p0(sm, slot, P.base, g0, P.hi, tc, false, need, P.pattern == 2, P.docmask)
-                               : tt_eval_chunk_p1(sm, slot, SC, g0, tc, false, need);
+        u32 S = PAT == TT_PATTERN_CUTS ? tt_eval_chunk_cuts(sm, slot, tc, false, need)
+              : PAT != 1 ? tt_eval_chunk_p0(sm, slot, P.base, g0, P.hi, tc, false, need, PAT == 2, P.docmask)
+                         : tt_eval_chunk_p1(sm, slot, SC, g0, tc, false, need);
         if (need) atomicOr(&s_need, need);
         __syncthreads();
         const u32 need_all = s_need;
@@ -325,9 +328,9 @@ k_pretok(const PretokParams P, const FrontParams F) {
             const long long below = (c_first - TT_LOW_HALO) * TT_CHUNK;    // first byte of the low halo
             if (need_all & NEED_N) tc.n_before = coop_back_num(P, T, below, scratch);
             if (need_all & NEED_A) tc.nl_absorbed_before = coop_back_nl(P, T, below, scratch);
-            if (need_all & NEED_S) tc.slash_absorbed_before = coop_back_slash(P, T, below, scratch);
+            if (PAT == 1 && (need_all & NEED_S)) tc.slash_absorbed_before = coop_back_slash(P, T, below, scratch);
             if (need_all & NEED_F) tc.nl_later_after = coop_fwd_nl(P, T, c_first + TT_TILE_CHUNKS + 1, scratch);
-            if (need_all & (NEED_H | NEED_C)) {
+            if (PAT == 1 && (need_all & (NEED_H | NEED_C))) {
                 // events of slot 0 (first halo chunk) are not examined by the walks in shared memory
                 const long long gend = below + TT_CHUNK;
                 const long long ev = coop_back_event(P, T, gend, false, scratch);
@@ -335,9 +338,9 @@ k_pretok(const PretokParams P, const FrontParams F) {
                 tc.sure_before = (ev & 1) ? (coop_back_event(P, T, (ev >> 1) + 1, true, scratch) >> 1) : (ev >> 1);
             }
             need = 0;
-            S = P.pattern == TT_PATTERN_CUTS ? tt_eval_chunk_cuts(sm, slot, tc, true, need)
-              : P.pattern != 1 ? tt_eval_chunk_p0(sm, slot, P.base, g0, P.hi, tc, true, need, P.pattern == 2, P.docmask)
-                               : tt_eval_chunk_p1(sm, slot, SC, g0, tc, true, need);
+            S = PAT == TT_PATTERN_CUTS ? tt_eval_chunk_cuts(sm, slot, tc, true, need)
+              : PAT != 1 ? tt_eval_chunk_p0(sm, slot, P.base, g0, P.hi, tc, true, need, PAT == 2, P.docmask)
+                         : tt_eval_chunk_p1(sm, slot, SC, g0, tc, true, need);
         }
         if (P.litstart && c_first + tid < P.nchunks) {                // an extracted literal is one piece whatever the pattern says
             const long long chunk = c_first + tid;

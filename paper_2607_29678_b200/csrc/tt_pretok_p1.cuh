@@ -141,7 +141,7 @@ TT_HD long long tt_next_doc_start(const u32* docmask, long long g, long long lim
 // provisional end a little past the chunk, and a match that examined the provisional end is repeated
 // with the end moved out geometrically (documents can be megabytes long; pieces rarely are).
 // doc_end returns an end that is exact whenever it is below g0 + 16.
-TT_HD u32 tt_seq_starts_p1(const SeqCtx& C, long long from, long long g0, long long& doc_end) {
+TT_HD_COLD u32 tt_seq_starts_p1(const SeqCtx& C, long long from, long long g0, long long& doc_end) {
     long long end = C.hi;
     bool exact = true;
     if (C.docmask) {

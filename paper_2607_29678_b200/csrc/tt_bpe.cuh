@@ -976,7 +976,7 @@ __device__ void merge_bulk_lists(const PieceParams& P, const u8* __restrict__ te
 
 // The merge kernel of bulk text (more tiles than a request's job search covers): works off the lists k_closing built.
 __global__ void __launch_bounds__(MERGE_THREADS, MERGE_CTAS_PER_SM)
-k_merge_bulk(const PieceParams P) {
+k_merge_bulk(const __grid_constant__ PieceParams P) {
     extern __shared__ __align__(16) u64 s_buf[];              // MERGE_SMEM_BYTES
     __shared__ u32 sc[SCR_WORDS];
     __shared__ u32 s_warps_done;
@@ -991,7 +991,7 @@ k_merge_bulk(const PieceParams P) {
 }
 
 __global__ void __launch_bounds__(MERGE_THREADS, MERGE_CTAS_PER_SM)
-k_merge(const PieceParams P) {
+k_merge(const __grid_constant__ PieceParams P) {
     extern __shared__ __align__(16) u64 s_buf[];              // MERGE_SMEM_BYTES
     __shared__ u32 sc[SCR_WORDS];
     __shared__ uint4 s_long[TT_TILE_LONGCAP + 2];             // the long pieces of one tile

@@ -249,7 +249,7 @@ constexpr int PRETOK_CTAS_REQUEST = 6, PRETOK_CTAS_BULK = 10;
 // the one it runs.
 template <bool FUSED, int MINB, int PAT>
 __global__ void __launch_bounds__(TT_TILE_CHUNKS, MINB)
-k_pretok(const PretokParams P, const FrontParams F) {
+k_pretok(const __grid_constant__ PretokParams P, const __grid_constant__ FrontParams F) {
     extern __shared__ __align__(16) u8 smem_raw[];
     u16 (*sm)[TT_SLOTS] = reinterpret_cast<u16 (*)[TT_SLOTS]>(smem_raw);        // class masks of the tile and its halo
     __shared__ long long scratch[40];

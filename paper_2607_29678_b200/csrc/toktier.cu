@@ -458,7 +458,7 @@ extern "C" size_t tt_workspace_bytes(const tt_vocab* v, size_t max_len, size_t m
 // One instance of the first kernel per pattern (the pattern's rules are compiled in), chosen here.
 template <bool FUSED, int MINB>
 static void launch_pretok(int grid, cudaStream_t st, const PretokParams& P, const FrontParams& F) {
-    const size_t smem = sizeof(u16) * F_COUNT * TT_SLOTS;
+    const size_t smem = TT_PRETOK_SMEM_BYTES;
     switch (P.pattern) {
     case TT_PATTERN_O200K:     k_pretok<FUSED, MINB, TT_PATTERN_O200K><<<grid, TT_TILE_CHUNKS, smem, st>>>(P, F); break;
     case TT_PATTERN_CL100K_N1: k_pretok<FUSED, MINB, TT_PATTERN_CL100K_N1><<<grid, TT_TILE_CHUNKS, smem, st>>>(P, F); break;

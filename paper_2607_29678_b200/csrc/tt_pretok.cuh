@@ -74,12 +74,70 @@ TT_HD int tt_popc(u32 x) {
 #endif
 }
 
+// ---- run summaries of the window's slots -----------------------------------------------------------------------
+// Kept behind the class masks in shared memory: per summary five words, a bit per slot that says "all sixteen bytes
+// are ASCII digits" (summary 0) or "all are blanks other than CR/LF" (summary 1), with no document start among them.
+// Words 0..3: the tile's own slots (bit = thread), word 4: the low halo slots (bits 0..13), the high one (bit 14) and,
+// in bit 31, whether the summary is filled at all (the kernel for bulk text leaves it empty).
+// A walk through a run that fills whole tiles -- a number of twenty thousand digits, 64 KB of blanks -- steps over
+// such slots at once instead of visiting them one by one from every chunk of the tile.
+constexpr int TT_RUNMASK_WORDS = TT_TILE_CHUNKS / 32 + 1;
+constexpr int TT_RUNMASK_OFFSET = (int)((sizeof(u16) * F_COUNT * TT_SLOTS + 15) / 16 * 16);      // bytes from the start of the masks
+constexpr int TT_PRETOK_SMEM_BYTES = TT_RUNMASK_OFFSET + 2 * TT_RUNMASK_WORDS * (int)sizeof(u32);
+TT_HD const u32* tt_runmask(const u16 (*sm)[TT_SLOTS], int which) {
+    return reinterpret_cast<const u32*>(reinterpret_cast<const u8*>(sm) + TT_RUNMASK_OFFSET) + which * TT_RUNMASK_WORDS;
+}
+// highest slot t <= s whose bit is clear (-1: none)
+TT_HD int tt_run_skip_back(const u32* rm, int s) {
+    constexpr int HW = TT_TILE_CHUNKS / 32;
+    if (s >= TT_LOW_HALO + TT_TILE_CHUNKS) { if (!((rm[HW] >> TT_LOW_HALO) & 1)) return s; s = TT_LOW_HALO + TT_TILE_CHUNKS - 1; }
+    if (s >= TT_LOW_HALO) {
+        const int idx = s - TT_LOW_HALO;
+        for (int w = idx >> 5; w >= 0; w--) {
+            u32 clear = ~rm[w];
+            if (w == (idx >> 5)) clear &= 0xFFFFFFFFu >> (31 - (idx & 31));
+            if (clear) return TT_LOW_HALO + w * 32 + tt_hibit(clear);
+        }
+        s = TT_LOW_HALO - 1;
+    }
+    const u32 clear = ~rm[HW] & (0xFFFFFFFFu >> (31 - s)) & ((1u << TT_LOW_HALO) - 1);
+    return clear ? tt_hibit(clear) : -1;
+}
+// lowest slot t >= s whose bit is clear (TT_SLOTS: none)
+TT_HD int tt_run_skip_fwd(const u32* rm, int s) {
+    constexpr int HW = TT_TILE_CHUNKS / 32;
+    if (s >= TT_SLOTS) return TT_SLOTS;
+    if (s < TT_LOW_HALO) {
+        const u32 clear = ~rm[HW] & ((1u << TT_LOW_HALO) - 1) & (0xFFFFFFFFu << s);
+        if (clear) return tt_lobit(clear);
+        s = TT_LOW_HALO;
+    }
+    if (s < TT_LOW_HALO + TT_TILE_CHUNKS) {
+        const int idx = s - TT_LOW_HALO;
+        for (int w = idx >> 5; w < HW; w++) {
+            u32 clear = ~rm[w];
+            if (w == (idx >> 5)) clear &= 0xFFFFFFFFu << (idx & 31);
+            if (clear) return TT_LOW_HALO + w * 32 + tt_lobit(clear);
+        }
+    }
+    return ((rm[HW] >> TT_LOW_HALO) & 1) ? TT_SLOTS : TT_SLOTS - 1;
+}
+
 // Number leads in the number run that ends at the last byte of slot `s` (walking down).
 // Returns the count; sets `open` when the run continues below slot 0.
 TT_HD u32 tt_walk_back_num(const u16 (*sm)[TT_SLOTS], int s, bool& open) {
     u32 cnt = 0;
     open = false;
+    const u32* rm = tt_runmask(sm, 0);
+    const bool summaries = (rm[TT_TILE_CHUNKS / 32] >> 31) != 0;
     for (; s >= 0; s--) {
+        if (summaries) {
+            int t = tt_run_skip_back(rm, s);                // slots of sixteen ASCII digits: sixteen leads each
+            if (t > s) t = s;                               // (never upwards: the loop ends whatever the summary holds)
+            cnt += 16u * (u32)(s - t);
+            s = t;
+            if (s < 0) break;
+        }
         u32 n = sm[F_NUM][s], d = sm[F_DOC][s], ld = sm[F_LEAD][s];
         u32 cut = (~n & 0xFFFFu) | (d >> 1);        // byte j ends the walk if it is not a number byte or j+1 starts a document
         if (cut) { int b = tt_hibit(cut); cnt += tt_popc(ld & n & (0xFFFFu << (b + 1)) & 0xFFFFu); return cnt; }
@@ -114,11 +172,17 @@ TT_HD u32 tt_walk_back_nl(const u16 (*sm)[TT_SLOTS], int s, u32 othmask_fields, 
 TT_HD u32 tt_walk_fwd_nl(const u16 (*sm)[TT_SLOTS], int s, int bit, bool& open) {
     open = false;
     u32 low = (0xFFFFu << (bit + 1)) & 0xFFFFu;
+    const u32* rm = tt_runmask(sm, 1);
+    const bool summaries = (rm[TT_TILE_CHUNKS / 32] >> 31) != 0;
     for (; s < TT_SLOTS; s++) {
         u32 w = sm[F_SPC][s], nl = sm[F_NL][s], d = sm[F_DOC][s];
         u32 ev = ((~w) | d | nl) & low;
         if (ev) { int j = tt_lobit(ev); return ((nl & w & ~d) >> j) & 1; }
         low = 0xFFFFu;
+        if (summaries) {
+            const int t = tt_run_skip_fwd(rm, s + 1);       // slots of sixteen plain blanks hold no event
+            if (t > s + 1) s = t - 1;                       // (never backwards: the loop ends whatever the summary holds)
+        }
     }
     open = true;
     return 0;
@@ -129,7 +193,21 @@ TT_HD u32 tt_walk_fwd_nl(const u16 (*sm)[TT_SLOTS], int s, int bit, bool& open) 
 // document boundary mask to consult; or more than `limit` bytes of blanks).  One thread, plain loads.
 TT_HD int tt_raw_fwd_nl(const u8* base, long long g, long long hi, const u32* docmask, int limit = 256) {
     if (docmask) return -1;
-    for (int k = 0; k < limit; k++, g++) {
+    int k = 0;
+    // sixteen bytes at a time while they are all blanks other than CR/LF (g is a multiple of 16 for every caller;
+    // `base` is 16-byte aligned)
+    if ((g & 15) == 0) {
+        for (; k + 16 <= limit && g + 16 <= hi; k += 16, g += 16) {
+            const uint4 v = *reinterpret_cast<const uint4*>(base + g);
+            const u32 w[4] = {v.x, v.y, v.z, v.w};
+            bool plain = ((v.x | v.y | v.z | v.w) & 0x80808080u) == 0;
+#pragma unroll
+            for (int j = 0; j < 4; j++)
+                plain = plain && (tt_swar_range(w[j], 0x09, 0x09) | tt_swar_range(w[j], 0x0B, 0x0C) | tt_swar_range(w[j], ' ', ' ')) == 0x80808080u;
+            if (!plain) break;
+        }
+    }
+    for (; k < limit; k++, g++) {
         if (g >= hi) return 0;
         const u32 b = base[g];
         if (b == '\n' || b == '\r') return 1;

@@ -70,6 +70,11 @@ __device__ __forceinline__ u32 doc_bits(const PretokParams& P, long long chunk) 
 // positions are in the aligned frame; `gend` is exclusive.
 
 enum { RUN_NUM = 0, RUN_NL = 1, RUN_SL = 2 };
+// The walks are rarely executed, so their instructions come from L2 or beyond, a cache line at a time: what a walk
+// costs is mostly the size of the code it runs through.  They share one copy of the classifier.
+TT_D_COLD ChunkMasks coop_classify(const PretokParams& P, const ClassTables& T, long long chunk) {
+    return tt_classify_chunk(P.base, chunk, P.nchunks, P.lo, P.hi, T);
+}
 constexpr long long COOP_NONE = -(1ll << 60);
 
 __device__ __forceinline__ u32 run_mask(const ChunkMasks& m, int kind) {
@@ -87,7 +92,7 @@ TT_D_COLD long long coop_back_run(const PretokParams& P, const ClassTables& T, l
     const long long ctop = (gend + TT_CHUNK - 1) / TT_CHUNK;          // chunks below ctop are examined
     for (long long cb = ctop - TT_TILE_CHUNKS;; cb -= TT_TILE_CHUNKS) {
         const long long chunk = cb + threadIdx.x;
-        const ChunkMasks m = tt_classify_chunk(P.base, chunk, P.nchunks, P.lo, P.hi, T);
+        const ChunkMasks m = coop_classify(P, T, chunk);
         const u32 d = doc_bits(P, chunk), dn = doc_bits(P, chunk + 1);
         u32 live = 0xFFFFu;                                          // bytes of this chunk below gend
         if (chunk * 16 + 16 > gend) live = gend > chunk * 16 ? (0xFFFFu >> (int)(chunk * 16 + 16 - gend)) : 0u;
@@ -146,7 +151,7 @@ TT_D_COLD u32 coop_back_slash(const PretokParams& P, const ClassTables& T, long 
 TT_D_COLD u32 coop_fwd_nl(const PretokParams& P, const ClassTables& T, long long c0, long long* scratch) {
     for (long long cb = c0;; cb += TT_TILE_CHUNKS) {
         long long chunk = cb + threadIdx.x;
-        ChunkMasks m = tt_classify_chunk(P.base, chunk, P.nchunks, P.lo, P.hi, T);
+        ChunkMasks m = coop_classify(P, T, chunk);
         u32 d = doc_bits(P, chunk);
         u32 ev = ((~(u32)m.spc) | d | m.nl) & 0xFFFFu;       // bytes past the end are not whitespace
         long long neg = COOP_NONE;
@@ -172,9 +177,9 @@ TT_D_COLD long long coop_back_event(const PretokParams& P, const ClassTables& T,
         long long pos = COOP_NONE;
         if (chunk >= 0) {
             ChunkDoc p, c, n;
-            p.m = tt_classify_chunk(P.base, chunk - 1, P.nchunks, P.lo, P.hi, T); p.doc = doc_bits(P, chunk - 1);
-            c.m = tt_classify_chunk(P.base, chunk, P.nchunks, P.lo, P.hi, T);     c.doc = doc_bits(P, chunk);
-            n.m = tt_classify_chunk(P.base, chunk + 1, P.nchunks, P.lo, P.hi, T); n.doc = doc_bits(P, chunk + 1);
+            p.m = coop_classify(P, T, chunk - 1); p.doc = doc_bits(P, chunk - 1);
+            c.m = coop_classify(P, T, chunk);     c.doc = doc_bits(P, chunk);
+            n.m = coop_classify(P, T, chunk + 1); n.doc = doc_bits(P, chunk + 1);
             tt_marks_inside_words_cm(p, c, n);
             u32 sure, hard;
             tt_sure_hard_cm(p, c, n, sure, hard);
@@ -252,6 +257,12 @@ __global__ void __launch_bounds__(TT_TILE_CHUNKS, MINB)
 k_pretok(const __grid_constant__ PretokParams P, const __grid_constant__ FrontParams F) {
     extern __shared__ __align__(16) u8 smem_raw[];
     u16 (*sm)[TT_SLOTS] = reinterpret_cast<u16 (*)[TT_SLOTS]>(smem_raw);        // class masks of the tile and its halo
+    u32* const s_runmask = reinterpret_cast<u32*>(smem_raw + TT_RUNMASK_OFFSET);   // run summaries of the slots, behind the masks
+    // Only the kernel compiled for requests fills them (a request may be one long run; its tiles each get a CTA that
+    // the others wait for).  Bulk text pays for every instruction per tile: there the summaries stay empty and the
+    // walks visit slot after slot.
+    constexpr bool RUN_SUMMARIES = MINB <= PRETOK_CTAS_REQUEST;
+    if (!RUN_SUMMARIES && threadIdx.x < 2 * TT_RUNMASK_WORDS) s_runmask[threadIdx.x] = 0;     // (the first barrier of the tile loop orders this)
     __shared__ long long scratch[40];
     __shared__ u32 s_need, s_first;
     __shared__ u32 s_islast;
@@ -287,11 +298,27 @@ k_pretok(const __grid_constant__ PretokParams P, const __grid_constant__ FrontPa
             const u32 d = doc_bits(P, chunk);
             store_slot(sm, tid + TT_LOW_HALO, m, d);
             any_bad |= m.bad | (d & ~(u32)m.lead & 0xFFFFu & (m.oth | m.mark | m.spc | m.num | m.low | m.upp | m.cless));
+            if (RUN_SUMMARIES) {      // (see tt_runmask) is the slot sixteen ASCII digits / sixteen blanks other than CR/LF?
+                const u32 bn = __ballot_sync(0xFFFFFFFFu, m.num == 0xFFFFu && m.lead == 0xFFFFu && d == 0);
+                const u32 bb = __ballot_sync(0xFFFFFFFFu, m.spc == 0xFFFFu && m.nl == 0 && d == 0);
+                if ((tid & 31) == 0) { s_runmask[tid >> 5] = bn; s_runmask[TT_RUNMASK_WORDS + (tid >> 5)] = bb; }
+            }
         }
-        if (tid < TT_LOW_HALO + 1) {
-            const long long chunk = tid < TT_LOW_HALO ? c_first - TT_LOW_HALO + tid : c_first + TT_TILE_CHUNKS;
-            const int s = tid < TT_LOW_HALO ? tid : TT_SLOTS - 1;
-            store_slot(sm, s, tt_classify_chunk(P.base, chunk, P.nchunks, P.lo, P.hi, T), doc_bits(P, chunk));
+        if (tid < 32) {                                               // the halo slots: the first warp
+            bool hn = false, hb = false;
+            if (tid < TT_LOW_HALO + 1) {
+                const long long chunk = tid < TT_LOW_HALO ? c_first - TT_LOW_HALO + tid : c_first + TT_TILE_CHUNKS;
+                const int s = tid < TT_LOW_HALO ? tid : TT_SLOTS - 1;
+                const ChunkMasks m = tt_classify_chunk(P.base, chunk, P.nchunks, P.lo, P.hi, T);
+                const u32 d = doc_bits(P, chunk);
+                store_slot(sm, s, m, d);
+                hn = m.num == 0xFFFFu && m.lead == 0xFFFFu && d == 0;
+                hb = m.spc == 0xFFFFu && m.nl == 0 && d == 0;
+            }
+            if (RUN_SUMMARIES) {
+                const u32 bn = __ballot_sync(0xFFFFFFFFu, hn), bb = __ballot_sync(0xFFFFFFFFu, hb);
+                if (tid == 0) { s_runmask[TT_TILE_CHUNKS / 32] = bn | 0x80000000u; s_runmask[TT_RUNMASK_WORDS + TT_TILE_CHUNKS / 32] = bb | 0x80000000u; }
+            }
         }
         __syncthreads();
         if (PAT == 1) {                                          // marks inside words count as caseless letters from here on

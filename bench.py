@@ -575,7 +575,7 @@ def main():
         "chars_per_s_single": round(cfg.n_chars / (ms_per_step * 1e-3), 1),
         "e2e": {"value": round(e2e_ms, 4), "unit": "ms", "h2d_bytes_per_step": nbytes, "d2h_bytes_per_step": 4 * n_ids + 12,
                 "p50": round(pct(e2e, 0.5), 4), "pageable_p50": round(pct(e2e_pageable, 0.5), 4),
-                "api": "tt_encode_host, wall clock of the synchronous call; pinned host buffers: text DMA'd from the caller's "
+                "api": "tt_encode_host, wall clock of the synchronous call; pinned host buffers: text read by the first kernel from the caller's "
                        "buffer, ids written by the scatter kernel into the caller's pinned buffer; pageable_p50: the same call "
                        "on pageable buffers (staged through pinned memory inside the library)"},
         "gpu_launches": KERNELS_PER_REQUEST * args.steps,

@@ -283,7 +283,8 @@ int tt_encode_timed(const tt_vocab* v, const uint8_t* text, size_t len, void* st
  * delivers the IDs to `ids_out` and synchronises.  Allocates and caches its own device and pinned staging
  * buffers inside the handle's context (not thread-safe per vocab).  ids_out HOST int32[ids_cap];
  * *count_out HOST.  Page-locked caller buffers (cudaHostAlloc / cudaHostRegister, a pinned tensor) are used
- * directly: `text` is the source of the DMA, and the IDs are written by the scatter kernel through the mapped
+ * directly: the first kernel reads `text` through the mapped pointer tile by tile (no copy in front of the chain; it
+ * leaves a device copy for the later kernels), and the IDs are written by the scatter kernel through the mapped
  * pointer straight into `ids_out` (entries beyond the count are unspecified); pageable buffers are staged.
  * Returns the host code, or the device status if that is not TT_OK.
  */

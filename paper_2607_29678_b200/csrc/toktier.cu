@@ -470,10 +470,16 @@ static void launch_pretok(int grid, cudaStream_t st, const PretokParams& P, cons
 // Enqueues K1+K2 (and K3 when piece_off_dst is given: only tt_pretokenize materialises the offsets;
 // the encode chain derives them per tile from the start flags).
 static int run_pretok(const tt_vocab* v, const uint8_t* text, size_t len, const int64_t* doc_off, size_t n_docs,
-                      cudaStream_t st, TTWorkspace& w, u32* piece_off_dst, PretokParams& P, bool literals = false, bool fused = false) {
+                      cudaStream_t st, TTWorkspace& w, u32* piece_off_dst, PretokParams& P, bool literals = false, bool fused = false,
+                      const uint8_t* host_src = nullptr) {
     const uintptr_t addr = (uintptr_t)text;
     const long long shift = (long long)(addr & 15);
     P.base = (const u8*)(addr - shift);
+    P.src = nullptr; P.copy = nullptr;
+    if (host_src) {                                           // pinned host text, read by the first kernel itself (tt_encode_host)
+        if ((long long)((uintptr_t)host_src & 15) != shift) return TT_ERR_ARG;     // the device copy shares the host text's 16-byte frame
+        P.src = host_src - shift; P.copy = (u8*)(addr - shift);
+    }
     P.lo = shift; P.hi = shift + (long long)len;
     P.nchunks = (P.hi + TT_CHUNK - 1) / TT_CHUNK;
     P.ntiles = (int)((P.nchunks + TT_TILE_CHUNKS - 1) / TT_TILE_CHUNKS);
@@ -555,7 +561,8 @@ static cudaError_t launch_after(void (*kernel)(const Params), int grid, int bloc
 
 static int encode_impl(const tt_vocab* v, const uint8_t* text, size_t len, const int64_t* doc_off, size_t n_docs,
                        cudaStream_t st, int32_t* ids_out, size_t ids_cap, int64_t* count_out, int64_t* ids_off_out,
-                       int32_t* status_out, void* workspace, cudaEvent_t* ev = nullptr, bool literals = false) {
+                       int32_t* status_out, void* workspace, cudaEvent_t* ev = nullptr, bool literals = false,
+                       const uint8_t* host_src = nullptr) {
 #define MARK(i) do { if (ev) cudaEventRecord(ev[i], st); } while (0)
     TTWorkspace w;
     carve(&w, workspace, len, n_docs);
@@ -576,7 +583,7 @@ static int encode_impl(const tt_vocab* v, const uint8_t* text, size_t len, const
     if (doc_off || literals || big || cap != cudaStreamCaptureStatusNone) CK(cudaMemsetAsync(w.hdr, 0, sizeof(TTHeader), st));
     MARK(0);
     PretokParams PP;
-    int rc = run_pretok(v, text, len, doc_off, n_docs, st, w, nullptr, PP, literals, true);
+    int rc = run_pretok(v, text, len, doc_off, n_docs, st, w, nullptr, PP, literals, true, host_src);
     if (rc != TT_OK) return rc;
     MARK(1);
     const int tile_grid = PP.ntiles < v->sm_count * 8 ? PP.ntiles : v->sm_count * 8;
@@ -805,10 +812,13 @@ extern "C" int tt_encode_host(tt_vocab* v, const uint8_t* text, size_t len, int3
     // buffer, and the scatter kernel writes the ids through the mapped pointer straight into the caller's
     // buffer, so no device-to-host copy follows.  Pageable buffers go through the handle's pinned staging.
     int32_t* ids_dev_view = nullptr;
-    const bool in_pinned = len && host_pointer_is_pinned(text, nullptr);
+    const uint8_t* text_dev_view = nullptr;
+    const bool in_pinned = len && host_pointer_is_pinned(text, (void**)&text_dev_view) && text_dev_view != nullptr;
     const bool out_pinned = len && host_pointer_is_pinned(ids_out, (void**)&ids_dev_view) && ids_dev_view != nullptr;
-    if (in_pinned) CK(cudaMemcpyAsync(v->d_text, text, len, cudaMemcpyHostToDevice, st));
-    else {
+    // Pinned text is not copied in front of the chain: the first kernel reads it through the mapped pointer, tile by
+    // tile, and leaves the device copy that the later kernels need -- the transfer runs under the kernel's own work.
+    const uint8_t* d_text = in_pinned ? v->d_text + ((uintptr_t)text_dev_view & 15) : v->d_text;
+    if (!in_pinned) {
         // pageable text is staged in slices, so that the DMA of one slice runs while the next is being staged
         const size_t slice = 256u << 10;
         for (size_t o = 0; o < len; o += slice) {
@@ -825,8 +835,9 @@ extern "C" int tt_encode_host(tt_vocab* v, const uint8_t* text, size_t len, int3
         count_dev = (long long*)p; status_dev = (int32_t*)((long long*)p + 1);
     }
     v->h_scalars[0] = 0; v->h_scalars[1] = 0;
-    int rc = tt_encode(v, v->d_text, len, st, out_pinned ? ids_dev_view : v->d_ids, out_pinned ? ids_cap : v->host_cap,
-                       (int64_t*)count_dev, status_dev, v->d_ws, v->ws_cap);
+    if (v->ws_cap < tt_workspace_bytes(v, len, 1)) return TT_ERR_ARG;
+    int rc = encode_impl(v, d_text, len, nullptr, 1, st, out_pinned ? ids_dev_view : v->d_ids, out_pinned ? ids_cap : v->host_cap,
+                         (int64_t*)count_dev, nullptr, status_dev, v->d_ws, nullptr, false, in_pinned ? text_dev_view : nullptr);
     if (rc != TT_OK) return rc;
     CK(cudaStreamSynchronize(st));
     const int status = (int)(v->h_scalars[1] & 0xFFFFFFFF);

@@ -133,7 +133,7 @@ __device__ __forceinline__ bool toktab_lookup(const TokTable& tab, const u8* __r
     const u32 sb = (u32)(addr & 3), sh = sb * 8, used = sb + n;           // bytes of the aligned window that hold the piece
     u32 x[7];
 #pragma unroll
-    for (int j = 0; j < 7; j++) x[j] = used > 4u * j ? __ldg(w + j) : 0u;  // only words that hold a piece byte
+    for (int j = 0; j < 7; j++) x[j] = used > 4u * j ? w[j] : 0u;          // only words that hold a piece byte (plain loads: the first kernel may have written the text itself)
     u32 k[6];
 #pragma unroll
     for (int j = 0; j < 6; j++) k[j] = toktab_mask_word(__funnelshift_r(x[j], x[j + 1], sh), n, j);

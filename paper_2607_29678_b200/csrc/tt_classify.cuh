@@ -186,18 +186,21 @@ TT_HD ChunkMasks tt_classify_words(const u32 (&w)[6], long long g0, long long lo
     return a;
 }
 
-// Loads the chunk and its two 4-byte neighbours with aligned accesses and classifies it.
-// `base` is 16-byte aligned; chunk in [0, nchunks); chunks outside that range are empty.
-TT_HD ChunkMasks tt_classify_chunk(const u8* base, long long chunk, long long nchunks, long long lo, long long hi,
-                                   const ClassTables& T) {
-    u32 w[6] = {0, 0, 0, 0, 0, 0};
-    if (chunk >= 0 && chunk < nchunks) {
-        const uint4 v = *reinterpret_cast<const uint4*>(base + chunk * TT_CHUNK);
-        w[1] = v.x; w[2] = v.y; w[3] = v.z; w[4] = v.w;
-        if (((v.x | v.y | v.z | v.w) & 0x80808080u) != 0) {       // the neighbours matter only to multi-byte characters
-            if (chunk > 0) w[0] = *reinterpret_cast<const u32*>(base + chunk * TT_CHUNK - 4);
-            if (chunk + 1 < nchunks) w[5] = *reinterpret_cast<const u32*>(base + (chunk + 1) * TT_CHUNK);
-        }
+// Classifies chunk `chunk`, whose sixteen bytes the caller has loaded (v; zero for a chunk outside [0, nchunks)); the
+// two 4-byte neighbours are fetched with aligned accesses where they matter.  `base` is 16-byte aligned.
+TT_HD ChunkMasks tt_classify_chunk_loaded(const uint4 v, const u8* base, long long chunk, long long nchunks, long long lo, long long hi,
+                                          const ClassTables& T) {
+    u32 w[6] = {0, v.x, v.y, v.z, v.w, 0};
+    if (chunk >= 0 && chunk < nchunks && ((v.x | v.y | v.z | v.w) & 0x80808080u) != 0) {       // the neighbours matter only to multi-byte characters
+        if (chunk > 0) w[0] = *reinterpret_cast<const u32*>(base + chunk * TT_CHUNK - 4);
+        if (chunk + 1 < nchunks) w[5] = *reinterpret_cast<const u32*>(base + (chunk + 1) * TT_CHUNK);
     }
     return tt_classify_words(w, chunk * TT_CHUNK, lo, hi, T);
+}
+// Loads the chunk and classifies it; chunks outside [0, nchunks) are empty.
+TT_HD ChunkMasks tt_classify_chunk(const u8* base, long long chunk, long long nchunks, long long lo, long long hi,
+                                   const ClassTables& T) {
+    uint4 v = make_uint4(0, 0, 0, 0);
+    if (chunk >= 0 && chunk < nchunks) v = *reinterpret_cast<const uint4*>(base + chunk * TT_CHUNK);
+    return tt_classify_chunk_loaded(v, base, chunk, nchunks, lo, hi, T);
 }

@@ -22,6 +22,8 @@ enum { NEED_N = 1, NEED_A = 2, NEED_F = 4, NEED_S = 8, NEED_H = 16, NEED_C = 32 
 
 struct PretokParams {
     const u8* base;          // 16-byte aligned address at or below the text
+    const u8* src;           // null, or the same frame in pinned host memory that the device can read: the kernel then takes the
+    u8* copy;                // text from there and leaves a copy of every chunk at `copy` (= base) for all that reads the text later
     long long lo, hi;        // the text occupies [lo, hi) in the aligned frame
     long long nchunks;       // ceil(hi / 16)
     int ntiles;

@@ -73,7 +73,7 @@ enum { RUN_NUM = 0, RUN_NL = 1, RUN_SL = 2 };
 // The walks are rarely executed, so their instructions come from L2 or beyond, a cache line at a time: what a walk
 // costs is mostly the size of the code it runs through.  They share one copy of the classifier.
 TT_D_COLD ChunkMasks coop_classify(const PretokParams& P, const ClassTables& T, long long chunk) {
-    return tt_classify_chunk(P.base, chunk, P.nchunks, P.lo, P.hi, T);
+    return tt_classify_chunk(P.src ? P.src : P.base, chunk, P.nchunks, P.lo, P.hi, T);
 }
 constexpr long long COOP_NONE = -(1ll << 60);
 
@@ -284,7 +284,11 @@ k_pretok(const __grid_constant__ PretokParams P, const __grid_constant__ FrontPa
     ClassTables T;
     T.stage1 = P.cls_tables; T.stage2 = P.cls_tables + 0x1100; T.ascii = P.cls_tables + P.cls_bytes - 128;
     SeqCtx SC;
-    SC.base = P.base; SC.lo = P.lo; SC.hi = P.hi; SC.docmask = P.docmask; SC.T = T;
+    // Where the text is read from: the device buffer, or (host calls with pinned text) the caller's host memory.  In
+    // the second case the CTA that classifies a chunk also writes it to the device copy; this kernel reads that copy
+    // only for the look-ups of the tile's own pieces, behind the tile's barriers.
+    const u8* const rd = P.src ? P.src : P.base;
+    SC.base = rd; SC.lo = P.lo; SC.hi = P.hi; SC.docmask = P.docmask; SC.T = T;
     u32 any_bad = 0;
 
     for (int tile = blockIdx.x; tile < P.ntiles; tile += gridDim.x) {
@@ -294,7 +298,12 @@ k_pretok(const __grid_constant__ PretokParams P, const __grid_constant__ FrontPa
         // phase A: classify own chunk (+ the halo chunks)
         {
             const long long chunk = c_first + tid;
-            const ChunkMasks m = tt_classify_chunk(P.base, chunk, P.nchunks, P.lo, P.hi, T);
+            uint4 v = make_uint4(0, 0, 0, 0);
+            if (chunk < P.nchunks) {
+                v = *reinterpret_cast<const uint4*>(rd + chunk * TT_CHUNK);
+                if (P.src) *reinterpret_cast<uint4*>(P.copy + chunk * TT_CHUNK) = v;
+            }
+            const ChunkMasks m = tt_classify_chunk_loaded(v, rd, chunk, P.nchunks, P.lo, P.hi, T);
             const u32 d = doc_bits(P, chunk);
             store_slot(sm, tid + TT_LOW_HALO, m, d);
             any_bad |= m.bad | (d & ~(u32)m.lead & 0xFFFFu & (m.oth | m.mark | m.spc | m.num | m.low | m.upp | m.cless));
@@ -309,7 +318,7 @@ k_pretok(const __grid_constant__ PretokParams P, const __grid_constant__ FrontPa
             if (tid < TT_LOW_HALO + 1) {
                 const long long chunk = tid < TT_LOW_HALO ? c_first - TT_LOW_HALO + tid : c_first + TT_TILE_CHUNKS;
                 const int s = tid < TT_LOW_HALO ? tid : TT_SLOTS - 1;
-                const ChunkMasks m = tt_classify_chunk(P.base, chunk, P.nchunks, P.lo, P.hi, T);
+                const ChunkMasks m = tt_classify_chunk(rd, chunk, P.nchunks, P.lo, P.hi, T);
                 const u32 d = doc_bits(P, chunk);
                 store_slot(sm, s, m, d);
                 hn = m.num == 0xFFFFu && m.lead == 0xFFFFu && d == 0;
@@ -333,9 +342,9 @@ k_pretok(const __grid_constant__ PretokParams P, const __grid_constant__ FrontPa
         if (PAT == 1) {                                          // sure starts / unresolved constructs per slot
             u32 su, ha;
             const long long gs0 = (c_first - TT_LOW_HALO) * TT_CHUNK;       // byte 0 of slot 0
-            tt_sure_hard(sm, tid + TT_LOW_HALO, su, ha, P.base, gs0, P.hi);
+            tt_sure_hard(sm, tid + TT_LOW_HALO, su, ha, rd, gs0, P.hi);
             sm[F_SURE][tid + TT_LOW_HALO] = (u16)su; sm[F_HARD][tid + TT_LOW_HALO] = (u16)ha;
-            if (tid >= 1 && tid < TT_LOW_HALO) { tt_sure_hard(sm, tid, su, ha, P.base, gs0, P.hi); sm[F_SURE][tid] = (u16)su; sm[F_HARD][tid] = (u16)ha; }
+            if (tid >= 1 && tid < TT_LOW_HALO) { tt_sure_hard(sm, tid, su, ha, rd, gs0, P.hi); sm[F_SURE][tid] = (u16)su; sm[F_HARD][tid] = (u16)ha; }
             __syncthreads();
         }
         // phase B: evaluate the piece-start predicate
@@ -346,7 +355,7 @@ k_pretok(const __grid_constant__ PretokParams P, const __grid_constant__ FrontPa
         const int slot = tid + TT_LOW_HALO;
         const long long g0 = (c_first + tid) * TT_CHUNK;
         u32 S = PAT == TT_PATTERN_CUTS ? tt_eval_chunk_cuts(sm, slot, tc, false, need)
-              : PAT != 1 ? tt_eval_chunk_p0(sm, slot, P.base, g0, P.hi, tc, false, need, PAT == 2, P.docmask)
+              : PAT != 1 ? tt_eval_chunk_p0(sm, slot, rd, g0, P.hi, tc, false, need, PAT == 2, P.docmask)
                          : tt_eval_chunk_p1(sm, slot, SC, g0, tc, false, need);
         if (need) atomicOr(&s_need, need);
         __syncthreads();
@@ -366,7 +375,7 @@ k_pretok(const __grid_constant__ PretokParams P, const __grid_constant__ FrontPa
             }
             need = 0;
             S = PAT == TT_PATTERN_CUTS ? tt_eval_chunk_cuts(sm, slot, tc, true, need)
-              : PAT != 1 ? tt_eval_chunk_p0(sm, slot, P.base, g0, P.hi, tc, true, need, PAT == 2, P.docmask)
+              : PAT != 1 ? tt_eval_chunk_p0(sm, slot, rd, g0, P.hi, tc, true, need, PAT == 2, P.docmask)
                          : tt_eval_chunk_p1(sm, slot, SC, g0, tc, true, need);
         }
         if (P.litstart && c_first + tid < P.nchunks) {                // an extracted literal is one piece whatever the pattern says
@@ -421,9 +430,9 @@ k_pretok(const __grid_constant__ PretokParams P, const __grid_constant__ FrontPa
                     const uintptr_t addr = (uintptr_t)(text + t0 + o[j]);
                     const u32* w = reinterpret_cast<const u32*>(addr & ~(uintptr_t)3);
                     const u32 used = (u32)(addr & 3) + n[j];
-                    x0[j] = __ldg(w);
-                    if (used > 4) x1[j] = __ldg(w + 1);
-                    if (used > 8) x2[j] = __ldg(w + 2);
+                    x0[j] = w[0];                                         // (plain loads: this CTA may have written these bytes itself)
+                    if (used > 4) x1[j] = w[1];
+                    if (used > 8) x2[j] = w[2];
                 }
             }
 #pragma unroll

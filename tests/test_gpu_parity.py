@@ -654,6 +654,15 @@ def test_host_entry_point_with_pinned_buffers():
     assert n == want.size and same(out[:n], want)
     n = gv.encode_host_into(text, pinned_ids)                     # pageable in, pinned out
     assert n == want.size and same(pinned_ids[:n].numpy(), want)
+    # more than 4 MB of pinned text takes the kernels for bulk text
+    big_cfg = wl.CONFIGS["C3"]
+    big = np.concatenate([wl.request(big_cfg, sample=s) for s in range(5)])
+    gb, cb = gpu_vocab("C3"), cpu_vocab("C3")
+    want_big, _ = cb.encode(big, big_cfg.pattern_id, nthreads=8)
+    pinned_big = torch.from_numpy(big).pin_memory()
+    ids_big = torch.empty(big.size, dtype=torch.int32).pin_memory()
+    n = gb.encode_host_into(pinned_big, ids_big)
+    assert n == want_big.size and same(ids_big[:n].numpy(), want_big)
     small = torch.empty(10, dtype=torch.int32).pin_memory()       # too small: capacity error, nothing written past it
     import paper_2607_29678_b200 as tt
     with pytest.raises(tt.TokTierError) as err:

@@ -142,6 +142,43 @@ def test_long_runs_across_tiles(pattern):
     _batch_pieces_check(name, pattern, docs)
 
 
+@pytest.mark.parametrize("pattern", [0, 1, 2])
+def test_long_runs_in_single_requests(pattern):
+    """Runs that fill whole tiles, each text a request of its own (no document mask: the walks may step over whole
+    slots of digits or blanks and look ahead in the raw text): digit runs with a non-ASCII digit, a letter or nothing
+    in them, blank runs with tabs, form feeds, no-break and ideographic spaces, with and without a CR/LF at the far
+    end, at every alignment to the 16-byte slots."""
+    name = "C4" if pattern == 1 else "C2"
+    gv, cv = gpu_vocab(name, pattern=pattern), cpu_vocab(name)
+    rng = random.Random(300 + pattern)
+    for trial in range(48):
+        parts = [rng.choice(["", "x", "ab ", "é", "12 "]) + "y" * rng.randrange(0, 40)]
+        for _ in range(rng.randrange(1, 4)):
+            k = rng.randrange(6)
+            n = rng.choice([rng.randrange(1, 300), rng.randrange(1000, 9000), rng.randrange(15000, 30000)])
+            if k == 0:
+                parts.append("7" * n)
+            elif k == 1:                                          # a digit run with one foreign character somewhere
+                cut = rng.randrange(0, n + 1)
+                parts.append("3" * cut + rng.choice(["٣", "²", "a", ".", " "]) + "8" * (n - cut))
+            elif k == 2:
+                parts.append(rng.choice(["", "!", "a", "\n"]) + " " * n + rng.choice(["", "x", "\n", "\r\n!", "1", "\u00a0\n"]))
+            elif k == 3:                                          # blanks of several kinds, a CR/LF somewhere or nowhere
+                blanks = "".join(rng.choice([" ", " ", " ", "\t", "\x0c", "\x0b"]) for _ in range(min(n, 4000))) + " " * max(n - 4000, 0)
+                cut = rng.randrange(0, len(blanks) + 1)
+                parts.append(blanks[:cut] + rng.choice(["", "\n", "\r", "\u3000", "\u00a0", "\u2028"]) + blanks[cut:] + rng.choice(["", "z", "\n"]))
+            elif k == 4:
+                parts.append(" " * rng.randrange(1, 40) + "word" + "\t" * n)
+            else:
+                parts.append("0" * n + " " * rng.randrange(1, 5000) + "9" * rng.randrange(1, 5000))
+        text = np.frombuffer("".join(parts).encode("utf-8"), dtype=np.uint8)
+        want_ids, want = cv.encode(text, pattern, nthreads=4)
+        got, status = gpu_pretok(gv, text)
+        assert status == 0 and same(got, want[:-1]), (trial, first_difference(got, want[:-1]))
+        ids, status = gpu_encode(gv, text)
+        assert status == 0 and same(ids, want_ids), trial
+
+
 def test_batch_ids_match_documents_alone():
     cfg = wl.CONFIGS["C5"]
     text, off = wl.batch(cfg, n_docs=12, scale=0.02)

@@ -48,7 +48,7 @@ struct tt_vocab {
     LitTable lit{};                      // added-token literals (tt_vocab_add_literals), n == 0: none
     u32 max_token_chars = 1;             // characters of the longest entry (stable boundary check of the sessions)
     // cached buffers of tt_encode_host
-    u8* h_text = nullptr; int32_t* h_ids = nullptr; long long* h_scalars = nullptr;
+    u8* h_text = nullptr; int32_t* h_ids = nullptr; long long* h_scalars = nullptr; long long* h_scalars_dev = nullptr;
     u8* d_text = nullptr; int32_t* d_ids = nullptr; long long* d_count = nullptr; int32_t* d_status = nullptr;
     void* d_ws = nullptr; size_t host_cap = 0, ws_cap = 0;
     cudaStream_t host_stream = nullptr;
@@ -830,9 +830,12 @@ extern "C" int tt_encode_host(tt_vocab* v, const uint8_t* text, size_t len, int3
     // count and status are written by the kernel into mapped pinned scalars of the handle
     long long* count_dev = nullptr; int32_t* status_dev = nullptr;
     {
-        void* p = nullptr;
-        if (!host_pointer_is_pinned(v->h_scalars, &p) || !p) return TT_ERR_CUDA;
-        count_dev = (long long*)p; status_dev = (int32_t*)((long long*)p + 1);
+        if (!v->h_scalars_dev) {                                  // looked up once: the buffer lives as long as the handle
+            void* p = nullptr;
+            if (!host_pointer_is_pinned(v->h_scalars, &p) || !p) return TT_ERR_CUDA;
+            v->h_scalars_dev = (long long*)p;
+        }
+        count_dev = v->h_scalars_dev; status_dev = (int32_t*)(v->h_scalars_dev + 1);
     }
     v->h_scalars[0] = 0; v->h_scalars[1] = 0;
     if (v->ws_cap < tt_workspace_bytes(v, len, 1)) return TT_ERR_ARG;

@@ -4,13 +4,13 @@
 // GPU hash tables; a round's minimum rank identifies one pair value, merging all its leftmost
 // non-overlapping occurrences equals iterated single merges, and only pairs next to a completed
 // merge need to be probed again.  Work is dispatched by piece length and difficulty:
-//   * k_lookup: a thread per piece looks the whole piece up as a vocabulary entry (one 32-byte probe); pieces
-//     that are not a single entry are appended to global queues by length class;
-//   * k_merge: every warp of the GPU draws from those queues -- a warp per piece (<= 32 bytes: tokens in
-//     registers, candidates as ballot masks; <= 256 bytes: several tokens per lane, compaction through shared
-//     memory), or, where the call has many pieces of <= 32 bytes, 32 of them at once, a thread per piece
-//     (lane_merge); longer pieces are merged by a whole CTA (cta_merge_long: state in shared memory, or in
-//     global scratch while the piece still has more than 4,096 tokens).
+//   * the first kernel (k_pretok, fused) has looked every piece up as a whole vocabulary entry (one 32-byte probe) and
+//     left the others in its tile's queue region by length class;
+//   * k_merge (a request) / k_closing + k_merge_bulk (bulk text): a warp per piece (<= 32 bytes: tokens in registers,
+//     candidates as ballot masks; <= 256 bytes: several tokens per lane, compaction through shared memory), or, where
+//     the call has many pieces of <= 32 bytes, 32 of them at once, a thread per piece (lane_merge); longer pieces
+//     are merged by a whole CTA of 768 threads (cta_merge_long: state in shared memory, or in global scratch while
+//     the piece still has more than 14,336 tokens).
 // Token ids inside the kernels are "internal": byte b -> b, result of the merge of rank r -> 256 + r;
 // the caller's ids are looked up when the tokens are staged.
 //

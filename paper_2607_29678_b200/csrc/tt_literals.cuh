@@ -9,8 +9,8 @@
 //                 it is selected in turn).  A selected literal becomes a document of its own in the boundary
 //                 mask (so the segments around it are tokenized as independent texts), its first byte is
 //                 marked in litstart and its other bytes in litin.
-// k_pretok then forces exactly one piece per literal (start bit at its first byte, none inside) and k_lookup
-// emits the staged id for a piece that begins at a litstart bit.
+// k_pretok then forces exactly one piece per literal (start bit at its first byte, none inside) and, in its look-up
+// half, takes the staged id for a piece that begins at a litstart bit.
 #pragma once
 #include "tt_common.cuh"
 

@@ -245,10 +245,12 @@ __device__ __forceinline__ void front_piece_queue(const FrontParams& F, int tile
 // otherwise.  Everything a tile leaves behind has this CTA as its only writer: no atomics on global memory, no
 // counter that would have to be cleared before the call.
 // MINB = CTAs per SM the kernel is compiled for.  A request (at most a few tiles per CTA) is a latency chain and
-// gets the registers it wants (6 CTAs of 128 threads, 80 registers); bulk text is bound by instruction issue and
-// by the latencies between its barriers, which more resident warps hide (10 CTAs, 48 registers, a few spills:
-// the 132 MB batch 1.80 -> 1.64 ms).
-constexpr int PRETOK_CTAS_REQUEST = 6, PRETOK_CTAS_BULK = 10;
+// gets the registers it wants (6 CTAs of 128 threads, 80 registers) and four table look-ups in flight per thread.
+// Bulk text is bound by instruction issue and by the latencies between its barriers, which more resident warps
+// hide better than anything a thread does for itself: 16 CTAs per SM (every warp slot taken, 32 registers, a few
+// spills) with one look-up at a time per thread.  The 132 MB batch: 1.80 ms at 6 CTAs, 1.64 at 10, 1.42 with the
+// rare paths out of line, 1.34 with one look-up in flight instead of four, 1.31 at 12 CTAs, 1.28 at 16.
+constexpr int PRETOK_CTAS_REQUEST = 6, PRETOK_CTAS_BULK = 16;
 // PAT = the pattern the kernel is compiled for (P.pattern says the same): each pattern's rules are a few hundred
 // kilobytes of code, and a kernel that carries all of them keeps missing the instruction caches on its way through
 // the one it runs.
@@ -418,11 +420,12 @@ k_pretok(const __grid_constant__ PretokParams P, const __grid_constant__ FrontPa
         const u32 nlook = np ? np - 1 : 0;
         const bool quick = P.litstart == nullptr && F.toktab.slots != nullptr;     // block-uniform
         u32 wsum = 0;
-        for (u32 ib = tid; ib < nlook; ib += 4 * TT_TILE_CHUNKS) {
-            u32 o[4], n[4], k0[4], k1[4], h[4], x0[4], x1[4], x2[4];
-            uint4 sl[4];
+        constexpr int LW = MINB > PRETOK_CTAS_REQUEST ? 1 : 4;       // look-ups in flight per thread
+        for (u32 ib = tid; ib < nlook; ib += LW * TT_TILE_CHUNKS) {
+            u32 o[LW], n[LW], k0[LW], k1[LW], h[LW], x0[LW], x1[LW], x2[LW];
+            uint4 sl[LW];
 #pragma unroll
-            for (int j = 0; j < 4; j++) {
+            for (int j = 0; j < LW; j++) {
                 const u32 i = ib + j * TT_TILE_CHUNKS;
                 o[j] = 0; n[j] = 0; x0[j] = 0; x1[j] = 0; x2[j] = 0;
                 if (i < nlook) { o[j] = s_off[i]; n[j] = (u32)s_off[i + 1] - o[j]; }
@@ -436,7 +439,7 @@ k_pretok(const __grid_constant__ PretokParams P, const __grid_constant__ FrontPa
                 }
             }
 #pragma unroll
-            for (int j = 0; j < 4; j++) {
+            for (int j = 0; j < LW; j++) {
                 k0[j] = 0; k1[j] = 0; h[j] = 0; sl[j] = make_uint4(0, 0, 0, 0);
                 if (quick && n[j] != 0 && n[j] <= 8) {
                     toktab_key01(x0[j], x1[j], x2[j], (u32)((uintptr_t)(text + t0 + o[j]) & 3), n[j], k0[j], k1[j]);
@@ -448,7 +451,7 @@ k_pretok(const __grid_constant__ PretokParams P, const __grid_constant__ FrontPa
                 }
             }
 #pragma unroll
-            for (int j = 0; j < 4; j++) {
+            for (int j = 0; j < LW; j++) {
                 const u32 i = ib + j * TT_TILE_CHUNKS;
                 if (n[j] == 0) continue;
                 bool settled = false;
@@ -523,7 +526,7 @@ k_pretok(const __grid_constant__ PretokParams P, const __grid_constant__ FrontPa
 
 // ---- K3: compaction of the start flags into piece offsets (tt_pretokenize) --------------------------
 // piece_off[i] = byte offset (relative to the text) of piece i; piece_off[n_pieces] = len.  The encode
-// chain does the same per tile in shared memory (tile_pieces in tt_bpe.cuh) and never stores the list.
+// chain does the same per tile in shared memory (the fused half of k_pretok) and keeps the offsets per tile.
 __global__ void __launch_bounds__(TT_TILE_CHUNKS)
 k_compact(const u16* __restrict__ startmask, const u32* __restrict__ tile_base, long long nchunks, int ntiles,
           long long shift, long long len, u32* __restrict__ piece_off, TTHeader* hdr, unsigned long long epoch) {

@@ -194,7 +194,7 @@ static int build_token_table(tt_vocab* v, const tt_merge* merges, size_t n_merge
         Q.hdr = d_hdr; Q.epoch = next_epoch(); Q.tab = v->tab;
         Q.toktab.slots = nullptr; Q.toktab.mask = 0; Q.toktab.shift = 0;      // no table yet: every piece is merged
         Q.longtab = LongTable{}; Q.litstart = nullptr;
-        Q.ext_id = v->d_ext_id; Q.piece_cnt = d_cnt; Q.stage = d_stage; Q.pairbuf = nullptr; Q.tile_tok = d_tt; Q.grp_tok = nullptr; Q.wq = nullptr; Q.gq = nullptr; Q.lq = nullptr;
+        Q.ext_id = v->d_ext_id; Q.piece_cnt = d_cnt; Q.stage = d_stage; Q.pairbuf = nullptr; Q.tile_tok = d_tt; Q.grp_tok = nullptr; Q.wq = nullptr; Q.gq = nullptr; Q.gq_x[0] = Q.gq_x[1] = Q.gq_x[2] = nullptr; Q.lq = nullptr;
         k_merge<<<v->sm_count * MERGE_CTAS_PER_SM, MERGE_THREADS, MERGE_SMEM_BYTES>>>(Q);
         ok = cudaGetLastError() == cudaSuccess && cudaDeviceSynchronize() == cudaSuccess;
     }
@@ -436,9 +436,18 @@ static size_t carve(TTWorkspace* w, void* base, size_t max_len, size_t max_docs)
     p = take(ntiles * TT_TILE_BYTES * sizeof(u16));          if (w) w->piece_off16 = (u16*)p;
     p = take(ntiles * TT_TILE_BYTES * sizeof(u32));          if (w) w->piece_cnt = (u32*)p;
     p = take(ntiles * TT_TILE_QCAP * sizeof(u32));           if (w) w->q = (u32*)p;
-    p = take((max_len / 33 + 64) * sizeof(u64));             if (w) w->wq = (u64*)p;
-    p = take((max_len / 2 + 64) * sizeof(u64));              if (w) w->gq = (u64*)p;
-    p = take((max_len / 257 + 16) * sizeof(uint4));          if (w) w->lq = (uint4*)p;
+    // the global lists of bulk text: only where a text can have more tiles than a request's job search covers (any
+    // alignment of the text counted in)
+    const bool bulk_lists = (15 + max_len + TT_TILE_BYTES - 1) / TT_TILE_BYTES > (size_t)MERGE_SR_MAX_TILES;
+    if (w) { w->wq = nullptr; w->gq = nullptr; w->lq = nullptr; for (int c = 0; c < TT_SHORT_CLASSES - 1; c++) w->gq_x[c] = nullptr; }
+    if (bulk_lists) {
+        p = take((max_len / 33 + 64) * sizeof(u64));             if (w) w->wq = (u64*)p;
+        p = take((max_len / 2 + 64) * sizeof(u64));              if (w) w->gq = (u64*)p;
+        for (int c = 1; c < TT_SHORT_CLASSES; c++) {              // a piece of class c has more bytes than class c - 1 allows
+            p = take((max_len / (tt_short_class_max(c - 1) + 1) + 64) * sizeof(u64));   if (w) w->gq_x[c - 1] = (u64*)p;
+        }
+        p = take((max_len / 257 + 16) * sizeof(uint4));          if (w) w->lq = (uint4*)p;
+    }
     p = take((max_len + 1) * sizeof(int32_t));  if (w) w->stage = (int32_t*)p;
     p = take((max_len + 1) * sizeof(u64));      if (w) w->pairbuf = (u64*)p;
     p = take(padded + 16);                      if (w) w->cand = (u8*)p;
@@ -595,7 +604,8 @@ static int encode_impl(const tt_vocab* v, const uint8_t* text, size_t len, const
     Q.hdr = w.hdr; Q.tab = v->tab; Q.toktab = v->toktab; Q.longtab = v->longtab; Q.litstart = literals ? w.litstart : nullptr; Q.epoch = PP.epoch;
     Q.ext_id = v->d_ext_id; Q.piece_cnt = w.piece_cnt; Q.stage = w.stage; Q.pairbuf = w.pairbuf; Q.tile_tok = w.tile_tok;
     Q.grp_tok = PP.ntiles > MERGE_SR_MAX_TILES ? w.grp_tok : nullptr;   // group totals only where k_scatter's CTAs would otherwise sum thousands of tiles each
-    Q.wq = big ? w.wq : nullptr; Q.gq = big ? w.gq : nullptr; Q.lq = big ? w.lq : nullptr;
+    Q.wq = big ? w.wq : nullptr; Q.gq = big ? w.gq : nullptr;
+    for (int c = 0; c < TT_SHORT_CLASSES - 1; c++) Q.gq_x[c] = big ? w.gq_x[c] : nullptr; Q.lq = big ? w.lq : nullptr;
     if (big) {                                                               // bulk text: closing pieces and the global lists first
         const int cgrid = (PP.ntiles + CLOSING_THREADS - 1) / CLOSING_THREADS;
         if (ev) k_closing<<<cgrid, CLOSING_THREADS, 0, st>>>(Q);

@@ -729,7 +729,8 @@ struct PieceParams {
     u32* tile_tok;
     u32* grp_tok;              // bulk text: tokens per group of TT_GROUP_TILES tiles (written by the last CTA), else null
     u64* wq;                   // bulk text: the warp-class pieces of all tiles (tile << 32 | queue entry), else null
-    u64* gq;                   // bulk text: the short pieces of all tiles, gathered by k_closing (tile << 32 | queue entry)
+    u64* gq;                   // bulk text: the short pieces of all tiles, gathered by k_closing (tile << 32 | queue entry),
+    u64* gq_x[3];              // one list per length class (tt_short_class_max); gq is the first
     uint4* lq;                 // bulk text: the long pieces of all tiles, listed by k_closing (text offset, bytes, piece slot, 0)
 };
 
@@ -823,6 +824,11 @@ __device__ __forceinline__ u64 warp_exscan_u64(u64 v, int lane, u64* total) {
 // closing pieces join the first kernel's list, long pieces get a list of their own.  The counters were cleared
 // by the memset in front of the chain.
 constexpr int CLOSING_THREADS = 256;
+// Length class of a short piece (2..32 bytes).
+__device__ __forceinline__ int short_class(u32 n) {
+    return n <= (u32)tt_short_class_max(0) ? 0 : n <= (u32)tt_short_class_max(1) ? 1 : n <= (u32)tt_short_class_max(2) ? 2 : 3;
+}
+
 __global__ void __launch_bounds__(CLOSING_THREADS)
 k_closing(const PieceParams P) {
     const int lane = threadIdx.x & 31;
@@ -859,17 +865,35 @@ k_closing(const PieceParams P) {
         }
         if (cn > (u32)TT_WARP_PIECE_MAX) P.lq[b] = make_uint4(ca, cn, cslot, 0u);
     }
-    // short pieces: one reservation per warp
-    const u32 mine = ns + (centry ? 1u : 0u);
-    u32 pre = mine;
+    // short pieces: three lists by length (a warp later merges 32 pieces of one list at a time, a thread each, and
+    // waits for the longest), one reservation per warp and list
+    u64 mine = 0;                                             // four counts of 16 bits (a warp's 32 tiles hold fewer than 2^16 pieces)
+    for (u32 e = 0; e < ns; e++) mine += 1ull << (16 * short_class((P.q[(size_t)t * TT_TILE_QCAP + e] >> 22) + 1));
+    if (centry) mine += 1ull << (16 * short_class(cn));
+    u64 pre = mine;
 #pragma unroll
-    for (int o = 1; o < 32; o <<= 1) { const u32 v = __shfl_up_sync(FULL, pre, o); if (lane >= o) pre += v; }
-    const u32 tot = __shfl_sync(FULL, pre, 31);
-    u32 base = 0;
-    if (lane == 31 && tot) base = atomicAdd(&P.hdr->nq_short, tot);
-    base = __shfl_sync(FULL, base, 31) + pre - mine;
-    for (u32 e = 0; e < ns; e++) P.gq[base + e] = ((u64)(u32)t << 32) | P.q[(size_t)t * TT_TILE_QCAP + e];
-    if (centry) P.gq[base + ns] = ((u64)(u32)t << 32) | centry;
+    for (int o = 1; o < 32; o <<= 1) { const u64 v = __shfl_up_sync(FULL, pre, o); if (lane >= o) pre += v; }
+    const u64 tot = __shfl_sync(FULL, pre, 31);
+    u32 base[TT_SHORT_CLASSES];
+#pragma unroll
+    for (int c = 0; c < TT_SHORT_CLASSES; c++) {
+        const u32 n = (u32)(tot >> (16 * c)) & 0xFFFFu;
+        base[c] = 0;
+        if (lane == 31 && n) base[c] = atomicAdd(c ? &P.hdr->nq_short_x[c - 1] : &P.hdr->nq_short, n);
+    }
+    pre -= mine;
+#pragma unroll
+    for (int c = 0; c < TT_SHORT_CLASSES; c++) base[c] = __shfl_sync(FULL, base[c], 31) + ((u32)(pre >> (16 * c)) & 0xFFFFu);
+    for (u32 e = 0; e <= ns; e++) {
+        if (e == ns && !centry) break;
+        const u32 entry = e < ns ? P.q[(size_t)t * TT_TILE_QCAP + e] : centry;
+        const int c = short_class((entry >> 22) + 1);
+        const u64 x = ((u64)(u32)t << 32) | entry;
+        if (c == 0) P.gq[base[0]++] = x;
+        else if (c == 1) P.gq_x[0][base[1]++] = x;
+        else if (c == 2) P.gq_x[1][base[2]++] = x;
+        else P.gq_x[2][base[3]++] = x;
+    }
 }
 
 // Long pieces of the tiles [t_lo, t_hi) (at most MERGE_THREADS of them), a whole CTA each.  Called by all threads
@@ -932,8 +956,8 @@ __device__ __forceinline__ void merge_group_totals(const PieceParams& P, u32* s_
     }
 }
 
-// Bulk text (k_closing has gathered one list per length class): long pieces a CTA each, warp-class pieces a warp
-// each by index, short pieces 32 at a time by ticket, a thread each.
+// Bulk text (k_closing has gathered the lists): long pieces a CTA each, warp-class pieces a warp each by index,
+// short pieces 32 of one length class at a time by ticket, a thread each.
 __device__ void merge_bulk_lists(const PieceParams& P, const u8* __restrict__ text, u64* s_buf, u32* sc, u32* s_warps_done) {
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
     const u32 FULL = 0xFFFFFFFFu;
@@ -954,13 +978,27 @@ __device__ void merge_bulk_lists(const PieceParams& P, const u8* __restrict__ te
         warp_merge_piece(P, text, (u32)((long long)t * TT_TILE_BYTES + (e & 2047u) - P.shift), (e >> 22) + 1, t * TT_TILE_BYTES + ((e >> 11) & 2047u), wbuf, lane);
     }
     u32* const tok = reinterpret_cast<u32*>(wbuf);
-    for (;;) {                                                        // bounded by the list length
-        u32 e0 = 0;
-        if (lane == 0) e0 = atomicAdd(&P.hdr->t_short, (u32)LANE_SLOTS);
-        e0 = __shfl_sync(FULL, e0, 0);
-        if (e0 >= ns) break;
-        if (e0 + lane < ns) {
-            const u64 x = P.gq[e0 + lane];
+    // tickets: 32 pieces of one list each, the list of the longest pieces first
+    u32 cnts[TT_SHORT_CLASSES], nb[TT_SHORT_CLASSES], nball = 0;
+#pragma unroll
+    for (int c = 0; c < TT_SHORT_CLASSES; c++) { cnts[c] = c ? P.hdr->nq_short_x[c - 1] : ns; nb[c] = (cnts[c] + LANE_SLOTS - 1) / LANE_SLOTS; nball += nb[c]; }
+    for (;;) {                                                        // bounded by the number of tickets
+        u32 tk = 0;
+        if (lane == 0) tk = atomicAdd(&P.hdr->t_short, 1u);
+        tk = __shfl_sync(FULL, tk, 0);
+        if (tk >= nball) break;
+        const u64* list = P.gq; u32 cnt = 0, e0 = 0;
+        {
+            u32 r = tk;
+            bool found = false;
+#pragma unroll
+            for (int c = TT_SHORT_CLASSES - 1; c >= 0; c--) {
+                if (!found && r < nb[c]) { list = c ? P.gq_x[c - 1] : P.gq; cnt = cnts[c]; e0 = r * LANE_SLOTS; found = true; }
+                if (!found) r -= nb[c];
+            }
+        }
+        if (e0 + lane < cnt) {
+            const u64 x = list[e0 + lane];
             const u32 t = (u32)(x >> 32), e = (u32)x;
             const u32 a = (u32)((long long)t * TT_TILE_BYTES + (e & 2047u) - P.shift), n = (e >> 22) + 1, slot = t * TT_TILE_BYTES + ((e >> 11) & 2047u);
             if (!piece_in_range(P, a, n, slot, 4u) || n < 2 || n > (u32)LANE_MAX) hdr_selfcheck_failed(P.hdr, P.epoch, 5u, a, n, slot, e0);

@@ -42,6 +42,9 @@ constexpr u32 TT_MAX_INTERNAL = 1u << TT_ID_BITS;
 constexpr u32 TT_RANK_INF = 0xFFFFFFFFu;
 constexpr u64 TT_SLOT_EMPTY = ~0ull;              // pair-table slot: (left << 38) | (right << 20) | rank
 constexpr int TT_WARP_PIECE_MAX = 256;            // bytes; longer pieces take the block-cooperative path
+// Bulk text: length classes of the pieces of at most 32 bytes (largest length of each class).
+constexpr int TT_SHORT_CLASSES = 4;
+TT_HD constexpr int tt_short_class_max(int c) { return c == 0 ? 6 : c == 1 ? 10 : c == 2 ? 16 : 32; }
 
 // ---- workspace header (device memory) -----------------------------------------------------------
 struct TTHeader {
@@ -53,8 +56,9 @@ struct TTHeader {
     u32 nwq;                 // bulk text: lengths of the global lists of warp-class, short and long pieces and the ticket
     u32 nq_short, nq_long;   //            counter of the short list (all cleared by a memset before the chain)
     u32 t_short;
+    u32 nq_short_x[3];       // bulk text: the short pieces have a list per length class; lengths of the other lists (cleared likewise)
     u32 dbg[8];              // first failed self-check of a kernel: site, then up to seven values (diagnostics only)
-    u32 pad[14];
+    u32 pad[11];
 };
 static_assert(sizeof(TTHeader) == 128, "header layout");
 
@@ -115,7 +119,8 @@ struct TTWorkspace {
     u32* piece_cnt;
     u32* q;
     u64* wq;           // bulk text only: warp-class pieces of all tiles (len / 33 + 64 entries)
-    u64* gq;           // bulk text only: short pieces of all tiles (len / 2 + 64 entries)
+    u64* gq;           // bulk text only: short pieces of all tiles by length class (see tt_short_class_max): a warp merges 32
+    u64* gq_x[3];      // pieces of one list at a time, a thread each, and is done when the longest of them is
     uint4* lq;         // bulk text only: long pieces of all tiles (len / 257 + 16 entries)
     int32_t* stage;    // token ids staged at the byte offset of their piece (len)
     u64* pairbuf;      // (token, rank) pairs of the long-piece path, indexed like the text (len)

@@ -61,7 +61,7 @@ class ClockSampler:
 
     def start(self):
         try:
-            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100",
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "20",
                                           "-i", str(self.gpu)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.t = threading.Thread(target=self._read, daemon=True)
             self.t.start()
@@ -71,6 +71,12 @@ class ClockSampler:
     def _read(self):
         for line in self.proc.stdout:
             self.lines.append(line.strip())
+
+    def wait_first_sample(self, limit_s: float = 2.0):
+        """Returns once nvidia-smi has delivered a sample (or after limit_s)."""
+        t0 = time.time()
+        while self.proc and not self.lines and time.time() - t0 < limit_s:
+            time.sleep(0.01)
 
     def stop(self):
         if not self.proc:
@@ -286,6 +292,11 @@ def main():
     def step(i):
         vocab.encode(dev_texts[i % N_DISTINCT_INPUTS], bufs)
 
+    # The clock sampler runs from before the warm-up to the end of the timed region (the region itself lasts a few
+    # milliseconds, less than nvidia-smi needs to start): its samples are taken under the same load.
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    sampler.wait_first_sample()
     for w in range(args.warmup):
         flush_l2(); step(w)
     torch.cuda.synchronize()
@@ -293,8 +304,6 @@ def main():
         dist.barrier()
 
     # ---- timed region: K steps, device time per step, L2 flushed (outside the events) before each ----
-    sampler = ClockSampler(local_rank)
-    sampler.start()
     ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
     torch.cuda.synchronize()
     for k in range(args.steps):

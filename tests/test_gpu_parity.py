@@ -179,6 +179,33 @@ def test_long_runs_in_single_requests(pattern):
         assert status == 0 and same(ids, want_ids), trial
 
 
+def test_bulk_text_short_pieces_of_every_length():
+    """More than 4 MB in one call (the kernels for bulk text), made of random-letter words of every length from 2 to
+    40 under a small vocabulary, so that nearly every word needs merging: all the length classes of the short-piece
+    lists, their boundaries, and the warp-per-piece list are filled, some of them with a single length only."""
+    rng = np.random.default_rng(77)
+    gv, cv = gpu_vocab("C1"), cpu_vocab("C1")
+    pattern = wl.CONFIGS["C1"].pattern_id
+    for lengths in (range(2, 41), (6, 7), (10, 11, 16, 17), (32, 33), (3,)):
+        lengths = list(lengths)
+        words = []
+        total = 0
+        while total < 4_400_000:
+            n = lengths[int(rng.integers(0, len(lengths)))]
+            w = (97 + rng.integers(0, 26, n)).astype(np.uint8)
+            words.append(w); words.append(np.frombuffer(b" ", dtype=np.uint8))
+            total += n + 1
+        text = np.concatenate(words)
+        doc_off = np.array([0, text.size // 3, text.size], dtype=np.int64)
+        while text[doc_off[1]] != 32:                            # cut between words
+            doc_off[1] += 1
+        ids, ioff, status = gpu_encode_batch(gv, text, doc_off)
+        want, woff = cv.encode_batch(text, doc_off, pattern, nthreads=8)
+        assert status == 0 and same(ioff, woff) and same(ids, want), (lengths[:4], first_difference(ids, want))
+        one, status = gpu_encode(gv, text)                       # the same text as one request of more than 4 MB
+        assert status == 0 and same(one, cv.encode(text, pattern, nthreads=8)[0])
+
+
 def test_batch_ids_match_documents_alone():
     cfg = wl.CONFIGS["C5"]
     text, off = wl.batch(cfg, n_docs=12, scale=0.02)

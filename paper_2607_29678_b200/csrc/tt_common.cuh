@@ -44,7 +44,7 @@ constexpr u64 TT_SLOT_EMPTY = ~0ull;              // pair-table slot: (left << 3
 constexpr int TT_WARP_PIECE_MAX = 256;            // bytes; longer pieces take the block-cooperative path
 // Bulk text: length classes of the pieces of at most 32 bytes (largest length of each class).
 constexpr int TT_SHORT_CLASSES = 4;
-TT_HD constexpr int tt_short_class_max(int c) { return c == 0 ? 6 : c == 1 ? 10 : c == 2 ? 16 : 32; }
+TT_HD constexpr int tt_short_class_max(int c) { return c == 0 ? 10 : c == 1 ? 16 : c == 2 ? 22 : 32; }
 
 // ---- workspace header (device memory) -----------------------------------------------------------
 struct TTHeader {

@@ -1446,6 +1446,15 @@ k_scatter_bulk(const ScatterParams P) {
         u32 skip = (lane >= 1 && lane < BPE_WARPS && tile + lane < tile_hi) ? P.tile_tok[tile + lane] : 0u;
         const size_t p0 = (size_t)tile * TT_TILE_BYTES;
         const long long t0 = (long long)tile * TT_TILE_BYTES - P.shift;      // text offset of the tile start
+        // does any document start in this tile?  (few tiles: the pieces of the others need not look)
+        bool tile_has_doc = false;
+        if (P.docmask) {
+            const size_t wi = (size_t)tile * (TT_TILE_BYTES / 32) + 2 * lane, nwords = (size_t)(P.hi >> 5) + 4;   // (the mask's cleared extent)
+            uint2 dm = make_uint2(0, 0);
+            if (wi + 1 < nwords) dm = *reinterpret_cast<const uint2*>(P.docmask + wi);
+            else if (wi < nwords) dm.x = P.docmask[wi];
+            tile_has_doc = __any_sync(FULL, (dm.x | dm.y) != 0);
+        }
         u32 run = carry;
         uint4 v = make_uint4(0, 0, 0, 0);
         uint2 o4 = make_uint2(0, 0);
@@ -1477,7 +1486,7 @@ k_scatter_bulk(const ScatterParams P) {
                     else if (x[h] >= 0) P.ids_out[dst] = x[h];
                     else if (c[h] <= 8) { for (u32 kk = 0; kk < c[h]; kk++) P.ids_out[dst + kk] = P.stage[src + kk]; }
                     else bigmask |= 1u << h;
-                    if (P.docmask) {
+                    if (tile_has_doc) {
                         const long long g = (long long)tile * TT_TILE_BYTES + off[h];
                         if ((P.docmask[g >> 5] >> (g & 31)) & 1) {
                             // every document that starts at this byte (empty ones included) gets this token offset

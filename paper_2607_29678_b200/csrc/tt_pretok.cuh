@@ -191,18 +191,18 @@ TT_HD u32 tt_walk_fwd_nl(const u16 (*sm)[TT_SLOTS], int s, int bit, bool& open) 
 }
 
 // The same question asked of the raw text from byte g on (the run has left the shared-memory window):
-// 1 / 0 = answered from ASCII bytes alone, -1 = undecided (a non-ASCII byte, which may be whitespace; a
-// document boundary mask to consult; or more than `limit` bytes of blanks).  One thread, plain loads.
+// 1 / 0 = answered from ASCII bytes alone, -1 = undecided (a non-ASCII byte, which may be whitespace, or more
+// than `limit` bytes of blanks).  A document start cuts the run.  One thread, plain loads.
 TT_HD int tt_raw_fwd_nl(const u8* base, long long g, long long hi, const u32* docmask, int limit = 256) {
-    if (docmask) return -1;
     int k = 0;
-    // sixteen bytes at a time while they are all blanks other than CR/LF (g is a multiple of 16 for every caller;
-    // `base` is 16-byte aligned)
+    // sixteen bytes at a time while they are all blanks other than CR/LF and no document starts among them (g is a
+    // multiple of 16 for every caller; `base` is 16-byte aligned)
     if ((g & 15) == 0) {
         for (; k + 16 <= limit && g + 16 <= hi; k += 16, g += 16) {
             const uint4 v = *reinterpret_cast<const uint4*>(base + g);
             const u32 w[4] = {v.x, v.y, v.z, v.w};
             bool plain = ((v.x | v.y | v.z | v.w) & 0x80808080u) == 0;
+            if (docmask) plain = plain && reinterpret_cast<const u16*>(docmask)[g >> 4] == 0;
 #pragma unroll
             for (int j = 0; j < 4; j++)
                 plain = plain && (tt_swar_range(w[j], 0x09, 0x09) | tt_swar_range(w[j], 0x0B, 0x0C) | tt_swar_range(w[j], ' ', ' ')) == 0x80808080u;
@@ -211,6 +211,7 @@ TT_HD int tt_raw_fwd_nl(const u8* base, long long g, long long hi, const u32* do
     }
     for (; k < limit; k++, g++) {
         if (g >= hi) return 0;
+        if (docmask && ((docmask[g >> 5] >> (g & 31)) & 1)) return 0;        // the run is cut by a document start
         const u32 b = base[g];
         if (b == '\n' || b == '\r') return 1;
         if (b >= 0x80) return -1;

@@ -629,12 +629,12 @@ def csrc_hash() -> str:
 # captures.  They belong to the source state whose hash is recorded with them; with other sources they are not
 # printed as measurements (the keys are null and "capture_stale" is true).
 NCU_CAPTURE = {
-    "csrc": "43bb8f501954a9eb",
+    "csrc": "f503444e9aebcd5b",
     # kernel -> dram__bytes_read.sum + dram__bytes_write.sum per launch, one cold C3 request (ncu --set full)
-    "c3_dram_bytes": {"front": 9472256, "merge": 10050560, "scatter": 1521920},
+    "c3_dram_bytes": {"front": 9474048, "merge": 10050048, "scatter": 1521920},
     # kernel -> smsp__inst_executed.sum per launch of the 256-request batch: captured on the first 32 documents of the same
     # batch (16,315,836 bytes) and scaled by text bytes to the full 132,689,913 (all work is per tile or per piece)
-    "batch_warp_inst": {"front": 481984000, "closing": 2743000, "merge_bulk": 110480000, "scatter_bulk": 101854000},
+    "batch_warp_inst": {"front": 475555000, "closing": 2742000, "merge_bulk": 110483000, "scatter_bulk": 90048000},
 }
 
 
